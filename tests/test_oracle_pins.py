@@ -1,0 +1,518 @@
+"""Pins for the CPU oracle: brute force in NumPy, library special cases, closed forms, invariants.
+
+None of these re-call the oracle's own routine: the NumPy side uses strided slicing, a normalised
+matrix product and full sorts, i.e. different index arithmetic from the C loops.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from paper_2607_23844_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def as_f64(x, dtype):
+    return x.astype(np.float64) if dtype == inputs.F32 else inputs.bf16_bits_to_f32(x).astype(np.float64)
+
+
+def np_token_match(x64, sy, sx, oy, ox, gy, gx, self_match=False, eps=1e-8):
+    """All-pairs brute force per patch with NumPy slicing. Returns best_sim(f64), best_idx, full list."""
+    B, T, H, W, C = x64.shape
+    Hp, Wp = H // gy, W // gx
+    idx = np.arange(B * T * H * W).reshape(B, T, H, W)
+    n = B * T * H * W
+    best_sim = np.full(n, -np.inf)
+    best_idx = np.arange(n)
+    second = np.full(n, -np.inf)
+    fulls = []
+    for b in range(B):
+        for t in range(T):
+            for py in range(gy):
+                for px in range(gx):
+                    xs = x64[b, t, py * Hp:(py + 1) * Hp, px * Wp:(px + 1) * Wp]
+                    ids = idx[b, t, py * Hp:(py + 1) * Hp, px * Wp:(px + 1) * Wp]
+                    if self_match:
+                        reps, rid = xs.reshape(-1, C), ids.reshape(-1)
+                        cands, cid = reps, rid
+                    else:
+                        mask = np.zeros((Hp, Wp), bool)
+                        mask[oy::sy, ox::sx] = True
+                        reps, rid = xs[mask], ids[mask]
+                        cands, cid = xs[~mask], ids[~mask]
+                    rn = reps / np.maximum(np.linalg.norm(reps, axis=1, keepdims=True), eps)
+                    cn = cands / np.maximum(np.linalg.norm(cands, axis=1, keepdims=True), eps)
+                    S = np.clip(cn @ rn.T, -1, 1)
+                    if self_match:
+                        np.fill_diagonal(S, -np.inf)
+                    a = S.argmax(axis=1)                      # first maximum = lowest index
+                    best_sim[cid] = S[np.arange(len(cid)), a]
+                    best_idx[cid] = rid[a]
+                    S2 = S.copy()
+                    S2[np.arange(len(cid)), a] = -np.inf
+                    second[cid] = S2.max(axis=1)
+                    fulls.append((cid, rid, S))
+    return best_sim, best_idx, second, fulls
+
+
+# ---------------------------------------------------------------------------------------------
+# hand-worked values (tests/golden/cosine_hand_cases.txt: integer vectors with rational cosines)
+# ---------------------------------------------------------------------------------------------
+def test_cosine_hand_cases(oracle):
+    rows = []
+    with open(os.path.join(GOLDEN, "cosine_hand_cases.txt")) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if not line:
+                continue
+            a, b, num, den = line.split(";")
+            rows.append((np.array(a.split(), np.float32), np.array(b.split(), np.float32),
+                         float(num) / float(den)))
+    assert len(rows) >= 6
+    for a, b, want in rows:
+        x = np.concatenate([a, b])
+        got = oracle.cosine(x, oracle.DT_F32, 0, a.size, a.size)
+        assert abs(got - want) < 1e-15, (a, b, got, want)
+        # same values stored as bf16 (small integers are exact in bf16)
+        xb = inputs.to_bf16_bits(x)
+        assert abs(oracle.cosine(xb, oracle.DT_BF16, 0, a.size, a.size) - want) < 1e-15
+
+
+def test_cosine_closed_forms(oracle):
+    rng = np.random.default_rng(3)
+    a = rng.standard_normal(257).astype(np.float32)
+    for s, want in ((2.0, 1.0), (0.5, 1.0), (-4.0, -1.0)):      # powers of two: scaling is exact
+        x = np.concatenate([a, (a * np.float32(s))])
+        assert abs(oracle.cosine(x, 0, 0, 257, 257) - want) < 1e-14
+    z = np.zeros(16, np.float32)
+    assert oracle.cosine(np.concatenate([z, a[:16]]), 0, 0, 16, 16) == 0.0   # zero row -> 0 (eps floor)
+    # operand order does not matter, and a transposed/offset read would break this antisymmetry pin
+    b = rng.standard_normal(257).astype(np.float32)
+    x = np.concatenate([a, b])
+    assert oracle.cosine(x, 0, 0, 257, 257) == oracle.cosine(x, 0, 257, 0, 257)
+    assert abs(oracle.cosine(np.concatenate([a, -b]), 0, 0, 257, 257) + oracle.cosine(x, 0, 0, 257, 257)) < 1e-15
+
+
+def test_bf16_widening_is_exact(oracle):
+    # every finite bf16 pattern widens to the fp32 with the same top bits: check through cos(a, e_k)
+    vals = np.array([1.0, -2.5, 3.0e-3, 1.5e10, -7.0], np.float32)
+    bits = inputs.to_bf16_bits(vals)
+    back = inputs.bf16_bits_to_f32(bits).astype(np.float64)
+    for k in range(vals.size):
+        e = np.zeros(vals.size, np.float32); e[k] = 1.0
+        x = np.concatenate([bits, inputs.to_bf16_bits(e)])
+        got = oracle.cosine(x, 1, 0, vals.size, vals.size)
+        assert abs(got - back[k] / np.linalg.norm(back)) < 1e-15
+
+
+# ---------------------------------------------------------------------------------------------
+# dense match vs NumPy brute force
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("shape,groups,lattice,dtype", [
+    ((1, 1, 16, 16, 64), (1, 1), (2, 2, 0, 0), inputs.F32),
+    ((2, 1, 8, 12, 24), (1, 1), (2, 2, 0, 0), inputs.BF16),
+    ((1, 3, 8, 8, 16), (2, 2), (2, 2, 1, 0), inputs.BF16),
+    ((2, 2, 8, 16, 8), (2, 4), (2, 2, 0, 1), inputs.F32),
+    ((1, 1, 6, 9, 8), (1, 1), (3, 3, 1, 2), inputs.F32),
+    ((1, 2, 4, 8, 8), (1, 2), (1, 2, 0, 1), inputs.BF16),
+])
+def test_match_token_bruteforce(oracle, shape, groups, lattice, dtype):
+    rng = np.random.default_rng(11)
+    xf = rng.standard_normal(shape).astype(np.float32)
+    # plant duplicates so that arg-max ties and high similarities occur
+    flat = xf.reshape(-1, shape[-1])
+    flat[5] = flat[0]; flat[9] = flat[0]; flat[-1] = 2 * flat[3]
+    x = xf if dtype == inputs.F32 else inputs.to_bf16_bits(xf)
+    sy, sx, oy, ox = lattice
+    L = oracle.Layout(oracle.KIND_TOKEN, dtype, *shape, sy=sy, sx=sx, oy=oy, ox=ox,
+                      gy=groups[0], gx=groups[1])
+    got = oracle.match_token(L, x, want_full=True)
+    bs, bi, sec, fulls = np_token_match(as_f64(x, dtype), sy, sx, oy, ox, *groups)
+    assert np.array_equal(got["best_idx"], bi)
+    cand = np.isfinite(bs)
+    assert np.allclose(got["best_sim"][cand], bs[cand], atol=1e-7, rtol=0)   # fp32 rounding of output
+    assert np.all(np.isneginf(got["best_sim"][~cand]))
+    assert np.allclose(got["second_sim"][cand], sec[cand].astype(np.float32), atol=1e-7, rtol=0)
+    # full matrix, element by element, to 1e-12
+    U = L.units_per_group
+    for g, (cid, rid, S) in enumerate(fulls):
+        loc = {L.unit_index(g, u): u for u in range(U)}
+        rows = [loc[i] for i in cid]
+        assert np.max(np.abs(got["full_sim"][g][rows] - S)) < 1e-12
+    # representative/candidate counts
+    assert cand.sum() == L.n_groups * (U - L.n_rep)
+
+
+def test_match_token_self_match_tiny_config(oracle):
+    w = inputs.tiny_token_cache()
+    L = oracle.Layout(oracle.KIND_TOKEN, w.dtype, *w.shape, self_match=1)
+    got = oracle.match_token(L, w.x, want_full=True)
+    bs, bi, sec, fulls = np_token_match(w.x.astype(np.float64), 2, 2, 0, 0, 1, 1, self_match=True)
+    assert np.array_equal(got["best_idx"], bi)
+    assert np.allclose(got["best_sim"], bs, atol=1e-7, rtol=0)
+    S = fulls[0][2]
+    off = ~np.eye(256, dtype=bool)
+    assert np.max(np.abs(got["full_sim"][0][off] - S[off])) < 1e-12
+    # sanity bands of the recipe: planted copies are near 1, everything else far below the threshold
+    assert (bs > 0.999).sum() >= 100 and ((bs > 0.6) & (bs < 0.999)).sum() == 0
+
+
+def test_match_token_rows_subset(oracle):
+    rng = np.random.default_rng(5)
+    x = inputs.to_bf16_bits(rng.standard_normal((2, 2, 8, 8, 16)).astype(np.float32))
+    L = oracle.Layout(oracle.KIND_TOKEN, oracle.DT_BF16, 2, 2, 8, 8, 16, gy=2, gx=2)
+    full = oracle.match_token(L, x)
+    rows = rng.choice(L.n_units, 40, replace=False)
+    sub = oracle.match_token(L, x, rows=rows)
+    assert np.array_equal(sub["best_idx"][rows], full["best_idx"][rows])
+    assert np.array_equal(sub["best_sim"][rows], full["best_sim"][rows])
+    untouched = np.setdiff1d(np.arange(L.n_units), rows)
+    assert np.all(sub["best_idx"][untouched] == -2)
+
+
+def test_match_token_library_special_case_midsize(oracle):
+    """Normalise rows, one float64 matrix product, row max: the textbook form, at several tiles' size."""
+    w = inputs.sd3_token_cache(seed=7, B=1, H=32, W=32, C=192)
+    L = oracle.Layout(oracle.KIND_TOKEN, w.dtype, *w.shape)
+    got = oracle.match_token(L, w.x)
+    x64 = as_f64(w.x, w.dtype)[0, 0]
+    reps = x64[0::2, 0::2].reshape(-1, 192)
+    rid = np.arange(32 * 32).reshape(32, 32)[0::2, 0::2].reshape(-1)
+    rn = reps / np.linalg.norm(reps, axis=1, keepdims=True)
+    xn = x64.reshape(-1, 192) / np.linalg.norm(x64.reshape(-1, 192), axis=1, keepdims=True)
+    S = xn @ rn.T
+    cand = np.setdiff1d(np.arange(1024), rid)
+    assert np.array_equal(got["best_idx"][cand], rid[S[cand].argmax(1)])
+    assert np.allclose(got["best_sim"][cand], S[cand].max(1), atol=1e-7, rtol=0)
+
+
+def test_match_token_duplicates_and_onehot(oracle):
+    # exact duplicate of a representative -> similarity exactly 1 and that representative wins,
+    # the lowest-indexed one when several representatives are identical
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((1, 1, 4, 4, 32)).astype(np.float32)
+    x[0, 0, 0, 2] = x[0, 0, 0, 0]        # rep (0,2) == rep (0,0)
+    x[0, 0, 1, 1] = x[0, 0, 0, 0]        # candidate copies them
+    x[0, 0, 3, 3] = 4 * x[0, 0, 2, 2]    # scaled copy of rep (2,2)
+    L = oracle.Layout(oracle.KIND_TOKEN, 0, 1, 1, 4, 4, 32)
+    got = oracle.match_token(L, x)
+    assert got["best_idx"][5] == 0 and abs(got["best_sim"][5] - 1) < 1e-7
+    assert abs(got["second_sim"][5] - 1) < 1e-7
+    assert got["best_idx"][15] == 10 and abs(got["best_sim"][15] - 1) < 1e-7
+    # one-hot rows: similarities are 0 or 1
+    eye = np.zeros((1, 1, 4, 4, 16), np.float32)
+    for k in range(16):
+        eye[0, 0, k // 4, k % 4, k % 4] = 1.0
+    got = oracle.match_token(oracle.Layout(0, 0, 1, 1, 4, 4, 16), eye, want_full=True)
+    f = got["full_sim"][0]
+    f = f[~np.isnan(f)]
+    assert set(np.unique(f)) <= {0.0, 1.0}
+    # permuting channels changes no index
+    perm = rng.permutation(32)
+    got_p = oracle.match_token(L, np.ascontiguousarray(x[..., perm]))
+    assert np.array_equal(got_p["best_idx"], oracle.match_token(L, x)["best_idx"])
+
+
+# ---------------------------------------------------------------------------------------------
+# frame and block match vs NumPy
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("T", [2, 5, 6])
+@pytest.mark.parametrize("stat", [0, 1])
+def test_match_frame_bruteforce(oracle, T, stat):
+    rng = np.random.default_rng(T)
+    B, H, W, Cc = 2, 3, 5, 16
+    xf = rng.standard_normal((B, T, H, W, Cc)).astype(np.float32)
+    xf[:, 1:] = 0.7 * xf[:, :-1] + 0.3 * xf[:, 1:]
+    x = inputs.to_bf16_bits(xf)
+    x64 = as_f64(x, inputs.BF16)
+    L = oracle.Layout(oracle.KIND_FRAME, oracle.DT_BF16, B, T, H, W, Cc, frame_stat=stat)
+    got = oracle.match_frame(L, x, want_pos=True)
+    a, b = x64[:, 1:], x64[:, :-1]
+    pos = (a * b).sum(-1) / (np.linalg.norm(a, axis=-1) * np.linalg.norm(b, axis=-1))
+    if stat == 0:
+        pair = pos.mean(axis=(2, 3))
+    else:
+        af, bf = a.reshape(B, T - 1, -1), b.reshape(B, T - 1, -1)
+        pair = (af * bf).sum(-1) / (np.linalg.norm(af, axis=-1) * np.linalg.norm(bf, axis=-1))
+    assert np.allclose(got["pos_sim"], pos.reshape(B, T - 1, -1), atol=1e-7, rtol=0)
+    assert np.allclose(got["pair_sim"], pair, atol=1e-7, rtol=0)
+    for bb in range(B):
+        for t in range(T):
+            i = bb * T + t
+            if t % 2 == 0:
+                assert got["best_idx"][i] == i and np.isneginf(got["best_sim"][i])
+                continue
+            opts = [(pair[bb, t - 1], i - 1)]
+            if t + 1 < T:
+                opts.append((pair[bb, t], i + 1))
+            want = max(opts, key=lambda o: (o[0], -o[1]))
+            assert got["best_idx"][i] == want[1]
+            assert abs(got["best_sim"][i] - want[0]) < 1e-7
+
+
+def test_match_frame_ar1_expectation(oracle):
+    """AR(1) frames: E[cos(x_t, x_{t-1})] = rho for unit-variance stationary rows (closed form)."""
+    rho = 0.95
+    rng = np.random.default_rng(8)
+    f0 = rng.standard_normal((8, 8, 320), dtype=np.float32)
+    x = inputs.ar1_frames(rng, f0, 9, rho).reshape(1, 9, 8, 8, 320)
+    L = oracle.Layout(oracle.KIND_FRAME, 0, 1, 9, 8, 8, 320)
+    got = oracle.match_frame(L, x)
+    assert np.all(np.abs(got["pair_sim"] - rho) < 3 * (1 - rho ** 2) / np.sqrt(320 * 64) + 2e-3)
+
+
+@pytest.mark.parametrize("lattice", [(2, 2, 0, 0), (2, 2, 1, 1), (1, 2, 0, 0)])
+def test_match_block_bruteforce(oracle, lattice):
+    sy, sx, oy, ox = lattice
+    rng = np.random.default_rng(4)
+    B, T, H, W, Cc = 2, 3, 4, 6, 8
+    x = inputs.to_bf16_bits(rng.standard_normal((B, T, H, W, Cc)).astype(np.float32))
+    x64 = as_f64(x, inputs.BF16)
+    desc = x64.transpose(0, 2, 3, 1, 4).reshape(B, H, W, T * Cc)       # (B, H*W, T*C) reshape
+    L = oracle.Layout(oracle.KIND_BLOCK, 1, B, T, H, W, Cc, sy=sy, sx=sx, oy=oy, ox=ox)
+    got = oracle.match_block(L, x)
+    for b in range(B):
+        for y in range(H):
+            for xx in range(W):
+                i = b * H * W + y * W + xx
+                ry, rx = (y // sy) * sy + oy, (xx // sx) * sx + ox
+                if (ry, rx) == (y, xx):
+                    assert got["best_idx"][i] == i and np.isneginf(got["best_sim"][i])
+                    continue
+                a, r = desc[b, y, xx], desc[b, ry, rx]
+                want = a @ r / (np.linalg.norm(a) * np.linalg.norm(r))
+                assert got["best_idx"][i] == b * H * W + ry * W + rx
+                assert abs(got["best_sim"][i] - want) < 1e-7
+
+
+# ---------------------------------------------------------------------------------------------
+# selection vs full sort in NumPy, and its invariants
+# ---------------------------------------------------------------------------------------------
+def np_select(L, best_sim, best_idx, mode, thr, n_reuse, stride):
+    G, U = L.n_groups, L.units_per_group
+    gi = np.array([[L.unit_index(g, u) for u in range(U)] for g in range(G)])
+    is_rep = np.array([L.is_rep(u) for u in range(U)])
+    n = G * U
+    reuse = np.zeros(n, bool)
+    for g in range(G):
+        cand = gi[g][~is_rep] if not L.self_match else gi[g]
+        if mode == 0:
+            r = best_sim[cand] >= np.float32(thr)
+            if L.self_match:
+                r &= best_idx[cand] < cand
+            reuse[cand[r]] = True
+        else:
+            order = np.lexsort((cand, -best_sim[cand].astype(np.float64)))   # sim desc, index asc
+            reuse[cand[order[:n_reuse]]] = True
+    kept_idx = np.full(G * stride, -1, np.int64)
+    slot_of = np.full(n, -1, np.int64)
+    cnt = np.zeros(G, np.int64)
+    for g in range(G):
+        kept = np.sort(gi[g][~reuse[gi[g]]])
+        kept_idx[g * stride: g * stride + kept.size] = kept
+        slot_of[kept] = g * stride + np.arange(kept.size)
+        cnt[g] = kept.size
+    mm = np.arange(n)
+    for i in np.nonzero(reuse)[0]:
+        m = i
+        while reuse[m]:
+            m = best_idx[m]
+        mm[i] = m
+    return kept_idx, cnt, mm, slot_of
+
+
+@pytest.mark.parametrize("kind,shape,groups", [
+    (0, (2, 1, 8, 8, 8), (1, 1)), (0, (1, 2, 8, 16, 8), (2, 2)),
+    (1, (3, 7, 2, 2, 8), (1, 1)), (2, (2, 3, 6, 8, 8), (1, 1)),
+])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_select_bruteforce(oracle, kind, shape, groups, mode):
+    rng = np.random.default_rng(kind * 10 + mode)
+    x = rng.standard_normal(shape).astype(np.float32)
+    L = oracle.Layout(kind, 0, *shape, gy=groups[0], gx=groups[1])
+    m = oracle.match(L, x)
+    bs = m["best_sim"].copy()
+    cand = np.isfinite(bs)
+    # quantise so that equal similarities occur and the index tie-break is exercised
+    bs[cand] = np.round(bs[cand] * 8) / 8
+    U = L.units_per_group
+    n_cand = U - L.n_rep
+    for thr, n_reuse in ((0.0, n_cand // 2), (0.125, 1), (2.0, 0), (-1.0, n_cand), (0.25, n_cand + 5)):
+        stride = U if mode == 0 else U - min(n_reuse, n_cand)
+        got = oracle.select(L, bs, m["best_idx"], mode, thr, n_reuse, stride)
+        ki, cnt, mm, so = np_select(L, bs, m["best_idx"], mode, thr, n_reuse, stride)
+        assert np.array_equal(got["kept_idx"], ki)
+        assert np.array_equal(got["kept_count"], cnt)
+        assert np.array_equal(got["match_map"], mm)
+        assert np.array_equal(got["slot_of"], so)
+        if mode == 1:
+            assert np.all(cnt == U - min(n_reuse, n_cand))
+
+
+def test_select_self_match_chain(oracle):
+    w = inputs.tiny_token_cache()
+    L = oracle.Layout(0, 0, *w.shape, self_match=1)
+    m = oracle.match_token(L, w.x)
+    got = oracle.select(L, m["best_sim"], m["best_idx"], 0, 0.9)
+    ki, cnt, mm, so = np_select(L, m["best_sim"], m["best_idx"], 0, 0.9, 0, 256)
+    assert np.array_equal(got["kept_idx"], ki) and np.array_equal(got["match_map"], mm)
+    reused = got["slot_of"] < 0
+    assert 40 <= reused.sum() <= 110
+    # every reused token maps to a kept token with a lower index and similar features
+    assert np.all(got["slot_of"][got["match_map"][reused]] >= 0)
+    assert np.all(got["match_map"][reused] < np.nonzero(reused)[0])
+
+
+def test_select_invariants(oracle):
+    w = inputs.sd3_token_cache(seed=3, B=2, H=16, W=16, C=32, groups=(2, 2))
+    L = oracle.Layout(0, w.dtype, *w.shape, gy=2, gx=2)
+    m = oracle.match_token(L, w.x)
+    U, G = L.units_per_group, L.n_groups
+    got = oracle.select(L, m["best_sim"], m["best_idx"], 1, 0.0, w.n_reuse, U - w.n_reuse)
+    stride = U - w.n_reuse
+    ki = got["kept_idx"].reshape(G, stride)
+    assert np.all(np.diff(ki, axis=1) > 0)                                    # strictly ascending
+    assert np.all(got["kept_count"] == stride)
+    reused = np.nonzero(got["slot_of"] < 0)[0]
+    assert reused.size == G * w.n_reuse
+    assert np.array_equal(np.sort(np.concatenate([ki.reshape(-1), reused])), np.arange(L.n_units))
+    rep_ids = [L.unit_index(g, u) for g in range(G) for u in range(U) if L.is_rep(u)]
+    assert np.all(got["slot_of"][rep_ids] >= 0)                               # representatives kept
+    assert np.array_equal(got["slot_of"][ki.reshape(-1)], np.arange(G * stride))
+    # match_map of a reused token is a kept representative of its own group
+    grp = {L.unit_index(g, u): g for g in range(G) for u in range(U)}
+    for i in reused:
+        r = got["match_map"][i]
+        assert grp[r] == grp[i] and got["slot_of"][r] >= 0 and r in set(rep_ids)
+    # the cut: every reused candidate is at least as similar as every kept candidate of its group
+    for g in range(G):
+        ids = np.array([L.unit_index(g, u) for u in range(U) if not L.is_rep(u)])
+        r = got["slot_of"][ids] < 0
+        assert m["best_sim"][ids][r].min() >= m["best_sim"][ids][~r].max()
+
+
+# ---------------------------------------------------------------------------------------------
+# gather / restore
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("kind", [0, 1, 2])
+def test_identity_selection_roundtrip(oracle, kind):
+    """Identity selection => kept_idx = 0..n-1, gather is a copy, restore(gather(x)) == x bitwise."""
+    rng = np.random.default_rng(kind)
+    shape = (2, 4, 4, 6, 8)
+    x = inputs.to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+    L = oracle.Layout(kind, 1, *shape)
+    m = oracle.match(L, x)
+    for mode, thr, n_reuse in ((0, 2.0, 0), (1, 0.0, 0)):
+        s = oracle.select(L, m["best_sim"], m["best_idx"], mode, thr, n_reuse)
+        assert np.array_equal(s["kept_idx"], np.arange(L.n_units))
+        assert np.array_equal(s["match_map"], np.arange(L.n_units))
+        R = oracle.rows_for(L, 8, 2)
+        y = oracle.gather(R, x, s["kept_idx"])
+        back = oracle.restore(R, y, np.zeros_like(x), L.n_units, s["slot_of"], s["match_map"])
+        assert back.tobytes() == x.tobytes()
+        if kind != 2:
+            assert y.tobytes() == x.tobytes()
+        else:   # block rows: the (T, HW, C) -> (HW, T, C) permutation
+            want = x.reshape(2, 4, 24, 8).transpose(0, 2, 1, 3)
+            assert y.tobytes() == np.ascontiguousarray(want).tobytes()
+
+
+@pytest.mark.parametrize("kind", [0, 1, 2])
+def test_restore_sources_no_averaging(oracle, kind):
+    rng = np.random.default_rng(20 + kind)
+    shape = (2, 6, 4, 4, 8)
+    Cout = 12
+    x = rng.standard_normal(shape).astype(np.float32)
+    L = oracle.Layout(kind, 0, *shape)
+    m = oracle.match(L, x)
+    n_cand = L.units_per_group - L.n_rep
+    s = oracle.select(L, m["best_sim"], m["best_idx"], 1, 0.0, n_cand // 2, L.units_per_group - n_cand // 2)
+    R = oracle.rows_for(L, Cout, 4)
+    out_shape = shape[:-1] + (Cout,)
+    cache = rng.standard_normal(out_shape).astype(np.float32)
+    n_slots = s["kept_idx"].size
+    z = rng.standard_normal((n_slots, R.row_bytes // 4)).astype(np.float32)
+    out = oracle.restore(R, z, cache, L.n_units, s["slot_of"], s["match_map"]).view(np.float32)
+
+    def unit_rows(t):      # [n_units, row elements] view of a [B,T,H,W,Cout] tensor, NumPy transposes
+        if kind == 0:
+            return t.reshape(-1, Cout)
+        if kind == 1:
+            return t.reshape(L.B * L.T, -1)
+        return np.ascontiguousarray(t.reshape(L.B, L.T, L.H * L.W, Cout).transpose(0, 2, 1, 3)).reshape(L.B * L.H * L.W, -1)
+
+    o, c = unit_rows(out.reshape(out_shape)), unit_rows(cache)
+    for i in range(L.n_units):
+        want = z[s["slot_of"][i]] if s["slot_of"][i] >= 0 else c[i]
+        assert o[i].tobytes() == want.tobytes()
+    # cold start: skipped units take the fresh row of their representative
+    out2 = oracle.restore(R, z, None, L.n_units, s["slot_of"], s["match_map"],
+                          src_mode=oracle.SRC_REPRESENTATIVE).view(np.float32)
+    o2 = unit_rows(out2.reshape(out_shape))
+    for i in range(L.n_units):
+        assert o2[i].tobytes() == z[s["slot_of"][s["match_map"][i]]].tobytes()
+    # in place: skipped rows untouched, computed rows overwritten
+    c2 = cache.copy()
+    oracle.restore(R, z, c2, L.n_units, s["slot_of"], s["match_map"], in_place=True)
+    assert c2.tobytes() == out.tobytes()
+    # gather lists exactly the kept rows of x in ascending order
+    Rx = oracle.rows_for(L, shape[-1], 4)
+    y = oracle.gather(Rx, x, s["kept_idx"]).view(np.float32)
+    xr = unit_rows_generic(x, L)
+    for slot, i in enumerate(s["kept_idx"]):
+        if i >= 0:
+            assert y[slot].tobytes() == xr[i].tobytes()
+
+
+def unit_rows_generic(t, L):
+    Cc = t.shape[-1]
+    if L.kind == 0:
+        return t.reshape(-1, Cc)
+    if L.kind == 1:
+        return t.reshape(L.B * L.T, -1)
+    return np.ascontiguousarray(t.reshape(L.B, L.T, L.H * L.W, Cc).transpose(0, 2, 1, 3)).reshape(L.B * L.H * L.W, -1)
+
+
+def test_layer_cache_rule(oracle):
+    lc = oracle.LayerCache()
+    a = np.arange(100, dtype=np.float32)
+    assert lc.get(3, 0, 5) is None
+    lc.put(3, 10, a)
+    for step, hit in ((9, False), (10, True), (14, True), (15, False), (100, False)):
+        got = lc.get(3, step, 5)
+        assert (got is not None) == hit
+        if hit:
+            assert got == a.tobytes()
+    assert lc.get(4, 10, 5) is None
+    lc.put(3, 15, a + 1)
+    assert lc.get(3, 14, 5) is None and lc.get(3, 16, 5) == (a + 1).tobytes()
+    lc.clear()
+    assert lc.get(3, 16, 5) is None
+
+
+# ---------------------------------------------------------------------------------------------
+# input recipes: sanity bands (properties of the generators, not parity targets)
+# ---------------------------------------------------------------------------------------------
+def test_input_recipes_shapes_and_bands(oracle):
+    w = inputs.sd3_token_cache(seed=1002, B=1, H=32, W=32, C=96)
+    assert w.x.dtype == np.uint16 and w.x.shape == (1, 1, 32, 32, 96)
+    assert w.n_reuse == (1024 - 256) // 2
+    f = inputs.bf16_bits_to_f32(w.x).astype(np.float64)
+    assert 0.7 < f.var() < 1.4
+    # neighbouring tokens of the smooth field are strongly correlated, distant ones are not
+    a, b, c = f[0, 0, :, :-1], f[0, 0, :, 1:], np.roll(f[0, 0], 16, axis=1)
+    near = (a * b).sum(-1) / (np.linalg.norm(a, axis=-1) * np.linalg.norm(b, axis=-1))
+    far = (f[0, 0] * c).sum(-1) / (np.linalg.norm(f[0, 0], axis=-1) * np.linalg.norm(c, axis=-1))
+    assert near.mean() > 0.95 and abs(far.mean()) < 0.3
+    blk = inputs.latte_blocks(T=4, H=8, W=8, C=64)
+    L = oracle.Layout(2, blk.dtype, *blk.shape)
+    sims = oracle.match_block(L, blk.x)["best_sim"]
+    sims = sims[np.isfinite(sims)]
+    assert sims.min() < 0.85 < sims.max()
+    assert inputs.keep_ratio_to_reuse(9216, 6912, 0.25) == 6912
+    assert inputs.keep_ratio_to_reuse(9216, 6912, 0.5) == 4608
+    assert inputs.keep_ratio_to_reuse(9216, 6912, 0.75) == 2304
+    # bf16 rounding is round-to-nearest-even
+    v = np.array([1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, 1.0 + 2 ** -9], np.float32)
+    assert list(inputs.to_bf16_bits(v)) == [0x3F80, 0x3F82, 0x3F80]
