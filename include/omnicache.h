@@ -1,0 +1,247 @@
+/*
+ * omnicache.h - C-ABI of the B200 (sm_100a) OmniCache hot path.
+ *
+ * The operator wrapped around one attention / FFN layer call by Token Cache, Frame Cache and Block
+ * Cache (Sections 3.2.1-3.2.3), plus the Layered Cache store (Section 3.4):
+ *
+ *     match  ->  select  ->  gather  ->  [ the wrapped layer, outside this library ]  ->  restore
+ *
+ * Conventions
+ *   - All data pointers are DEVICE pointers unless a name ends in `_host`.  The caller owns every
+ *     feature / index / output buffer and the stream.  The library never allocates caller-visible
+ *     memory, never frees caller memory and never synchronises the stream (exceptions are stated).
+ *   - `stream` is a cudaStream_t passed as void*.  All work is stream-ordered.
+ *   - Feature tensors are row-major [B][T][H][W][C], channel last (Section 3.2.2 writes spatial
+ *     inputs as (B, T, H, W, C)); images have T = 1.  Base pointers are 16-byte aligned and
+ *     C * element size is a multiple of 16 bytes.
+ *   - A "unit" is a token (OC_KIND_TOKEN), a frame (OC_KIND_FRAME) or a 1x1xT temporal block
+ *     (OC_KIND_BLOCK).  Unit indices are global and int32:
+ *         token ((b*T + t)*H + y)*W + x,     frame b*T + t,     block b*H*W + y*W + x.
+ *   - Every call returns an oc_status.  On a host-detected error nothing is launched and no output
+ *     is written.  Device-side conditions (an expired bounded wait) land in a status word read by
+ *     oc_device_status().  No call aborts or throws.
+ *   - A context is bound to one device and is not thread-safe; use one per host thread.
+ */
+#ifndef OMNICACHE_H_
+#define OMNICACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int oc_status;
+enum {
+    OC_OK = 0,
+    OC_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, inconsistent layout            */
+    OC_ERR_ALIGNMENT = 2,    /* pointer or row size not a multiple of 16 bytes                  */
+    OC_ERR_UNSUPPORTED = 3,  /* valid request outside what the kernels implement                */
+    OC_ERR_WORKSPACE = 4,    /* context workspace smaller than oc_match_workspace_bytes()       */
+    OC_ERR_CUDA = 5,         /* a CUDA runtime / driver call failed (no device, launch error)   */
+    OC_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired (see oc_device_status)       */
+    OC_ERR_OOM = 7,          /* device allocation for library-owned storage failed              */
+    OC_CACHE_MISS = 8        /* oc_layer_cache_get: nothing reusable for (layer, step)          */
+};
+
+enum { OC_KIND_TOKEN = 0, OC_KIND_FRAME = 1, OC_KIND_BLOCK = 2 };
+enum { OC_DTYPE_F32 = 0, OC_DTYPE_BF16 = 1 };
+enum { OC_SELECT_THRESHOLD = 0, OC_SELECT_COUNT = 1 };
+enum { OC_RESTORE_FROM_CACHE = 0, OC_RESTORE_FROM_REPRESENTATIVE = 1 };
+enum { OC_FRAME_MEAN_POS_COS = 0, OC_FRAME_FLAT_COS = 1 };
+
+/* Which units are compared with which (Sections 3.2.1-3.2.3, 3.3).
+ *   TOKEN: each frame is cut into gy x gx equal patches ("token groups", Section 3.3); inside a
+ *          patch the tokens on the (oy, ox) + (sy, sx)-strided lattice are the representatives and
+ *          every other token is a candidate, compared with all representatives of its patch.
+ *          self_match = 1: every token is both (all pairs, self excluded); needs gy = gx = 1.
+ *   FRAME: even frames are representatives, odd frames candidates, each compared with its two
+ *          adjacent frames (alternating sets, Section 3.2.2).  sy..gx are ignored (gy = gx = 1).
+ *   BLOCK: positions are cut into sy x sx neighbourhoods; the (oy, ox) member is the
+ *          representative, the others are compared with it over the T*C block descriptor
+ *          (Section 3.2.1).  gy = gx = 1.
+ * H/gy must be a multiple of sy and W/gx of sx (TOKEN, BLOCK). */
+typedef struct oc_layout {
+    int kind;        /* OC_KIND_*  */
+    int dtype;       /* OC_DTYPE_* of the feature tensor */
+    int B, T, H, W, C;
+    int sy, sx;      /* representative lattice stride, >= 1, sy*sx >= 2 unless self_match */
+    int oy, ox;      /* representative offset inside a neighbourhood, 0 <= oy < sy, 0 <= ox < sx */
+    int gy, gx;      /* patches per frame */
+    int self_match;  /* TOKEN only */
+    int frame_stat;  /* FRAME only: OC_FRAME_* */
+    float eps;       /* floor applied to each vector norm; cos = <a,b> / (max(|a|,eps) max(|b|,eps)) */
+} oc_layout;
+
+/* Rows of a strided tensor, used by gather / restore so that one pair of kernels moves tokens,
+ * whole frames and 1x1xT blocks (the fused permutation/scatter of Appendix A).  The row of unit i
+ * is n_seg segments of seg_bytes; segment s starts at byte
+ *     (i / units_per_outer) * outer_pitch + (i % units_per_outer) * unit_pitch + s * seg_stride.
+ * The dense side (gather output, restore input) is packed [row][segment][seg_bytes].
+ * seg_bytes and all pitches are multiples of 16. */
+typedef struct oc_rows {
+    int64_t seg_bytes;
+    int64_t n_seg;
+    int64_t seg_stride;
+    int64_t unit_pitch;
+    int64_t units_per_outer;
+    int64_t outer_pitch;
+} oc_rows;
+
+typedef struct oc_ctx oc_ctx;
+
+/* ---------------------------------------------------------------------------------------------
+ * Host-only helpers: no device is touched, usable without a GPU.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Human-readable name of a status code (static storage). */
+const char* oc_status_str(oc_status s);
+
+/* Validates a layout against the rules above.  OC_OK, OC_ERR_INVALID_ARG, OC_ERR_ALIGNMENT
+ * (C * element size not a multiple of 16) or OC_ERR_UNSUPPORTED (e.g. more than 2^31-1 units). */
+oc_status oc_layout_check(const oc_layout* layout);
+
+/* Group structure of a layout: a group is an independent selection problem (TOKEN: one patch of one
+ * frame; FRAME, BLOCK: one batch element).  Any output pointer may be null. */
+oc_status oc_layout_counts(const oc_layout* layout, int64_t* n_groups, int64_t* units_per_group,
+                           int64_t* reps_per_group);
+
+/* Bytes of context workspace oc_match() needs for this layout (norms, packed arg-max keys,
+ * partial sums). */
+oc_status oc_match_workspace_bytes(const oc_layout* layout, size_t* bytes);
+
+/* Row geometry of this layout's units inside a [B][T][H][W][channels] tensor of elem_bytes-sized
+ * elements (the layer input, or a layer output with another channel count). */
+oc_status oc_rows_from_layout(const oc_layout* layout, int channels, int elem_bytes, oc_rows* rows);
+
+/* The Layered Cache reuse rule (Section 3.4; the (l, t, N) triples of Algorithm 1): an output stored
+ * at stored_step serves step iff 0 <= step - stored_step < interval.  Returns 1 or 0. */
+int oc_layer_cache_would_hit(int stored_step, int step, int interval);
+
+/* Kernel ids for the launch counters / timers below. */
+enum {
+    OC_K_NORMS = 0,       /* row inverse norms + key reset (dense match pre-pass)     */
+    OC_K_MATCH_TC = 1,    /* tcgen05 dense matcher                                    */
+    OC_K_MATCH_SIMT = 2,  /* FFMA dense matcher (fp32 inputs, self-match, odd shapes) */
+    OC_K_MATCH_FIN = 3,   /* key unpack -> best_sim / best_idx                        */
+    OC_K_FRAME = 4,       /* Frame Cache streaming cosine                             */
+    OC_K_FRAME_FIN = 5,
+    OC_K_BLOCK = 6,       /* Block Cache streaming cosine                             */
+    OC_K_BLOCK_FIN = 7,
+    OC_K_SELECT = 8,
+    OC_K_GATHER = 9,
+    OC_K_RESTORE = 10,
+    OC_K_COPY = 11,       /* layered-cache put / copying get                          */
+    OC_K_COUNT = 12
+};
+const char* oc_kernel_name(int kernel_id);
+
+/* ---------------------------------------------------------------------------------------------
+ * Context
+ * ------------------------------------------------------------------------------------------- */
+
+/* Creates a context on `device` with `workspace_bytes` of library-owned scratch (may be 0 if
+ * oc_match is never called).  The context also owns the Layered Cache storage and a device status
+ * word.  OC_ERR_CUDA if the device cannot be used, OC_ERR_OOM if the scratch cannot be allocated. */
+oc_status oc_create(oc_ctx** out, int device, size_t workspace_bytes);
+
+/* Frees everything the context owns.  Synchronises the device. */
+oc_status oc_destroy(oc_ctx* ctx);
+
+/* Synchronises the device, reads and clears the device status word: *code is OC_OK or the first
+ * device-side condition recorded since the last call (OC_ERR_TIMEOUT). */
+oc_status oc_device_status(oc_ctx* ctx, int* code);
+
+/* Launch counters and optional per-kernel timers.  Counters always run.  With timers enabled each
+ * kernel launch is bracketed by CUDA events on the caller's stream; oc_profile_read waits for the
+ * recorded events and returns the number of launches and their summed device time since the last
+ * reset.  total_ms is 0 when timers were off. */
+oc_status oc_profile_enable(oc_ctx* ctx, int on);
+oc_status oc_profile_reset(oc_ctx* ctx);
+oc_status oc_profile_read(oc_ctx* ctx, int kernel_id, int64_t* launches, double* total_ms);
+
+/* ---------------------------------------------------------------------------------------------
+ * The hot path
+ * ------------------------------------------------------------------------------------------- */
+
+/* match (Background: "matches similar pairs by cosine similarity"; Sections 3.2.1-3.2.3).
+ * For every candidate unit: the most similar representative it may be matched with.
+ *   x         [B][T][H][W][C] features of layout->dtype (the wrapped layer's input)
+ *   best_sim  [n_units] float: cosine of the best match; -inf for representatives
+ *   best_idx  [n_units] int32: global unit index of that representative (ties: lowest index);
+ *             a representative's own index for representatives
+ *   aux_sim   nullable.  TOKEN: [n_groups][units_per_group][reps_per_group] float, every candidate
+ *             row's full similarity row (rows of representatives and the self-match diagonal are
+ *             not written).  FRAME: [B][T-1][H*W] per-position cosines of frame t vs t-1.
+ *   pair_sim  nullable, FRAME only: [B][T-1] statistic of every adjacent pair (t, t-1).
+ * bf16 TOKEN layouts without self_match run on the tcgen05 tensor cores (fp32 accumulation);
+ * everything else on fp32 FMA pipelines.  Needs oc_match_workspace_bytes() of context workspace
+ * (OC_ERR_WORKSPACE otherwise).  Calls on one context must not overlap on the device. */
+oc_status oc_match(oc_ctx* ctx, const oc_layout* layout, const void* x, float* best_sim,
+                   int32_t* best_idx, float* aux_sim, float* pair_sim, void* stream);
+
+/* select ("the r most redundant ... are marked for cached restoration while the retained
+ * representatives are computed normally", Sections 3.2.1-3.2.3).  Representatives are always kept.
+ *   mode OC_SELECT_THRESHOLD: a candidate is reused iff best_sim >= thr (self_match: and its best
+ *        match has a lower index; match_map then follows best_idx down to a kept token).
+ *   mode OC_SELECT_COUNT: in every group the n_reuse_per_group candidates with the largest
+ *        best_sim are reused (equal values: lower index first; clamped to the candidates present).
+ *   y_group_stride  rows reserved per group in the dense buffer: at least the number of kept units
+ *        (units_per_group always suffices; units_per_group - n_reuse in COUNT mode packs it tight)
+ *   kept_idx   [n_groups][y_group_stride] int32: kept units in ascending original index, tail -1
+ *   kept_count [n_groups] int32 (stays on the device: no host synchronisation)
+ *   match_map  [n_units] int32: i for kept units, else the representative standing for i
+ *   slot_of    [n_units] int32: row of unit i in the dense buffer (g*y_group_stride + rank), -1 if reused
+ * OC_ERR_UNSUPPORTED for COUNT with self_match or more than 65536 units per group. */
+oc_status oc_select(oc_ctx* ctx, const oc_layout* layout, const float* best_sim,
+                    const int32_t* best_idx, int mode, float thr, int64_t n_reuse_per_group,
+                    int64_t y_group_stride, int32_t* kept_idx, int32_t* kept_count,
+                    int32_t* match_map, int32_t* slot_of, void* stream);
+
+/* gather (Appendix A: "compact retained tokens"): y[slot] = row kept_idx[slot] of x for every slot
+ * in [0, n_slots) with kept_idx[slot] >= 0; other slots of y are left untouched.  Bit copy. */
+oc_status oc_gather(oc_ctx* ctx, const oc_rows* rows, const void* x, const int32_t* kept_idx,
+                    int64_t n_slots, void* y, void* stream);
+
+/* restore (Sections 3.2.1-3.2.3: skipped positions "are restored from cached activations
+ * associated with the same positions at the previous denoising step"; no averaging).
+ *   z      dense layer output, row slot_of[i] belongs to unit i
+ *   cache  strided like out: the previous step's restored output (nullable in
+ *          OC_RESTORE_FROM_REPRESENTATIVE mode)
+ *   out    out[i] = z[slot_of[i]] if slot_of[i] >= 0; otherwise cache[i] (FROM_CACHE) or
+ *          z[slot_of[match_map[i]]] (FROM_REPRESENTATIVE, for a first step without a cache).
+ *          out may equal cache: then only computed rows are written. */
+oc_status oc_restore(oc_ctx* ctx, const oc_rows* rows, const void* z, const void* cache,
+                     int64_t n_units, const int32_t* slot_of, const int32_t* match_map, void* out,
+                     int src_mode, void* stream);
+
+/* Layered Cache (Section 3.4): keep a layer's output at a scheduled step and reuse it for the
+ * following steps of the interval.
+ *   put  copies `bytes` from src into library-owned storage for `layer` (allocated on the first
+ *        put of that size: that put calls cudaMalloc) and records `step`.
+ *   get  OC_OK iff an entry exists and 0 <= step - stored_step < interval, else OC_CACHE_MISS.
+ *        On a hit: if dst != null the stored bytes are copied to dst (stream-ordered); if
+ *        view != null *view receives the library-owned device pointer (zero copy, valid until the
+ *        next put / clear for that layer); if bytes != null *bytes receives the entry size.
+ *   clear frees all entries (synchronises the device). */
+oc_status oc_layer_cache_put(oc_ctx* ctx, int layer, int step, const void* src, size_t bytes,
+                             void* stream);
+oc_status oc_layer_cache_get(oc_ctx* ctx, int layer, int step, int interval, void* dst,
+                             const void** view, size_t* bytes, void* stream);
+oc_status oc_layer_cache_clear(oc_ctx* ctx);
+
+/* One whole cache-wrapped layer call on HOST buffers, for callers that keep activations in host
+ * memory: copies x_host (layer input) and cache_host (previous output, same shape) to library-owned
+ * device staging, runs match -> select -> gather -> restore with the identity as the wrapped layer
+ * (z = the gathered rows), copies the restored tensor to out_host and the per-group kept counts to
+ * kept_count_host, and synchronises the stream before returning.  Pinned host memory makes the
+ * copies asynchronous to the host but the call still waits for completion. */
+oc_status oc_cache_step_host(oc_ctx* ctx, const oc_layout* layout, int mode, float thr,
+                             int64_t n_reuse_per_group, const void* x_host, const void* cache_host,
+                             void* out_host, int32_t* kept_count_host, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OMNICACHE_H_ */

@@ -1,0 +1,217 @@
+// Shared internals of the OmniCache sm_100a library: context, launch bookkeeping, small device helpers.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <map>
+#include <vector>
+
+#include "omnicache.h"
+
+namespace oc {
+
+struct KernelProf {
+    int64_t launches = 0;
+    double total_ms = 0.0;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> pending;
+};
+
+struct LayerEntry {
+    void* ptr = nullptr;
+    size_t bytes = 0;
+    size_t capacity = 0;
+    int step = 0;
+};
+
+}  // namespace oc
+
+struct oc_ctx {
+    int device = 0;
+    int sm_count = 0;
+    void* workspace = nullptr;
+    size_t workspace_bytes = 0;
+    int* d_status = nullptr;                 // device status word (first device-side error)
+    bool profile_on = false;
+    oc::KernelProf prof[OC_K_COUNT];
+    std::vector<cudaEvent_t> free_events;
+    std::map<int, oc::LayerEntry> layers;    // Layered Cache store
+    // staging for oc_cache_step_host
+    void* stage = nullptr;
+    size_t stage_bytes = 0;
+    // cached tensor maps of the tcgen05 matcher (opaque to the other files)
+    void* tc_cache = nullptr;
+};
+
+namespace oc {
+
+// RAII: makes ctx->device current for the duration of a call and restores the caller's device.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// Counts a kernel launch and, if timers are on, brackets it with events on the launching stream.
+struct LaunchScope {
+    oc_ctx* ctx; int k; cudaStream_t s; cudaEvent_t e0 = nullptr, e1 = nullptr;
+    LaunchScope(oc_ctx* c, int kernel, cudaStream_t stream);
+    ~LaunchScope();
+};
+
+inline oc_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? OC_OK : OC_ERR_CUDA; }
+inline oc_status last_launch_status() { return cuda_ok(cudaGetLastError()); }
+
+// Host-side geometry derived from a layout (validated before use).
+struct Geo {
+    int kind, dtype, B, T, H, W, C, sy, sx, oy, ox, gy, gx, self_match, frame_stat;
+    float eps;
+    int Hp, Wp;          // patch size (TOKEN) or frame size
+    int Hs, Ws;          // representative lattice size inside a patch
+    int64_t n_groups, units_per_group, reps_per_group, n_units;
+    int elem_bytes;
+};
+oc_status make_geo(const oc_layout* L, Geo* g);
+
+// Device-side description of the select / match group structure.
+struct GroupMap {
+    int kind, self_match;
+    int H, W, gy, gx, Hp, Wp, sy, sx, oy, ox;
+    int units_per_group;
+};
+GroupMap make_group_map(const Geo& g);
+
+__host__ __device__ inline int64_t gm_unit_index(const GroupMap& m, int64_t g, int u) {
+    if (m.kind == OC_KIND_TOKEN) {
+        int px = (int)(g % m.gx);
+        int py = (int)((g / m.gx) % m.gy);
+        int64_t bt = g / ((int64_t)m.gx * m.gy);
+        int ly = u / m.Wp, lx = u - ly * m.Wp;
+        return (bt * m.H + (int64_t)py * m.Hp + ly) * m.W + (int64_t)px * m.Wp + lx;
+    }
+    return g * m.units_per_group + u;
+}
+__host__ __device__ inline bool gm_is_rep(const GroupMap& m, int u) {
+    if (m.kind == OC_KIND_FRAME) return (u & 1) == 0;
+    if (m.self_match) return true;
+    int Wl = (m.kind == OC_KIND_TOKEN) ? m.Wp : m.W;
+    int ly = u / Wl, lx = u - ly * Wl;
+    return (ly % m.sy) == m.oy && (lx % m.sx) == m.ox;
+}
+__host__ __device__ inline bool gm_is_cand(const GroupMap& m, int u) {
+    if (m.kind == OC_KIND_TOKEN && m.self_match) return true;
+    return !gm_is_rep(m, u);
+}
+
+// ---- internal launchers (each validates nothing: the C-ABI layer in api.cu has done so) --------
+oc_status launch_gather(oc_ctx*, const oc_rows&, const void* x, const int32_t* kept_idx, int64_t n_slots,
+                        void* y, cudaStream_t);
+oc_status launch_restore(oc_ctx*, const oc_rows&, const void* z, const void* cache, int64_t n_units,
+                         const int32_t* slot_of, const int32_t* match_map, void* out, int src_mode,
+                         cudaStream_t);
+oc_status launch_copy(oc_ctx*, const void* src, void* dst, size_t bytes, cudaStream_t);
+oc_status launch_select(oc_ctx*, const Geo&, const float* best_sim, const int32_t* best_idx, int mode,
+                        float thr, int64_t n_reuse, int64_t y_stride, int32_t* kept_idx,
+                        int32_t* kept_count, int32_t* match_map, int32_t* slot_of, cudaStream_t);
+oc_status launch_match_frame(oc_ctx*, const Geo&, const void* x, float* best_sim, int32_t* best_idx,
+                             float* pos_sim, float* pair_sim, cudaStream_t);
+oc_status launch_match_block(oc_ctx*, const Geo&, const void* x, float* best_sim, int32_t* best_idx,
+                             cudaStream_t);
+oc_status launch_match_token(oc_ctx*, const Geo&, const void* x, float* best_sim, int32_t* best_idx,
+                             float* aux_sim, cudaStream_t);
+// tcgen05 path of launch_match_token; returns OC_ERR_UNSUPPORTED if the shape is not covered.
+bool tc_match_supported(const Geo&);
+oc_status launch_match_token_tc(oc_ctx*, const Geo&, const void* x, const float* inv_norm,
+                                unsigned long long* keys, float* aux_sim, cudaStream_t);
+void tc_cache_free(oc_ctx*);
+
+size_t match_workspace_bytes(const Geo&);
+
+// ---- device helpers ---------------------------------------------------------------------------
+#ifdef __CUDACC__
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_v4(void* p, uint4 v) {
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xFFFF0000u); }
+
+// Order-preserving map float -> uint32 (larger float <=> larger key) and back.
+__device__ __forceinline__ uint32_t f32_to_ordered(float f) {
+    uint32_t b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_to_f32(uint32_t k) {
+    uint32_t b = (k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k;
+    return __uint_as_float(b);
+}
+// (value, index) -> 64-bit key whose maximum is the largest value, then the lowest index.
+__device__ __forceinline__ unsigned long long pack_key(float v, uint32_t idx) {
+    return ((unsigned long long)f32_to_ordered(v) << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
+}
+
+// fp32 partial products of one 16-byte chunk of two rows: dot, |a|^2, |b|^2.
+template <int DT> struct Chunk;
+template <> struct Chunk<OC_DTYPE_BF16> {
+    static __device__ __forceinline__ void acc3(const uint4& a, const uint4& b, float& dot, float& na, float& nb) {
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float a0 = bf16_lo(aw[i]), a1 = bf16_hi(aw[i]), b0 = bf16_lo(bw[i]), b1 = bf16_hi(bw[i]);
+            dot = fmaf(a0, b0, dot); dot = fmaf(a1, b1, dot);
+            na = fmaf(a0, a0, na);   na = fmaf(a1, a1, na);
+            nb = fmaf(b0, b0, nb);   nb = fmaf(b1, b1, nb);
+        }
+    }
+    static __device__ __forceinline__ void acc2(const uint4& a, const uint4& b, float& dot, float& na) {
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float a0 = bf16_lo(aw[i]), a1 = bf16_hi(aw[i]), b0 = bf16_lo(bw[i]), b1 = bf16_hi(bw[i]);
+            dot = fmaf(a0, b0, dot); dot = fmaf(a1, b1, dot);
+            na = fmaf(a0, a0, na);   na = fmaf(a1, a1, na);
+        }
+    }
+    static __device__ __forceinline__ void sq(const uint4& a, float& na) {
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float a0 = bf16_lo(aw[i]), a1 = bf16_hi(aw[i]);
+            na = fmaf(a0, a0, na); na = fmaf(a1, a1, na);
+        }
+    }
+};
+template <> struct Chunk<OC_DTYPE_F32> {
+    static __device__ __forceinline__ void acc3(const uint4& a, const uint4& b, float& dot, float& na, float& nb) {
+        const float av[4] = {__uint_as_float(a.x), __uint_as_float(a.y), __uint_as_float(a.z), __uint_as_float(a.w)};
+        const float bv[4] = {__uint_as_float(b.x), __uint_as_float(b.y), __uint_as_float(b.z), __uint_as_float(b.w)};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            dot = fmaf(av[i], bv[i], dot); na = fmaf(av[i], av[i], na); nb = fmaf(bv[i], bv[i], nb);
+        }
+    }
+    static __device__ __forceinline__ void acc2(const uint4& a, const uint4& b, float& dot, float& na) {
+        const float av[4] = {__uint_as_float(a.x), __uint_as_float(a.y), __uint_as_float(a.z), __uint_as_float(a.w)};
+        const float bv[4] = {__uint_as_float(b.x), __uint_as_float(b.y), __uint_as_float(b.z), __uint_as_float(b.w)};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { dot = fmaf(av[i], bv[i], dot); na = fmaf(av[i], av[i], na); }
+    }
+    static __device__ __forceinline__ void sq(const uint4& a, float& na) {
+        const float av[4] = {__uint_as_float(a.x), __uint_as_float(a.y), __uint_as_float(a.z), __uint_as_float(a.w)};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) na = fmaf(av[i], av[i], na);
+    }
+};
+
+__device__ __forceinline__ float clamp_unit(float v) { return fminf(1.0f, fmaxf(-1.0f, v)); }
+#endif  // __CUDACC__
+
+}  // namespace oc

@@ -1,0 +1,303 @@
+// Frame Cache and Block Cache matching: a handful of cosine comparisons over very long descriptors
+// (Sections 3.2.1, 3.2.2).  About 3 FMA per element read, so both are HBM-bound streaming
+// reductions: 16-byte loads, fp32 accumulators for <a,b>, |a|^2, |b|^2, sub-warp shuffle
+// reductions, and a fixed-order two-level sum (no floating-point atomics) so results are
+// reproducible run to run.
+#include "common.cuh"
+
+namespace oc {
+
+static constexpr int PAIR_THREADS = 256;
+
+// lanes cooperating on one row: power of two, about 4 chunks per lane
+static int lanes_per_row(int64_t chunks_per_row) {
+    int l = 1;
+    while (l < 32 && (int64_t)l * 4 < chunks_per_row) l <<= 1;
+    return l;
+}
+
+template <int LPR>
+__device__ __forceinline__ float group_sum(float v) {
+#pragma unroll
+    for (int d = LPR / 2; d >= 1; d >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, d);
+    return v;
+}
+
+// fixed-order CTA reduction of one value per thread-group; result valid in thread 0
+__device__ __forceinline__ float cta_sum_fixed(float v, float* sh /*[PAIR_THREADS]*/) {
+    sh[threadIdx.x] = v;
+    __syncthreads();
+    for (int w = PAIR_THREADS / 2; w >= 1; w >>= 1) {
+        if ((int)threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+        __syncthreads();
+    }
+    float r = sh[0];
+    __syncthreads();
+    return r;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Frame Cache: for every adjacent pair (t, t-1) and position p, cos(x[t,p,:], x[t-1,p,:]).
+// grid = (position tiles, B*(T-1)).  A CTA covers POS_PER_CTA consecutive positions of one pair and
+// writes one partial record {sum cos, sum dot, sum |a|^2, sum |b|^2}.  Frame t is read from HBM by
+// pair (t, t-1) and again, out of L2, by pair (t+1, t).
+// ------------------------------------------------------------------------------------------------
+template <int DT, int LPR>
+__global__ void __launch_bounds__(PAIR_THREADS)
+frame_pair_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float eps,
+                  float* __restrict__ pos_sim, float4* __restrict__ partial, int pos_per_cta) {
+    __shared__ float sh[PAIR_THREADS];
+    const int q = blockIdx.y;                       // pair index b*(T-1) + (t-1)
+    const int b = q / (T - 1), t = q - b * (T - 1) + 1;
+    const int groups = PAIR_THREADS / LPR;
+    const int grp = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+    const long long row_bytes = (long long)cpr * 16;
+    const uint8_t* cur = x + ((long long)(b * T + t) * P) * row_bytes;
+    const uint8_t* prv = cur - (long long)P * row_bytes;
+    const int p_begin = blockIdx.x * pos_per_cta;
+    const int p_end = min(P, p_begin + pos_per_cta);
+
+    float s_cos = 0.f, s_dot = 0.f, s_na = 0.f, s_nb = 0.f;
+    // the trip count is the same for every thread of the CTA: the shuffles below name all 32 lanes
+    for (int p0 = p_begin; p0 < p_end; p0 += groups) {
+        const int p = p0 + grp;
+        const bool valid = p < p_end;
+        float dot = 0.f, na = 0.f, nb = 0.f;
+        if (valid) {
+            const uint8_t* a = cur + (long long)p * row_bytes;
+            const uint8_t* bb = prv + (long long)p * row_bytes;
+            int c = lane;
+            for (; c + LPR < cpr; c += 2 * LPR) {                   // two chunks in flight per row
+                uint4 a0 = ld_nc_v4(a + (long long)c * 16), b0 = ld_nc_v4(bb + (long long)c * 16);
+                uint4 a1 = ld_nc_v4(a + (long long)(c + LPR) * 16), b1 = ld_nc_v4(bb + (long long)(c + LPR) * 16);
+                Chunk<DT>::acc3(a0, b0, dot, na, nb);
+                Chunk<DT>::acc3(a1, b1, dot, na, nb);
+            }
+            if (c < cpr) {
+                uint4 a0 = ld_nc_v4(a + (long long)c * 16), b0 = ld_nc_v4(bb + (long long)c * 16);
+                Chunk<DT>::acc3(a0, b0, dot, na, nb);
+            }
+        }
+        dot = group_sum<LPR>(dot); na = group_sum<LPR>(na); nb = group_sum<LPR>(nb);
+        if (valid && lane == 0) {
+            float cs = clamp_unit(dot / (fmaxf(sqrtf(na), eps) * fmaxf(sqrtf(nb), eps)));
+            if (pos_sim) pos_sim[(long long)q * P + p] = cs;
+            s_cos += cs; s_dot += dot; s_na += na; s_nb += nb;
+        }
+    }
+    float r0 = cta_sum_fixed(s_cos, sh), r1 = cta_sum_fixed(s_dot, sh);
+    float r2 = cta_sum_fixed(s_na, sh), r3 = cta_sum_fixed(s_nb, sh);
+    if (threadIdx.x == 0) partial[(long long)q * gridDim.x + blockIdx.x] = make_float4(r0, r1, r2, r3);
+}
+
+// One warp per adjacent pair sums the CTA partials in a fixed order; then thread per frame picks the
+// better adjacent representative.
+__global__ void __launch_bounds__(PAIR_THREADS)
+frame_finalize_kernel(const float4* __restrict__ partial, int n_tiles, int B, int T, int P, int stat,
+                      float eps, float* __restrict__ pair_ws, float* __restrict__ pair_sim,
+                      float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
+    const int n_pairs = B * (T - 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int q = warp; q < n_pairs; q += PAIR_THREADS / 32) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        for (int i = lane; i < n_tiles; i += 32) {
+            float4 v = partial[(long long)q * n_tiles + i];
+            a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+        }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            a0 += __shfl_xor_sync(0xFFFFFFFFu, a0, d); a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, d);
+            a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, d); a3 += __shfl_xor_sync(0xFFFFFFFFu, a3, d);
+        }
+        if (lane == 0) {
+            float v = stat == OC_FRAME_FLAT_COS
+                          ? clamp_unit(a1 / (fmaxf(sqrtf(a2), eps) * fmaxf(sqrtf(a3), eps)))
+                          : a0 / (float)P;
+            pair_ws[q] = v;
+            if (pair_sim) pair_sim[q] = v;
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < B * T; i += PAIR_THREADS) {
+        const int b = i / T, t = i - b * T;
+        if ((t & 1) == 0) { best_sim[i] = -INFINITY; best_idx[i] = i; continue; }
+        float best = pair_ws[b * (T - 1) + t - 1]; int arg = i - 1;
+        if (t + 1 < T) {
+            float nxt = pair_ws[b * (T - 1) + t];
+            if (nxt > best) { best = nxt; arg = i + 1; }
+        }
+        best_sim[i] = best; best_idx[i] = arg;
+    }
+}
+
+template <int DT>
+static void frame_dispatch(int lpr, dim3 grid, cudaStream_t s, const uint8_t* x, int T, int P, int cpr, float eps,
+                           float* pos_sim, float4* partial, int ppc) {
+    switch (lpr) {
+        case 1:  frame_pair_kernel<DT, 1><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 2:  frame_pair_kernel<DT, 2><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 4:  frame_pair_kernel<DT, 4><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 8:  frame_pair_kernel<DT, 8><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 16: frame_pair_kernel<DT, 16><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        default: frame_pair_kernel<DT, 32><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+    }
+}
+
+static int frame_pos_per_cta(const Geo& g, int lpr) {
+    // every thread-group takes about 4 positions
+    return (PAIR_THREADS / lpr) * 4;
+}
+static int frame_tiles(const Geo& g) {
+    int cpr = g.C * g.elem_bytes / 16;
+    int ppc = frame_pos_per_cta(g, lanes_per_row(cpr));
+    return (g.H * g.W + ppc - 1) / ppc;
+}
+
+size_t frame_workspace_bytes(const Geo& g) {
+    size_t pairs = (size_t)g.B * (size_t)(g.T > 1 ? g.T - 1 : 0);
+    return pairs * (size_t)frame_tiles(g) * sizeof(float4) + pairs * sizeof(float) + 256;
+}
+
+oc_status launch_match_frame(oc_ctx* ctx, const Geo& g, const void* x, float* best_sim, int32_t* best_idx,
+                             float* pos_sim, float* pair_sim, cudaStream_t s) {
+    const int P = g.H * g.W, cpr = g.C * g.elem_bytes / 16;
+    const int n_pairs = g.B * (g.T - 1);
+    const int lpr = lanes_per_row(cpr);
+    const int ppc = frame_pos_per_cta(g, lpr);
+    const int n_tiles = frame_tiles(g);
+    float4* partial = (float4*)ctx->workspace;
+    float* pair_ws = (float*)((uint8_t*)ctx->workspace + ((size_t)(n_pairs > 0 ? n_pairs : 0) * n_tiles * sizeof(float4)));
+    if (n_pairs > 0) {
+        if (n_pairs > 65535) return OC_ERR_UNSUPPORTED;
+        dim3 grid((unsigned)n_tiles, (unsigned)n_pairs);
+        LaunchScope scope(ctx, OC_K_FRAME, s);
+        if (g.dtype == OC_DTYPE_BF16)
+            frame_dispatch<OC_DTYPE_BF16>(lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, ppc);
+        else
+            frame_dispatch<OC_DTYPE_F32>(lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, ppc);
+    }
+    {
+        LaunchScope scope(ctx, OC_K_FRAME_FIN, s);
+        frame_finalize_kernel<<<1, PAIR_THREADS, 0, s>>>(partial, n_tiles, g.B, g.T, P, g.frame_stat, g.eps,
+                                                         pair_ws, pair_sim, best_sim, best_idx);
+    }
+    return last_launch_status();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Block Cache: inside every sy x sx neighbourhood, each non-representative position's T*C
+// descriptor against the representative's.  grid = (cell tiles, B*T): a thread-group handles one
+// (cell, t) and writes the C-long partial sums {|rep|^2, then (dot, |cand|^2) per member}; the
+// finalize kernel adds the T partials of a cell in order of t.
+// ------------------------------------------------------------------------------------------------
+static constexpr int MAX_MEMBERS = 16;
+
+template <int DT, int LPR>
+__global__ void __launch_bounds__(PAIR_THREADS)
+block_partial_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr, int sy, int sx, int oy, int ox,
+                     float* __restrict__ partial, int rec /*floats per (cell,t)*/) {
+    const int bt = blockIdx.y;
+    const int cells_x = W / sx, cells = (H / sy) * cells_x;
+    const int groups = PAIR_THREADS / LPR;
+    const int grp = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+    const int cell_raw = blockIdx.x * groups + grp;
+    const bool valid = cell_raw < cells;             // out-of-range groups redo cell 0 and write nothing,
+    const int cell = valid ? cell_raw : 0;           // so that every lane takes part in the shuffles
+    const int cy = cell / cells_x, cx = cell - cy * cells_x;
+    const long long row_bytes = (long long)cpr * 16;
+    const uint8_t* frame = x + (long long)bt * H * W * row_bytes;
+    const uint8_t* rep = frame + ((long long)(cy * sy + oy) * W + (cx * sx + ox)) * row_bytes;
+    const int b = bt / T, t = bt - b * T;
+    float* out = partial + (((long long)b * cells + cell) * T + t) * rec;
+
+    float rn = 0.f;
+    for (int c = lane; c < cpr; c += LPR) { uint4 r = ld_nc_v4(rep + (long long)c * 16); Chunk<DT>::sq(r, rn); }
+    rn = group_sum<LPR>(rn);
+    if (valid && lane == 0) out[0] = rn;
+    int k = 0;
+    for (int my = 0; my < sy; ++my)
+        for (int mx = 0; mx < sx; ++mx) {
+            if (my == oy && mx == ox) continue;
+            const uint8_t* cand = frame + ((long long)(cy * sy + my) * W + (cx * sx + mx)) * row_bytes;
+            float dot = 0.f, na = 0.f;
+            int c = lane;
+            for (; c + LPR < cpr; c += 2 * LPR) {
+                uint4 a0 = ld_nc_v4(cand + (long long)c * 16), r0 = ld_nc_v4(rep + (long long)c * 16);
+                uint4 a1 = ld_nc_v4(cand + (long long)(c + LPR) * 16), r1 = ld_nc_v4(rep + (long long)(c + LPR) * 16);
+                Chunk<DT>::acc2(a0, r0, dot, na);
+                Chunk<DT>::acc2(a1, r1, dot, na);
+            }
+            if (c < cpr) {
+                uint4 a0 = ld_nc_v4(cand + (long long)c * 16), r0 = ld_nc_v4(rep + (long long)c * 16);
+                Chunk<DT>::acc2(a0, r0, dot, na);
+            }
+            dot = group_sum<LPR>(dot); na = group_sum<LPR>(na);
+            if (valid && lane == 0) { out[1 + 2 * k] = dot; out[2 + 2 * k] = na; }
+            ++k;
+        }
+}
+
+__global__ void __launch_bounds__(PAIR_THREADS)
+block_finalize_kernel(const float* __restrict__ partial, int B, int T, int H, int W, int sy, int sx, int oy, int ox,
+                      int rec, float eps, float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
+    const long long n = (long long)B * H * W;
+    const long long i = (long long)blockIdx.x * PAIR_THREADS + threadIdx.x;
+    if (i >= n) return;
+    const int P = H * W;
+    const int b = (int)(i / P), p = (int)(i - (long long)b * P);
+    const int y = p / W, xx = p - y * W;
+    const int my = y % sy, mx = xx % sx;
+    if (my == oy && mx == ox) { best_sim[i] = -INFINITY; best_idx[i] = (int32_t)i; return; }
+    const int cells_x = W / sx, cells = (H / sy) * cells_x;
+    const int cell = (y / sy) * cells_x + xx / sx;
+    int k = my * sx + mx;                        // rank among the neighbourhood's non-representatives
+    if (k > oy * sx + ox) --k;
+    const float* recs = partial + ((long long)b * cells + cell) * T * rec;
+    float rn = 0.f, dot = 0.f, na = 0.f;
+    for (int t = 0; t < T; ++t) { rn += recs[t * rec]; dot += recs[t * rec + 1 + 2 * k]; na += recs[t * rec + 2 + 2 * k]; }
+    best_sim[i] = clamp_unit(dot / (fmaxf(sqrtf(na), eps) * fmaxf(sqrtf(rn), eps)));
+    best_idx[i] = (int32_t)((long long)b * P + (y - my + oy) * W + (xx - mx + ox));
+}
+
+size_t block_workspace_bytes(const Geo& g) {
+    size_t cells = (size_t)(g.H / g.sy) * (size_t)(g.W / g.sx);
+    size_t rec = 1 + 2 * (size_t)(g.sy * g.sx - 1);
+    return (size_t)g.B * cells * (size_t)g.T * rec * sizeof(float) + 256;
+}
+
+template <int DT>
+static void block_dispatch(int lpr, dim3 grid, cudaStream_t s, const uint8_t* x, const Geo& g, int cpr, float* partial, int rec) {
+#define OC_BLK(L) block_partial_kernel<DT, L><<<grid, PAIR_THREADS, 0, s>>>(x, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec)
+    switch (lpr) {
+        case 1: OC_BLK(1); break; case 2: OC_BLK(2); break; case 4: OC_BLK(4); break;
+        case 8: OC_BLK(8); break; case 16: OC_BLK(16); break; default: OC_BLK(32); break;
+    }
+#undef OC_BLK
+}
+
+oc_status launch_match_block(oc_ctx* ctx, const Geo& g, const void* x, float* best_sim, int32_t* best_idx,
+                             cudaStream_t s) {
+    if (g.sy * g.sx > MAX_MEMBERS) return OC_ERR_UNSUPPORTED;
+    const int cpr = g.C * g.elem_bytes / 16;
+    const int lpr = lanes_per_row(cpr);
+    const int cells = (g.H / g.sy) * (g.W / g.sx);
+    const int rec = 1 + 2 * (g.sy * g.sx - 1);
+    float* partial = (float*)ctx->workspace;
+    if ((int64_t)g.B * g.T > 65535) return OC_ERR_UNSUPPORTED;
+    {
+        const int groups = PAIR_THREADS / lpr;
+        dim3 grid((unsigned)((cells + groups - 1) / groups), (unsigned)(g.B * g.T));
+        LaunchScope scope(ctx, OC_K_BLOCK, s);
+        if (g.dtype == OC_DTYPE_BF16) block_dispatch<OC_DTYPE_BF16>(lpr, grid, s, (const uint8_t*)x, g, cpr, partial, rec);
+        else block_dispatch<OC_DTYPE_F32>(lpr, grid, s, (const uint8_t*)x, g, cpr, partial, rec);
+    }
+    {
+        const long long n = (long long)g.B * g.H * g.W;
+        LaunchScope scope(ctx, OC_K_BLOCK_FIN, s);
+        block_finalize_kernel<<<(unsigned)((n + PAIR_THREADS - 1) / PAIR_THREADS), PAIR_THREADS, 0, s>>>(
+            partial, g.B, g.T, g.H, g.W, g.sy, g.sx, g.oy, g.ox, rec, g.eps, best_sim, best_idx);
+    }
+    return last_launch_status();
+}
+
+}  // namespace oc

@@ -1,0 +1,304 @@
+"""ctypes binding of the OmniCache C-ABI (``include/omnicache.h``); same names, marshalling only.
+
+Every function here turns torch tensors into raw device pointers and the current torch stream into a
+``cudaStream_t`` and calls the shared library: all arithmetic and data movement happen in the CUDA
+kernels.  There is no CPU fallback: a missing library raises at import, a failing call raises
+``OmniCacheError``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libomnicache_b200.so")
+
+OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_OOM, CACHE_MISS = range(9)
+KIND_TOKEN, KIND_FRAME, KIND_BLOCK = 0, 1, 2
+DTYPE_F32, DTYPE_BF16 = 0, 1
+SELECT_THRESHOLD, SELECT_COUNT = 0, 1
+RESTORE_FROM_CACHE, RESTORE_FROM_REPRESENTATIVE = 0, 1
+FRAME_MEAN_POS_COS, FRAME_FLAT_COS = 0, 1
+(K_NORMS, K_MATCH_TC, K_MATCH_SIMT, K_MATCH_FIN, K_FRAME, K_FRAME_FIN, K_BLOCK, K_BLOCK_FIN, K_SELECT,
+ K_GATHER, K_RESTORE, K_COPY) = range(12)
+K_COUNT = 12
+
+EXPORTS = (
+    "oc_status_str", "oc_layout_check", "oc_layout_counts", "oc_match_workspace_bytes",
+    "oc_rows_from_layout", "oc_layer_cache_would_hit", "oc_kernel_name", "oc_create", "oc_destroy",
+    "oc_device_status", "oc_profile_enable", "oc_profile_reset", "oc_profile_read", "oc_match",
+    "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
+    "oc_layer_cache_clear", "oc_cache_step_host",
+)
+
+
+class OmniCacheError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_str(status)}")
+
+
+class CLayout(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("kind", "dtype", "B", "T", "H", "W", "C", "sy", "sx", "oy", "ox",
+                                      "gy", "gx", "self_match", "frame_stat")] + [("eps", C.c_float)]
+
+
+class CRows(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("seg_bytes", "n_seg", "seg_stride", "unit_pitch",
+                                        "units_per_outer", "outer_pitch")]
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_23844_b200.build`")
+_lib = C.CDLL(LIB_PATH)
+
+_vp, _i, _i64, _f = C.c_void_p, C.c_int, C.c_int64, C.c_float
+_lib.oc_status_str.restype = C.c_char_p
+_lib.oc_status_str.argtypes = [_i]
+_lib.oc_kernel_name.restype = C.c_char_p
+_lib.oc_kernel_name.argtypes = [_i]
+_lib.oc_layout_check.argtypes = [_vp]
+_lib.oc_layout_counts.argtypes = [_vp, _vp, _vp, _vp]
+_lib.oc_match_workspace_bytes.argtypes = [_vp, _vp]
+_lib.oc_rows_from_layout.argtypes = [_vp, _i, _i, _vp]
+_lib.oc_layer_cache_would_hit.argtypes = [_i, _i, _i]
+_lib.oc_create.argtypes = [_vp, _i, C.c_size_t]
+_lib.oc_destroy.argtypes = [_vp]
+_lib.oc_device_status.argtypes = [_vp, _vp]
+_lib.oc_profile_enable.argtypes = [_vp, _i]
+_lib.oc_profile_reset.argtypes = [_vp]
+_lib.oc_profile_read.argtypes = [_vp, _i, _vp, _vp]
+_lib.oc_match.argtypes = [_vp] * 8
+_lib.oc_select.argtypes = [_vp, _vp, _vp, _vp, _i, _f, _i64, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.oc_gather.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp]
+_lib.oc_restore.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _i, _vp]
+_lib.oc_layer_cache_put.argtypes = [_vp, _i, _i, _vp, C.c_size_t, _vp]
+_lib.oc_layer_cache_get.argtypes = [_vp, _i, _i, _i, _vp, _vp, _vp, _vp]
+_lib.oc_layer_cache_clear.argtypes = [_vp]
+_lib.oc_cache_step_host.argtypes = [_vp, _vp, _i, _f, _i64, _vp, _vp, _vp, _vp, _vp]
+
+
+def status_str(s: int) -> str:
+    return _lib.oc_status_str(s).decode()
+
+
+def kernel_name(k: int) -> str:
+    return _lib.oc_kernel_name(k).decode()
+
+
+def _chk(st: int, where: str) -> None:
+    if st != OK:
+        raise OmniCacheError(st, where)
+
+
+@dataclass
+class Layout:
+    kind: int
+    dtype: int
+    B: int
+    T: int
+    H: int
+    W: int
+    C: int
+    sy: int = 2
+    sx: int = 2
+    oy: int = 0
+    ox: int = 0
+    gy: int = 1
+    gx: int = 1
+    self_match: int = 0
+    frame_stat: int = 0
+    eps: float = 1e-8
+
+    def c(self) -> CLayout:
+        return CLayout(self.kind, self.dtype, self.B, self.T, self.H, self.W, self.C, self.sy, self.sx,
+                       self.oy, self.ox, self.gy, self.gx, self.self_match, self.frame_stat, self.eps)
+
+    def check(self) -> int:
+        return layout_check(self)
+
+    def counts(self) -> tuple[int, int, int]:
+        return layout_counts(self)
+
+    @property
+    def n_groups(self) -> int:
+        return self.counts()[0]
+
+    @property
+    def units_per_group(self) -> int:
+        return self.counts()[1]
+
+    @property
+    def reps_per_group(self) -> int:
+        return self.counts()[2]
+
+    @property
+    def n_units(self) -> int:
+        g, u, _ = self.counts()
+        return g * u
+
+    @property
+    def elem_bytes(self) -> int:
+        return 4 if self.dtype == DTYPE_F32 else 2
+
+
+def layout_check(layout: Layout) -> int:
+    """oc_layout_check: returns the status code (no exception), host only."""
+    cl = layout.c()
+    return _lib.oc_layout_check(C.byref(cl))
+
+
+def layout_counts(layout: Layout) -> tuple[int, int, int]:
+    cl = layout.c()
+    g, u, r = C.c_int64(), C.c_int64(), C.c_int64()
+    _chk(_lib.oc_layout_counts(C.byref(cl), C.byref(g), C.byref(u), C.byref(r)), "oc_layout_counts")
+    return g.value, u.value, r.value
+
+
+def match_workspace_bytes(layout: Layout) -> int:
+    cl = layout.c()
+    n = C.c_size_t()
+    _chk(_lib.oc_match_workspace_bytes(C.byref(cl), C.byref(n)), "oc_match_workspace_bytes")
+    return n.value
+
+
+def rows_from_layout(layout: Layout, channels: int, elem_bytes: int) -> CRows:
+    cl, rows = layout.c(), CRows()
+    _chk(_lib.oc_rows_from_layout(C.byref(cl), channels, elem_bytes, C.byref(rows)), "oc_rows_from_layout")
+    return rows
+
+
+def layer_cache_would_hit(stored_step: int, step: int, interval: int) -> bool:
+    return bool(_lib.oc_layer_cache_would_hit(stored_step, step, interval))
+
+
+def _ptr(t) -> int | None:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_contiguous(), "tensors handed to the C-ABI must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+class Context:
+    """oc_create / oc_destroy and the per-context calls."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+        self._h = C.c_void_p()
+        _chk(_lib.oc_create(C.byref(self._h), device, workspace_bytes), "oc_create")
+        self.device = device
+        self.workspace_bytes = workspace_bytes
+
+    def close(self) -> None:
+        if self._h:
+            _lib.oc_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- status / profile ------------------------------------------------------------------------
+    def device_status(self) -> int:
+        code = C.c_int()
+        _chk(_lib.oc_device_status(self._h, C.byref(code)), "oc_device_status")
+        return code.value
+
+    def profile_enable(self, on: bool) -> None:
+        _chk(_lib.oc_profile_enable(self._h, int(on)), "oc_profile_enable")
+
+    def profile_reset(self) -> None:
+        _chk(_lib.oc_profile_reset(self._h), "oc_profile_reset")
+
+    def profile_read(self, kernel_id: int) -> tuple[int, float]:
+        n, ms = C.c_int64(), C.c_double()
+        _chk(_lib.oc_profile_read(self._h, kernel_id, C.byref(n), C.byref(ms)), "oc_profile_read")
+        return n.value, ms.value
+
+    def launches(self) -> dict[str, int]:
+        return {kernel_name(k): self.profile_read(k)[0] for k in range(K_COUNT)}
+
+    # -- hot path --------------------------------------------------------------------------------
+    def match(self, layout: Layout, x, best_sim, best_idx, aux_sim=None, pair_sim=None, stream=None,
+              check: bool = True) -> int:
+        cl = layout.c()
+        st = _lib.oc_match(self._h, C.byref(cl), _ptr(x), _ptr(best_sim), _ptr(best_idx), _ptr(aux_sim),
+                           _ptr(pair_sim), _stream(stream))
+        if check:
+            _chk(st, "oc_match")
+        return st
+
+    def select(self, layout: Layout, best_sim, best_idx, mode: int, thr: float, n_reuse_per_group: int,
+               y_group_stride: int, kept_idx, kept_count, match_map, slot_of, stream=None,
+               check: bool = True) -> int:
+        cl = layout.c()
+        st = _lib.oc_select(self._h, C.byref(cl), _ptr(best_sim), _ptr(best_idx), mode, thr,
+                            n_reuse_per_group, y_group_stride, _ptr(kept_idx), _ptr(kept_count),
+                            _ptr(match_map), _ptr(slot_of), _stream(stream))
+        if check:
+            _chk(st, "oc_select")
+        return st
+
+    def gather(self, rows: CRows, x, kept_idx, n_slots: int, y, stream=None, check: bool = True) -> int:
+        st = _lib.oc_gather(self._h, C.byref(rows), _ptr(x), _ptr(kept_idx), n_slots, _ptr(y), _stream(stream))
+        if check:
+            _chk(st, "oc_gather")
+        return st
+
+    def restore(self, rows: CRows, z, cache, n_units: int, slot_of, match_map, out,
+                src_mode: int = RESTORE_FROM_CACHE, stream=None, check: bool = True) -> int:
+        st = _lib.oc_restore(self._h, C.byref(rows), _ptr(z), _ptr(cache), n_units, _ptr(slot_of),
+                             _ptr(match_map), _ptr(out), src_mode, _stream(stream))
+        if check:
+            _chk(st, "oc_restore")
+        return st
+
+    def layer_cache_put(self, layer: int, step: int, src, nbytes: int | None = None, stream=None,
+                        check: bool = True) -> int:
+        if nbytes is None:
+            nbytes = src.numel() * src.element_size()
+        st = _lib.oc_layer_cache_put(self._h, layer, step, _ptr(src), nbytes, _stream(stream))
+        if check:
+            _chk(st, "oc_layer_cache_put")
+        return st
+
+    def layer_cache_get(self, layer: int, step: int, interval: int, dst=None, stream=None):
+        """Returns (hit, view pointer, bytes).  Raises on errors other than a miss."""
+        view, nbytes = C.c_void_p(), C.c_size_t()
+        st = _lib.oc_layer_cache_get(self._h, layer, step, interval, _ptr(dst), C.byref(view), C.byref(nbytes),
+                                     _stream(stream))
+        if st == CACHE_MISS:
+            return False, None, 0
+        _chk(st, "oc_layer_cache_get")
+        return True, view.value, nbytes.value
+
+    def layer_cache_clear(self) -> None:
+        _chk(_lib.oc_layer_cache_clear(self._h), "oc_layer_cache_clear")
+
+    def cache_step_host(self, layout: Layout, mode: int, thr: float, n_reuse_per_group: int, x_host, cache_host,
+                        out_host, kept_count_host=None, stream=None, check: bool = True) -> int:
+        """Host-buffer call: tensors are CPU (ideally pinned) torch tensors."""
+        cl = layout.c()
+        st = _lib.oc_cache_step_host(self._h, C.byref(cl), mode, thr, n_reuse_per_group, _ptr(x_host),
+                                     _ptr(cache_host), _ptr(out_host), _ptr(kept_count_host), _stream(stream))
+        if check:
+            _chk(st, "oc_cache_step_host")
+        return st

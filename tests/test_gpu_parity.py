@@ -1,0 +1,398 @@
+"""GPU parity: every op of the path, called through the C-ABI binding, against the CPU oracle on the
+same seeded inputs.  Tolerances: similarities 1e-3 absolute for bf16 inputs (fp32 accumulation),
+1e-5 for fp32 inputs; indices exact except near-ties (oracle top-two gap, or distance to the
+selection cut, below 1e-4); gather / restore / layered cache bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_23844_b200 import inputs
+
+import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+TOL = {inputs.F32: 1e-5, inputs.BF16: 1e-3}
+
+
+@pytest.fixture(scope="module")
+def oc():
+    from paper_2607_23844_b200 import build
+    build.build()
+    from paper_2607_23844_b200 import omnicache
+    assert torch.cuda.is_available()
+    return omnicache
+
+
+def run_chain(oc, oracle, w, Cout=None, full_oracle=True, sample_rows=0, want_aux=False, **layout_kw):
+    """match -> select -> gather -> restore for one workload, each stage compared with the oracle.
+    Returns a small report dict."""
+    L, Lo = H.layouts(oc, oracle, w, **layout_kw)
+    rep = {}
+    x_dev = H.to_dev(w.x)
+    with H.make_ctx(oc, L) as ctx:
+        # ---- match -----------------------------------------------------------------------------
+        m = H.gpu_match(oc, ctx, L, x_dev, want_aux=want_aux and L.kind != oc.KIND_BLOCK,
+                        want_pair=L.kind == oc.KIND_FRAME)
+        gs, gi = m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy()
+        if L.kind == oc.KIND_TOKEN:
+            if full_oracle:
+                ref = oracle.match_token(Lo, w.x, want_full=want_aux)
+                rows = None
+            else:
+                rng = np.random.default_rng(99)
+                rows = np.sort(rng.choice(Lo.n_units, sample_rows, replace=False))
+                ref = oracle.match_token(Lo, w.x, rows=rows)
+            rep["near_tie_rows"], rep["near_tie_differ"] = H.check_match_against_oracle(
+                oracle, Lo, w.x, gs, gi, ref, TOL[w.dtype], rows)
+            if want_aux and full_oracle:
+                a = m["aux"].cpu().numpy().astype(np.float64)
+                f = ref["full_sim"]
+                written = ~np.isnan(f)
+                assert np.array_equal(~np.isnan(a), written), "aux rows written differ from the oracle's"
+                assert np.abs(a[written] - f[written]).max() <= TOL[w.dtype]
+        elif L.kind == oc.KIND_FRAME:
+            ref = oracle.match_frame(Lo, w.x, want_pos=want_aux)
+            H.check_match_against_oracle(oracle, Lo, w.x, gs, gi, ref, TOL[w.dtype])
+            if L.T > 1:
+                assert np.abs(m["pair_sim"].cpu().numpy() - ref["pair_sim"]).max() <= TOL[w.dtype]
+            if want_aux and L.T > 1:
+                assert np.abs(m["aux"].cpu().numpy() - ref["pos_sim"]).max() <= TOL[w.dtype]
+        else:
+            ref = oracle.match_block(Lo, w.x)
+            H.check_match_against_oracle(oracle, Lo, w.x, gs, gi, ref, TOL[w.dtype])
+
+        # ---- select: (a) on the GPU's own similarities, oracle given the same arrays (exact) -----
+        mode = oc.SELECT_COUNT if w.mode == "count" else oc.SELECT_THRESHOLD
+        U = L.units_per_group
+        n_cand = U if w.self_match else U - L.reps_per_group
+        stride = U - min(w.n_reuse, n_cand) if mode == oc.SELECT_COUNT else U
+        s = H.gpu_select(oc, ctx, L, m["best_sim"], m["best_idx"], mode, w.thr, w.n_reuse, stride)
+        ref_s = H.check_select_against_oracle(oracle, Lo, gs, gi, mode, w.thr, w.n_reuse, stride, s)
+        # ---- select: (b) on the oracle's similarities uploaded to the GPU (exact, no exceptions) ---
+        if full_oracle:
+            os_, oi = ref["best_sim"], ref["best_idx"]
+            s2 = H.gpu_select(oc, ctx, L, H.to_dev(os_), H.to_dev(oi), mode, w.thr, w.n_reuse, stride)
+            ref_s2 = H.check_select_against_oracle(oracle, Lo, os_, oi, mode, w.thr, w.n_reuse, stride, s2)
+            # (c) the two selections may differ only at units whose oracle similarity is within 1e-4
+            # of the cut (count mode: the last reused value; threshold mode: thr)
+            kept_a, kept_b = ref_s["slot_of"] >= 0, ref_s2["slot_of"] >= 0
+            differ = np.nonzero(kept_a != kept_b)[0]
+            if differ.size:
+                G = Lo.n_groups
+                grp_of = np.empty(Lo.n_units, np.int64)
+                for g in range(G):
+                    grp_of[[Lo.unit_index(g, u) for u in range(U)]] = g
+                for i in differ:
+                    if mode == oc.SELECT_COUNT:
+                        ids = np.nonzero((grp_of == grp_of[i]) & ~kept_b & np.isfinite(os_))[0]
+                        cut = os_[ids].min()
+                    else:
+                        cut = w.thr
+                    assert abs(float(os_[i]) - float(cut)) < H.NEAR_TIE, (i, os_[i], cut)
+            rep["cut_differ"] = int(differ.size)
+            assert np.array_equal(ref_s["kept_count"], ref_s2["kept_count"]) or mode == oc.SELECT_THRESHOLD
+
+        # ---- gather ------------------------------------------------------------------------------
+        Ro = oracle.rows_for(Lo, w.shape[-1], w.elem_bytes)
+        n_slots = s["kept_idx"].numel()
+        y = torch.full((n_slots, Ro.row_bytes), 0xAB, device="cuda", dtype=torch.uint8)
+        ctx.gather(H.crows(oc, Ro), x_dev, s["kept_idx"], n_slots, y)
+        y_ref = oracle.gather(Ro, w.x, ref_s["kept_idx"], fill=0xAB)
+        assert H.dev_bytes(y) == y_ref.tobytes()
+
+        # ---- wrapped layer stand-in (outside the path) and restore ---------------------------------
+        Cout = Cout or w.shape[-1]
+        eb = w.elem_bytes
+        Rz = oracle.rows_for(Lo, Cout, eb)
+        rng = np.random.default_rng(123)
+        if "layer_weight" in w.extra and Cout == w.shape[-1] and L.kind == oc.KIND_TOKEN:
+            wt = w.extra["layer_weight"].astype(np.float64)
+            yv = y_ref.view(np.float32).reshape(n_slots, -1).astype(np.float64)
+            z_np = (yv @ wt).astype(np.float32)
+            cache_np = (w.extra["x_prev"].reshape(-1, Cout).astype(np.float64) @ wt).astype(np.float32)
+        else:
+            n_el = n_slots * Rz.row_bytes // eb
+            z_np = inputs.random_rows(5, (n_el,), w.dtype)
+            cache_np = inputs.random_rows(6, w.shape[:-1] + (Cout,), w.dtype)
+        z_dev, cache_dev = H.to_dev(z_np), H.to_dev(cache_np)
+        n_units = Lo.n_units
+        for src_mode in (oc.RESTORE_FROM_CACHE, oc.RESTORE_FROM_REPRESENTATIVE):
+            out = torch.full((cache_np.nbytes,), 0xCD, device="cuda", dtype=torch.uint8)
+            ctx.restore(H.crows(oc, Rz), z_dev, cache_dev, n_units, s["slot_of"], s["match_map"], out, src_mode)
+            want = oracle.restore(Rz, z_np, cache_np, n_units, ref_s["slot_of"], ref_s["match_map"], src_mode)
+            assert H.dev_bytes(out) == want.tobytes(), f"restore mode {src_mode}"
+        inplace = cache_dev.clone()
+        ctx.restore(H.crows(oc, Rz), z_dev, inplace, n_units, s["slot_of"], s["match_map"], inplace)
+        want = oracle.restore(Rz, z_np, cache_np.copy(), n_units, ref_s["slot_of"], ref_s["match_map"], in_place=True)
+        assert H.dev_bytes(inplace) == want.tobytes()
+        torch.cuda.synchronize()
+        assert ctx.device_status() == oc.OK
+        rep["reused"] = int((ref_s["slot_of"] < 0).sum())
+        rep["launches"] = ctx.launches()
+    return rep
+
+
+# ---------------------------------------------------------------------------------------------------
+# config 1 exactly, and small versions of configs 2-4 that span several tiles with ragged tails
+# ---------------------------------------------------------------------------------------------------
+def test_config1_tiny_token_cache_fp32(oc, oracle):
+    rep = run_chain(oc, oracle, inputs.tiny_token_cache(), want_aux=True)
+    assert 40 <= rep["reused"] <= 110
+    assert rep["launches"]["match_simt"] == 1
+
+
+@pytest.mark.parametrize("shape,groups,lattice,dtype", [
+    ((2, 1, 24, 40, 200), (1, 1), (2, 2, 0, 0), inputs.BF16),     # K tail (200 % 64), 240 reps
+    ((1, 2, 32, 32, 128), (2, 2), (2, 2, 1, 1), inputs.BF16),     # patches, other lattice offset
+    ((1, 1, 36, 72, 64), (1, 1), (2, 2, 0, 1), inputs.BF16),      # 18 x 36 lattice: ragged both ways
+    ((2, 1, 16, 48, 96), (2, 4), (2, 2, 0, 0), inputs.BF16),      # 8 token groups per frame
+    ((1, 1, 12, 18, 40), (1, 1), (3, 3, 1, 2), inputs.BF16),      # 3 x 3 neighbourhoods
+    ((1, 2, 16, 16, 36), (1, 1), (2, 2, 0, 0), inputs.F32),       # fp32, C % 32 != 0
+    ((1, 1, 64, 64, 320), (1, 1), (2, 2, 0, 0), inputs.BF16),     # 1024 reps: several N tiles
+])
+def test_token_chain_small(oc, oracle, shape, groups, lattice, dtype):
+    B, T, Hh, W, C = shape
+    w = inputs.sd3_token_cache(seed=21, B=B * T, H=Hh, W=W, C=C, groups=groups, dtype=dtype)
+    w.x = w.x.reshape(shape); w.shape = shape
+    sy, sx, oy, ox = lattice
+    U = (Hh // groups[0]) * (W // groups[1])
+    w.n_reuse = (U - U // (sy * sx)) // 2
+    rep = run_chain(oc, oracle, w, want_aux=True, sy=sy, sx=sx, oy=oy, ox=ox)
+    if dtype == inputs.BF16:
+        assert rep["launches"]["match_tc"] + rep["launches"]["match_simt"] == 1
+
+
+@pytest.mark.parametrize("dtype", [inputs.BF16, inputs.F32])
+@pytest.mark.parametrize("T,stat", [(7, 0), (6, 1), (2, 0), (1, 0)])
+def test_frame_chain_small(oc, oracle, dtype, T, stat):
+    w = inputs.svd_frames(seed=31, T=T, H=9, W=13, C=40, dtype=dtype, thr=0.9)
+    rep = run_chain(oc, oracle, w, Cout=24, want_aux=True, frame_stat=stat)
+    assert rep["reused"] == T // 2          # rho = 0.95 > 0.9: every odd frame is reused
+
+
+@pytest.mark.parametrize("dtype,lattice", [(inputs.BF16, (2, 2, 0, 0)), (inputs.F32, (2, 2, 1, 0)),
+                                          (inputs.BF16, (1, 2, 0, 1)), (inputs.BF16, (3, 2, 2, 1))])
+def test_block_chain_small(oc, oracle, dtype, lattice):
+    sy, sx, oy, ox = lattice
+    w = inputs.latte_blocks(seed=41, T=5, H=6, W=10, C=72, dtype=dtype)
+    rep = run_chain(oc, oracle, w, Cout=40, sy=sy, sx=sx, oy=oy, ox=ox)
+    assert 0 < rep["reused"] < 60
+
+
+# ---------------------------------------------------------------------------------------------------
+# full-size configs 2-4
+# ---------------------------------------------------------------------------------------------------
+def test_config2_sd3_token_cache_full(oc, oracle):
+    w = inputs.sd3_token_cache()
+    rep = run_chain(oc, oracle, w, full_oracle=True)
+    assert rep["launches"]["match_tc"] == 1, "the bf16 dense matcher must run on the tcgen05 kernel"
+    assert rep["reused"] == 2 * 1536
+    print("config2 report:", rep)
+
+
+@pytest.mark.parametrize("groups", [(2, 1), (2, 2), (4, 2)])
+def test_config2_token_groups_sampled(oc, oracle, groups):
+    w = inputs.sd3_token_cache(groups=groups)
+    rep = run_chain(oc, oracle, w, full_oracle=False, sample_rows=384)
+    assert rep["launches"]["match_tc"] == 1
+
+
+def test_config3_svd_frame_cache_full(oc, oracle):
+    w = inputs.svd_frames()
+    rep = run_chain(oc, oracle, w, want_aux=True)
+    assert rep["reused"] == 12
+
+
+def test_config4_latte_block_cache_full(oc, oracle):
+    w = inputs.latte_blocks()
+    rep = run_chain(oc, oracle, w)
+    assert 40 <= rep["reused"] <= 160
+
+
+# ---------------------------------------------------------------------------------------------------
+# config 5: three U-Net levels x three caches x keep ratios, with step drift and the Layered Cache
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("level", [0, 1, 2])
+def test_config5_levels(oc, oracle, level):
+    Hh, W, C = inputs.SVD_LEVELS[level]
+    base = inputs.svd_frames(seed=1005 + level, T=25, H=Hh, W=W, C=C, rho=0.95, kind="token")
+    steps = (0, 1, 24) if level > 0 else (0, 1)
+    rng = np.random.default_rng(77)
+    x = base.x
+    lc_ref = oracle.LayerCache()
+    L_any = oc.Layout(oc.KIND_TOKEN, base.dtype, *base.shape)
+    with oc.Context(0, oc.match_workspace_bytes(L_any)) as lc_ctx:
+        for step in range(max(steps) + 1):
+            if step > 0:
+                x = inputs.drift_step(rng, x, base.dtype)
+            # Layered Cache: put every 5 steps, get on the others (interval N = 5), bit-exact
+            x_dev = H.to_dev(x)
+            if step % 5 == 0:
+                lc_ctx.layer_cache_put(level, step, x_dev)
+                lc_ref.put(level, step, x)
+            dst = torch.zeros_like(x_dev)
+            hit, view, nbytes = lc_ctx.layer_cache_get(level, step, 5, dst)
+            want = lc_ref.get(level, step, 5)
+            assert hit == (want is not None)
+            if hit:
+                assert nbytes == len(want) and H.dev_bytes(dst) == want
+            if step not in steps:
+                continue
+            for kind in ("token", "frame", "block"):
+                ratios = (0.25, 0.5, 0.75) if step == 0 else (0.5,)
+                for ratio in ratios:
+                    w = inputs.Workload(f"svd_l{level}_{kind}", kind, base.dtype, base.shape, x, mode="count")
+                    if kind == "token":
+                        U, R = Hh * W, (Hh // 2) * (W // 2)
+                    elif kind == "frame":
+                        U, R = 25, 13
+                    else:
+                        U, R = Hh * W, (Hh // 2) * (W // 2)
+                    w.n_reuse = inputs.keep_ratio_to_reuse(U, U - R, ratio)
+                    full = kind != "token"
+                    run_chain(oc, oracle, w, full_oracle=full, sample_rows=160)
+        assert lc_ctx.layer_cache_get(level, max(steps) + 5, 5)[0] is False
+
+
+# ---------------------------------------------------------------------------------------------------
+# edge cases
+# ---------------------------------------------------------------------------------------------------
+def test_identity_selection_roundtrip_and_extremes(oc, oracle):
+    w = inputs.sd3_token_cache(seed=5, B=2, H=16, W=24, C=64)
+    L, Lo = H.layouts(oc, oracle, w)
+    x_dev = H.to_dev(w.x)
+    U, n_cand = L.units_per_group, L.units_per_group - L.reps_per_group
+    R = H.crows(oc, oracle.rows_for(Lo, 64, 2))
+    with H.make_ctx(oc, L) as ctx:
+        m = H.gpu_match(oc, ctx, L, x_dev)
+        for mode, thr, n_reuse in ((oc.SELECT_COUNT, 0.0, 0), (oc.SELECT_THRESHOLD, 2.0, 0)):
+            s = H.gpu_select(oc, ctx, L, m["best_sim"], m["best_idx"], mode, thr, n_reuse, U)
+            assert torch.equal(s["kept_idx"].cpu(), torch.arange(L.n_units, dtype=torch.int32))
+            y = torch.zeros_like(x_dev)
+            ctx.gather(R, x_dev, s["kept_idx"], L.n_units, y)
+            out = torch.zeros_like(x_dev)
+            ctx.restore(R, y, torch.zeros_like(x_dev), L.n_units, s["slot_of"], s["match_map"], out)
+            assert torch.equal(out, x_dev), "restore after an identity selection must reproduce the input"
+        # everything reusable is reused: count >= candidates, threshold -inf
+        for mode, thr, n_reuse, stride in ((oc.SELECT_COUNT, 0.0, n_cand + 7, U - n_cand),
+                                           (oc.SELECT_THRESHOLD, -float("inf"), 0, U)):
+            s = H.gpu_select(oc, ctx, L, m["best_sim"], m["best_idx"], mode, thr, n_reuse, stride)
+            H.check_select_against_oracle(oracle, Lo, m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy(),
+                                          mode, thr, n_reuse, stride, s)
+            assert int(s["kept_count"].sum()) == L.n_groups * L.reps_per_group
+
+
+def test_duplicates_zero_rows_and_ties(oc, oracle):
+    rng = np.random.default_rng(9)
+    xf = rng.standard_normal((1, 1, 32, 32, 128)).astype(np.float32)
+    xf[0, 0, 0, 2] = xf[0, 0, 0, 0]          # two identical representatives
+    xf[0, 0, 1, 1] = xf[0, 0, 0, 0]          # a candidate equal to both: lowest index must win
+    xf[0, 0, 5, 5] = 0.0                     # all-zero candidate: similarity 0 with everything
+    xf[0, 0, 6, 6] = 0.0                     # all-zero representative
+    xf[0, 0, 9, 9] = 4.0 * xf[0, 0, 8, 8]    # scaled copy: similarity 1
+    for dtype in (inputs.BF16, inputs.F32):
+        x = xf if dtype == inputs.F32 else inputs.to_bf16_bits(xf)
+        w = inputs.Workload("dups", "token", dtype, xf.shape, x, mode="count", n_reuse=100)
+        L, Lo = H.layouts(oc, oracle, w)
+        with H.make_ctx(oc, L) as ctx:
+            m = H.gpu_match(oc, ctx, L, H.to_dev(x))
+        gs, gi = m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy()
+        assert gi[33] == 0 and abs(gs[33] - 1.0) <= 1e-6
+        assert gi[9 * 32 + 9] == 8 * 32 + 8 and abs(gs[9 * 32 + 9] - 1.0) <= 1e-6
+        assert gs[5 * 32 + 5] == 0.0 and gi[5 * 32 + 5] == 0     # all similarities 0: lowest index
+        ref = oracle.match_token(Lo, x)
+        H.check_match_against_oracle(oracle, Lo, x, gs, gi, ref, TOL[dtype])
+
+
+def test_determinism_and_profile_counters(oc, oracle):
+    w = inputs.sd3_token_cache(seed=8, B=2, H=32, W=32, C=256)
+    L, _ = H.layouts(oc, oracle, w)
+    x_dev = H.to_dev(w.x)
+    with H.make_ctx(oc, L) as ctx:
+        ctx.profile_enable(True)
+        a = H.gpu_match(oc, ctx, L, x_dev)
+        b = H.gpu_match(oc, ctx, L, x_dev)
+        assert torch.equal(a["best_sim"], b["best_sim"]) and torch.equal(a["best_idx"], b["best_idx"])
+        n, ms = ctx.profile_read(oc.K_NORMS)
+        assert n == 2 and ms > 0.0
+        n_tc, ms_tc = ctx.profile_read(oc.K_MATCH_TC)
+        n_si, ms_si = ctx.profile_read(oc.K_MATCH_SIMT)
+        assert n_tc + n_si == 2 and ms_tc + ms_si > 0.0
+        ctx.profile_reset()
+        assert ctx.profile_read(oc.K_NORMS) == (0, 0.0)
+
+
+def test_runtime_argument_errors_launch_nothing(oc, oracle):
+    w = inputs.sd3_token_cache(seed=5, B=1, H=16, W=16, C=64)
+    L, Lo = H.layouts(oc, oracle, w)
+    x_dev = H.to_dev(w.x)
+    n = L.n_units
+    sim = torch.zeros(n, device="cuda"); idx = torch.zeros(n, device="cuda", dtype=torch.int32)
+    sentinel = torch.full((n,), 7, device="cuda", dtype=torch.int32)
+    with oc.Context(0, 16) as small:
+        assert small.match(L, x_dev, sim, idx, check=False) == oc.ERR_WORKSPACE
+    with H.make_ctx(oc, L) as ctx:
+        before = dict(ctx.launches())
+        assert ctx.match(L, x_dev.view(torch.uint8)[2:].data_ptr(), sim, idx, check=False) == oc.ERR_ALIGNMENT
+        U = L.units_per_group
+        k = sentinel.clone()
+        args = (k, k.clone(), k.clone(), k.clone())
+        assert ctx.select(L, sim, idx, 5, 0.5, 0, U, *args, check=False) == oc.ERR_INVALID_ARG
+        assert ctx.select(L, sim, idx, oc.SELECT_COUNT, 0.0, -1, U, *args, check=False) == oc.ERR_INVALID_ARG
+        assert ctx.select(L, sim, idx, oc.SELECT_COUNT, 0.0, 10, U - 11, *args, check=False) == oc.ERR_INVALID_ARG
+        assert ctx.select(L, sim, idx, oc.SELECT_THRESHOLD, float("nan"), 0, U, *args, check=False) == oc.ERR_INVALID_ARG
+        Ls = oc.Layout(oc.KIND_TOKEN, w.dtype, *w.shape, self_match=1)
+        assert ctx.select(Ls, sim, idx, oc.SELECT_COUNT, 0.0, 4, U, *args, check=False) == oc.ERR_UNSUPPORTED
+        rows = oc.CRows(24, 1, 0, 24, 1 << 40, 0)
+        assert ctx.gather(rows, x_dev, k, 4, x_dev, check=False) == oc.ERR_ALIGNMENT
+        good = H.crows(oc, oracle.rows_for(Lo, 64, 2))
+        assert ctx.restore(good, x_dev, None, n, k, k, x_dev.clone(), oc.RESTORE_FROM_CACHE, check=False) == oc.ERR_INVALID_ARG
+        assert ctx.restore(good, x_dev, x_dev, n, k, k, x_dev, check=False) == oc.ERR_INVALID_ARG     # out == z
+        assert ctx.layer_cache_get(0, 0, 5)[0] is False
+        torch.cuda.synchronize()
+        assert torch.equal(k, sentinel), "a rejected call must not write outputs"
+        assert ctx.launches() == before, "a rejected call must not launch"
+        assert ctx.device_status() == oc.OK
+
+
+def test_select_capacity_limits(oc, oracle):
+    # 65536 units per group is the supported maximum; one more patch row is rejected
+    L = oc.Layout(oc.KIND_TOKEN, oc.DTYPE_BF16, 1, 1, 256, 256, 8)
+    n = L.n_units
+    rng = np.random.default_rng(1)
+    sim_np = np.round(rng.uniform(-1, 1, n).astype(np.float32) * 64) / 64        # many equal values
+    Lo = oracle.Layout(0, 1, 1, 1, 256, 256, 8)
+    rep_mask = np.array([Lo.is_rep(u) for u in range(n)])
+    sim_np[rep_mask] = -np.inf
+    idx_np = np.where(rep_mask, np.arange(n), 0).astype(np.int32)
+    with oc.Context(0, 0) as ctx:
+        n_reuse = 20000
+        s = H.gpu_select(oc, ctx, L, H.to_dev(sim_np), H.to_dev(idx_np), oc.SELECT_COUNT, 0.0, n_reuse, n - n_reuse)
+        H.check_select_against_oracle(oracle, Lo, sim_np, idx_np, oc.SELECT_COUNT, 0.0, n_reuse, n - n_reuse, s)
+        big = oc.Layout(oc.KIND_TOKEN, oc.DTYPE_BF16, 1, 1, 258, 256, 8)
+        t = torch.zeros(big.n_units, device="cuda")
+        ti = torch.zeros(big.n_units, device="cuda", dtype=torch.int32)
+        assert ctx.select(big, t, ti, oc.SELECT_THRESHOLD, 0.5, 0, big.units_per_group, ti.clone(), ti.clone(),
+                          ti.clone(), ti.clone(), check=False) == oc.ERR_UNSUPPORTED
+
+
+def test_cache_step_host_matches_device_path(oc, oracle):
+    w = inputs.sd3_token_cache(seed=12, B=2, H=32, W=32, C=128)
+    L, Lo = H.layouts(oc, oracle, w)
+    cache_np = inputs.random_rows(3, w.shape, w.dtype)
+    xh = torch.from_numpy(w.x.view(np.int16)).pin_memory()
+    ch = torch.from_numpy(cache_np.view(np.int16)).pin_memory()
+    oh = torch.zeros_like(xh).pin_memory()
+    kh = torch.zeros(L.n_groups, dtype=torch.int32).pin_memory()
+    with H.make_ctx(oc, L) as ctx:
+        ctx.cache_step_host(L, oc.SELECT_COUNT, 0.0, w.n_reuse, xh, ch, oh, kh)
+        m = H.gpu_match(oc, ctx, L, H.to_dev(w.x))
+    gs, gi = m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy()
+    U = L.units_per_group
+    s = oracle.select(Lo, gs, gi, 1, 0.0, w.n_reuse, U)
+    R = oracle.rows_for(Lo, 128, 2)
+    y = oracle.gather(R, w.x, s["kept_idx"])
+    want = oracle.restore(R, y, cache_np, Lo.n_units, s["slot_of"], s["match_map"])
+    assert oh.numpy().tobytes() == want.tobytes()
+    assert np.array_equal(kh.numpy(), s["kept_count"])
