@@ -84,7 +84,8 @@ def check_match_against_oracle(oracle, Lo, x_np, got_sim, got_idx, ref, tol, row
     diff = np.nonzero(cand & (gi != ri))[0]
     near = 0
     if "second_sim" in ref:
-        gap = rs.astype(np.float64) - ref["second_sim"][sel].astype(np.float64)
+        with np.errstate(invalid="ignore"):      # representative rows: -inf - -inf
+            gap = rs.astype(np.float64) - ref["second_sim"][sel].astype(np.float64)
         near = int((cand & (gap < NEAR_TIE)).sum())
         C = Lo.C
         for k in diff:
