@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the OmniCache hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A "step" is one pass of the whole path over one batch of synthetic input:
+    match -> select -> gather -> restore -> layer_cache_put -> layer_cache_get (copying)
+with the identity as the wrapped layer (restore reads the gathered rows).  The default workload is
+the SD3-shaped Token Cache (batch 2 x 64x64 tokens x 1536 channels, bf16, reuse the 50 % most similar
+candidates).  Prints ONE JSON line on rank 0.
+
+`value` counts, per second, the candidates matched plus the rows restored by all ranks, with the
+inputs resident in HBM; `e2e` is the same count through the host-buffer C-ABI call, host<->device
+copies included.  Buffers rotate through a ring larger than 4x L2, so every step starts L2-cold.
+`--impl reference` times the CPU oracle (the only reference implementation that exists) instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_23844_b200 import inputs, sharding  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists for the workload.
+NCU_TRAFFIC_BYTES = {"sd3_token": None}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK)
+    d["_source"] = "fallback"
+    return d
+
+
+def make_workload(name: str, seed_offset: int = 0) -> inputs.Workload:
+    if name == "sd3_token":
+        return inputs.sd3_token_cache(seed=1002 + seed_offset)
+    if name == "svd_frame":
+        return inputs.svd_frames(seed=1003 + seed_offset)
+    if name == "latte_block":
+        return inputs.latte_blocks(seed=1004 + seed_offset)
+    if name.startswith("svd_token_l"):
+        H, W, C = inputs.SVD_LEVELS[int(name[-1])]
+        w = inputs.svd_frames(seed=1005 + seed_offset, H=H, W=W, C=C, kind="token")
+        w.mode = "count"
+        w.n_reuse = inputs.keep_ratio_to_reuse(H * W, H * W - (H // 2) * (W // 2), 0.5)
+        return w
+    raise SystemExit(f"unknown workload {name}")
+
+
+KIND = {"token": 0, "frame": 1, "block": 2}
+
+
+def unit_counts(w: inputs.Workload):
+    """(groups, units per group, representatives per group) without touching any library."""
+    B, T, H, W, C = w.shape
+    if w.kind == "token":
+        gy, gx = w.groups
+        u = (H // gy) * (W // gx)
+        return B * T * gy * gx, u, (u if w.self_match else u // 4)
+    if w.kind == "frame":
+        return B, T, (T + 1) // 2
+    return B, H * W, (H // 2) * (W // 2)
+
+
+# ---------------------------------------------------------------------------------------------------
+# clocks during the timed region (NVML, read only)
+# ---------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, uuid: str):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if r & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.005)
+
+    def __enter__(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "samples": len(self.samples), "reasons": sorted(self.reasons)}
+
+
+# ---------------------------------------------------------------------------------------------------
+# CPU oracle timing (baseline leg and --impl reference)
+# ---------------------------------------------------------------------------------------------------
+def oracle_sample_step(w: inputs.Workload, n_rows: int, seed: int = 0):
+    """Times the oracle, as it stands, on a bounded sample of one step of workload `w`:
+    match on `n_rows` sampled candidates (scaled to all candidates), then select / gather / restore
+    at full size.  Returns (tokens_per_s, seconds, description, threads)."""
+    import oracle
+    oracle.build()
+    Lo = oracle.Layout(KIND[w.kind], w.dtype, *w.shape, gy=w.groups[0], gx=w.groups[1],
+                       self_match=int(w.self_match))
+    G, U, R = unit_counts(w)
+    n_units = G * U
+    n_cand = G * (U if w.self_match else U - R)
+    mode = 1 if w.mode == "count" else 0
+    if w.kind == "token":
+        rng = np.random.default_rng(seed)
+        cands = np.array([i for i in rng.permutation(n_units) if not _is_rep_token(w, int(i))][:n_rows],
+                         dtype=np.int32)
+    t0 = time.perf_counter()
+    if w.kind == "token":
+        m = oracle.match_token(Lo, w.x, rows=np.sort(cands))
+        t_match = (time.perf_counter() - t0) * (n_cand / max(len(cands), 1))
+        sample = ("full step" if len(cands) == n_cand else
+                  f"match on {len(cands)} of {n_cand} sampled candidates (time scaled), select/gather/restore full size")
+        best_sim = np.where(np.isnan(m["best_sim"]), np.float32(-np.inf), m["best_sim"])
+        best_idx = np.where(m["best_idx"] < 0, np.arange(n_units, dtype=np.int32), m["best_idx"])
+        # unsampled candidates get a deterministic filler similarity so that select sees full-size input
+        filler = np.random.default_rng(1).uniform(0.9, 0.99, n_units).astype(np.float32)
+        unsampled = np.ones(n_units, bool); unsampled[cands] = False
+        cand_mask = np.array([not _is_rep_token(w, i) for i in range(n_units)])
+        best_sim = np.where(unsampled & cand_mask, filler, best_sim).astype(np.float32)
+        best_idx = np.where(unsampled & cand_mask, 0, best_idx).astype(np.int32)
+    else:
+        m = oracle.match(Lo, w.x)
+        t_match = time.perf_counter() - t0
+        sample = "full step"
+        best_sim, best_idx = m["best_sim"], m["best_idx"]
+    t1 = time.perf_counter()
+    n_cand_g = U if w.self_match else U - R
+    stride = U - min(w.n_reuse, n_cand_g) if mode == 1 else U
+    s = oracle.select(Lo, best_sim, best_idx, mode, w.thr, w.n_reuse, stride)
+    Rw = oracle.rows_for(Lo, w.shape[-1], w.elem_bytes)
+    y = oracle.gather(Rw, w.x, s["kept_idx"])
+    cache = w.x            # any tensor of the right shape: restore is a bit copy
+    oracle.restore(Rw, y, cache, n_units, s["slot_of"], s["match_map"])
+    t_rest = time.perf_counter() - t1
+    total = t_match + t_rest
+    return (n_cand + n_units) / total, total, sample, oracle.num_threads()
+
+
+def _is_rep_token(w: inputs.Workload, i: int) -> bool:
+    if w.self_match:
+        return False
+    B, T, H, W, C = w.shape
+    x, y = i % W, (i // W) % H
+    gy, gx = w.groups
+    return ((y % (H // gy)) % 2 == 0) and ((x % (W // gx)) % 2 == 0)
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    w = make_workload(args.workload)
+    n_rows = args.ref_rows
+    for _ in range(args.warmup if args.warmup < 2 else 1):
+        oracle_sample_step(w, max(n_rows // 8, 8))
+    times, vals = [], []
+    sample = threads = None
+    wall0 = time.perf_counter()
+    for k in range(args.steps):
+        v, t, sample, threads = oracle_sample_step(w, n_rows, seed=k)
+        vals.append(v); times.append(t)
+    wall = time.perf_counter() - wall0
+    value = statistics.mean(vals)
+    G, U, R = unit_counts(w)
+    line = {
+        "impl": "reference", "metric": "matched+restored tokens/s per cache op", "value": value,
+        "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * statistics.mean(times), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "shape": list(w.shape), "groups": G, "units_per_group": U,
+                   "note": "CPU oracle, scaled from a bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "wall_s": wall,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------------------------------
+def run_ours(args, rank, local_rank, world):
+    import torch
+    from paper_2607_23844_b200 import build
+    if rank == 0:
+        build.build()
+    sharding.barrier()
+    from paper_2607_23844_b200 import omnicache as oc
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    w = make_workload(args.workload, seed_offset=rank)          # weak scaling: each rank its own batch
+    G, U, R = unit_counts(w)
+    n_units, n_cand_g = G * U, (U if w.self_match else U - R)
+    n_cand = G * n_cand_g
+    mode = oc.SELECT_COUNT if w.mode == "count" else oc.SELECT_THRESHOLD
+    stride = U - min(w.n_reuse, n_cand_g) if mode == oc.SELECT_COUNT else U
+    L = oc.Layout(KIND[w.kind], w.dtype, *w.shape, gy=w.groups[0], gx=w.groups[1], self_match=int(w.self_match))
+    rows = oc.rows_from_layout(L, w.shape[-1], w.elem_bytes)
+    row_bytes = rows.seg_bytes * rows.n_seg
+    tensor_bytes = int(np.prod(w.shape)) * w.elem_bytes
+
+    def host_tensor(a):
+        return torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a)
+
+    x_host = host_tensor(w.x).pin_memory()
+    cache_host = host_tensor(inputs.random_rows(7 + rank, w.shape, w.dtype)).pin_memory()
+
+    per_set = 5 * tensor_bytes + G * stride * row_bytes          # x, cache, out, dst, layered-cache entry, y
+    ring = max(2, -(-4 * L2_BYTES // per_set))
+    sets = []
+    for r in range(ring):
+        s = dict(
+            x=x_host.to(dev), cache=cache_host.to(dev),
+            out=torch.empty(tensor_bytes, dtype=torch.uint8, device=dev),
+            y=torch.empty(G * stride * row_bytes, dtype=torch.uint8, device=dev),
+            dst=torch.empty(tensor_bytes, dtype=torch.uint8, device=dev),
+            best_sim=torch.empty(n_units, dtype=torch.float32, device=dev),
+            best_idx=torch.empty(n_units, dtype=torch.int32, device=dev),
+            kept_idx=torch.empty(G * stride, dtype=torch.int32, device=dev),
+            kept_count=torch.empty(G, dtype=torch.int32, device=dev),
+            match_map=torch.empty(n_units, dtype=torch.int32, device=dev),
+            slot_of=torch.empty(n_units, dtype=torch.int32, device=dev))
+        sets.append(s)
+    ctx = oc.Context(local_rank, oc.match_workspace_bytes(L))
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        s = sets[i % ring]
+        ctx.match(L, s["x"], s["best_sim"], s["best_idx"], stream=stream)
+        ctx.select(L, s["best_sim"], s["best_idx"], mode, w.thr, w.n_reuse, stride, s["kept_idx"], s["kept_count"],
+                   s["match_map"], s["slot_of"], stream=stream)
+        ctx.gather(rows, s["x"], s["kept_idx"], G * stride, s["y"], stream=stream)
+        ctx.restore(rows, s["y"], s["cache"], n_units, s["slot_of"], s["match_map"], s["out"], stream=stream)
+        ctx.layer_cache_put(i % ring, i, s["out"], tensor_bytes, stream=stream)
+        ctx.layer_cache_get(i % ring, i, 5, s["dst"], stream=stream)
+
+    for i in range(max(args.warmup, ring)):            # also allocates every layered-cache entry
+        step(i)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == oc.OK
+    ctx.profile_reset()
+    ctx.profile_enable(True)
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sharding.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)) as clk:
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    sharding.barrier()
+    ms_total = sharding.max_over_ranks(e0.elapsed_time(e1), dev)
+    ctx.profile_enable(False)
+    prof = {oc.kernel_name(k): ctx.profile_read(k) for k in range(oc.K_COUNT)}
+    launches = sum(n for n, _ in prof.values())
+    assert ctx.device_status() == oc.OK
+
+    tokens_per_step = n_cand + n_units
+    value = world * tokens_per_step * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end through the host-buffer call ------------------------------------------------
+    out_host = torch.empty_like(x_host).pin_memory()
+    kc_host = torch.zeros(G, dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, args.e2e_steps))
+    for _ in range(2):
+        ctx.cache_step_host(L, mode, w.thr, w.n_reuse, x_host, cache_host, out_host, kc_host, stream=stream)
+    sharding.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        ctx.cache_step_host(L, mode, w.thr, w.n_reuse, x_host, cache_host, out_host, kc_host, stream=stream)
+    torch.cuda.synchronize()
+    e2e_s = sharding.max_over_ranks(time.perf_counter() - t0, dev)
+    e2e_value = world * tokens_per_step * e2e_steps / e2e_s
+
+    # ---- roofline of the dominant kernel and per-op table -----------------------------------------
+    peaks = measured_peaks()
+    ops = {}
+    for name, (n, ms) in prof.items():
+        if n:
+            ops[name] = {"launches": n, "avg_us": 1e3 * ms / n, "share": None}
+    tot_ms = sum(ms for _, ms in prof.values()) or 1.0
+    for name, (n, ms) in prof.items():
+        if n:
+            ops[name]["share"] = ms / tot_ms
+    n_keep = G * stride
+    alg_bytes = {"gather": 2 * n_keep * row_bytes, "restore": 2 * n_units * row_bytes, "copy": 2 * tensor_bytes,
+                 "norms": tensor_bytes, "frame_pair": tensor_bytes, "block_partial": tensor_bytes}
+    for name, b in alg_bytes.items():
+        if name in ops:
+            ops[name]["GB/s"] = b / (ops[name]["avg_us"] * 1e-6) / 1e9
+            ops[name]["frac_hbm"] = ops[name]["GB/s"] / peaks["hbm_gbs"]
+    if w.kind == "token" and not w.self_match and "match_tc" in ops:
+        flops = 2.0 * n_cand * R * w.shape[-1]
+        achieved = flops / (ops["match_tc"]["avg_us"] * 1e-6) / 1e12
+        peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        roofline = {"kernel": "match_tc", "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                    "peak_source": f"{peaks['_source']} bf16 sustained", "frac_of_burst": achieved / peaks["bf16_tflops"],
+                    "frac_of_nominal": achieved / NOMINAL["bf16_tflops"], "flops_per_launch": flops}
+    else:
+        dom = max((k for k in ops if k in alg_bytes), key=lambda k: ops[k]["share"])
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": ops[dom]["GB/s"], "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": ops[dom]["frac_hbm"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                    "peak_source": f"{peaks['_source']} copy bandwidth", "bytes_per_launch": alg_bytes[dom]}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, t, sample, threads = oracle_sample_step(w, args.ref_rows)
+        cpu_baseline = {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample,
+                        "seconds": t}
+
+    if rank == 0:
+        line = {
+            "metric": "matched+restored tokens/s per cache op", "value": value, "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if w.dtype == inputs.BF16 else "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "shape": list(w.shape), "kind": w.kind, "mode": w.mode,
+                       "n_reuse_per_group": w.n_reuse, "thr": w.thr, "groups": G, "units_per_group": U,
+                       "reps_per_group": R, "tokens_per_step": tokens_per_step,
+                       "l2": f"inputs rotate through a ring of {ring} buffer sets ({ring * per_set >> 20} MiB > 4x L2)",
+                       "wrapped_layer": "identity stand-in (outside the path)", "parallelism": f"replicas x{world}"},
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": 2 * tensor_bytes,
+                    "d2h_bytes_per_step": tensor_bytes + 4 * G, "steps": e2e_steps,
+                    "ms_per_step": 1e3 * e2e_s / e2e_steps},
+            "gpu_launches": launches, "clocks": clk.summary(), "ops": ops,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="sd3_token")
+    ap.add_argument("--ref-rows", type=int, default=8192,
+                    help="candidates the CPU oracle matches per step (all of them if the workload has fewer)")
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 1000 if args.impl == "ours" else 3
+    if args.warmup is None:
+        args.warmup = 50 if args.impl == "ours" else 1
+    if args.impl == "ours":
+        args.warmup = max(args.warmup, 3)
+    rank, local_rank, world = sharding.env_rank_world()
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    rank, local_rank, world = sharding.init()
+    try:
+        run_ours(args, rank, local_rank, world)
+    finally:
+        sharding.finalize()
+
+
+if __name__ == "__main__":
+    main()
