@@ -147,6 +147,7 @@ __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u 
 // Order-preserving map float -> uint32 (larger float <=> larger key) and back.
 __device__ __forceinline__ uint32_t f32_to_ordered(float f) {
     uint32_t b = __float_as_uint(f);
+    if (b == 0x80000000u) b = 0u;                           // -0.0 and +0.0 compare equal: one key
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 __device__ __forceinline__ float ordered_to_f32(uint32_t k) {

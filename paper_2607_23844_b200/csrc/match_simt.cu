@@ -19,12 +19,15 @@ norms_kernel(const uint8_t* __restrict__ x, long long n_tok, int cpr, float eps,
     if (row >= n_tok) return;
     const uint8_t* r = x + row * (long long)cpr * 16;
     float s0 = 0.f, s1 = 0.f;
-    int c = lane;
-    for (; c + 32 < cpr; c += 64) {
-        uint4 a = ld_nc_v4(r + (long long)c * 16), b = ld_nc_v4(r + (long long)(c + 32) * 16);
-        Chunk<DT>::sq(a, s0); Chunk<DT>::sq(b, s1);
+    for (int c = lane; c < cpr; c += 128) {                 // up to four 16-byte loads in flight per lane
+        uint4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (c + 32 * k < cpr) v[k] = ld_nc_v4(r + (long long)(c + 32 * k) * 16);
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (c + 32 * k < cpr) Chunk<DT>::sq(v[k], (k & 1) ? s1 : s0);
     }
-    if (c < cpr) { uint4 a = ld_nc_v4(r + (long long)c * 16); Chunk<DT>::sq(a, s0); }
     float s = s0 + s1;
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, d);

@@ -2,142 +2,195 @@
 //
 // One CTA per group (a group is an independent selection problem).  Everything is decided in
 // ascending unit order, so the result is deterministic and comparable bit for bit:
-//   COUNT mode  - 4 x 8-bit radix select over order-preserving keys of the candidates' best_sim
-//                 finds the value at the cut; candidates above it are reused, candidates equal to it
-//                 are admitted lowest index first;
-//   both modes  - reuse flags live in a shared-memory bitmask; kept units are compacted with a
-//                 warp-ballot prefix sum (stable, ascending original index).
+//   COUNT mode  - the candidates' best_sim are staged once in shared memory as order-preserving
+//                 keys; a 4 x 8-bit radix select (warp-aggregated histogram updates, warp-parallel
+//                 bin search) finds the value at the cut; candidates above it are reused, candidates
+//                 equal to it are admitted lowest index first;
+//   both modes  - kept units are compacted with block-wide prefix sums (stable, ascending original
+//                 index).
+// Two kernels: select_fast_kernel (groups up to 40960 units, the usual case) reads every input once
+// up front, gives each thread a contiguous run of units so that only two block-wide scans are needed,
+// and writes all outputs in one coalesced pass at the end; select_general_kernel covers self-match
+// and larger groups with a round-by-round loop.
 #include "common.cuh"
 
 namespace oc {
 
 static constexpr int SEL_THREADS = 1024;
 static constexpr int SEL_MAX_UNITS = 65536;
+static constexpr int SEL_SMEM_KEYS = 40960;          // keys cached in shared memory up to this many units
 
-struct BlockScan {
-    // exclusive prefix of a per-thread 0/1 flag over the CTA (thread order), plus the CTA total.
-    __device__ static int run(bool flag, int* warp_sums /*[33]*/, int& total) {
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-        unsigned b = __ballot_sync(0xFFFFFFFFu, flag);
-        int within = __popc(b & ((1u << lane) - 1u));
-        if (lane == 0) warp_sums[warp] = __popc(b);
-        __syncthreads();
-        if (warp == 0) {
-            int v = warp_sums[lane];
-            int incl = v;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                int n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                if (lane >= d) incl += n;
-            }
-            warp_sums[lane] = incl - v;
-            if (lane == 31) warp_sums[32] = incl;
+// Per-CTA view of one group: unit index arithmetic without 64-bit divisions in the loops.
+struct GroupView {
+    long long base;     // global index of local unit 0 (TOKEN: of the patch's first token)
+    int row_pitch;      // TOKEN: frame width W; others unused
+    __device__ GroupView(const GroupMap& m, long long g) {
+        if (m.kind == OC_KIND_TOKEN) {
+            const int px = (int)(g % m.gx), py = (int)((g / m.gx) % m.gy);
+            const long long bt = g / ((long long)m.gx * m.gy);
+            base = (bt * m.H + (long long)py * m.Hp) * m.W + (long long)px * m.Wp;
+            row_pitch = m.W;
+        } else {
+            base = g * m.units_per_group;
+            row_pitch = 0;
         }
-        __syncthreads();
-        int res = warp_sums[warp] + within;
-        total = warp_sums[32];
-        __syncthreads();          // warp_sums is reused by the next call
-        return res;
+    }
+    __device__ __forceinline__ long long index(const GroupMap& m, int u) const {
+        if (m.kind != OC_KIND_TOKEN) return base + u;
+        const int ly = u / m.Wp, lx = u - ly * m.Wp;
+        return base + (long long)ly * row_pitch + lx;
     }
 };
 
+// exclusive prefix of a per-thread 0/1 flag over the CTA (thread order) and the CTA total; `sums`
+// is one of two alternating 33-int buffers, so consecutive calls need no trailing barrier.
+__device__ __forceinline__ int block_scan(bool flag, int* sums, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned b = __ballot_sync(0xFFFFFFFFu, flag);
+    const int within = __popc(b & ((1u << lane) - 1u));
+    if (lane == 0) sums[warp] = __popc(b);
+    __syncthreads();
+    if (warp == 0) {
+        const int v = sums[lane];
+        int incl = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= d) incl += n;
+        }
+        sums[lane] = incl - v;
+        if (lane == 31) sums[32] = incl;
+    }
+    __syncthreads();
+    total = sums[32];
+    return sums[warp] + within;
+}
+
 __global__ void __launch_bounds__(SEL_THREADS)
-select_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_t* __restrict__ best_idx,
-              int mode, float thr, int n_reuse, int y_stride, int32_t* __restrict__ kept_idx,
-              int32_t* __restrict__ kept_count, int32_t* __restrict__ match_map,
-              int32_t* __restrict__ slot_of) {
+select_general_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_t* __restrict__ best_idx,
+              int mode, float thr, int n_reuse, int y_stride, int keys_in_smem,
+              int32_t* __restrict__ kept_idx, int32_t* __restrict__ kept_count,
+              int32_t* __restrict__ match_map, int32_t* __restrict__ slot_of) {
+    extern __shared__ unsigned key_cache[];                    // [U] when keys_in_smem
     __shared__ unsigned reuse_bits[SEL_MAX_UNITS / 32];
-    __shared__ int warp_sums[33];
+    __shared__ int scan_sums[2][33];
     __shared__ unsigned hist[256];
     __shared__ unsigned sh_prefix, sh_remaining;
+    __shared__ int sh_ncand;
 
     const int U = gm.units_per_group;
     const long long g = blockIdx.x;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_rounds = (U + SEL_THREADS - 1) / SEL_THREADS;
+    const GroupView gv(gm, g);
+    int scan_flip = 0;
 
     // ---- COUNT mode: value at the cut ----------------------------------------------------------
-    unsigned cut_key = 0;       // candidates with key > cut_key are reused
-    int need_eq = 0;            // ... plus the first need_eq candidates with key == cut_key
+    unsigned cut_key = 0xFFFFFFFFu;  // candidates with key > cut_key are reused
+    int need_eq = 0;                 // ... plus the first need_eq candidates with key == cut_key
     bool all_reused = false;
     if (mode == OC_SELECT_COUNT) {
-        // number of candidates in the group
+        // stage keys (0 marks a non-candidate: every real key is > 0) and count the candidates
+        if (tid == 0) sh_ncand = 0;
+        __syncthreads();
         int local = 0;
-        for (int u = tid; u < U; u += SEL_THREADS) local += gm_is_cand(gm, u) ? 1 : 0;
-        // CTA sum through the scan helper (flag-wise), done on counts via shared atomics instead
-        if (tid == 0) sh_remaining = 0;
+        for (int u = tid; u < U; u += SEL_THREADS) {
+            unsigned key = 0;
+            if (gm_is_cand(gm, u)) { key = f32_to_ordered(best_sim[gv.index(gm, u)]); key = key ? key : 1u; ++local; }
+            if (keys_in_smem) key_cache[u] = key;
+        }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, d);
+        if (lane == 0 && local) atomicAdd(&sh_ncand, local);
         __syncthreads();
-        if (local) atomicAdd(&sh_remaining, (unsigned)local);
-        __syncthreads();
-        const int n_cand = (int)sh_remaining;
-        __syncthreads();
+        const int n_cand = sh_ncand;
         const int k = n_reuse < n_cand ? n_reuse : n_cand;
         if (k >= n_cand) {
             all_reused = true;
         } else if (k > 0) {
             if (tid == 0) { sh_prefix = 0; sh_remaining = (unsigned)k; }
-            __syncthreads();
             for (int pass = 0; pass < 4; ++pass) {
                 const int shift = 24 - 8 * pass;
                 if (tid < 256) hist[tid] = 0;
                 __syncthreads();
                 const unsigned prefix = sh_prefix;
                 const unsigned himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-                for (int u = tid; u < U; u += SEL_THREADS) {
-                    if (!gm_is_cand(gm, u)) continue;
-                    unsigned key = f32_to_ordered(best_sim[gm_unit_index(gm, g, u)]);
-                    if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+                for (int r = 0; r < n_rounds; ++r) {
+                    const int u = r * SEL_THREADS + tid;
+                    unsigned key = 0;
+                    if (u < U) {
+                        if (keys_in_smem) key = key_cache[u];
+                        else if (gm_is_cand(gm, u)) { key = f32_to_ordered(best_sim[gv.index(gm, u)]); key = key ? key : 1u; }
+                    }
+                    const bool take = key != 0 && (key & himask) == prefix;
+                    // warp-aggregated update: one shared-memory atomic per distinct digit in the warp
+                    const unsigned digit = take ? ((key >> shift) & 255u) : 256u;
+                    const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
+                    if (take && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
                 }
                 __syncthreads();
-                if (tid == 0) {
-                    unsigned rem = sh_remaining;   // how many still to take among keys matching prefix
-                    int d = 255;
-                    for (; d > 0; --d) {
-                        if (hist[d] >= rem) break;
-                        rem -= hist[d];
+                if (warp == 0) {
+                    // lane l owns bins 255-8l .. 248-8l (descending); find where the running count reaches rem
+                    const unsigned rem = sh_remaining;
+                    unsigned c[8], tot = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { c[i] = hist[255 - 8 * lane - i]; tot += c[i]; }
+                    unsigned incl = tot;
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        const unsigned n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                        if (lane >= d) incl += n;
                     }
-                    sh_prefix = prefix | ((unsigned)d << shift);
-                    sh_remaining = rem;            // taken from bin d (1 <= rem <= hist[d])
+                    const unsigned before = incl - tot;           // count in higher bins owned by lower lanes
+                    const bool here = before < rem && rem <= incl;
+                    if (here) {
+                        unsigned acc = before;
+                        int bin = 255 - 8 * lane;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (acc + c[i] >= rem) { bin = 255 - 8 * lane - i; break; }
+                            acc += c[i];
+                        }
+                        sh_prefix = prefix | ((unsigned)bin << shift);
+                        sh_remaining = rem - acc;                 // still to take inside that bin (>= 1)
+                    }
                 }
                 __syncthreads();
             }
             cut_key = sh_prefix;
             need_eq = (int)sh_remaining;
         }
-        // k == 0: nothing reused (cut_key = 0xFFFFFFFF semantics handled below)
-        if (k == 0) { cut_key = 0xFFFFFFFFu; need_eq = 0; }
     }
 
     // ---- reuse flags, ascending unit order -----------------------------------------------------
     int eq_seen = 0;
     for (int r = 0; r < n_rounds; ++r) {
         const int u = r * SEL_THREADS + tid;
-        bool cand = false, reuse = false, eq = false;
-        if (u < U) {
-            cand = gm_is_cand(gm, u);
-            if (cand) {
-                const long long i = gm_unit_index(gm, g, u);
-                const float s = best_sim[i];
-                if (mode == OC_SELECT_THRESHOLD) {
-                    reuse = s >= thr;
-                    if (gm.self_match) reuse = reuse && (best_idx[i] < (int)i);
-                } else if (all_reused) {
-                    reuse = true;
-                } else {
-                    unsigned key = f32_to_ordered(s);
-                    reuse = key > cut_key;
-                    eq = key == cut_key;
-                }
+        bool reuse = false, eq = false;
+        if (u < U && gm_is_cand(gm, u)) {
+            if (mode == OC_SELECT_THRESHOLD) {
+                const long long i = gv.index(gm, u);
+                reuse = best_sim[i] >= thr;
+                if (gm.self_match) reuse = reuse && (best_idx[i] < (int)i);
+            } else if (all_reused) {
+                reuse = true;
+            } else {
+                unsigned key;
+                if (keys_in_smem) key = key_cache[u];
+                else { key = f32_to_ordered(best_sim[gv.index(gm, u)]); key = key ? key : 1u; }
+                reuse = key > cut_key;
+                eq = key == cut_key;
             }
         }
-        if (mode == OC_SELECT_COUNT && !all_reused && need_eq > 0) {
+        if (need_eq > 0) {                                         // uniform over the CTA
             int tot;
-            int rank = BlockScan::run(eq, warp_sums, tot);
+            const int rank = block_scan(eq, scan_sums[scan_flip], tot);
+            scan_flip ^= 1;
             if (eq && eq_seen + rank < need_eq) reuse = true;
             eq_seen += tot;
         }
-        unsigned bits = __ballot_sync(0xFFFFFFFFu, reuse);
-        if ((tid & 31) == 0 && (u < U)) reuse_bits[u >> 5] = bits;
+        const unsigned bits = __ballot_sync(0xFFFFFFFFu, reuse);
+        if (lane == 0 && u < U) reuse_bits[u >> 5] = bits;
     }
     __syncthreads();
 
@@ -149,9 +202,10 @@ select_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_t* __
         const bool reuse = valid && ((reuse_bits[u >> 5] >> (u & 31)) & 1u);
         const bool kept = valid && !reuse;
         int tot;
-        int rank = BlockScan::run(kept, warp_sums, tot);
+        const int rank = block_scan(kept, scan_sums[scan_flip], tot);
+        scan_flip ^= 1;
         if (valid) {
-            const long long i = gm_unit_index(gm, g, u);
+            const long long i = gv.index(gm, u);
             if (kept) {
                 const int pos = kept_base + rank;
                 if (pos < y_stride) kept_idx[g * y_stride + pos] = (int32_t)i;
@@ -178,6 +232,174 @@ select_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_t* __
     if (tid == 0) kept_count[g] = kept_base;
 }
 
+// inclusive-to-exclusive block scan of one int per thread; returns this thread's exclusive prefix
+__device__ __forceinline__ int block_scan_int(int v, int* sums /*[33]*/, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += n;
+    }
+    if (lane == 31) sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const int w = sums[lane];
+        int wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int n = __shfl_up_sync(0xFFFFFFFFu, wi, d);
+            if (lane >= d) wi += n;
+        }
+        sums[lane] = wi - w;
+        if (lane == 31) sums[32] = wi;
+    }
+    __syncthreads();
+    total = sums[32];
+    return sums[warp] + incl - v;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS)
+select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_t* __restrict__ best_idx,
+                   int mode, float thr, int n_reuse, int y_stride,
+                   int32_t* __restrict__ kept_idx, int32_t* __restrict__ kept_count,
+                   int32_t* __restrict__ match_map, int32_t* __restrict__ slot_of) {
+    extern __shared__ unsigned key_cache[];                    // [U] keys, later reused as kept positions
+    __shared__ int scan_sums[2][33];
+    __shared__ unsigned hist[256];
+    __shared__ unsigned sh_prefix, sh_remaining;
+    __shared__ int sh_ncand;
+
+    const int U = gm.units_per_group;
+    const long long g = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_rounds = (U + SEL_THREADS - 1) / SEL_THREADS;
+    const GroupView gv(gm, g);
+
+    // ---- phase 0: every similarity is read once, coalesced, all loads independent ----------------
+    // key 0 marks a non-candidate (every real key is >= 1)
+    if (tid == 0) sh_ncand = 0;
+    __syncthreads();
+    int local = 0;
+    for (int u = tid; u < U; u += SEL_THREADS) {
+        unsigned key = 0;
+        if (gm_is_cand(gm, u)) { key = f32_to_ordered(best_sim[gv.index(gm, u)]); key = key ? key : 1u; ++local; }
+        key_cache[u] = key;
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, d);
+    if (lane == 0 && local) atomicAdd(&sh_ncand, local);
+    __syncthreads();
+
+    // ---- the cut: candidates with key > cut_key are reused, plus the first need_eq with key == cut_key
+    unsigned cut_key = 0xFFFFFFFFu;
+    int need_eq = 0;
+    bool all_reused = false;
+    if (mode == OC_SELECT_THRESHOLD) {
+        // sim >= thr  <=>  key >= ordered(thr)  (-0.0 and +0.0 share one key); as "key > cut": cut = ordered(thr) - 1
+        unsigned tk = f32_to_ordered(thr); tk = tk ? tk : 1u;
+        cut_key = tk - 1u;
+    } else {
+        const int n_cand = sh_ncand;
+        const int k = n_reuse < n_cand ? n_reuse : n_cand;
+        if (k >= n_cand) {
+            all_reused = true;
+        } else if (k > 0) {
+            if (tid == 0) { sh_prefix = 0; sh_remaining = (unsigned)k; }
+            for (int pass = 0; pass < 4; ++pass) {
+                const int shift = 24 - 8 * pass;
+                if (tid < 256) hist[tid] = 0;
+                __syncthreads();
+                const unsigned prefix = sh_prefix;
+                const unsigned himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+                for (int r = 0; r < n_rounds; ++r) {
+                    const int u = r * SEL_THREADS + tid;
+                    const unsigned key = u < U ? key_cache[u] : 0u;
+                    const bool take = key != 0 && (key & himask) == prefix;
+                    // warp-aggregated update: one shared-memory atomic per distinct digit in the warp
+                    const unsigned digit = take ? ((key >> shift) & 255u) : 256u;
+                    const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
+                    if (take && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+                }
+                __syncthreads();
+                if (warp == 0) {
+                    // lane l owns bins 255-8l .. 248-8l (descending); find where the running count reaches rem
+                    const unsigned rem = sh_remaining;
+                    unsigned c[8], tot = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { c[i] = hist[255 - 8 * lane - i]; tot += c[i]; }
+                    unsigned incl = tot;
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        const unsigned n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                        if (lane >= d) incl += n;
+                    }
+                    const unsigned before = incl - tot;
+                    if (before < rem && rem <= incl) {
+                        unsigned acc = before;
+                        int bin = 255 - 8 * lane;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (acc + c[i] >= rem) { bin = 255 - 8 * lane - i; break; }
+                            acc += c[i];
+                        }
+                        sh_prefix = prefix | ((unsigned)bin << shift);
+                        sh_remaining = rem - acc;
+                    }
+                }
+                __syncthreads();
+            }
+            cut_key = sh_prefix;
+            need_eq = (int)sh_remaining;
+        }
+    }
+
+    // ---- phase 2: each thread owns a contiguous run of units -------------------------------------
+    const int run = n_rounds;                                   // units per thread
+    const int u0 = tid * run, u1 = min(U, u0 + run);
+    int eq_base = 0;
+    if (need_eq > 0) {
+        int n_eq = 0;
+        for (int u = u0; u < u1; ++u) n_eq += key_cache[u] == cut_key ? 1 : 0;
+        int tot;
+        eq_base = block_scan_int(n_eq, scan_sums[0], tot);
+    }
+    unsigned long long reuse_mask = 0;                          // run <= 40 units
+    int n_kept = 0;
+    for (int u = u0; u < u1; ++u) {
+        const unsigned key = key_cache[u];
+        bool reuse = false;
+        if (key != 0) {
+            if (all_reused) reuse = true;
+            else if (key > cut_key) reuse = true;
+            else if (need_eq > 0 && key == cut_key) { reuse = eq_base < need_eq; ++eq_base; }
+        }
+        if (reuse) reuse_mask |= 1ull << (u - u0); else ++n_kept;
+    }
+    int kept_total;
+    int pos = block_scan_int(n_kept, scan_sums[1], kept_total);
+    __syncthreads();                                            // all reads of the keys are done
+    for (int u = u0; u < u1; ++u)
+        key_cache[u] = ((reuse_mask >> (u - u0)) & 1ull) ? 0xFFFFFFFFu : (unsigned)pos++;
+    __syncthreads();
+
+    // ---- phase 3: one coalesced pass writes every output ------------------------------------------
+    for (int u = tid; u < U; u += SEL_THREADS) {
+        const long long i = gv.index(gm, u);
+        const unsigned p = key_cache[u];
+        if (p != 0xFFFFFFFFu) {
+            if ((int)p < y_stride) kept_idx[g * y_stride + p] = (int32_t)i;
+            slot_of[i] = (int32_t)(g * y_stride + p);
+            match_map[i] = (int32_t)i;
+        } else {
+            slot_of[i] = -1;
+            match_map[i] = best_idx[i];
+        }
+    }
+    for (int p = kept_total + tid; p < y_stride; p += SEL_THREADS) kept_idx[g * y_stride + p] = -1;
+    if (tid == 0) kept_count[g] = kept_total;
+}
+
 oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, const int32_t* best_idx,
                         int mode, float thr, int64_t n_reuse, int64_t y_stride, int32_t* kept_idx,
                         int32_t* kept_count, int32_t* match_map, int32_t* slot_of, cudaStream_t s) {
@@ -185,10 +407,26 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
     if (geo.n_groups == 0) return OC_OK;
     GroupMap gm = make_group_map(geo);
     int nr = (int)(n_reuse > 0x7FFFFFFF ? 0x7FFFFFFF : n_reuse);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(select_general_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess ||
+            cudaFuncSetAttribute(select_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess)
+            return OC_ERR_CUDA;
+        attr_set = true;
+    }
     LaunchScope scope(ctx, OC_K_SELECT, s);
-    select_kernel<<<(unsigned)geo.n_groups, SEL_THREADS, 0, s>>>(gm, best_sim, best_idx, mode, thr, nr,
-                                                                  (int)y_stride, kept_idx, kept_count,
-                                                                  match_map, slot_of);
+    if (!geo.self_match && geo.units_per_group <= SEL_SMEM_KEYS) {
+        select_fast_kernel<<<(unsigned)geo.n_groups, SEL_THREADS, (size_t)geo.units_per_group * sizeof(unsigned), s>>>(
+            gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);
+    } else {
+        const int keys_in_smem = (mode == OC_SELECT_COUNT && geo.units_per_group <= SEL_SMEM_KEYS) ? 1 : 0;
+        const size_t dyn = keys_in_smem ? (size_t)geo.units_per_group * sizeof(unsigned) : 0;
+        select_general_kernel<<<(unsigned)geo.n_groups, SEL_THREADS, dyn, s>>>(gm, best_sim, best_idx, mode, thr, nr,
+                                                                                (int)y_stride, keys_in_smem, kept_idx,
+                                                                                kept_count, match_map, slot_of);
+    }
     return last_launch_status();
 }
 
