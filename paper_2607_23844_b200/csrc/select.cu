@@ -20,25 +20,45 @@ static constexpr int SEL_THREADS = 1024;
 static constexpr int SEL_MAX_UNITS = 65536;
 static constexpr int SEL_SMEM_KEYS = 40960;          // keys cached in shared memory up to this many units
 
-// Per-CTA view of one group: unit index arithmetic without 64-bit divisions in the loops.
+// Per-CTA view of one group: unit index and candidate test with as few instructions as possible
+// (one CTA serves a whole group, so the kernel is bound by instruction issue on a single SM):
+// shifts and masks when the row width / lattice strides are powers of two, divisions otherwise.
 struct GroupView {
     long long base;     // global index of local unit 0 (TOKEN: of the patch's first token)
     int row_pitch;      // TOKEN: frame width W; others unused
+    int w_local;        // row width of the local unit grid (TOKEN: Wp, BLOCK: W, FRAME: 0)
+    int w_shift;        // log2(w_local) if it is a power of two, else -1
+    int lat_pow2;       // sy and sx are both powers of two
     __device__ GroupView(const GroupMap& m, long long g) {
         if (m.kind == OC_KIND_TOKEN) {
             const int px = (int)(g % m.gx), py = (int)((g / m.gx) % m.gy);
             const long long bt = g / ((long long)m.gx * m.gy);
             base = (bt * m.H + (long long)py * m.Hp) * m.W + (long long)px * m.Wp;
             row_pitch = m.W;
+            w_local = m.Wp;
         } else {
             base = g * m.units_per_group;
             row_pitch = 0;
+            w_local = m.kind == OC_KIND_BLOCK ? m.W : 0;
         }
+        w_shift = (w_local > 0 && (w_local & (w_local - 1)) == 0) ? 31 - __clz(w_local) : -1;
+        lat_pow2 = (m.sy & (m.sy - 1)) == 0 && (m.sx & (m.sx - 1)) == 0;
+    }
+    __device__ __forceinline__ void split(int u, int& ly, int& lx) const {
+        if (w_shift >= 0) { ly = u >> w_shift; lx = u & (w_local - 1); }
+        else { ly = u / w_local; lx = u - ly * w_local; }
     }
     __device__ __forceinline__ long long index(const GroupMap& m, int u) const {
         if (m.kind != OC_KIND_TOKEN) return base + u;
-        const int ly = u / m.Wp, lx = u - ly * m.Wp;
+        int ly, lx; split(u, ly, lx);
         return base + (long long)ly * row_pitch + lx;
+    }
+    __device__ __forceinline__ bool is_cand(const GroupMap& m, int u) const {
+        if (m.kind == OC_KIND_FRAME) return (u & 1) != 0;
+        if (m.self_match) return true;
+        int ly, lx; split(u, ly, lx);
+        if (lat_pow2) return !(((ly & (m.sy - 1)) == m.oy) && ((lx & (m.sx - 1)) == m.ox));
+        return !((ly % m.sy) == m.oy && (lx % m.sx) == m.ox);
     }
 };
 
@@ -269,6 +289,7 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     __shared__ unsigned hist[256];
     __shared__ unsigned sh_prefix, sh_remaining;
     __shared__ int sh_ncand;
+    __shared__ unsigned sh_kmin, sh_kmax;
 
     const int U = gm.units_per_group;
     const long long g = blockIdx.x;
@@ -276,19 +297,47 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     const int n_rounds = (U + SEL_THREADS - 1) / SEL_THREADS;
     const GroupView gv(gm, g);
 
-    // ---- phase 0: every similarity is read once, coalesced, all loads independent ----------------
+    // ---- phase 0: every input is read once, coalesced, all loads issued before any is used --------
     // key 0 marks a non-candidate (every real key is >= 1)
-    if (tid == 0) sh_ncand = 0;
+    constexpr int PF = 8;                                       // rounds whose loads are kept in registers
+    if (tid == 0) { sh_ncand = 0; sh_kmin = 0xFFFFFFFFu; sh_kmax = 0u; }
     __syncthreads();
     int local = 0;
-    for (int u = tid; u < U; u += SEL_THREADS) {
-        unsigned key = 0;
-        if (gm_is_cand(gm, u)) { key = f32_to_ordered(best_sim[gv.index(gm, u)]); key = key ? key : 1u; ++local; }
-        key_cache[u] = key;
+    unsigned kmin = 0xFFFFFFFFu, kmax = 0u;
+    int idx_pf[PF];                                             // best_idx of this thread's units (phase 3)
+    for (int r0 = 0; r0 < n_rounds; r0 += PF) {
+        float sim_pf[PF];
+        long long gi[PF];
+#pragma unroll
+        for (int k = 0; k < PF; ++k) {
+            const int u = (r0 + k) * SEL_THREADS + tid;
+            gi[k] = u < U ? gv.index(gm, u) : -1;
+        }
+#pragma unroll
+        for (int k = 0; k < PF; ++k) {
+            sim_pf[k] = gi[k] >= 0 ? best_sim[gi[k]] : 0.f;
+            if (r0 == 0) idx_pf[k] = gi[k] >= 0 ? best_idx[gi[k]] : 0;
+        }
+#pragma unroll
+        for (int k = 0; k < PF; ++k) {
+            const int u = (r0 + k) * SEL_THREADS + tid;
+            if (u < U) {
+                unsigned key = 0;
+                if (gv.is_cand(gm, u)) {
+                    key = f32_to_ordered(sim_pf[k]); key = key ? key : 1u; ++local;
+                    kmin = min(kmin, key); kmax = max(kmax, key);
+                }
+                key_cache[u] = key;
+            }
+        }
     }
 #pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, d);
-    if (lane == 0 && local) atomicAdd(&sh_ncand, local);
+    for (int d = 16; d >= 1; d >>= 1) {
+        local += __shfl_xor_sync(0xFFFFFFFFu, local, d);
+        kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, d));
+        kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, d));
+    }
+    if (lane == 0 && local) { atomicAdd(&sh_ncand, local); atomicMin(&sh_kmin, kmin); atomicMax(&sh_kmax, kmax); }
     __syncthreads();
 
     // ---- the cut: candidates with key > cut_key are reused, plus the first need_eq with key == cut_key
@@ -306,8 +355,15 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
             all_reused = true;
         } else if (k > 0) {
             if (tid == 0) { sh_prefix = 0; sh_remaining = (unsigned)k; }
+            const unsigned span = sh_kmin ^ sh_kmax;            // bits in which candidates differ at all
             for (int pass = 0; pass < 4; ++pass) {
                 const int shift = 24 - 8 * pass;
+                if ((span >> shift) == 0) {                         // every candidate shares this digit: no histogram needed
+                    __syncthreads();
+                    if (tid == 0) sh_prefix |= ((sh_kmax >> shift) & 255u) << shift;
+                    __syncthreads();
+                    continue;
+                }
                 if (tid < 256) hist[tid] = 0;
                 __syncthreads();
                 const unsigned prefix = sh_prefix;
@@ -316,10 +372,18 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
                     const int u = r * SEL_THREADS + tid;
                     const unsigned key = u < U ? key_cache[u] : 0u;
                     const bool take = key != 0 && (key & himask) == prefix;
-                    // warp-aggregated update: one shared-memory atomic per distinct digit in the warp
-                    const unsigned digit = take ? ((key >> shift) & 255u) : 256u;
-                    const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
-                    if (take && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+                    const unsigned digit = (key >> shift) & 255u;
+                    // high digits are usually shared by the whole warp: one atomic for all of them;
+                    // otherwise plain shared-memory atomics (distinct bins rarely collide)
+                    const unsigned takers = __ballot_sync(0xFFFFFFFFu, take);
+                    if (takers) {
+                        const unsigned dref = __shfl_sync(0xFFFFFFFFu, digit, __ffs(takers) - 1);
+                        if (__all_sync(0xFFFFFFFFu, !take || digit == dref)) {
+                            if (lane == 0) atomicAdd(&hist[dref], (unsigned)__popc(takers));
+                        } else if (take) {
+                            atomicAdd(&hist[digit], 1u);
+                        }
+                    }
                 }
                 __syncthreads();
                 if (warp == 0) {
@@ -384,7 +448,9 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     __syncthreads();
 
     // ---- phase 3: one coalesced pass writes every output ------------------------------------------
-    for (int u = tid; u < U; u += SEL_THREADS) {
+    for (int r = 0; r < n_rounds; ++r) {
+        const int u = r * SEL_THREADS + tid;
+        if (u >= U) break;
         const long long i = gv.index(gm, u);
         const unsigned p = key_cache[u];
         if (p != 0xFFFFFFFFu) {
@@ -393,7 +459,13 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
             match_map[i] = (int32_t)i;
         } else {
             slot_of[i] = -1;
-            match_map[i] = best_idx[i];
+            int m;
+            switch (r) {                                            // registers of the first PF rounds, else reload
+                case 0: m = idx_pf[0]; break; case 1: m = idx_pf[1]; break; case 2: m = idx_pf[2]; break;
+                case 3: m = idx_pf[3]; break; case 4: m = idx_pf[4]; break; case 5: m = idx_pf[5]; break;
+                case 6: m = idx_pf[6]; break; case 7: m = idx_pf[7]; break; default: m = best_idx[i]; break;
+            }
+            match_map[i] = m;
         }
     }
     for (int p = kept_total + tid; p < y_stride; p += SEL_THREADS) kept_idx[g * y_stride + p] = -1;

@@ -94,6 +94,9 @@ def _chk(st: int, where: str) -> None:
         raise OmniCacheError(st, where)
 
 
+_LAYOUT_CACHE: dict = {}
+
+
 @dataclass
 class Layout:
     kind: int
@@ -114,8 +117,12 @@ class Layout:
     eps: float = 1e-8
 
     def c(self) -> CLayout:
-        return CLayout(self.kind, self.dtype, self.B, self.T, self.H, self.W, self.C, self.sy, self.sx,
-                       self.oy, self.ox, self.gy, self.gx, self.self_match, self.frame_stat, self.eps)
+        key = (self.kind, self.dtype, self.B, self.T, self.H, self.W, self.C, self.sy, self.sx,
+               self.oy, self.ox, self.gy, self.gx, self.self_match, self.frame_stat, self.eps)
+        hit = _LAYOUT_CACHE.get(key)
+        if hit is None:
+            hit = _LAYOUT_CACHE[key] = CLayout(*key)
+        return hit
 
     def check(self) -> int:
         return layout_check(self)
