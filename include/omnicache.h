@@ -231,6 +231,31 @@ oc_status oc_layer_cache_get(oc_ctx* ctx, int layer, int step, int interval, voi
                              const void** view, size_t* bytes, void* stream);
 oc_status oc_layer_cache_clear(oc_ctx* ctx);
 
+/* Frame Cache match for callers that must not allocate.  The paper has no counterpart for this
+ * call; it exists for hosts where the calling code is not allowed to obtain device memory at all:
+ * an inference server that hands its whole memory budget to one pool at start-up and treats any
+ * later driver allocation as a fault, a plug-in running inside another framework's allocator, or
+ * code that may already be inside a region where cudaMalloc is illegal or would stall every stream.
+ * oc_match() needs a context, and a context owns cudaMalloc'd scratch; this variant needs neither.
+ *
+ * It computes exactly what oc_match() computes for an OC_KIND_FRAME layout (best_sim, best_idx and,
+ * if pair_sim is not null, the [B][T-1] adjacent-pair statistic), with the same kernels, but keeps
+ * its partial sums in a fixed array of OC_NOALLOC_SCRATCH_BYTES bytes that is part of the library
+ * image: every GPU that loads the library holds that array until the process exits.
+ *   - A layout whose scratch need (oc_match_workspace_bytes) exceeds OC_NOALLOC_SCRATCH_BYTES is
+ *     refused with OC_ERR_WORKSPACE and nothing is launched.  Other kinds: OC_ERR_INVALID_ARG.
+ *   - The call itself makes no cudaMalloc / cudaFree and uses no allocating library routine; the
+ *     caller passes every input and output buffer.
+ *   - The first call on each device looks up the array's device address (with that device current)
+ *     and remembers it; make that first call before any stream capture begins.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left.  No
+ *     part of it needs to start at zero (each call writes every value it later reads), but two calls
+ *     whose kernels overlap on the GPU - different streams, or one stream replayed concurrently -
+ *     race on it.  Serialise them. */
+#define OC_NOALLOC_SCRATCH_BYTES (1u << 20)
+oc_status oc_match_frame_noalloc(int device, const oc_layout* layout, const void* x, float* best_sim,
+                                 int32_t* best_idx, float* pair_sim, void* stream);
+
 /* One whole cache-wrapped layer call on HOST buffers, for callers that keep activations in host
  * memory: copies x_host (layer input) and cache_host (previous output, same shape) to library-owned
  * device staging, runs match -> select -> gather -> restore with the identity as the wrapped layer

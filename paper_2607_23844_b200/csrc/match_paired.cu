@@ -301,3 +301,69 @@ oc_status launch_match_block(oc_ctx* ctx, const Geo& g, const void* x, float* be
 }
 
 }  // namespace oc
+
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free Frame Cache match (see oc_match_frame_noalloc in omnicache.h).
+//
+// Same two kernels as launch_match_frame, but the partial sums live in a fixed array that is part
+// of the library image, so the call never asks the driver (or anybody's allocator) for memory.
+// ------------------------------------------------------------------------------------------------
+namespace oc {
+
+static constexpr size_t NOALLOC_SCRATCH_BYTES = OC_NOALLOC_SCRATCH_BYTES;
+static constexpr int NOALLOC_MAX_DEVICES = 64;
+
+// Every GPU that loads this library carries this array until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
+
+// In host code `g_noalloc_scratch` is only a handle for the runtime, not a device address.  The
+// address each device gave the array is looked up once per device and kept here.
+static void* g_noalloc_dev_ptr[NOALLOC_MAX_DEVICES] = {};
+
+}  // namespace oc
+
+extern "C" oc_status oc_match_frame_noalloc(int device, const oc_layout* layout, const void* x, float* best_sim,
+                                            int32_t* best_idx, float* pair_sim, void* stream) {
+    using namespace oc;
+    if (device < 0 || device >= NOALLOC_MAX_DEVICES || !x || !best_sim || !best_idx) return OC_ERR_INVALID_ARG;
+    Geo g;
+    oc_status st = make_geo(layout, &g);
+    if (st != OC_OK) return st;
+    if (g.kind != OC_KIND_FRAME) return OC_ERR_INVALID_ARG;
+    if (((uintptr_t)x & 15u) != 0) return OC_ERR_ALIGNMENT;
+    const int n_pairs = g.B * (g.T - 1);
+    if (n_pairs > 65535) return OC_ERR_UNSUPPORTED;
+    // the fixed array must hold what the context workspace would hold for this layout
+    if (frame_workspace_bytes(g) > NOALLOC_SCRATCH_BYTES) return OC_ERR_WORKSPACE;
+
+    DeviceGuard guard(device);
+    if (!guard.ok) return OC_ERR_CUDA;
+    if (!g_noalloc_dev_ptr[device]) {
+        // set-up, once per device, with that device current
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) { cudaGetLastError(); return OC_ERR_CUDA; }
+        g_noalloc_dev_ptr[device] = p;
+    }
+    uint8_t* scratch = (uint8_t*)g_noalloc_dev_ptr[device];
+
+    cudaStream_t s = (cudaStream_t)stream;
+    const int P = g.H * g.W, cpr = g.C * g.elem_bytes / 16;
+    const int lpr = lanes_per_row(cpr);
+    const int ppc = frame_pos_per_cta(g, lpr);
+    const int n_tiles = frame_tiles(g);
+    float4* partial = (float4*)scratch;
+    float* pair_ws = (float*)(scratch + (size_t)(n_pairs > 0 ? n_pairs : 0) * n_tiles * sizeof(float4));
+    // nothing in the array has to start at zero: every partial record and every pair value read
+    // below is written first by this call's own kernels
+    if (n_pairs > 0) {
+        dim3 grid((unsigned)n_tiles, (unsigned)n_pairs);
+        if (g.dtype == OC_DTYPE_BF16)
+            frame_dispatch<OC_DTYPE_BF16>(lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, nullptr, partial, ppc);
+        else
+            frame_dispatch<OC_DTYPE_F32>(lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, nullptr, partial, ppc);
+    }
+    frame_finalize_kernel<<<1, PAIR_THREADS, 0, s>>>(partial, n_tiles, g.B, g.T, P, g.frame_stat, g.eps, pair_ws,
+                                                     pair_sim, best_sim, best_idx);
+    return last_launch_status();
+}

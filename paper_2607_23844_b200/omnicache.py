@@ -31,7 +31,7 @@ EXPORTS = (
     "oc_rows_from_layout", "oc_layer_cache_would_hit", "oc_kernel_name", "oc_create", "oc_destroy",
     "oc_device_status", "oc_profile_enable", "oc_profile_reset", "oc_profile_read", "oc_match",
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
-    "oc_layer_cache_clear", "oc_cache_step_host",
+    "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc",
 )
 
 
@@ -79,6 +79,8 @@ _lib.oc_layer_cache_put.argtypes = [_vp, _i, _i, _vp, C.c_size_t, _vp]
 _lib.oc_layer_cache_get.argtypes = [_vp, _i, _i, _i, _vp, _vp, _vp, _vp]
 _lib.oc_layer_cache_clear.argtypes = [_vp]
 _lib.oc_cache_step_host.argtypes = [_vp, _vp, _i, _f, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.oc_match_frame_noalloc.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp]
+NOALLOC_SCRATCH_BYTES = 1 << 20
 
 
 def status_str(s: int) -> str:
@@ -195,6 +197,22 @@ def _stream(stream) -> int:
     if stream is None:
         return torch.cuda.current_stream().cuda_stream
     return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def match_frame_noalloc(device: int, layout: Layout, x, best_sim, best_idx, pair_sim=None, stream=None,
+                        check: bool = True) -> int:
+    """oc_match_frame_noalloc: the Frame Cache match for callers that may not allocate device memory.
+
+    No context is involved: the partial sums go to a fixed array inside the library (at most
+    NOALLOC_SCRATCH_BYTES; larger layouts come back as ERR_WORKSPACE).  Calls on one device share that
+    array, so do not let two of them overlap on the GPU, and make the first call on a device outside
+    of any stream capture."""
+    cl = layout.c()
+    st = _lib.oc_match_frame_noalloc(device, C.byref(cl), _ptr(x), _ptr(best_sim), _ptr(best_idx), _ptr(pair_sim),
+                                     _stream(stream))
+    if check:
+        _chk(st, "oc_match_frame_noalloc")
+    return st
 
 
 class Context:
