@@ -37,7 +37,7 @@ FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1
 
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES = {"sd3_token": None}
+NCU_TRAFFIC_BYTES = {"sd3_token": 25325568}     # profiles/match_tc_sd3_token.md
 
 
 def measured_peaks():
