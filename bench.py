@@ -364,7 +364,7 @@ def run_ours(args, rank, local_rank, world):
     for name, (n, ms) in prof.items():
         if n:
             ops[name]["share"] = ms / tot_ms
-    n_keep = G * stride
+    n_keep = int(sets[0]["kept_count"].sum().item())       # rows actually kept (threshold mode keeps fewer than G*stride)
     alg_bytes = {"gather": 2 * n_keep * row_bytes, "restore": 2 * n_units * row_bytes, "copy": 2 * tensor_bytes,
                  "norms": tensor_bytes, "frame_pair": tensor_bytes, "block_partial": tensor_bytes}
     for name, b in alg_bytes.items():

@@ -90,43 +90,117 @@ frame_pair_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float ep
     if (threadIdx.x == 0) partial[(long long)q * gridDim.x + blockIdx.x] = make_float4(r0, r1, r2, r3);
 }
 
-// One warp per adjacent pair sums the CTA partials in a fixed order; then thread per frame picks the
-// better adjacent representative.
+// Time-marching variant: a thread-group owns ONE position and walks a segment of frames, keeping the
+// previous frame's row in registers and prefetching the next one, so every row is read exactly once
+// (the pair kernel above reads each row twice, the second time out of L2).  Segments overlap by one
+// frame.  Per pair and CTA the groups' values are combined in a fixed order (shuffles inside a warp,
+// then the warps in index order), written as one partial record per (pair, position tile).
+static constexpr int MARCH_CPL = 8;      // most 16-byte chunks a lane may hold per row (instantiated for 5 and 8)
+
+template <int DT, int LPR, int CPL>
+__global__ void __launch_bounds__(PAIR_THREADS)
+frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float eps, int seg_len, int n_seg,
+                   float* __restrict__ pos_sim, float4* __restrict__ partial) {
+    extern __shared__ float4 warp_part[];                 // [seg_len][PAIR_THREADS / 32]
+    constexpr int GROUPS = PAIR_THREADS / LPR, WARPS = PAIR_THREADS / 32;
+    const int b = blockIdx.y / n_seg, seg = blockIdx.y - b * n_seg;
+    const int t0 = seg * seg_len;                         // first frame of the segment (as "previous")
+    const int t1 = min(T - 1, t0 + seg_len);              // last frame of the segment
+    const int grp = threadIdx.x / LPR, lane = threadIdx.x % LPR, warp = threadIdx.x >> 5, wl = threadIdx.x & 31;
+    const int p = blockIdx.x * GROUPS + grp;
+    const bool valid = p < P;
+    const long long row_bytes = (long long)cpr * 16;
+    const long long frame_bytes = (long long)P * row_bytes;
+    const uint8_t* base = x + ((long long)b * T * P + (valid ? p : 0)) * row_bytes;
+
+    uint4 prev[CPL], cur[CPL], nxt[CPL];
+    auto load_row = [&](uint4* dst, int t) {
+#pragma unroll
+        for (int k = 0; k < CPL; ++k)
+            if (lane + k * LPR < cpr) dst[k] = ld_nc_v4(base + (long long)t * frame_bytes + (long long)(lane + k * LPR) * 16);
+    };
+    load_row(prev, t0);
+    if (t0 + 1 <= t1) load_row(cur, t0 + 1);
+    float n_prev = 0.f;
+#pragma unroll
+    for (int k = 0; k < CPL; ++k)
+        if (lane + k * LPR < cpr) Chunk<DT>::sq(prev[k], n_prev);
+    n_prev = group_sum<LPR>(n_prev);
+
+    for (int t = t0 + 1; t <= t1; ++t) {
+        if (t + 1 <= t1) load_row(nxt, t + 1);            // in flight while frame t is reduced
+        float dot = 0.f, n_cur = 0.f;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k)
+            if (lane + k * LPR < cpr) Chunk<DT>::acc2(cur[k], prev[k], dot, n_cur);
+        dot = group_sum<LPR>(dot); n_cur = group_sum<LPR>(n_cur);
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (valid && lane == 0) {
+            const float cs = clamp_unit(dot / (fmaxf(sqrtf(n_cur), eps) * fmaxf(sqrtf(n_prev), eps)));
+            if (pos_sim) pos_sim[((long long)b * (T - 1) + (t - 1)) * P + p] = cs;
+            v = make_float4(cs, dot, n_cur, n_prev);
+        }
+        // groups of one warp, fixed order
+#pragma unroll
+        for (int d = 16; d >= LPR; d >>= 1) {
+            v.x += __shfl_xor_sync(0xFFFFFFFFu, v.x, d); v.y += __shfl_xor_sync(0xFFFFFFFFu, v.y, d);
+            v.z += __shfl_xor_sync(0xFFFFFFFFu, v.z, d); v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, d);
+        }
+        if (wl == 0) warp_part[(t - t0 - 1) * WARPS + warp] = v;
+        n_prev = n_cur;
+#pragma unroll
+        for (int k = 0; k < CPL; ++k) { prev[k] = cur[k]; cur[k] = nxt[k]; }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < t1 - t0; i += PAIR_THREADS) {
+        float4 a = warp_part[i * WARPS];
+        for (int w = 1; w < WARPS; ++w) {
+            const float4 c = warp_part[i * WARPS + w];
+            a.x += c.x; a.y += c.y; a.z += c.z; a.w += c.w;
+        }
+        const int q = b * (T - 1) + t0 + i;               // pair (t0+i+1, t0+i)
+        partial[(long long)q * gridDim.x + blockIdx.x] = a;
+    }
+}
+
+// One warp per frame: it sums, in a fixed order, the CTA partials of the pair (t, t-1) and of the
+// pair (t+1, t), publishes the first as pair_sim[t-1] and, for an odd (candidate) frame, picks the
+// better of its two adjacent representatives.  Every warp is independent, so frames run in parallel.
+__device__ __forceinline__ float frame_pair_value(const float4* __restrict__ partial, int n_tiles, int q, int P,
+                                                  int stat, float eps) {
+    const int lane = threadIdx.x & 31;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int i = lane; i < n_tiles; i += 32) {
+        const float4 v = partial[(long long)q * n_tiles + i];
+        a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        a0 += __shfl_xor_sync(0xFFFFFFFFu, a0, d); a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, d);
+        a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, d); a3 += __shfl_xor_sync(0xFFFFFFFFu, a3, d);
+    }
+    return stat == OC_FRAME_FLAT_COS ? clamp_unit(a1 / (fmaxf(sqrtf(a2), eps) * fmaxf(sqrtf(a3), eps)))
+                                     : a0 / (float)P;
+}
+
 __global__ void __launch_bounds__(PAIR_THREADS)
 frame_finalize_kernel(const float4* __restrict__ partial, int n_tiles, int B, int T, int P, int stat,
                       float eps, float* __restrict__ pair_ws, float* __restrict__ pair_sim,
                       float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
-    const int n_pairs = B * (T - 1);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int q = warp; q < n_pairs; q += PAIR_THREADS / 32) {
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        for (int i = lane; i < n_tiles; i += 32) {
-            float4 v = partial[(long long)q * n_tiles + i];
-            a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
-        }
-#pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) {
-            a0 += __shfl_xor_sync(0xFFFFFFFFu, a0, d); a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, d);
-            a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, d); a3 += __shfl_xor_sync(0xFFFFFFFFu, a3, d);
-        }
-        if (lane == 0) {
-            float v = stat == OC_FRAME_FLAT_COS
-                          ? clamp_unit(a1 / (fmaxf(sqrtf(a2), eps) * fmaxf(sqrtf(a3), eps)))
-                          : a0 / (float)P;
-            pair_ws[q] = v;
-            if (pair_sim) pair_sim[q] = v;
-        }
+    const int i = blockIdx.x * (PAIR_THREADS / 32) + (threadIdx.x >> 5);     // frame index b*T + t
+    const int lane = threadIdx.x & 31;
+    if (i >= B * T) return;                                                   // whole warps leave together
+    const int b = i / T, t = i - b * T;
+    float with_prev = -INFINITY, with_next = -INFINITY;
+    if (t >= 1) {
+        with_prev = frame_pair_value(partial, n_tiles, b * (T - 1) + t - 1, P, stat, eps);
+        if (lane == 0) { pair_ws[b * (T - 1) + t - 1] = with_prev; if (pair_sim) pair_sim[b * (T - 1) + t - 1] = with_prev; }
     }
-    __syncthreads();
-    for (int i = threadIdx.x; i < B * T; i += PAIR_THREADS) {
-        const int b = i / T, t = i - b * T;
-        if ((t & 1) == 0) { best_sim[i] = -INFINITY; best_idx[i] = i; continue; }
-        float best = pair_ws[b * (T - 1) + t - 1]; int arg = i - 1;
-        if (t + 1 < T) {
-            float nxt = pair_ws[b * (T - 1) + t];
-            if (nxt > best) { best = nxt; arg = i + 1; }
-        }
-        best_sim[i] = best; best_idx[i] = arg;
+    if ((t & 1) && t + 1 < T) with_next = frame_pair_value(partial, n_tiles, b * (T - 1) + t, P, stat, eps);
+    if (lane == 0) {
+        if ((t & 1) == 0) { best_sim[i] = -INFINITY; best_idx[i] = i; }
+        else if (with_next > with_prev) { best_sim[i] = with_next; best_idx[i] = i + 1; }
+        else { best_sim[i] = with_prev; best_idx[i] = i - 1; }
     }
 }
 
@@ -143,45 +217,93 @@ static void frame_dispatch(int lpr, dim3 grid, cudaStream_t s, const uint8_t* x,
     }
 }
 
-static int frame_pos_per_cta(const Geo& g, int lpr) {
-    // every thread-group takes about 4 positions
-    return (PAIR_THREADS / lpr) * 4;
-}
-static int frame_tiles(const Geo& g) {
-    int cpr = g.C * g.elem_bytes / 16;
-    int ppc = frame_pos_per_cta(g, lanes_per_row(cpr));
-    return (g.H * g.W + ppc - 1) / ppc;
+struct FramePlan {
+    bool march;          // time-marching kernel (rows short enough to keep in registers) or pair kernel
+    int lpr, n_tiles, ppc, seg_len, n_seg;
+};
+static FramePlan frame_plan(const Geo& g) {
+    FramePlan f;
+    const int cpr = g.C * g.elem_bytes / 16, P = g.H * g.W;
+    int l = 4;
+    while (l < 32 && l * 5 < cpr) l <<= 1;               // about 5 chunks per lane
+    f.march = g.T >= 2 && cpr <= l * MARCH_CPL;
+    if (f.march) {
+        f.lpr = l;
+        f.n_tiles = (P + PAIR_THREADS / l - 1) / (PAIR_THREADS / l);
+        f.ppc = PAIR_THREADS / l;
+        // segments: enough CTAs for a few waves, but at least 6 pairs per segment (one frame re-read each)
+        int n_seg = 1;
+        while ((long long)f.n_tiles * g.B * n_seg < 148 * 4 && (g.T - 1) / (n_seg + 1) >= 6) ++n_seg;
+        f.seg_len = (g.T - 1 + n_seg - 1) / n_seg;
+        if (f.seg_len > 256) f.seg_len = 256;            // per-pair warp records live in shared memory
+        f.n_seg = (g.T - 1 + f.seg_len - 1) / f.seg_len;
+    } else {
+        f.lpr = lanes_per_row(cpr);
+        f.ppc = (PAIR_THREADS / f.lpr) * 4;              // every thread-group takes about 4 positions
+        f.n_tiles = (P + f.ppc - 1) / f.ppc;
+        f.seg_len = f.n_seg = 0;
+    }
+    return f;
 }
 
 size_t frame_workspace_bytes(const Geo& g) {
     size_t pairs = (size_t)g.B * (size_t)(g.T > 1 ? g.T - 1 : 0);
-    return pairs * (size_t)frame_tiles(g) * sizeof(float4) + pairs * sizeof(float) + 256;
+    return pairs * (size_t)frame_plan(g).n_tiles * sizeof(float4) + pairs * sizeof(float) + 256;
+}
+
+template <int DT>
+static void march_dispatch(int lpr, dim3 grid, size_t smem, cudaStream_t s, const uint8_t* x, int T, int P, int cpr,
+                           float eps, int seg_len, int n_seg, float* pos_sim, float4* partial) {
+#define OC_MARCH(L) do { if (cpr <= 5 * L) frame_march_kernel<DT, L, 5><<<grid, PAIR_THREADS, smem, s>>>(x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial); \
+                         else frame_march_kernel<DT, L, 8><<<grid, PAIR_THREADS, smem, s>>>(x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial); } while (0)
+    switch (lpr) {
+        case 4: OC_MARCH(4); break; case 8: OC_MARCH(8); break; case 16: OC_MARCH(16); break; default: OC_MARCH(32); break;
+    }
+#undef OC_MARCH
+}
+
+// Both frame entry points run this: `scratch` holds the partial records and the pair values.
+// ctx may be null (no launch counters then).
+static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, const void* x, float* best_sim,
+                                 int32_t* best_idx, float* pos_sim, float* pair_sim, cudaStream_t s) {
+    const int P = g.H * g.W, cpr = g.C * g.elem_bytes / 16;
+    const int n_pairs = g.B * (g.T - 1);
+    const FramePlan f = frame_plan(g);
+    float4* partial = (float4*)scratch;
+    float* pair_ws = (float*)(scratch + (size_t)(n_pairs > 0 ? n_pairs : 0) * f.n_tiles * sizeof(float4));
+    if (n_pairs > 65535 || (long long)g.B * (f.march ? f.n_seg : 1) > 65535) return OC_ERR_UNSUPPORTED;
+    struct Scope { oc_ctx* c; int k; cudaStream_t s; LaunchScope* l; 
+                   Scope(oc_ctx* c_, int k_, cudaStream_t s_) : c(c_), k(k_), s(s_), l(c_ ? new LaunchScope(c_, k_, s_) : nullptr) {}
+                   ~Scope() { delete l; } };
+    if (n_pairs > 0) {
+        Scope scope(ctx, OC_K_FRAME, s);
+        if (f.march) {
+            dim3 grid((unsigned)f.n_tiles, (unsigned)(g.B * f.n_seg));
+            const size_t smem = (size_t)f.seg_len * (PAIR_THREADS / 32) * sizeof(float4);
+            if (g.dtype == OC_DTYPE_BF16)
+                march_dispatch<OC_DTYPE_BF16>(f.lpr, grid, smem, s, (const uint8_t*)x, g.T, P, cpr, g.eps, f.seg_len, f.n_seg, pos_sim, partial);
+            else
+                march_dispatch<OC_DTYPE_F32>(f.lpr, grid, smem, s, (const uint8_t*)x, g.T, P, cpr, g.eps, f.seg_len, f.n_seg, pos_sim, partial);
+        } else {
+            dim3 grid((unsigned)f.n_tiles, (unsigned)n_pairs);
+            if (g.dtype == OC_DTYPE_BF16)
+                frame_dispatch<OC_DTYPE_BF16>(f.lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, f.ppc);
+            else
+                frame_dispatch<OC_DTYPE_F32>(f.lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, f.ppc);
+        }
+    }
+    {
+        Scope scope(ctx, OC_K_FRAME_FIN, s);
+        const int warps = PAIR_THREADS / 32;
+        frame_finalize_kernel<<<(unsigned)((g.B * g.T + warps - 1) / warps), PAIR_THREADS, 0, s>>>(
+            partial, f.n_tiles, g.B, g.T, P, g.frame_stat, g.eps, pair_ws, pair_sim, best_sim, best_idx);
+    }
+    return last_launch_status();
 }
 
 oc_status launch_match_frame(oc_ctx* ctx, const Geo& g, const void* x, float* best_sim, int32_t* best_idx,
                              float* pos_sim, float* pair_sim, cudaStream_t s) {
-    const int P = g.H * g.W, cpr = g.C * g.elem_bytes / 16;
-    const int n_pairs = g.B * (g.T - 1);
-    const int lpr = lanes_per_row(cpr);
-    const int ppc = frame_pos_per_cta(g, lpr);
-    const int n_tiles = frame_tiles(g);
-    float4* partial = (float4*)ctx->workspace;
-    float* pair_ws = (float*)((uint8_t*)ctx->workspace + ((size_t)(n_pairs > 0 ? n_pairs : 0) * n_tiles * sizeof(float4)));
-    if (n_pairs > 0) {
-        if (n_pairs > 65535) return OC_ERR_UNSUPPORTED;
-        dim3 grid((unsigned)n_tiles, (unsigned)n_pairs);
-        LaunchScope scope(ctx, OC_K_FRAME, s);
-        if (g.dtype == OC_DTYPE_BF16)
-            frame_dispatch<OC_DTYPE_BF16>(lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, ppc);
-        else
-            frame_dispatch<OC_DTYPE_F32>(lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, ppc);
-    }
-    {
-        LaunchScope scope(ctx, OC_K_FRAME_FIN, s);
-        frame_finalize_kernel<<<1, PAIR_THREADS, 0, s>>>(partial, n_tiles, g.B, g.T, P, g.frame_stat, g.eps,
-                                                         pair_ws, pair_sim, best_sim, best_idx);
-    }
-    return last_launch_status();
+    return run_frame_match(ctx, (uint8_t*)ctx->workspace, g, x, best_sim, best_idx, pos_sim, pair_sim, s);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -192,7 +314,7 @@ oc_status launch_match_frame(oc_ctx* ctx, const Geo& g, const void* x, float* be
 // ------------------------------------------------------------------------------------------------
 static constexpr int MAX_MEMBERS = 16;
 
-template <int DT, int LPR>
+template <int DT, int LPR, int NCMAX>
 __global__ void __launch_bounds__(PAIR_THREADS)
 block_partial_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr, int sy, int sx, int oy, int ox,
                      float* __restrict__ partial, int rec /*floats per (cell,t)*/) {
@@ -210,31 +332,41 @@ block_partial_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr
     const int b = bt / T, t = bt - b * T;
     float* out = partial + (((long long)b * cells + cell) * T + t) * rec;
 
-    float rn = 0.f;
-    for (int c = lane; c < cpr; c += LPR) { uint4 r = ld_nc_v4(rep + (long long)c * 16); Chunk<DT>::sq(r, rn); }
+    // the neighbourhood's other members, in (my, mx) order
+    const int nc = sy * sx - 1;
+    const uint8_t* cand[NCMAX];
+    const int rep_m = oy * sx + ox;
+#pragma unroll
+    for (int k = 0; k < NCMAX; ++k) {
+        const int m = k + (k >= rep_m ? 1 : 0);      // k-th non-representative member
+        const int my = m / sx, mx = m - my * sx;
+        cand[k] = k < nc ? frame + ((long long)(cy * sy + my) * W + (cx * sx + mx)) * row_bytes : rep;
+    }
+    // one pass over the channels: the representative's chunk and every member's chunk are loaded
+    // together, so up to 1 + nc loads are in flight per lane and step
+    float rn = 0.f, dot[NCMAX], na[NCMAX];
+#pragma unroll
+    for (int k = 0; k < NCMAX; ++k) { dot[k] = 0.f; na[k] = 0.f; }
+    for (int c = lane; c < cpr; c += LPR) {
+        const uint4 r = ld_nc_v4(rep + (long long)c * 16);
+        uint4 a[NCMAX];
+#pragma unroll
+        for (int k = 0; k < NCMAX; ++k)
+            if (k < nc) a[k] = ld_nc_v4(cand[k] + (long long)c * 16);
+        Chunk<DT>::sq(r, rn);
+#pragma unroll
+        for (int k = 0; k < NCMAX; ++k)
+            if (k < nc) Chunk<DT>::acc2(a[k], r, dot[k], na[k]);
+    }
     rn = group_sum<LPR>(rn);
     if (valid && lane == 0) out[0] = rn;
-    int k = 0;
-    for (int my = 0; my < sy; ++my)
-        for (int mx = 0; mx < sx; ++mx) {
-            if (my == oy && mx == ox) continue;
-            const uint8_t* cand = frame + ((long long)(cy * sy + my) * W + (cx * sx + mx)) * row_bytes;
-            float dot = 0.f, na = 0.f;
-            int c = lane;
-            for (; c + LPR < cpr; c += 2 * LPR) {
-                uint4 a0 = ld_nc_v4(cand + (long long)c * 16), r0 = ld_nc_v4(rep + (long long)c * 16);
-                uint4 a1 = ld_nc_v4(cand + (long long)(c + LPR) * 16), r1 = ld_nc_v4(rep + (long long)(c + LPR) * 16);
-                Chunk<DT>::acc2(a0, r0, dot, na);
-                Chunk<DT>::acc2(a1, r1, dot, na);
-            }
-            if (c < cpr) {
-                uint4 a0 = ld_nc_v4(cand + (long long)c * 16), r0 = ld_nc_v4(rep + (long long)c * 16);
-                Chunk<DT>::acc2(a0, r0, dot, na);
-            }
-            dot = group_sum<LPR>(dot); na = group_sum<LPR>(na);
-            if (valid && lane == 0) { out[1 + 2 * k] = dot; out[2 + 2 * k] = na; }
-            ++k;
+#pragma unroll
+    for (int k = 0; k < NCMAX; ++k) {
+        if (k < nc) {                                 // nc is uniform over the grid
+            const float d = group_sum<LPR>(dot[k]), n = group_sum<LPR>(na[k]);
+            if (valid && lane == 0) { out[1 + 2 * k] = d; out[2 + 2 * k] = n; }
         }
+    }
 }
 
 __global__ void __launch_bounds__(PAIR_THREADS)
@@ -267,7 +399,8 @@ size_t block_workspace_bytes(const Geo& g) {
 
 template <int DT>
 static void block_dispatch(int lpr, dim3 grid, cudaStream_t s, const uint8_t* x, const Geo& g, int cpr, float* partial, int rec) {
-#define OC_BLK(L) block_partial_kernel<DT, L><<<grid, PAIR_THREADS, 0, s>>>(x, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec)
+#define OC_BLK(L) do { if (g.sy * g.sx - 1 <= 3) block_partial_kernel<DT, L, 3><<<grid, PAIR_THREADS, 0, s>>>(x, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec); \
+                       else block_partial_kernel<DT, L, 15><<<grid, PAIR_THREADS, 0, s>>>(x, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec); } while (0)
     switch (lpr) {
         case 1: OC_BLK(1); break; case 2: OC_BLK(2); break; case 4: OC_BLK(4); break;
         case 8: OC_BLK(8); break; case 16: OC_BLK(16); break; default: OC_BLK(32); break;
@@ -346,24 +479,7 @@ extern "C" oc_status oc_match_frame_noalloc(int device, const oc_layout* layout,
         g_noalloc_dev_ptr[device] = p;
     }
     uint8_t* scratch = (uint8_t*)g_noalloc_dev_ptr[device];
-
-    cudaStream_t s = (cudaStream_t)stream;
-    const int P = g.H * g.W, cpr = g.C * g.elem_bytes / 16;
-    const int lpr = lanes_per_row(cpr);
-    const int ppc = frame_pos_per_cta(g, lpr);
-    const int n_tiles = frame_tiles(g);
-    float4* partial = (float4*)scratch;
-    float* pair_ws = (float*)(scratch + (size_t)(n_pairs > 0 ? n_pairs : 0) * n_tiles * sizeof(float4));
-    // nothing in the array has to start at zero: every partial record and every pair value read
-    // below is written first by this call's own kernels
-    if (n_pairs > 0) {
-        dim3 grid((unsigned)n_tiles, (unsigned)n_pairs);
-        if (g.dtype == OC_DTYPE_BF16)
-            frame_dispatch<OC_DTYPE_BF16>(lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, nullptr, partial, ppc);
-        else
-            frame_dispatch<OC_DTYPE_F32>(lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, nullptr, partial, ppc);
-    }
-    frame_finalize_kernel<<<1, PAIR_THREADS, 0, s>>>(partial, n_tiles, g.B, g.T, P, g.frame_stat, g.eps, pair_ws,
-                                                     pair_sim, best_sim, best_idx);
-    return last_launch_status();
+    // nothing in the array has to start at zero: every partial record and every pair value that
+    // the kernels read is written first by this call's own kernels
+    return run_frame_match(nullptr, scratch, g, x, best_sim, best_idx, nullptr, pair_sim, (cudaStream_t)stream);
 }
