@@ -48,7 +48,7 @@ static constexpr int BK = 64;            // channels per stage: 128 bytes of bf1
 static constexpr int A_BYTES = BM * BK * 2;
 static constexpr int Q_BYTES = QN * BK * 2;
 static constexpr int MAX_STAGES = 8;
-static constexpr int TILE_BYTES = 192 * 1024;    // operand ring
+static constexpr int SMEM_LIMIT = 232448;         // 227 KB: the most dynamic shared memory a CTA may have
 static constexpr int TC_THREADS = 320;   // producer warp, MMA warp, 8 epilogue warps
 static constexpr int EPI_THREADS = 256;
 static constexpr int MAX_LATTICES = 9;
@@ -201,12 +201,16 @@ struct Walk {
 
 static constexpr int COL_BYTES = 256 * 8;                               // {scale, bias} per column of a piece
 static constexpr int N_BARS = 2 * MAX_STAGES + 3;                       // full[], empty[], acc_full, acc_empty, drain
-static constexpr int SMEM_TOTAL = 1024 + TILE_BYTES + COL_BYTES + N_BARS * 8 + 16;
+static constexpr int TAIL_BYTES = COL_BYTES + N_BARS * 8 + 32;        // column table, barriers, TMEM slot, flags
+static constexpr int TILE_BYTES = (SMEM_LIMIT - TAIL_BYTES) / 1024 * 1024;   // operand ring: everything else
+static constexpr int SMEM_TOTAL = TILE_BYTES + TAIL_BYTES;
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 match_tc_kernel(const __grid_constant__ TcParams P) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // The operand ring starts at the base of dynamic shared memory, which must be 1024-byte aligned
+    // for the 128-byte swizzle (this kernel has no static shared memory in front of it; checked below).
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = smem_raw;
     float4* colsb = (float4*)(smem + TILE_BYTES);                      // 128 pairs of {scale, bias}
     uint64_t* bars = (uint64_t*)(smem + TILE_BYTES + COL_BYTES);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * MAX_STAGES;
@@ -218,6 +222,10 @@ match_tc_kernel(const __grid_constant__ TcParams P) {
     const int STAGES = P.n_stages, STAGE_BYTES = P.stage_bytes;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if ((tiles_base & 1023u) != 0) {                                   // never expected; refuse rather than compute garbage
+        if (threadIdx.x == 0) atomicCAS(P.status, 0, OC_ERR_ALIGNMENT);
+        return;
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
