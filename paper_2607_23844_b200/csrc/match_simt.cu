@@ -10,30 +10,54 @@
 namespace oc {
 
 // ---- pre-pass ----------------------------------------------------------------------------------
-template <int DT>
+// Persistent warps; a thread-group of LPR lanes owns a row (about five 16-byte chunks per lane), so a
+// warp has 32/LPR rows in flight and every lane keeps several independent loads outstanding.
+template <int DT, int LPR>
 __global__ void __launch_bounds__(256)
 norms_kernel(const uint8_t* __restrict__ x, long long n_tok, int cpr, float eps,
              float* __restrict__ inv_norm, unsigned long long* __restrict__ keys) {
-    const int lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (row >= n_tok) return;
-    const uint8_t* r = x + row * (long long)cpr * 16;
-    float s0 = 0.f, s1 = 0.f;
-    for (int c = lane; c < cpr; c += 128) {                 // up to four 16-byte loads in flight per lane
-        uint4 v[4];
+    constexpr int CPL = 8;                                   // chunks a lane holds at once
+    const int lane = threadIdx.x % LPR;
+    const long long groups_total = (long long)gridDim.x * (256 / LPR);
+    const long long grp0 = (long long)blockIdx.x * (256 / LPR) + threadIdx.x / LPR;
+    const long long n_iter = (n_tok + groups_total - 1) / groups_total;   // same trip count for every thread
+    for (long long it = 0; it < n_iter; ++it) {
+        const long long row = grp0 + it * groups_total;
+        const bool valid = row < n_tok;
+        const uint8_t* r = x + (valid ? row : 0) * (long long)cpr * 16;
+        float s = 0.f;
+        for (int c0 = 0; c0 < cpr; c0 += CPL * LPR) {
+            uint4 v[CPL];
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (c + 32 * k < cpr) v[k] = ld_nc_v4(r + (long long)(c + 32 * k) * 16);
+            for (int k = 0; k < CPL; ++k)
+                if (c0 + lane + k * LPR < cpr) v[k] = ld_nc_v4(r + (long long)(c0 + lane + k * LPR) * 16);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (c + 32 * k < cpr) Chunk<DT>::sq(v[k], (k & 1) ? s1 : s0);
+            for (int k = 0; k < CPL; ++k)
+                if (c0 + lane + k * LPR < cpr) Chunk<DT>::sq(v[k], s);
+        }
+#pragma unroll
+        for (int d = LPR / 2; d >= 1; d >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
+        if (valid && lane == 0) {
+            inv_norm[row] = 1.0f / fmaxf(sqrtf(s), eps);
+            keys[row] = 0ull;
+        }
     }
-    float s = s0 + s1;
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, d);
-    if (lane == 0) {
-        inv_norm[row] = 1.0f / fmaxf(sqrtf(s), eps);
-        keys[row] = 0ull;
+}
+
+template <int DT>
+static void norms_dispatch(int sm_count, cudaStream_t s, const uint8_t* x, long long n_tok, int cpr, float eps,
+                           float* inv_norm, unsigned long long* keys) {
+    int lpr = 4;
+    while (lpr < 32 && lpr * 5 < cpr) lpr <<= 1;
+    const long long rows_per_block = 256 / lpr;
+    long long blocks = (n_tok + rows_per_block - 1) / rows_per_block;
+    const long long cap = (long long)sm_count * 4;           // 4 resident CTAs of 256 threads per SM (64 registers)
+    if (blocks > cap) blocks = cap;
+    switch (lpr) {
+        case 4:  norms_kernel<DT, 4><<<(unsigned)blocks, 256, 0, s>>>(x, n_tok, cpr, eps, inv_norm, keys); break;
+        case 8:  norms_kernel<DT, 8><<<(unsigned)blocks, 256, 0, s>>>(x, n_tok, cpr, eps, inv_norm, keys); break;
+        case 16: norms_kernel<DT, 16><<<(unsigned)blocks, 256, 0, s>>>(x, n_tok, cpr, eps, inv_norm, keys); break;
+        default: norms_kernel<DT, 32><<<(unsigned)blocks, 256, 0, s>>>(x, n_tok, cpr, eps, inv_norm, keys); break;
     }
 }
 
@@ -205,11 +229,10 @@ oc_status launch_match_token(oc_ctx* ctx, const Geo& g, const void* x, float* be
     const int cpr = g.C * g.elem_bytes / 16;
     {
         LaunchScope scope(ctx, OC_K_NORMS, s);
-        unsigned blocks = (unsigned)((n_tok + 7) / 8);
         if (g.dtype == OC_DTYPE_BF16)
-            norms_kernel<OC_DTYPE_BF16><<<blocks, 256, 0, s>>>((const uint8_t*)x, n_tok, cpr, g.eps, inv_norm, keys);
+            norms_dispatch<OC_DTYPE_BF16>(ctx->sm_count, s, (const uint8_t*)x, n_tok, cpr, g.eps, inv_norm, keys);
         else
-            norms_kernel<OC_DTYPE_F32><<<blocks, 256, 0, s>>>((const uint8_t*)x, n_tok, cpr, g.eps, inv_norm, keys);
+            norms_dispatch<OC_DTYPE_F32>(ctx->sm_count, s, (const uint8_t*)x, n_tok, cpr, g.eps, inv_norm, keys);
     }
     oc_status st = OC_ERR_UNSUPPORTED;
     if (tc_match_supported(g)) st = launch_match_token_tc(ctx, g, x, inv_norm, keys, aux_sim, s);
