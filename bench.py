@@ -414,6 +414,131 @@ def run_ours(args, rank, local_rank, world):
     ctx.close()
 
 
+# ---------------------------------------------------------------------------------------------------
+# config 5: the SVD-XT sweep (three U-Net levels x Token / Frame / Block Cache x keep ratios + the
+# Layered Cache), per-op and summed device times.  One JSON line; an extra mode, not the default.
+# ---------------------------------------------------------------------------------------------------
+def run_sweep(args):
+    import torch
+    from paper_2607_23844_b200 import build
+    build.build()
+    from paper_2607_23844_b200 import omnicache as oc
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    stream = torch.cuda.current_stream()
+
+    def graph_time_us(fn, reps):
+        """fn() enqueues one pass over the ring; returns device microseconds per pass (graph replay)."""
+        fn(); torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        g.replay(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record(); torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / reps
+
+    results = []
+    for level, (H, W, C) in enumerate(inputs.SVD_LEVELS):
+        base = inputs.svd_frames(seed=1005 + level, T=25, H=H, W=W, C=C, kind="token")
+        tensor_bytes = int(np.prod(base.shape)) * 2
+        ring = max(2, -(-4 * L2_BYTES // (3 * tensor_bytes)))
+        xs = [torch.from_numpy(base.x.view(np.int16)).to(dev) for _ in range(ring)]
+        caches = [torch.empty_like(xs[0]) for _ in range(ring)]
+        outs = [torch.empty_like(xs[0]) for _ in range(ring)]
+        for kind in ("token", "frame", "block"):
+            L = oc.Layout(KIND[kind], inputs.BF16, *base.shape)
+            G, U, R = L.counts()
+            n_units, n_cand = G * U, G * (U - R)
+            rows = oc.rows_from_layout(L, C, 2)
+            row_bytes = rows.seg_bytes * rows.n_seg
+            ctx = oc.Context(0, oc.match_workspace_bytes(L))
+            sims = [torch.empty(n_units, dtype=torch.float32, device=dev) for _ in range(ring)]
+            idxs = [torch.empty(n_units, dtype=torch.int32, device=dev) for _ in range(ring)]
+
+            def f_match():
+                for r in range(ring):
+                    ctx.match(L, xs[r], sims[r], idxs[r], stream=torch.cuda.current_stream())
+            reps = max(3, args.steps // 10)
+            t_match = graph_time_us(f_match, reps) / ring
+            if kind == "token":
+                flops = 2.0 * n_cand * R * C
+                match_rate = {"TFLOP/s": flops / (t_match * 1e-6) / 1e12}
+            else:
+                match_rate = {"GB/s": tensor_bytes / (t_match * 1e-6) / 1e9,
+                              "frac_hbm": tensor_bytes / (t_match * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+            for ratio in (0.25, 0.5, 0.75):
+                n_reuse = inputs.keep_ratio_to_reuse(U, U - R, ratio)
+                stride = U - n_reuse
+                kept = [torch.empty(G * stride, dtype=torch.int32, device=dev) for _ in range(ring)]
+                cnt = [torch.empty(G, dtype=torch.int32, device=dev) for _ in range(ring)]
+                mm = [torch.empty(n_units, dtype=torch.int32, device=dev) for _ in range(ring)]
+                so = [torch.empty(n_units, dtype=torch.int32, device=dev) for _ in range(ring)]
+                ys = [torch.empty(G * stride * row_bytes, dtype=torch.uint8, device=dev) for _ in range(ring)]
+
+                def f_select():
+                    for r in range(ring):
+                        ctx.select(L, sims[r], idxs[r], oc.SELECT_COUNT, 0.0, n_reuse, stride, kept[r], cnt[r], mm[r], so[r],
+                                   stream=torch.cuda.current_stream())
+
+                def f_gather():
+                    for r in range(ring):
+                        ctx.gather(rows, xs[r], kept[r], G * stride, ys[r], stream=torch.cuda.current_stream())
+
+                def f_restore():
+                    for r in range(ring):
+                        ctx.restore(rows, ys[r], caches[r], n_units, so[r], mm[r], outs[r], stream=torch.cuda.current_stream())
+                t_sel = graph_time_us(f_select, reps) / ring
+                t_gat = graph_time_us(f_gather, reps) / ring
+                t_res = graph_time_us(f_restore, reps) / ring
+                gb = lambda b, t: b / (t * 1e-6) / 1e9
+                res = {
+                    "level": level, "shape": list(base.shape), "cache": kind, "keep_ratio": ratio, "n_reuse_per_group": n_reuse,
+                    "match_us": t_match, "select_us": t_sel, "gather_us": t_gat, "restore_us": t_res,
+                    "summed_us": t_match + t_sel + t_gat + t_res,
+                    "matched_units_per_s": n_cand / ((t_match + t_sel) * 1e-6),
+                    "restored_units_per_s": n_units / (t_res * 1e-6),
+                    "match": match_rate,
+                    "gather_GB/s": gb(2 * G * stride * row_bytes, t_gat),
+                    "gather_frac_hbm": gb(2 * G * stride * row_bytes, t_gat) / peaks["hbm_gbs"],
+                    "restore_GB/s": gb(2 * n_units * row_bytes, t_res),
+                    "restore_frac_hbm": gb(2 * n_units * row_bytes, t_res) / peaks["hbm_gbs"],
+                }
+                results.append(res)
+            assert ctx.device_status() == oc.OK
+            ctx.close()
+        # Layered Cache: put every 5th step, copying get on the others (25 steps, N = 5)
+        ctx = oc.Context(0, 0)
+        for r in range(ring):
+            ctx.layer_cache_put(r, 0, xs[r], tensor_bytes)
+
+        def f_put():
+            for r in range(ring):
+                ctx.layer_cache_put(r, 0, xs[r], tensor_bytes, stream=torch.cuda.current_stream())
+
+        def f_get():
+            for r in range(ring):
+                ctx.layer_cache_get(r, 3, 5, outs[r], stream=torch.cuda.current_stream())
+        t_put = graph_time_us(f_put, max(3, args.steps // 10)) / ring
+        t_get = graph_time_us(f_get, max(3, args.steps // 10)) / ring
+        results.append({"level": level, "cache": "layered", "entry_bytes": tensor_bytes, "put_us": t_put, "get_copy_us": t_get,
+                        "put_frac_hbm": 2 * tensor_bytes / (t_put * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                        "get_frac_hbm": 2 * tensor_bytes / (t_get * 1e-6) / 1e9 / peaks["hbm_gbs"],
+                        "steps_25_interval_5_total_us": 5 * t_put + 20 * t_get})
+        ctx.close()
+        del xs, caches, outs
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "per-op and summed device time, SVD-XT sweep (config 5)", "unit": "us",
+                      "timing": "CUDA-graph replay per op over a ring of buffers larger than 4x L2",
+                      "peaks": {"hbm_gbs": peaks["hbm_gbs"], "source": peaks["_source"]}, "data": "synthetic",
+                      "results": results}), flush=True)
+
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -433,6 +558,10 @@ def main():
     if args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     rank, local_rank, world = sharding.env_rank_world()
+    if args.workload == "svd_sweep":
+        if rank == 0:
+            run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args, rank)
         return

@@ -330,7 +330,7 @@ block_partial_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr
     const uint8_t* frame = x + (long long)bt * H * W * row_bytes;
     const uint8_t* rep = frame + ((long long)(cy * sy + oy) * W + (cx * sx + ox)) * row_bytes;
     const int b = bt / T, t = bt - b * T;
-    float* out = partial + (((long long)b * cells + cell) * T + t) * rec;
+    float* out = partial + (((long long)b * T + t) * cells + cell) * rec;     // [b][t][cell][rec]
 
     // the neighbourhood's other members, in (my, mx) order
     const int nc = sy * sx - 1;
@@ -369,6 +369,67 @@ block_partial_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr
     }
 }
 
+// Variant for neighbourhoods with at most three candidates and rows short enough to hold in
+// registers (CPL chunks per lane): every load of the item - the representative's row and all
+// candidates' rows - is issued before the first one is used.
+template <int DT, int LPR, int CPL>
+__global__ void __launch_bounds__(PAIR_THREADS)
+block_partial_reg_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr, int sy, int sx, int oy, int ox,
+                         float* __restrict__ partial, int rec) {
+    constexpr int NC = 3;
+    const int bt = blockIdx.y;
+    const int cells_x = W / sx, cells = (H / sy) * cells_x;
+    const int groups = PAIR_THREADS / LPR;
+    const int grp = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+    const int cell_raw = blockIdx.x * groups + grp;
+    const bool valid = cell_raw < cells;
+    const int cell = valid ? cell_raw : 0;
+    const int cy = cell / cells_x, cx = cell - cy * cells_x;
+    const long long row_bytes = (long long)cpr * 16;
+    const uint8_t* frame = x + (long long)bt * H * W * row_bytes;
+    const uint8_t* rep = frame + ((long long)(cy * sy + oy) * W + (cx * sx + ox)) * row_bytes;
+    const int b = bt / T, t = bt - b * T;
+    float* out = partial + (((long long)b * T + t) * cells + cell) * rec;     // [b][t][cell][rec]
+    const int nc = sy * sx - 1, rep_m = oy * sx + ox;
+    const uint8_t* cand[NC];
+#pragma unroll
+    for (int k = 0; k < NC; ++k) {
+        const int m = k + (k >= rep_m ? 1 : 0);
+        const int my = m / sx, mx = m - my * sx;
+        cand[k] = k < nc ? frame + ((long long)(cy * sy + my) * W + (cx * sx + mx)) * row_bytes : rep;
+    }
+    uint4 r[CPL], a[NC][CPL];
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) {
+        const int c = lane + j * LPR;
+        if (c < cpr) {
+            r[j] = ld_nc_v4(rep + (long long)c * 16);
+#pragma unroll
+            for (int k = 0; k < NC; ++k)
+                if (k < nc) a[k][j] = ld_nc_v4(cand[k] + (long long)c * 16);
+        }
+    }
+    float rn = 0.f, dot[NC] = {0.f, 0.f, 0.f}, na[NC] = {0.f, 0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) {
+        if (lane + j * LPR < cpr) {
+            Chunk<DT>::sq(r[j], rn);
+#pragma unroll
+            for (int k = 0; k < NC; ++k)
+                if (k < nc) Chunk<DT>::acc2(a[k][j], r[j], dot[k], na[k]);
+        }
+    }
+    rn = group_sum<LPR>(rn);
+    if (valid && lane == 0) out[0] = rn;
+#pragma unroll
+    for (int k = 0; k < NC; ++k) {
+        if (k < nc) {
+            const float d = group_sum<LPR>(dot[k]), n = group_sum<LPR>(na[k]);
+            if (valid && lane == 0) { out[1 + 2 * k] = d; out[2 + 2 * k] = n; }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(PAIR_THREADS)
 block_finalize_kernel(const float* __restrict__ partial, int B, int T, int H, int W, int sy, int sx, int oy, int ox,
                       int rec, float eps, float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
@@ -384,9 +445,13 @@ block_finalize_kernel(const float* __restrict__ partial, int B, int T, int H, in
     const int cell = (y / sy) * cells_x + xx / sx;
     int k = my * sx + mx;                        // rank among the neighbourhood's non-representatives
     if (k > oy * sx + ox) --k;
-    const float* recs = partial + ((long long)b * cells + cell) * T * rec;
+    // records are laid out [b][t][cell][rec]: neighbouring threads (cells) read neighbouring records
+    const float* recs = partial + ((long long)b * T * cells + cell) * rec;
+    const long long t_stride = (long long)cells * rec;
     float rn = 0.f, dot = 0.f, na = 0.f;
-    for (int t = 0; t < T; ++t) { rn += recs[t * rec]; dot += recs[t * rec + 1 + 2 * k]; na += recs[t * rec + 2 + 2 * k]; }
+    for (int t = 0; t < T; ++t) {
+        rn += recs[t * t_stride]; dot += recs[t * t_stride + 1 + 2 * k]; na += recs[t * t_stride + 2 + 2 * k];
+    }
     best_sim[i] = clamp_unit(dot / (fmaxf(sqrtf(na), eps) * fmaxf(sqrtf(rn), eps)));
     best_idx[i] = (int32_t)((long long)b * P + (y - my + oy) * W + (xx - mx + ox));
 }
@@ -412,17 +477,35 @@ oc_status launch_match_block(oc_ctx* ctx, const Geo& g, const void* x, float* be
                              cudaStream_t s) {
     if (g.sy * g.sx > MAX_MEMBERS) return OC_ERR_UNSUPPORTED;
     const int cpr = g.C * g.elem_bytes / 16;
-    const int lpr = lanes_per_row(cpr);
     const int cells = (g.H / g.sy) * (g.W / g.sx);
     const int rec = 1 + 2 * (g.sy * g.sx - 1);
     float* partial = (float*)ctx->workspace;
     if ((int64_t)g.B * g.T > 65535) return OC_ERR_UNSUPPORTED;
+    // register-resident variant: about five chunks per lane, at most three candidates
+    int lr = 4;
+    while (lr < 32 && lr * 5 < cpr) lr <<= 1;
+    const bool reg_variant = g.sy * g.sx - 1 <= 3 && cpr <= 5 * lr;
+    const int lpr = reg_variant ? lr : lanes_per_row(cpr);
     {
         const int groups = PAIR_THREADS / lpr;
         dim3 grid((unsigned)((cells + groups - 1) / groups), (unsigned)(g.B * g.T));
         LaunchScope scope(ctx, OC_K_BLOCK, s);
-        if (g.dtype == OC_DTYPE_BF16) block_dispatch<OC_DTYPE_BF16>(lpr, grid, s, (const uint8_t*)x, g, cpr, partial, rec);
-        else block_dispatch<OC_DTYPE_F32>(lpr, grid, s, (const uint8_t*)x, g, cpr, partial, rec);
+        const uint8_t* xb = (const uint8_t*)x;
+        if (reg_variant) {
+#define OC_BLKR(DTV, L) block_partial_reg_kernel<DTV, L, 5><<<grid, PAIR_THREADS, 0, s>>>(xb, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec)
+            if (g.dtype == OC_DTYPE_BF16) {
+                switch (lpr) { case 4: OC_BLKR(OC_DTYPE_BF16, 4); break; case 8: OC_BLKR(OC_DTYPE_BF16, 8); break;
+                               case 16: OC_BLKR(OC_DTYPE_BF16, 16); break; default: OC_BLKR(OC_DTYPE_BF16, 32); break; }
+            } else {
+                switch (lpr) { case 4: OC_BLKR(OC_DTYPE_F32, 4); break; case 8: OC_BLKR(OC_DTYPE_F32, 8); break;
+                               case 16: OC_BLKR(OC_DTYPE_F32, 16); break; default: OC_BLKR(OC_DTYPE_F32, 32); break; }
+            }
+#undef OC_BLKR
+        } else if (g.dtype == OC_DTYPE_BF16) {
+            block_dispatch<OC_DTYPE_BF16>(lpr, grid, s, xb, g, cpr, partial, rec);
+        } else {
+            block_dispatch<OC_DTYPE_F32>(lpr, grid, s, xb, g, cpr, partial, rec);
+        }
     }
     {
         const long long n = (long long)g.B * g.H * g.W;
