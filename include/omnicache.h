@@ -153,6 +153,13 @@ oc_status oc_destroy(oc_ctx* ctx);
  * device-side condition recorded since the last call (OC_ERR_TIMEOUT). */
 oc_status oc_device_status(oc_ctx* ctx, int* code);
 
+/* Self-test of the device-side failure path.  Every wait inside the kernels is bounded; when one
+ * runs out the kernel records OC_ERR_TIMEOUT in the status word and returns instead of hanging.
+ * This call launches a one-warp kernel that waits, for at most limit_us microseconds
+ * (1 .. 1000000), on a barrier that nothing completes, so that path can be observed on demand:
+ * afterwards oc_device_status() reports OC_ERR_TIMEOUT once, and the context works as before. */
+oc_status oc_selftest_bounded_wait(oc_ctx* ctx, unsigned int limit_us, void* stream);
+
 /* Launch counters and optional per-kernel timers.  Counters always run.  With timers enabled each
  * kernel launch is bracketed by CUDA events on the caller's stream; oc_profile_read waits for the
  * recorded events and returns the number of launches and their summed device time since the last

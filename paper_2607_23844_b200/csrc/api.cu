@@ -234,6 +234,13 @@ oc_status oc_device_status(oc_ctx* c, int* code) {
     return OC_OK;
 }
 
+oc_status oc_selftest_bounded_wait(oc_ctx* c, unsigned int limit_us, void* stream) {
+    if (!c || limit_us == 0 || limit_us > 1000000u) return OC_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return OC_ERR_CUDA;
+    return launch_bounded_wait_selftest(c, (unsigned long long)limit_us * 1000ull, (cudaStream_t)stream);
+}
+
 oc_status oc_profile_enable(oc_ctx* c, int on) {
     if (!c) return OC_ERR_INVALID_ARG;
     c->profile_on = on != 0;

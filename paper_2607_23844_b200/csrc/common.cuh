@@ -127,6 +127,7 @@ bool tc_match_supported(const Geo&);
 oc_status launch_match_token_tc(oc_ctx*, const Geo&, const void* x, const float* inv_norm,
                                 unsigned long long* keys, float* aux_sim, cudaStream_t);
 void tc_cache_free(oc_ctx*);
+oc_status launch_bounded_wait_selftest(oc_ctx*, unsigned long long limit_ns, cudaStream_t);
 
 size_t match_workspace_bytes(const Geo&);
 

@@ -463,6 +463,34 @@ match_tc_kernel(const __grid_constant__ TcParams P) {
     }
 }
 
+// ---- self-test of the bounded wait ---------------------------------------------------------------
+// One warp waits on an mbarrier that nothing ever completes, with the same try_wait / %globaltimer
+// loop the matcher uses but a caller-chosen limit.  The wait runs out, the kernel records
+// OC_ERR_TIMEOUT in the status word and returns normally: the context stays usable.
+__global__ void bounded_wait_selftest_kernel(unsigned long long limit_ns, int* status) {
+    __shared__ uint64_t bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        const unsigned long long t0 = global_ns();
+        bool done = false;
+        unsigned spins = 0;
+        while (!(done = mbar_try_wait(b, 0))) {
+            if ((++spins & 63u) == 0 && global_ns() - t0 > limit_ns) break;
+        }
+        if (!done) atomicCAS(status, 0, OC_ERR_TIMEOUT);
+    }
+}
+
+oc_status launch_bounded_wait_selftest(oc_ctx* ctx, unsigned long long limit_ns, cudaStream_t s) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(limit_ns, ctx->d_status);
+    return last_launch_status();
+}
+
 // ---- host side ---------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

@@ -31,7 +31,7 @@ EXPORTS = (
     "oc_rows_from_layout", "oc_layer_cache_would_hit", "oc_kernel_name", "oc_create", "oc_destroy",
     "oc_device_status", "oc_profile_enable", "oc_profile_reset", "oc_profile_read", "oc_match",
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
-    "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc",
+    "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
 )
 
 
@@ -68,6 +68,7 @@ _lib.oc_layer_cache_would_hit.argtypes = [_i, _i, _i]
 _lib.oc_create.argtypes = [_vp, _i, C.c_size_t]
 _lib.oc_destroy.argtypes = [_vp]
 _lib.oc_device_status.argtypes = [_vp, _vp]
+_lib.oc_selftest_bounded_wait.argtypes = [_vp, C.c_uint, _vp]
 _lib.oc_profile_enable.argtypes = [_vp, _i]
 _lib.oc_profile_reset.argtypes = [_vp]
 _lib.oc_profile_read.argtypes = [_vp, _i, _vp, _vp]
@@ -246,6 +247,10 @@ class Context:
         code = C.c_int()
         _chk(_lib.oc_device_status(self._h, C.byref(code)), "oc_device_status")
         return code.value
+
+    def selftest_bounded_wait(self, limit_us: int = 2000, stream=None) -> None:
+        """Makes a bounded device-side wait run out on purpose (see oc_selftest_bounded_wait)."""
+        _chk(_lib.oc_selftest_bounded_wait(self._h, limit_us, _stream(stream)), "oc_selftest_bounded_wait")
 
     def profile_enable(self, on: bool) -> None:
         _chk(_lib.oc_profile_enable(self._h, int(on)), "oc_profile_enable")

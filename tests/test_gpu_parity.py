@@ -397,3 +397,20 @@ def test_cache_step_host_matches_device_path(oc, oracle):
     want = oracle.restore(R, y, cache_np, Lo.n_units, s["slot_of"], s["match_map"])
     assert oh.numpy().tobytes() == want.tobytes()
     assert np.array_equal(kh.numpy(), s["kept_count"])
+
+
+def test_bounded_wait_expires_into_the_status_word_and_context_stays_usable(oc, oracle):
+    """Failure detection without a fault: a wait that nothing satisfies gives up after its limit,
+    the status word says OC_ERR_TIMEOUT once, and the same context then matches correctly."""
+    w = inputs.sd3_token_cache(seed=14, B=1, H=32, W=32, C=128)
+    L, Lo = H.layouts(oc, oracle, w)
+    with H.make_ctx(oc, L) as ctx:
+        assert ctx.device_status() == oc.OK
+        ctx.selftest_bounded_wait(2000)
+        assert ctx.device_status() == oc.ERR_TIMEOUT
+        assert ctx.device_status() == oc.OK                      # read-and-clear
+        m = H.gpu_match(oc, ctx, L, H.to_dev(w.x))
+        ref = oracle.match_token(Lo, w.x)
+        H.check_match_against_oracle(oracle, Lo, w.x, m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy(),
+                                     ref, TOL[w.dtype])
+        assert oc._lib.oc_selftest_bounded_wait(ctx._h, 0, None) == oc.ERR_INVALID_ARG
