@@ -539,6 +539,92 @@ def run_sweep(args):
 
 
 
+# ---------------------------------------------------------------------------------------------------
+# SD3 shape at token-group counts 1, 2, 4, 8 (the setting of Appendix A.1's kernel comparison):
+# per-op device times.  One JSON line; an extra mode, not the default.
+# ---------------------------------------------------------------------------------------------------
+def run_token_groups(args):
+    import torch
+    from paper_2607_23844_b200 import build
+    build.build()
+    from paper_2607_23844_b200 import omnicache as oc
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+
+    def graph_time_us(fn, reps):
+        fn(); torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        g.replay(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record(); torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / reps
+
+    base = inputs.sd3_token_cache()
+    C = base.shape[-1]
+    tensor_bytes = int(np.prod(base.shape)) * 2
+    ring = max(2, -(-4 * L2_BYTES // (3 * tensor_bytes)))
+    xs = [torch.from_numpy(base.x.view(np.int16)).to(dev) for _ in range(ring)]
+    caches = [torch.empty_like(xs[0]) for _ in range(ring)]
+    outs = [torch.empty_like(xs[0]) for _ in range(ring)]
+    reps = max(3, args.steps // 10)
+    results = []
+    for gy, gx in ((1, 1), (2, 1), (2, 2), (4, 2)):
+        L = oc.Layout(oc.KIND_TOKEN, inputs.BF16, *base.shape, gy=gy, gx=gx)
+        G, U, R = L.counts()
+        n_units, n_cand = G * U, G * (U - R)
+        n_reuse = (U - R) // 2
+        stride = U - n_reuse
+        rows = oc.rows_from_layout(L, C, 2)
+        row_bytes = rows.seg_bytes
+        ctx = oc.Context(0, oc.match_workspace_bytes(L))
+        sims = [torch.empty(n_units, dtype=torch.float32, device=dev) for _ in range(ring)]
+        idxs = [torch.empty(n_units, dtype=torch.int32, device=dev) for _ in range(ring)]
+        kept = [torch.empty(G * stride, dtype=torch.int32, device=dev) for _ in range(ring)]
+        cnt = [torch.empty(G, dtype=torch.int32, device=dev) for _ in range(ring)]
+        mm = [torch.empty(n_units, dtype=torch.int32, device=dev) for _ in range(ring)]
+        so = [torch.empty(n_units, dtype=torch.int32, device=dev) for _ in range(ring)]
+        ys = [torch.empty(G * stride * row_bytes, dtype=torch.uint8, device=dev) for _ in range(ring)]
+
+        def f_match():
+            for r in range(ring):
+                ctx.match(L, xs[r], sims[r], idxs[r], stream=torch.cuda.current_stream())
+
+        def f_select():
+            for r in range(ring):
+                ctx.select(L, sims[r], idxs[r], oc.SELECT_COUNT, 0.0, n_reuse, stride, kept[r], cnt[r], mm[r], so[r],
+                           stream=torch.cuda.current_stream())
+
+        def f_gather():
+            for r in range(ring):
+                ctx.gather(rows, xs[r], kept[r], G * stride, ys[r], stream=torch.cuda.current_stream())
+
+        def f_restore():
+            for r in range(ring):
+                ctx.restore(rows, ys[r], caches[r], n_units, so[r], mm[r], outs[r], stream=torch.cuda.current_stream())
+        t = {k: graph_time_us(f, reps) / ring for k, f in
+             (("match", f_match), ("select", f_select), ("gather", f_gather), ("restore", f_restore))}
+        flops = 2.0 * n_cand * R * C
+        results.append({
+            "token_groups": gy * gx, "grid": [gy, gx], "groups": G, "units_per_group": U, "n_reuse_per_group": n_reuse,
+            "match_us": t["match"], "select_us": t["select"], "gather_us": t["gather"], "restore_us": t["restore"],
+            "selection_plus_restoration_us": t["select"] + t["gather"] + t["restore"],
+            "summed_us": sum(t.values()), "match_TFLOP/s": flops / (t["match"] * 1e-6) / 1e12,
+            "gather_frac_hbm": 2 * G * stride * row_bytes / (t["gather"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
+            "restore_frac_hbm": 2 * n_units * row_bytes / (t["restore"] * 1e-6) / 1e9 / peaks["hbm_gbs"]})
+        assert ctx.device_status() == oc.OK
+        ctx.close()
+    print(json.dumps({"metric": "per-op device time, SD3 shape at token-group counts 1/2/4/8", "unit": "us",
+                      "timing": "CUDA-graph replay per op over a ring of buffers larger than 4x L2",
+                      "shape": list(base.shape), "data": "synthetic", "results": results}), flush=True)
+
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -558,9 +644,9 @@ def main():
     if args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     rank, local_rank, world = sharding.env_rank_world()
-    if args.workload == "svd_sweep":
+    if args.workload in ("svd_sweep", "sd3_groups"):
         if rank == 0:
-            run_sweep(args)
+            (run_sweep if args.workload == "svd_sweep" else run_token_groups)(args)
         return
     if args.impl == "reference":
         run_reference(args, rank)

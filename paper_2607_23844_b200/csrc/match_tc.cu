@@ -64,7 +64,8 @@ struct TcParams {
     int n_cand_lat;                      // sy*sx - 1
     int kblocks;
     int bwA_log2, bhA, n_wtA, n_tilesA;  // candidate box: (1 << bwA_log2) x bhA lattice points = 128 rows
-    int n_apairs;                        // candidate tiles are processed two at a time
+    int tpp;                             // candidate tiles per piece: 2 (M = 256), or 1 for small problems
+    int n_apairs;                        // tile rows per lattice member = ceil(n_tilesA / tpp)
     int bwQ_log2, bhQ, n_wq, n_quanta;   // quantum box:   (1 << bwQ_log2) x bhQ lattice points = 32 rows
     int pieces_per_row, total_items;     // a row = one pair of candidate tiles against all representatives
     int n_stages, stage_bytes;           // operand ring of this launch
@@ -265,19 +266,20 @@ match_tc_kernel(const __grid_constant__ TcParams P) {
         while (ok && walk.next(P, c)) {
             const CUtensorMap* map = &P.mapQ;
             int w, h;
-            if (lane < 2) {
+            if (lane < P.tpp) {
                 map = &P.mapsA[c.member];
-                const int ta = 2 * c.a_pair + lane;   // may lie past the lattice: the box is then masked
+                const int ta = P.tpp * c.a_pair + lane;   // may lie past the lattice: the box is then masked
                 const int htA = ta / P.n_wtA, wtA = ta - htA * P.n_wtA;
                 w = c.px * P.Ws + wtA * bwA; h = c.py * P.Hs + htA * P.bhA;
             } else {
-                const int qi = c.q0 + lane - 2;
+                const int qi = c.q0 + lane - P.tpp;
                 const int hq = qi / P.n_wq, wq = qi - hq * P.n_wq;
                 w = c.px * P.Ws + wq * bwQ; h = c.py * P.Hs + hq * P.bhQ;
             }
-            const bool active = lane < c.nq + 2;
-            const uint32_t dst_off = lane < 2 ? (uint32_t)(lane * A_BYTES) : (uint32_t)(2 * A_BYTES + (lane - 2) * Q_BYTES);
-            const uint32_t bytes = (uint32_t)(2 * A_BYTES + c.nq * Q_BYTES);
+            const bool active = lane < c.nq + P.tpp;
+            const uint32_t dst_off = lane < P.tpp ? (uint32_t)(lane * A_BYTES)
+                                                  : (uint32_t)(P.tpp * A_BYTES + (lane - P.tpp) * Q_BYTES);
+            const uint32_t bytes = (uint32_t)(P.tpp * A_BYTES + c.nq * Q_BYTES);
             for (int kb = 0; kb < P.kblocks; ++kb) {
                 const uint32_t full = bar_full + 8 * stage;
                 bool go = true;
@@ -325,12 +327,13 @@ match_tc_kernel(const __grid_constant__ TcParams P) {
                     const uint32_t a_addr = tiles_base + stage * STAGE_BYTES;
                     const uint64_t a0_desc = make_smem_desc(a_addr);
                     const uint64_t a1_desc = make_smem_desc(a_addr + A_BYTES);
-                    const uint64_t b_desc = make_smem_desc(a_addr + 2 * A_BYTES);
+                    const uint64_t b_desc = make_smem_desc(a_addr + P.tpp * A_BYTES);
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 16; ++k4) {            // UMMA K = 16: 32 bytes along the row
                         const uint32_t acc = (uint32_t)((kb | k4) != 0);
                         tc_mma_bf16(tmem_base, a0_desc + (uint64_t)(2 * k4), b_desc + (uint64_t)(2 * k4), idesc, acc);
-                        tc_mma_bf16(tmem_base + 256u, a1_desc + (uint64_t)(2 * k4), b_desc + (uint64_t)(2 * k4), idesc, acc);
+                        if (P.tpp == 2)
+                            tc_mma_bf16(tmem_base + 256u, a1_desc + (uint64_t)(2 * k4), b_desc + (uint64_t)(2 * k4), idesc, acc);
                     }
                     tc_commit(bar_empty + 8 * stage);                  // frees the stage when the MMAs retire
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -382,8 +385,8 @@ match_tc_kernel(const __grid_constant__ TcParams P) {
                 const int ch_split = (c.nq + 1) >> 1;
                 const int ch_begin = half ? ch_split : 0, ch_end = half ? c.nq : ch_split;
 #pragma unroll 1
-                for (int t = 0; t < 2; ++t) {                          // the two candidate tiles
-                    const int ta = 2 * c.a_pair + t;
+                for (int t = 0; t < P.tpp; ++t) {                      // the piece's candidate tiles
+                    const int ta = P.tpp * c.a_pair + t;
                     const int htA = ta / P.n_wtA, wtA = ta - htA * P.n_wtA;
                     const int hsA = htA * P.bhA + (row >> P.bwA_log2), wsA = wtA * bwA + (row & (bwA - 1));
                     const bool row_ok = hsA < P.Hs && wsA < P.Ws;
@@ -514,7 +517,7 @@ static EncodeTiledFn encode_fn() {
 static int pow2_ceil_log2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
 
 struct TcPlan {
-    int bwA_log2, bhA, n_wtA, n_tilesA, n_apairs, bwQ_log2, bhQ, n_wq, n_quanta;
+    int bwA_log2, bhA, n_wtA, n_tilesA, tpp, n_apairs, bwQ_log2, bhQ, n_wq, n_quanta;
     int pieces_per_row, qmax, n_stages, stage_bytes;
     long long rows, items;
 };
@@ -525,29 +528,37 @@ static TcPlan make_plan(const Geo& g, int sm_count) {
     p.bwA_log2 = la; p.bhA = BM >> la;
     p.n_wtA = (g.Ws + (1 << la) - 1) >> la;
     p.n_tilesA = p.n_wtA * ((g.Hs + p.bhA - 1) / p.bhA);
-    p.n_apairs = (p.n_tilesA + 1) / 2;
     int lq = pow2_ceil_log2(g.Ws); if ((1 << lq) > QN) lq = pow2_ceil_log2(QN);
     p.bwQ_log2 = lq; p.bhQ = QN >> lq;
     p.n_wq = (g.Ws + (1 << lq) - 1) >> lq;
     p.n_quanta = p.n_wq * ((g.Hs + p.bhQ - 1) / p.bhQ);
-    p.rows = g.n_groups * (long long)(g.sy * g.sx - 1) * p.n_apairs;
-    // Pieces per row: estimated cycles = waves x per-piece cycles.  Per 64-channel step a piece of q
-    // quanta fetches 32 + 4q KB at ~48 B/clk/SM (the measured L2 -> shared-memory feed) and needs
-    // 128q tensor cycles; its epilogue (~400 cycles per quantum for both tiles) is not overlapped.
+    // Tiles per piece (1 or 2) and pieces per row: estimated cycles = waves x per-piece cycles.  Per
+    // 64-channel step a piece fetches tpp*16 + 4q KB; the step takes the longest of: that fetch at
+    // ~48 B/clk/SM (measured L2 -> shared-memory feed), the fetch round trip (~3000 cycles) divided
+    // by the stages that fit in the ring, and tpp*64q tensor cycles.  The epilogue (~200 cycles per
+    // quantum and tile) is not overlapped.
     const int kblocks = (g.C + BK - 1) / BK;
-    double best_cost = 0; int best_P = 0;
-    for (int P = (p.n_quanta + MAXQ - 1) / MAXQ; P <= p.n_quanta; ++P) {
-        const int q = (p.n_quanta + P - 1) / P;
-        const long long items = p.rows * P;
-        const long long waves = (items + sm_count - 1) / sm_count;
-        const double fetch = (32.0 + 4.0 * q) * 1024.0 / 48.0, mma = 128.0 * q;
-        const double piece = kblocks * (fetch > mma ? fetch : mma) + 400.0 * q + 1500.0;
-        const double cost = waves * piece;
-        if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; }
+    double best_cost = 0; int best_P = 0, best_tpp = 2;
+    for (int tpp = 1; tpp <= 2; ++tpp) {
+        const long long rows = g.n_groups * (long long)(g.sy * g.sx - 1) * ((p.n_tilesA + tpp - 1) / tpp);
+        for (int P = (p.n_quanta + MAXQ - 1) / MAXQ; P <= p.n_quanta; ++P) {
+            const int q = (p.n_quanta + P - 1) / P;
+            const double stage_kb = tpp * 16.0 + 4.0 * q;
+            int stages = (int)(TILE_BYTES / 1024 / stage_kb); if (stages > MAX_STAGES) stages = MAX_STAGES;
+            const long long waves = (rows * P + sm_count - 1) / sm_count;
+            const double fetch = stage_kb * 1024.0 / 48.0, lat = 3000.0 / stages, mma = tpp * 64.0 * q;
+            double step = fetch > lat ? fetch : lat; if (mma > step) step = mma;
+            const double piece = kblocks * step + 200.0 * q * tpp + 1500.0;
+            const double cost = waves * piece;
+            if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; best_tpp = tpp; }
+        }
     }
+    p.tpp = best_tpp;
+    p.n_apairs = (p.n_tilesA + p.tpp - 1) / p.tpp;
+    p.rows = g.n_groups * (long long)(g.sy * g.sx - 1) * p.n_apairs;
     p.pieces_per_row = best_P;
     p.qmax = (p.n_quanta + best_P - 1) / best_P;
-    p.stage_bytes = 2 * A_BYTES + p.qmax * Q_BYTES;
+    p.stage_bytes = p.tpp * A_BYTES + p.qmax * Q_BYTES;
     p.n_stages = TILE_BYTES / p.stage_bytes;
     if (p.n_stages > MAX_STAGES) p.n_stages = MAX_STAGES;
     p.items = p.rows * p.pieces_per_row;
@@ -596,7 +607,7 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
     P.Hp = g.Hp; P.Wp = g.Wp; P.Hs = g.Hs; P.Ws = g.Ws;
     P.rep_member = rep_member; P.n_cand_lat = g.sy * g.sx - 1;
     P.kblocks = (g.C + BK - 1) / BK;
-    P.bwA_log2 = p.bwA_log2; P.bhA = p.bhA; P.n_wtA = p.n_wtA; P.n_tilesA = p.n_tilesA; P.n_apairs = p.n_apairs;
+    P.bwA_log2 = p.bwA_log2; P.bhA = p.bhA; P.n_wtA = p.n_wtA; P.n_tilesA = p.n_tilesA; P.tpp = p.tpp; P.n_apairs = p.n_apairs;
     P.bwQ_log2 = p.bwQ_log2; P.bhQ = p.bhQ; P.n_wq = p.n_wq; P.n_quanta = p.n_quanta;
     P.pieces_per_row = p.pieces_per_row; P.total_items = (int)p.items;
     P.n_stages = p.n_stages; P.stage_bytes = p.stage_bytes;
