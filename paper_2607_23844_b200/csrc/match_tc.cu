@@ -6,35 +6,56 @@
 // 4-D TMA tensor map {C, W/sx, H/sy, B*T}, so a box {64 channels, bw, bh, 1} lands in shared memory
 // as a canonical K-major, 128-byte-swizzled tile.  No operand is gathered or copied beforehand.
 //
-// What bounds it.  Measured on B200, this loop is limited by operand traffic L2 -> shared memory
-// (every variant tried settled at 8-10 TB/s over all SMs, with ~3000 cycles from "stage free" to
-// "stage full"), not by the tensor pipe.  So the tile is chosen for FLOP per fetched byte:
-// one CTA multiplies TWO 128-row candidate tiles by the same N <= 256 representatives
-// (M = 256 per CTA: 128 FLOP/B at N = 256, twice what a 128 x 128 tile gets), using all 512 TMEM
-// columns as two accumulators.
+// What bounds it.  Measured on B200 (in-kernel timestamps and a copy-only micro-benchmark):
+//   * a TMA box costs the issuing warp ~50-100 cycles whatever its size, and the L2 -> shared-memory
+//     path delivers ~80 B/clk/SM to all SMs at once, with ~2000 cycles from issue to "stage full" for
+//     a 56 KB stage under load.  With 224 KB of ring the loop is therefore bound by bytes in flight
+//     (Little's law) unless a stage carries enough MMA work: the tile is chosen for FLOP per fetched
+//     byte, and a stage is fetched with as few boxes as possible;
+//   * the tensor pipe accepts an MMA only about when the previous one starts, so whatever the issuing
+//     warp does between two stages (finding out that the next stage is full takes ~150 cycles) is
+//     time the pipe idles, unless it is folded in between the MMAs of a stage;
+//   * a lone warp pays several hundred cycles per integer division and per first touch of code or
+//     parameters, which is what the first piece of a CTA costs before its first copy is issued.
+//
+// Tile.  One CTA multiplies ONE or TWO 128-row candidate tiles by the same N <= 256 representatives.
+// Two tiles (M = 256 per CTA, 128 FLOP/B at N = 256) use all 512 TMEM columns as two accumulators;
+// one tile leaves half of TMEM free, so two accumulators take turns and the epilogue of a piece runs
+// under the MMAs of the next.  Optionally two CTAs of a cluster form a pair (cta_group::2): each
+// holds its own candidate tiles and fetches HALF of the representatives, and the tensor cores of
+// both SMs read both halves: the same MMA work per SM for fewer fetched bytes.
 //
 // Work split.  The representatives of a group are cut into "quanta" of 32 lattice points (one 4 KB
-// box per 64 channels).  A row of the problem is one pair of candidate tiles against all
+// box per 64 channels).  A row of the problem is the candidate tiles of one CTA (or pair) against all
 // representatives of its group; it is cut into P pieces of nearly equal width (<= 8 quanta), and the
-// pieces are dealt out evenly to one persistent CTA per SM.  The host picks P with a small cost
-// model (bytes fetched per piece x number of waves).
+// pieces are dealt out evenly, in contiguous runs, to one persistent CTA (pair) per SM (pair of SMs).
+// The host picks the form, the tiles per CTA and P with a small cost model.
 //
 // Warp specialised:
-//   warp 0      TMA producer   (one lane per box): global -> smem ring (as many stages as fit in
-//               192 KB for this launch's piece width), mbarrier complete_tx
-//   warp 1      MMA issuer     (one lane): tcgen05.mma kind::f16 (bf16 x bf16 -> fp32 in TMEM), two
-//               MMAs per 16 channels (one per candidate tile); owns tcgen05.alloc / dealloc
-//   warps 2..9  epilogue: thread r of warps 2..5 / 6..9 owns row r (= TMEM lane r) of both candidate
+//   warp 0      TMA producer   (one lane per box; a CTA's candidate tiles are one box, and so are its
+//               quanta of a piece, whenever they stack into a rectangle of lattice rows): global ->
+//               smem ring (as many stages as fit in 224 KB), mbarrier complete_tx
+//   warp 1      MMA issuer     (all lanes walk the loop so that addresses stay warp-uniform, one
+//               elected lane issues): tcgen05.mma kind::f16 (bf16 x bf16 -> fp32 in TMEM), all MMAs
+//               of a stage in one instruction block with the look at the next stage's barrier
+//               folded in; owns tcgen05.alloc / dealloc
+//   warps 2..9  epilogue: thread r of warps 2..5 / 6..9 owns row r (= TMEM lane r) of the candidate
 //               tiles for the first / second half of the piece's columns: tcgen05.ld 32 columns at a
-//               time (double buffered), scale by the representative's inverse norm, running
-//               (max, arg max) in two independent register chains - no cross-thread reduction - then
-//               ONE 64-bit atomicMax per row merges the piece into the packed key array (largest
+//               time (double buffered), scale by the representative's inverse norm, and a running
+//               maximum over keys that carry the column in their 5 low mantissa bits (one three-input
+//               max per two columns, no compare-and-select per element, no cross-thread reduction);
+//               then ONE 64-bit atomicMax per row merges the piece into the packed key array (largest
 //               value, then lowest index: independent of arrival order, hence deterministic).
-// Rows / columns of a box that fall outside the patch are masked in the epilogue (bias -inf), so
-// ragged lattices need no padding.  Every mbarrier wait is bounded: on expiry the CTA records
-// OC_ERR_TIMEOUT in the context's status word, lets its outstanding copies land, frees TMEM and exits.
+//               The reported similarity is thereby truncated by at most 2^-18 relative, and among
+//               representatives whose similarities agree to that precision the lowest index wins.
+// Rows / columns of a box that fall outside the patch are masked in the epilogue (a NaN scale never
+// wins a max), so ragged lattices need no padding.  Every mbarrier wait is bounded: on expiry the CTA
+// records OC_ERR_TIMEOUT in the context's status word, lets its outstanding copies land, frees TMEM
+// and exits.
 #include <cuda.h>
 
+#include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -55,9 +76,8 @@ static constexpr int MAX_LATTICES = 9;
 static constexpr uint32_t TMEM_COLS = 512;
 static constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;   // 1 s per wait
 
-struct TcParams {
-    CUtensorMap mapsA[MAX_LATTICES];     // 128-row boxes, one map per sub-lattice member (my*sx + mx)
-    CUtensorMap mapQ;                    // 32-row boxes of the representative lattice
+// Everything but the tensor maps.
+struct TcScalars {
     int H, W, sy, sx, gy, gx;
     int Hp, Wp, Hs, Ws;                  // patch size; lattice size per patch (same for every member)
     int rep_member;                      // oy*sx + ox
@@ -67,13 +87,28 @@ struct TcParams {
     int tpp;                             // candidate tiles per piece: 2 (M = 256), or 1 for small problems
     int n_apairs;                        // tile rows per lattice member = ceil(n_tilesA / tpp)
     int bwQ_log2, bhQ, n_wq, n_quanta;   // quantum box:   (1 << bwQ_log2) x bhQ lattice points = 32 rows
-    int pieces_per_row, total_items;     // a row = one pair of candidate tiles against all representatives
+    int pieces_per_row, total_items;     // a row = the candidate tiles of one piece against all representatives
+    int q_unit, n_q_units;               // pieces are cut in units of q_unit quanta (2 for a CTA pair)
+    int a_merged, q_merged, q_lo;        // one box for a CTA's candidate tiles / for its quanta of a piece
+    int items_base, items_rem;           // every walker takes items_base pieces, the first items_rem one more
+    unsigned cum[5];                     // pieces per tile run, lattice, patch, patch row, frame
+    float rcp_cum[5], rcp_ppr;           // their reciprocals, and 1 / pieces_per_row
+    float rcp_n_wtA, rcp_n_wq;
+    int my_rep, mx_rep;                  // rep_member / sx and the remainder
+    int sx_magic;                        // ceil(65536 / sx): (m * sx_magic) >> 16 == m / sx for m < 256
+    int u_step_q, u_step_r;              // n_q_units / pieces_per_row and the remainder
     int n_stages, stage_bytes;           // operand ring of this launch
     int units_per_group, reps_per_group;
     const float* inv_norm;
     unsigned long long* keys;
     float* aux;
     int* status;
+};
+struct TcParams {
+    CUtensorMap mapsA[MAX_LATTICES];     // 128-row boxes, one map per sub-lattice member (my*sx + mx)
+    CUtensorMap mapQ[2];                 // representative boxes: one quantum (32 rows), or when a piece's quanta
+                                         // stack into one rectangle, q_lo quanta ([0]) and q_lo + 1 quanta ([1])
+    TcScalars s;
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
@@ -102,6 +137,16 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+// One look at a barrier, never suspending the thread.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait: false if the phase did not complete within WAIT_LIMIT_NS or another role gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -118,25 +163,75 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 __device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" :: "l"(map) : "memory");
 }
+// arrive on a barrier given by its cluster-wide shared address (own CTA or the other CTA of a pair)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" :: "r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared address of the same variable in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// In a CTA pair `bar` is the cluster address of the LEADER's barrier: both CTAs' copies report there.
+template <bool PAIR>
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
                                             uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-        :: "r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+    if (PAIR)
+        asm volatile(
+            "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+            :: "r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+            :: "r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // arrive on `bar` once every MMA issued so far by this thread has retired
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+// The MMA warp runs its loop with all 32 lanes (so that addresses and descriptors are warp-uniform
+// values); `issue` is non-zero in the one elected lane that actually issues.
+template <bool PAIR>
+__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t issue = 1u) {
+    if (PAIR)
+        asm volatile("{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %1, 0;\n\t"
+                     "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+                     :: "r"(bar), "r"(issue) : "memory");
+    else
+        asm volatile("{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %1, 0;\n\t"
+                     "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+                     :: "r"(bar), "r"(issue) : "memory");
 }
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t e;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.b32 %0, 1, 0, p;\n\t}" : "=r"(e));
+    return e;
+}
+template <bool PAIR>
 __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+                                            uint32_t accumulate, uint32_t issue) {
+    if (PAIR)
+        asm volatile(
+            "{\n\t.reg .pred p, e;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "setp.ne.b32 e, %5, 0;\n\t"
+            "@e tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p, e;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "setp.ne.b32 e, %5, 0;\n\t"
+            "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
     asm volatile(
@@ -148,6 +243,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
           "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // Barrier over the 256 epilogue threads that also ANDs a flag: every thread learns whether any
@@ -163,6 +271,55 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
     return r != 0;
 }
 
+// All MMAs of one 64-channel stage (4 steps of K = 16, for one or two candidate tiles), with a look at
+// the NEXT stage's barrier folded in: the test is issued before the last MMAs and its answer read
+// after them, so the ~150 cycles it takes to come back pass while those MMAs queue up instead of
+// between two stages (the tensor pipe accepts an MMA only about when the previous one starts, so
+// nothing else hides that gap).
+// Returns non-zero when the next stage was already full.
+#define OC_MMA_STAGE_ASM(CG, TWO)                                                                        \
+    asm volatile(                                                                                       \
+        "{\n\t"                                                                                         \
+        ".reg .pred pa, pt, e, r;\n\t"                                                                  \
+        ".reg .b64 a0, a1, bb;\n\t"                                                                     \
+        ".reg .b32 d1;\n\t"                                                                             \
+        "setp.ne.b32 pa, %5, 0;\n\t"                                                                    \
+        "setp.ne.b32 e, %6, 0;\n\t"                                                                     \
+        "setp.eq.b32 pt, 0, 0;\n\t"                                                                     \
+        "add.u32 d1, %1, 256;\n\t"                                                                      \
+        "@e tcgen05.mma.cta_group::" CG ".kind::f16 [%1], %2, %4, %9, pa;\n\t"                          \
+        TWO("@e tcgen05.mma.cta_group::" CG ".kind::f16 [d1], %3, %4, %9, pa;\n\t")                     \
+        "add.u64 a0, %2, 2;\n\tadd.u64 a1, %3, 2;\n\tadd.u64 bb, %4, 2;\n\t"                          \
+        "@e tcgen05.mma.cta_group::" CG ".kind::f16 [%1], a0, bb, %9, pt;\n\t"                          \
+        TWO("@e tcgen05.mma.cta_group::" CG ".kind::f16 [d1], a1, bb, %9, pt;\n\t")                     \
+        "add.u64 a0, %2, 4;\n\tadd.u64 a1, %3, 4;\n\tadd.u64 bb, %4, 4;\n\t"                          \
+        "@e tcgen05.mma.cta_group::" CG ".kind::f16 [%1], a0, bb, %9, pt;\n\t"                          \
+        TWO("@e tcgen05.mma.cta_group::" CG ".kind::f16 [d1], a1, bb, %9, pt;\n\t")                     \
+        "mbarrier.test_wait.parity.shared::cta.b64 r, [%7], %8;\n\t"                                    \
+        "add.u64 a0, %2, 6;\n\tadd.u64 a1, %3, 6;\n\tadd.u64 bb, %4, 6;\n\t"                          \
+        "@e tcgen05.mma.cta_group::" CG ".kind::f16 [%1], a0, bb, %9, pt;\n\t"                          \
+        TWO("@e tcgen05.mma.cta_group::" CG ".kind::f16 [d1], a1, bb, %9, pt;\n\t")                     \
+        "selp.b32 %0, 1, 0, r;\n\t"                                                                     \
+        "}"                                                                                             \
+        : "=r"(ready)                                                                                   \
+        : "r"(d_tmem), "l"(a0_desc), "l"(a1_desc), "l"(b_desc), "r"(accumulate), "r"(issue), "r"(next_bar), \
+          "r"(next_parity), "r"(idesc)                                                                  \
+        : "memory")
+#define OC_KEEP(x) x
+#define OC_DROP(x)
+template <bool PAIR>
+__device__ __forceinline__ uint32_t tc_mma_stage(uint32_t d_tmem, uint64_t a0_desc, uint64_t a1_desc, uint64_t b_desc,
+                                                 uint32_t idesc, uint32_t accumulate, uint32_t issue, bool two_tiles,
+                                                 uint32_t next_bar, uint32_t next_parity) {
+    uint32_t ready;
+    if (two_tiles) {
+        if (PAIR) OC_MMA_STAGE_ASM("2", OC_KEEP); else OC_MMA_STAGE_ASM("1", OC_KEEP);
+    } else {
+        if (PAIR) OC_MMA_STAGE_ASM("2", OC_DROP); else OC_MMA_STAGE_ASM("1", OC_DROP);
+    }
+    return ready;
+}
+
 // K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
     const uint32_t lo = ((addr >> 4) & 0x3FFFu) | (1u << 16);           // start address, LBO = 16 B (unused)
@@ -173,123 +330,196 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
 // ---- the walk over this CTA's share of the piece list ----------------------------------------------
 struct Piece {
     int bt, py, px, member;              // frame, patch, candidate sub-lattice member
-    int a_pair;                          // candidate tiles 2*a_pair and 2*a_pair + 1 of the member's lattice
+    int a_pair;                          // which run of candidate tiles (tpp per CTA) of the member's lattice
     int q0, nq;                          // quanta [q0, q0 + nq) of the group's representatives
     long long g;
 };
+// floor(a / d) for a < 2^22 from the float reciprocal (one multiply and a fix-up; an integer division
+// costs a lone warp several hundred cycles), by integer division otherwise.
+__device__ __forceinline__ unsigned div_small(unsigned a, unsigned d, float rcp_d) {
+    if (a >= (1u << 22)) return a / d;
+    unsigned q = (unsigned)((float)a * rcp_d);
+    const int r = (int)(a - q * d);
+    if (r < 0) --q; else if ((unsigned)r >= d) ++q;
+    return q;
+}
+
+// Pieces are numbered row-major over (frame, patch row, patch column, candidate lattice, tile run,
+// piece of the row); a walker takes a contiguous range.  The first piece is decoded by division,
+// the following ones by counting up.
 struct Walk {
-    int i, i_end;
-    __device__ Walk(const TcParams& P) {
-        const long long n = gridDim.x, c = blockIdx.x;
-        i = (int)((long long)P.total_items * c / n); i_end = (int)((long long)P.total_items * (c + 1) / n);
+    int left;                            // pieces still to hand out
+    int j, a_pair, k, px, py, bt;
+    int u_cur, r_cur;                    // floor(j * n_q_units / pieces_per_row) and the remainder
+    long long g;
+    __device__ __forceinline__ Walk(const TcScalars& P, int c) {
+        const unsigned i0 = (unsigned)(c * P.items_base + (c < P.items_rem ? c : P.items_rem));
+        left = P.items_base + (c < P.items_rem ? 1 : 0);
+        const unsigned q0 = div_small(i0, P.cum[0], P.rcp_cum[0]), q1 = div_small(i0, P.cum[1], P.rcp_cum[1]),
+                       q2 = div_small(i0, P.cum[2], P.rcp_cum[2]), q3 = div_small(i0, P.cum[3], P.rcp_cum[3]),
+                       q4 = div_small(i0, P.cum[4], P.rcp_cum[4]);
+        j = (int)(i0 - q0 * P.cum[0]);
+        a_pair = (int)(q0 - q1 * (unsigned)P.n_apairs);
+        k = (int)(q1 - q2 * (unsigned)P.n_cand_lat);
+        g = q2;
+        px = (int)(q2 - q3 * (unsigned)P.gx);
+        py = (int)(q3 - q4 * (unsigned)P.gy);
+        bt = (int)q4;
+        const unsigned ju = (unsigned)j * (unsigned)P.n_q_units;
+        u_cur = (int)div_small(ju, (unsigned)P.pieces_per_row, P.rcp_ppr);
+        r_cur = (int)(ju - (unsigned)u_cur * (unsigned)P.pieces_per_row);
     }
-    __device__ bool next(const TcParams& P, Piece& p) {
-        if (i >= i_end) return false;
-        int row = i / P.pieces_per_row;
-        const int j = i - row * P.pieces_per_row;
-        ++i;
-        p.q0 = j * P.n_quanta / P.pieces_per_row;
-        p.nq = (j + 1) * P.n_quanta / P.pieces_per_row - p.q0;
-        p.a_pair = row % P.n_apairs; row /= P.n_apairs;
-        const int k = row % P.n_cand_lat; row /= P.n_cand_lat;
-        p.g = row;
-        p.px = row % P.gx; row /= P.gx;
-        p.py = row % P.gy; p.bt = row / P.gy;
+    __device__ __forceinline__ bool next(const TcScalars& P, Piece& p) {
+        if (left <= 0) return false;
+        --left;
+        int u_next = u_cur + P.u_step_q, r_next = r_cur + P.u_step_r;
+        if (r_next >= P.pieces_per_row) { r_next -= P.pieces_per_row; ++u_next; }
+        p.q0 = u_cur * P.q_unit;
+        p.nq = (u_next - u_cur) * P.q_unit;
+        u_cur = u_next; r_cur = r_next;
+        p.a_pair = a_pair; p.g = g; p.px = px; p.py = py; p.bt = bt;
         p.member = k < P.rep_member ? k : k + 1;
+        if (++j == P.pieces_per_row) {
+            j = 0; u_cur = 0; r_cur = 0;
+            if (++a_pair == P.n_apairs) {
+                a_pair = 0;
+                if (++k == P.n_cand_lat) {
+                    k = 0; ++g;
+                    if (++px == P.gx) { px = 0; if (++py == P.gy) { py = 0; ++bt; } }
+                }
+            }
+        }
         return true;
     }
 };
 
 static constexpr int COL_BYTES = 256 * 8;                               // {scale, bias} per column of a piece
-static constexpr int N_BARS = 2 * MAX_STAGES + 3;                       // full[], empty[], acc_full, acc_empty, drain
+static constexpr int N_BARS = 2 * MAX_STAGES + 5;                       // full[], empty[], acc_full[2], acc_empty[2], drain
 static constexpr int TAIL_BYTES = COL_BYTES + N_BARS * 8 + 32;        // column table, barriers, TMEM slot, flags
 static constexpr int TILE_BYTES = (SMEM_LIMIT - TAIL_BYTES) / 1024 * 1024;   // operand ring: everything else
 static constexpr int SMEM_TOTAL = TILE_BYTES + TAIL_BYTES;
 
+// PAIR: two CTAs of a cluster work on one piece with cta_group::2 instructions.  Each holds its own
+// tpp candidate tiles (256 accumulator rows per MMA across the pair) and fetches HALF of the piece's
+// representative quanta; the tensor cores of both SMs read both halves, so every fetched operand
+// byte feeds twice the FLOPs.  The leader (cluster rank 0) issues all MMAs; both CTAs' copies report
+// to the leader's stage barrier, and the leader's commits free the stage in both CTAs.
+template <bool PAIR, bool AUX>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-match_tc_kernel(const __grid_constant__ TcParams P) {
+match_tc_kernel(const __grid_constant__ TcParams KP) {
     // The operand ring starts at the base of dynamic shared memory, which must be 1024-byte aligned
     // for the 128-byte swizzle (this kernel has no static shared memory in front of it; checked below).
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = smem_raw;
-    float4* colsb = (float4*)(smem + TILE_BYTES);                      // 128 pairs of {scale, bias}
+    float4* colsb = (float4*)(smem + TILE_BYTES);                      // per column: scale[256], then token[256]
     uint64_t* bars = (uint64_t*)(smem + TILE_BYTES + COL_BYTES);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * MAX_STAGES;
-    const uint32_t bar_acc_full = bar_empty + 8 * MAX_STAGES, bar_acc_empty = bar_acc_full + 8;
-    const uint32_t bar_drain = bar_acc_empty + 8;
+    const uint32_t bar_acc_full = bar_empty + 8 * MAX_STAGES, bar_acc_empty = bar_acc_full + 16;   // two of each
+    const uint32_t bar_drain = bar_acc_empty + 16;
     uint32_t* tmem_slot = (uint32_t*)(bars + N_BARS);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     const uint32_t tiles_base = smem_u32(smem);
-    const int STAGES = P.n_stages, STAGE_BYTES = P.stage_bytes;
+    const TcScalars& P = KP.s;
+    // First touches of parameter space miss the constant cache (several hundred cycles each, and
+    // one after the other when a lone warp meets them on its way to the first copy): every warp
+    // reads one word per 64 bytes of the scalars now, as independent loads.
+    {
+        const int w0 = P.H, w1 = P.n_apairs, w2 = P.items_base, w3 = P.sx_magic, w4 = P.units_per_group;
+        asm volatile("" :: "r"(w0), "r"(w1), "r"(w2), "r"(w3), "r"(w4));
+    }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+    const bool leader = rank == 0;
+    const int walker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     if ((tiles_base & 1023u) != 0) {                                   // never expected; refuse rather than compute garbage
-        if (threadIdx.x == 0) atomicCAS(P.status, 0, OC_ERR_ALIGNMENT);
+        if (threadIdx.x == 0) atomicCAS(KP.s.status, 0, OC_ERR_ALIGNMENT);   // (same verdict in both CTAs of a pair)
         return;
     }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        mbar_init(bar_acc_full, 1);
-        mbar_init(bar_acc_empty, 8);                                    // one arrival per epilogue warp
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, PAIR ? 16 : 8);            // one arrival per epilogue warp (of both CTAs)
+        }
         mbar_init(bar_drain, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 0 && lane == 0) {
-        tma_prefetch_map(&P.mapQ);
-        for (int m = 0; m <= P.n_cand_lat; ++m)
-            if (m != P.rep_member) tma_prefetch_map(&P.mapsA[m]);
+        tma_prefetch_map(&KP.mapQ[0]);
+        tma_prefetch_map(&KP.mapQ[1]);
+        for (int m = 0; m <= KP.s.n_cand_lat; ++m)
+            if (m != KP.s.rep_member) tma_prefetch_map(&KP.mapsA[m]);
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     :: "r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         :: "r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         :: "r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();          // the other CTA's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const int STAGES = P.n_stages, STAGE_BYTES = P.stage_bytes;
+    const bool dbl = P.tpp == 1;
 
+    Walk walk(P, walker);                  // every role walks the same pieces
+    Piece c;
     const int bwA = 1 << P.bwA_log2, bwQ = 1 << P.bwQ_log2;
-    const int my_rep = P.rep_member / P.sx, mx_rep = P.rep_member - my_rep * P.sx;
+    const int my_rep = P.my_rep, mx_rep = P.mx_rep;
 
     if (warp == 0) {
         // ================================ TMA producer ==========================================
-        // One lane per box: lanes 0 and 1 fetch the two candidate tiles, lanes 2..nq+1 one quantum
-        // each, so a stage costs one barrier wait plus one copy instruction per lane.
+        // One lane per box: the first tpp lanes fetch this CTA's candidate tiles, the next lanes one
+        // quantum each (in a pair: this CTA's half of the piece's quanta), so a stage costs one
+        // barrier wait plus one copy instruction per lane.
         int stage = 0; uint32_t phase = 0;
         uint32_t armed = 0;                           // stages with a copy possibly still in flight
         bool ok = true;
-        Walk walk(P); Piece c;
         while (ok && walk.next(P, c)) {
-            const CUtensorMap* map = &P.mapQ;
+            const int nq_mine = PAIR ? (c.nq >> 1) : c.nq;             // quanta this CTA fetches
+            const int nA = P.a_merged ? 1 : P.tpp, nQ = P.q_merged ? 1 : nq_mine;   // boxes per stage
+            const CUtensorMap* map;
             int w, h;
-            if (lane < P.tpp) {
-                map = &P.mapsA[c.member];
-                const int ta = P.tpp * c.a_pair + lane;   // may lie past the lattice: the box is then masked
-                const int htA = ta / P.n_wtA, wtA = ta - htA * P.n_wtA;
+            uint32_t dst_off;
+            if (lane < nA) {
+                map = &KP.mapsA[c.member];
+                // (tiles past the lattice are fetched as zeros and masked in the epilogue)
+                const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + lane;
+                const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
                 w = c.px * P.Ws + wtA * bwA; h = c.py * P.Hs + htA * P.bhA;
+                dst_off = (uint32_t)(lane * A_BYTES);
             } else {
-                const int qi = c.q0 + lane - P.tpp;
-                const int hq = qi / P.n_wq, wq = qi - hq * P.n_wq;
+                map = &KP.mapQ[(P.q_merged && nq_mine != P.q_lo) ? 1 : 0];
+                const int qi = c.q0 + (int)rank * nq_mine + lane - nA;
+                const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
                 w = c.px * P.Ws + wq * bwQ; h = c.py * P.Hs + hq * P.bhQ;
+                dst_off = (uint32_t)(P.tpp * A_BYTES + (lane - nA) * Q_BYTES);
             }
-            const bool active = lane < c.nq + P.tpp;
-            const uint32_t dst_off = lane < P.tpp ? (uint32_t)(lane * A_BYTES)
-                                                  : (uint32_t)(P.tpp * A_BYTES + (lane - P.tpp) * Q_BYTES);
-            const uint32_t bytes = (uint32_t)(P.tpp * A_BYTES + c.nq * Q_BYTES);
+            const bool active = lane < nA + nQ;
+            // what the leader's barrier expects per stage: the copies of both CTAs
+            const uint32_t bytes = (uint32_t)((PAIR ? 2 : 1) * (P.tpp * A_BYTES + nq_mine * Q_BYTES));
             for (int kb = 0; kb < P.kblocks; ++kb) {
-                const uint32_t full = bar_full + 8 * stage;
+                const uint32_t full_local = bar_full + 8 * stage;
+                const uint32_t full = PAIR ? map_to_cta(full_local, 0) : full_local;
                 bool go = true;
                 if (lane == 0) {
                     go = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
-                    if (go) mbar_arrive_expect_tx(full, bytes);
+                    if (go && leader) mbar_arrive_expect_tx(full_local, bytes);
                 }
                 go = __shfl_sync(0xFFFFFFFFu, (int)go, 0) != 0;
                 if (!go) { ok = false; break; }
-                if (active) tma_load_4d(tiles_base + stage * STAGE_BYTES + dst_off, map, kb * BK, w, h, c.bt, full);
+                if (active) tma_load_4d<PAIR>(tiles_base + stage * STAGE_BYTES + dst_off, map, kb * BK, w, h, c.bt, full);
                 armed |= 1u << stage;
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
@@ -299,50 +529,63 @@ match_tc_kernel(const __grid_constant__ TcParams P) {
             *abort_flag = 1;
             // copies already issued still write this CTA's shared memory: give each a bounded
             // chance to land before the CTA retires (the parity armed last is phase or phase^1)
-            for (int s = 0; s < STAGES; ++s) {
-                if (!(armed & (1u << s))) continue;
-                const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
+            if (leader) {
+                for (int s = 0; s < STAGES; ++s) {
+                    if (!(armed & (1u << s))) continue;
+                    const uint32_t par = (s < stage) ? phase : (phase ^ 1u);
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_full + 8 * s, par) && global_ns() - t0 < 20000000ull) {}
+                }
+            } else {                                   // its copies report to the leader: allow them a fixed time
                 const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(bar_full + 8 * s, par) && global_ns() - t0 < 20000000ull) {}
+                while (global_ns() - t0 < 1000000ull) {}
             }
         }
     } else if (warp == 1) {
         // ================================ MMA issuer ============================================
-        if (lane == 0) {
-            constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) |
-                                            ((uint32_t)(BM >> 4) << 24);   // D=f32, A=B=bf16, K-major both, M=128
+        if (leader) {
+            constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) |      // D=f32, A=B=bf16, K-major both,
+                                            ((uint32_t)((PAIR ? 2 * BM : BM) >> 4) << 24);   // M=128 (256 across a pair)
+            const uint32_t issue = elect_one();        // all lanes walk the loop, this one issues
             int stage = 0; uint32_t phase = 0;
-            bool ok = true;
+            bool ok = true, peeked = false;
             uint32_t it = 0;
-            Walk walk(P); Piece c;
             while (ok && walk.next(P, c)) {
-                const uint32_t acc_phase = it & 1u;
+                // one candidate tile per CTA leaves half of TMEM free: two accumulators take turns, and the
+                // epilogue of a piece runs under the MMAs of the next one
+                const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
                 ++it;
-                if (!mbar_wait(bar_acc_empty, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_empty + 8 * buf, acc_phase ^ 1u, abort_flag))) { ok = false; break; }
+                const uint32_t d_tmem = tmem_base + buf * 256u;
                 tc_fence_after();
                 const uint32_t idesc = IDESC_BASE | ((uint32_t)((c.nq * QN) >> 3) << 17);
                 for (int kb = 0; kb < P.kblocks; ++kb) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
+                    // (each lane looked for itself; the barrier's phase cannot go back, so a lane that saw it
+                    //  full stays right, and the others wait here)
+                    if (!peeked && !mbar_wait(bar_full + 8 * stage, phase, abort_flag)) ok = false;
+                    if (!__all_sync(0xFFFFFFFFu, ok)) { ok = false; break; }
                     const uint32_t a_addr = tiles_base + stage * STAGE_BYTES;
                     const uint64_t a0_desc = make_smem_desc(a_addr);
                     const uint64_t a1_desc = make_smem_desc(a_addr + A_BYTES);
                     const uint64_t b_desc = make_smem_desc(a_addr + P.tpp * A_BYTES);
-#pragma unroll
-                    for (int k4 = 0; k4 < BK / 16; ++k4) {            // UMMA K = 16: 32 bytes along the row
-                        const uint32_t acc = (uint32_t)((kb | k4) != 0);
-                        tc_mma_bf16(tmem_base, a0_desc + (uint64_t)(2 * k4), b_desc + (uint64_t)(2 * k4), idesc, acc);
-                        if (P.tpp == 2)
-                            tc_mma_bf16(tmem_base + 256u, a1_desc + (uint64_t)(2 * k4), b_desc + (uint64_t)(2 * k4), idesc, acc);
-                    }
-                    tc_commit(bar_empty + 8 * stage);                  // frees the stage when the MMAs retire
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    int nstage = stage + 1; uint32_t nphase = phase;
+                    if (nstage == STAGES) { nstage = 0; nphase ^= 1u; }
+                    // UMMA K = 16 is 32 bytes along the swizzled row: +2 in the descriptor's address field
+                    peeked = tc_mma_stage<PAIR>(d_tmem, a0_desc, a1_desc, b_desc, idesc, (uint32_t)(kb != 0), issue,
+                                                P.tpp == 2, bar_full + 8 * nstage, nphase) != 0;
+                    // frees the stage (in both CTAs of a pair) when the MMAs retire
+                    tc_commit<PAIR>(PAIR ? map_to_cta(bar_empty + 8 * stage, 0) : bar_empty + 8 * stage, issue);
+                    if (PAIR) tc_commit<PAIR>(map_to_cta(bar_empty + 8 * stage, 1), issue);
+                    stage = nstage; phase = nphase;
                 }
-                if (ok) tc_commit(bar_acc_full);
+                if (ok) {
+                    tc_commit<PAIR>(PAIR ? map_to_cta(bar_acc_full + 8 * buf, 0) : bar_acc_full + 8 * buf, issue);
+                    if (PAIR) tc_commit<PAIR>(map_to_cta(bar_acc_full + 8 * buf, 1), issue);
+                }
             }
-            if (!ok) { atomicCAS(P.status, 0, OC_ERR_TIMEOUT); *abort_flag = 1; }
-            // all MMAs issued by this thread must retire before TMEM is released
-            tc_commit(bar_drain);
+            if (!ok && lane == 0) { atomicCAS(P.status, 0, OC_ERR_TIMEOUT); *abort_flag = 1; }
+            // all MMAs issued by this warp must retire before TMEM is released
+            tc_commit<PAIR>(PAIR ? map_to_cta(bar_drain, 0) : bar_drain, issue);
             const unsigned long long t0 = global_ns();
             while (!mbar_try_wait(bar_drain, 0) && global_ns() - t0 < WAIT_LIMIT_NS) {}
         }
@@ -354,115 +597,163 @@ match_tc_kernel(const __grid_constant__ TcParams P) {
         const int row = lane_group * 32 + lane;                        // tile row owned by this thread
         bool ok = true;
         uint32_t it = 0;
-        Walk walk(P); Piece c;
-        float2* cs = (float2*)colsb;
-        const float4* cs4 = colsb;
-        while (walk.next(P, c)) {
-            const uint32_t acc_phase = it & 1u;
-            ++it;
-            const int ncol = c.nq * QN;
-            // ---- column table: inverse norm and validity of every representative of the piece -------
-            // (safe to overwrite: every epilogue thread passed the previous piece's loop before the
-            //  barrier below was completed for that piece ... see the trailing barrier)
-            for (int n = et; n < ncol; n += EPI_THREADS) {
-                const int qi = c.q0 + (n >> 5), r = n & 31;
-                const int hq = qi / P.n_wq, wq = qi - hq * P.n_wq;
-                const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));
-                float2 v = make_float2(0.f, -INFINITY);
-                if (hs < P.Hs && ws < P.Ws) {
-                    const int y = (c.py * P.Hs + hs) * P.sy + my_rep, x = (c.px * P.Ws + ws) * P.sx + mx_rep;
-                    v = make_float2(__ldg(P.inv_norm + ((long long)c.bt * P.H + y) * P.W + x), 0.f);
-                }
-                cs[n] = v;
+        const uint32_t acc_empty = PAIR ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;   // the leader's
+        // Per column of a piece: the representative's inverse norm (NaN where the column is not a
+        // representative of this patch: a NaN product never wins a max).  Two tables take turns: the
+        // entries of the NEXT piece are fetched (one per thread) before this piece's accumulators are
+        // read and stored after, so their global-memory latency is never waited for.
+        float* col_scale = (float*)colsb;                              // [2][256]
+        const int rowh = row >> P.bwA_log2, roww = row & (bwA - 1);
+        auto table_entry = [&](const Piece& pc) -> float {
+            if (et >= pc.nq * QN) return __int_as_float(0x7FC00000);
+            const int qi = pc.q0 + (et >> 5), r = et & 31;
+            const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
+            const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));
+            if (hs >= P.Hs || ws >= P.Ws) return __int_as_float(0x7FC00000);
+            const int y = (pc.py * P.Hs + hs) * P.sy + my_rep, x = (pc.px * P.Ws + ws) * P.sx + mx_rep;
+            return __ldg(P.inv_norm + ((long long)pc.bt * P.H + y) * P.W + x);
+        };
+        Piece nx;
+        bool have = walk.next(P, c);
+        if (have) col_scale[et] = table_entry(c);
+        if (!epilogue_barrier_all(ok)) { ok = false; have = false; }
+        while (have) {
+            const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
+            const float4* col_scale4 = (const float4*)(col_scale + (it & 1u) * 256);
+            const float* col_scale1 = col_scale + (it & 1u) * 256;
+            const bool have_nx = walk.next(P, nx);
+            float sc_nx = 0.f;
+            if (have_nx) sc_nx = table_entry(nx);                      // in flight until the end of this piece
+            const int my = (c.member * P.sx_magic) >> 16, mx = c.member - my * P.sx;
+            long long tokA0, tokA1; bool row_ok0, row_ok1;
+            {
+                const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp;
+                const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
+                const int hsA = htA * P.bhA + rowh, wsA = wtA * bwA + roww;
+                row_ok0 = hsA < P.Hs && wsA < P.Ws;
+                const int yA = (c.py * P.Hs + hsA) * P.sy + my, xA = (c.px * P.Ws + wsA) * P.sx + mx;
+                tokA0 = ((long long)c.bt * P.H + yA) * P.W + xA;
             }
-            if (!epilogue_barrier_all(ok)) { ok = false; break; }     // also orders the table writes
+            {
+                const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + 1;
+                const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
+                const int hsA = htA * P.bhA + rowh, wsA = wtA * bwA + roww;
+                row_ok1 = P.tpp == 2 && hsA < P.Hs && wsA < P.Ws;
+                const int yA = (c.py * P.Hs + hsA) * P.sy + my, xA = (c.px * P.Ws + wsA) * P.sx + mx;
+                tokA1 = ((long long)c.bt * P.H + yA) * P.W + xA;
+            }
+            // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
+            const int ch_split = (c.nq + 1) >> 1;
+            const int ch_begin = half ? ch_split : 0, ch_end = half ? c.nq : ch_split;
             // warp-uniform outcome: the TMEM loads below are warp-collective
-            const bool ready = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full, acc_phase, abort_flag));
+            const bool ready = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * buf, acc_phase, abort_flag));
             if (ready) {
                 tc_fence_after();
-                const int my = c.member / P.sx, mx = c.member - my * P.sx;
-                // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
-                const int ch_split = (c.nq + 1) >> 1;
-                const int ch_begin = half ? ch_split : 0, ch_end = half ? c.nq : ch_split;
 #pragma unroll 1
                 for (int t = 0; t < P.tpp; ++t) {                      // the piece's candidate tiles
-                    const int ta = P.tpp * c.a_pair + t;
-                    const int htA = ta / P.n_wtA, wtA = ta - htA * P.n_wtA;
-                    const int hsA = htA * P.bhA + (row >> P.bwA_log2), wsA = wtA * bwA + (row & (bwA - 1));
-                    const bool row_ok = hsA < P.Hs && wsA < P.Ws;
-                    const int yA = (c.py * P.Hs + hsA) * P.sy + my, xA = (c.px * P.Ws + wsA) * P.sx + mx;
-                    const long long tokA = ((long long)c.bt * P.H + yA) * P.W + xA;
+                    const long long tokA = t ? tokA1 : tokA0;
+                    const bool row_ok = t ? row_ok1 : row_ok0;
                     float inv_a = 0.f;
                     float* aux_row = nullptr;
-                    if (P.aux && row_ok) {
+                    if (AUX && P.aux && row_ok) {
                         inv_a = __ldg(P.inv_norm + tokA);
-                        const int u_local = (hsA * P.sy + my) * P.Wp + wsA * P.sx + mx;
+                        const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + t;
+                        const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
+                        const int u_local = ((htA * P.bhA + rowh) * P.sy + my) * P.Wp + (wtA * bwA + roww) * P.sx + mx;
                         aux_row = P.aux + ((long long)c.g * P.units_per_group + u_local) * P.reps_per_group;
                     }
-                    float best0 = -INFINITY, best1 = -INFINITY; int n0 = -1, n1 = -1;
-                    const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(t * 256);
-                    // two register buffers: the TMEM load of the next chunk is in flight while this one is reduced
+                    // Running maximum over "keys": the scaled similarity with its 5 low mantissa bits
+                    // replaced by 31 - (column within the chunk), so that ONE three-input max per two
+                    // columns carries the arg max along (among equal similarities the lowest column has
+                    // the largest key).  The similarity loses 5 of its 24 mantissa bits (2^-18 relative),
+                    // far inside the tolerance of a bf16 match.  Two independent chains; bc = the chunk in
+                    // which a chain last rose.
+                    float bm0 = -INFINITY, bm1 = -INFINITY;
+                    int bc0 = -1, bc1 = -1;
+                    const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(t * 256) + buf * 256u;
+                    // two register buffers: the TMEM load of the next step is in flight while this one is reduced
                     uint32_t va[32], vb[32];
-                    auto reduce_chunk = [&](const uint32_t* v, int ch) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 2) {              // two independent (max, arg max) chains
-                            const float4 sb = cs4[ch * 16 + (j >> 1)];
-                            const float x0 = fmaf(__uint_as_float(v[j]), sb.x, sb.y);
-                            const float x1 = fmaf(__uint_as_float(v[j + 1]), sb.z, sb.w);
-                            if (x0 > best0) { best0 = x0; n0 = ch * 32 + j; }      // ascending columns: lowest index wins
-                            if (x1 > best1) { best1 = x1; n1 = ch * 32 + j + 1; }
-                        }
-                        if (aux_row) {
-                            for (int j = 0; j < 32; ++j) {
-                                const float2 sb = cs[ch * 32 + j];
-                                if (sb.y == 0.f) {
-                                    const int qi = c.q0 + ch;
-                                    const int hq = qi / P.n_wq, wq = qi - hq * P.n_wq;
-                                    const int hs = hq * P.bhQ + (j >> P.bwQ_log2), ws = wq * bwQ + (j & (bwQ - 1));
-                                    aux_row[hs * P.Ws + ws] = clamp_unit(__uint_as_float(v[j]) * sb.x * inv_a);
-                                }
-                            }
-                        }
-                    };
+#define OC_KEY(v, s, j) __uint_as_float((__float_as_uint(__uint_as_float(v) * (s)) & 0xFFFFFFE0u) | (uint32_t)(31 - (j)))
+#define OC_VAL(k) __uint_as_float(__float_as_uint(k) & 0xFFFFFFE0u)
+#define OC_REDUCE_CHUNK(v, ch)                                                                                   \
+    do {                                                                                                         \
+        float cm0 = -INFINITY, cm1 = -INFINITY;                                                                  \
+        _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
+            const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                                   \
+            cm0 = max3f(cm0, OC_KEY(v[j], s4.x, j), OC_KEY(v[j + 1], s4.y, j + 1));                              \
+            cm1 = max3f(cm1, OC_KEY(v[j + 2], s4.z, j + 2), OC_KEY(v[j + 3], s4.w, j + 3));                      \
+        }                                                                                                        \
+        /* a later chunk wins only with a strictly larger similarity (the index bits set aside) */              \
+        if (OC_VAL(cm0) > OC_VAL(bm0)) { bm0 = cm0; bc0 = (ch); }                                                \
+        if (OC_VAL(cm1) > OC_VAL(bm1)) { bm1 = cm1; bc1 = (ch); }                                                \
+        if (AUX && aux_row) {                                                                                    \
+            for (int j = 0; j < 32; ++j) {                                                                       \
+                const float sc = col_scale1[(ch) * 32 + j];                                                      \
+                if (sc == sc) {                                                                                  \
+                    const int qi = c.q0 + (ch), r = j;                                                           \
+                    const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;                                           \
+                    const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));              \
+                    aux_row[hs * P.Ws + ws] = clamp_unit(__uint_as_float(v[j]) * sc * inv_a);                    \
+                }                                                                                                \
+            }                                                                                                    \
+        }                                                                                                        \
+    } while (0)
                     if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
 #pragma unroll 1
                     for (int ch = ch_begin; ch < ch_end; ch += 2) {
                         tmem_ld_wait();
                         if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);
-                        reduce_chunk(va, ch);
+                        OC_REDUCE_CHUNK(va, ch);
                         if (ch + 1 < ch_end) {
                             tmem_ld_wait();
                             if (ch + 2 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), va);
-                            reduce_chunk(vb, ch + 1);
+                            OC_REDUCE_CHUNK(vb, ch + 1);
                         }
                     }
-                    if (best1 > best0 || (best1 == best0 && n1 >= 0 && (n0 < 0 || n1 < n0))) { best0 = best1; n0 = n1; }
+#undef OC_REDUCE_CHUNK
+#undef OC_KEY
+                    // the better chain; among equal similarities the lower column
+                    int n0 = bc0 < 0 ? -1 : bc0 * 32 + 31 - (int)(__float_as_uint(bm0) & 31u);
+                    const int n1 = bc1 < 0 ? -1 : bc1 * 32 + 31 - (int)(__float_as_uint(bm1) & 31u);
+                    float best = OC_VAL(bm0);
+                    if (n1 >= 0 && (n0 < 0 || OC_VAL(bm1) > best || (OC_VAL(bm1) == best && n1 < n0))) { best = OC_VAL(bm1); n0 = n1; }
+#undef OC_VAL
                     if (row_ok && n0 >= 0) {
                         const int qi = c.q0 + (n0 >> 5), r = n0 & 31;
-                        const int hq = qi / P.n_wq, wq = qi - hq * P.n_wq;
+                        const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
                         const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));
                         const int y = (c.py * P.Hs + hs) * P.sy + my_rep, x = (c.px * P.Ws + ws) * P.sx + mx_rep;
                         const long long tokB = ((long long)c.bt * P.H + y) * P.W + x;
-                        atomicMax(P.keys + tokA, pack_key(best0, (uint32_t)tokB));
+                        atomicMax(P.keys + tokA, pack_key(best, (uint32_t)tokB));
                     }
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_acc_empty);              // both accumulators may be overwritten
+                if (lane == 0) {                                       // both accumulators may be overwritten
+                    if (PAIR) mbar_arrive_cluster(acc_empty + 8 * buf); else mbar_arrive(bar_acc_empty + 8 * buf);
+                }
             } else {
                 ok = false;
             }
-            // the column table is rewritten for the next piece: everyone must be done reading it
+            // the next piece's table entries; the barrier publishes them, and keeps the table just read
+            // from being overwritten (in the next turn) while a slower warp still reads it
+            if (have_nx) col_scale[((it + 1u) & 1u) * 256 + et] = sc_nx;
             if (!epilogue_barrier_all(ok)) { ok = false; break; }
+            c = nx; have = have_nx;
+            ++it;
         }
         if (!ok) { atomicCAS(P.status, 0, OC_ERR_TIMEOUT); *abort_flag = 1; }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();          // nobody signals a barrier of, or reads operands from, a retired CTA
     tc_fence_after();
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(TMEM_COLS) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -518,11 +809,13 @@ static int pow2_ceil_log2(int v) { int l = 0; while ((1 << l) < v) ++l; return l
 
 struct TcPlan {
     int bwA_log2, bhA, n_wtA, n_tilesA, tpp, n_apairs, bwQ_log2, bhQ, n_wq, n_quanta;
+    int pair, q_unit, n_q_units, a_merged, q_merged, q_lo;
     int pieces_per_row, qmax, n_stages, stage_bytes;
     long long rows, items;
 };
 
-static TcPlan make_plan(const Geo& g, int sm_count) {
+// walkers: CTAs that can run at once; pair_walkers: CTA pairs that can (0 = pairs not available)
+static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
     TcPlan p;
     int la = pow2_ceil_log2(g.Ws); if ((1 << la) > BM) la = pow2_ceil_log2(BM);
     p.bwA_log2 = la; p.bhA = BM >> la;
@@ -532,36 +825,64 @@ static TcPlan make_plan(const Geo& g, int sm_count) {
     p.bwQ_log2 = lq; p.bhQ = QN >> lq;
     p.n_wq = (g.Ws + (1 << lq) - 1) >> lq;
     p.n_quanta = p.n_wq * ((g.Hs + p.bhQ - 1) / p.bhQ);
-    // Tiles per piece (1 or 2) and pieces per row: estimated cycles = waves x per-piece cycles.  Per
-    // 64-channel step a piece fetches tpp*16 + 4q KB; the step takes the longest of: that fetch at
-    // ~48 B/clk/SM (measured L2 -> shared-memory feed), the fetch round trip (~3000 cycles) divided
-    // by the stages that fit in the ring, and tpp*64q tensor cycles.  The epilogue (~200 cycles per
-    // quantum and tile) is not overlapped.
+    // Form (single CTA or CTA pair), candidate tiles per CTA (1 or 2) and pieces per row: estimated
+    // cycles = waves x per-piece cycles.  Per 64-channel step a CTA fetches tpp*16 KB of candidates
+    // plus 4 KB per quantum it loads (all q of the piece, or q/2 in a pair); the step takes the
+    // longest of: that fetch at the measured L2 -> shared-memory feed rate, the fetch round trip
+    // divided by the stages that fit in the ring, and tpp*64q tensor cycles.  The epilogue (~200
+    // cycles per quantum and tile) is not overlapped.
     const int kblocks = (g.C + BK - 1) / BK;
-    double best_cost = 0; int best_P = 0, best_tpp = 2;
-    for (int tpp = 1; tpp <= 2; ++tpp) {
-        const long long rows = g.n_groups * (long long)(g.sy * g.sx - 1) * ((p.n_tilesA + tpp - 1) / tpp);
-        for (int P = (p.n_quanta + MAXQ - 1) / MAXQ; P <= p.n_quanta; ++P) {
-            const int q = (p.n_quanta + P - 1) / P;
-            const double stage_kb = tpp * 16.0 + 4.0 * q;
-            int stages = (int)(TILE_BYTES / 1024 / stage_kb); if (stages > MAX_STAGES) stages = MAX_STAGES;
-            const long long waves = (rows * P + sm_count - 1) / sm_count;
-            const double fetch = stage_kb * 1024.0 / 48.0, lat = 3000.0 / stages, mma = tpp * 64.0 * q;
-            double step = fetch > lat ? fetch : lat; if (mma > step) step = mma;
-            const double piece = kblocks * step + 200.0 * q * tpp + 1500.0;
-            const double cost = waves * piece;
-            if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; best_tpp = tpp; }
+    const double FEED_B_PER_CLK = 36.0;
+    double best_cost = 0; int best_P = 0, best_tpp = 2, best_pair = 0;
+    for (int pair = 0; pair <= (pair_walkers > 0 ? 1 : 0); ++pair) {
+        const int ncta = pair ? 2 : 1, q_unit = pair ? 2 : 1;
+        const int n_units = (p.n_quanta + q_unit - 1) / q_unit, max_units = MAXQ / q_unit;
+        const int nw = pair ? pair_walkers : walkers;
+        for (int tpp = 1; tpp <= 2; ++tpp) {
+            const long long rows = g.n_groups * (long long)(g.sy * g.sx - 1) *
+                                   ((p.n_tilesA + tpp * ncta - 1) / (tpp * ncta));
+            for (int P = (n_units + max_units - 1) / max_units; P <= n_units; ++P) {
+                const int q = ((n_units + P - 1) / P) * q_unit;       // quanta of the largest piece
+                const double stage_kb = tpp * 16.0 + 4.0 * q / ncta;
+                int stages = (int)(TILE_BYTES / 1024 / stage_kb); if (stages > MAX_STAGES) stages = MAX_STAGES;
+                const long long waves = (rows * P + nw - 1) / nw;
+                const double fetch = stage_kb * 1024.0 / FEED_B_PER_CLK, lat = (pair ? 3600.0 : 3000.0) / stages,
+                             mma = tpp * 64.0 * q;
+                double step = fetch > lat ? fetch : lat; if (mma > step) step = mma;
+                const double piece = kblocks * step + 200.0 * q * tpp + (pair ? 2500.0 : 1500.0);
+                const double cost = waves * piece;
+                if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; best_tpp = tpp; best_pair = pair; }
+            }
         }
     }
-    p.tpp = best_tpp;
-    p.n_apairs = (p.n_tilesA + p.tpp - 1) / p.tpp;
+    // Experiments may override the choice: OC_TC_PLAN="pair,tiles,pieces" (ignored unless valid).
+    if (const char* e = getenv("OC_TC_PLAN")) {
+        int o_pair = 0, o_tpp = 0, o_P = 0;
+        if (sscanf(e, "%d,%d,%d", &o_pair, &o_tpp, &o_P) == 3 && (o_pair == 0 || (o_pair == 1 && pair_walkers > 0)) &&
+            (o_tpp == 1 || o_tpp == 2)) {
+            const int q_unit = o_pair ? 2 : 1;
+            const int n_units = (p.n_quanta + q_unit - 1) / q_unit, max_units = MAXQ / q_unit;
+            if (o_P >= (n_units + max_units - 1) / max_units && o_P <= n_units) { best_pair = o_pair; best_tpp = o_tpp; best_P = o_P; }
+        }
+    }
+    p.pair = best_pair; p.tpp = best_tpp;
+    p.q_unit = p.pair ? 2 : 1;
+    p.n_q_units = (p.n_quanta + p.q_unit - 1) / p.q_unit;
+    const int ncta = p.pair ? 2 : 1;
+    p.n_apairs = (p.n_tilesA + p.tpp * ncta - 1) / (p.tpp * ncta);
     p.rows = g.n_groups * (long long)(g.sy * g.sx - 1) * p.n_apairs;
     p.pieces_per_row = best_P;
-    p.qmax = (p.n_quanta + best_P - 1) / best_P;
-    p.stage_bytes = p.tpp * A_BYTES + p.qmax * Q_BYTES;
+    p.qmax = ((p.n_q_units + best_P - 1) / best_P) * p.q_unit;
+    p.stage_bytes = p.tpp * A_BYTES + (p.qmax / ncta) * Q_BYTES;
     p.n_stages = TILE_BYTES / p.stage_bytes;
     if (p.n_stages > MAX_STAGES) p.n_stages = MAX_STAGES;
     p.items = p.rows * p.pieces_per_row;
+    // One copy instruction costs the producer ~100 cycles whatever the box size, so a CTA's candidate
+    // tiles, and its quanta of a piece, travel as ONE box each whenever they stack into a rectangle
+    // of lattice rows (always the case when the patch's lattice is at most one box wide).
+    p.a_merged = (p.tpp == 1 || p.n_wtA == 1) ? 1 : 0;
+    p.q_merged = p.n_wq == 1 ? 1 : 0;
+    p.q_lo = p.n_q_units / best_P;
     return p;
 }
 
@@ -579,28 +900,64 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
                                 unsigned long long* keys, float* aux_sim, cudaStream_t s) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return OC_ERR_UNSUPPORTED;
-    const TcPlan p = make_plan(g, ctx->sm_count);
+    // once per process: opt in to the large dynamic shared memory, and ask how many CTA pairs fit
+    static std::once_flag attr_once;
+    static bool attr_ok = false;
+    static int max_pairs[64];
+    std::call_once(attr_once, [] {
+        attr_ok = cudaFuncSetAttribute(match_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+                  cudaFuncSetAttribute(match_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+                  cudaFuncSetAttribute(match_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+                  cudaFuncSetAttribute(match_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess;
+        for (int i = 0; i < 64; ++i) max_pairs[i] = -1;
+        if (!attr_ok) cudaGetLastError();
+    });
+    if (!attr_ok) return OC_ERR_CUDA;
+    const int dev = ctx->device;
+    int pair_walkers = 0;
+    if (dev >= 0 && dev < 64) {
+        if (max_pairs[dev] < 0) {                     // (context's device is current here)
+            cudaLaunchConfig_t q = {};
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+            q.gridDim = dim3(2 * (unsigned)(ctx->sm_count / 2)); q.blockDim = dim3(TC_THREADS);
+            q.dynamicSmemBytes = SMEM_TOTAL; q.attrs = qa; q.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, match_tc_kernel<true, false>, &q) != cudaSuccess) { cudaGetLastError(); n = 0; }
+            if (n > ctx->sm_count / 2) n = ctx->sm_count / 2;
+            max_pairs[dev] = n;
+        }
+        pair_walkers = max_pairs[dev];
+    }
+    const TcPlan p = make_plan(g, ctx->sm_count, pair_walkers);
     if (p.items > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
 
-    TcParams P;
-    memset(&P, 0, sizeof(P));
+    TcParams KP;
+    memset(&KP, 0, sizeof(KP));
+    TcScalars& P = KP.s;
     const cuuint64_t dims[4] = {(cuuint64_t)g.C, (cuuint64_t)(g.W / g.sx), (cuuint64_t)(g.H / g.sy),
                                 (cuuint64_t)g.B * g.T};
     const cuuint64_t strides[3] = {(cuuint64_t)g.sx * g.C * 2, (cuuint64_t)g.sy * g.W * g.C * 2,
                                    (cuuint64_t)g.H * g.W * g.C * 2};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    const cuuint32_t boxA[4] = {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwA_log2), (cuuint32_t)p.bhA, 1};
-    const cuuint32_t boxQ[4] = {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwQ_log2), (cuuint32_t)p.bhQ, 1};
+    const cuuint32_t boxA[4] = {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwA_log2),
+                                (cuuint32_t)(p.bhA * (p.a_merged ? p.tpp : 1)), 1};
+    const int q_hi = (p.n_q_units % p.pieces_per_row) ? p.q_lo + 1 : p.q_lo;
+    const cuuint32_t boxQ[2][4] = {
+        {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwQ_log2), (cuuint32_t)(p.bhQ * (p.q_merged ? p.q_lo : 1)), 1},
+        {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwQ_log2), (cuuint32_t)(p.bhQ * (p.q_merged ? q_hi : 1)), 1}};
     const int rep_member = g.oy * g.sx + g.ox;
-    for (int m = 0; m <= g.sy * g.sx; ++m) {
-        const bool quantum_map = m == g.sy * g.sx;
+    const int n_members = g.sy * g.sx;
+    for (int m = 0; m < n_members + 2; ++m) {
+        const bool quantum_map = m >= n_members;
         const int member = quantum_map ? rep_member : m;
         if (!quantum_map && member == rep_member) continue;              // representatives are never candidates
         const int my = member / g.sx, mx = member - my * g.sx;
         void* base = (uint8_t*)x + ((size_t)my * g.W + mx) * g.C * 2;
-        CUresult r = enc(quantum_map ? &P.mapQ : &P.mapsA[m], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides,
-                         quantum_map ? boxQ : boxA, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        CUresult r = enc(quantum_map ? &KP.mapQ[m - n_members] : &KP.mapsA[m], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base,
+                         dims, strides, quantum_map ? boxQ[m - n_members] : boxA, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return OC_ERR_UNSUPPORTED;     // the FMA matcher takes over
     }
     P.H = g.H; P.W = g.W; P.sy = g.sy; P.sx = g.sx; P.gy = g.gy; P.gx = g.gx;
@@ -610,22 +967,40 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
     P.bwA_log2 = p.bwA_log2; P.bhA = p.bhA; P.n_wtA = p.n_wtA; P.n_tilesA = p.n_tilesA; P.tpp = p.tpp; P.n_apairs = p.n_apairs;
     P.bwQ_log2 = p.bwQ_log2; P.bhQ = p.bhQ; P.n_wq = p.n_wq; P.n_quanta = p.n_quanta;
     P.pieces_per_row = p.pieces_per_row; P.total_items = (int)p.items;
+    P.q_unit = p.q_unit; P.n_q_units = p.n_q_units;
+    P.a_merged = p.a_merged; P.q_merged = p.q_merged; P.q_lo = p.q_lo;
     P.n_stages = p.n_stages; P.stage_bytes = p.stage_bytes;
     P.units_per_group = (int)g.units_per_group; P.reps_per_group = (int)g.reps_per_group;
     P.inv_norm = inv_norm; P.keys = keys; P.aux = aux_sim; P.status = ctx->d_status;
-
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(match_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) != cudaSuccess)
-            return OC_ERR_CUDA;
-        attr_set = true;
-    }
-    // one CTA per SM, or one per piece when there are fewer pieces
-    long long grid = p.items;
-    if (grid > ctx->sm_count) grid = ctx->sm_count;
-    if (grid < 1) grid = 1;
+    // one walker (CTA or CTA pair) per SM (pair of SMs), or one per piece when there are fewer pieces
+    long long walkers = p.items;
+    const int cap = p.pair ? pair_walkers : ctx->sm_count;
+    if (walkers > cap) walkers = cap;
+    if (walkers < 1) walkers = 1;
+    P.items_base = (int)(p.items / walkers); P.items_rem = (int)(p.items % walkers);
+    P.cum[0] = (unsigned)p.pieces_per_row; P.cum[1] = P.cum[0] * (unsigned)p.n_apairs;
+    P.cum[2] = P.cum[1] * (unsigned)P.n_cand_lat; P.cum[3] = P.cum[2] * (unsigned)g.gx; P.cum[4] = P.cum[3] * (unsigned)g.gy;
+    P.u_step_q = p.n_q_units / p.pieces_per_row; P.u_step_r = p.n_q_units % p.pieces_per_row;
+    for (int i = 0; i < 5; ++i) P.rcp_cum[i] = 1.0f / (float)P.cum[i];
+    P.rcp_ppr = 1.0f / (float)p.pieces_per_row;
+    P.rcp_n_wtA = 1.0f / (float)p.n_wtA; P.rcp_n_wq = 1.0f / (float)p.n_wq;
+    P.my_rep = rep_member / g.sx; P.mx_rep = rep_member % g.sx;
+    P.sx_magic = (65536 + g.sx - 1) / g.sx;
     LaunchScope scope(ctx, OC_K_MATCH_TC, s);
-    match_tc_kernel<<<(unsigned)grid, TC_THREADS, SMEM_TOTAL, s>>>(P);
+    if (p.pair) {
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3(2 * (unsigned)walkers); cfg.blockDim = dim3(TC_THREADS);
+        cfg.dynamicSmemBytes = SMEM_TOTAL; cfg.stream = s; cfg.attrs = at; cfg.numAttrs = 1;
+        const cudaError_t e = aux_sim ? cudaLaunchKernelEx(&cfg, match_tc_kernel<true, true>, KP)
+                                      : cudaLaunchKernelEx(&cfg, match_tc_kernel<true, false>, KP);
+        if (e != cudaSuccess) { cudaGetLastError(); return OC_ERR_CUDA; }
+        return OC_OK;
+    }
+    if (aux_sim) match_tc_kernel<false, true><<<(unsigned)walkers, TC_THREADS, SMEM_TOTAL, s>>>(KP);
+    else match_tc_kernel<false, false><<<(unsigned)walkers, TC_THREADS, SMEM_TOTAL, s>>>(KP);
     return last_launch_status();
 }
 
