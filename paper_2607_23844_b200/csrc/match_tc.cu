@@ -825,14 +825,20 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
     p.bwQ_log2 = lq; p.bhQ = QN >> lq;
     p.n_wq = (g.Ws + (1 << lq) - 1) >> lq;
     p.n_quanta = p.n_wq * ((g.Hs + p.bhQ - 1) / p.bhQ);
-    // Form (single CTA or CTA pair), candidate tiles per CTA (1 or 2) and pieces per row: estimated
-    // cycles = waves x per-piece cycles.  Per 64-channel step a CTA fetches tpp*16 KB of candidates
-    // plus 4 KB per quantum it loads (all q of the piece, or q/2 in a pair); the step takes the
-    // longest of: that fetch at the measured L2 -> shared-memory feed rate, the fetch round trip
-    // divided by the stages that fit in the ring, and tpp*64q tensor cycles.  The epilogue (~200
-    // cycles per quantum and tile) is not overlapped.
+    // Form (single CTA or CTA pair), candidate tiles per CTA (1 or 2) and pieces per row, by estimated
+    // cycles of the busiest walker.  The shape of the estimate follows the kernel; its constants were
+    // fitted to timed sweeps of all valid plans on six workloads (SD3-shaped token cache at 1/4/8
+    // token groups per image, the three SVD UNet levels):
+    //   * per 64-channel stage a CTA fetches tpp*16 KB of candidates plus 4 KB per quantum it loads
+    //     (all q of the piece, or q/2 in a pair) and issues tpp*64*q tensor cycles; the stage takes the
+    //     longest of the MMAs (+~50 cycles between stages), the fetch at ~74 B/clk, and - once the ring
+    //     has been drained - the refill round trip (MMAs + ~330 + ~1500 cycles of copy latency, ~1000
+    //     more in a pair) divided by the stages that fit in the ring;
+    //   * the epilogue costs ~250 + ~410 cycles per 32 columns of each thread's half, per tile; with two
+    //     tiles per CTA it follows the MMAs of the piece, with one tile it runs under the next piece's
+    //     MMAs, where the two slow each other down (~0.8 of the shorter one is not hidden);
+    //   * ~6500 cycles before a CTA's first MMA and after its last.
     const int kblocks = (g.C + BK - 1) / BK;
-    const double FEED_B_PER_CLK = 36.0;
     double best_cost = 0; int best_P = 0, best_tpp = 2, best_pair = 0;
     for (int pair = 0; pair <= (pair_walkers > 0 ? 1 : 0); ++pair) {
         const int ncta = pair ? 2 : 1, q_unit = pair ? 2 : 1;
@@ -845,12 +851,22 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
                 const int q = ((n_units + P - 1) / P) * q_unit;       // quanta of the largest piece
                 const double stage_kb = tpp * 16.0 + 4.0 * q / ncta;
                 int stages = (int)(TILE_BYTES / 1024 / stage_kb); if (stages > MAX_STAGES) stages = MAX_STAGES;
-                const long long waves = (rows * P + nw - 1) / nw;
-                const double fetch = stage_kb * 1024.0 / FEED_B_PER_CLK, lat = (pair ? 3600.0 : 3000.0) / stages,
-                             mma = tpp * 64.0 * q;
-                double step = fetch > lat ? fetch : lat; if (mma > step) step = mma;
-                const double piece = kblocks * step + 200.0 * q * tpp + (pair ? 2500.0 : 1500.0);
-                const double cost = waves * piece;
+                const long long per_walker = (rows * P + nw - 1) / nw;
+                const double mma = tpp * 64.0 * q, fetch = stage_kb * 1024.0 / 74.0;
+                const double refill = (mma + 330.0 + 1450.0 + 1.35 * stage_kb + (pair ? 980.0 : 0.0)) / stages;
+                double fast = mma + 53.0; if (fetch > fast) fast = fetch;
+                const double slow = refill > fast ? refill : fast;
+                const double epi = tpp * (246.0 + 413.0 * ((q + 1) / 2));
+                double piece;
+                if (tpp == 1) {
+                    const double loop = kblocks * slow;
+                    piece = (loop + 440.0 > epi ? loop + 440.0 : epi) + 0.79 * (loop < epi ? loop : epi);
+                } else {
+                    const int nf = kblocks < stages ? kblocks : stages;
+                    piece = nf * fast + (kblocks - nf) * slow + epi + 534.0;
+                }
+                if (pair) piece += 850.0;
+                const double cost = 6550.0 + (pair ? 616.0 : 0.0) + per_walker * piece + (tpp == 1 ? epi : 0.0);
                 if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; best_tpp = tpp; best_pair = pair; }
             }
         }
