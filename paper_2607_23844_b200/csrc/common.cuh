@@ -62,6 +62,36 @@ struct LaunchScope {
     ~LaunchScope();
 };
 
+// Launch with programmatic stream serialization: the grid may be scheduled while the kernel before it
+// in the stream is still running, once every CTA of that kernel has executed
+// griddepcontrol.launch_dependents (or exited), which hides the launch latency between the kernels of
+// a step.  Kernels launched this way execute griddepcontrol.wait (pdl_wait) before they touch
+// anything the earlier kernel reads or writes, and only then let their own dependents go, so a grid
+// never runs ahead of more than the one kernel before it.  Use as
+//     OC_LAUNCH((kernel<T, N>), grid, block, smem_bytes, stream, args...);
+struct PdlLaunch {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    PdlLaunch(dim3 grid, dim3 block, size_t smem, cudaStream_t s, unsigned cluster_x = 0) {
+        cfg = cudaLaunchConfig_t{};
+        cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 1;
+        if (cluster_x > 1) {
+            attr[1].id = cudaLaunchAttributeClusterDimension;
+            attr[1].val.clusterDim.x = cluster_x; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+            cfg.numAttrs = 2;
+        }
+        cfg.attrs = attr;
+    }
+};
+#define OC_LAUNCH(kernel, grid, block, smem, stream, ...)                      \
+    do {                                                                       \
+        ::oc::PdlLaunch oc_l_((grid), (block), (smem), (stream));              \
+        cudaLaunchKernelEx(&oc_l_.cfg, kernel, __VA_ARGS__);                   \
+    } while (0)
+
 inline oc_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? OC_OK : OC_ERR_CUDA; }
 inline oc_status last_launch_status() { return cuda_ok(cudaGetLastError()); }
 
@@ -133,6 +163,12 @@ size_t match_workspace_bytes(const Geo&);
 
 // ---- device helpers ---------------------------------------------------------------------------
 #ifdef __CUDACC__
+// See PdlLaunch: wait for the kernel before this one in the stream (all of it, memory included), and
+// let the kernel after this one be scheduled.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_launch_dependents(); }
+
 __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"

@@ -16,6 +16,7 @@ template <int DT, int LPR>
 __global__ void __launch_bounds__(256)
 norms_kernel(const uint8_t* __restrict__ x, long long n_tok, int cpr, float eps,
              float* __restrict__ inv_norm, unsigned long long* __restrict__ keys) {
+    pdl_enter();
     constexpr int CPL = 8;                                   // chunks a lane holds at once
     const int lane = threadIdx.x % LPR;
     const long long groups_total = (long long)gridDim.x * (256 / LPR);
@@ -54,10 +55,10 @@ static void norms_dispatch(int sm_count, cudaStream_t s, const uint8_t* x, long 
     const long long cap = (long long)sm_count * 4;           // 4 resident CTAs of 256 threads per SM (64 registers)
     if (blocks > cap) blocks = cap;
     switch (lpr) {
-        case 4:  norms_kernel<DT, 4><<<(unsigned)blocks, 256, 0, s>>>(x, n_tok, cpr, eps, inv_norm, keys); break;
-        case 8:  norms_kernel<DT, 8><<<(unsigned)blocks, 256, 0, s>>>(x, n_tok, cpr, eps, inv_norm, keys); break;
-        case 16: norms_kernel<DT, 16><<<(unsigned)blocks, 256, 0, s>>>(x, n_tok, cpr, eps, inv_norm, keys); break;
-        default: norms_kernel<DT, 32><<<(unsigned)blocks, 256, 0, s>>>(x, n_tok, cpr, eps, inv_norm, keys); break;
+        case 4:  OC_LAUNCH((norms_kernel<DT, 4>), (unsigned)blocks, 256, 0, s, x, n_tok, cpr, eps, inv_norm, keys); break;
+        case 8:  OC_LAUNCH((norms_kernel<DT, 8>), (unsigned)blocks, 256, 0, s, x, n_tok, cpr, eps, inv_norm, keys); break;
+        case 16: OC_LAUNCH((norms_kernel<DT, 16>), (unsigned)blocks, 256, 0, s, x, n_tok, cpr, eps, inv_norm, keys); break;
+        default: OC_LAUNCH((norms_kernel<DT, 32>), (unsigned)blocks, 256, 0, s, x, n_tok, cpr, eps, inv_norm, keys); break;
     }
 }
 
@@ -106,6 +107,7 @@ template <int DT>
 __global__ void __launch_bounds__(256)
 dense_simt_kernel(const uint8_t* __restrict__ x, SimtGeo sg, const float* __restrict__ inv_norm,
                   unsigned long long* __restrict__ keys, float* __restrict__ aux_sim) {
+    pdl_enter();
     __shared__ __align__(16) float As[SK][ST + 4];
     __shared__ __align__(16) float Bs[SK][ST + 4];
     __shared__ long long a_tok[ST], b_tok[ST];          // global token index, -1 = masked
@@ -194,6 +196,7 @@ __global__ void __launch_bounds__(256)
 finalize_kernel(GroupMap gm, long long n_groups, const float* __restrict__ inv_norm,
                 const unsigned long long* __restrict__ keys, float* __restrict__ best_sim,
                 int32_t* __restrict__ best_idx) {
+    pdl_enter();
     const long long w = (long long)blockIdx.x * 256 + threadIdx.x;
     const int U = gm.units_per_group;
     if (w >= n_groups * U) return;
@@ -245,16 +248,16 @@ oc_status launch_match_token(oc_ctx* ctx, const Geo& g, const void* x, float* be
         if (grid.y > 65535) return OC_ERR_UNSUPPORTED;
         LaunchScope scope(ctx, OC_K_MATCH_SIMT, s);
         if (g.dtype == OC_DTYPE_BF16)
-            dense_simt_kernel<OC_DTYPE_BF16><<<grid, 256, 0, s>>>((const uint8_t*)x, sg, inv_norm, keys, aux_sim);
+            OC_LAUNCH(dense_simt_kernel<OC_DTYPE_BF16>, grid, 256, 0, s, (const uint8_t*)x, sg, inv_norm, keys, aux_sim);
         else
-            dense_simt_kernel<OC_DTYPE_F32><<<grid, 256, 0, s>>>((const uint8_t*)x, sg, inv_norm, keys, aux_sim);
+            OC_LAUNCH(dense_simt_kernel<OC_DTYPE_F32>, grid, 256, 0, s, (const uint8_t*)x, sg, inv_norm, keys, aux_sim);
         st = last_launch_status();
     }
     if (st != OC_OK) return st;
     {
         LaunchScope scope(ctx, OC_K_MATCH_FIN, s);
-        finalize_kernel<<<(unsigned)((n_tok + 255) / 256), 256, 0, s>>>(make_group_map(g), g.n_groups, inv_norm, keys,
-                                                                        best_sim, best_idx);
+        OC_LAUNCH(finalize_kernel, (unsigned)((n_tok + 255) / 256), 256, 0, s, make_group_map(g), g.n_groups, inv_norm, keys,
+                  best_sim, best_idx);
     }
     return last_launch_status();
 }

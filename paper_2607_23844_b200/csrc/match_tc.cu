@@ -613,6 +613,10 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             const int y = (pc.py * P.Hs + hs) * P.sy + my_rep, x = (pc.px * P.Ws + ws) * P.sx + mx_rep;
             return __ldg(P.inv_norm + ((long long)pc.bt * P.H + y) * P.W + x);
         };
+        // Only from here on does this kernel touch what the norm pre-pass (the kernel before it in the
+        // stream) writes: its operand copies and MMAs may run while that kernel still does.
+        pdl_wait();
+        if (et == 0) pdl_launch_dependents();
         Piece nx;
         bool have = walk.next(P, c);
         if (have) col_scale[et] = table_entry(c);
@@ -1004,19 +1008,14 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
     P.sx_magic = (65536 + g.sx - 1) / g.sx;
     LaunchScope scope(ctx, OC_K_MATCH_TC, s);
     if (p.pair) {
-        cudaLaunchConfig_t cfg = {};
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeClusterDimension;
-        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-        cfg.gridDim = dim3(2 * (unsigned)walkers); cfg.blockDim = dim3(TC_THREADS);
-        cfg.dynamicSmemBytes = SMEM_TOTAL; cfg.stream = s; cfg.attrs = at; cfg.numAttrs = 1;
-        const cudaError_t e = aux_sim ? cudaLaunchKernelEx(&cfg, match_tc_kernel<true, true>, KP)
-                                      : cudaLaunchKernelEx(&cfg, match_tc_kernel<true, false>, KP);
+        PdlLaunch l(dim3(2 * (unsigned)walkers), dim3(TC_THREADS), SMEM_TOTAL, s, 2);
+        const cudaError_t e = aux_sim ? cudaLaunchKernelEx(&l.cfg, match_tc_kernel<true, true>, KP)
+                                      : cudaLaunchKernelEx(&l.cfg, match_tc_kernel<true, false>, KP);
         if (e != cudaSuccess) { cudaGetLastError(); return OC_ERR_CUDA; }
         return OC_OK;
     }
-    if (aux_sim) match_tc_kernel<false, true><<<(unsigned)walkers, TC_THREADS, SMEM_TOTAL, s>>>(KP);
-    else match_tc_kernel<false, false><<<(unsigned)walkers, TC_THREADS, SMEM_TOTAL, s>>>(KP);
+    if (aux_sim) OC_LAUNCH((match_tc_kernel<false, true>), (unsigned)walkers, TC_THREADS, SMEM_TOTAL, s, KP);
+    else OC_LAUNCH((match_tc_kernel<false, false>), (unsigned)walkers, TC_THREADS, SMEM_TOTAL, s, KP);
     return last_launch_status();
 }
 

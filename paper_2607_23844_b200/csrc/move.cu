@@ -49,6 +49,7 @@ template <bool SEG>
 __global__ void __launch_bounds__(MOVE_THREADS)
 gather_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ kept_idx,
               uint8_t* __restrict__ y, unsigned total_chunks, RowsDev R) {
+    pdl_enter();
     const unsigned base = blockIdx.x * (MOVE_THREADS * MOVE_UNROLL) + threadIdx.x;
     uint4 v[MOVE_UNROLL];
     bool ok[MOVE_UNROLL];
@@ -79,6 +80,7 @@ __global__ void __launch_bounds__(MOVE_THREADS)
 restore_kernel(const uint8_t* __restrict__ z, const uint8_t* __restrict__ cache,
                const int32_t* __restrict__ slot_of, const int32_t* __restrict__ match_map,
                uint8_t* __restrict__ out, unsigned total_chunks, RowsDev R) {
+    pdl_enter();
     const unsigned base = blockIdx.x * (MOVE_THREADS * MOVE_UNROLL) + threadIdx.x;
     uint4 v[MOVE_UNROLL];
     long long dst[MOVE_UNROLL];
@@ -108,6 +110,7 @@ restore_kernel(const uint8_t* __restrict__ z, const uint8_t* __restrict__ cache,
 __global__ void __launch_bounds__(MOVE_THREADS)
 copy_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, unsigned long long n_chunks,
             unsigned long long tail_begin, unsigned tail_bytes) {
+    pdl_enter();
     const unsigned long long base = (unsigned long long)blockIdx.x * (MOVE_THREADS * MOVE_UNROLL) + threadIdx.x;
     uint4 v[MOVE_UNROLL];
 #pragma unroll
@@ -139,8 +142,8 @@ oc_status launch_gather(oc_ctx* ctx, const oc_rows& rows, const void* x, const i
         unsigned blocks = (total + MOVE_THREADS * MOVE_UNROLL - 1) / (MOVE_THREADS * MOVE_UNROLL);
         uint8_t* yy = (uint8_t*)y + s0 * (int64_t)R.cpr * 16;
         LaunchScope scope(ctx, OC_K_GATHER, s);
-        if (seg) gather_kernel<true><<<blocks, MOVE_THREADS, 0, s>>>((const uint8_t*)x, kept_idx + s0, yy, total, R);
-        else     gather_kernel<false><<<blocks, MOVE_THREADS, 0, s>>>((const uint8_t*)x, kept_idx + s0, yy, total, R);
+        if (seg) OC_LAUNCH(gather_kernel<true>, blocks, MOVE_THREADS, 0, s, (const uint8_t*)x, kept_idx + s0, yy, total, R);
+        else     OC_LAUNCH(gather_kernel<false>, blocks, MOVE_THREADS, 0, s, (const uint8_t*)x, kept_idx + s0, yy, total, R);
     }
     return last_launch_status();
 }
@@ -149,9 +152,9 @@ template <bool SEG>
 static void restore_dispatch(int mode, unsigned blocks, cudaStream_t s, const uint8_t* z, const uint8_t* cache,
                              const int32_t* slot_of, const int32_t* match_map, uint8_t* out, unsigned total,
                              const RowsDev& R) {
-    if (mode == 0) restore_kernel<SEG, 0><<<blocks, MOVE_THREADS, 0, s>>>(z, cache, slot_of, match_map, out, total, R);
-    else if (mode == 1) restore_kernel<SEG, 1><<<blocks, MOVE_THREADS, 0, s>>>(z, cache, slot_of, match_map, out, total, R);
-    else restore_kernel<SEG, 2><<<blocks, MOVE_THREADS, 0, s>>>(z, cache, slot_of, match_map, out, total, R);
+    if (mode == 0) OC_LAUNCH((restore_kernel<SEG, 0>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, out, total, R);
+    else if (mode == 1) OC_LAUNCH((restore_kernel<SEG, 1>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, out, total, R);
+    else OC_LAUNCH((restore_kernel<SEG, 2>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, out, total, R);
 }
 
 oc_status launch_restore(oc_ctx* ctx, const oc_rows& rows, const void* z, const void* cache,
@@ -190,7 +193,7 @@ oc_status launch_copy(oc_ctx* ctx, const void* src, void* dst, size_t bytes, cud
     if (blocks == 0) blocks = 1;
     if (blocks > 0x7FFFFFFFull) return OC_ERR_UNSUPPORTED;
     LaunchScope scope(ctx, OC_K_COPY, s);
-    copy_kernel<<<(unsigned)blocks, MOVE_THREADS, 0, s>>>((const uint8_t*)src, (uint8_t*)dst, n_chunks, tail_begin, (unsigned)tail);
+    OC_LAUNCH(copy_kernel, (unsigned)blocks, MOVE_THREADS, 0, s, (const uint8_t*)src, (uint8_t*)dst, n_chunks, tail_begin, (unsigned)tail);
     return last_launch_status();
 }
 

@@ -91,6 +91,7 @@ select_general_kernel(GroupMap gm, const float* __restrict__ best_sim, const int
               int mode, float thr, int n_reuse, int y_stride, int keys_in_smem,
               int32_t* __restrict__ kept_idx, int32_t* __restrict__ kept_count,
               int32_t* __restrict__ match_map, int32_t* __restrict__ slot_of) {
+    pdl_enter();
     extern __shared__ unsigned key_cache[];                    // [U] when keys_in_smem
     __shared__ unsigned reuse_bits[SEL_MAX_UNITS / 32];
     __shared__ int scan_sums[2][33];
@@ -284,6 +285,7 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
                    int mode, float thr, int n_reuse, int y_stride,
                    int32_t* __restrict__ kept_idx, int32_t* __restrict__ kept_count,
                    int32_t* __restrict__ match_map, int32_t* __restrict__ slot_of) {
+    pdl_enter();
     extern __shared__ unsigned key_cache[];                    // [U] keys, later reused as kept positions
     __shared__ int scan_sums[2][33];
     __shared__ unsigned hist[256];
@@ -490,14 +492,13 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
     }
     LaunchScope scope(ctx, OC_K_SELECT, s);
     if (!geo.self_match && geo.units_per_group <= SEL_SMEM_KEYS) {
-        select_fast_kernel<<<(unsigned)geo.n_groups, SEL_THREADS, (size_t)geo.units_per_group * sizeof(unsigned), s>>>(
-            gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);
+        OC_LAUNCH(select_fast_kernel, (unsigned)geo.n_groups, SEL_THREADS, (size_t)geo.units_per_group * sizeof(unsigned), s,
+                  gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);
     } else {
         const int keys_in_smem = (mode == OC_SELECT_COUNT && geo.units_per_group <= SEL_SMEM_KEYS) ? 1 : 0;
         const size_t dyn = keys_in_smem ? (size_t)geo.units_per_group * sizeof(unsigned) : 0;
-        select_general_kernel<<<(unsigned)geo.n_groups, SEL_THREADS, dyn, s>>>(gm, best_sim, best_idx, mode, thr, nr,
-                                                                                (int)y_stride, keys_in_smem, kept_idx,
-                                                                                kept_count, match_map, slot_of);
+        OC_LAUNCH(select_general_kernel, (unsigned)geo.n_groups, SEL_THREADS, dyn, s, gm, best_sim, best_idx, mode, thr, nr,
+                  (int)y_stride, keys_in_smem, kept_idx, kept_count, match_map, slot_of);
     }
     return last_launch_status();
 }
