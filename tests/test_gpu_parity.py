@@ -163,6 +163,38 @@ def test_token_chain_small(oc, oracle, shape, groups, lattice, dtype):
         assert rep["launches"]["match_tc"] + rep["launches"]["match_simt"] == 1
 
 
+@pytest.mark.parametrize("shape,groups", [
+    ((2, 1, 64, 64, 192), (1, 1)),       # 1024 representatives: 32 quanta, 8 candidate tiles per lattice
+    ((1, 3, 40, 56, 136), (1, 1)),       # ragged 20 x 28 lattice, K tail, three frames
+    ((1, 1, 64, 64, 128), (2, 2)),       # four patches per frame
+])
+@pytest.mark.parametrize("plan", ["0,1,1", "0,1,3", "0,2,2", "0,2,5", "1,1,1", "1,1,2", "1,2,1", "1,2,4", "0,2,64", "1,1,64"])
+def test_tensor_core_matcher_every_plan(oc, oracle, shape, groups, plan, monkeypatch):
+    """The planner's choice (single CTA or CTA pair, one or two candidate tiles per CTA, pieces per
+    row) changes the work split only: every valid plan must reproduce the oracle.  A plan the shape
+    does not admit is ignored by the library (the planner's own choice runs instead)."""
+    B, T, Hh, W, C = shape
+    w = inputs.sd3_token_cache(seed=33, B=B * T, H=Hh, W=W, C=C, groups=groups)
+    w.x = w.x.reshape(shape); w.shape = shape
+    L, Lo = H.layouts(oc, oracle, w)
+    ref = oracle.match_token(Lo, w.x, want_full=True)
+    monkeypatch.setenv("OC_TC_PLAN", plan)
+    x_dev = H.to_dev(w.x)
+    with H.make_ctx(oc, L) as ctx:
+        ctx.profile_enable(True)
+        for want_aux in (False, True):
+            m = H.gpu_match(oc, ctx, L, x_dev, want_aux=want_aux)
+            gs, gi = m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy()
+            H.check_match_against_oracle(oracle, Lo, w.x, gs, gi, ref, TOL[inputs.BF16])
+            if want_aux:
+                a = m["aux"].cpu().numpy().astype(np.float64)
+                f = ref["full_sim"]
+                written = ~np.isnan(f)
+                assert np.array_equal(~np.isnan(a), written), "aux rows written differ from the oracle's"
+                assert np.abs(a[written] - f[written]).max() <= TOL[inputs.BF16]
+        assert ctx.profile_read(oc.K_MATCH_TC)[0] == 2
+
+
 @pytest.mark.parametrize("dtype", [inputs.BF16, inputs.F32])
 @pytest.mark.parametrize("T,stat", [(7, 0), (6, 1), (2, 0), (1, 0)])
 def test_frame_chain_small(oc, oracle, dtype, T, stat):
