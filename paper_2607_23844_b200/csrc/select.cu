@@ -3,8 +3,10 @@
 // One CTA per group (a group is an independent selection problem).  Everything is decided in
 // ascending unit order, so the result is deterministic and comparable bit for bit:
 //   COUNT mode  - the candidates' best_sim are staged once in shared memory as order-preserving
-//                 keys; a 4 x 8-bit radix select (warp-aggregated histogram updates, warp-parallel
-//                 bin search) finds the value at the cut; candidates above it are reused, candidates
+//                 keys; a radix select finds the value at the cut (fast kernel: 12-bit digits of the
+//                 key relative to the smallest candidate key, two passes for the narrow range one
+//                 group's similarities span; general kernel: 4 x 8-bit digits of the raw key with
+//                 warp-aggregated histogram updates); candidates above the cut are reused, candidates
 //                 equal to it are admitted lowest index first;
 //   both modes  - kept units are compacted with block-wide prefix sums (stable, ascending original
 //                 index).
@@ -288,14 +290,14 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     pdl_enter();
     extern __shared__ unsigned key_cache[];                    // [U] keys, later reused as kept positions
     __shared__ int scan_sums[2][33];
-    __shared__ unsigned hist[256];
+    __shared__ unsigned hist[4096];
     __shared__ unsigned sh_prefix, sh_remaining;
     __shared__ int sh_ncand;
     __shared__ unsigned sh_kmin, sh_kmax;
 
     const int U = gm.units_per_group;
     const long long g = blockIdx.x;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int n_rounds = (U + SEL_THREADS - 1) / SEL_THREADS;
     const GroupView gv(gm, g);
 
@@ -312,16 +314,19 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
         long long gi[PF];
 #pragma unroll
         for (int k = 0; k < PF; ++k) {
+            if (r0 + k >= n_rounds) break;                          // (uniform: whole rounds that do not exist)
             const int u = (r0 + k) * SEL_THREADS + tid;
             gi[k] = u < U ? gv.index(gm, u) : -1;
         }
 #pragma unroll
         for (int k = 0; k < PF; ++k) {
+            if (r0 + k >= n_rounds) break;
             sim_pf[k] = gi[k] >= 0 ? best_sim[gi[k]] : 0.f;
             if (r0 == 0) idx_pf[k] = gi[k] >= 0 ? best_idx[gi[k]] : 0;
         }
 #pragma unroll
         for (int k = 0; k < PF; ++k) {
+            if (r0 + k >= n_rounds) break;
             const int u = (r0 + k) * SEL_THREADS + tid;
             if (u < U) {
                 unsigned key = 0;
@@ -356,66 +361,51 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
         if (k >= n_cand) {
             all_reused = true;
         } else if (k > 0) {
+            // Radix select of the k-th largest key, 12 bits at a time, on keys taken relative to the
+            // smallest candidate key: similarities of one group span a narrow range, so two passes
+            // cover it where 8-bit digits of the raw key needed four (three cover any 32-bit span).
             if (tid == 0) { sh_prefix = 0; sh_remaining = (unsigned)k; }
-            const unsigned span = sh_kmin ^ sh_kmax;            // bits in which candidates differ at all
-            for (int pass = 0; pass < 4; ++pass) {
-                const int shift = 24 - 8 * pass;
-                if ((span >> shift) == 0) {                         // every candidate shares this digit: no histogram needed
-                    __syncthreads();
-                    if (tid == 0) sh_prefix |= ((sh_kmax >> shift) & 255u) << shift;
-                    __syncthreads();
-                    continue;
-                }
-                if (tid < 256) hist[tid] = 0;
+            const unsigned base = sh_kmin;
+            const unsigned span = sh_kmax - base;
+            const int nbits = 32 - __clz(span);                    // 0 when all candidate keys are equal
+            const int n_pass = (nbits + 11) / 12;
+            for (int pass = 0; pass < n_pass; ++pass) {
+                const int shift = 12 * (n_pass - 1 - pass);
+                for (int i = tid; i < 4096; i += SEL_THREADS) hist[i] = 0;
                 __syncthreads();
-                const unsigned prefix = sh_prefix;
-                const unsigned himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+                const unsigned prefix = sh_prefix;                  // the digits fixed so far (high part of rel)
                 for (int r = 0; r < n_rounds; ++r) {
                     const int u = r * SEL_THREADS + tid;
                     const unsigned key = u < U ? key_cache[u] : 0u;
-                    const bool take = key != 0 && (key & himask) == prefix;
-                    const unsigned digit = (key >> shift) & 255u;
-                    // high digits are usually shared by the whole warp: one atomic for all of them;
-                    // otherwise plain shared-memory atomics (distinct bins rarely collide)
-                    const unsigned takers = __ballot_sync(0xFFFFFFFFu, take);
-                    if (takers) {
-                        const unsigned dref = __shfl_sync(0xFFFFFFFFu, digit, __ffs(takers) - 1);
-                        if (__all_sync(0xFFFFFFFFu, !take || digit == dref)) {
-                            if (lane == 0) atomicAdd(&hist[dref], (unsigned)__popc(takers));
-                        } else if (take) {
-                            atomicAdd(&hist[digit], 1u);
-                        }
+                    if (key != 0) {
+                        const unsigned rel = key - base;
+                        // (a shift by 32 would be undefined: the first pass has no fixed digits)
+                        if (pass == 0 || (rel >> (shift + 12)) == prefix) atomicAdd(&hist[(rel >> shift) & 4095u], 1u);
                     }
                 }
                 __syncthreads();
-                if (warp == 0) {
-                    // lane l owns bins 255-8l .. 248-8l (descending); find where the running count reaches rem
-                    const unsigned rem = sh_remaining;
-                    unsigned c[8], tot = 0;
+                // thread t owns bins 4095-4t .. 4092-4t (descending): where does the running count reach rem?
+                const unsigned rem = sh_remaining;
+                unsigned c[4], tot = 0;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) { c[i] = hist[255 - 8 * lane - i]; tot += c[i]; }
-                    unsigned incl = tot;
+                for (int i = 0; i < 4; ++i) { c[i] = hist[4095 - 4 * tid - i]; tot += c[i]; }
+                int all;
+                const unsigned before = (unsigned)block_scan_int((int)tot, scan_sums[pass & 1], all);
+                if (before < rem && rem <= before + tot) {
+                    unsigned acc = before;
+                    int bin = 4095 - 4 * tid;
 #pragma unroll
-                    for (int d = 1; d < 32; d <<= 1) {
-                        const unsigned n = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                        if (lane >= d) incl += n;
+                    for (int i = 0; i < 4; ++i) {
+                        if (acc + c[i] >= rem) { bin = 4095 - 4 * tid - i; break; }
+                        acc += c[i];
                     }
-                    const unsigned before = incl - tot;
-                    if (before < rem && rem <= incl) {
-                        unsigned acc = before;
-                        int bin = 255 - 8 * lane;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            if (acc + c[i] >= rem) { bin = 255 - 8 * lane - i; break; }
-                            acc += c[i];
-                        }
-                        sh_prefix = prefix | ((unsigned)bin << shift);
-                        sh_remaining = rem - acc;
-                    }
+                    sh_prefix = (prefix << 12) | (unsigned)bin;
+                    sh_remaining = rem - acc;
                 }
                 __syncthreads();
             }
-            cut_key = sh_prefix;
+            // (with no pass at all every candidate has the key `base`: the cut is that key, k of them reused)
+            cut_key = base + sh_prefix;
             need_eq = (int)sh_remaining;
         }
     }
@@ -450,9 +440,7 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     __syncthreads();
 
     // ---- phase 3: one coalesced pass writes every output ------------------------------------------
-    for (int r = 0; r < n_rounds; ++r) {
-        const int u = r * SEL_THREADS + tid;
-        if (u >= U) break;
+    auto emit = [&](int u, int m_pf, bool have_pf) {
         const long long i = gv.index(gm, u);
         const unsigned p = key_cache[u];
         if (p != 0xFFFFFFFFu) {
@@ -461,14 +449,17 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
             match_map[i] = (int32_t)i;
         } else {
             slot_of[i] = -1;
-            int m;
-            switch (r) {                                            // registers of the first PF rounds, else reload
-                case 0: m = idx_pf[0]; break; case 1: m = idx_pf[1]; break; case 2: m = idx_pf[2]; break;
-                case 3: m = idx_pf[3]; break; case 4: m = idx_pf[4]; break; case 5: m = idx_pf[5]; break;
-                case 6: m = idx_pf[6]; break; case 7: m = idx_pf[7]; break; default: m = best_idx[i]; break;
-            }
-            match_map[i] = m;
+            match_map[i] = have_pf ? m_pf : best_idx[i];            // registers of the first PF rounds, else reload
         }
+    };
+#pragma unroll
+    for (int r = 0; r < PF; ++r) {
+        const int u = r * SEL_THREADS + tid;
+        if (r < n_rounds && u < U) emit(u, idx_pf[r], true);
+    }
+    for (int r = PF; r < n_rounds; ++r) {
+        const int u = r * SEL_THREADS + tid;
+        if (u < U) emit(u, 0, false);
     }
     for (int p = kept_total + tid; p < y_stride; p += SEL_THREADS) kept_idx[g * y_stride + p] = -1;
     if (tid == 0) kept_count[g] = kept_total;
