@@ -349,6 +349,22 @@ def run_ours(args, rank, local_rank, world):
     ctx.profile_enable(False)
     n_tiny, ms_tiny = ctx.profile_read(oc.K_COPY)
     bracket_us = 1e3 * ms_tiny / max(n_tiny, 1)
+    # A third pass, for the tensor-core matcher only: the same K steps with the kernel stamping the GPU
+    # timer when its first CTA starts and when its last CTA ends (no events): the time its CTAs occupy
+    # the device, without launch latency and event records.
+    span_us = None
+    if w.kind == "token" and not w.self_match and prof.get("match_tc", (0, 0.0))[0]:
+        ctx.profile_reset()
+        ctx.profile_enable(2)
+        for i in range(args.steps):
+            if i % 20 == 0:
+                torch.cuda._sleep(int(2.0e9 * 0.004))
+            step(i)
+        torch.cuda.synchronize()
+        n_span, ms_span = ctx.profile_span_read(oc.K_MATCH_TC)
+        ctx.profile_enable(False)
+        if n_span:
+            span_us = 1e3 * ms_span / n_span
 
     tokens_per_step = n_cand + n_units
     value = world * tokens_per_step * args.steps / (ms_total * 1e-3)
@@ -396,6 +412,12 @@ def run_ours(args, rank, local_rank, world):
                     # the same with the bracket's own cost (see timing.event_bracket_us) taken off the duration
                     "achieved_net_of_bracket": flops / (max(ops["match_tc"]["net_us"], 1e-3) * 1e-6) / 1e12,
                     "frac_net_of_bracket": flops / (max(ops["match_tc"]["net_us"], 1e-3) * 1e-6) / 1e12 / peak}
+        if span_us:
+            # first-CTA-entry -> last-CTA-exit by the GPU timer (oc_profile_span_read): device occupancy only
+            roofline["device_span_us"] = span_us
+            roofline["achieved_device_span"] = flops / (span_us * 1e-6) / 1e12
+            roofline["frac_device_span"] = roofline["achieved_device_span"] / peak
+            roofline["frac_device_span_of_nominal"] = roofline["achieved_device_span"] / NOMINAL["bf16_tflops"]
     else:
         dom = max((k for k in ops if k in alg_bytes), key=lambda k: ops[k]["share"])
         roofline = {"kernel": dom, "bound": "hbm", "achieved": ops[dom]["GB/s"], "peak": peaks["hbm_gbs"],

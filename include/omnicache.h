@@ -160,13 +160,24 @@ oc_status oc_device_status(oc_ctx* ctx, int* code);
  * afterwards oc_device_status() reports OC_ERR_TIMEOUT once, and the context works as before. */
 oc_status oc_selftest_bounded_wait(oc_ctx* ctx, unsigned int limit_us, void* stream);
 
-/* Launch counters and optional per-kernel timers.  Counters always run.  With timers enabled each
- * kernel launch is bracketed by CUDA events on the caller's stream; oc_profile_read waits for the
- * recorded events and returns the number of launches and their summed device time since the last
- * reset.  total_ms is 0 when timers were off. */
+/* Launch counters and optional per-kernel timers.  Counters always run.  oc_profile_enable takes
+ * 0 (timers off), 1 (each kernel launch is bracketed by CUDA events on the caller's stream) or 2
+ * (device-side spans of the tensor-core matcher, see oc_profile_span_read; no events).
+ * oc_profile_read waits for the recorded events and returns the number of launches and their
+ * summed device time since the last reset.  total_ms is 0 when the event timers were off. */
 oc_status oc_profile_enable(oc_ctx* ctx, int on);
 oc_status oc_profile_reset(oc_ctx* ctx);
 oc_status oc_profile_read(oc_ctx* ctx, int kernel_id, int64_t* launches, double* total_ms);
+
+/* Device-side span of the tensor-core matcher (kernel_id must be OC_K_MATCH_TC).  With
+ * oc_profile_enable(ctx, 2) every launch of that kernel stamps the GPU's nanosecond timer when its
+ * first CTA starts and when its last CTA ends (two atomics per CTA; no events are recorded in this
+ * mode).  oc_profile_span_read synchronises the device and returns how many launches were stamped
+ * since the last reset (at most the 256 most recent are kept) and the sum of their spans.  A span
+ * leaves out what an event bracket adds around a kernel (launch latency, the event records
+ * themselves): it is the time the kernel's CTAs occupy the device.  The paper has no counterpart;
+ * this is a measurement aid. */
+oc_status oc_profile_span_read(oc_ctx* ctx, int kernel_id, int64_t* launches, double* total_ms);
 
 /* ---------------------------------------------------------------------------------------------
  * The hot path

@@ -197,6 +197,10 @@ oc_status oc_create(oc_ctx** out, int device, size_t workspace_bytes) {
     c->device = device; c->sm_count = prop.multiProcessorCount;
     if (cudaMalloc(&c->d_status, 256) != cudaSuccess) { delete c; cudaGetLastError(); return OC_ERR_OOM; }
     cudaMemset(c->d_status, 0, 256);
+    if (cudaMalloc(&c->d_span, 512 * sizeof(unsigned long long)) != cudaSuccess) {
+        cudaFree(c->d_status); delete c; cudaGetLastError(); return OC_ERR_OOM;
+    }
+    cudaMemset(c->d_span, 0, 512 * sizeof(unsigned long long));
     if (workspace_bytes) {
         if (cudaMalloc(&c->workspace, workspace_bytes) != cudaSuccess) {
             cudaFree(c->d_status); delete c; cudaGetLastError(); return OC_ERR_OOM;
@@ -218,6 +222,7 @@ oc_status oc_destroy(oc_ctx* c) {
     tc_cache_free(c);
     cudaFree(c->stage);
     cudaFree(c->workspace);
+    cudaFree(c->d_span);
     cudaFree(c->d_status);
     delete c;
     return cuda_ok(cudaGetLastError());
@@ -243,7 +248,8 @@ oc_status oc_selftest_bounded_wait(oc_ctx* c, unsigned int limit_us, void* strea
 
 oc_status oc_profile_enable(oc_ctx* c, int on) {
     if (!c) return OC_ERR_INVALID_ARG;
-    c->profile_on = on != 0;
+    c->profile_on = on == 1;
+    c->span_on = on == 2;
     return OC_OK;
 }
 
@@ -261,6 +267,7 @@ oc_status oc_profile_reset(oc_ctx* c) {
     if (!c) return OC_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);
     for (int k = 0; k < OC_K_COUNT; ++k) { drain(c, k); c->prof[k].launches = 0; c->prof[k].total_ms = 0.0; }
+    c->span_count = 0;
     return OC_OK;
 }
 
@@ -270,6 +277,27 @@ oc_status oc_profile_read(oc_ctx* c, int k, int64_t* launches, double* total_ms)
     drain(c, k);
     if (launches) *launches = c->prof[k].launches;
     if (total_ms) *total_ms = c->prof[k].total_ms;
+    return OC_OK;
+}
+
+oc_status oc_profile_span_read(oc_ctx* c, int k, int64_t* launches, double* total_ms) {
+    if (!c || k < 0 || k >= OC_K_COUNT) return OC_ERR_INVALID_ARG;
+    if (k != OC_K_MATCH_TC) return OC_ERR_UNSUPPORTED;
+    DeviceGuard guard(c->device);
+    if (!guard.ok || cudaDeviceSynchronize() != cudaSuccess) return OC_ERR_CUDA;
+    const long long n = c->span_count < 256 ? c->span_count : 256;
+    std::vector<unsigned long long> h(512);
+    if (cudaMemcpy(h.data(), c->d_span, 512 * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return OC_ERR_CUDA;
+    double ns = 0.0;
+    long long counted = 0;
+    for (long long i = 0; i < n; ++i) {
+        const long long slot = (c->span_count - 1 - i) & 255;
+        const unsigned long long entry = ~h[2 * slot], exit = h[2 * slot + 1];
+        if (h[2 * slot] != 0 && exit >= entry) { ns += (double)(exit - entry); ++counted; }
+    }
+    if (launches) *launches = counted;
+    if (total_ms) *total_ms = ns * 1e-6;
     return OC_OK;
 }
 

@@ -31,7 +31,10 @@ struct oc_ctx {
     void* workspace = nullptr;
     size_t workspace_bytes = 0;
     int* d_status = nullptr;                 // device status word (first device-side error)
-    bool profile_on = false;
+    bool profile_on = false;                 // event brackets around every launch
+    bool span_on = false;                    // device-side spans of the tensor-core matcher instead
+    unsigned long long* d_span = nullptr;    // 256 slots of {~first entry, last exit} in GPU-timer ns
+    long long span_count = 0;                // launches stamped since the last reset
     oc::KernelProf prof[OC_K_COUNT];
     std::vector<cudaEvent_t> free_events;
     std::map<int, oc::LayerEntry> layers;    // Layered Cache store

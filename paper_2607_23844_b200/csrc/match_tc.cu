@@ -102,6 +102,7 @@ struct TcScalars {
     const float* inv_norm;
     unsigned long long* keys;
     float* aux;
+    unsigned long long* span;            // nullable: {~first entry, last exit} of this launch, GPU-timer ns
     int* status;
 };
 struct TcParams {
@@ -420,6 +421,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     const uint32_t tiles_base = smem_u32(smem);
     const TcScalars& P = KP.s;
+    if (P.span && threadIdx.x == 0) atomicMax(P.span, ~global_ns());
     // First touches of parameter space miss the constant cache (several hundred cycles each, and
     // one after the other when a lone warp meets them on its way to the first copy): every warp
     // reads one word per 64 bytes of the scalars now, as independent loads.
@@ -759,6 +761,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         else
             asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
+    if (P.span && threadIdx.x == 0) atomicMax(P.span + 1, global_ns());
 }
 
 // ---- self-test of the bounded wait ---------------------------------------------------------------
@@ -992,6 +995,11 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
     P.n_stages = p.n_stages; P.stage_bytes = p.stage_bytes;
     P.units_per_group = (int)g.units_per_group; P.reps_per_group = (int)g.reps_per_group;
     P.inv_norm = inv_norm; P.keys = keys; P.aux = aux_sim; P.status = ctx->d_status;
+    if (ctx->span_on) {
+        P.span = ctx->d_span + 2 * (ctx->span_count & 255);
+        ++ctx->span_count;
+        if (cudaMemsetAsync(P.span, 0, 2 * sizeof(unsigned long long), s) != cudaSuccess) return OC_ERR_CUDA;
+    }
     // one walker (CTA or CTA pair) per SM (pair of SMs), or one per piece when there are fewer pieces
     long long walkers = p.items;
     const int cap = p.pair ? pair_walkers : ctx->sm_count;

@@ -29,7 +29,8 @@ K_COUNT = 12
 EXPORTS = (
     "oc_status_str", "oc_layout_check", "oc_layout_counts", "oc_match_workspace_bytes",
     "oc_rows_from_layout", "oc_layer_cache_would_hit", "oc_kernel_name", "oc_create", "oc_destroy",
-    "oc_device_status", "oc_profile_enable", "oc_profile_reset", "oc_profile_read", "oc_match",
+    "oc_device_status", "oc_profile_enable", "oc_profile_reset", "oc_profile_read", "oc_profile_span_read",
+    "oc_match",
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
     "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
 )
@@ -72,6 +73,7 @@ _lib.oc_selftest_bounded_wait.argtypes = [_vp, C.c_uint, _vp]
 _lib.oc_profile_enable.argtypes = [_vp, _i]
 _lib.oc_profile_reset.argtypes = [_vp]
 _lib.oc_profile_read.argtypes = [_vp, _i, _vp, _vp]
+_lib.oc_profile_span_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_match.argtypes = [_vp] * 8
 _lib.oc_select.argtypes = [_vp, _vp, _vp, _vp, _i, _f, _i64, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.oc_gather.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp]
@@ -252,7 +254,9 @@ class Context:
         """Makes a bounded device-side wait run out on purpose (see oc_selftest_bounded_wait)."""
         _chk(_lib.oc_selftest_bounded_wait(self._h, limit_us, _stream(stream)), "oc_selftest_bounded_wait")
 
-    def profile_enable(self, on: bool) -> None:
+    def profile_enable(self, on) -> None:
+        """False/0: timers off; True/1: CUDA events around every launch; 2: device-side spans of the
+        tensor-core matcher (read with profile_span_read)."""
         _chk(_lib.oc_profile_enable(self._h, int(on)), "oc_profile_enable")
 
     def profile_reset(self) -> None:
@@ -261,6 +265,12 @@ class Context:
     def profile_read(self, kernel_id: int) -> tuple[int, float]:
         n, ms = C.c_int64(), C.c_double()
         _chk(_lib.oc_profile_read(self._h, kernel_id, C.byref(n), C.byref(ms)), "oc_profile_read")
+        return n.value, ms.value
+
+    def profile_span_read(self, kernel_id: int) -> tuple[int, float]:
+        """(launches stamped, summed first-CTA-entry -> last-CTA-exit time in ms); see profile_enable(2)."""
+        n, ms = C.c_int64(), C.c_double()
+        _chk(_lib.oc_profile_span_read(self._h, kernel_id, C.byref(n), C.byref(ms)), "oc_profile_span_read")
         return n.value, ms.value
 
     def launches(self) -> dict[str, int]:

@@ -359,6 +359,31 @@ def test_determinism_and_profile_counters(oc, oracle):
         assert ctx.profile_read(oc.K_NORMS) == (0, 0.0)
 
 
+def test_device_span_of_the_tensor_core_matcher(oc, oracle):
+    """Span mode stamps first-CTA entry and last-CTA exit of every match_tc launch; the span is
+    positive, shorter than the event bracket around the same kernel, and results are unchanged."""
+    w = inputs.sd3_token_cache(seed=8, B=2, H=32, W=32, C=256)
+    L, _ = H.layouts(oc, oracle, w)
+    x_dev = H.to_dev(w.x)
+    with H.make_ctx(oc, L) as ctx:
+        ctx.profile_enable(1)
+        a = H.gpu_match(oc, ctx, L, x_dev)
+        for _ in range(4):
+            H.gpu_match(oc, ctx, L, x_dev)
+        n_ev, ms_ev = ctx.profile_read(oc.K_MATCH_TC)
+        ctx.profile_reset()
+        ctx.profile_enable(2)
+        for _ in range(5):
+            b = H.gpu_match(oc, ctx, L, x_dev)
+        n_sp, ms_sp = ctx.profile_span_read(oc.K_MATCH_TC)
+        ctx.profile_enable(0)
+        assert n_ev == 5 and n_sp == 5
+        assert 0.0 < ms_sp < ms_ev
+        assert torch.equal(a["best_sim"], b["best_sim"]) and torch.equal(a["best_idx"], b["best_idx"])
+        with pytest.raises(oc.OmniCacheError):
+            ctx.profile_span_read(oc.K_SELECT)
+
+
 def test_runtime_argument_errors_launch_nothing(oc, oracle):
     w = inputs.sd3_token_cache(seed=5, B=1, H=16, W=16, C=64)
     L, Lo = H.layouts(oc, oracle, w)
