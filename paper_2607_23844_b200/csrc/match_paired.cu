@@ -46,6 +46,7 @@ template <int DT, int LPR>
 __global__ void __launch_bounds__(PAIR_THREADS)
 frame_pair_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float eps,
                   float* __restrict__ pos_sim, float4* __restrict__ partial, int pos_per_cta) {
+    pdl_enter();
     __shared__ float sh[PAIR_THREADS];
     const int q = blockIdx.y;                       // pair index b*(T-1) + (t-1)
     const int b = q / (T - 1), t = q - b * (T - 1) + 1;
@@ -101,6 +102,7 @@ template <int DT, int LPR, int CPL>
 __global__ void __launch_bounds__(PAIR_THREADS)
 frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float eps, int seg_len, int n_seg,
                    float* __restrict__ pos_sim, float4* __restrict__ partial) {
+    pdl_enter();
     extern __shared__ float4 warp_part[];                 // [seg_len][PAIR_THREADS / 32]
     constexpr int GROUPS = PAIR_THREADS / LPR, WARPS = PAIR_THREADS / 32;
     const int b = blockIdx.y / n_seg, seg = blockIdx.y - b * n_seg;
@@ -187,6 +189,7 @@ __global__ void __launch_bounds__(PAIR_THREADS)
 frame_finalize_kernel(const float4* __restrict__ partial, int n_tiles, int B, int T, int P, int stat,
                       float eps, float* __restrict__ pair_ws, float* __restrict__ pair_sim,
                       float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
+    pdl_enter();
     const int i = blockIdx.x * (PAIR_THREADS / 32) + (threadIdx.x >> 5);     // frame index b*T + t
     const int lane = threadIdx.x & 31;
     if (i >= B * T) return;                                                   // whole warps leave together
@@ -208,12 +211,12 @@ template <int DT>
 static void frame_dispatch(int lpr, dim3 grid, cudaStream_t s, const uint8_t* x, int T, int P, int cpr, float eps,
                            float* pos_sim, float4* partial, int ppc) {
     switch (lpr) {
-        case 1:  frame_pair_kernel<DT, 1><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        case 2:  frame_pair_kernel<DT, 2><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        case 4:  frame_pair_kernel<DT, 4><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        case 8:  frame_pair_kernel<DT, 8><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        case 16: frame_pair_kernel<DT, 16><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        default: frame_pair_kernel<DT, 32><<<grid, PAIR_THREADS, 0, s>>>(x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 1:  OC_LAUNCH((frame_pair_kernel<DT, 1>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 2:  OC_LAUNCH((frame_pair_kernel<DT, 2>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 4:  OC_LAUNCH((frame_pair_kernel<DT, 4>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 8:  OC_LAUNCH((frame_pair_kernel<DT, 8>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 16: OC_LAUNCH((frame_pair_kernel<DT, 16>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        default: OC_LAUNCH((frame_pair_kernel<DT, 32>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
     }
 }
 
@@ -254,8 +257,8 @@ size_t frame_workspace_bytes(const Geo& g) {
 template <int DT>
 static void march_dispatch(int lpr, dim3 grid, size_t smem, cudaStream_t s, const uint8_t* x, int T, int P, int cpr,
                            float eps, int seg_len, int n_seg, float* pos_sim, float4* partial) {
-#define OC_MARCH(L) do { if (cpr <= 5 * L) frame_march_kernel<DT, L, 5><<<grid, PAIR_THREADS, smem, s>>>(x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial); \
-                         else frame_march_kernel<DT, L, 8><<<grid, PAIR_THREADS, smem, s>>>(x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial); } while (0)
+#define OC_MARCH(L) do { if (cpr <= 5 * L) OC_LAUNCH((frame_march_kernel<DT, L, 5>), grid, PAIR_THREADS, smem, s, x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial); \
+                         else OC_LAUNCH((frame_march_kernel<DT, L, 8>), grid, PAIR_THREADS, smem, s, x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial); } while (0)
     switch (lpr) {
         case 4: OC_MARCH(4); break; case 8: OC_MARCH(8); break; case 16: OC_MARCH(16); break; default: OC_MARCH(32); break;
     }
@@ -295,7 +298,7 @@ static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, co
     {
         Scope scope(ctx, OC_K_FRAME_FIN, s);
         const int warps = PAIR_THREADS / 32;
-        frame_finalize_kernel<<<(unsigned)((g.B * g.T + warps - 1) / warps), PAIR_THREADS, 0, s>>>(
+        OC_LAUNCH((frame_finalize_kernel), (unsigned)((g.B * g.T + warps - 1) / warps), PAIR_THREADS, 0, s, 
             partial, f.n_tiles, g.B, g.T, P, g.frame_stat, g.eps, pair_ws, pair_sim, best_sim, best_idx);
     }
     return last_launch_status();
@@ -318,6 +321,7 @@ template <int DT, int LPR, int NCMAX>
 __global__ void __launch_bounds__(PAIR_THREADS)
 block_partial_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr, int sy, int sx, int oy, int ox,
                      float* __restrict__ partial, int rec /*floats per (cell,t)*/) {
+    pdl_enter();
     const int bt = blockIdx.y;
     const int cells_x = W / sx, cells = (H / sy) * cells_x;
     const int groups = PAIR_THREADS / LPR;
@@ -376,6 +380,7 @@ template <int DT, int LPR, int CPL>
 __global__ void __launch_bounds__(PAIR_THREADS)
 block_partial_reg_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr, int sy, int sx, int oy, int ox,
                          float* __restrict__ partial, int rec) {
+    pdl_enter();
     constexpr int NC = 3;
     const int bt = blockIdx.y;
     const int cells_x = W / sx, cells = (H / sy) * cells_x;
@@ -433,6 +438,7 @@ block_partial_reg_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int
 __global__ void __launch_bounds__(PAIR_THREADS)
 block_finalize_kernel(const float* __restrict__ partial, int B, int T, int H, int W, int sy, int sx, int oy, int ox,
                       int rec, float eps, float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
+    pdl_enter();
     const long long n = (long long)B * H * W;
     const long long i = (long long)blockIdx.x * PAIR_THREADS + threadIdx.x;
     if (i >= n) return;
@@ -464,8 +470,8 @@ size_t block_workspace_bytes(const Geo& g) {
 
 template <int DT>
 static void block_dispatch(int lpr, dim3 grid, cudaStream_t s, const uint8_t* x, const Geo& g, int cpr, float* partial, int rec) {
-#define OC_BLK(L) do { if (g.sy * g.sx - 1 <= 3) block_partial_kernel<DT, L, 3><<<grid, PAIR_THREADS, 0, s>>>(x, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec); \
-                       else block_partial_kernel<DT, L, 15><<<grid, PAIR_THREADS, 0, s>>>(x, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec); } while (0)
+#define OC_BLK(L) do { if (g.sy * g.sx - 1 <= 3) OC_LAUNCH((block_partial_kernel<DT, L, 3>), grid, PAIR_THREADS, 0, s, x, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec); \
+                       else OC_LAUNCH((block_partial_kernel<DT, L, 15>), grid, PAIR_THREADS, 0, s, x, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec); } while (0)
     switch (lpr) {
         case 1: OC_BLK(1); break; case 2: OC_BLK(2); break; case 4: OC_BLK(4); break;
         case 8: OC_BLK(8); break; case 16: OC_BLK(16); break; default: OC_BLK(32); break;
@@ -492,7 +498,7 @@ oc_status launch_match_block(oc_ctx* ctx, const Geo& g, const void* x, float* be
         LaunchScope scope(ctx, OC_K_BLOCK, s);
         const uint8_t* xb = (const uint8_t*)x;
         if (reg_variant) {
-#define OC_BLKR(DTV, L) block_partial_reg_kernel<DTV, L, 5><<<grid, PAIR_THREADS, 0, s>>>(xb, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec)
+#define OC_BLKR(DTV, L) OC_LAUNCH((block_partial_reg_kernel<DTV, L, 5>), grid, PAIR_THREADS, 0, s, xb, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, partial, rec)
             if (g.dtype == OC_DTYPE_BF16) {
                 switch (lpr) { case 4: OC_BLKR(OC_DTYPE_BF16, 4); break; case 8: OC_BLKR(OC_DTYPE_BF16, 8); break;
                                case 16: OC_BLKR(OC_DTYPE_BF16, 16); break; default: OC_BLKR(OC_DTYPE_BF16, 32); break; }
@@ -510,7 +516,7 @@ oc_status launch_match_block(oc_ctx* ctx, const Geo& g, const void* x, float* be
     {
         const long long n = (long long)g.B * g.H * g.W;
         LaunchScope scope(ctx, OC_K_BLOCK_FIN, s);
-        block_finalize_kernel<<<(unsigned)((n + PAIR_THREADS - 1) / PAIR_THREADS), PAIR_THREADS, 0, s>>>(
+        OC_LAUNCH((block_finalize_kernel), (unsigned)((n + PAIR_THREADS - 1) / PAIR_THREADS), PAIR_THREADS, 0, s, 
             partial, g.B, g.T, g.H, g.W, g.sy, g.sx, g.oy, g.ox, rec, g.eps, best_sim, best_idx);
     }
     return last_launch_status();
