@@ -467,11 +467,18 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         }
     }
-    tc_fence_before();
-    __syncthreads();
-    if (PAIR) cluster_sync_all();          // the other CTA's barriers exist before anything signals them
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    // The producer warp initialised the barriers itself (its lane 0, above), so in the single-CTA form
+    // it does not wait for the rest of the set-up (the TMEM allocation): it goes on to decode its
+    // first piece and issue its first stage, and joins this barrier from inside its loop.  In a pair the other
+    // CTA's barriers must exist first, so everybody meets here.
+    const bool early_producer = !PAIR && warp == 0;
+    __syncwarp();
+    if (!early_producer) {
+        tc_fence_before();
+        __syncthreads();
+        if (PAIR) cluster_sync_all();      // the other CTA's barriers exist before anything signals them
+        tc_fence_after();
+    }
     const int STAGES = P.n_stages, STAGE_BYTES = P.stage_bytes;
     const bool dbl = P.tpp == 1;
 
@@ -479,6 +486,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     Piece c;
     const int bwA = 1 << P.bwA_log2, bwQ = 1 << P.bwQ_log2;
     const int my_rep = P.my_rep, mx_rep = P.mx_rep;
+    const uint32_t tmem_base = early_producer ? 0u : *tmem_slot;    // (the producer warp never touches TMEM)
 
     if (warp == 0) {
         // ================================ TMA producer ==========================================
@@ -488,6 +496,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         int stage = 0; uint32_t phase = 0;
         uint32_t armed = 0;                           // stages with a copy possibly still in flight
         bool ok = true;
+        bool joined = !early_producer;                // whether this warp has met the set-up barrier yet
         while (ok && walk.next(P, c)) {
             const int nq_mine = PAIR ? (c.nq >> 1) : c.nq;             // quanta this CTA fetches
             const int nA = P.a_merged ? 1 : P.tpp, nQ = P.q_merged ? 1 : nq_mine;   // boxes per stage
@@ -524,8 +533,10 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 if (active) tma_load_4d<PAIR>(tiles_base + stage * STAGE_BYTES + dst_off, map, kb * BK, w, h, c.bt, full);
                 armed |= 1u << stage;
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                if (!joined) { __syncthreads(); joined = true; }   // first stage on its way: meet the others
             }
         }
+        if (!joined) { __syncthreads(); joined = true; }
         if (!ok && lane == 0) {
             atomicCAS(P.status, 0, OC_ERR_TIMEOUT);
             *abort_flag = 1;
