@@ -3,7 +3,8 @@
 TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's CPU-baseline leg may
 import this package; the product package never does.  The arithmetic lives in
 ``omnicache_oracle.c`` (plain C, double precision, compiled here with gcc); this file only builds
-it, marshals NumPy arrays into it and keeps the dictionary behind the Layered Cache oracle.
+it, marshals NumPy arrays into it and keeps the dictionary behind the Layered Cache oracle and the
+few lines of the Layered Cache schedule proposal (Algorithm 1).
 Nothing in here imports the CUDA package.
 """
 from __future__ import annotations
@@ -284,6 +285,35 @@ class LayerCache:
 
     def clear(self) -> None:
         self.store.clear()
+
+
+def schedule_proposal(L, Q, s_r: float):
+    """Cache schedule proposal (Algorithm 1, Section 3.4), step by step in the paper's notation.
+
+    L[i], Q[i]: latency and quality loss of candidate i (a layer-timestep pair); s_r: target speedup.
+    Scores w = Q / L; candidates sorted by increasing w (equal scores: lower candidate index first,
+    a point the paper leaves open); TargetSave = (1 - 1/s_r) * sum(L); candidates are taken in that
+    order while Saved < TargetSave, each adding its L to Saved.  Returns the taken candidate indices
+    in the order taken (every one of them carries the same cache interval N, which is not used to
+    choose).  Double precision throughout."""
+    L = [float(v) for v in L]
+    Q = [float(v) for v in Q]
+    assert len(L) == len(Q) and all(v > 0.0 for v in L) and s_r >= 1.0
+    w = [Q[i] / L[i] for i in range(len(L))]
+    order = sorted(range(len(L)), key=lambda i: (w[i], i))
+    total = 0.0
+    for v in L:
+        total += v
+    target_save = (1.0 - 1.0 / s_r) * total
+    saved = 0.0
+    chosen = []
+    k = 0
+    while saved < target_save and k < len(order):
+        i = order[k]
+        k += 1
+        chosen.append(i)
+        saved += L[i]
+    return chosen
 
 
 def num_threads() -> int:

@@ -492,6 +492,61 @@ def test_layer_cache_rule(oracle):
 
 
 # ---------------------------------------------------------------------------------------------
+# Layered Cache schedule proposal (Algorithm 1)
+# ---------------------------------------------------------------------------------------------
+def test_schedule_proposal_hand_cases(oracle):
+    path = os.path.join(os.path.dirname(__file__), "golden", "schedule_hand_cases.txt")
+    n = 0
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        Ls, Qs, s_r, exp = [f.strip() for f in line.split(";")]
+        got = oracle.schedule_proposal([float(v) for v in Ls.split()], [float(v) for v in Qs.split()], float(s_r))
+        assert got == [int(v) for v in exp.split()], line
+        n += 1
+    assert n == 7
+
+
+def test_schedule_proposal_is_the_shortest_sorted_prefix_that_meets_the_budget(oracle):
+    """Exact-rational restatement: sort by (Q/L, index) with Fractions, take the shortest prefix whose
+    latency sum reaches (1 - 1/s_r) * sum(L).  Inputs are small dyadic rationals, so the oracle's
+    doubles are exact too and the two must agree to the index."""
+    from fractions import Fraction as Fr
+    rng = np.random.default_rng(5)
+    for trial in range(200):
+        n = int(rng.integers(1, 9))
+        L = [Fr(int(rng.integers(1, 64)), 8) for _ in range(n)]
+        Q = [Fr(int(rng.integers(0, 64)), 16) for _ in range(n)]
+        s_r = Fr(int(rng.integers(8, 64)), 8)                       # 1 .. 8 in eighths
+        order = sorted(range(n), key=lambda i: (Q[i] / L[i], i))
+        target = (1 - 1 / s_r) * sum(L)
+        exp, saved = [], Fr(0)
+        for i in order:
+            if not saved < target:
+                break
+            exp.append(i); saved += L[i]
+        got = oracle.schedule_proposal([float(v) for v in L], [float(v) for v in Q], float(s_r))
+        # 1/s_r may round in binary; the budget then moves by one ulp, which only matters when a prefix
+        # sum lands exactly on it: accept either side in that single case
+        if got != exp:
+            pref = [sum(L[i] for i in order[:k]) for k in range(n + 1)]
+            assert any(p == target for p in pref) and abs(len(got) - len(exp)) == 1 and got[:len(exp)] == exp[:len(got)]
+        else:
+            assert got == exp
+        # invariants that hold whatever the rounding
+        assert got == order[:len(got)]
+        if got:
+            assert sum(L[i] for i in got[:-1]) < target or abs(float(sum(L[i] for i in got[:-1]) - target)) < 1e-12
+    assert oracle.schedule_proposal([1.0, 2.0], [0.5, 0.1], 1.0) == []
+    assert oracle.schedule_proposal([1.0, 2.0], [0.5, 0.1], 1e9) == [1, 0]
+    # a larger target speedup never takes fewer candidates
+    L = list(rng.uniform(0.5, 4.0, 30)); Q = list(rng.uniform(0.0, 1.0, 30))
+    sizes = [len(oracle.schedule_proposal(L, Q, s)) for s in (1.0, 1.1, 1.5, 2.0, 3.0, 10.0)]
+    assert sizes == sorted(sizes) and sizes[0] == 0 and sizes[-1] <= 30
+
+
+# ---------------------------------------------------------------------------------------------
 # input recipes: sanity bands (properties of the generators, not parity targets)
 # ---------------------------------------------------------------------------------------------
 def test_input_recipes_shapes_and_bands(oracle):
