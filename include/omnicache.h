@@ -274,6 +274,24 @@ oc_status oc_layer_cache_clear(oc_ctx* ctx);
 oc_status oc_match_frame_noalloc(int device, const oc_layout* layout, const void* x, float* best_sim,
                                  int32_t* best_idx, float* pair_sim, void* stream);
 
+/* Layered Cache schedule proposal (Algorithm 1, "Cache Schedule Proposal", Section 3.4).  Host-side;
+ * launches nothing and needs no context.
+ *   latency[i], quality_loss[i]  the profiled L and Q of candidate i (a layer-timestep pair), n of
+ *                                them, host arrays; every latency must be > 0 and finite, every
+ *                                quality loss finite
+ *   target_speedup               s_r >= 1
+ * Candidates are ranked by w = Q / L ascending (equal scores: lower index first) and taken in that
+ * order while Saved < (1 - 1/s_r) * sum(L), each adding its L to Saved, all in double precision.
+ *   chosen     host array of capacity n: receives the taken candidate indices in the order taken
+ *              (each is to be cached with the caller's interval N, which does not influence the choice)
+ *   n_chosen   receives how many were taken
+ *   saved      nullable: receives the accumulated latency of the taken candidates
+ * OC_ERR_INVALID_ARG on null pointers, n < 0, s_r < 1 or non-finite / non-positive inputs; nothing
+ * is written then.  The refinement pass over the model graph (Algorithm 2) is not part of this
+ * library. */
+oc_status oc_schedule_propose(const double* latency, const double* quality_loss, int64_t n, double target_speedup,
+                              int32_t* chosen, int64_t* n_chosen, double* saved);
+
 /* One whole cache-wrapped layer call on HOST buffers, for callers that keep activations in host
  * memory: copies x_host (layer input) and cache_host (previous output, same shape) to library-owned
  * device staging, runs match -> select -> gather -> restore with the identity as the wrapped layer

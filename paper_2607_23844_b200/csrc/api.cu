@@ -5,6 +5,8 @@
 
 #include <new>
 
+#include <algorithm>
+#include <cmath>
 #include "common.cuh"
 
 namespace oc {
@@ -418,6 +420,32 @@ oc_status oc_layer_cache_clear(oc_ctx* c) {
 }
 
 // ---- host-buffer call --------------------------------------------------------------------------
+oc_status oc_schedule_propose(const double* latency, const double* quality_loss, int64_t n, double target_speedup,
+                              int32_t* chosen, int64_t* n_chosen, double* saved) {
+    if (!latency || !quality_loss || !chosen || !n_chosen || n < 0 || n > 0x7FFFFFFF) return OC_ERR_INVALID_ARG;
+    if (!(target_speedup >= 1.0)) return OC_ERR_INVALID_ARG;
+    double total = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (!(latency[i] > 0.0) || !std::isfinite(latency[i]) || !std::isfinite(quality_loss[i])) return OC_ERR_INVALID_ARG;
+        total += latency[i];
+    }
+    std::vector<double> w((size_t)n);
+    std::vector<int32_t> order((size_t)n);
+    for (int64_t i = 0; i < n; ++i) { w[(size_t)i] = quality_loss[i] / latency[i]; order[(size_t)i] = (int32_t)i; }
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return w[(size_t)a] < w[(size_t)b]; });
+    const double target_save = (1.0 - 1.0 / target_speedup) * total;
+    double acc = 0.0;
+    int64_t k = 0;
+    while (acc < target_save && k < n) {
+        const int32_t i = order[(size_t)k];
+        chosen[k++] = i;
+        acc += latency[i];
+    }
+    *n_chosen = k;
+    if (saved) *saved = acc;
+    return OC_OK;
+}
+
 oc_status oc_cache_step_host(oc_ctx* c, const oc_layout* layout, int mode, float thr, int64_t n_reuse,
                              const void* x_host, const void* cache_host, void* out_host, int32_t* kept_count_host,
                              void* stream) {

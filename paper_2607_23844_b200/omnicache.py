@@ -33,6 +33,7 @@ EXPORTS = (
     "oc_match",
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
     "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
+    "oc_schedule_propose",
 )
 
 
@@ -82,6 +83,7 @@ _lib.oc_layer_cache_put.argtypes = [_vp, _i, _i, _vp, C.c_size_t, _vp]
 _lib.oc_layer_cache_get.argtypes = [_vp, _i, _i, _i, _vp, _vp, _vp, _vp]
 _lib.oc_layer_cache_clear.argtypes = [_vp]
 _lib.oc_cache_step_host.argtypes = [_vp, _vp, _i, _f, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.oc_schedule_propose.argtypes = [_vp, _vp, _i64, C.c_double, _vp, _vp, _vp]
 _lib.oc_match_frame_noalloc.argtypes = [_i, _vp, _vp, _vp, _vp, _vp, _vp]
 NOALLOC_SCRATCH_BYTES = 1 << 20
 
@@ -200,6 +202,21 @@ def _stream(stream) -> int:
     if stream is None:
         return torch.cuda.current_stream().cuda_stream
     return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+def schedule_propose(latency, quality_loss, target_speedup: float):
+    """Layered Cache schedule proposal (Algorithm 1).  Returns (chosen candidate indices in the order
+    taken, saved latency).  Host-side: no device work."""
+    import numpy as np
+    L = np.ascontiguousarray(latency, dtype=np.float64)
+    Q = np.ascontiguousarray(quality_loss, dtype=np.float64)
+    if L.shape != Q.shape or L.ndim != 1:
+        raise ValueError("latency and quality_loss must be 1-D arrays of one length")
+    chosen = np.empty(max(L.size, 1), dtype=np.int32)
+    n, saved = C.c_int64(), C.c_double()
+    _chk(_lib.oc_schedule_propose(L.ctypes.data_as(_vp), Q.ctypes.data_as(_vp), L.size, float(target_speedup),
+                                  chosen.ctypes.data_as(_vp), C.byref(n), C.byref(saved)), "oc_schedule_propose")
+    return chosen[:n.value].tolist(), saved.value
 
 
 def match_frame_noalloc(device: int, layout: Layout, x, best_sim, best_idx, pair_sim=None, stream=None,

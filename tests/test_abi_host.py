@@ -133,6 +133,37 @@ def test_null_context_and_bad_arguments_are_rejected_before_any_launch(oc):
     assert lib.oc_create(C.byref(h), -1, 0) == oc.ERR_INVALID_ARG
 
 
+def test_schedule_proposal_matches_oracle(oc, oracle):
+    """Algorithm 1 is host logic: the library's answer must equal the oracle's to the index."""
+    import numpy as np
+    rng = np.random.default_rng(17)
+    for trial in range(300):
+        n = int(rng.integers(0, 40))
+        L = rng.uniform(0.05, 5.0, n)
+        Q = rng.uniform(0.0, 2.0, n)
+        if n > 3 and trial % 3 == 0:                       # ties in the score and zero losses
+            Q[1] = Q[0] / L[0] * L[1]; Q[2] = 0.0; Q[3] = 0.0
+        s_r = float(rng.choice([1.0, 1.05, 1.5, 2.0, 3.7, 50.0]))
+        got, saved = oc.schedule_propose(L, Q, s_r)
+        ref = oracle.schedule_proposal(L, Q, s_r)
+        assert got == ref
+        assert abs(saved - L[ref].sum()) < 1e-9
+    # the 28-layer x 25-step table of a DiT-sized model, as one call
+    L = rng.uniform(0.5, 2.0, 28 * 25); Q = rng.gamma(2.0, 0.1, 28 * 25)
+    got, saved = oc.schedule_propose(L, Q, 2.0)
+    assert got == oracle.schedule_proposal(L, Q, 2.0) and saved >= 0.5 * L.sum() > saved - L[got[-1]]
+    lib = oc._lib
+    one = C.c_void_p(16)
+    n_out = C.c_int64()
+    assert lib.oc_schedule_propose(None, one, 1, 2.0, one, C.byref(n_out), None) == oc.ERR_INVALID_ARG
+    bad = np.array([1.0, 0.0]); q = np.array([0.1, 0.1]); ch = np.empty(2, np.int32)
+    assert lib.oc_schedule_propose(bad.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), 2, 2.0,
+                                   ch.ctypes.data_as(C.c_void_p), C.byref(n_out), None) == oc.ERR_INVALID_ARG
+    ok = np.array([1.0, 1.0])
+    assert lib.oc_schedule_propose(ok.ctypes.data_as(C.c_void_p), q.ctypes.data_as(C.c_void_p), 2, 0.5,
+                                   ch.ctypes.data_as(C.c_void_p), C.byref(n_out), None) == oc.ERR_INVALID_ARG
+
+
 def test_create_fails_loudly_without_a_device(oc):
     import torch
     if torch.cuda.is_available():
