@@ -585,7 +585,8 @@ def run_sweep(args):
 # SD3 shape at token-group counts 1, 2, 4, 8 (the setting of Appendix A.1's kernel comparison):
 # per-op device times.  One JSON line; an extra mode, not the default.
 # ---------------------------------------------------------------------------------------------------
-def run_token_groups(args):
+def run_token_groups(args, bases=None, metric="per-op device time, SD3 shape at token-group counts 1/2/4/8"):
+    """bases: list of (label, workload, patch grids); default: the SD3 shape at 1/2/4/8 token groups."""
     import torch
     from paper_2607_23844_b200 import build
     build.build()
@@ -607,7 +608,17 @@ def run_token_groups(args):
         e1.record(); torch.cuda.synchronize()
         return 1e3 * e0.elapsed_time(e1) / reps
 
-    base = inputs.sd3_token_cache()
+    if bases is None:
+        bases = [("sd3", inputs.sd3_token_cache(), ((1, 1), (2, 1), (2, 2), (4, 2)))]
+    results = []
+    for label, base, grids in bases:
+        results += _token_groups_one(args, oc, torch, dev, peaks, graph_time_us, label, base, grids)
+    print(json.dumps({"metric": metric, "unit": "us",
+                      "timing": "CUDA-graph replay per op over a ring of buffers larger than 4x L2",
+                      "data": "synthetic", "results": results}), flush=True)
+
+
+def _token_groups_one(args, oc, torch, dev, peaks, graph_time_us, label, base, grids):
     C = base.shape[-1]
     tensor_bytes = int(np.prod(base.shape)) * 2
     ring = max(2, -(-4 * L2_BYTES // (3 * tensor_bytes)))
@@ -616,7 +627,7 @@ def run_token_groups(args):
     outs = [torch.empty_like(xs[0]) for _ in range(ring)]
     reps = max(3, args.steps // 10)
     results = []
-    for gy, gx in ((1, 1), (2, 1), (2, 2), (4, 2)):
+    for gy, gx in grids:
         L = oc.Layout(oc.KIND_TOKEN, inputs.BF16, *base.shape, gy=gy, gx=gx)
         G, U, R = L.counts()
         n_units, n_cand = G * U, G * (U - R)
@@ -653,6 +664,7 @@ def run_token_groups(args):
              (("match", f_match), ("select", f_select), ("gather", f_gather), ("restore", f_restore))}
         flops = 2.0 * n_cand * R * C
         results.append({
+            "workload": label, "shape": list(base.shape), "match_GFLOP": flops / 1e9,
             "token_groups": gy * gx, "grid": [gy, gx], "groups": G, "units_per_group": U, "n_reuse_per_group": n_reuse,
             "match_us": t["match"], "select_us": t["select"], "gather_us": t["gather"], "restore_us": t["restore"],
             "selection_plus_restoration_us": t["select"] + t["gather"] + t["restore"],
@@ -661,9 +673,15 @@ def run_token_groups(args):
             "restore_frac_hbm": 2 * n_units * row_bytes / (t["restore"] * 1e-6) / 1e9 / peaks["hbm_gbs"]})
         assert ctx.device_status() == oc.OK
         ctx.close()
-    print(json.dumps({"metric": "per-op device time, SD3 shape at token-group counts 1/2/4/8", "unit": "us",
-                      "timing": "CUDA-graph replay per op over a ring of buffers larger than 4x L2",
-                      "shape": list(base.shape), "data": "synthetic", "results": results}), flush=True)
+    # patch-local against whole-frame matching (Hierarchical Caching, Section 3.3): cost ratios
+    t_global = results[0]["match_us"] if grids[0] == (1, 1) else None
+    for r in results:
+        if t_global:
+            r["match_time_ratio_vs_whole_frame"] = t_global / r["match_us"]
+            r["match_flop_ratio_vs_whole_frame"] = results[0]["match_GFLOP"] / r["match_GFLOP"]
+    del xs, caches, outs
+    torch.cuda.empty_cache()
+    return results
 
 
 
@@ -686,9 +704,17 @@ def main():
     if args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     rank, local_rank, world = sharding.env_rank_world()
-    if args.workload in ("svd_sweep", "sd3_groups"):
+    if args.workload in ("svd_sweep", "sd3_groups", "svd_patches"):
         if rank == 0:
-            (run_sweep if args.workload == "svd_sweep" else run_token_groups)(args)
+            if args.workload == "svd_sweep":
+                run_sweep(args)
+            elif args.workload == "sd3_groups":
+                run_token_groups(args)
+            else:
+                # patch-local Token Cache matching on the three SVD U-Net levels (per-frame groups cut into k x k patches)
+                grids = {0: ((1, 1), (2, 2), (4, 4), (6, 8)), 1: ((1, 1), (2, 2), (6, 8)), 2: ((1, 1), (3, 4))}
+                run_token_groups(args, [(f"svd_token_l{lv}", make_workload(f"svd_token_l{lv}"), grids[lv]) for lv in (0, 1, 2)],
+                                 metric="per-op device time, Token Cache on the SVD levels, whole-frame vs patch-local matching")
         return
     if args.impl == "reference":
         run_reference(args, rank)

@@ -267,7 +267,7 @@ __device__ __forceinline__ int block_scan_int(int v, int* sums /*[33]*/, int& to
     if (lane == 31) sums[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-        const int w = sums[lane];
+        const int w = lane < (int)(blockDim.x >> 5) ? sums[lane] : 0;     // (CTAs of fewer than 32 warps)
         int wi = w;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -282,7 +282,7 @@ __device__ __forceinline__ int block_scan_int(int v, int* sums /*[33]*/, int& to
     return sums[warp] + incl - v;
 }
 
-__global__ void __launch_bounds__(SEL_THREADS)
+__global__ void __launch_bounds__(1024)
 select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_t* __restrict__ best_idx,
                    int mode, float thr, int n_reuse, int y_stride,
                    int32_t* __restrict__ kept_idx, int32_t* __restrict__ kept_count,
@@ -295,10 +295,11 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     __shared__ int sh_ncand;
     __shared__ unsigned sh_kmin, sh_kmax;
 
+    const int NT = (int)blockDim.x;                             // 128..1024 threads, chosen by the host for the group size
     const int U = gm.units_per_group;
     const long long g = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31;
-    const int n_rounds = (U + SEL_THREADS - 1) / SEL_THREADS;
+    const int n_rounds = (U + NT - 1) / NT;
     const GroupView gv(gm, g);
 
     // ---- phase 0: every input is read once, coalesced, all loads issued before any is used --------
@@ -315,7 +316,7 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
 #pragma unroll
         for (int k = 0; k < PF; ++k) {
             if (r0 + k >= n_rounds) break;                          // (uniform: whole rounds that do not exist)
-            const int u = (r0 + k) * SEL_THREADS + tid;
+            const int u = (r0 + k) * NT + tid;
             gi[k] = u < U ? gv.index(gm, u) : -1;
         }
 #pragma unroll
@@ -327,7 +328,7 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
 #pragma unroll
         for (int k = 0; k < PF; ++k) {
             if (r0 + k >= n_rounds) break;
-            const int u = (r0 + k) * SEL_THREADS + tid;
+            const int u = (r0 + k) * NT + tid;
             if (u < U) {
                 unsigned key = 0;
                 if (gv.is_cand(gm, u)) {
@@ -371,11 +372,11 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
             const int n_pass = (nbits + 11) / 12;
             for (int pass = 0; pass < n_pass; ++pass) {
                 const int shift = 12 * (n_pass - 1 - pass);
-                for (int i = tid; i < 4096; i += SEL_THREADS) hist[i] = 0;
+                for (int i = tid; i < 4096; i += NT) hist[i] = 0;
                 __syncthreads();
                 const unsigned prefix = sh_prefix;                  // the digits fixed so far (high part of rel)
                 for (int r = 0; r < n_rounds; ++r) {
-                    const int u = r * SEL_THREADS + tid;
+                    const int u = r * NT + tid;
                     const unsigned key = u < U ? key_cache[u] : 0u;
                     if (key != 0) {
                         const unsigned rel = key - base;
@@ -384,20 +385,21 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
                     }
                 }
                 __syncthreads();
-                // thread t owns bins 4095-4t .. 4092-4t (descending): where does the running count reach rem?
+                // thread t owns bins 4095 - bpt*t downwards (bpt = 4096 / threads): where does the running
+                // count reach rem?
                 const unsigned rem = sh_remaining;
-                unsigned c[4], tot = 0;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { c[i] = hist[4095 - 4 * tid - i]; tot += c[i]; }
+                const int bpt = 4096 / NT, top = 4095 - bpt * tid;
+                unsigned tot = 0;
+                for (int i = 0; i < bpt; ++i) tot += hist[top - i];
                 int all;
                 const unsigned before = (unsigned)block_scan_int((int)tot, scan_sums[pass & 1], all);
                 if (before < rem && rem <= before + tot) {
                     unsigned acc = before;
-                    int bin = 4095 - 4 * tid;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        if (acc + c[i] >= rem) { bin = 4095 - 4 * tid - i; break; }
-                        acc += c[i];
+                    int bin = top;
+                    for (int i = 0; i < bpt; ++i) {
+                        const unsigned ci = hist[top - i];
+                        if (acc + ci >= rem) { bin = top - i; break; }
+                        acc += ci;
                     }
                     sh_prefix = (prefix << 12) | (unsigned)bin;
                     sh_remaining = rem - acc;
@@ -454,14 +456,14 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     };
 #pragma unroll
     for (int r = 0; r < PF; ++r) {
-        const int u = r * SEL_THREADS + tid;
+        const int u = r * NT + tid;
         if (r < n_rounds && u < U) emit(u, idx_pf[r], true);
     }
     for (int r = PF; r < n_rounds; ++r) {
-        const int u = r * SEL_THREADS + tid;
+        const int u = r * NT + tid;
         if (u < U) emit(u, 0, false);
     }
-    for (int p = kept_total + tid; p < y_stride; p += SEL_THREADS) kept_idx[g * y_stride + p] = -1;
+    for (int p = kept_total + tid; p < y_stride; p += NT) kept_idx[g * y_stride + p] = -1;
     if (tid == 0) kept_count[g] = kept_total;
 }
 
@@ -483,7 +485,13 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
     }
     LaunchScope scope(ctx, OC_K_SELECT, s);
     if (!geo.self_match && geo.units_per_group <= SEL_SMEM_KEYS) {
-        OC_LAUNCH(select_fast_kernel, (unsigned)geo.n_groups, SEL_THREADS, (size_t)geo.units_per_group * sizeof(unsigned), s,
+        // A big group wants every thread it can get (the kernel is latency-bound per thread); many small
+        // groups want small CTAs so that several share an SM.  A thread's run of units must fit its
+        // 64-bit reuse mask.
+        int nt = 128;
+        while (nt < SEL_THREADS && nt * 4 < geo.units_per_group) nt <<= 1;
+        while (nt < SEL_THREADS && (geo.units_per_group + nt - 1) / nt > 40) nt <<= 1;
+        OC_LAUNCH(select_fast_kernel, (unsigned)geo.n_groups, nt, (size_t)geo.units_per_group * sizeof(unsigned), s,
                   gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);
     } else {
         const int keys_in_smem = (mode == OC_SELECT_COUNT && geo.units_per_group <= SEL_SMEM_KEYS) ? 1 : 0;
