@@ -572,6 +572,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 const uint32_t d_tmem = tmem_base + buf * 256u;
                 tc_fence_after();
                 const uint32_t idesc = IDESC_BASE | ((uint32_t)((c.nq * QN) >> 3) << 17);
+                // an odd number of candidate tiles leaves the last run with an empty second tile (in a pair:
+                // empty in both CTAs): its MMAs are not issued, and the epilogue skips it likewise
+                const bool two_tiles = P.tpp == 2 && (PAIR ? 2 : 1) * P.tpp * c.a_pair + 1 < P.n_tilesA;
                 for (int kb = 0; kb < P.kblocks; ++kb) {
                     // (each lane looked for itself; the barrier's phase cannot go back, so a lane that saw it
                     //  full stays right, and the others wait here)
@@ -585,7 +588,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     if (nstage == STAGES) { nstage = 0; nphase ^= 1u; }
                     // UMMA K = 16 is 32 bytes along the swizzled row: +2 in the descriptor's address field
                     peeked = tc_mma_stage<PAIR>(d_tmem, a0_desc, a1_desc, b_desc, idesc, (uint32_t)(kb != 0), issue,
-                                                P.tpp == 2, bar_full + 8 * nstage, nphase) != 0;
+                                                two_tiles, bar_full + 8 * nstage, nphase) != 0;
                     // frees the stage (in both CTAs of a pair) when the MMAs retire
                     tc_commit<PAIR>(PAIR ? map_to_cta(bar_empty + 8 * stage, 0) : bar_empty + 8 * stage, issue);
                     if (PAIR) tc_commit<PAIR>(map_to_cta(bar_empty + 8 * stage, 1), issue);
@@ -668,6 +671,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 tc_fence_after();
 #pragma unroll 1
                 for (int t = 0; t < P.tpp; ++t) {                      // the piece's candidate tiles
+                    if ((PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + t >= P.n_tilesA) continue;   // past the lattice
                     const long long tokA = t ? tokA1 : tokA0;
                     const bool row_ok = t ? row_ok1 : row_ok0;
                     float inv_a = 0.f;
