@@ -296,8 +296,11 @@ oc_status oc_schedule_propose(const double* latency, const double* quality_loss,
  * memory: copies x_host (layer input) and cache_host (previous output, same shape) to library-owned
  * device staging, runs match -> select -> gather -> restore with the identity as the wrapped layer
  * (z = the gathered rows), copies the restored tensor to out_host and the per-group kept counts to
- * kept_count_host, and synchronises the stream before returning.  Pinned host memory makes the
- * copies asynchronous to the host but the call still waits for completion. */
+ * kept_count_host, and synchronises the stream before returning.  When cache_host / out_host are
+ * pinned (page-locked, device-mapped, 16-byte aligned) the restore kernel reads and writes them in
+ * place: of the cache only the rows of reused units cross the bus, and the output streams out while
+ * they stream in; pageable buffers go through staging copies of the whole tensors.  x_host is always
+ * copied whole (the matcher reads it several times). */
 oc_status oc_cache_step_host(oc_ctx* ctx, const oc_layout* layout, int mode, float thr,
                              int64_t n_reuse_per_group, const void* x_host, const void* cache_host,
                              void* out_host, int32_t* kept_count_host, void* stream);

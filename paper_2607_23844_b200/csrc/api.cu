@@ -485,17 +485,31 @@ oc_status oc_cache_step_host(oc_ctx* c, const oc_layout* layout, int mode, float
     int32_t* dslot = (int32_t*)p; p += up(nu * 4);
     int32_t* dcount = (int32_t*)p;
 
+    // Pinned (page-locked, device-mapped) host buffers are read and written by the restore kernel
+    // itself: of the cache only the rows of reused units then cross the bus, and the output streams
+    // to the host while those rows stream in (the link is full duplex).  Pageable buffers go through
+    // staging copies.
+    auto mapped = [](const void* h) -> void* {
+        cudaPointerAttributes a;
+        if (cudaPointerGetAttributes(&a, h) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        return (a.type == cudaMemoryTypeHost && ((uintptr_t)a.devicePointer & 15) == 0) ? a.devicePointer : nullptr;
+    };
+    void* cache_dev = mapped(cache_host);
+    void* out_dev = mapped(out_host);
     if (cudaMemcpyAsync(dx, x_host, tensor_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return OC_ERR_CUDA;
-    if (cudaMemcpyAsync(dcache, cache_host, tensor_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return OC_ERR_CUDA;
+    if (!cache_dev && cudaMemcpyAsync(dcache, cache_host, tensor_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return OC_ERR_CUDA;
     st = oc_match(c, layout, dx, dsim, didx, nullptr, nullptr, stream);
     if (st != OC_OK) return st;
     st = oc_select(c, layout, dsim, didx, mode, thr, n_reuse, g.units_per_group, dkept, dcount, dmap, dslot, stream);
     if (st != OC_OK) return st;
     st = oc_gather(c, &rows, dx, dkept, (int64_t)nu, dy, stream);
     if (st != OC_OK) return st;
-    st = oc_restore(c, &rows, dy, dcache, (int64_t)nu, dslot, dmap, dout, OC_RESTORE_FROM_CACHE, stream);
+    st = oc_restore(c, &rows, dy, cache_dev ? cache_dev : dcache, (int64_t)nu, dslot, dmap, out_dev ? out_dev : dout,
+                    OC_RESTORE_FROM_CACHE, stream);
     if (st != OC_OK) return st;
-    if (cudaMemcpyAsync(out_host, dout, tensor_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return OC_ERR_CUDA;
+    if (!out_dev && cudaMemcpyAsync(out_host, dout, tensor_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return OC_ERR_CUDA;
     if (kept_count_host &&
         cudaMemcpyAsync(kept_count_host, dcount, ng * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return OC_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return OC_ERR_CUDA;

@@ -438,14 +438,18 @@ def test_select_capacity_limits(oc, oracle):
                           ti.clone(), ti.clone(), check=False) == oc.ERR_UNSUPPORTED
 
 
-def test_cache_step_host_matches_device_path(oc, oracle):
+@pytest.mark.parametrize("pinned", [True, False])
+def test_cache_step_host_matches_device_path(oc, oracle, pinned):
+    """Pinned buffers: the restore kernel reads the cache and writes the output in host memory itself;
+    pageable buffers: staging copies.  Same bytes either way."""
     w = inputs.sd3_token_cache(seed=12, B=2, H=32, W=32, C=128)
     L, Lo = H.layouts(oc, oracle, w)
     cache_np = inputs.random_rows(3, w.shape, w.dtype)
-    xh = torch.from_numpy(w.x.view(np.int16)).pin_memory()
-    ch = torch.from_numpy(cache_np.view(np.int16)).pin_memory()
-    oh = torch.zeros_like(xh).pin_memory()
-    kh = torch.zeros(L.n_groups, dtype=torch.int32).pin_memory()
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    xh = pin(torch.from_numpy(w.x.view(np.int16).copy()))
+    ch = pin(torch.from_numpy(cache_np.view(np.int16).copy()))
+    oh = pin(torch.zeros_like(xh))
+    kh = pin(torch.zeros(L.n_groups, dtype=torch.int32))
     with H.make_ctx(oc, L) as ctx:
         ctx.cache_step_host(L, oc.SELECT_COUNT, 0.0, w.n_reuse, xh, ch, oh, kh)
         m = H.gpu_match(oc, ctx, L, H.to_dev(w.x))
