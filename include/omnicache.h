@@ -300,7 +300,10 @@ oc_status oc_schedule_propose(const double* latency, const double* quality_loss,
  * pinned (page-locked, device-mapped, 16-byte aligned) the restore kernel reads and writes them in
  * place: of the cache only the rows of reused units cross the bus, and the output streams out while
  * they stream in; pageable buffers go through staging copies of the whole tensors.  x_host is always
- * copied whole (the matcher reads it several times). */
+ * copied whole (the matcher reads it several times).  Token Cache layouts of several frames are
+ * processed in up to 8 chunks of whole frames, the copies of later chunks overlapping the work on
+ * earlier ones (a second, library-owned stream carries those copies; the caller's stream orders the
+ * call as a whole). */
 oc_status oc_cache_step_host(oc_ctx* ctx, const oc_layout* layout, int mode, float thr,
                              int64_t n_reuse_per_group, const void* x_host, const void* cache_host,
                              void* out_host, int32_t* kept_count_host, void* stream);

@@ -224,6 +224,8 @@ oc_status oc_destroy(oc_ctx* c) {
     tc_cache_free(c);
     cudaFree(c->stage);
     cudaFree(c->workspace);
+    for (auto e : c->chunk_events) cudaEventDestroy(e);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     cudaFree(c->d_span);
     cudaFree(c->d_status);
     delete c;
@@ -496,20 +498,80 @@ oc_status oc_cache_step_host(oc_ctx* c, const oc_layout* layout, int mode, float
     };
     void* cache_dev = mapped(cache_host);
     void* out_dev = mapped(out_host);
-    if (cudaMemcpyAsync(dx, x_host, tensor_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return OC_ERR_CUDA;
-    if (!cache_dev && cudaMemcpyAsync(dcache, cache_host, tensor_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return OC_ERR_CUDA;
-    st = oc_match(c, layout, dx, dsim, didx, nullptr, nullptr, stream);
-    if (st != OC_OK) return st;
-    st = oc_select(c, layout, dsim, didx, mode, thr, n_reuse, g.units_per_group, dkept, dcount, dmap, dslot, stream);
-    if (st != OC_OK) return st;
-    st = oc_gather(c, &rows, dx, dkept, (int64_t)nu, dy, stream);
-    if (st != OC_OK) return st;
-    st = oc_restore(c, &rows, dy, cache_dev ? cache_dev : dcache, (int64_t)nu, dslot, dmap, out_dev ? out_dev : dout,
-                    OC_RESTORE_FROM_CACHE, stream);
-    if (st != OC_OK) return st;
-    if (!out_dev && cudaMemcpyAsync(out_host, dout, tensor_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return OC_ERR_CUDA;
+
+    // Token Cache groups never span frames, so the call is cut into up to 8 chunks of whole frames:
+    // all host->device copies of x are queued at once on a second stream, and chunk k is matched,
+    // selected, gathered and restored (its output streaming back to the host) while the copies of the
+    // chunks after it are still arriving.  Other kinds, and single frames, are one chunk.
+    const int64_t frames = (int64_t)g.B * g.T;
+    int n_chunks = (g.kind == OC_KIND_TOKEN && frames > 1) ? (int)(frames < 8 ? frames : 8) : 1;
+    if (n_chunks > 1) {
+        if (!c->copy_stream && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess) {
+            cudaGetLastError(); n_chunks = 1;
+        }
+        while (n_chunks > 1 && (int)c->chunk_events.size() < n_chunks + 1) {
+            cudaEvent_t e;
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); n_chunks = 1; break; }
+            c->chunk_events.push_back(e);
+        }
+    }
+    if (n_chunks == 1) {
+        if (cudaMemcpyAsync(dx, x_host, tensor_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return OC_ERR_CUDA;
+        if (!cache_dev && cudaMemcpyAsync(dcache, cache_host, tensor_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return OC_ERR_CUDA;
+        st = oc_match(c, layout, dx, dsim, didx, nullptr, nullptr, stream);
+        if (st != OC_OK) return st;
+        st = oc_select(c, layout, dsim, didx, mode, thr, n_reuse, g.units_per_group, dkept, dcount, dmap, dslot, stream);
+        if (st != OC_OK) return st;
+        st = oc_gather(c, &rows, dx, dkept, (int64_t)nu, dy, stream);
+        if (st != OC_OK) return st;
+        st = oc_restore(c, &rows, dy, cache_dev ? cache_dev : dcache, (int64_t)nu, dslot, dmap, out_dev ? out_dev : dout,
+                        OC_RESTORE_FROM_CACHE, stream);
+        if (st != OC_OK) return st;
+        if (!out_dev && cudaMemcpyAsync(out_host, dout, tensor_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return OC_ERR_CUDA;
+    } else {
+        const int64_t fpc = (frames + n_chunks - 1) / n_chunks;              // frames per chunk
+        const size_t frame_bytes = tensor_bytes / (size_t)frames;
+        const size_t units_pf = nu / (size_t)frames, groups_pf = ng / (size_t)frames;
+        cudaStream_t cs = c->copy_stream;
+        // the copies may not overtake earlier work of the caller's stream on the staging buffers
+        if (cudaEventRecord(c->chunk_events[n_chunks], s) != cudaSuccess ||
+            cudaStreamWaitEvent(cs, c->chunk_events[n_chunks], 0) != cudaSuccess) return OC_ERR_CUDA;
+        for (int k = 0; k < n_chunks; ++k) {
+            const int64_t f0 = k * fpc, f1 = (f0 + fpc < frames) ? f0 + fpc : frames;
+            if (f0 >= f1) { n_chunks = k; break; }
+            const size_t off = (size_t)f0 * frame_bytes, len = (size_t)(f1 - f0) * frame_bytes;
+            if (cudaMemcpyAsync((uint8_t*)dx + off, (const uint8_t*)x_host + off, len, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+                return OC_ERR_CUDA;
+            if (!cache_dev && cudaMemcpyAsync((uint8_t*)dcache + off, (const uint8_t*)cache_host + off, len,
+                                              cudaMemcpyHostToDevice, cs) != cudaSuccess) return OC_ERR_CUDA;
+            if (cudaEventRecord(c->chunk_events[k], cs) != cudaSuccess) return OC_ERR_CUDA;
+        }
+        for (int k = 0; k < n_chunks; ++k) {
+            const int64_t f0 = k * fpc, f1 = (f0 + fpc < frames) ? f0 + fpc : frames;
+            oc_layout sub = *layout;
+            sub.B = (int)(f1 - f0); sub.T = 1;
+            oc_rows sub_rows;
+            st = oc_rows_from_layout(&sub, g.C, g.elem_bytes, &sub_rows);
+            if (st != OC_OK) return st;
+            const size_t off = (size_t)f0 * frame_bytes, uoff = (size_t)f0 * units_pf, goff = (size_t)f0 * groups_pf;
+            const int64_t sub_units = (int64_t)((size_t)(f1 - f0) * units_pf);
+            if (cudaStreamWaitEvent(s, c->chunk_events[k], 0) != cudaSuccess) return OC_ERR_CUDA;
+            st = oc_match(c, &sub, (uint8_t*)dx + off, dsim + uoff, didx + uoff, nullptr, nullptr, stream);
+            if (st != OC_OK) return st;
+            st = oc_select(c, &sub, dsim + uoff, didx + uoff, mode, thr, n_reuse, g.units_per_group, dkept + uoff,
+                           dcount + goff, dmap + uoff, dslot + uoff, stream);
+            if (st != OC_OK) return st;
+            st = oc_gather(c, &sub_rows, (uint8_t*)dx + off, dkept + uoff, sub_units, (uint8_t*)dy + off, stream);
+            if (st != OC_OK) return st;
+            st = oc_restore(c, &sub_rows, (uint8_t*)dy + off, (uint8_t*)(cache_dev ? cache_dev : dcache) + off, sub_units,
+                            dslot + uoff, dmap + uoff, (uint8_t*)(out_dev ? out_dev : dout) + off, OC_RESTORE_FROM_CACHE, stream);
+            if (st != OC_OK) return st;
+            if (!out_dev && cudaMemcpyAsync((uint8_t*)out_host + off, (uint8_t*)dout + off, (size_t)(f1 - f0) * frame_bytes,
+                                            cudaMemcpyDeviceToHost, s) != cudaSuccess) return OC_ERR_CUDA;
+        }
+    }
     if (kept_count_host &&
         cudaMemcpyAsync(kept_count_host, dcount, ng * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return OC_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return OC_ERR_CUDA;

@@ -41,6 +41,8 @@ struct oc_ctx {
     // staging for oc_cache_step_host
     void* stage = nullptr;
     size_t stage_bytes = 0;
+    cudaStream_t copy_stream = nullptr;      // host->device copies of the chunks of oc_cache_step_host
+    std::vector<cudaEvent_t> chunk_events;
     // cached tensor maps of the tcgen05 matcher (opaque to the other files)
     void* tc_cache = nullptr;
 };

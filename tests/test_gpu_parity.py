@@ -439,10 +439,14 @@ def test_select_capacity_limits(oc, oracle):
 
 
 @pytest.mark.parametrize("pinned", [True, False])
-def test_cache_step_host_matches_device_path(oc, oracle, pinned):
+@pytest.mark.parametrize("frames", [(2, 1), (3, 3), (1, 1)])
+def test_cache_step_host_matches_device_path(oc, oracle, pinned, frames):
     """Pinned buffers: the restore kernel reads the cache and writes the output in host memory itself;
-    pageable buffers: staging copies.  Same bytes either way."""
-    w = inputs.sd3_token_cache(seed=12, B=2, H=32, W=32, C=128)
+    pageable buffers: staging copies.  Several frames are processed in chunks whose copies overlap the
+    work on earlier chunks (9 frames: chunks of 2, 2, 2, 2, 1).  Same bytes every way."""
+    w = inputs.sd3_token_cache(seed=12, B=frames[0] * frames[1], H=32, W=32, C=128)
+    shape = (frames[0], frames[1]) + tuple(w.shape[2:])
+    w.x = w.x.reshape(shape); w.shape = shape
     L, Lo = H.layouts(oc, oracle, w)
     cache_np = inputs.random_rows(3, w.shape, w.dtype)
     pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
