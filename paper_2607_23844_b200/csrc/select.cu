@@ -485,11 +485,12 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
     }
     LaunchScope scope(ctx, OC_K_SELECT, s);
     if (!geo.self_match && geo.units_per_group <= SEL_SMEM_KEYS) {
-        // A big group wants every thread it can get (the kernel is latency-bound per thread); many small
-        // groups want small CTAs so that several share an SM.  A thread's run of units must fit its
-        // 64-bit reuse mask.
-        int nt = 128;
-        while (nt < SEL_THREADS && nt * 4 < geo.units_per_group) nt <<= 1;
+        // A group wants every thread it can get (the kernel is latency-bound per thread); only when the
+        // groups do not all fit on the device at once, and are small, do smaller CTAs pay (more groups in
+        // flight).  A thread's run of units must fit its 64-bit reuse mask.
+        int nt = SEL_THREADS, min_nt = 512;          // (measured: below 512 threads a group only gets slower)
+        while (min_nt < SEL_THREADS && min_nt * 4 < geo.units_per_group) min_nt <<= 1;      // at most ~4 units per thread
+        while (nt > min_nt && (long long)geo.n_groups * nt > 2048ll * ctx->sm_count) nt >>= 1;
         while (nt < SEL_THREADS && (geo.units_per_group + nt - 1) / nt > 40) nt <<= 1;
         OC_LAUNCH(select_fast_kernel, (unsigned)geo.n_groups, nt, (size_t)geo.units_per_group * sizeof(unsigned), s,
                   gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);
