@@ -27,8 +27,11 @@
 //
 // Work split.  The representatives of a group are cut into "quanta" of 32 lattice points (one 4 KB
 // box per 64 channels).  A row of the problem is the candidate tiles of one CTA (or pair) against all
-// representatives of its group; it is cut into P pieces of nearly equal width (<= 8 quanta), and the
-// pieces are dealt out evenly, in contiguous runs, to one persistent CTA (pair) per SM (pair of SMs).
+// representatives of its group; it is cut into P pieces of nearly equal width (<= 256 columns; in the
+// single-CTA form in steps of half a quantum, so that 1024 columns split six ways as 176/176/160
+// rather than 192/160/160: a piece that begins in mid-quantum fetches that quantum whole and starts
+// its B descriptor 16 rows in), and the pieces are dealt out evenly, in contiguous runs, to one
+// persistent CTA (pair) per SM (pair of SMs).
 // The host picks the form, the tiles per CTA and P with a small cost model.
 //
 // Warp specialised:
@@ -88,7 +91,8 @@ struct TcScalars {
     int n_apairs;                        // tile rows per lattice member = ceil(n_tilesA / tpp)
     int bwQ_log2, bhQ, n_wq, n_quanta;   // quantum box:   (1 << bwQ_log2) x bhQ lattice points = 32 rows
     int pieces_per_row, total_items;     // a row = the candidate tiles of one piece against all representatives
-    int q_unit, n_q_units;               // pieces are cut in units of q_unit quanta (2 for a CTA pair)
+    int q_unit, n_q_units;               // pieces are cut in units of q_unit quanta (2 for a CTA pair), or, when
+    int half_units;                      // half_units is set, in units of half a quantum (16 columns)
     int a_merged, q_merged, q_lo;        // one box for a CTA's candidate tiles / for its quanta of a piece
     int items_base, items_rem;           // every walker takes items_base pieces, the first items_rem one more
     unsigned cum[5];                     // pieces per tile run, lattice, patch, patch row, frame
@@ -332,7 +336,9 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
 struct Piece {
     int bt, py, px, member;              // frame, patch, candidate sub-lattice member
     int a_pair;                          // which run of candidate tiles (tpp per CTA) of the member's lattice
-    int q0, nq;                          // quanta [q0, q0 + nq) of the group's representatives
+    int q0, nq;                          // quanta [q0, q0 + nq) of the group's representatives are fetched
+    int c_off, ncol;                     // of which columns [c_off, c_off + ncol) are the piece (c_off is 0 or 16,
+                                         // ncol a multiple of 16: pieces may begin and end in mid-quantum)
     long long g;
 };
 // floor(a / d) for a < 2^22 from the float reciprocal (one multiply and a fix-up; an integer division
@@ -375,8 +381,17 @@ struct Walk {
         --left;
         int u_next = u_cur + P.u_step_q, r_next = r_cur + P.u_step_r;
         if (r_next >= P.pieces_per_row) { r_next -= P.pieces_per_row; ++u_next; }
-        p.q0 = u_cur * P.q_unit;
-        p.nq = (u_next - u_cur) * P.q_unit;
+        if (P.half_units) {                  // units of 16 columns: half a quantum
+            p.q0 = u_cur >> 1;
+            p.nq = ((u_next - 1) >> 1) - p.q0 + 1;
+            p.c_off = (u_cur & 1) << 4;
+            p.ncol = (u_next - u_cur) << 4;
+        } else {
+            p.q0 = u_cur * P.q_unit;
+            p.nq = (u_next - u_cur) * P.q_unit;
+            p.c_off = 0;
+            p.ncol = p.nq * QN;
+        }
         u_cur = u_next; r_cur = r_next;
         p.a_pair = a_pair; p.g = g; p.px = px; p.py = py; p.bt = bt;
         p.member = k < P.rep_member ? k : k + 1;
@@ -571,7 +586,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_empty + 8 * buf, acc_phase ^ 1u, abort_flag))) { ok = false; break; }
                 const uint32_t d_tmem = tmem_base + buf * 256u;
                 tc_fence_after();
-                const uint32_t idesc = IDESC_BASE | ((uint32_t)((c.nq * QN) >> 3) << 17);
+                const uint32_t idesc = IDESC_BASE | ((uint32_t)(c.ncol >> 3) << 17);
                 // an odd number of candidate tiles leaves the last run with an empty second tile (in a pair:
                 // empty in both CTAs): its MMAs are not issued, and the epilogue skips it likewise
                 const bool two_tiles = P.tpp == 2 && (PAIR ? 2 : 1) * P.tpp * c.a_pair + 1 < P.n_tilesA;
@@ -583,7 +598,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     const uint32_t a_addr = tiles_base + stage * STAGE_BYTES;
                     const uint64_t a0_desc = make_smem_desc(a_addr);
                     const uint64_t a1_desc = make_smem_desc(a_addr + A_BYTES);
-                    const uint64_t b_desc = make_smem_desc(a_addr + P.tpp * A_BYTES);
+                    // (a piece that begins in mid-quantum skips 16 rows = 2 KB of its first box: a whole number
+                    //  of 8-row swizzle groups)
+                    const uint64_t b_desc = make_smem_desc(a_addr + P.tpp * A_BYTES + (uint32_t)c.c_off * 128u);
                     int nstage = stage + 1; uint32_t nphase = phase;
                     if (nstage == STAGES) { nstage = 0; nphase ^= 1u; }
                     // UMMA K = 16 is 32 bytes along the swizzled row: +2 in the descriptor's address field
@@ -621,8 +638,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         float* col_scale = (float*)colsb;                              // [2][256]
         const int rowh = row >> P.bwA_log2, roww = row & (bwA - 1);
         auto table_entry = [&](const Piece& pc) -> float {
-            if (et >= pc.nq * QN) return __int_as_float(0x7FC00000);
-            const int qi = pc.q0 + (et >> 5), r = et & 31;
+            if (et >= pc.ncol) return __int_as_float(0x7FC00000);
+            const int gp = pc.c_off + et;
+            const int qi = pc.q0 + (gp >> 5), r = gp & 31;
             const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
             const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));
             if (hs >= P.Hs || ws >= P.Ws) return __int_as_float(0x7FC00000);
@@ -663,8 +681,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 tokA1 = ((long long)c.bt * P.H + yA) * P.W + xA;
             }
             // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
-            const int ch_split = (c.nq + 1) >> 1;
-            const int ch_begin = half ? ch_split : 0, ch_end = half ? c.nq : ch_split;
+            const int n_ch = (c.ncol + 31) >> 5;                        // (a last half chunk reads 16 columns of
+            const int ch_split = (n_ch + 1) >> 1;                      //  nothing: their table entries are NaN)
+            const int ch_begin = half ? ch_split : 0, ch_end = half ? n_ch : ch_split;
             // warp-uniform outcome: the TMEM loads below are warp-collective
             const bool ready = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * buf, acc_phase, abort_flag));
             if (ready) {
@@ -711,7 +730,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             for (int j = 0; j < 32; ++j) {                                                                       \
                 const float sc = col_scale1[(ch) * 32 + j];                                                      \
                 if (sc == sc) {                                                                                  \
-                    const int qi = c.q0 + (ch), r = j;                                                           \
+                    const int gp_ = c.c_off + (ch) * 32 + j;                                                     \
+                    const int qi = c.q0 + (gp_ >> 5), r = gp_ & 31;                                              \
                     const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;                                           \
                     const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));              \
                     aux_row[hs * P.Ws + ws] = clamp_unit(__uint_as_float(v[j]) * sc * inv_a);                    \
@@ -740,7 +760,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     if (n1 >= 0 && (n0 < 0 || OC_VAL(bm1) > best || (OC_VAL(bm1) == best && n1 < n0))) { best = OC_VAL(bm1); n0 = n1; }
 #undef OC_VAL
                     if (row_ok && n0 >= 0) {
-                        const int qi = c.q0 + (n0 >> 5), r = n0 & 31;
+                        const int gp = c.c_off + n0;
+                        const int qi = c.q0 + (gp >> 5), r = gp & 31;
                         const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
                         const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));
                         const int y = (c.py * P.Hs + hs) * P.sy + my_rep, x = (c.px * P.Ws + ws) * P.sx + mx_rep;
@@ -831,7 +852,7 @@ static int pow2_ceil_log2(int v) { int l = 0; while ((1 << l) < v) ++l; return l
 
 struct TcPlan {
     int bwA_log2, bhA, n_wtA, n_tilesA, tpp, n_apairs, bwQ_log2, bhQ, n_wq, n_quanta;
-    int pair, q_unit, n_q_units, a_merged, q_merged, q_lo;
+    int pair, q_unit, n_q_units, half_units, a_merged, q_merged, q_lo, q_hi;
     int pieces_per_row, qmax, n_stages, stage_bytes;
     long long rows, items;
 };
@@ -861,6 +882,17 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
     //     MMAs, where the two slow each other down (~0.8 of the shorter one is not hidden);
     //   * ~6500 cycles before a CTA's first MMA and after its last.
     const int kblocks = (g.C + BK - 1) / BK;
+    // Single-CTA pieces are cut in units of HALF a quantum (16 columns) whenever that is valid: no piece
+    // wider than 256 columns, none that would have to fetch more than MAXQ quanta (one that begins in
+    // mid-quantum fetches its first quantum whole).  Returns the widest piece in half units, or 0.
+    const int n_half = 2 * p.n_quanta;
+    auto half_widest = [&](int P) -> int {
+        if (P < 1 || P > p.n_quanta) return 0;
+        const int h_max = (n_half + P - 1) / P;
+        if (h_max > 2 * MAXQ) return 0;
+        if (h_max == 2 * MAXQ && !(n_half % P == 0 && (h_max & 1) == 0)) return 0;   // 256 columns only from even starts
+        return h_max;
+    };
     double best_cost = 0; int best_P = 0, best_tpp = 2, best_pair = 0;
     for (int pair = 0; pair <= (pair_walkers > 0 ? 1 : 0); ++pair) {
         const int ncta = pair ? 2 : 1, q_unit = pair ? 2 : 1;
@@ -870,11 +902,16 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
             const long long rows = g.n_groups * (long long)(g.sy * g.sx - 1) *
                                    ((p.n_tilesA + tpp * ncta - 1) / (tpp * ncta));
             for (int P = (n_units + max_units - 1) / max_units; P <= n_units; ++P) {
-                const int q = ((n_units + P - 1) / P) * q_unit;       // quanta of the largest piece
-                const double stage_kb = tpp * 16.0 + 4.0 * q / ncta;
+                int q = ((n_units + P - 1) / P) * q_unit;             // quanta of the largest piece: for the MMAs ...
+                int q_load = q;                                       // ... and fetched per stage
+                const int hw = pair ? 0 : half_widest(P);
+                if (hw) { q_load = (hw + 2) >> 1; if (q_load > MAXQ) q_load = MAXQ; }
+                const double qe = hw ? hw * 0.5 : (double)q;          // width in quanta (may end in a half)
+                if (hw) q = (hw + 1) >> 1;
+                const double stage_kb = tpp * 16.0 + 4.0 * q_load / ncta;
                 int stages = (int)(TILE_BYTES / 1024 / stage_kb); if (stages > MAX_STAGES) stages = MAX_STAGES;
                 const long long per_walker = (rows * P + nw - 1) / nw;
-                const double mma = tpp * 64.0 * q, fetch = stage_kb * 1024.0 / 74.0;
+                const double mma = tpp * 64.0 * qe, fetch = stage_kb * 1024.0 / 74.0;
                 const double refill = (mma + 330.0 + 1450.0 + 1.35 * stage_kb + (pair ? 980.0 : 0.0)) / stages;
                 double fast = mma + 53.0; if (fetch > fast) fast = fetch;
                 const double slow = refill > fast ? refill : fast;
@@ -904,14 +941,23 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
         }
     }
     p.pair = best_pair; p.tpp = best_tpp;
+    p.half_units = (!p.pair && half_widest(best_P)) ? 1 : 0;
     p.q_unit = p.pair ? 2 : 1;
-    p.n_q_units = (p.n_quanta + p.q_unit - 1) / p.q_unit;
+    p.n_q_units = p.half_units ? n_half : (p.n_quanta + p.q_unit - 1) / p.q_unit;
     const int ncta = p.pair ? 2 : 1;
     p.n_apairs = (p.n_tilesA + p.tpp * ncta - 1) / (p.tpp * ncta);
     p.rows = g.n_groups * (long long)(g.sy * g.sx - 1) * p.n_apairs;
     p.pieces_per_row = best_P;
-    p.qmax = ((p.n_q_units + best_P - 1) / best_P) * p.q_unit;
-    p.stage_bytes = p.tpp * A_BYTES + (p.qmax / ncta) * Q_BYTES;
+    // fewest and most quanta any piece fetches (per CTA)
+    int q_min = 1 << 30, q_max = 0;
+    for (int j = 0; j < best_P; ++j) {
+        const int u0 = (int)((long long)j * p.n_q_units / best_P), u1 = (int)((long long)(j + 1) * p.n_q_units / best_P);
+        int nq = p.half_units ? ((u1 - 1) >> 1) - (u0 >> 1) + 1 : (u1 - u0) * p.q_unit / ncta;
+        if (nq < q_min) q_min = nq;
+        if (nq > q_max) q_max = nq;
+    }
+    p.qmax = q_max * ncta;
+    p.stage_bytes = p.tpp * A_BYTES + q_max * Q_BYTES;
     p.n_stages = TILE_BYTES / p.stage_bytes;
     if (p.n_stages > MAX_STAGES) p.n_stages = MAX_STAGES;
     p.items = p.rows * p.pieces_per_row;
@@ -920,7 +966,8 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
     // of lattice rows (always the case when the patch's lattice is at most one box wide).
     p.a_merged = (p.tpp == 1 || p.n_wtA == 1) ? 1 : 0;
     p.q_merged = p.n_wq == 1 ? 1 : 0;
-    p.q_lo = p.n_q_units / best_P;
+    p.q_lo = q_min;                           // merged boxes come in two heights: q_lo and q_lo + 1 quanta
+    p.q_hi = q_max;
     return p;
 }
 
@@ -981,7 +1028,7 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const cuuint32_t boxA[4] = {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwA_log2),
                                 (cuuint32_t)(p.bhA * (p.a_merged ? p.tpp : 1)), 1};
-    const int q_hi = (p.n_q_units % p.pieces_per_row) ? p.q_lo + 1 : p.q_lo;
+    const int q_hi = p.q_hi;
     const cuuint32_t boxQ[2][4] = {
         {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwQ_log2), (cuuint32_t)(p.bhQ * (p.q_merged ? p.q_lo : 1)), 1},
         {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwQ_log2), (cuuint32_t)(p.bhQ * (p.q_merged ? q_hi : 1)), 1}};
@@ -1005,7 +1052,7 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
     P.bwA_log2 = p.bwA_log2; P.bhA = p.bhA; P.n_wtA = p.n_wtA; P.n_tilesA = p.n_tilesA; P.tpp = p.tpp; P.n_apairs = p.n_apairs;
     P.bwQ_log2 = p.bwQ_log2; P.bhQ = p.bhQ; P.n_wq = p.n_wq; P.n_quanta = p.n_quanta;
     P.pieces_per_row = p.pieces_per_row; P.total_items = (int)p.items;
-    P.q_unit = p.q_unit; P.n_q_units = p.n_q_units;
+    P.q_unit = p.q_unit; P.n_q_units = p.n_q_units; P.half_units = p.half_units;
     P.a_merged = p.a_merged; P.q_merged = p.q_merged; P.q_lo = p.q_lo;
     P.n_stages = p.n_stages; P.stage_bytes = p.stage_bytes;
     P.units_per_group = (int)g.units_per_group; P.reps_per_group = (int)g.reps_per_group;
