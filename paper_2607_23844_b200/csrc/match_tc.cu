@@ -450,7 +450,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     const bool leader = rank == 0;
     const int walker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     if ((tiles_base & 1023u) != 0) {                                   // never expected; refuse rather than compute garbage
-        if (threadIdx.x == 0) atomicCAS(KP.s.status, 0, OC_ERR_ALIGNMENT);   // (same verdict in both CTAs of a pair)
+        if (threadIdx.x == 0) atomicCAS(KP.s.status, 0, OC_ERR_ALIGNMENT);   // (same outcome in both CTAs of a pair)
         return;
     }
 
