@@ -163,6 +163,54 @@ def test_token_chain_small(oc, oracle, shape, groups, lattice, dtype):
         assert rep["launches"]["match_tc"] + rep["launches"]["match_simt"] == 1
 
 
+def _random_token_layouts(n, seed):
+    """Seeded random valid Token Cache shapes: lattice strides 2 or 3 with any offset, 1-8 patches per
+    frame, ragged lattice sizes, channel counts with and without a 64-channel tail, 1-3 frames."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < n:
+        sy, sx = int(rng.integers(2, 4)), int(rng.integers(2, 4))
+        gy, gx = int(rng.choice([1, 1, 2, 3])), int(rng.choice([1, 1, 2, 4]))
+        hp, wp = sy * int(rng.integers(2, 14)), sx * int(rng.integers(2, 22))
+        C = int(rng.choice([8, 24, 64, 72, 128, 200, 320]))
+        B, T = int(rng.integers(1, 3)), int(rng.integers(1, 3))
+        if B * T * gy * hp * gx * wp * C > 6_000_000:
+            continue
+        out.append(((B, T, gy * hp, gx * wp, C), (gy, gx), (sy, sx, int(rng.integers(0, sy)), int(rng.integers(0, sx)))))
+    return out
+
+
+@pytest.mark.parametrize("shape,groups,lattice", _random_token_layouts(24, seed=20260701))
+def test_token_chain_random_layouts(oc, oracle, shape, groups, lattice):
+    """The whole chain against the oracle on shapes nobody picked by hand (the matcher's tiling,
+    piece cutting and masking depend on every one of these numbers)."""
+    B, T, Hh, W, C = shape
+    w = inputs.sd3_token_cache(seed=int(np.prod(shape)) % 9973, B=B * T, H=Hh, W=W, C=C, groups=groups)
+    w.x = w.x.reshape(shape); w.shape = shape
+    sy, sx, oy, ox = lattice
+    U = (Hh // groups[0]) * (W // groups[1])
+    reps = ((Hh // groups[0]) // sy) * ((W // groups[1]) // sx)
+    w.n_reuse = (U - reps) // 3
+    rep = run_chain(oc, oracle, w, want_aux=True, sy=sy, sx=sx, oy=oy, ox=ox)
+    assert rep["launches"]["match_tc"] + rep["launches"]["match_simt"] == 1
+
+
+@pytest.mark.parametrize("plan", ["0,1,2", "0,2,3", "1,1,1", "1,2,2"])
+@pytest.mark.parametrize("shape,groups,lattice", _random_token_layouts(8, seed=7))
+def test_token_match_random_layouts_forced_plans(oc, oracle, shape, groups, lattice, plan, monkeypatch):
+    B, T, Hh, W, C = shape
+    w = inputs.sd3_token_cache(seed=int(np.prod(shape)) % 9973, B=B * T, H=Hh, W=W, C=C, groups=groups)
+    w.x = w.x.reshape(shape); w.shape = shape
+    sy, sx, oy, ox = lattice
+    L, Lo = H.layouts(oc, oracle, w, sy=sy, sx=sx, oy=oy, ox=ox)
+    ref = oracle.match_token(Lo, w.x)
+    monkeypatch.setenv("OC_TC_PLAN", plan)
+    with H.make_ctx(oc, L) as ctx:
+        m = H.gpu_match(oc, ctx, L, H.to_dev(w.x))
+    H.check_match_against_oracle(oracle, Lo, w.x, m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy(), ref,
+                                 TOL[inputs.BF16])
+
+
 @pytest.mark.parametrize("shape,groups", [
     ((2, 1, 64, 64, 192), (1, 1)),       # 1024 representatives: 32 quanta, 8 candidate tiles per lattice
     ((1, 3, 40, 56, 136), (1, 1)),       # ragged 20 x 28 lattice, K tail, three frames
