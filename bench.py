@@ -349,6 +349,36 @@ def run_ours(args, rank, local_rank, world):
     ctx.profile_enable(False)
     n_tiny, ms_tiny = ctx.profile_read(oc.K_COPY)
     bracket_us = 1e3 * ms_tiny / max(n_tiny, 1)
+    # The same brackets INSIDE the timed region's kind of execution: one more graph per ring slot,
+    # captured with the timers on, so that every launch sits between two event-record nodes of the graph;
+    # replayed K times, the brackets read after each replay.  No eager launch latency, no host in the loop.
+    graph_us = {}
+    ctx.profile_enable(True)
+    pgraphs = []
+    for r in range(ring):
+        gph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gph):
+            stream = torch.cuda.current_stream()
+            step(r)
+        pgraphs.append(gph)
+    ctx.profile_enable(False)
+    stream = torch.cuda.current_stream()
+    acc = {}
+    n_rep = 0
+    for i in range(min(args.steps, 200)):
+        pgraphs[i % ring].replay()
+        torch.cuda.synchronize()
+        if i < ring:            # every slot's graph has to have run once before all captured brackets are valid
+            continue
+        n_rep += 1
+        for k in range(oc.K_COUNT):
+            n_c, ms_c = ctx.profile_captured_read(k)
+            if n_c:
+                acc[k] = acc.get(k, 0.0) + ms_c / n_c      # mean over the slots' brackets (each holds its latest run)
+    if n_rep:
+        graph_us = {oc.kernel_name(k): 1e3 * v / n_rep for k, v in acc.items()}
+    del pgraphs
+
     # A third pass, for the tensor-core matcher only: the same K steps with the kernel stamping the GPU
     # timer when its first CTA starts and when its last CTA ends (no events): the time its CTAs occupy
     # the device, without launch latency and event records.
@@ -390,6 +420,8 @@ def run_ours(args, rank, local_rank, world):
     for name, (n, ms) in prof.items():
         if n:
             ops[name] = {"launches": n, "avg_us": 1e3 * ms / n, "net_us": max(1e3 * ms / n - bracket_us, 0.0), "share": None}
+            if name in graph_us:
+                ops[name]["in_graph_us"] = graph_us[name]       # CUDA events around the launch inside a replayed graph
     tot_ms = sum(ms for _, ms in prof.values()) or 1.0
     for name, (n, ms) in prof.items():
         if n:
@@ -412,6 +444,10 @@ def run_ours(args, rank, local_rank, world):
                     # the same with the bracket's own cost (see timing.event_bracket_us) taken off the duration
                     "achieved_net_of_bracket": flops / (max(ops["match_tc"]["net_us"], 1e-3) * 1e-6) / 1e12,
                     "frac_net_of_bracket": flops / (max(ops["match_tc"]["net_us"], 1e-3) * 1e-6) / 1e12 / peak}
+        if "in_graph_us" in ops["match_tc"]:
+            roofline["in_graph_us"] = ops["match_tc"]["in_graph_us"]
+            roofline["achieved_in_graph"] = flops / (ops["match_tc"]["in_graph_us"] * 1e-6) / 1e12
+            roofline["frac_in_graph"] = roofline["achieved_in_graph"] / peak
         if span_us:
             # first-CTA-entry -> last-CTA-exit by the GPU timer (oc_profile_span_read): device occupancy only
             roofline["device_span_us"] = span_us

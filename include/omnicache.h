@@ -179,6 +179,15 @@ oc_status oc_profile_read(oc_ctx* ctx, int kernel_id, int64_t* launches, double*
  * this is a measurement aid. */
 oc_status oc_profile_span_read(oc_ctx* ctx, int kernel_id, int64_t* launches, double* total_ms);
 
+/* Event brackets inside a CUDA graph.  Launches made while the event timers are on (mode 1) AND the
+ * caller's stream is being captured are bracketed by event-record nodes of the captured graph; those
+ * brackets are taken again every time the graph runs and are not counted by oc_profile_read.
+ * oc_profile_captured_read returns, for one kernel, how many such brackets exist (over all graphs
+ * captured so far with this context) and the sum of their MOST RECENT recordings; call it after
+ * synchronising a replay.  The events live until oc_destroy: graphs captured this way must not be
+ * launched after the context is destroyed. */
+oc_status oc_profile_captured_read(oc_ctx* ctx, int kernel_id, int64_t* launches, double* total_ms);
+
 /* ---------------------------------------------------------------------------------------------
  * The hot path
  * ------------------------------------------------------------------------------------------- */

@@ -22,14 +22,20 @@ static cudaEvent_t take_event(oc_ctx* c) {
 LaunchScope::LaunchScope(oc_ctx* c, int kernel, cudaStream_t stream) : ctx(c), k(kernel), s(stream) {
     ctx->prof[k].launches += 1;
     if (ctx->profile_on) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) { cudaGetLastError(); cap = cudaStreamCaptureStatusNone; }
+        capturing = cap == cudaStreamCaptureStatusActive;
         e0 = take_event(ctx); e1 = take_event(ctx);
-        if (e0 && e1) cudaEventRecord(e0, s);
+        // in a capture the records become event-record nodes of the graph (external events), so that the
+        // bracket is taken again on every replay
+        if (e0 && e1) cudaEventRecordWithFlags(e0, s, capturing ? cudaEventRecordExternal : cudaEventRecordDefault);
     }
 }
 LaunchScope::~LaunchScope() {
     if (e0 && e1) {
-        cudaEventRecord(e1, s);
-        ctx->prof[k].pending.emplace_back(e0, e1);
+        cudaEventRecordWithFlags(e1, s, capturing ? cudaEventRecordExternal : cudaEventRecordDefault);
+        if (capturing) ctx->prof[k].captured.emplace_back(e0, e1);
+        else ctx->prof[k].pending.emplace_back(e0, e1);
     } else {
         if (e0) ctx->free_events.push_back(e0);
         if (e1) ctx->free_events.push_back(e1);
@@ -218,8 +224,10 @@ oc_status oc_destroy(oc_ctx* c) {
     DeviceGuard guard(c->device);
     cudaDeviceSynchronize();
     for (auto& kv : c->layers) cudaFree(kv.second.ptr);
-    for (int k = 0; k < OC_K_COUNT; ++k)
+    for (int k = 0; k < OC_K_COUNT; ++k) {
         for (auto& p : c->prof[k].pending) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
+        for (auto& p : c->prof[k].captured) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
+    }
     for (auto e : c->free_events) cudaEventDestroy(e);
     tc_cache_free(c);
     cudaFree(c->stage);
@@ -281,6 +289,24 @@ oc_status oc_profile_read(oc_ctx* c, int k, int64_t* launches, double* total_ms)
     drain(c, k);
     if (launches) *launches = c->prof[k].launches;
     if (total_ms) *total_ms = c->prof[k].total_ms;
+    return OC_OK;
+}
+
+oc_status oc_profile_captured_read(oc_ctx* c, int k, int64_t* launches, double* total_ms) {
+    if (!c || k < 0 || k >= OC_K_COUNT) return OC_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    double sum = 0.0;
+    int64_t n = 0;
+    for (auto& p : c->prof[k].captured) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(p.second) == cudaSuccess && cudaEventElapsedTime(&ms, p.first, p.second) == cudaSuccess) {
+            sum += ms; ++n;
+        } else {
+            cudaGetLastError();                  // captured but its graph has not run yet
+        }
+    }
+    if (launches) *launches = n;
+    if (total_ms) *total_ms = sum;
     return OC_OK;
 }
 

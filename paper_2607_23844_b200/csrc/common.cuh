@@ -14,6 +14,9 @@ struct KernelProf {
     int64_t launches = 0;
     double total_ms = 0.0;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> pending;
+    // brackets recorded while the stream was being captured: event-record nodes of that graph, recorded
+    // anew on every replay (never recycled while the context lives)
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> captured;
 };
 
 struct LayerEntry {
@@ -62,7 +65,7 @@ struct DeviceGuard {
 
 // Counts a kernel launch and, if timers are on, brackets it with events on the launching stream.
 struct LaunchScope {
-    oc_ctx* ctx; int k; cudaStream_t s; cudaEvent_t e0 = nullptr, e1 = nullptr;
+    oc_ctx* ctx; int k; cudaStream_t s; cudaEvent_t e0 = nullptr, e1 = nullptr; bool capturing = false;
     LaunchScope(oc_ctx* c, int kernel, cudaStream_t stream);
     ~LaunchScope();
 };

@@ -30,7 +30,7 @@ EXPORTS = (
     "oc_status_str", "oc_layout_check", "oc_layout_counts", "oc_match_workspace_bytes",
     "oc_rows_from_layout", "oc_layer_cache_would_hit", "oc_kernel_name", "oc_create", "oc_destroy",
     "oc_device_status", "oc_profile_enable", "oc_profile_reset", "oc_profile_read", "oc_profile_span_read",
-    "oc_match",
+    "oc_profile_captured_read", "oc_match",
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
     "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
     "oc_schedule_propose",
@@ -75,6 +75,7 @@ _lib.oc_profile_enable.argtypes = [_vp, _i]
 _lib.oc_profile_reset.argtypes = [_vp]
 _lib.oc_profile_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_profile_span_read.argtypes = [_vp, _i, _vp, _vp]
+_lib.oc_profile_captured_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_match.argtypes = [_vp] * 8
 _lib.oc_select.argtypes = [_vp, _vp, _vp, _vp, _i, _f, _i64, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.oc_gather.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp]
@@ -282,6 +283,12 @@ class Context:
     def profile_read(self, kernel_id: int) -> tuple[int, float]:
         n, ms = C.c_int64(), C.c_double()
         _chk(_lib.oc_profile_read(self._h, kernel_id, C.byref(n), C.byref(ms)), "oc_profile_read")
+        return n.value, ms.value
+
+    def profile_captured_read(self, kernel_id: int) -> tuple[int, float]:
+        """(brackets captured into CUDA graphs, sum of their most recent recordings in ms)."""
+        n, ms = C.c_int64(), C.c_double()
+        _chk(_lib.oc_profile_captured_read(self._h, kernel_id, C.byref(n), C.byref(ms)), "oc_profile_captured_read")
         return n.value, ms.value
 
     def profile_span_read(self, kernel_id: int) -> tuple[int, float]:

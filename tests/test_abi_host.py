@@ -125,6 +125,7 @@ def test_null_context_and_bad_arguments_are_rejected_before_any_launch(oc):
     assert lib.oc_device_status(None, None) == oc.ERR_INVALID_ARG
     assert lib.oc_profile_read(None, 0, None, None) == oc.ERR_INVALID_ARG
     assert lib.oc_profile_span_read(None, 1, None, None) == oc.ERR_INVALID_ARG
+    assert lib.oc_profile_captured_read(None, 1, None, None) == oc.ERR_INVALID_ARG
     assert lib.oc_selftest_bounded_wait(None, 100, None) == oc.ERR_INVALID_ARG
     assert lib.oc_match_frame_noalloc(-1, C.byref(L), one, one, one, None, None) == oc.ERR_INVALID_ARG
     assert lib.oc_cache_step_host(None, C.byref(L), 0, 0.5, 0, one, one, one, None, None) == oc.ERR_INVALID_ARG

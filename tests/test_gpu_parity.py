@@ -432,6 +432,35 @@ def test_device_span_of_the_tensor_core_matcher(oc, oracle):
             ctx.profile_span_read(oc.K_SELECT)
 
 
+def test_event_brackets_captured_into_a_graph_are_taken_on_every_replay(oc, oracle):
+    w = inputs.sd3_token_cache(seed=8, B=2, H=32, W=32, C=256)
+    L, _ = H.layouts(oc, oracle, w)
+    x_dev = H.to_dev(w.x)
+    n = L.n_units
+    sim = torch.empty(n, device="cuda"); idx = torch.empty(n, dtype=torch.int32, device="cuda")
+    with H.make_ctx(oc, L) as ctx:
+        ctx.match(L, x_dev, sim, idx); torch.cuda.synchronize()
+        ref = idx.clone()
+        ctx.profile_reset()
+        ctx.profile_enable(1)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            ctx.match(L, x_dev, sim, idx, stream=torch.cuda.current_stream())
+        ctx.profile_enable(0)
+        assert ctx.profile_captured_read(oc.K_MATCH_FIN) == (0, 0.0)        # captured, never run
+        seen = []
+        for _ in range(3):
+            idx.zero_()
+            g.replay(); torch.cuda.synchronize()
+            k, ms = ctx.profile_captured_read(oc.K_MATCH_FIN)
+            assert k == 1 and ms > 0.0
+            seen.append(ms)
+            assert torch.equal(idx, ref)
+        # the eager counters saw the captured launches as launches, their timers did not
+        assert ctx.profile_read(oc.K_MATCH_FIN) == (1, 0.0)
+        del g
+
+
 def test_runtime_argument_errors_launch_nothing(oc, oracle):
     w = inputs.sd3_token_cache(seed=5, B=1, H=16, W=16, C=64)
     L, Lo = H.layouts(oc, oracle, w)
