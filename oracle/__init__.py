@@ -152,8 +152,14 @@ def rows_for(L: Layout, channels: int, elem_bytes: int) -> Rows:
     if L.kind == KIND_TOKEN:
         return Rows(cb, 1, 0, cb, 1 << 40, 0)
     if L.kind == KIND_FRAME:
-        fb = L.H * L.W * cb
-        return Rows(fb, 1, 0, fb, 1 << 40, 0)
+        if L.gy * L.gx == 1:
+            fb = L.H * L.W * cb
+            return Rows(fb, 1, 0, fb, 1 << 40, 0)
+        # a patch of a frame: H/gy segments of (W/gx)*C' elements, one per image row; the gx
+        # patches of a patch row sit side by side, and patch rows follow one another uniformly
+        # through frames and batch elements (Section 3.3)
+        hp, wp = L.H // L.gy, L.W // L.gx
+        return Rows(wp * cb, hp, L.W * cb, wp * cb, L.gx, hp * L.W * cb)
     return Rows(cb, L.T, L.H * L.W * cb, cb, L.H * L.W, L.T * L.H * L.W * cb)
 
 
@@ -191,10 +197,10 @@ def match_token(L: Layout, x: np.ndarray, rows=None, want_full: bool = False):
 
 def match_frame(L: Layout, x: np.ndarray, want_pos: bool = False):
     _check(x, L)
-    n = L.B * L.T
+    n = L.B * L.T * L.gy * L.gx
     best_sim = np.empty(n, np.float32)
     best_idx = np.empty(n, np.int32)
-    pair = np.empty((L.B, max(L.T - 1, 0)), np.float32)
+    pair = np.empty((L.B, max(L.T - 1, 0)) + ((L.gy * L.gx,) if L.gy * L.gx > 1 else ()), np.float32)
     pos = np.empty((L.B, max(L.T - 1, 0), L.H * L.W), np.float32) if want_pos else None
     rc = lib().ocr_match_frame(C.byref(L.c()), _p(x), _p(best_sim), _p(best_idx), _p(pair), _p(pos))
     assert rc == 0, rc

@@ -11,7 +11,9 @@
  *   - dtype 0 = IEEE fp32, dtype 1 = bf16 stored as 16-bit patterns; every stored value is
  *     widened exactly to double and all arithmetic is double;
  *   - a unit is a token (kind 0), a frame (kind 1) or a 1x1xT block (kind 2); unit indices are
- *     global: token ((b*T+t)*H+y)*W+x, frame b*T+t, block b*H*W + y*W+x;
+ *     global: token ((b*T+t)*H+y)*W+x, frame b*T+t, block b*H*W + y*W+x; with patch-local
+ *     Frame Cache (Section 3.3, gy*gx > 1) the unit is one patch of one frame,
+ *     ((b*T+t)*gy+py)*gx+px;
  *   - outputs that the library produces in fp32 are rounded to fp32 once, at the end.
  *
  * Every function has at least one pin in the CPU test-suite (brute force in NumPy, closed forms,
@@ -31,7 +33,7 @@ typedef struct {
     int B, T, H, W, C;
     int sy, sx;      /* representative lattice stride (Section 3.2.1 / 3.2.3: local 2x2 groups) */
     int oy, ox;      /* which member of a group is the representative */
-    int gy, gx;      /* token groups (patches) per frame, Section 3.3 */
+    int gy, gx;      /* patches per frame, Section 3.3 (token and frame kinds) */
     int self_match;  /* every token is candidate and representative (tiny all-pairs config) */
     int frame_stat;  /* 0 mean of same-position token cosines, 1 cosine of the flat H*W*C descriptor */
     double eps;      /* floor applied to each norm */
@@ -82,10 +84,13 @@ double ocr_cosine(const void* x, int dtype, int64_t a_off, int64_t b_off, int64_
 /* ---- group structure -----------------------------------------------------------------------
  * token kind : a group is one patch of one frame, (b, t, py, px); units = (H/gy)*(W/gx) tokens,
  *              local index u = ly*(W/gx)+lx in row-major order of the patch.
- * frame kind : a group is one batch element; units = its T frames.
+ * frame kind : a group is one patch position of one batch element, (b, py, px) (Section 3.3's
+ *              (B*k*k, T, .) arrangement; gy = gx = 1 is the whole frame); units = the T
+ *              frame-patches at that position, local index u = t.
  * block kind : a group is one batch element; units = its H*W spatial positions. */
 int64_t ocr_num_groups(const ocr_layout* L) {
     if (L->kind == 0) return (int64_t)L->B * L->T * L->gy * L->gx;
+    if (L->kind == 1) return (int64_t)L->B * L->gy * L->gx;
     return L->B;
 }
 int64_t ocr_units_per_group(const ocr_layout* L) {
@@ -102,6 +107,10 @@ int64_t ocr_unit_index(const ocr_layout* L, int64_t g, int64_t u) {
         int64_t px = g % L->gx, py = (g / L->gx) % L->gy, bt = g / ((int64_t)L->gx * L->gy);
         int64_t ly = u / Wp, lx = u % Wp;
         return (bt * L->H + py * Hp + ly) * L->W + px * Wp + lx;
+    }
+    if (L->kind == 1) {
+        int64_t np = (int64_t)L->gy * L->gx, b = g / np, patch = g % np;
+        return (b * L->T + u) * np + patch;
     }
     return g * ocr_units_per_group(L) + u;
 }
@@ -194,46 +203,70 @@ int ocr_match_token(const ocr_layout* L, const void* x, const int32_t* rows, int
  * similarity of two frames is, by default, the mean over positions p of cos(x[t,p,:], x[u,p,:]);
  * with frame_stat = 1 it is the cosine of the two flattened H*W*C descriptors (the paper's literal
  * (B, T, H*W*C) reshape).  A candidate t is compared with its adjacent frames t-1 and t+1 only;
- * best = maximum, ties to the lower frame.  pair_sim[b][t-1], t = 1..T-1, is the statistic of
- * (t, t-1) for every adjacent pair; pos_sim (nullable) [b][t-1][p] the per-position cosines. */
-static double frame_stat(const ocr_layout* L, const void* x, int64_t fa, int64_t fb, float* pos_out) {
-    const int64_t P = (int64_t)L->H * L->W, C = L->C;
-    if (L->frame_stat == 1 && !pos_out)
-        return ocr_cosine(x, L->dtype, fa * P * C, fb * P * C, P * C, L->eps);
-    double acc = 0.0;
-    for (int64_t p = 0; p < P; ++p) {
-        double c = ocr_cosine(x, L->dtype, (fa * P + p) * C, (fb * P + p) * C, C, L->eps);
-        if (pos_out) pos_out[p] = (float)c;
-        acc += c;
+ * best = maximum, ties to the lower frame.
+ * Patch-local form (Section 3.3): the frame is cut into gy x gx equal patches and everything above
+ * is done per patch position, the descriptor being the patch's (H/gy)*(W/gx)*C elements; a unit is
+ * one patch of one frame and best_idx names the matched patch of the adjacent frame.
+ * pair_sim[b][t-1][patch], t = 1..T-1, is the statistic of (t, t-1) for every adjacent pair;
+ * pos_sim (nullable) [b][t-1][p] the per-position cosines (p = y*W+x in the frame). */
+static double patch_stat(const ocr_layout* L, const void* x, int64_t fa, int64_t fb, int64_t py, int64_t px) {
+    const int64_t Hp = L->H / L->gy, Wp = L->W / L->gx, C = L->C, P = (int64_t)L->H * L->W;
+    double acc = 0.0, dot = 0.0, na = 0.0, nb = 0.0;
+    for (int64_t ly = 0; ly < Hp; ++ly)
+        for (int64_t lx = 0; lx < Wp; ++lx) {
+            int64_t p = (py * Hp + ly) * L->W + px * Wp + lx;
+            int64_t ao = (fa * P + p) * C, bo = (fb * P + p) * C;
+            if (L->frame_stat == 1) {
+                for (int64_t c = 0; c < C; ++c) {
+                    double a = load_elem(x, L->dtype, ao + c), b = load_elem(x, L->dtype, bo + c);
+                    dot += a * b; na += a * a; nb += b * b;
+                }
+            } else {
+                acc += ocr_cosine(x, L->dtype, ao, bo, C, L->eps);
+            }
+        }
+    if (L->frame_stat == 1) {
+        na = sqrt(na); nb = sqrt(nb);
+        if (na < L->eps) na = L->eps;
+        if (nb < L->eps) nb = L->eps;
+        return clamp1(dot / (na * nb));
     }
-    if (L->frame_stat == 1) return ocr_cosine(x, L->dtype, fa * P * C, fb * P * C, P * C, L->eps);
-    return acc / (double)P;
+    return acc / (double)(Hp * Wp);
 }
 
 int ocr_match_frame(const ocr_layout* L, const void* x, float* best_sim, int32_t* best_idx,
                     float* pair_sim, float* pos_sim) {
     if (L->kind != 1) return 1;
-    const int64_t T = L->T, P = (int64_t)L->H * L->W;
+    if (L->gy <= 0 || L->gx <= 0 || L->H % L->gy || L->W % L->gx) return 1;
+    const int64_t T = L->T, P = (int64_t)L->H * L->W, C = L->C;
+    const int64_t np = (int64_t)L->gy * L->gx;
     const int64_t n_pairs = (int64_t)L->B * (T - 1);
-    double* pair = (double*)malloc(sizeof(double) * (size_t)(n_pairs > 0 ? n_pairs : 1));
+    double* pair = (double*)malloc(sizeof(double) * (size_t)(n_pairs * np > 0 ? n_pairs * np : 1));
     if (!pair) return 2;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int64_t q = 0; q < n_pairs; ++q) {
         int64_t b = q / (T - 1), t = q % (T - 1) + 1;
-        pair[q] = frame_stat(L, x, b * T + t, b * T + t - 1, pos_sim ? pos_sim + q * P : NULL);
-        if (pair_sim) pair_sim[q] = (float)pair[q];
+        int64_t fa = b * T + t, fb = fa - 1;
+        for (int64_t patch = 0; patch < np; ++patch) {
+            pair[q * np + patch] = patch_stat(L, x, fa, fb, patch / L->gx, patch % L->gx);
+            if (pair_sim) pair_sim[q * np + patch] = (float)pair[q * np + patch];
+        }
+        if (pos_sim)
+            for (int64_t p = 0; p < P; ++p)
+                pos_sim[q * P + p] = (float)ocr_cosine(x, L->dtype, (fa * P + p) * C, (fb * P + p) * C, C, L->eps);
     }
     for (int64_t b = 0; b < L->B; ++b)
-        for (int64_t t = 0; t < T; ++t) {
-            int64_t i = b * T + t;
-            if (t % 2 == 0) { best_sim[i] = -INFINITY; best_idx[i] = (int32_t)i; continue; }
-            double best = pair[b * (T - 1) + (t - 1)]; int64_t arg = i - 1;      /* (t, t-1) */
-            if (t + 1 < T) {
-                double nxt = pair[b * (T - 1) + t];                             /* (t+1, t) */
-                if (nxt > best) { best = nxt; arg = i + 1; }
+        for (int64_t t = 0; t < T; ++t)
+            for (int64_t patch = 0; patch < np; ++patch) {
+                int64_t i = (b * T + t) * np + patch;
+                if (t % 2 == 0) { best_sim[i] = -INFINITY; best_idx[i] = (int32_t)i; continue; }
+                double best = pair[(b * (T - 1) + (t - 1)) * np + patch]; int64_t arg = i - np;   /* (t, t-1) */
+                if (t + 1 < T) {
+                    double nxt = pair[(b * (T - 1) + t) * np + patch];                             /* (t+1, t) */
+                    if (nxt > best) { best = nxt; arg = i + np; }
+                }
+                best_sim[i] = (float)best; best_idx[i] = (int32_t)arg;
             }
-            best_sim[i] = (float)best; best_idx[i] = (int32_t)arg;
-        }
     free(pair);
     return 0;
 }

@@ -251,6 +251,84 @@ def test_match_frame_bruteforce(oracle, T, stat):
             assert abs(got["best_sim"][i] - want[0]) < 1e-7
 
 
+def patch_major(x, gy, gx):
+    """Section 3.3's rearrangement, written with NumPy: (B,T,k,H/k,k,W/k,C) -> (B*k*k, T, (H/k)*(W/k), C)."""
+    B, T, H, W, Cc = x.shape
+    hp, wp = H // gy, W // gx
+    return x.reshape(B, T, gy, hp, gx, wp, Cc).transpose(0, 2, 4, 1, 3, 5, 6).reshape(B * gy * gx, T, hp * wp, Cc)
+
+
+@pytest.mark.parametrize("grid", [(2, 2), (1, 3), (3, 1), (2, 4), (6, 12)])
+@pytest.mark.parametrize("stat", [0, 1])
+def test_match_frame_patch_local_is_the_reshaped_problem(oracle, grid, stat):
+    """Patch-local Frame Cache = the whole-frame rule applied to every row of the rearranged array."""
+    gy, gx = grid
+    rng = np.random.default_rng(100 + gy * 16 + gx)
+    B, T, H, W, Cc = 2, 6, 6, 12, 8
+    xf = rng.standard_normal((B, T, H, W, Cc)).astype(np.float32)
+    xf[:, 1:] = 0.6 * xf[:, :-1] + 0.4 * xf[:, 1:]
+    x = inputs.to_bf16_bits(xf)
+    x64 = as_f64(x, inputs.BF16)
+    L = oracle.Layout(oracle.KIND_FRAME, oracle.DT_BF16, B, T, H, W, Cc, gy=gy, gx=gx, frame_stat=stat)
+    got = oracle.match_frame(L, x, want_pos=True)
+    npatch = gy * gx
+    assert L.n_groups == B * npatch and L.units_per_group == T and L.n_units == B * T * npatch
+    xp = patch_major(x64, gy, gx)                                  # [B*np, T, Pp, C]
+    a, b = xp[:, 1:], xp[:, :-1]
+    pos = (a * b).sum(-1) / (np.linalg.norm(a, axis=-1) * np.linalg.norm(b, axis=-1))
+    if stat == 0:
+        pair = pos.mean(axis=-1)                                   # [B*np, T-1]
+    else:
+        af, bf = a.reshape(B * npatch, T - 1, -1), b.reshape(B * npatch, T - 1, -1)
+        pair = (af * bf).sum(-1) / (np.linalg.norm(af, axis=-1) * np.linalg.norm(bf, axis=-1))
+    want_pair = pair.reshape(B, npatch, T - 1).transpose(0, 2, 1)  # [B, T-1, np]
+    assert np.allclose(got["pair_sim"].reshape(B, T - 1, npatch), want_pair, atol=1e-7, rtol=0)
+    # per-position cosines stay in frame order
+    a5, b5 = x64[:, 1:], x64[:, :-1]
+    pos5 = (a5 * b5).sum(-1) / (np.linalg.norm(a5, axis=-1) * np.linalg.norm(b5, axis=-1))
+    assert np.allclose(got["pos_sim"], pos5.reshape(B, T - 1, -1), atol=1e-7, rtol=0)
+    for bb in range(B):
+        for t in range(T):
+            for pt in range(npatch):
+                i = ((bb * T + t) * gy + pt // gx) * gx + pt % gx
+                assert L.unit_index(bb * npatch + pt, t) == i
+                if t % 2 == 0:
+                    assert got["best_idx"][i] == i and np.isneginf(got["best_sim"][i])
+                    continue
+                opts = [(want_pair[bb, t - 1, pt], i - npatch)]
+                if t + 1 < T:
+                    opts.append((want_pair[bb, t, pt], i + npatch))
+                want = max(opts, key=lambda o: (o[0], -o[1]))
+                assert got["best_idx"][i] == want[1]
+                assert abs(got["best_sim"][i] - want[0]) < 1e-7
+
+
+def test_match_frame_patch_local_equals_whole_frame_match_of_each_patch(oracle):
+    """Cutting a patch out and matching it as a frame of its own gives that patch's results."""
+    rng = np.random.default_rng(77)
+    B, T, H, W, Cc, gy, gx = 2, 5, 4, 6, 8, 2, 3
+    x = rng.standard_normal((B, T, H, W, Cc)).astype(np.float32)
+    x[:, 1:] = 0.5 * x[:, :-1] + 0.5 * x[:, 1:]
+    hp, wp, npatch = H // gy, W // gx, gy * gx
+    for stat in (0, 1):
+        L = oracle.Layout(oracle.KIND_FRAME, 0, B, T, H, W, Cc, gy=gy, gx=gx, frame_stat=stat)
+        got = oracle.match_frame(L, x)
+        for py in range(gy):
+            for px in range(gx):
+                sub = np.ascontiguousarray(x[:, :, py * hp:(py + 1) * hp, px * wp:(px + 1) * wp, :])
+                Ls = oracle.Layout(oracle.KIND_FRAME, 0, B, T, hp, wp, Cc, frame_stat=stat)
+                ws = oracle.match_frame(Ls, sub)
+                pt = py * gx + px
+                assert np.array_equal(got["pair_sim"][:, :, pt], ws["pair_sim"])
+                assert np.array_equal(got["best_sim"][pt::npatch], ws["best_sim"])
+                assert np.array_equal(got["best_idx"][pt::npatch], ws["best_idx"] * npatch + pt)
+    # the patch means, weighted equally (equal areas), average to the whole-frame mean
+    L1 = oracle.Layout(oracle.KIND_FRAME, 0, B, T, H, W, Cc)
+    Lp = oracle.Layout(oracle.KIND_FRAME, 0, B, T, H, W, Cc, gy=gy, gx=gx)
+    assert np.allclose(oracle.match_frame(Lp, x)["pair_sim"].astype(np.float64).mean(-1),
+                       oracle.match_frame(L1, x)["pair_sim"], atol=2e-7, rtol=0)
+
+
 def test_match_frame_ar1_expectation(oracle):
     """AR(1) frames: E[cos(x_t, x_{t-1})] = rho for unit-variance stationary rows (closed form)."""
     rho = 0.95
@@ -325,6 +403,7 @@ def np_select(L, best_sim, best_idx, mode, thr, n_reuse, stride):
 @pytest.mark.parametrize("kind,shape,groups", [
     (0, (2, 1, 8, 8, 8), (1, 1)), (0, (1, 2, 8, 16, 8), (2, 2)),
     (1, (3, 7, 2, 2, 8), (1, 1)), (2, (2, 3, 6, 8, 8), (1, 1)),
+    (1, (2, 7, 4, 6, 8), (2, 3)),
 ])
 @pytest.mark.parametrize("mode", [0, 1])
 def test_select_bruteforce(oracle, kind, shape, groups, mode):
@@ -463,6 +542,56 @@ def test_restore_sources_no_averaging(oracle, kind):
     for slot, i in enumerate(s["kept_idx"]):
         if i >= 0:
             assert y[slot].tobytes() == xr[i].tobytes()
+
+
+def patch_rows(t, gy, gx):
+    """[B*T*gy*gx, (H/gy)*(W/gx)*C] rows of the frame patches, unit order ((b*T+t)*gy+py)*gx+px."""
+    B, T, H, W, Cc = t.shape
+    hp, wp = H // gy, W // gx
+    return np.ascontiguousarray(t.reshape(B, T, gy, hp, gx, wp, Cc).transpose(0, 1, 2, 4, 3, 5, 6)).reshape(
+        B * T * gy * gx, hp * wp * Cc)
+
+
+@pytest.mark.parametrize("grid", [(2, 3), (1, 2), (4, 1)])
+def test_frame_patch_rows_gather_restore(oracle, grid):
+    """Patch-local Frame Cache moves patches of frames: the rows are the NumPy patch slices."""
+    gy, gx = grid
+    rng = np.random.default_rng(300 + gy * 8 + gx)
+    shape = (2, 5, 4, 6, 8)
+    Cout = 12
+    x = rng.standard_normal(shape).astype(np.float32)
+    x[:, 1:] = 0.5 * x[:, :-1] + 0.5 * x[:, 1:]
+    L = oracle.Layout(oracle.KIND_FRAME, 0, *shape, gy=gy, gx=gx)
+    m = oracle.match(L, x)
+    # identity selection: gather is the patch-major copy, restore brings the frames back
+    s0 = oracle.select(L, m["best_sim"], m["best_idx"], 0, 2.0, 0)
+    Rx = oracle.rows_for(L, shape[-1], 4)
+    y0 = oracle.gather(Rx, x, s0["kept_idx"]).view(np.float32)
+    xr = patch_rows(x, gy, gx)
+    assert np.array_equal(np.sort(s0["kept_idx"]), np.arange(L.n_units))
+    assert y0.reshape(L.n_units, -1).tobytes() == xr[s0["kept_idx"]].tobytes()
+    back = oracle.restore(Rx, y0, np.zeros_like(x), L.n_units, s0["slot_of"], s0["match_map"])
+    assert back.tobytes() == x.tobytes()
+    # a real selection: every output patch is bit-identical to exactly one source
+    thr = float(np.median(m["best_sim"][np.isfinite(m["best_sim"])]))
+    s = oracle.select(L, m["best_sim"], m["best_idx"], 0, thr, 0)
+    assert 0 < (s["slot_of"] < 0).sum() < L.n_units
+    y = oracle.gather(Rx, x, s["kept_idx"]).view(np.float32).reshape(s["kept_idx"].size, -1)
+    for slot, i in enumerate(s["kept_idx"]):
+        if i >= 0:
+            assert y[slot].tobytes() == xr[i].tobytes()
+    R = oracle.rows_for(L, Cout, 4)
+    out_shape = shape[:-1] + (Cout,)
+    cache = rng.standard_normal(out_shape).astype(np.float32)
+    z = rng.standard_normal((s["kept_idx"].size, R.row_bytes // 4)).astype(np.float32)
+    out = oracle.restore(R, z, cache, L.n_units, s["slot_of"], s["match_map"]).view(np.float32)
+    o, c = patch_rows(out.reshape(out_shape), gy, gx), patch_rows(cache, gy, gx)
+    for i in range(L.n_units):
+        want = z[s["slot_of"][i]] if s["slot_of"][i] >= 0 else c[i]
+        assert o[i].tobytes() == want.tobytes()
+        # the stand-in of a skipped patch is the same patch position of an adjacent frame
+        if s["slot_of"][i] < 0:
+            assert abs(s["match_map"][i] - i) == gy * gx
 
 
 def unit_rows_generic(t, L):
