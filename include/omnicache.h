@@ -16,7 +16,9 @@
  *     C * element size is a multiple of 16 bytes.
  *   - A "unit" is a token (OC_KIND_TOKEN), a frame (OC_KIND_FRAME) or a 1x1xT temporal block
  *     (OC_KIND_BLOCK).  Unit indices are global and int32:
- *         token ((b*T + t)*H + y)*W + x,     frame b*T + t,     block b*H*W + y*W + x.
+ *         token ((b*T + t)*H + y)*W + x,     frame b*T + t,     block b*H*W + y*W + x;
+ *     with patch-local Frame Cache (gy*gx > 1) the unit is one patch of one frame,
+ *         ((b*T + t)*gy + py)*gx + px.
  *   - Every call returns an oc_status.  On a host-detected error nothing is launched and no output
  *     is written.  Device-side conditions (an expired bounded wait) land in a status word read by
  *     oc_device_status().  No call aborts or throws.
@@ -57,18 +59,22 @@ enum { OC_FRAME_MEAN_POS_COS = 0, OC_FRAME_FLAT_COS = 1 };
  *          every other token is a candidate, compared with all representatives of its patch.
  *          self_match = 1: every token is both (all pairs, self excluded); needs gy = gx = 1.
  *   FRAME: even frames are representatives, odd frames candidates, each compared with its two
- *          adjacent frames (alternating sets, Section 3.2.2).  sy..gx are ignored (gy = gx = 1).
+ *          adjacent frames (alternating sets, Section 3.2.2).  sy..ox are ignored.  gy x gx > 1
+ *          is the patch-local form of Section 3.3: each frame is cut into gy x gx equal patches,
+ *          every patch position (b, py, px) is a matching and selection problem of its own over
+ *          its T frame-patches (the paper's (B*k*k, T, (H/k)*(W/k)*C) arrangement, read in place),
+ *          and the statistic runs over the patch's positions only.  gy = gx = 0 means 1.
  *   BLOCK: positions are cut into sy x sx neighbourhoods; the (oy, ox) member is the
  *          representative, the others are compared with it over the T*C block descriptor
  *          (Section 3.2.1).  gy = gx = 1.
- * H/gy must be a multiple of sy and W/gx of sx (TOKEN, BLOCK). */
+ * H must be a multiple of gy and W of gx; H/gy must be a multiple of sy and W/gx of sx (TOKEN, BLOCK). */
 typedef struct oc_layout {
     int kind;        /* OC_KIND_*  */
     int dtype;       /* OC_DTYPE_* of the feature tensor */
     int B, T, H, W, C;
     int sy, sx;      /* representative lattice stride, >= 1, sy*sx >= 2 unless self_match */
     int oy, ox;      /* representative offset inside a neighbourhood, 0 <= oy < sy, 0 <= ox < sx */
-    int gy, gx;      /* patches per frame */
+    int gy, gx;      /* patches per frame (TOKEN, FRAME) */
     int self_match;  /* TOKEN only */
     int frame_stat;  /* FRAME only: OC_FRAME_* */
     float eps;       /* floor applied to each vector norm; cos = <a,b> / (max(|a|,eps) max(|b|,eps)) */
@@ -103,7 +109,8 @@ const char* oc_status_str(oc_status s);
 oc_status oc_layout_check(const oc_layout* layout);
 
 /* Group structure of a layout: a group is an independent selection problem (TOKEN: one patch of one
- * frame; FRAME, BLOCK: one batch element).  Any output pointer may be null. */
+ * frame; FRAME: one patch position of one batch element, its units being T frame-patches that lie
+ * gy*gx apart in unit order; BLOCK: one batch element).  Any output pointer may be null. */
 oc_status oc_layout_counts(const oc_layout* layout, int64_t* n_groups, int64_t* units_per_group,
                            int64_t* reps_per_group);
 
@@ -201,7 +208,8 @@ oc_status oc_profile_captured_read(oc_ctx* ctx, int kernel_id, int64_t* launches
  *   aux_sim   nullable.  TOKEN: [n_groups][units_per_group][reps_per_group] float, every candidate
  *             row's full similarity row (rows of representatives and the self-match diagonal are
  *             not written).  FRAME: [B][T-1][H*W] per-position cosines of frame t vs t-1.
- *   pair_sim  nullable, FRAME only: [B][T-1] statistic of every adjacent pair (t, t-1).
+ *   pair_sim  nullable, FRAME only: [B][T-1][gy*gx] statistic of every adjacent pair (t, t-1),
+ *             per patch.
  * bf16 TOKEN layouts without self_match run on the tcgen05 tensor cores (fp32 accumulation);
  * everything else on fp32 FMA pipelines.  Needs oc_match_workspace_bytes() of context workspace
  * (OC_ERR_WORKSPACE otherwise).  Calls on one context must not overlap on the device. */
@@ -266,7 +274,7 @@ oc_status oc_layer_cache_clear(oc_ctx* ctx);
  * oc_match() needs a context, and a context owns cudaMalloc'd scratch; this variant needs neither.
  *
  * It computes exactly what oc_match() computes for an OC_KIND_FRAME layout (best_sim, best_idx and,
- * if pair_sim is not null, the [B][T-1] adjacent-pair statistic), with the same kernels, but keeps
+ * if pair_sim is not null, the [B][T-1][gy*gx] adjacent-pair statistic), with the same kernels, but keeps
  * its partial sums in a fixed array of OC_NOALLOC_SCRATCH_BYTES bytes that is part of the library
  * image: every GPU that loads the library holds that array until the process exits.
  *   - A layout whose scratch need (oc_match_workspace_bytes) exceeds OC_NOALLOC_SCRATCH_BYTES is

@@ -87,39 +87,37 @@ double ocr_cosine(const void* x, int dtype, int64_t a_off, int64_t b_off, int64_
  * frame kind : a group is one patch position of one batch element, (b, py, px) (Section 3.3's
  *              (B*k*k, T, .) arrangement; gy = gx = 1 is the whole frame); units = the T
  *              frame-patches at that position, local index u = t.
- * block kind : a group is one batch element; units = its H*W spatial positions. */
+ * block kind : a group is one patch of one batch element, (b, py, px) (gy = gx = 1: all positions);
+ *              units = the (H/gy)*(W/gx) spatial positions of the patch, row-major.  A block is
+ *              always compared with the representative of its own sy x sx neighbourhood; the patch
+ *              confines the selection ("the r most redundant" of the patch, Section 3.3). */
 int64_t ocr_num_groups(const ocr_layout* L) {
     if (L->kind == 0) return (int64_t)L->B * L->T * L->gy * L->gx;
-    if (L->kind == 1) return (int64_t)L->B * L->gy * L->gx;
-    return L->B;
+    return (int64_t)L->B * L->gy * L->gx;
 }
 int64_t ocr_units_per_group(const ocr_layout* L) {
-    if (L->kind == 0) return (int64_t)(L->H / L->gy) * (L->W / L->gx);
     if (L->kind == 1) return L->T;
-    return (int64_t)L->H * L->W;
+    return (int64_t)(L->H / L->gy) * (L->W / L->gx);
 }
 int64_t ocr_num_units(const ocr_layout* L) { return ocr_num_groups(L) * ocr_units_per_group(L); }
 
 /* global unit index of local unit u of group g */
 int64_t ocr_unit_index(const ocr_layout* L, int64_t g, int64_t u) {
-    if (L->kind == 0) {
+    if (L->kind != 1) {                        /* token: bt = frame b*T+t; block: bt = batch element */
         int Hp = L->H / L->gy, Wp = L->W / L->gx;
         int64_t px = g % L->gx, py = (g / L->gx) % L->gy, bt = g / ((int64_t)L->gx * L->gy);
         int64_t ly = u / Wp, lx = u % Wp;
         return (bt * L->H + py * Hp + ly) * L->W + px * Wp + lx;
     }
-    if (L->kind == 1) {
-        int64_t np = (int64_t)L->gy * L->gx, b = g / np, patch = g % np;
-        return (b * L->T + u) * np + patch;
-    }
-    return g * ocr_units_per_group(L) + u;
+    int64_t np = (int64_t)L->gy * L->gx, b = g / np, patch = g % np;
+    return (b * L->T + u) * np + patch;
 }
 
 /* is local unit u a representative (always computed, never reused)? */
 int ocr_is_rep(const ocr_layout* L, int64_t u) {
     if (L->kind == 1) return (u % 2) == 0;                 /* alternating frame sets, Section 3.2.2 */
     if (L->self_match) return 1;
-    int Wl = (L->kind == 0) ? L->W / L->gx : L->W;
+    int Wl = L->W / L->gx;                     /* patches hold whole sy x sx neighbourhoods */
     int64_t ly = u / Wl, lx = u % Wl;
     return (ly % L->sy) == L->oy && (lx % L->sx) == L->ox;
 }
@@ -277,6 +275,7 @@ int ocr_match_frame(const ocr_layout* L, const void* x, float* best_sim, int32_t
  * the (oy, ox) member is the representative, every other member is compared with it. */
 int ocr_match_block(const ocr_layout* L, const void* x, float* best_sim, int32_t* best_idx) {
     if (L->kind != 2) return 1;
+    if (L->gy <= 0 || L->gx <= 0 || L->H % (L->gy * L->sy) || L->W % (L->gx * L->sx)) return 1;
     const int64_t T = L->T, H = L->H, W = L->W, C = L->C, P = H * W;
 #pragma omp parallel for schedule(dynamic, 16)
     for (int64_t i = 0; i < (int64_t)L->B * P; ++i) {

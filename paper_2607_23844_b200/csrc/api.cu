@@ -58,10 +58,15 @@ oc_status make_geo(const oc_layout* L, Geo* g) {
     if (n_tok > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
     if (L->kind == OC_KIND_FRAME) {
         if (L->frame_stat != OC_FRAME_MEAN_POS_COS && L->frame_stat != OC_FRAME_FLAT_COS) return OC_ERR_INVALID_ARG;
-        g->sy = g->sx = 1; g->oy = g->ox = 0; g->gy = g->gx = 1; g->self_match = 0;
-        g->Hp = L->H; g->Wp = L->W; g->Hs = L->H; g->Ws = L->W;
-        g->n_groups = L->B; g->units_per_group = L->T; g->reps_per_group = (L->T + 1) / 2;
-        g->n_units = (int64_t)L->B * L->T;
+        // patch-local Frame Cache (Section 3.3): gy x gx equal patches per frame, one group per
+        // patch position of a batch element; a layout that leaves gy = gx = 0 means whole frames
+        g->gy = L->gy > 0 ? L->gy : 1; g->gx = L->gx > 0 ? L->gx : 1;
+        if (L->gy < 0 || L->gx < 0 || L->H % g->gy != 0 || L->W % g->gx != 0) return OC_ERR_INVALID_ARG;
+        g->sy = g->sx = 1; g->oy = g->ox = 0; g->self_match = 0;
+        g->Hp = L->H / g->gy; g->Wp = L->W / g->gx; g->Hs = g->Hp; g->Ws = g->Wp;
+        g->n_groups = (int64_t)L->B * g->gy * g->gx; g->units_per_group = L->T; g->reps_per_group = (L->T + 1) / 2;
+        g->n_units = g->n_groups * L->T;
+        if (g->n_units > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
         return OC_OK;
     }
     if (L->gy <= 0 || L->gx <= 0) return OC_ERR_INVALID_ARG;
@@ -177,7 +182,10 @@ oc_status oc_rows_from_layout(const oc_layout* layout, int channels, int elem_by
     if (g.kind == OC_KIND_TOKEN) {
         *rows = oc_rows{cb, 1, 0, cb, (int64_t)1 << 40, 0};
     } else if (g.kind == OC_KIND_FRAME) {
-        *rows = oc_rows{P * cb, 1, 0, P * cb, (int64_t)1 << 40, 0};
+        if (g.gy * g.gx == 1) *rows = oc_rows{P * cb, 1, 0, P * cb, (int64_t)1 << 40, 0};
+        // a patch of a frame: Hp segments of Wp*C' elements; the gx patches of a patch row sit side by
+        // side and patch rows follow one another at one pitch through frames and batch elements
+        else *rows = oc_rows{g.Wp * cb, g.Hp, (int64_t)g.W * cb, g.Wp * cb, g.gx, (int64_t)g.Hp * g.W * cb};
     } else {
         *rows = oc_rows{cb, g.T, P * cb, cb, P, (int64_t)g.T * P * cb};
     }

@@ -130,6 +130,10 @@ __host__ __device__ inline int64_t gm_unit_index(const GroupMap& m, int64_t g, i
         int ly = u / m.Wp, lx = u - ly * m.Wp;
         return (bt * m.H + (int64_t)py * m.Hp + ly) * m.W + (int64_t)px * m.Wp + lx;
     }
+    if (m.kind == OC_KIND_FRAME) {                     // group (b, patch): its frames are n_patches apart
+        const int64_t np = (int64_t)m.gy * m.gx, b = g / np, patch = g - b * np;
+        return (b * m.units_per_group + u) * np + patch;
+    }
     return g * m.units_per_group + u;
 }
 __host__ __device__ inline bool gm_is_rep(const GroupMap& m, int u) {

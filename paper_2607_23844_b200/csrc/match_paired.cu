@@ -37,15 +37,42 @@ __device__ __forceinline__ float cta_sum_fixed(float v, float* sh /*[PAIR_THREAD
 }
 
 // ------------------------------------------------------------------------------------------------
+// Patch-local Frame Cache (Section 3.3): the frame is cut into gy x gx equal patches and every
+// patch position is a matching problem of its own.  The position tiles of the kernels below never
+// straddle a patch: tile i covers local positions of patch i / tiles_per_patch, so a partial record
+// belongs to one (pair, patch) and the per-patch statistics are sums of whole records.  With one
+// patch the local position IS the frame position and no index arithmetic is added.
+// ------------------------------------------------------------------------------------------------
+struct PatchGrid {
+    int n_patches, gx, Hp, Wp, W;
+    int Pp;                 // positions per patch
+    int tiles_per_patch;
+};
+static PatchGrid make_patch_grid(const Geo& g, int pos_per_tile) {
+    PatchGrid pg;
+    pg.n_patches = g.gy * g.gx; pg.gx = g.gx; pg.Hp = g.Hp; pg.Wp = g.Wp; pg.W = g.W;
+    pg.Pp = g.Hp * g.Wp;
+    pg.tiles_per_patch = (pg.Pp + pos_per_tile - 1) / pos_per_tile;
+    return pg;
+}
+// frame position of local position lp of a patch
+__device__ __forceinline__ int patch_position(const PatchGrid& pg, int patch, int lp) {
+    if (pg.n_patches == 1) return lp;
+    const int py = patch / pg.gx, px = patch - py * pg.gx;
+    const int ly = lp / pg.Wp, lx = lp - ly * pg.Wp;
+    return (py * pg.Hp + ly) * pg.W + px * pg.Wp + lx;
+}
+
+// ------------------------------------------------------------------------------------------------
 // Frame Cache: for every adjacent pair (t, t-1) and position p, cos(x[t,p,:], x[t-1,p,:]).
-// grid = (position tiles, B*(T-1)).  A CTA covers POS_PER_CTA consecutive positions of one pair and
-// writes one partial record {sum cos, sum dot, sum |a|^2, sum |b|^2}.  Frame t is read from HBM by
-// pair (t, t-1) and again, out of L2, by pair (t+1, t).
+// grid = (position tiles, B*(T-1)).  A CTA covers POS_PER_CTA consecutive positions of one patch of
+// one pair and writes one partial record {sum cos, sum dot, sum |a|^2, sum |b|^2}.  Frame t is read
+// from HBM by pair (t, t-1) and again, out of L2, by pair (t+1, t).
 // ------------------------------------------------------------------------------------------------
 template <int DT, int LPR>
 __global__ void __launch_bounds__(PAIR_THREADS)
 frame_pair_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float eps,
-                  float* __restrict__ pos_sim, float4* __restrict__ partial, int pos_per_cta) {
+                  float* __restrict__ pos_sim, float4* __restrict__ partial, int pos_per_cta, PatchGrid pg) {
     pdl_enter();
     __shared__ float sh[PAIR_THREADS];
     const int q = blockIdx.y;                       // pair index b*(T-1) + (t-1)
@@ -55,14 +82,16 @@ frame_pair_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float ep
     const long long row_bytes = (long long)cpr * 16;
     const uint8_t* cur = x + ((long long)(b * T + t) * P) * row_bytes;
     const uint8_t* prv = cur - (long long)P * row_bytes;
-    const int p_begin = blockIdx.x * pos_per_cta;
-    const int p_end = min(P, p_begin + pos_per_cta);
+    int patch = 0, tile = blockIdx.x;
+    if (pg.n_patches > 1) { patch = tile / pg.tiles_per_patch; tile -= patch * pg.tiles_per_patch; }
+    const int p_begin = tile * pos_per_cta;
+    const int p_end = min(pg.Pp, p_begin + pos_per_cta);
 
     float s_cos = 0.f, s_dot = 0.f, s_na = 0.f, s_nb = 0.f;
     // the trip count is the same for every thread of the CTA: the shuffles below name all 32 lanes
     for (int p0 = p_begin; p0 < p_end; p0 += groups) {
-        const int p = p0 + grp;
-        const bool valid = p < p_end;
+        const bool valid = p0 + grp < p_end;
+        const int p = valid ? patch_position(pg, patch, p0 + grp) : 0;
         float dot = 0.f, na = 0.f, nb = 0.f;
         if (valid) {
             const uint8_t* a = cur + (long long)p * row_bytes;
@@ -101,7 +130,7 @@ static constexpr int MARCH_CPL = 8;      // most 16-byte chunks a lane may hold 
 template <int DT, int LPR, int CPL>
 __global__ void __launch_bounds__(PAIR_THREADS)
 frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float eps, int seg_len, int n_seg,
-                   float* __restrict__ pos_sim, float4* __restrict__ partial) {
+                   float* __restrict__ pos_sim, float4* __restrict__ partial, PatchGrid pg) {
     pdl_enter();
     extern __shared__ float4 warp_part[];                 // [seg_len][PAIR_THREADS / 32]
     constexpr int GROUPS = PAIR_THREADS / LPR, WARPS = PAIR_THREADS / 32;
@@ -109,8 +138,10 @@ frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float e
     const int t0 = seg * seg_len;                         // first frame of the segment (as "previous")
     const int t1 = min(T - 1, t0 + seg_len);              // last frame of the segment
     const int grp = threadIdx.x / LPR, lane = threadIdx.x % LPR, warp = threadIdx.x >> 5, wl = threadIdx.x & 31;
-    const int p = blockIdx.x * GROUPS + grp;
-    const bool valid = p < P;
+    int patch = 0, tile = blockIdx.x;
+    if (pg.n_patches > 1) { patch = tile / pg.tiles_per_patch; tile -= patch * pg.tiles_per_patch; }
+    const bool valid = tile * GROUPS + grp < pg.Pp;
+    const int p = valid ? patch_position(pg, patch, tile * GROUPS + grp) : 0;
     const long long row_bytes = (long long)cpr * 16;
     const long long frame_bytes = (long long)P * row_bytes;
     const uint8_t* base = x + ((long long)b * T * P + (valid ? p : 0)) * row_bytes;
@@ -165,15 +196,16 @@ frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float e
     }
 }
 
-// One warp per frame: it sums, in a fixed order, the CTA partials of the pair (t, t-1) and of the
-// pair (t+1, t), publishes the first as pair_sim[t-1] and, for an odd (candidate) frame, picks the
-// better of its two adjacent representatives.  Every warp is independent, so frames run in parallel.
-__device__ __forceinline__ float frame_pair_value(const float4* __restrict__ partial, int n_tiles, int q, int P,
+// One warp per unit (a frame, or one patch of a frame): it sums, in a fixed order, the CTA partials
+// of the pair (t, t-1) and of the pair (t+1, t) that belong to its patch, publishes the first as
+// pair_sim[t-1][patch] and, for an odd (candidate) frame, picks the better of its two adjacent
+// representatives.  Every warp is independent, so units run in parallel.
+__device__ __forceinline__ float frame_pair_value(const float4* __restrict__ rec, int n_rec, int n_pos,
                                                   int stat, float eps) {
     const int lane = threadIdx.x & 31;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    for (int i = lane; i < n_tiles; i += 32) {
-        const float4 v = partial[(long long)q * n_tiles + i];
+    for (int i = lane; i < n_rec; i += 32) {
+        const float4 v = rec[i];
         a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
     }
 #pragma unroll
@@ -182,47 +214,51 @@ __device__ __forceinline__ float frame_pair_value(const float4* __restrict__ par
         a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, d); a3 += __shfl_xor_sync(0xFFFFFFFFu, a3, d);
     }
     return stat == OC_FRAME_FLAT_COS ? clamp_unit(a1 / (fmaxf(sqrtf(a2), eps) * fmaxf(sqrtf(a3), eps)))
-                                     : a0 / (float)P;
+                                     : a0 / (float)n_pos;
 }
 
 __global__ void __launch_bounds__(PAIR_THREADS)
-frame_finalize_kernel(const float4* __restrict__ partial, int n_tiles, int B, int T, int P, int stat,
-                      float eps, float* __restrict__ pair_ws, float* __restrict__ pair_sim,
+frame_finalize_kernel(const float4* __restrict__ partial, int tiles_per_patch, int n_patches, int B, int T,
+                      int Pp, int stat, float eps, float* __restrict__ pair_ws, float* __restrict__ pair_sim,
                       float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
     pdl_enter();
-    const int i = blockIdx.x * (PAIR_THREADS / 32) + (threadIdx.x >> 5);     // frame index b*T + t
+    const int i = blockIdx.x * (PAIR_THREADS / 32) + (threadIdx.x >> 5);     // unit index (b*T + t)*n_patches + patch
     const int lane = threadIdx.x & 31;
-    if (i >= B * T) return;                                                   // whole warps leave together
-    const int b = i / T, t = i - b * T;
+    if (i >= B * T * n_patches) return;                                       // whole warps leave together
+    const int bt = i / n_patches, patch = i - bt * n_patches;
+    const int b = bt / T, t = bt - b * T;
+    const long long q_prev = (long long)(b * (T - 1) + t - 1) * n_patches + patch;   // record run of (t, t-1)
     float with_prev = -INFINITY, with_next = -INFINITY;
     if (t >= 1) {
-        with_prev = frame_pair_value(partial, n_tiles, b * (T - 1) + t - 1, P, stat, eps);
-        if (lane == 0) { pair_ws[b * (T - 1) + t - 1] = with_prev; if (pair_sim) pair_sim[b * (T - 1) + t - 1] = with_prev; }
+        with_prev = frame_pair_value(partial + q_prev * tiles_per_patch, tiles_per_patch, Pp, stat, eps);
+        if (lane == 0) { pair_ws[q_prev] = with_prev; if (pair_sim) pair_sim[q_prev] = with_prev; }
     }
-    if ((t & 1) && t + 1 < T) with_next = frame_pair_value(partial, n_tiles, b * (T - 1) + t, P, stat, eps);
+    if ((t & 1) && t + 1 < T)
+        with_next = frame_pair_value(partial + (q_prev + n_patches) * tiles_per_patch, tiles_per_patch, Pp, stat, eps);
     if (lane == 0) {
         if ((t & 1) == 0) { best_sim[i] = -INFINITY; best_idx[i] = i; }
-        else if (with_next > with_prev) { best_sim[i] = with_next; best_idx[i] = i + 1; }
-        else { best_sim[i] = with_prev; best_idx[i] = i - 1; }
+        else if (with_next > with_prev) { best_sim[i] = with_next; best_idx[i] = i + n_patches; }
+        else { best_sim[i] = with_prev; best_idx[i] = i - n_patches; }
     }
 }
 
 template <int DT>
 static void frame_dispatch(int lpr, dim3 grid, cudaStream_t s, const uint8_t* x, int T, int P, int cpr, float eps,
-                           float* pos_sim, float4* partial, int ppc) {
+                           float* pos_sim, float4* partial, int ppc, const PatchGrid& pg) {
     switch (lpr) {
-        case 1:  OC_LAUNCH((frame_pair_kernel<DT, 1>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        case 2:  OC_LAUNCH((frame_pair_kernel<DT, 2>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        case 4:  OC_LAUNCH((frame_pair_kernel<DT, 4>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        case 8:  OC_LAUNCH((frame_pair_kernel<DT, 8>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        case 16: OC_LAUNCH((frame_pair_kernel<DT, 16>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
-        default: OC_LAUNCH((frame_pair_kernel<DT, 32>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc); break;
+        case 1:  OC_LAUNCH((frame_pair_kernel<DT, 1>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc, pg); break;
+        case 2:  OC_LAUNCH((frame_pair_kernel<DT, 2>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc, pg); break;
+        case 4:  OC_LAUNCH((frame_pair_kernel<DT, 4>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc, pg); break;
+        case 8:  OC_LAUNCH((frame_pair_kernel<DT, 8>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc, pg); break;
+        case 16: OC_LAUNCH((frame_pair_kernel<DT, 16>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc, pg); break;
+        default: OC_LAUNCH((frame_pair_kernel<DT, 32>), grid, PAIR_THREADS, 0, s, x, T, P, cpr, eps, pos_sim, partial, ppc, pg); break;
     }
 }
 
 struct FramePlan {
     bool march;          // time-marching kernel (rows short enough to keep in registers) or pair kernel
-    int lpr, n_tiles, ppc, seg_len, n_seg;
+    int lpr, n_tiles, ppc, seg_len, n_seg;     // n_tiles = patches * tiles per patch
+    PatchGrid pg;
 };
 static FramePlan frame_plan(const Geo& g) {
     FramePlan f;
@@ -232,8 +268,9 @@ static FramePlan frame_plan(const Geo& g) {
     f.march = g.T >= 2 && cpr <= l * MARCH_CPL;
     if (f.march) {
         f.lpr = l;
-        f.n_tiles = (P + PAIR_THREADS / l - 1) / (PAIR_THREADS / l);
         f.ppc = PAIR_THREADS / l;
+        f.pg = make_patch_grid(g, f.ppc);
+        f.n_tiles = f.pg.n_patches * f.pg.tiles_per_patch;
         // segments: enough CTAs for a few waves, but at least 6 pairs per segment (one frame re-read each)
         int n_seg = 1;
         while ((long long)f.n_tiles * g.B * n_seg < 148 * 4 && (g.T - 1) / (n_seg + 1) >= 6) ++n_seg;
@@ -243,7 +280,8 @@ static FramePlan frame_plan(const Geo& g) {
     } else {
         f.lpr = lanes_per_row(cpr);
         f.ppc = (PAIR_THREADS / f.lpr) * 4;              // every thread-group takes about 4 positions
-        f.n_tiles = (P + f.ppc - 1) / f.ppc;
+        f.pg = make_patch_grid(g, f.ppc);
+        f.n_tiles = f.pg.n_patches * f.pg.tiles_per_patch;
         f.seg_len = f.n_seg = 0;
     }
     return f;
@@ -251,14 +289,14 @@ static FramePlan frame_plan(const Geo& g) {
 
 size_t frame_workspace_bytes(const Geo& g) {
     size_t pairs = (size_t)g.B * (size_t)(g.T > 1 ? g.T - 1 : 0);
-    return pairs * (size_t)frame_plan(g).n_tiles * sizeof(float4) + pairs * sizeof(float) + 256;
+    return pairs * (size_t)frame_plan(g).n_tiles * sizeof(float4) + pairs * (size_t)(g.gy * g.gx) * sizeof(float) + 256;
 }
 
 template <int DT>
 static void march_dispatch(int lpr, dim3 grid, size_t smem, cudaStream_t s, const uint8_t* x, int T, int P, int cpr,
-                           float eps, int seg_len, int n_seg, float* pos_sim, float4* partial) {
-#define OC_MARCH(L) do { if (cpr <= 5 * L) OC_LAUNCH((frame_march_kernel<DT, L, 5>), grid, PAIR_THREADS, smem, s, x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial); \
-                         else OC_LAUNCH((frame_march_kernel<DT, L, 8>), grid, PAIR_THREADS, smem, s, x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial); } while (0)
+                           float eps, int seg_len, int n_seg, float* pos_sim, float4* partial, const PatchGrid& pg) {
+#define OC_MARCH(L) do { if (cpr <= 5 * L) OC_LAUNCH((frame_march_kernel<DT, L, 5>), grid, PAIR_THREADS, smem, s, x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial, pg); \
+                         else OC_LAUNCH((frame_march_kernel<DT, L, 8>), grid, PAIR_THREADS, smem, s, x, T, P, cpr, eps, seg_len, n_seg, pos_sim, partial, pg); } while (0)
     switch (lpr) {
         case 4: OC_MARCH(4); break; case 8: OC_MARCH(8); break; case 16: OC_MARCH(16); break; default: OC_MARCH(32); break;
     }
@@ -284,22 +322,23 @@ static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, co
             dim3 grid((unsigned)f.n_tiles, (unsigned)(g.B * f.n_seg));
             const size_t smem = (size_t)f.seg_len * (PAIR_THREADS / 32) * sizeof(float4);
             if (g.dtype == OC_DTYPE_BF16)
-                march_dispatch<OC_DTYPE_BF16>(f.lpr, grid, smem, s, (const uint8_t*)x, g.T, P, cpr, g.eps, f.seg_len, f.n_seg, pos_sim, partial);
+                march_dispatch<OC_DTYPE_BF16>(f.lpr, grid, smem, s, (const uint8_t*)x, g.T, P, cpr, g.eps, f.seg_len, f.n_seg, pos_sim, partial, f.pg);
             else
-                march_dispatch<OC_DTYPE_F32>(f.lpr, grid, smem, s, (const uint8_t*)x, g.T, P, cpr, g.eps, f.seg_len, f.n_seg, pos_sim, partial);
+                march_dispatch<OC_DTYPE_F32>(f.lpr, grid, smem, s, (const uint8_t*)x, g.T, P, cpr, g.eps, f.seg_len, f.n_seg, pos_sim, partial, f.pg);
         } else {
             dim3 grid((unsigned)f.n_tiles, (unsigned)n_pairs);
             if (g.dtype == OC_DTYPE_BF16)
-                frame_dispatch<OC_DTYPE_BF16>(f.lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, f.ppc);
+                frame_dispatch<OC_DTYPE_BF16>(f.lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, f.ppc, f.pg);
             else
-                frame_dispatch<OC_DTYPE_F32>(f.lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, f.ppc);
+                frame_dispatch<OC_DTYPE_F32>(f.lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, f.ppc, f.pg);
         }
     }
     {
         Scope scope(ctx, OC_K_FRAME_FIN, s);
         const int warps = PAIR_THREADS / 32;
-        OC_LAUNCH((frame_finalize_kernel), (unsigned)((g.B * g.T + warps - 1) / warps), PAIR_THREADS, 0, s, 
-            partial, f.n_tiles, g.B, g.T, P, g.frame_stat, g.eps, pair_ws, pair_sim, best_sim, best_idx);
+        OC_LAUNCH((frame_finalize_kernel), (unsigned)((g.n_units + warps - 1) / warps), PAIR_THREADS, 0, s,
+            partial, f.pg.tiles_per_patch, f.pg.n_patches, g.B, g.T, f.pg.Pp, g.frame_stat, g.eps, pair_ws, pair_sim,
+            best_sim, best_idx);
     }
     return last_launch_status();
 }

@@ -47,7 +47,8 @@ def gpu_match(oc, ctx, L, x_dev, want_aux=False, want_pair=False):
         else:
             aux = torch.full((L.B, L.T - 1, L.H * L.W), float("nan"), device="cuda", dtype=torch.float32)
     if want_pair:
-        pair = torch.full((L.B, max(L.T - 1, 0)), float("nan"), device="cuda", dtype=torch.float32)
+        shape = (L.B, max(L.T - 1, 0)) + ((L.gy * L.gx,) if L.kind == oc.KIND_FRAME and L.gy * L.gx > 1 else ())
+        pair = torch.full(shape, float("nan"), device="cuda", dtype=torch.float32)
     ctx.match(L, x_dev, best_sim, best_idx, aux, pair)
     torch.cuda.synchronize()
     assert ctx.device_status() == oc.OK

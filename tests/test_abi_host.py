@@ -62,6 +62,10 @@ def test_layout_check_rules(oc):
     assert L(oc.KIND_TOKEN, oc.DTYPE_BF16, 1, 1, 8, 8, 8, eps=-1.0).check() == oc.ERR_INVALID_ARG
     assert L(oc.KIND_FRAME, oc.DTYPE_BF16, 1, 25, 72, 128, 320).check() == oc.OK
     assert L(oc.KIND_FRAME, oc.DTYPE_BF16, 1, 25, 72, 128, 320, frame_stat=2).check() == oc.ERR_INVALID_ARG
+    assert L(oc.KIND_FRAME, oc.DTYPE_BF16, 1, 25, 72, 128, 320, gy=4, gx=4).check() == oc.OK     # patch-local
+    assert L(oc.KIND_FRAME, oc.DTYPE_BF16, 1, 25, 72, 128, 320, gy=5).check() == oc.ERR_INVALID_ARG
+    assert L(oc.KIND_FRAME, oc.DTYPE_BF16, 1, 25, 72, 128, 320, gx=-1).check() == oc.ERR_INVALID_ARG
+    assert L(oc.KIND_FRAME, oc.DTYPE_BF16, 1, 25, 72, 128, 320, gy=0, gx=0).counts()[0] == 1
     assert L(oc.KIND_BLOCK, oc.DTYPE_BF16, 1, 16, 16, 16, 1152).check() == oc.OK
     assert L(oc.KIND_BLOCK, oc.DTYPE_BF16, 1, 16, 16, 16, 1152, gy=2).check() == oc.ERR_UNSUPPORTED
     assert L(oc.KIND_TOKEN, oc.DTYPE_BF16, 64, 64, 1024, 1024, 8).check() == oc.ERR_UNSUPPORTED   # > 2^31-1 units
@@ -73,6 +77,8 @@ def test_layout_check_rules(oc):
     (0, (1, 25, 18, 32, 1280), {}), (0, (1, 1, 16, 16, 64), dict(self_match=1)),
     (0, (1, 2, 12, 18, 8), dict(sy=3, sx=3, oy=1, ox=2, gy=2, gx=2)),
     (1, (3, 25, 72, 128, 320), {}), (2, (2, 16, 16, 16, 1152), {}),
+    (1, (2, 25, 72, 128, 320), dict(gy=4, gx=4)), (1, (2, 5, 12, 16, 8), dict(gy=3, gx=1)),
+    (1, (1, 4, 12, 16, 8), dict(gy=1, gx=8)),
 ])
 def test_counts_and_rows_agree_with_oracle(oc, oracle, kind, shape, kw):
     L = oc.Layout(kind, oc.DTYPE_BF16, *shape, **kw)
@@ -85,7 +91,7 @@ def test_counts_and_rows_agree_with_oracle(oc, oracle, kind, shape, kw):
         # both describe the same byte offsets for every unit and segment
         assert (a.seg_bytes, a.n_seg) == (b.seg_bytes, b.n_seg)
         n_units = g * u
-        for i in (0, 1, n_units // 2, n_units - 1):
+        for i in (0, 1, n_units // 2, n_units // 3 + 1, n_units - 1):
             for s in (0, a.n_seg - 1):
                 off_a = (i // a.units_per_outer) * a.outer_pitch + (i % a.units_per_outer) * a.unit_pitch + s * a.seg_stride
                 off_b = (i // b.units_per_outer) * b.outer_pitch + (i % b.units_per_outer) * b.unit_pitch + s * b.seg_stride

@@ -251,6 +251,45 @@ def test_frame_chain_small(oc, oracle, dtype, T, stat):
     assert rep["reused"] == T // 2          # rho = 0.95 > 0.9: every odd frame is reused
 
 
+def _frame_patch_workload(seed, B, T, Hh, W, C, dtype, grid, mode, rho=0.95):
+    """AR(1) frames as in the SVD recipe, B batch elements, cut into grid patches per frame."""
+    rng = np.random.default_rng(seed)
+    x = np.stack([inputs.ar1_frames(rng, inputs.smooth_field(rng, Hh, W, C, 4.0), T, rho) for _ in range(B)])
+    x = np.ascontiguousarray(x.reshape(B, T, Hh, W, C), dtype=np.float32)
+    w = inputs.Workload(f"frame_patches_{grid[0]}x{grid[1]}", "frame", dtype, (B, T, Hh, W, C),
+                        x if dtype == inputs.F32 else inputs.to_bf16_bits(x), mode=mode, thr=rho, n_reuse=max(1, (T // 2) // 2))
+    w.groups = grid
+    return w
+
+
+@pytest.mark.parametrize("dtype", [inputs.BF16, inputs.F32])
+@pytest.mark.parametrize("B,T,grid,stat,mode", [
+    (2, 7, (3, 1), 0, "threshold"), (1, 6, (2, 4), 1, "count"), (2, 5, (1, 2), 0, "count"),
+    (1, 2, (4, 4), 0, "threshold"), (2, 1, (2, 2), 0, "threshold"), (1, 9, (12, 16), 1, "threshold"),
+])
+def test_frame_patch_chain_small(oc, oracle, dtype, B, T, grid, stat, mode):
+    """Patch-local Frame Cache (Section 3.3): every stage against the oracle, patches of frames as units."""
+    w = _frame_patch_workload(41 + T, B, T, 12, 16, 40, dtype, grid, mode)
+    rep = run_chain(oc, oracle, w, Cout=24, want_aux=True, frame_stat=stat)
+    if T > 1 and grid != (12, 16):
+        assert 0 < rep["reused"] <= B * (T // 2) * grid[0] * grid[1]
+
+
+def test_frame_patch_chain_long_rows(oc, oracle):
+    """Rows too long for the time-marching kernel: the pair kernel's tiles follow the patches too."""
+    w = _frame_patch_workload(5, 1, 4, 4, 6, 2176, inputs.BF16, (2, 3), "threshold")
+    run_chain(oc, oracle, w, Cout=16, want_aux=True)
+
+
+def test_frame_patches_svd_level0(oc, oracle):
+    """Config-3 tensor cut 4 x 4 (18 x 32-token patches): sims, indices and the whole chain."""
+    w = inputs.svd_frames()
+    w.groups = (4, 4)
+    w.thr = 0.95
+    rep = run_chain(oc, oracle, w)
+    assert 0 < rep["reused"] < 12 * 16
+
+
 @pytest.mark.parametrize("dtype,lattice", [(inputs.BF16, (2, 2, 0, 0)), (inputs.F32, (2, 2, 1, 0)),
                                           (inputs.BF16, (1, 2, 0, 1)), (inputs.BF16, (3, 2, 2, 1))])
 def test_block_chain_small(oc, oracle, dtype, lattice):

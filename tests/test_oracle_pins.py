@@ -403,7 +403,7 @@ def np_select(L, best_sim, best_idx, mode, thr, n_reuse, stride):
 @pytest.mark.parametrize("kind,shape,groups", [
     (0, (2, 1, 8, 8, 8), (1, 1)), (0, (1, 2, 8, 16, 8), (2, 2)),
     (1, (3, 7, 2, 2, 8), (1, 1)), (2, (2, 3, 6, 8, 8), (1, 1)),
-    (1, (2, 7, 4, 6, 8), (2, 3)),
+    (1, (2, 7, 4, 6, 8), (2, 3)), (2, (2, 3, 8, 12, 8), (2, 3)),
 ])
 @pytest.mark.parametrize("mode", [0, 1])
 def test_select_bruteforce(oracle, kind, shape, groups, mode):
@@ -427,6 +427,38 @@ def test_select_bruteforce(oracle, kind, shape, groups, mode):
         assert np.array_equal(got["slot_of"], so)
         if mode == 1:
             assert np.all(cnt == U - min(n_reuse, n_cand))
+
+
+def test_block_patches_confine_the_selection_only(oracle):
+    """Patch-local Block Cache: matching is unchanged (own 2x2 neighbourhood), the count-mode
+    selection is taken per patch; unit indices stay the frame positions."""
+    rng = np.random.default_rng(55)
+    shape, gy, gx = (2, 3, 8, 12, 8), 2, 3
+    x = rng.standard_normal(shape).astype(np.float32)
+    L1 = oracle.Layout(2, 0, *shape)
+    Lp = oracle.Layout(2, 0, *shape, gy=gy, gx=gx)
+    m1, mp = oracle.match_block(L1, x), oracle.match_block(Lp, x)
+    assert np.array_equal(m1["best_sim"], mp["best_sim"]) and np.array_equal(m1["best_idx"], mp["best_idx"])
+    B, T, Hh, W, Cc = shape
+    hp, wp = Hh // gy, W // gx
+    assert Lp.n_groups == B * gy * gx and Lp.units_per_group == hp * wp and Lp.n_rep == hp * wp // 4
+    pos = np.arange(B * Hh * W).reshape(B, gy, hp, gx, wp).transpose(0, 1, 3, 2, 4).reshape(B * gy * gx, hp * wp)
+    for g in range(Lp.n_groups):
+        for u in (0, 1, wp, hp * wp - 1):
+            assert Lp.unit_index(g, u) == pos[g, u]
+    n_reuse = 5
+    s = oracle.select(Lp, mp["best_sim"], mp["best_idx"], 1, 0.0, n_reuse, hp * wp - n_reuse)
+    reused = s["slot_of"] < 0
+    for g in range(Lp.n_groups):
+        ids = pos[g]
+        assert reused[ids].sum() == n_reuse
+        cand = ids[np.isfinite(mp["best_sim"][ids])]
+        order = cand[np.lexsort((cand, -mp["best_sim"][cand].astype(np.float64)))]
+        assert set(order[:n_reuse]) == set(ids[reused[ids]])
+        assert np.array_equal(s["kept_idx"][g * (hp * wp - n_reuse):(g + 1) * (hp * wp - n_reuse)], ids[~reused[ids]][np.argsort(ids[~reused[ids]])])
+    # rows are still whole blocks addressed by frame position
+    R1, Rp = oracle.rows_for(L1, Cc, 4), oracle.rows_for(Lp, Cc, 4)
+    assert R1 == Rp
 
 
 def test_select_self_match_chain(oracle):
