@@ -66,7 +66,8 @@ enum { OC_FRAME_MEAN_POS_COS = 0, OC_FRAME_FLAT_COS = 1 };
  *          and the statistic runs over the patch's positions only.  gy = gx = 0 means 1.
  *   BLOCK: positions are cut into sy x sx neighbourhoods; the (oy, ox) member is the
  *          representative, the others are compared with it over the T*C block descriptor
- *          (Section 3.2.1).  gy = gx = 1.
+ *          (Section 3.2.1).  gy x gx > 1 cuts the positions into patches of whole neighbourhoods
+ *          (Section 3.3): matching is unchanged, the selection is taken per patch (b, py, px).
  * H must be a multiple of gy and W of gx; H/gy must be a multiple of sy and W/gx of sx (TOKEN, BLOCK). */
 typedef struct oc_layout {
     int kind;        /* OC_KIND_*  */
@@ -215,6 +216,23 @@ oc_status oc_profile_captured_read(oc_ctx* ctx, int kernel_id, int64_t* launches
  * (OC_ERR_WORKSPACE otherwise).  Calls on one context must not overlap on the device. */
 oc_status oc_match(oc_ctx* ctx, const oc_layout* layout, const void* x, float* best_sim,
                    int32_t* best_idx, float* aux_sim, float* pair_sim, void* stream);
+
+/* Frame Cache at several patch sizes from ONE pass over the tensor (Section 3.3: after patch-level
+ * caching "the patch size can be increased for coarser reuse, or patches can be restored to full
+ * frames").  `layout` is an OC_KIND_FRAME layout whose (gy, gx) is the finest grid; `grids` (HOST
+ * memory, [n_levels][2] ints) lists (gy_l, gx_l) per level, each dividing (gy, gx) -- (1, 1) is the
+ * whole frame.  Level l's results are what oc_match() gives for the same layout with (gy_l, gx_l)
+ * (equal up to fp32 summation order), stored one level after another:
+ *   best_sim, best_idx  [sum_l B*T*gy_l*gx_l], unit indices local to their level
+ *   pair_sim  nullable, [sum_l B*(T-1)*gy_l*gx_l]
+ *   pos_sim   nullable, [B][T-1][H*W] per-position cosines (shared by all levels)
+ * The streaming kernel runs once; only the small per-unit reduction runs per level.
+ * 1 <= n_levels <= OC_MAX_FRAME_LEVELS.  Workspace: oc_match_workspace_bytes(layout).
+ * Errors: as oc_match(); OC_ERR_INVALID_ARG for a grid that does not divide the layout's. */
+#define OC_MAX_FRAME_LEVELS 8
+oc_status oc_match_frame_levels(oc_ctx* ctx, const oc_layout* layout, const void* x, int n_levels,
+                                const int32_t* grids, float* best_sim, int32_t* best_idx, float* pos_sim,
+                                float* pair_sim, void* stream);
 
 /* select ("the r most redundant ... are marked for cached restoration while the retained
  * representatives are computed normally", Sections 3.2.1-3.2.3).  Representatives are always kept.

@@ -70,7 +70,6 @@ oc_status make_geo(const oc_layout* L, Geo* g) {
         return OC_OK;
     }
     if (L->gy <= 0 || L->gx <= 0) return OC_ERR_INVALID_ARG;
-    if (L->kind == OC_KIND_BLOCK && (L->gy != 1 || L->gx != 1)) return OC_ERR_UNSUPPORTED;
     if (L->kind == OC_KIND_BLOCK && L->self_match) return OC_ERR_INVALID_ARG;
     if (L->H % L->gy != 0 || L->W % L->gx != 0) return OC_ERR_INVALID_ARG;
     g->Hp = L->H / L->gy; g->Wp = L->W / L->gx;
@@ -89,10 +88,12 @@ oc_status make_geo(const oc_layout* L, Geo* g) {
         g->units_per_group = (int64_t)g->Hp * g->Wp;
         g->reps_per_group = (int64_t)g->Hs * g->Ws;
     } else {
-        g->n_groups = L->B;
-        g->units_per_group = (int64_t)L->H * L->W;
+        // a patch confines the selection; matching stays inside the sy x sx neighbourhood, which a
+        // patch never cuts (Hp % sy == 0, Wp % sx == 0 above)
+        g->n_groups = (int64_t)L->B * L->gy * L->gx;
+        g->units_per_group = (int64_t)g->Hp * g->Wp;
         g->reps_per_group = (int64_t)g->Hs * g->Ws;
-        if (g->units_per_group * L->B > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
+        if ((int64_t)L->H * L->W * L->B > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
     }
     g->n_units = g->n_groups * g->units_per_group;
     return OC_OK;
@@ -356,6 +357,29 @@ oc_status oc_match(oc_ctx* c, const oc_layout* layout, const void* x, float* bes
     if (g.kind == OC_KIND_TOKEN) return launch_match_token(c, g, x, best_sim, best_idx, aux_sim, s);
     if (g.kind == OC_KIND_FRAME) return launch_match_frame(c, g, x, best_sim, best_idx, aux_sim, pair_sim, s);
     return launch_match_block(c, g, x, best_sim, best_idx, s);
+}
+
+oc_status oc_match_frame_levels(oc_ctx* c, const oc_layout* layout, const void* x, int n_levels,
+                                const int32_t* grids, float* best_sim, int32_t* best_idx, float* pos_sim,
+                                float* pair_sim, void* stream) {
+    if (!c || !x || !best_sim || !best_idx || !grids || n_levels < 1 || n_levels > OC_MAX_FRAME_LEVELS)
+        return OC_ERR_INVALID_ARG;
+    Geo g;
+    oc_status st = make_geo(layout, &g);
+    if (st != OC_OK) return st;
+    if (g.kind != OC_KIND_FRAME) return OC_ERR_INVALID_ARG;
+    long long units = 0;
+    for (int l = 0; l < n_levels; ++l) {
+        const int gy = grids[2 * l], gx = grids[2 * l + 1];
+        if (gy <= 0 || gx <= 0 || g.gy % gy != 0 || g.gx % gx != 0) return OC_ERR_INVALID_ARG;
+        units += (long long)g.B * g.T * gy * gx;
+    }
+    if (units > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
+    if (misaligned(x)) return OC_ERR_ALIGNMENT;
+    if (match_workspace_bytes(g) > c->workspace_bytes) return OC_ERR_WORKSPACE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return OC_ERR_CUDA;
+    return launch_match_frame_levels(c, g, x, n_levels, grids, best_sim, best_idx, pos_sim, pair_sim, (cudaStream_t)stream);
 }
 
 oc_status oc_select(oc_ctx* c, const oc_layout* layout, const float* best_sim, const int32_t* best_idx, int mode,

@@ -123,24 +123,21 @@ struct GroupMap {
 GroupMap make_group_map(const Geo& g);
 
 __host__ __device__ inline int64_t gm_unit_index(const GroupMap& m, int64_t g, int u) {
-    if (m.kind == OC_KIND_TOKEN) {
+    if (m.kind != OC_KIND_FRAME) {                     // TOKEN: bt = frame; BLOCK: bt = batch element
         int px = (int)(g % m.gx);
         int py = (int)((g / m.gx) % m.gy);
         int64_t bt = g / ((int64_t)m.gx * m.gy);
         int ly = u / m.Wp, lx = u - ly * m.Wp;
         return (bt * m.H + (int64_t)py * m.Hp + ly) * m.W + (int64_t)px * m.Wp + lx;
     }
-    if (m.kind == OC_KIND_FRAME) {                     // group (b, patch): its frames are n_patches apart
-        const int64_t np = (int64_t)m.gy * m.gx, b = g / np, patch = g - b * np;
-        return (b * m.units_per_group + u) * np + patch;
-    }
-    return g * m.units_per_group + u;
+    // FRAME group (b, patch): its frames are n_patches apart
+    const int64_t np = (int64_t)m.gy * m.gx, b = g / np, patch = g - b * np;
+    return (b * m.units_per_group + u) * np + patch;
 }
 __host__ __device__ inline bool gm_is_rep(const GroupMap& m, int u) {
     if (m.kind == OC_KIND_FRAME) return (u & 1) == 0;
     if (m.self_match) return true;
-    int Wl = (m.kind == OC_KIND_TOKEN) ? m.Wp : m.W;
-    int ly = u / Wl, lx = u - ly * Wl;
+    int ly = u / m.Wp, lx = u - ly * m.Wp;
     return (ly % m.sy) == m.oy && (lx % m.sx) == m.ox;
 }
 __host__ __device__ inline bool gm_is_cand(const GroupMap& m, int u) {
@@ -160,6 +157,8 @@ oc_status launch_select(oc_ctx*, const Geo&, const float* best_sim, const int32_
                         int32_t* kept_count, int32_t* match_map, int32_t* slot_of, cudaStream_t);
 oc_status launch_match_frame(oc_ctx*, const Geo&, const void* x, float* best_sim, int32_t* best_idx,
                              float* pos_sim, float* pair_sim, cudaStream_t);
+oc_status launch_match_frame_levels(oc_ctx*, const Geo&, const void* x, int n_levels, const int32_t* levels,
+                                    float* best_sim, int32_t* best_idx, float* pos_sim, float* pair_sim, cudaStream_t);
 oc_status launch_match_block(oc_ctx*, const Geo&, const void* x, float* best_sim, int32_t* best_idx,
                              cudaStream_t);
 oc_status launch_match_token(oc_ctx*, const Geo&, const void* x, float* best_sim, int32_t* best_idx,

@@ -200,13 +200,39 @@ frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float e
 // of the pair (t, t-1) and of the pair (t+1, t) that belong to its patch, publishes the first as
 // pair_sim[t-1][patch] and, for an odd (candidate) frame, picks the better of its two adjacent
 // representatives.  Every warp is independent, so units run in parallel.
-__device__ __forceinline__ float frame_pair_value(const float4* __restrict__ rec, int n_rec, int n_pos,
-                                                  int stat, float eps) {
+//
+// The partial records are laid out for the FINEST patch grid; a coarser level of the hierarchy
+// (Section 3.3: "the patch size can be increased for coarser reuse, or patches can be restored to
+// full frames") whose patches are unions of ry x rx fine patches is finalized from the same records,
+// so one pass over the tensor serves every level.
+struct FinLevel {
+    int gy, gx;             // this level's patch grid
+    int ry, rx;             // fine patches per patch of this level, per axis
+    int gx_fine, np_fine;   // finest grid: patches per row, patches per frame
+    int tiles_per_patch;    // records per (pair, fine patch)
+    int n_pos;              // positions per patch of this level
+};
+
+__device__ __forceinline__ float frame_pair_value(const float4* __restrict__ partial, long long q, int patch,
+                                                  const FinLevel& lv, int stat, float eps) {
     const int lane = threadIdx.x & 31;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    for (int i = lane; i < n_rec; i += 32) {
-        const float4 v = rec[i];
-        a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+    if (lv.ry * lv.rx == 1) {
+        const float4* rec = partial + (q * lv.np_fine + patch) * lv.tiles_per_patch;
+        for (int i = lane; i < lv.tiles_per_patch; i += 32) {
+            const float4 v = rec[i];
+            a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+        }
+    } else {
+        const int py = patch / lv.gx, px = patch - py * lv.gx;
+        const int per_row = lv.rx * lv.tiles_per_patch, n_rec = lv.ry * per_row;
+        for (int j = lane; j < n_rec; j += 32) {
+            const int fy = j / per_row, r = j - fy * per_row;
+            const int fx = r / lv.tiles_per_patch, k = r - fx * lv.tiles_per_patch;
+            const int fine = (py * lv.ry + fy) * lv.gx_fine + px * lv.rx + fx;
+            const float4 v = partial[(q * lv.np_fine + fine) * lv.tiles_per_patch + k];
+            a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+        }
     }
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {
@@ -214,27 +240,26 @@ __device__ __forceinline__ float frame_pair_value(const float4* __restrict__ rec
         a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, d); a3 += __shfl_xor_sync(0xFFFFFFFFu, a3, d);
     }
     return stat == OC_FRAME_FLAT_COS ? clamp_unit(a1 / (fmaxf(sqrtf(a2), eps) * fmaxf(sqrtf(a3), eps)))
-                                     : a0 / (float)n_pos;
+                                     : a0 / (float)lv.n_pos;
 }
 
 __global__ void __launch_bounds__(PAIR_THREADS)
-frame_finalize_kernel(const float4* __restrict__ partial, int tiles_per_patch, int n_patches, int B, int T,
-                      int Pp, int stat, float eps, float* __restrict__ pair_ws, float* __restrict__ pair_sim,
-                      float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
+frame_finalize_kernel(const float4* __restrict__ partial, FinLevel lv, int B, int T, int stat, float eps,
+                      float* __restrict__ pair_sim, float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
     pdl_enter();
+    const int n_patches = lv.gy * lv.gx;
     const int i = blockIdx.x * (PAIR_THREADS / 32) + (threadIdx.x >> 5);     // unit index (b*T + t)*n_patches + patch
     const int lane = threadIdx.x & 31;
     if (i >= B * T * n_patches) return;                                       // whole warps leave together
     const int bt = i / n_patches, patch = i - bt * n_patches;
     const int b = bt / T, t = bt - b * T;
-    const long long q_prev = (long long)(b * (T - 1) + t - 1) * n_patches + patch;   // record run of (t, t-1)
+    const long long q_prev = (long long)b * (T - 1) + t - 1;                  // pair (t, t-1)
     float with_prev = -INFINITY, with_next = -INFINITY;
     if (t >= 1) {
-        with_prev = frame_pair_value(partial + q_prev * tiles_per_patch, tiles_per_patch, Pp, stat, eps);
-        if (lane == 0) { pair_ws[q_prev] = with_prev; if (pair_sim) pair_sim[q_prev] = with_prev; }
+        with_prev = frame_pair_value(partial, q_prev, patch, lv, stat, eps);
+        if (lane == 0 && pair_sim) pair_sim[q_prev * n_patches + patch] = with_prev;
     }
-    if ((t & 1) && t + 1 < T)
-        with_next = frame_pair_value(partial + (q_prev + n_patches) * tiles_per_patch, tiles_per_patch, Pp, stat, eps);
+    if ((t & 1) && t + 1 < T) with_next = frame_pair_value(partial, q_prev + 1, patch, lv, stat, eps);
     if (lane == 0) {
         if ((t & 1) == 0) { best_sim[i] = -INFINITY; best_idx[i] = i; }
         else if (with_next > with_prev) { best_sim[i] = with_next; best_idx[i] = i + n_patches; }
@@ -289,7 +314,7 @@ static FramePlan frame_plan(const Geo& g) {
 
 size_t frame_workspace_bytes(const Geo& g) {
     size_t pairs = (size_t)g.B * (size_t)(g.T > 1 ? g.T - 1 : 0);
-    return pairs * (size_t)frame_plan(g).n_tiles * sizeof(float4) + pairs * (size_t)(g.gy * g.gx) * sizeof(float) + 256;
+    return pairs * (size_t)frame_plan(g).n_tiles * sizeof(float4) + 256;
 }
 
 template <int DT>
@@ -303,15 +328,17 @@ static void march_dispatch(int lpr, dim3 grid, size_t smem, cudaStream_t s, cons
 #undef OC_MARCH
 }
 
-// Both frame entry points run this: `scratch` holds the partial records and the pair values.
-// ctx may be null (no launch counters then).
+// Every frame entry point runs this: `scratch` holds the partial records.  ctx may be null (no launch
+// counters then).  levels == nullptr: one level, the layout's own grid; otherwise n_levels grids
+// (gy_l, gx_l), each dividing the layout's, whose outputs follow one another in best_sim / best_idx
+// (B*T*gy_l*gx_l entries each) and pair_sim (B*(T-1)*gy_l*gx_l each).
 static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, const void* x, float* best_sim,
-                                 int32_t* best_idx, float* pos_sim, float* pair_sim, cudaStream_t s) {
+                                 int32_t* best_idx, float* pos_sim, float* pair_sim, cudaStream_t s,
+                                 int n_levels = 1, const int32_t* levels = nullptr) {
     const int P = g.H * g.W, cpr = g.C * g.elem_bytes / 16;
     const int n_pairs = g.B * (g.T - 1);
     const FramePlan f = frame_plan(g);
     float4* partial = (float4*)scratch;
-    float* pair_ws = (float*)(scratch + (size_t)(n_pairs > 0 ? n_pairs : 0) * f.n_tiles * sizeof(float4));
     if (n_pairs > 65535 || (long long)g.B * (f.march ? f.n_seg : 1) > 65535) return OC_ERR_UNSUPPORTED;
     struct Scope { oc_ctx* c; int k; cudaStream_t s; LaunchScope* l; 
                    Scope(oc_ctx* c_, int k_, cudaStream_t s_) : c(c_), k(k_), s(s_), l(c_ ? new LaunchScope(c_, k_, s_) : nullptr) {}
@@ -333,12 +360,20 @@ static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, co
                 frame_dispatch<OC_DTYPE_F32>(f.lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, f.ppc, f.pg);
         }
     }
-    {
+    for (int l = 0; l < n_levels; ++l) {
+        FinLevel lv;
+        lv.gy = levels ? levels[2 * l] : g.gy; lv.gx = levels ? levels[2 * l + 1] : g.gx;
+        lv.ry = g.gy / lv.gy; lv.rx = g.gx / lv.gx;
+        lv.gx_fine = g.gx; lv.np_fine = g.gy * g.gx;
+        lv.tiles_per_patch = f.pg.tiles_per_patch;
+        lv.n_pos = f.pg.Pp * lv.ry * lv.rx;
+        const long long units = (long long)g.B * g.T * lv.gy * lv.gx;
         Scope scope(ctx, OC_K_FRAME_FIN, s);
         const int warps = PAIR_THREADS / 32;
-        OC_LAUNCH((frame_finalize_kernel), (unsigned)((g.n_units + warps - 1) / warps), PAIR_THREADS, 0, s,
-            partial, f.pg.tiles_per_patch, f.pg.n_patches, g.B, g.T, f.pg.Pp, g.frame_stat, g.eps, pair_ws, pair_sim,
-            best_sim, best_idx);
+        OC_LAUNCH((frame_finalize_kernel), (unsigned)((units + warps - 1) / warps), PAIR_THREADS, 0, s,
+            partial, lv, g.B, g.T, g.frame_stat, g.eps, pair_sim, best_sim, best_idx);
+        best_sim += units; best_idx += units;
+        if (pair_sim) pair_sim += (long long)n_pairs * lv.gy * lv.gx;
     }
     return last_launch_status();
 }
@@ -346,6 +381,11 @@ static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, co
 oc_status launch_match_frame(oc_ctx* ctx, const Geo& g, const void* x, float* best_sim, int32_t* best_idx,
                              float* pos_sim, float* pair_sim, cudaStream_t s) {
     return run_frame_match(ctx, (uint8_t*)ctx->workspace, g, x, best_sim, best_idx, pos_sim, pair_sim, s);
+}
+
+oc_status launch_match_frame_levels(oc_ctx* ctx, const Geo& g, const void* x, int n_levels, const int32_t* levels,
+                                    float* best_sim, int32_t* best_idx, float* pos_sim, float* pair_sim, cudaStream_t s) {
+    return run_frame_match(ctx, (uint8_t*)ctx->workspace, g, x, best_sim, best_idx, pos_sim, pair_sim, s, n_levels, levels);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -27,31 +27,28 @@ static constexpr int SEL_SMEM_KEYS = 40960;          // keys cached in shared me
 // shifts and masks when the row width / lattice strides are powers of two, divisions otherwise.
 struct GroupView {
     long long base;     // global index of local unit 0 (TOKEN: of the patch's first token)
-    int unit_stride;    // FRAME: distance between consecutive frames of a patch position; BLOCK: 1
-    int row_pitch;      // TOKEN: frame width W; others unused
-    int w_local;        // row width of the local unit grid (TOKEN: Wp, BLOCK: W, FRAME: 0)
+    int unit_stride;    // FRAME: distance between consecutive frames of a patch position
+    int row_pitch;      // TOKEN, BLOCK: frame width W
+    int w_local;        // row width of the local unit grid (TOKEN, BLOCK: Wp; FRAME: 0)
     int w_shift;        // log2(w_local) if it is a power of two, else -1
     int lat_pow2;       // sy and sx are both powers of two
+    int contig;         // local units are equally spaced in unit order (FRAME; patches as wide as the frame)
     __device__ GroupView(const GroupMap& m, long long g) {
-        if (m.kind == OC_KIND_TOKEN) {
+        if (m.kind != OC_KIND_FRAME) {                  // TOKEN: bt = frame; BLOCK: bt = batch element
             const int px = (int)(g % m.gx), py = (int)((g / m.gx) % m.gy);
             const long long bt = g / ((long long)m.gx * m.gy);
             base = (bt * m.H + (long long)py * m.Hp) * m.W + (long long)px * m.Wp;
             row_pitch = m.W;
             w_local = m.Wp;
             unit_stride = 1;
-        } else if (m.kind == OC_KIND_FRAME) {
+        } else {
             const long long np = (long long)m.gy * m.gx, b = g / np;
             base = b * m.units_per_group * np + (g - b * np);
             unit_stride = (int)np;
             row_pitch = 0;
             w_local = 0;
-        } else {
-            base = g * m.units_per_group;
-            unit_stride = 1;
-            row_pitch = 0;
-            w_local = m.kind == OC_KIND_BLOCK ? m.W : 0;
         }
+        contig = m.kind == OC_KIND_FRAME || m.Wp == m.W;
         w_shift = (w_local > 0 && (w_local & (w_local - 1)) == 0) ? 31 - __clz(w_local) : -1;
         lat_pow2 = (m.sy & (m.sy - 1)) == 0 && (m.sx & (m.sx - 1)) == 0;
     }
@@ -60,7 +57,7 @@ struct GroupView {
         else { ly = u / w_local; lx = u - ly * w_local; }
     }
     __device__ __forceinline__ long long index(const GroupMap& m, int u) const {
-        if (m.kind != OC_KIND_TOKEN) return base + (long long)u * unit_stride;
+        if (contig) return base + (long long)u * unit_stride;
         int ly, lx; split(u, ly, lx);
         return base + (long long)ly * row_pitch + lx;
     }

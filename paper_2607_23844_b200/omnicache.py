@@ -30,7 +30,7 @@ EXPORTS = (
     "oc_status_str", "oc_layout_check", "oc_layout_counts", "oc_match_workspace_bytes",
     "oc_rows_from_layout", "oc_layer_cache_would_hit", "oc_kernel_name", "oc_create", "oc_destroy",
     "oc_device_status", "oc_profile_enable", "oc_profile_reset", "oc_profile_read", "oc_profile_span_read",
-    "oc_profile_captured_read", "oc_match",
+    "oc_profile_captured_read", "oc_match", "oc_match_frame_levels",
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
     "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
     "oc_schedule_propose",
@@ -77,6 +77,7 @@ _lib.oc_profile_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_profile_span_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_profile_captured_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_match.argtypes = [_vp] * 8
+_lib.oc_match_frame_levels.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.oc_select.argtypes = [_vp, _vp, _vp, _vp, _i, _f, _i64, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.oc_gather.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp]
 _lib.oc_restore.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _i, _vp]
@@ -308,6 +309,18 @@ class Context:
                            _ptr(pair_sim), _stream(stream))
         if check:
             _chk(st, "oc_match")
+        return st
+
+    def match_frame_levels(self, layout: Layout, x, grids, best_sim, best_idx, pos_sim=None, pair_sim=None,
+                           stream=None, check: bool = True) -> int:
+        """oc_match_frame_levels: ``grids`` is a sequence of (gy, gx) pairs (host side)."""
+        cl = layout.c()
+        flat = [int(v) for g in grids for v in g]
+        arr = (C.c_int32 * max(len(flat), 1))(*flat)
+        st = _lib.oc_match_frame_levels(self._h, C.byref(cl), _ptr(x), len(grids), arr, _ptr(best_sim),
+                                        _ptr(best_idx), _ptr(pos_sim), _ptr(pair_sim), _stream(stream))
+        if check:
+            _chk(st, "oc_match_frame_levels")
         return st
 
     def select(self, layout: Layout, best_sim, best_idx, mode: int, thr: float, n_reuse_per_group: int,

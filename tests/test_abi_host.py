@@ -67,7 +67,8 @@ def test_layout_check_rules(oc):
     assert L(oc.KIND_FRAME, oc.DTYPE_BF16, 1, 25, 72, 128, 320, gx=-1).check() == oc.ERR_INVALID_ARG
     assert L(oc.KIND_FRAME, oc.DTYPE_BF16, 1, 25, 72, 128, 320, gy=0, gx=0).counts()[0] == 1
     assert L(oc.KIND_BLOCK, oc.DTYPE_BF16, 1, 16, 16, 16, 1152).check() == oc.OK
-    assert L(oc.KIND_BLOCK, oc.DTYPE_BF16, 1, 16, 16, 16, 1152, gy=2).check() == oc.ERR_UNSUPPORTED
+    assert L(oc.KIND_BLOCK, oc.DTYPE_BF16, 1, 16, 16, 16, 1152, gy=2).check() == oc.OK          # patch-local selection
+    assert L(oc.KIND_BLOCK, oc.DTYPE_BF16, 1, 16, 16, 16, 1152, gy=16).check() == oc.ERR_INVALID_ARG  # cuts a 2x2 group
     assert L(oc.KIND_TOKEN, oc.DTYPE_BF16, 64, 64, 1024, 1024, 8).check() == oc.ERR_UNSUPPORTED   # > 2^31-1 units
     assert oc._lib.oc_layout_check(None) == oc.ERR_INVALID_ARG
 
@@ -78,7 +79,7 @@ def test_layout_check_rules(oc):
     (0, (1, 2, 12, 18, 8), dict(sy=3, sx=3, oy=1, ox=2, gy=2, gx=2)),
     (1, (3, 25, 72, 128, 320), {}), (2, (2, 16, 16, 16, 1152), {}),
     (1, (2, 25, 72, 128, 320), dict(gy=4, gx=4)), (1, (2, 5, 12, 16, 8), dict(gy=3, gx=1)),
-    (1, (1, 4, 12, 16, 8), dict(gy=1, gx=8)),
+    (1, (1, 4, 12, 16, 8), dict(gy=1, gx=8)), (2, (2, 16, 16, 24, 1152), dict(gy=2, gx=3)),
 ])
 def test_counts_and_rows_agree_with_oracle(oc, oracle, kind, shape, kw):
     L = oc.Layout(kind, oc.DTYPE_BF16, *shape, **kw)
@@ -121,6 +122,7 @@ def test_null_context_and_bad_arguments_are_rejected_before_any_launch(oc):
     rows = oc.CRows(16, 1, 0, 16, 1 << 40, 0)
     one = C.c_void_p(16)   # a non-null, 16-byte aligned dummy; never dereferenced on these paths
     assert lib.oc_match(None, C.byref(L), one, one, one, None, None, None) == oc.ERR_INVALID_ARG
+    assert lib.oc_match_frame_levels(None, C.byref(L), one, 1, one, one, one, None, None, None) == oc.ERR_INVALID_ARG
     assert lib.oc_select(None, C.byref(L), one, one, 0, 0.5, 0, 64, one, one, one, one, None) == oc.ERR_INVALID_ARG
     assert lib.oc_gather(None, C.byref(rows), one, one, 4, one, None) == oc.ERR_INVALID_ARG
     assert lib.oc_restore(None, C.byref(rows), one, one, 4, one, one, one, 0, None) == oc.ERR_INVALID_ARG

@@ -275,6 +275,39 @@ def test_frame_patch_chain_small(oc, oracle, dtype, B, T, grid, stat, mode):
         assert 0 < rep["reused"] <= B * (T // 2) * grid[0] * grid[1]
 
 
+@pytest.mark.parametrize("dtype,stat", [(inputs.BF16, 0), (inputs.F32, 1)])
+def test_frame_hierarchy_levels_from_one_pass(oc, oracle, dtype, stat):
+    """Every level of the patch hierarchy (Section 3.3) equals the oracle's match at that patch size."""
+    B, T, Hh, W, C = 2, 7, 12, 16, 40
+    w = _frame_patch_workload(3, B, T, Hh, W, C, dtype, (6, 8), "threshold")
+    grids = [(6, 8), (3, 4), (3, 1), (1, 2), (1, 1)]
+    L = oc.Layout(oc.KIND_FRAME, dtype, B, T, Hh, W, C, gy=6, gx=8, frame_stat=stat)
+    n_units = [B * T * gy * gx for gy, gx in grids]
+    n_pairs = [B * (T - 1) * gy * gx for gy, gx in grids]
+    with H.make_ctx(oc, L) as ctx:
+        bs = torch.full((sum(n_units),), float("nan"), device="cuda")
+        bi = torch.full((sum(n_units),), -2, device="cuda", dtype=torch.int32)
+        ps = torch.full((sum(n_pairs),), float("nan"), device="cuda")
+        pos = torch.full((B, T - 1, Hh * W), float("nan"), device="cuda")
+        ctx.match_frame_levels(L, H.to_dev(w.x), grids, bs, bi, pos, ps)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == oc.OK
+        assert ctx.launches()["frame_pair"] == 1            # one streaming pass for all levels
+        uo = po = 0
+        for (gy, gx), nu, npair in zip(grids, n_units, n_pairs):
+            Lo = oracle.Layout(oracle.KIND_FRAME, dtype, B, T, Hh, W, C, gy=gy, gx=gx, frame_stat=stat)
+            ref = oracle.match_frame(Lo, w.x, want_pos=True)
+            H.check_match_against_oracle(oracle, Lo, w.x, bs[uo:uo + nu].cpu().numpy(), bi[uo:uo + nu].cpu().numpy(),
+                                         ref, TOL[dtype])
+            assert np.abs(ps[po:po + npair].cpu().numpy() - ref["pair_sim"].reshape(-1)).max() <= TOL[dtype]
+            assert np.abs(pos.cpu().numpy() - ref["pos_sim"]).max() <= TOL[dtype]
+            uo += nu
+            po += npair
+        # argument checks: a grid that does not divide the finest one, too many levels
+        assert ctx.match_frame_levels(L, H.to_dev(w.x), [(4, 8)], bs, bi, check=False) == oc.ERR_INVALID_ARG
+        assert ctx.match_frame_levels(L, H.to_dev(w.x), [(1, 1)] * 9, bs, bi, check=False) == oc.ERR_INVALID_ARG
+
+
 def test_frame_patch_chain_long_rows(oc, oracle):
     """Rows too long for the time-marching kernel: the pair kernel's tiles follow the patches too."""
     w = _frame_patch_workload(5, 1, 4, 4, 6, 2176, inputs.BF16, (2, 3), "threshold")
@@ -303,6 +336,18 @@ def test_block_chain_small(oc, oracle, dtype, lattice):
 # ---------------------------------------------------------------------------------------------------
 # full-size configs 2-4
 # ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("grid,mode", [((2, 2), "count"), ((1, 4), "count"), ((4, 1), "threshold"), ((2, 3), "count")])
+def test_block_patches_chain(oc, oracle, grid, mode):
+    """Patch-local Block Cache (Section 3.3): the selection is taken per patch of positions."""
+    w = inputs.latte_blocks(seed=77, T=5, H=16, W=24, C=72)
+    w.groups = grid
+    w.mode = mode
+    w.n_reuse = 7
+    rep = run_chain(oc, oracle, w, Cout=40)
+    if mode == "count":
+        assert rep["reused"] == 7 * grid[0] * grid[1]
+
+
 def test_config2_sd3_token_cache_full(oc, oracle):
     w = inputs.sd3_token_cache()
     rep = run_chain(oc, oracle, w, full_oracle=True)
