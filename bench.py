@@ -665,14 +665,15 @@ def _token_groups_one(args, oc, torch, dev, peaks, graph_time_us, label, base, g
     outs = [torch.empty_like(xs[0]) for _ in range(ring)]
     reps = max(3, args.steps // 10)
     results = []
+    kind = KIND[base.kind]
     for gy, gx in grids:
-        L = oc.Layout(oc.KIND_TOKEN, inputs.BF16, *base.shape, gy=gy, gx=gx)
+        L = oc.Layout(kind, inputs.BF16, *base.shape, gy=gy, gx=gx)
         G, U, R = L.counts()
         n_units, n_cand = G * U, G * (U - R)
         n_reuse = (U - R) // 2
         stride = U - n_reuse
         rows = oc.rows_from_layout(L, C, 2)
-        row_bytes = rows.seg_bytes
+        row_bytes = rows.seg_bytes * rows.n_seg
         ctx = oc.Context(0, oc.match_workspace_bytes(L))
         sims = [torch.empty(n_units, dtype=torch.float32, device=dev) for _ in range(ring)]
         idxs = [torch.empty(n_units, dtype=torch.int32, device=dev) for _ in range(ring)]
@@ -700,15 +701,22 @@ def _token_groups_one(args, oc, torch, dev, peaks, graph_time_us, label, base, g
                 ctx.restore(rows, ys[r], caches[r], n_units, so[r], mm[r], outs[r], stream=torch.cuda.current_stream())
         t = {k: graph_time_us(f, reps) / ring for k, f in
              (("match", f_match), ("select", f_select), ("gather", f_gather), ("restore", f_restore))}
-        flops = 2.0 * n_cand * R * C
-        results.append({
-            "workload": label, "shape": list(base.shape), "match_GFLOP": flops / 1e9,
-            "token_groups": gy * gx, "grid": [gy, gx], "groups": G, "units_per_group": U, "n_reuse_per_group": n_reuse,
+        # token: dense contraction; frame / block: every element is read once (about 3 FLOP per byte)
+        flops = 2.0 * n_cand * R * C if kind == 0 else 0.0
+        rec = {
+            "workload": label, "shape": list(base.shape),
+            "patches_per_frame": gy * gx, "grid": [gy, gx], "groups": G, "units_per_group": U, "n_reuse_per_group": n_reuse,
             "match_us": t["match"], "select_us": t["select"], "gather_us": t["gather"], "restore_us": t["restore"],
             "selection_plus_restoration_us": t["select"] + t["gather"] + t["restore"],
-            "summed_us": sum(t.values()), "match_TFLOP/s": flops / (t["match"] * 1e-6) / 1e12,
+            "summed_us": sum(t.values()),
             "gather_frac_hbm": 2 * G * stride * row_bytes / (t["gather"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
-            "restore_frac_hbm": 2 * n_units * row_bytes / (t["restore"] * 1e-6) / 1e9 / peaks["hbm_gbs"]})
+            "restore_frac_hbm": 2 * n_units * row_bytes / (t["restore"] * 1e-6) / 1e9 / peaks["hbm_gbs"]}
+        if kind == 0:
+            rec.update({"match_GFLOP": flops / 1e9, "token_groups": gy * gx,
+                        "match_TFLOP/s": flops / (t["match"] * 1e-6) / 1e12})
+        else:
+            rec["match_frac_hbm"] = tensor_bytes / (t["match"] * 1e-6) / 1e9 / peaks["hbm_gbs"]
+        results.append(rec)
         assert ctx.device_status() == oc.OK
         ctx.close()
     # patch-local against whole-frame matching (Hierarchical Caching, Section 3.3): cost ratios
@@ -716,7 +724,29 @@ def _token_groups_one(args, oc, torch, dev, peaks, graph_time_us, label, base, g
     for r in results:
         if t_global:
             r["match_time_ratio_vs_whole_frame"] = t_global / r["match_us"]
-            r["match_flop_ratio_vs_whole_frame"] = results[0]["match_GFLOP"] / r["match_GFLOP"]
+            if kind == 0:
+                r["match_flop_ratio_vs_whole_frame"] = results[0]["match_GFLOP"] / r["match_GFLOP"]
+    if kind == 1 and len(grids) > 1:
+        # the whole hierarchy from one streaming pass (oc_match_frame_levels) against one pass per level
+        fine = max(grids, key=lambda g: g[0] * g[1])
+        levels = [g for g in grids if fine[0] % g[0] == 0 and fine[1] % g[1] == 0]
+        L = oc.Layout(kind, inputs.BF16, *base.shape, gy=fine[0], gx=fine[1])
+        B, T = base.shape[0], base.shape[1]
+        nu = sum(B * T * a * b for a, b in levels)
+        ctx = oc.Context(0, oc.match_workspace_bytes(L))
+        sims = [torch.empty(nu, dtype=torch.float32, device=dev) for _ in range(ring)]
+        idxs = [torch.empty(nu, dtype=torch.int32, device=dev) for _ in range(ring)]
+
+        def f_levels():
+            for r in range(ring):
+                ctx.match_frame_levels(L, xs[r], levels, sims[r], idxs[r], stream=torch.cuda.current_stream())
+        t_lv = graph_time_us(f_levels, reps) / ring
+        separate = sum(r["match_us"] for r in results if tuple(r["grid"]) in levels)
+        results.append({"workload": label, "hierarchy_levels": [list(g) for g in levels],
+                        "one_pass_all_levels_us": t_lv, "one_pass_per_level_us": separate,
+                        "match_frac_hbm_one_pass": tensor_bytes / (t_lv * 1e-6) / 1e9 / peaks["hbm_gbs"]})
+        assert ctx.device_status() == oc.OK
+        ctx.close()
     del xs, caches, outs
     torch.cuda.empty_cache()
     return results
@@ -742,12 +772,20 @@ def main():
     if args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     rank, local_rank, world = sharding.env_rank_world()
-    if args.workload in ("svd_sweep", "sd3_groups", "svd_patches"):
+    if args.workload in ("svd_sweep", "sd3_groups", "svd_patches", "frame_block_patches"):
         if rank == 0:
             if args.workload == "svd_sweep":
                 run_sweep(args)
             elif args.workload == "sd3_groups":
                 run_token_groups(args)
+            elif args.workload == "frame_block_patches":
+                # patch-local Frame Cache (SVD frame tensor) and Block Cache (SVD level 0 and the Latte tensor)
+                blk = make_workload("svd_token_l0")
+                blk.kind = "block"
+                run_token_groups(args, [("svd_frame", make_workload("svd_frame"), ((1, 1), (2, 2), (4, 4), (12, 16))),
+                                        ("svd_block_l0", blk, ((1, 1), (2, 2), (4, 4), (12, 16))),
+                                        ("latte_block", make_workload("latte_block"), ((1, 1), (2, 2), (4, 4)))],
+                                 metric="per-op device time, Frame and Block Cache, whole-frame vs patch-local (Section 3.3)")
             else:
                 # patch-local Token Cache matching on the three SVD U-Net levels (per-frame groups cut into k x k patches)
                 grids = {0: ((1, 1), (2, 2), (4, 4), (6, 8)), 1: ((1, 1), (2, 2), (6, 8)), 2: ((1, 1), (3, 4))}

@@ -180,6 +180,58 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_launch_dependents(); }
 
+// ---- shared-memory barriers (mbarrier) with bounded waits ----------------------------------------
+// Every wait in this library gives up after WAIT_LIMIT_NS, so that a lost copy shows up as
+// OC_ERR_TIMEOUT in the context's status word instead of a hung device.
+static constexpr unsigned long long WAIT_LIMIT_NS = 1000000000ull;   // 1 s per wait
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// One look at a barrier, never suspending the thread.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within WAIT_LIMIT_NS or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    unsigned spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+        }
+    }
+    return true;
+}
 __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -209,33 +261,41 @@ __device__ __forceinline__ unsigned long long pack_key(float v, uint32_t idx) {
 
 // fp32 partial products of one 16-byte chunk of two rows: dot, |a|^2, |b|^2.
 template <int DT> struct Chunk;
+// bf16 operands go straight into the fp32 FMA (fma.rn.f32.bf16: bf16 x bf16 + fp32, one rounding), so a
+// pair of packed elements costs its FMAs and nothing else -- no shift/mask to widen them first.  The
+// product of two bf16 values is exact in fp32, so the result equals that of widening and fmaf().
 template <> struct Chunk<OC_DTYPE_BF16> {
+    static __device__ __forceinline__ void word3(uint32_t a, uint32_t b, float& dot, float& na, float& nb) {
+        asm("{\n\t.reg .b16 al, ah, bl, bh;\n\t"
+            "mov.b32 {al, ah}, %3;\n\tmov.b32 {bl, bh}, %4;\n\t"
+            "fma.rn.f32.bf16 %0, al, bl, %0;\n\tfma.rn.f32.bf16 %0, ah, bh, %0;\n\t"
+            "fma.rn.f32.bf16 %1, al, al, %1;\n\tfma.rn.f32.bf16 %1, ah, ah, %1;\n\t"
+            "fma.rn.f32.bf16 %2, bl, bl, %2;\n\tfma.rn.f32.bf16 %2, bh, bh, %2;\n\t}"
+            : "+f"(dot), "+f"(na), "+f"(nb) : "r"(a), "r"(b));
+    }
+    static __device__ __forceinline__ void word2(uint32_t a, uint32_t b, float& dot, float& na) {
+        asm("{\n\t.reg .b16 al, ah, bl, bh;\n\t"
+            "mov.b32 {al, ah}, %2;\n\tmov.b32 {bl, bh}, %3;\n\t"
+            "fma.rn.f32.bf16 %0, al, bl, %0;\n\tfma.rn.f32.bf16 %0, ah, bh, %0;\n\t"
+            "fma.rn.f32.bf16 %1, al, al, %1;\n\tfma.rn.f32.bf16 %1, ah, ah, %1;\n\t}"
+            : "+f"(dot), "+f"(na) : "r"(a), "r"(b));
+    }
+    static __device__ __forceinline__ void word1(uint32_t a, float& na) {
+        asm("{\n\t.reg .b16 al, ah;\n\t"
+            "mov.b32 {al, ah}, %1;\n\t"
+            "fma.rn.f32.bf16 %0, al, al, %0;\n\tfma.rn.f32.bf16 %0, ah, ah, %0;\n\t}"
+            : "+f"(na) : "r"(a));
+    }
     static __device__ __forceinline__ void acc3(const uint4& a, const uint4& b, float& dot, float& na, float& nb) {
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float a0 = bf16_lo(aw[i]), a1 = bf16_hi(aw[i]), b0 = bf16_lo(bw[i]), b1 = bf16_hi(bw[i]);
-            dot = fmaf(a0, b0, dot); dot = fmaf(a1, b1, dot);
-            na = fmaf(a0, a0, na);   na = fmaf(a1, a1, na);
-            nb = fmaf(b0, b0, nb);   nb = fmaf(b1, b1, nb);
-        }
+        word3(a.x, b.x, dot, na, nb); word3(a.y, b.y, dot, na, nb);
+        word3(a.z, b.z, dot, na, nb); word3(a.w, b.w, dot, na, nb);
     }
     static __device__ __forceinline__ void acc2(const uint4& a, const uint4& b, float& dot, float& na) {
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float a0 = bf16_lo(aw[i]), a1 = bf16_hi(aw[i]), b0 = bf16_lo(bw[i]), b1 = bf16_hi(bw[i]);
-            dot = fmaf(a0, b0, dot); dot = fmaf(a1, b1, dot);
-            na = fmaf(a0, a0, na);   na = fmaf(a1, a1, na);
-        }
+        word2(a.x, b.x, dot, na); word2(a.y, b.y, dot, na);
+        word2(a.z, b.z, dot, na); word2(a.w, b.w, dot, na);
     }
     static __device__ __forceinline__ void sq(const uint4& a, float& na) {
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float a0 = bf16_lo(aw[i]), a1 = bf16_hi(aw[i]);
-            na = fmaf(a0, a0, na); na = fmaf(a1, a1, na);
-        }
+        word1(a.x, na); word1(a.y, na); word1(a.z, na); word1(a.w, na);
     }
 };
 template <> struct Chunk<OC_DTYPE_F32> {

@@ -128,7 +128,7 @@ frame_pair_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float ep
 static constexpr int MARCH_CPL = 8;      // most 16-byte chunks a lane may hold per row (instantiated for 5 and 8)
 
 template <int DT, int LPR, int CPL>
-__global__ void __launch_bounds__(PAIR_THREADS)
+__global__ void __launch_bounds__(PAIR_THREADS, CPL <= 5 ? 3 : 2)
 frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float eps, int seg_len, int n_seg,
                    float* __restrict__ pos_sim, float4* __restrict__ partial, PatchGrid pg) {
     pdl_enter();
@@ -213,57 +213,91 @@ struct FinLevel {
     int n_pos;              // positions per patch of this level
 };
 
-__device__ __forceinline__ float frame_pair_value(const float4* __restrict__ partial, long long q, int patch,
-                                                  const FinLevel& lv, int stat, float eps) {
+// record j (0 <= j < ry*rx*tiles_per_patch, a fixed enumeration) of patch `patch` of pair q at this level
+__device__ __forceinline__ float4 level_record(const float4* __restrict__ partial, long long q, int patch,
+                                               const FinLevel& lv, int j) {
+    if (lv.ry * lv.rx == 1) return partial[(q * lv.np_fine + patch) * lv.tiles_per_patch + j];
+    const int py = patch / lv.gx, px = patch - py * lv.gx;
+    const int per_row = lv.rx * lv.tiles_per_patch;
+    const int fy = j / per_row, r = j - fy * per_row;
+    const int fx = r / lv.tiles_per_patch, k = r - fx * lv.tiles_per_patch;
+    const int fine = (py * lv.ry + fy) * lv.gx_fine + px * lv.rx + fx;
+    return partial[(q * lv.np_fine + fine) * lv.tiles_per_patch + k];
+}
+
+// The statistics of pair q0 (if has0) and pair q1 (if has1) for one patch, by one warp.  The kernel is
+// pure latency (a few hundred records out of L2), so a lane issues the loads of eight rounds of both
+// pairs before it adds anything; the order of the additions is fixed.
+__device__ __forceinline__ void frame_pair_values(const float4* __restrict__ partial, long long q0, bool has0,
+                                                  long long q1, bool has1, int patch, const FinLevel& lv, int stat,
+                                                  float eps, float& out0, float& out1) {
     const int lane = threadIdx.x & 31;
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    if (lv.ry * lv.rx == 1) {
-        const float4* rec = partial + (q * lv.np_fine + patch) * lv.tiles_per_patch;
-        for (int i = lane; i < lv.tiles_per_patch; i += 32) {
-            const float4 v = rec[i];
-            a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+    const int n_rec = lv.ry * lv.rx * lv.tiles_per_patch;
+    float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+    constexpr int BATCH = 8;
+    for (int j0 = lane; j0 < n_rec; j0 += 32 * BATCH) {
+        float4 v0[BATCH], v1[BATCH];
+#pragma unroll
+        for (int k = 0; k < BATCH; ++k) {
+            const int j = j0 + 32 * k;
+            v0[k] = (has0 && j < n_rec) ? level_record(partial, q0, patch, lv, j) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v1[k] = (has1 && j < n_rec) ? level_record(partial, q1, patch, lv, j) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-    } else {
-        const int py = patch / lv.gx, px = patch - py * lv.gx;
-        const int per_row = lv.rx * lv.tiles_per_patch, n_rec = lv.ry * per_row;
-        for (int j = lane; j < n_rec; j += 32) {
-            const int fy = j / per_row, r = j - fy * per_row;
-            const int fx = r / lv.tiles_per_patch, k = r - fx * lv.tiles_per_patch;
-            const int fine = (py * lv.ry + fy) * lv.gx_fine + px * lv.rx + fx;
-            const float4 v = partial[(q * lv.np_fine + fine) * lv.tiles_per_patch + k];
-            a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+#pragma unroll
+        for (int k = 0; k < BATCH; ++k) {
+            s0.x += v0[k].x; s0.y += v0[k].y; s0.z += v0[k].z; s0.w += v0[k].w;
+            s1.x += v1[k].x; s1.y += v1[k].y; s1.z += v1[k].z; s1.w += v1[k].w;
         }
     }
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {
-        a0 += __shfl_xor_sync(0xFFFFFFFFu, a0, d); a1 += __shfl_xor_sync(0xFFFFFFFFu, a1, d);
-        a2 += __shfl_xor_sync(0xFFFFFFFFu, a2, d); a3 += __shfl_xor_sync(0xFFFFFFFFu, a3, d);
+        s0.x += __shfl_xor_sync(0xFFFFFFFFu, s0.x, d); s0.y += __shfl_xor_sync(0xFFFFFFFFu, s0.y, d);
+        s0.z += __shfl_xor_sync(0xFFFFFFFFu, s0.z, d); s0.w += __shfl_xor_sync(0xFFFFFFFFu, s0.w, d);
+        s1.x += __shfl_xor_sync(0xFFFFFFFFu, s1.x, d); s1.y += __shfl_xor_sync(0xFFFFFFFFu, s1.y, d);
+        s1.z += __shfl_xor_sync(0xFFFFFFFFu, s1.z, d); s1.w += __shfl_xor_sync(0xFFFFFFFFu, s1.w, d);
     }
-    return stat == OC_FRAME_FLAT_COS ? clamp_unit(a1 / (fmaxf(sqrtf(a2), eps) * fmaxf(sqrtf(a3), eps)))
-                                     : a0 / (float)lv.n_pos;
+    if (stat == OC_FRAME_FLAT_COS) {
+        out0 = clamp_unit(s0.y / (fmaxf(sqrtf(s0.z), eps) * fmaxf(sqrtf(s0.w), eps)));
+        out1 = clamp_unit(s1.y / (fmaxf(sqrtf(s1.z), eps) * fmaxf(sqrtf(s1.w), eps)));
+    } else {
+        out0 = s0.x / (float)lv.n_pos;
+        out1 = s1.x / (float)lv.n_pos;
+    }
 }
 
+struct FinLevels {
+    int n;
+    FinLevel lv[OC_MAX_FRAME_LEVELS];
+    int unit_off[OC_MAX_FRAME_LEVELS + 1];      // first output unit of each level (levels are stored one after another)
+    int pair_off[OC_MAX_FRAME_LEVELS + 1];      // first pair_sim entry of each level
+};
+
 __global__ void __launch_bounds__(PAIR_THREADS)
-frame_finalize_kernel(const float4* __restrict__ partial, FinLevel lv, int B, int T, int stat, float eps,
-                      float* __restrict__ pair_sim, float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
+frame_finalize_kernel(const float4* __restrict__ partial, const __grid_constant__ FinLevels F, int B, int T, int stat,
+                      float eps, float* __restrict__ pair_sim, float* __restrict__ best_sim,
+                      int32_t* __restrict__ best_idx) {
     pdl_enter();
-    const int n_patches = lv.gy * lv.gx;
-    const int i = blockIdx.x * (PAIR_THREADS / 32) + (threadIdx.x >> 5);     // unit index (b*T + t)*n_patches + patch
+    const int w = blockIdx.x * (PAIR_THREADS / 32) + (threadIdx.x >> 5);     // output unit over all levels
     const int lane = threadIdx.x & 31;
-    if (i >= B * T * n_patches) return;                                       // whole warps leave together
+    if (w >= F.unit_off[F.n]) return;                                         // whole warps leave together
+    int l = 0;
+    while (l + 1 < F.n && w >= F.unit_off[l + 1]) ++l;
+    const FinLevel& lv = F.lv[l];
+    const int n_patches = lv.gy * lv.gx;
+    const int i = w - F.unit_off[l];                                          // unit index (b*T + t)*n_patches + patch
     const int bt = i / n_patches, patch = i - bt * n_patches;
     const int b = bt / T, t = bt - b * T;
     const long long q_prev = (long long)b * (T - 1) + t - 1;                  // pair (t, t-1)
-    float with_prev = -INFINITY, with_next = -INFINITY;
-    if (t >= 1) {
-        with_prev = frame_pair_value(partial, q_prev, patch, lv, stat, eps);
-        if (lane == 0 && pair_sim) pair_sim[q_prev * n_patches + patch] = with_prev;
-    }
-    if ((t & 1) && t + 1 < T) with_next = frame_pair_value(partial, q_prev + 1, patch, lv, stat, eps);
+    const bool has_prev = t >= 1, has_next = (t & 1) && t + 1 < T;
+    float with_prev, with_next;
+    frame_pair_values(partial, q_prev, has_prev, q_prev + 1, has_next, patch, lv, stat, eps, with_prev, with_next);
+    if (!has_prev) with_prev = -INFINITY;
+    if (!has_next) with_next = -INFINITY;
+    if (lane == 0 && has_prev && pair_sim) pair_sim[F.pair_off[l] + q_prev * n_patches + patch] = with_prev;
     if (lane == 0) {
-        if ((t & 1) == 0) { best_sim[i] = -INFINITY; best_idx[i] = i; }
-        else if (with_next > with_prev) { best_sim[i] = with_next; best_idx[i] = i + n_patches; }
-        else { best_sim[i] = with_prev; best_idx[i] = i - n_patches; }
+        if ((t & 1) == 0) { best_sim[w] = -INFINITY; best_idx[w] = i; }
+        else if (with_next > with_prev) { best_sim[w] = with_next; best_idx[w] = i + n_patches; }
+        else { best_sim[w] = with_prev; best_idx[w] = i - n_patches; }
     }
 }
 
@@ -360,20 +394,24 @@ static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, co
                 frame_dispatch<OC_DTYPE_F32>(f.lpr, grid, s, (const uint8_t*)x, g.T, P, cpr, g.eps, pos_sim, partial, f.ppc, f.pg);
         }
     }
+    FinLevels F;
+    F.n = n_levels;
+    F.unit_off[0] = F.pair_off[0] = 0;
     for (int l = 0; l < n_levels; ++l) {
-        FinLevel lv;
+        FinLevel& lv = F.lv[l];
         lv.gy = levels ? levels[2 * l] : g.gy; lv.gx = levels ? levels[2 * l + 1] : g.gx;
         lv.ry = g.gy / lv.gy; lv.rx = g.gx / lv.gx;
         lv.gx_fine = g.gx; lv.np_fine = g.gy * g.gx;
         lv.tiles_per_patch = f.pg.tiles_per_patch;
         lv.n_pos = f.pg.Pp * lv.ry * lv.rx;
-        const long long units = (long long)g.B * g.T * lv.gy * lv.gx;
+        F.unit_off[l + 1] = F.unit_off[l] + g.B * g.T * lv.gy * lv.gx;
+        F.pair_off[l + 1] = F.pair_off[l] + n_pairs * lv.gy * lv.gx;
+    }
+    {
         Scope scope(ctx, OC_K_FRAME_FIN, s);
         const int warps = PAIR_THREADS / 32;
-        OC_LAUNCH((frame_finalize_kernel), (unsigned)((units + warps - 1) / warps), PAIR_THREADS, 0, s,
-            partial, lv, g.B, g.T, g.frame_stat, g.eps, pair_sim, best_sim, best_idx);
-        best_sim += units; best_idx += units;
-        if (pair_sim) pair_sim += (long long)n_pairs * lv.gy * lv.gx;
+        OC_LAUNCH((frame_finalize_kernel), (unsigned)((F.unit_off[n_levels] + warps - 1) / warps), PAIR_THREADS, 0, s,
+            partial, F, g.B, g.T, g.frame_stat, g.eps, pair_sim, best_sim, best_idx);
     }
     return last_launch_status();
 }

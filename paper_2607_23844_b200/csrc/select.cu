@@ -473,6 +473,86 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     if (tid == 0) kept_count[g] = kept_total;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Small groups (at most 64 units: the frames of a clip, the positions of a small patch): one WARP
+// per group, two units per lane, everything in registers.  The count-mode rank of a candidate is
+// counted directly -- how many candidates of the group precede it in (similarity descending, index
+// ascending) order -- by passing every key round the warp; positions come from ballots.  No shared
+// memory, no CTA barrier: the kernel costs a launch plus a few hundred cycles.
+// ------------------------------------------------------------------------------------------------
+static constexpr int SEL_SMALL_UNITS = 64;
+static constexpr int SEL_SMALL_THREADS = 128;
+
+__global__ void __launch_bounds__(SEL_SMALL_THREADS)
+select_small_kernel(GroupMap gm, long long n_groups, const float* __restrict__ best_sim,
+                    const int32_t* __restrict__ best_idx, int mode, float thr, int n_reuse, int y_stride,
+                    int32_t* __restrict__ kept_idx, int32_t* __restrict__ kept_count,
+                    int32_t* __restrict__ match_map, int32_t* __restrict__ slot_of) {
+    pdl_enter();
+    const long long g = (long long)blockIdx.x * (SEL_SMALL_THREADS / 32) + (threadIdx.x >> 5);
+    if (g >= n_groups) return;                                 // whole warps leave together
+    const int lane = threadIdx.x & 31;
+    const int U = gm.units_per_group;
+    const GroupView gv(gm, g);
+    long long gi[2];
+    unsigned key[2];
+    int m_idx[2];
+    bool valid[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int u = lane + 32 * h;
+        valid[h] = u < U;
+        gi[h] = valid[h] ? gv.index(gm, u) : 0;
+        key[h] = 0; m_idx[h] = 0;
+        if (valid[h] && gv.is_cand(gm, u)) {
+            key[h] = f32_to_ordered(best_sim[gi[h]]); key[h] = key[h] ? key[h] : 1u;   // 0 marks a non-candidate
+            m_idx[h] = best_idx[gi[h]];
+        }
+    }
+    bool reuse[2] = {false, false};
+    if (mode == OC_SELECT_THRESHOLD) {
+        unsigned tk = f32_to_ordered(thr); tk = tk ? tk : 1u;      // sim >= thr  <=>  key >= ordered(thr)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) reuse[h] = key[h] != 0 && key[h] >= tk;
+    } else {
+        const int n_cand = __popc(__ballot_sync(0xFFFFFFFFu, key[0] != 0)) + __popc(__ballot_sync(0xFFFFFFFFu, key[1] != 0));
+        const int k = n_reuse < n_cand ? n_reuse : n_cand;
+        int rank[2] = {0, 0};
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+            if (32 * h2 >= U) break;                            // (uniform)
+            for (int l = 0; l < 32; ++l) {
+                const unsigned ko = __shfl_sync(0xFFFFFFFFu, key[h2], l);
+                const int uo = l + 32 * h2;
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+                    rank[h] += (ko != 0 && (ko > key[h] || (ko == key[h] && uo < lane + 32 * h))) ? 1 : 0;
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) reuse[h] = key[h] != 0 && rank[h] < k;
+    }
+    const unsigned lt = (1u << lane) - 1u;
+    const unsigned k0 = __ballot_sync(0xFFFFFFFFu, valid[0] && !reuse[0]);
+    const unsigned k1 = __ballot_sync(0xFFFFFFFFu, valid[1] && !reuse[1]);
+    const int pos[2] = {__popc(k0 & lt), __popc(k0) + __popc(k1 & lt)};
+    const int kept_total = __popc(k0) + __popc(k1);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        if (!valid[h]) continue;
+        if (!reuse[h]) {
+            if (pos[h] < y_stride) kept_idx[g * y_stride + pos[h]] = (int32_t)gi[h];
+            slot_of[gi[h]] = (int32_t)(g * y_stride + pos[h]);
+            match_map[gi[h]] = (int32_t)gi[h];
+        } else {
+            slot_of[gi[h]] = -1;
+            match_map[gi[h]] = m_idx[h];
+        }
+    }
+    for (int p = kept_total + lane; p < y_stride; p += 32) kept_idx[g * y_stride + p] = -1;
+    if (lane == 0) kept_count[g] = kept_total;
+}
+
 oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, const int32_t* best_idx,
                         int mode, float thr, int64_t n_reuse, int64_t y_stride, int32_t* kept_idx,
                         int32_t* kept_count, int32_t* match_map, int32_t* slot_of, cudaStream_t s) {
@@ -490,7 +570,12 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
         attr_set = true;
     }
     LaunchScope scope(ctx, OC_K_SELECT, s);
-    if (!geo.self_match && geo.units_per_group <= SEL_SMEM_KEYS) {
+    if (!geo.self_match && geo.units_per_group <= SEL_SMALL_UNITS) {
+        const int wpc = SEL_SMALL_THREADS / 32;
+        OC_LAUNCH(select_small_kernel, (unsigned)((geo.n_groups + wpc - 1) / wpc), SEL_SMALL_THREADS, 0, s,
+                  gm, (long long)geo.n_groups, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count,
+                  match_map, slot_of);
+    } else if (!geo.self_match && geo.units_per_group <= SEL_SMEM_KEYS) {
         // A group wants every thread it can get (the kernel is latency-bound per thread); only when the
         // groups do not all fit on the device at once, and are small, do smaller CTAs pay (more groups in
         // flight).  A thread's run of units must fit its 64-bit reuse mask.

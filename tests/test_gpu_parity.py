@@ -578,6 +578,45 @@ def test_runtime_argument_errors_launch_nothing(oc, oracle):
         assert ctx.device_status() == oc.OK
 
 
+@pytest.mark.parametrize("kind,shape,kw", [
+    (1, (3, 25, 4, 4, 8), {}), (1, (2, 64, 4, 6, 8), dict(gy=2, gx=3)), (1, (1, 1, 4, 4, 8), {}),
+    (1, (2, 33, 2, 2, 8), dict(gy=2, gx=1)), (1, (1, 65, 2, 2, 8), {}),
+    (2, (2, 3, 16, 24, 8), dict(gy=2, gx=3)), (2, (1, 2, 16, 16, 8), dict(gy=4, gx=4)), (2, (3, 2, 6, 10, 8), {}),
+    (0, (1, 3, 8, 8, 8), {}), (0, (2, 2, 12, 20, 8), dict(gy=3, gx=2, sy=2, sx=5, oy=1, ox=3)),
+    (0, (1, 2, 16, 16, 8), dict(gy=2, gx=4)),
+])
+def test_select_small_and_strided_groups_with_ties(oc, oracle, kind, shape, kw):
+    """Groups of at most 64 units (one warp each) and just above; quantised similarities give many ties."""
+    L = oc.Layout(kind, oc.DTYPE_BF16, *shape, **kw)
+    Lo = oracle.Layout(kind, oracle.DT_BF16, *shape, **kw)
+    G, U, R = L.counts()
+    n = G * U
+    rng = np.random.default_rng(G * 1000 + U)
+    sim_np = (np.round(rng.uniform(-1, 1, n) * 6) / 6).astype(np.float32)
+    sim_np[rng.integers(0, n, 3)] = 0.0
+    sim_np[rng.integers(0, n, 3)] = -0.0
+    idx_np = np.zeros(n, np.int32)
+    reps = [u for u in range(U) if Lo.is_rep(u)]
+    for g in range(G):
+        for u in range(U):
+            i = Lo.unit_index(g, u)
+            if Lo.is_rep(u):
+                sim_np[i] = -np.inf
+                idx_np[i] = i
+            else:                                   # a match is always a representative of the same group
+                idx_np[i] = Lo.unit_index(g, reps[int(rng.integers(0, len(reps)))])
+    n_cand = U - R
+    with oc.Context(0, 0) as ctx:
+        for mode, thr, n_reuse in ((oc.SELECT_COUNT, 0.0, 0), (oc.SELECT_COUNT, 0.0, 1), (oc.SELECT_COUNT, 0.0, n_cand // 2),
+                                   (oc.SELECT_COUNT, 0.0, max(n_cand - 1, 0)), (oc.SELECT_COUNT, 0.0, n_cand + 3),
+                                   (oc.SELECT_THRESHOLD, 0.0, 0), (oc.SELECT_THRESHOLD, 1 / 3, 0),
+                                   (oc.SELECT_THRESHOLD, -1.0, 0), (oc.SELECT_THRESHOLD, 1.5, 0)):
+            stride = U - min(n_reuse, n_cand) if mode == oc.SELECT_COUNT else U
+            s = H.gpu_select(oc, ctx, L, H.to_dev(sim_np), H.to_dev(idx_np), mode, thr, n_reuse, stride)
+            H.check_select_against_oracle(oracle, Lo, sim_np, idx_np, mode, thr, n_reuse, stride, s)
+        assert ctx.device_status() == oc.OK
+
+
 def test_select_capacity_limits(oc, oracle):
     # 65536 units per group is the supported maximum; one more patch row is rejected
     L = oc.Layout(oc.KIND_TOKEN, oc.DTYPE_BF16, 1, 1, 256, 256, 8)
