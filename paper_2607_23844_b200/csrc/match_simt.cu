@@ -10,7 +10,7 @@
 namespace oc {
 
 // ---- pre-pass ----------------------------------------------------------------------------------
-// Persistent warps; a thread-group of LPR lanes owns a row (about five 16-byte chunks per lane), so a
+// A thread-group of LPR lanes owns a row (about five 16-byte chunks per lane), so a
 // warp has 32/LPR rows in flight and every lane keeps several independent loads outstanding.
 template <int DT, int LPR>
 __global__ void __launch_bounds__(256)
@@ -52,7 +52,10 @@ static void norms_dispatch(int sm_count, cudaStream_t s, const uint8_t* x, long 
     while (lpr < 32 && lpr * 5 < cpr) lpr <<= 1;
     const long long rows_per_block = 256 / lpr;
     long long blocks = (n_tok + rows_per_block - 1) / rows_per_block;
-    const long long cap = (long long)sm_count * 4;           // 4 resident CTAs of 256 threads per SM (64 registers)
+    // one pass per CTA: short CTAs that retire and are replaced keep more loads in flight than a
+    // persistent grid does (measured: 0.75 against 0.71 of the copy bandwidth on a 147 MB tensor)
+    const long long cap = 0x7FFFFFFFll;
+    (void)sm_count;
     if (blocks > cap) blocks = cap;
     switch (lpr) {
         case 4:  OC_LAUNCH((norms_kernel<DT, 4>), (unsigned)blocks, 256, 0, s, x, n_tok, cpr, eps, inv_norm, keys); break;
