@@ -67,6 +67,10 @@ def lib():
         _lib.ocr_match_token.argtypes = [C.c_void_p] * 3 + [C.c_int64] + [C.c_void_p] * 4
         _lib.ocr_match_frame.argtypes = [C.c_void_p] * 6
         _lib.ocr_match_block.argtypes = [C.c_void_p] * 4
+        _lib.ocr_joint_groups.argtypes = [C.c_int, C.c_int] + [C.c_void_p] * 4
+        _lib.ocr_match_joint.argtypes = [C.c_void_p] * 6
+        _lib.ocr_select_joint.argtypes = ([C.c_void_p] * 4 + [C.c_int, C.c_float, C.c_int64, C.c_int64, C.c_int64]
+                                          + [C.c_void_p] * 4)
         _lib.ocr_select.argtypes = ([C.c_void_p] * 3 + [C.c_int, C.c_float, C.c_int64, C.c_int64]
                                     + [C.c_void_p] * 4)
         _lib.ocr_gather.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
@@ -268,6 +272,48 @@ def restore(R: Rows, z: np.ndarray, cache: np.ndarray | None, n_units: int, slot
                            _p(out), src_mode)
     assert rc == 0
     return out
+
+
+def joint_groups(B: int, T: int, frame_best_sim, frame_best_idx, frame_slot_of) -> np.ndarray:
+    """Frame pairs of Frame Cache as token groups (Section 3.2.3): [B*T, 2] int32 (u, t) per slot."""
+    fs = np.ascontiguousarray(frame_best_sim, np.float32)
+    fi = np.ascontiguousarray(frame_best_idx, np.int32)
+    so = np.ascontiguousarray(frame_slot_of, np.int32)
+    frames = np.empty((B * T, 2), np.int32)
+    rc = lib().ocr_joint_groups(B, T, _p(fs), _p(fi), _p(so), _p(frames))
+    assert rc == 0, rc
+    return frames
+
+
+def match_joint(L: Layout, x: np.ndarray, frames: np.ndarray):
+    _check(x, L)
+    n = L.B * L.T * L.H * L.W
+    frames = np.ascontiguousarray(frames, np.int32)
+    best_sim = np.full(n, np.nan, np.float32)
+    best_idx = np.full(n, -7, np.int32)
+    second = np.full(n, np.nan, np.float32)
+    rc = lib().ocr_match_joint(C.byref(L.c()), _p(x), _p(frames), _p(best_sim), _p(best_idx), _p(second))
+    assert rc == 0, rc
+    return dict(best_sim=best_sim, best_idx=best_idx, second_sim=second)
+
+
+def select_joint(L: Layout, frames: np.ndarray, best_sim, best_idx, mode: int, thr: float = 0.0,
+                 n_reuse_pair: int = 0, n_reuse_single: int = 0, y_group_stride: int | None = None):
+    F, P = L.B * L.T, L.H * L.W
+    if y_group_stride is None:
+        y_group_stride = 2 * P
+    frames = np.ascontiguousarray(frames, np.int32)
+    best_sim = np.ascontiguousarray(best_sim, np.float32)
+    best_idx = np.ascontiguousarray(best_idx, np.int32)
+    kept_idx = np.full(F * y_group_stride, -7, np.int32)
+    kept_count = np.full(F, -7, np.int32)
+    match_map = np.full(F * P, -7, np.int32)
+    slot_of = np.full(F * P, -7, np.int32)
+    rc = lib().ocr_select_joint(C.byref(L.c()), _p(frames), _p(best_sim), _p(best_idx), mode, thr,
+                                n_reuse_pair, n_reuse_single, y_group_stride, _p(kept_idx),
+                                _p(kept_count), _p(match_map), _p(slot_of))
+    assert rc == 0, rc
+    return dict(kept_idx=kept_idx, kept_count=kept_count, match_map=match_map, slot_of=slot_of)
 
 
 def layer_cache_hit(stored_step: int, step: int, interval: int) -> bool:

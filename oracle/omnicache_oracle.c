@@ -365,6 +365,134 @@ int ocr_select(const ocr_layout* L, const float* best_sim, const int32_t* best_i
     return 0;
 }
 
+/* ---- O5b: Token Cache on the frame pairs of Frame Cache (Section 3.2.3) -----------------------
+ * "Token Cache consumes the same feature map and frame-pair metadata used by Frame Cache ... For
+ * frame pairs selected by Frame Cache, we reshape the paired features from (B, 2 r_f, H, W, C) to
+ * (B r_f, 2HW, C).  Within each local 2x2x2 cube, Token Cache retains representative tokens ...
+ * For unmatched frames, the same procedure is applied within local 2x2 spatial neighborhoods."
+ *
+ * Reading (the paper fixes neither the cube's representative nor what happens when two candidate
+ * frames pick the same representative frame):
+ *   - a candidate frame t that Frame Cache marked for reuse claims its matched representative
+ *     frame u = frame_best_idx[t]; if both neighbours of u claim it, the one with the larger frame
+ *     similarity wins (equal: the earlier frame), the other stays unmatched;
+ *   - a pair (u, t) is ONE token group of 2HW tokens: the lattice tokens of frame u are its
+ *     representatives (one per 2x2x2 cube: the cube's (oy, ox) member in the representative
+ *     frame), the other 3HW/4 tokens of u and ALL HW tokens of t are candidates, each compared
+ *     with all representatives of the group;
+ *   - every other frame is a group of its own with the usual lattice (unmatched frames).
+ * frames[f] = (u, t) for slot f: (f, partner) if f is the representative frame of a pair,
+ * (f, -1) if f is a group of its own, (-1, -1) if f was absorbed into its partner's group.
+ * Units of a pair are ordered by time: the earlier frame's tokens first. */
+int ocr_joint_groups(int B, int T, const float* frame_best_sim, const int32_t* frame_best_idx,
+                     const int32_t* frame_slot_of, int32_t* frames) {
+    for (int64_t f = 0; f < (int64_t)B * T; ++f) { frames[2 * f] = (int32_t)f; frames[2 * f + 1] = -1; }
+    for (int b = 0; b < B; ++b)
+        for (int u = 0; u < T; u += 2) {                       /* representative frames */
+            int64_t fu = (int64_t)b * T + u, win = -1;
+            for (int d = -1; d <= 1; d += 2) {
+                int t = u + d;
+                if (t < 0 || t >= T) continue;
+                int64_t ft = (int64_t)b * T + t;
+                if (frame_slot_of[ft] >= 0 || frame_best_idx[ft] != fu) continue;   /* not reused / matched elsewhere */
+                if (win < 0 || frame_best_sim[ft] > frame_best_sim[win]) win = ft;  /* equal: the earlier one stays */
+            }
+            if (win >= 0) { frames[2 * fu + 1] = (int32_t)win; frames[2 * win] = -1; frames[2 * win + 1] = -1; }
+        }
+    return 0;
+}
+
+/* is token i (frame f = i / HW) a representative of its joint group? */
+static int joint_is_rep(const ocr_layout* L, const int32_t* frames, int64_t i) {
+    int64_t P = (int64_t)L->H * L->W, f = i / P, p = i % P, y = p / L->W, xx = p % L->W;
+    if (frames[2 * f] < 0) return 0;                            /* absorbed frame: all candidates */
+    return (y % L->sy) == L->oy && (xx % L->sx) == L->ox;
+}
+
+int ocr_match_joint(const ocr_layout* L, const void* x, const int32_t* frames, float* best_sim,
+                    int32_t* best_idx, float* second_sim) {
+    if (L->kind != 0 || L->gy != 1 || L->gx != 1 || L->self_match) return 1;
+    const int64_t P = (int64_t)L->H * L->W, F = (int64_t)L->B * L->T, C = L->C;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t slot = 0; slot < F; ++slot) {
+        int64_t u = frames[2 * slot], t = frames[2 * slot + 1];
+        if (u < 0) continue;
+        for (int half = 0; half < 2; ++half) {
+            int64_t f = half ? t : u;
+            if (f < 0) continue;
+            for (int64_t p = 0; p < P; ++p) {
+                int64_t i = f * P + p;
+                if (joint_is_rep(L, frames, i)) {
+                    best_sim[i] = -INFINITY; best_idx[i] = (int32_t)i;
+                    if (second_sim) second_sim[i] = -INFINITY;
+                    continue;
+                }
+                double best = -INFINITY, second = -INFINITY; int64_t arg = i;
+                for (int64_t r = 0; r < P; ++r) {             /* representatives: the lattice of frame u */
+                    int64_t j = u * P + r;
+                    if (!joint_is_rep(L, frames, j)) continue;
+                    double s = ocr_cosine(x, L->dtype, i * C, j * C, C, L->eps);
+                    if (s > best) { second = best; best = s; arg = j; }
+                    else if (s > second) second = s;
+                }
+                best_sim[i] = (float)best; best_idx[i] = (int32_t)arg;
+                if (second_sim) second_sim[i] = (float)second;
+            }
+        }
+    }
+    return 0;
+}
+
+/* Selection over the joint groups: as ocr_select, the group of slot f being the tokens of its one
+ * or two frames in time order.  n_reuse_pair / n_reuse_single: count-mode budgets of a pair group
+ * and of a single-frame group.  kept_idx: [B*T slots][y_group_stride]; absorbed slots keep nothing. */
+int ocr_select_joint(const ocr_layout* L, const int32_t* frames, const float* best_sim,
+                     const int32_t* best_idx, int mode, float thr, int64_t n_reuse_pair,
+                     int64_t n_reuse_single, int64_t y_group_stride, int32_t* kept_idx,
+                     int32_t* kept_count, int32_t* match_map, int32_t* slot_of) {
+    if (L->kind != 0 || L->gy != 1 || L->gx != 1 || L->self_match) return 1;
+    const int64_t P = (int64_t)L->H * L->W, F = (int64_t)L->B * L->T;
+    uint8_t* reuse = (uint8_t*)calloc((size_t)(F * P > 0 ? F * P : 1), 1);
+    ocr_rank* rk = (ocr_rank*)malloc(sizeof(ocr_rank) * (size_t)(2 * P > 0 ? 2 * P : 1));
+    int64_t* unit = (int64_t*)malloc(sizeof(int64_t) * (size_t)(2 * P > 0 ? 2 * P : 1));
+    if (!reuse || !rk || !unit) { free(reuse); free(rk); free(unit); return 2; }
+    for (int64_t slot = 0; slot < F; ++slot) {
+        int64_t u = frames[2 * slot], t = frames[2 * slot + 1];
+        for (int64_t s = 0; s < y_group_stride; ++s) kept_idx[slot * y_group_stride + s] = -1;
+        kept_count[slot] = 0;
+        if (u < 0) continue;
+        /* the group's tokens in time order */
+        int64_t n = 0, f0 = (t >= 0 && t < u) ? t : u, f1 = (t >= 0 && t < u) ? u : t;
+        for (int64_t p = 0; p < P; ++p) unit[n++] = f0 * P + p;
+        if (f1 >= 0) for (int64_t p = 0; p < P; ++p) unit[n++] = f1 * P + p;
+        if (mode == 0) {
+            for (int64_t k = 0; k < n; ++k)
+                if (!joint_is_rep(L, frames, unit[k])) reuse[unit[k]] = best_sim[unit[k]] >= thr;
+        } else {
+            int64_t m = 0;
+            for (int64_t k = 0; k < n; ++k)
+                if (!joint_is_rep(L, frames, unit[k])) { rk[m].sim = best_sim[unit[k]]; rk[m].u = k; ++m; }
+            qsort(rk, (size_t)m, sizeof(ocr_rank), rank_cmp);
+            int64_t want = t >= 0 ? n_reuse_pair : n_reuse_single;
+            if (want > m) want = m;
+            for (int64_t k = 0; k < want; ++k) reuse[unit[rk[k].u]] = 1;
+        }
+        int64_t pos = 0;
+        for (int64_t k = 0; k < n; ++k) {
+            int64_t i = unit[k];
+            if (reuse[i]) { slot_of[i] = -1; match_map[i] = best_idx[i]; continue; }
+            if (pos >= y_group_stride) { free(reuse); free(rk); free(unit); return 3; }
+            kept_idx[slot * y_group_stride + pos] = (int32_t)i;
+            slot_of[i] = (int32_t)(slot * y_group_stride + pos);
+            match_map[i] = (int32_t)i;
+            ++pos;
+        }
+        kept_count[slot] = (int32_t)pos;
+    }
+    free(reuse); free(rk); free(unit);
+    return 0;
+}
+
 /* ---- rows of a strided tensor --------------------------------------------------------------
  * A unit's row is n_seg segments of seg_bytes; segment s of unit i starts at byte
  *   (i / units_per_outer) * outer_pitch + (i % units_per_outer) * unit_pitch + s * seg_stride.

@@ -504,6 +504,150 @@ def test_select_invariants(oracle):
 
 
 # ---------------------------------------------------------------------------------------------
+# Token Cache on the frame pairs of Frame Cache (Section 3.2.3)
+# ---------------------------------------------------------------------------------------------
+def test_joint_groups_hand_cases(oracle):
+    """Which frames pair up, written out by hand for one clip of five frames (candidates 1 and 3)."""
+    ninf = -np.inf
+    def groups(sim1, idx1, so1, sim3, idx3, so3):
+        fs = np.array([ninf, sim1, ninf, sim3, ninf], np.float32)
+        fi = np.array([0, idx1, 2, idx3, 4], np.int32)
+        so = np.array([0, so1, 1, so3, 2], np.int32)
+        return oracle.joint_groups(1, 5, fs, fi, so).tolist()
+    # both candidates reused, different representatives
+    assert groups(0.9, 0, -1, 0.8, 4, -1) == [[0, 1], [-1, -1], [2, -1], [-1, -1], [4, 3]]
+    # both claim frame 2: the more similar one wins, the other stays a group of its own
+    assert groups(0.9, 2, -1, 0.8, 2, -1) == [[0, -1], [-1, -1], [2, 1], [3, -1], [4, -1]]
+    assert groups(0.7, 2, -1, 0.8, 2, -1) == [[0, -1], [1, -1], [2, 3], [-1, -1], [4, -1]]
+    assert groups(0.8, 2, -1, 0.8, 2, -1) == [[0, -1], [-1, -1], [2, 1], [3, -1], [4, -1]]   # equal: the earlier frame
+    # a candidate that Frame Cache keeps (slot >= 0) claims nothing
+    assert groups(0.9, 2, 3, 0.8, 2, -1) == [[0, -1], [1, -1], [2, 3], [-1, -1], [4, -1]]
+    assert groups(0.9, 0, 1, 0.8, 4, 3) == [[f, -1] for f in range(5)]
+    # two batch elements are independent
+    fs = np.array([ninf, 0.9, ninf, ninf, 0.5, ninf], np.float32)
+    fi = np.array([0, 2, 2, 3, 3, 5], np.int32)
+    so = np.array([0, -1, 1, 2, -1, 3], np.int32)
+    assert oracle.joint_groups(2, 3, fs, fi, so).tolist() == [[0, -1], [-1, -1], [2, 1], [3, 4], [-1, -1], [5, -1]]
+
+
+def np_joint(x64, frames, sy, sx, oy, ox):
+    """NumPy brute force of the joint match: per group normalised matrix product, row arg-max."""
+    B, T, Hh, W, Cc = x64.shape
+    P = Hh * W
+    tok = x64.reshape(B * T * P, Cc)
+    nrm = tok / np.maximum(np.linalg.norm(tok, axis=1, keepdims=True), 1e-8)
+    yy, xx = np.divmod(np.arange(P), W)
+    lat = (yy % sy == oy) & (xx % sx == ox)
+    best = np.full(B * T * P, -np.inf)
+    arg = np.arange(B * T * P)
+    is_rep = np.zeros(B * T * P, bool)
+    for slot, (u, t) in enumerate(frames):
+        if u < 0:
+            continue
+        reps = u * P + np.nonzero(lat)[0]
+        is_rep[reps] = True
+        cands = u * P + np.nonzero(~lat)[0]
+        if t >= 0:
+            cands = np.concatenate([cands, t * P + np.arange(P)])
+        sim = np.clip(nrm[cands] @ nrm[reps].T, -1, 1)
+        k = sim.argmax(axis=1)                      # first maximum = lowest representative index
+        best[cands] = sim[np.arange(cands.size), k]
+        arg[cands] = reps[k]
+    return best, arg, is_rep
+
+
+@pytest.mark.parametrize("lattice", [(2, 2, 0, 0), (2, 2, 1, 0), (1, 2, 0, 1)])
+def test_match_joint_bruteforce(oracle, lattice):
+    sy, sx, oy, ox = lattice
+    rng = np.random.default_rng(sum(lattice) + 11)
+    B, T, Hh, W, Cc = 2, 5, 4, 6, 16
+    xf = rng.standard_normal((B, T, Hh, W, Cc)).astype(np.float32)
+    xf[:, 1:] = 0.6 * xf[:, :-1] + 0.4 * xf[:, 1:]
+    x = inputs.to_bf16_bits(xf)
+    x64 = as_f64(x, inputs.BF16)
+    frames = np.array([[0, 1], [-1, -1], [2, -1], [3, -1], [4, -1],        # b = 0: (0,1) pair, 3 unmatched
+                       [5, -1], [-1, -1], [7, 6], [-1, -1], [9, 8]], np.int32)   # b = 1: pairs with t < u
+    L = oracle.Layout(0, oracle.DT_BF16, B, T, Hh, W, Cc, sy=sy, sx=sx, oy=oy, ox=ox)
+    got = oracle.match_joint(L, x, frames)
+    best, arg, is_rep = np_joint(x64, frames, sy, sx, oy, ox)
+    assert np.array_equal(np.isneginf(got["best_sim"]), is_rep)
+    assert np.array_equal(got["best_idx"][is_rep], np.nonzero(is_rep)[0])
+    c = ~is_rep
+    assert np.abs(got["best_sim"][c] - best[c]).max() < 1e-7
+    differ = np.nonzero(c & (got["best_idx"] != arg))[0]
+    for i in differ:       # float32 rounding of the NumPy product can reorder exact ties only
+        assert abs(best[i] - got["second_sim"][i]) < 1e-7
+
+
+def test_match_joint_reduces_to_token_cache_and_to_copies(oracle):
+    rng = np.random.default_rng(3)
+    B, T, Hh, W, Cc = 1, 4, 4, 4, 8
+    x = rng.standard_normal((B, T, Hh, W, Cc)).astype(np.float32)
+    L = oracle.Layout(0, 0, B, T, Hh, W, Cc)
+    # no pairs: every frame on its own = per-frame Token Cache
+    singles = np.array([[f, -1] for f in range(T)], np.int32)
+    a, b = oracle.match_joint(L, x, singles), oracle.match_token(L, x)
+    assert np.array_equal(a["best_sim"], b["best_sim"]) and np.array_equal(a["best_idx"], b["best_idx"])
+    s_a = oracle.select_joint(L, singles, a["best_sim"], a["best_idx"], 1, 0.0, 0, 5, 11)
+    s_b = oracle.select(L, b["best_sim"], b["best_idx"], 1, 0.0, 5, 11)
+    for k in ("kept_idx", "kept_count", "match_map", "slot_of"):
+        assert np.array_equal(s_a[k], s_b[k])
+    # frame 1 an exact copy of frame 0, paired: a copy of a lattice token matches that token with
+    # similarity 1; a copy of any other token has the same match as its original
+    x[0, 1] = x[0, 0]
+    frames = np.array([[0, 1], [-1, -1], [2, -1], [3, -1]], np.int32)
+    m = oracle.match_joint(L, x, frames)
+    P = Hh * W
+    yy, xx = np.divmod(np.arange(P), W)
+    lat = (yy % 2 == 0) & (xx % 2 == 0)
+    assert np.allclose(m["best_sim"][P + np.nonzero(lat)[0]], 1.0, atol=1e-7)
+    assert np.array_equal(m["best_idx"][P + np.nonzero(lat)[0]], np.nonzero(lat)[0])
+    assert np.array_equal(m["best_sim"][P + np.nonzero(~lat)[0]], m["best_sim"][np.nonzero(~lat)[0]])
+    assert np.array_equal(m["best_idx"][P + np.nonzero(~lat)[0]], m["best_idx"][np.nonzero(~lat)[0]])
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_select_joint_bruteforce_and_invariants(oracle, mode):
+    rng = np.random.default_rng(40 + mode)
+    B, T, Hh, W, Cc = 2, 5, 4, 6, 8
+    P = Hh * W
+    x = rng.standard_normal((B, T, Hh, W, Cc)).astype(np.float32)
+    frames = np.array([[0, 1], [-1, -1], [2, -1], [3, -1], [4, -1],
+                       [5, -1], [-1, -1], [7, 6], [-1, -1], [9, 8]], np.int32)
+    L = oracle.Layout(0, 0, B, T, Hh, W, Cc)
+    m = oracle.match_joint(L, x, frames)
+    bs = m["best_sim"].copy()
+    c = np.isfinite(bs)
+    bs[c] = np.round(bs[c] * 8) / 8                  # equal similarities: the index tie-break matters
+    for thr, n_pair, n_single in ((0.0, 20, 7), (0.125, 1, 0), (2.0, 0, 0), (-1.0, 42, 18), (0.25, 100, 100)):
+        stride = 2 * P
+        got = oracle.select_joint(L, frames, bs, m["best_idx"], mode, thr, n_pair, n_single, stride)
+        reused = got["slot_of"] < 0
+        for slot, (u, t) in enumerate(frames):
+            lo = slot * stride
+            if u < 0:
+                assert got["kept_count"][slot] == 0 and np.all(got["kept_idx"][lo:lo + stride] == -1)
+                continue
+            fr = sorted(f for f in (u, t) if f >= 0)
+            ids = np.concatenate([f * P + np.arange(P) for f in fr])         # time order = ascending index
+            cand = ids[np.isfinite(bs[ids])]
+            if mode == 0:
+                want = cand[bs[cand] >= np.float32(thr)]
+            else:
+                order = cand[np.lexsort((cand, -bs[cand].astype(np.float64)))]
+                want = order[:min(n_pair if t >= 0 else n_single, cand.size)]
+            assert set(ids[reused[ids]]) == set(want)
+            kept = ids[~reused[ids]]
+            n = kept.size
+            assert got["kept_count"][slot] == n
+            assert np.array_equal(got["kept_idx"][lo:lo + n], kept) and np.all(got["kept_idx"][lo + n:lo + stride] == -1)
+            assert np.array_equal(got["slot_of"][kept], lo + np.arange(n))
+            assert np.array_equal(got["match_map"][kept], kept)
+            assert np.array_equal(got["match_map"][ids[reused[ids]]], m["best_idx"][ids[reused[ids]]])
+            # a reused token's stand-in is a kept representative of its own group
+            assert np.all(~reused[got["match_map"][ids]]) and np.all(got["match_map"][ids[reused[ids]]] // P == u)
+
+
 # gather / restore
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("kind", [0, 1, 2])
