@@ -234,6 +234,42 @@ oc_status oc_match_frame_levels(oc_ctx* ctx, const oc_layout* layout, const void
                                 const int32_t* grids, float* best_sim, int32_t* best_idx, float* pos_sim,
                                 float* pair_sim, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Token Cache on the frame pairs of Frame Cache (Section 3.2.3): "Token Cache consumes the same
+ * feature map and frame-pair metadata used by Frame Cache"; matched pairs become token groups of
+ * 2*H*W tokens with one representative per 2x2x2 cube, unmatched frames keep their 2x2 groups.
+ * `layout` is the OC_KIND_TOKEN layout of the tensor (bf16, gy = gx = 1, no self_match;
+ * OC_ERR_UNSUPPORTED otherwise).  `frames` is a device array of B*T slots {rep, partner} (int32
+ * pairs, 8-byte aligned): slot f = {f, t} if frame f is the representative frame of the pair
+ * (f, t), {f, -1} if frame f is a group of its own, {-1, -1} if frame f was absorbed into its
+ * partner's group.
+ *
+ * oc_joint_groups: builds `frames` from a Frame Cache result on the same tensor (whole frames,
+ *   gy = gx = 1): a candidate frame t with frame_slot_of[t] < 0 (reused) claims the representative
+ *   frame_best_idx[t]; if both neighbours of a representative claim it, the one with the larger
+ *   frame_best_sim wins (equal: the earlier frame) and the other stays on its own.
+ * oc_match_joint: for every group, every candidate token against all representatives of the group
+ *   (the lattice tokens of the representative frame); candidates are the other tokens of that frame
+ *   and ALL tokens of the partner frame.  Outputs as oc_match (indexed by token).  One launch of
+ *   the tensor-core matcher over a device-side work list; needs oc_joint_workspace_bytes().
+ * oc_select_joint: as oc_select with one group per slot, a pair's units being the tokens of its two
+ *   frames in time order; n_reuse_pair / n_reuse_single are the count-mode budgets of the two kinds
+ *   of group; kept_idx is [B*T][y_stride] (absorbed slots keep nothing, kept_count 0), y_stride at
+ *   most 2*H*W and at least what either kind of group can keep; 2*H*W at most 40960.
+ * gather / restore then move token rows as for any Token Cache selection (n_slots = B*T*y_stride).
+ * Errors: as oc_match / oc_select.
+ * ------------------------------------------------------------------------------------------- */
+oc_status oc_joint_workspace_bytes(const oc_layout* layout, size_t* bytes);
+oc_status oc_joint_groups(oc_ctx* ctx, const oc_layout* layout, const float* frame_best_sim,
+                          const int32_t* frame_best_idx, const int32_t* frame_slot_of, int32_t* frames,
+                          void* stream);
+oc_status oc_match_joint(oc_ctx* ctx, const oc_layout* layout, const void* x, const int32_t* frames,
+                         float* best_sim, int32_t* best_idx, void* stream);
+oc_status oc_select_joint(oc_ctx* ctx, const oc_layout* layout, const int32_t* frames, const float* best_sim,
+                          const int32_t* best_idx, int mode, float thr, int64_t n_reuse_pair,
+                          int64_t n_reuse_single, int64_t y_stride, int32_t* kept_idx, int32_t* kept_count,
+                          int32_t* match_map, int32_t* slot_of, void* stream);
+
 /* select ("the r most redundant ... are marked for cached restoration while the retained
  * representatives are computed normally", Sections 3.2.1-3.2.3).  Representatives are always kept.
  *   mode OC_SELECT_THRESHOLD: a candidate is reused iff best_sim >= thr (self_match: and its best

@@ -104,6 +104,7 @@ GroupMap make_group_map(const Geo& g) {
     m.kind = g.kind; m.self_match = g.self_match; m.H = g.H; m.W = g.W; m.gy = g.gy; m.gx = g.gx;
     m.Hp = g.Hp; m.Wp = g.Wp; m.sy = g.sy; m.sx = g.sx; m.oy = g.oy; m.ox = g.ox;
     m.units_per_group = (int)g.units_per_group;
+    m.frames = nullptr; m.n_reuse_single = 0;
     return m;
 }
 
@@ -380,6 +381,74 @@ oc_status oc_match_frame_levels(oc_ctx* c, const oc_layout* layout, const void* 
     DeviceGuard guard(c->device);
     if (!guard.ok) return OC_ERR_CUDA;
     return launch_match_frame_levels(c, g, x, n_levels, grids, best_sim, best_idx, pos_sim, pair_sim, (cudaStream_t)stream);
+}
+
+// ---- Token Cache on the frame pairs of Frame Cache (Section 3.2.3) ---------------------------------
+static oc_status joint_geo(const oc_layout* layout, Geo* g) {
+    oc_status st = make_geo(layout, g);
+    if (st != OC_OK) return st;
+    if (g->kind != OC_KIND_TOKEN || g->self_match) return OC_ERR_INVALID_ARG;
+    if (g->gy != 1 || g->gx != 1 || g->dtype != OC_DTYPE_BF16) return OC_ERR_UNSUPPORTED;
+    return OC_OK;
+}
+
+oc_status oc_joint_workspace_bytes(const oc_layout* layout, size_t* bytes) {
+    if (!bytes) return OC_ERR_INVALID_ARG;
+    Geo g;
+    oc_status st = joint_geo(layout, &g);
+    if (st != OC_OK) return st;
+    *bytes = joint_workspace_bytes(g);
+    return OC_OK;
+}
+
+oc_status oc_joint_groups(oc_ctx* c, const oc_layout* layout, const float* frame_best_sim,
+                          const int32_t* frame_best_idx, const int32_t* frame_slot_of, int32_t* frames, void* stream) {
+    if (!c || !frame_best_sim || !frame_best_idx || !frame_slot_of || !frames) return OC_ERR_INVALID_ARG;
+    Geo g;
+    oc_status st = joint_geo(layout, &g);
+    if (st != OC_OK) return st;
+    if (((uintptr_t)frames & 7u) != 0) return OC_ERR_ALIGNMENT;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return OC_ERR_CUDA;
+    return launch_joint_groups(c, g.B, g.T, frame_best_sim, frame_best_idx, frame_slot_of, (int2*)frames, (cudaStream_t)stream);
+}
+
+oc_status oc_match_joint(oc_ctx* c, const oc_layout* layout, const void* x, const int32_t* frames, float* best_sim,
+                         int32_t* best_idx, void* stream) {
+    if (!c || !x || !frames || !best_sim || !best_idx) return OC_ERR_INVALID_ARG;
+    Geo g;
+    oc_status st = joint_geo(layout, &g);
+    if (st != OC_OK) return st;
+    if (misaligned(x) || ((uintptr_t)frames & 7u) != 0) return OC_ERR_ALIGNMENT;
+    if (joint_workspace_bytes(g) > c->workspace_bytes) return OC_ERR_WORKSPACE;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return OC_ERR_CUDA;
+    return launch_match_joint(c, g, x, (const int2*)frames, best_sim, best_idx, (cudaStream_t)stream);
+}
+
+oc_status oc_select_joint(oc_ctx* c, const oc_layout* layout, const int32_t* frames, const float* best_sim,
+                          const int32_t* best_idx, int mode, float thr, int64_t n_reuse_pair, int64_t n_reuse_single,
+                          int64_t y_stride, int32_t* kept_idx, int32_t* kept_count, int32_t* match_map,
+                          int32_t* slot_of, void* stream) {
+    if (!c || !frames || !best_sim || !best_idx || !kept_idx || !kept_count || !match_map || !slot_of)
+        return OC_ERR_INVALID_ARG;
+    if (mode != OC_SELECT_THRESHOLD && mode != OC_SELECT_COUNT) return OC_ERR_INVALID_ARG;
+    Geo g;
+    oc_status st = joint_geo(layout, &g);
+    if (st != OC_OK) return st;
+    const int64_t P = (int64_t)g.H * g.W;
+    if (n_reuse_pair < 0 || n_reuse_single < 0 || y_stride <= 0 || y_stride > 2 * P) return OC_ERR_INVALID_ARG;
+    // capacity: a pair keeps at least 2P - min(n_reuse_pair, 7P/4-ish candidates), a single frame P - ...
+    const int64_t cand_single = P - g.reps_per_group, cand_pair = 2 * P - g.reps_per_group;
+    const int64_t keep_pair = mode == OC_SELECT_COUNT ? 2 * P - (n_reuse_pair < cand_pair ? n_reuse_pair : cand_pair) : 2 * P;
+    const int64_t keep_single = mode == OC_SELECT_COUNT ? P - (n_reuse_single < cand_single ? n_reuse_single : cand_single) : P;
+    if (y_stride < keep_pair || y_stride < keep_single) return OC_ERR_INVALID_ARG;
+    if ((int64_t)g.B * g.T * y_stride > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
+    if (((uintptr_t)frames & 7u) != 0) return OC_ERR_ALIGNMENT;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return OC_ERR_CUDA;
+    return launch_select_joint(c, g, (const int2*)frames, best_sim, best_idx, mode, thr, n_reuse_pair, n_reuse_single,
+                               y_stride, kept_idx, kept_count, match_map, slot_of, (cudaStream_t)stream);
 }
 
 oc_status oc_select(oc_ctx* c, const oc_layout* layout, const float* best_sim, const int32_t* best_idx, int mode,

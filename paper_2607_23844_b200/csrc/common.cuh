@@ -119,6 +119,11 @@ struct GroupMap {
     int kind, self_match;
     int H, W, gy, gx, Hp, Wp, sy, sx, oy, ox;
     int units_per_group;
+    // Joint form (Token Cache on frame pairs, Section 3.2.3): group g is slot g of this table,
+    // {representative frame, partner frame or -1}, {-1, -1} for a frame absorbed into its partner's
+    // group; a pair's units are the tokens of its two frames in time order.  Null otherwise.
+    const int2* frames;
+    int n_reuse_single;                  // count-mode budget of a single-frame group (pairs take n_reuse)
 };
 GroupMap make_group_map(const Geo& g);
 
@@ -165,6 +170,17 @@ oc_status launch_match_token(oc_ctx*, const Geo&, const void* x, float* best_sim
                              float* aux_sim, cudaStream_t);
 // tcgen05 path of launch_match_token; returns OC_ERR_UNSUPPORTED if the shape is not covered.
 bool tc_match_supported(const Geo&);
+size_t joint_workspace_bytes(const Geo&);
+oc_status launch_joint_groups(oc_ctx*, int B, int T, const float* frame_best_sim, const int32_t* frame_best_idx,
+                              const int32_t* frame_slot_of, int2* frames, cudaStream_t);
+oc_status launch_match_joint(oc_ctx*, const Geo&, const void* x, const int2* frames, float* best_sim, int32_t* best_idx,
+                             cudaStream_t);
+oc_status launch_select_joint(oc_ctx*, const Geo&, const int2* frames, const float* best_sim, const int32_t* best_idx,
+                              int mode, float thr, int64_t n_reuse_pair, int64_t n_reuse_single, int64_t y_stride,
+                              int32_t* kept_idx, int32_t* kept_count, int32_t* match_map, int32_t* slot_of, cudaStream_t);
+bool tc_match_supported(const Geo&);
+oc_status launch_match_joint_tc(oc_ctx*, const Geo&, const void* x, const float* inv_norm, unsigned long long* keys,
+                                const int4* units, const int* n_units_dev, long long max_units, cudaStream_t);
 oc_status launch_match_token_tc(oc_ctx*, const Geo&, const void* x, const float* inv_norm,
                                 unsigned long long* keys, float* aux_sim, cudaStream_t);
 void tc_cache_free(oc_ctx*);

@@ -226,6 +226,16 @@ size_t match_workspace_bytes(const Geo& g) {
     return n * sizeof(unsigned long long) + ((n * sizeof(float) + 255) / 256) * 256 + 256;
 }
 
+// the pre-pass alone (also used by the joint frame-pair matcher)
+void launch_norms(oc_ctx* ctx, const Geo& g, const void* x, float* inv_norm, unsigned long long* keys, cudaStream_t s) {
+    const int cpr = g.C * g.elem_bytes / 16;
+    LaunchScope scope(ctx, OC_K_NORMS, s);
+    if (g.dtype == OC_DTYPE_BF16)
+        norms_dispatch<OC_DTYPE_BF16>(ctx->sm_count, s, (const uint8_t*)x, g.n_units, cpr, g.eps, inv_norm, keys);
+    else
+        norms_dispatch<OC_DTYPE_F32>(ctx->sm_count, s, (const uint8_t*)x, g.n_units, cpr, g.eps, inv_norm, keys);
+}
+
 oc_status launch_match_token(oc_ctx* ctx, const Geo& g, const void* x, float* best_sim, int32_t* best_idx,
                              float* aux_sim, cudaStream_t s) {
     const long long n_tok = g.n_units;

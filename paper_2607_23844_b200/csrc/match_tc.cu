@@ -102,6 +102,13 @@ struct TcScalars {
     int u_step_q, u_step_r;              // n_q_units / pieces_per_row and the remainder
     int n_stages, stage_bytes;           // operand ring of this launch
     int units_per_group, reps_per_group;
+    // Joint form (Token Cache on the frame pairs of Frame Cache, Section 3.2.3): the work is a list of
+    // units {representative frame, candidate frame, candidate sub-lattice member} written by another
+    // kernel, whose length is only known on the device; every walker derives its share from it.
+    const int4* units;                   // null: the regular (frame, patch, member) enumeration
+    const int* n_units_dev;
+    unsigned n_walkers;
+    float rcp_walkers;
     const float* inv_norm;
     unsigned long long* keys;
     float* aux;
@@ -285,7 +292,8 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
 
 // ---- the walk over this CTA's share of the piece list ----------------------------------------------
 struct Piece {
-    int bt, py, px, member;              // frame, patch, candidate sub-lattice member
+    int bt, py, px, member;              // frame (of the representatives), patch, candidate sub-lattice member
+    int bt_a;                            // frame of the candidates (differs from bt only in the joint form)
     int a_pair;                          // which run of candidate tiles (tpp per CTA) of the member's lattice
     int q0, nq;                          // quanta [q0, q0 + nq) of the group's representatives are fetched
     int c_off, ncol;                     // of which columns [c_off, c_off + ncol) are the piece (c_off is 0 or 16,
@@ -309,8 +317,30 @@ struct Walk {
     int left;                            // pieces still to hand out
     int j, a_pair, k, px, py, bt;
     int u_cur, r_cur;                    // floor(j * n_q_units / pieces_per_row) and the remainder
+    int bt_a, member_u;                  // joint form: the current unit's candidate frame and member
     long long g;
+    __device__ __forceinline__ void load_unit(const TcScalars& P) {
+        const int4 v = __ldg(P.units + g);
+        bt = v.x; bt_a = v.y; member_u = v.z;
+    }
     __device__ __forceinline__ Walk(const TcScalars& P, int c) {
+        if (P.units) {
+            // pieces are numbered (unit, tile run, piece of the row); the list length is read here
+            const unsigned total = (unsigned)__ldg(P.n_units_dev) * P.cum[1];
+            const unsigned base = div_small(total, P.n_walkers, P.rcp_walkers), rem = total - base * P.n_walkers;
+            const unsigned i0 = (unsigned)c * base + ((unsigned)c < rem ? (unsigned)c : rem);
+            left = (int)(base + ((unsigned)c < rem ? 1u : 0u));
+            const unsigned q0 = div_small(i0, P.cum[0], P.rcp_cum[0]), q1 = div_small(i0, P.cum[1], P.rcp_cum[1]);
+            j = (int)(i0 - q0 * P.cum[0]);
+            a_pair = (int)(q0 - q1 * (unsigned)P.n_apairs);
+            g = q1; k = 0; px = 0; py = 0; bt = 0; bt_a = 0; member_u = 0;
+            if (left > 0) load_unit(P);
+            const unsigned ju = (unsigned)j * (unsigned)P.n_q_units;
+            u_cur = (int)div_small(ju, (unsigned)P.pieces_per_row, P.rcp_ppr);
+            r_cur = (int)(ju - (unsigned)u_cur * (unsigned)P.pieces_per_row);
+            return;
+        }
+        bt_a = 0; member_u = 0;
         const unsigned i0 = (unsigned)(c * P.items_base + (c < P.items_rem ? c : P.items_rem));
         left = P.items_base + (c < P.items_rem ? 1 : 0);
         const unsigned q0 = div_small(i0, P.cum[0], P.rcp_cum[0]), q1 = div_small(i0, P.cum[1], P.rcp_cum[1]),
@@ -345,12 +375,16 @@ struct Walk {
         }
         u_cur = u_next; r_cur = r_next;
         p.a_pair = a_pair; p.g = g; p.px = px; p.py = py; p.bt = bt;
-        p.member = k < P.rep_member ? k : k + 1;
+        p.bt_a = P.units ? bt_a : bt;
+        p.member = P.units ? member_u : (k < P.rep_member ? k : k + 1);
         if (++j == P.pieces_per_row) {
             j = 0; u_cur = 0; r_cur = 0;
             if (++a_pair == P.n_apairs) {
                 a_pair = 0;
-                if (++k == P.n_cand_lat) {
+                if (P.units) {
+                    ++g;
+                    if (left > 0) load_unit(P);
+                } else if (++k == P.n_cand_lat) {
                     k = 0; ++g;
                     if (++px == P.gx) { px = 0; if (++py == P.gy) { py = 0; ++bt; } }
                 }
@@ -420,7 +454,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         tma_prefetch_map(&KP.mapQ[0]);
         tma_prefetch_map(&KP.mapQ[1]);
         for (int m = 0; m <= KP.s.n_cand_lat; ++m)
-            if (m != KP.s.rep_member) tma_prefetch_map(&KP.mapsA[m]);
+            if (m != KP.s.rep_member || KP.s.units) tma_prefetch_map(&KP.mapsA[m]);
     }
     if (warp == 1) {
         if (PAIR) {
@@ -448,6 +482,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     const int STAGES = P.n_stages, STAGE_BYTES = P.stage_bytes;
     const bool dbl = P.tpp == 1;
 
+    // (the joint form's work list is written by a kernel earlier in the stream: wait for it)
+    if (P.units) pdl_wait();
     Walk walk(P, walker);                  // every role walks the same pieces
     Piece c;
     const int bwA = 1 << P.bwA_log2, bwQ = 1 << P.bwQ_log2;
@@ -496,7 +532,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 }
                 go = __shfl_sync(0xFFFFFFFFu, (int)go, 0) != 0;
                 if (!go) { ok = false; break; }
-                if (active) tma_load_4d<PAIR>(tiles_base + stage * STAGE_BYTES + dst_off, map, kb * BK, w, h, c.bt, full);
+                if (active) tma_load_4d<PAIR>(tiles_base + stage * STAGE_BYTES + dst_off, map, kb * BK, w, h, lane < nA ? c.bt_a : c.bt, full);
                 armed |= 1u << stage;
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 if (!joined) { __syncthreads(); joined = true; }   // first stage on its way: meet the others
@@ -621,7 +657,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 const int hsA = htA * P.bhA + rowh, wsA = wtA * bwA + roww;
                 row_ok0 = hsA < P.Hs && wsA < P.Ws;
                 const int yA = (c.py * P.Hs + hsA) * P.sy + my, xA = (c.px * P.Ws + wsA) * P.sx + mx;
-                tokA0 = ((long long)c.bt * P.H + yA) * P.W + xA;
+                tokA0 = ((long long)c.bt_a * P.H + yA) * P.W + xA;
             }
             {
                 const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + 1;
@@ -629,7 +665,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 const int hsA = htA * P.bhA + rowh, wsA = wtA * bwA + roww;
                 row_ok1 = P.tpp == 2 && hsA < P.Hs && wsA < P.Ws;
                 const int yA = (c.py * P.Hs + hsA) * P.sy + my, xA = (c.px * P.Ws + wsA) * P.sx + mx;
-                tokA1 = ((long long)c.bt * P.H + yA) * P.W + xA;
+                tokA1 = ((long long)c.bt_a * P.H + yA) * P.W + xA;
             }
             // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
             const int n_ch = (c.ncol + 31) >> 5;                        // (a last half chunk reads 16 columns of
@@ -932,8 +968,25 @@ bool tc_match_supported(const Geo& g) {
 
 void tc_cache_free(oc_ctx*) {}
 
+static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm, unsigned long long* keys,
+                           float* aux_sim, const int4* units, const int* n_units_dev, long long max_units, cudaStream_t s);
+
 oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm,
                                 unsigned long long* keys, float* aux_sim, cudaStream_t s) {
+    return launch_tc(ctx, g, x, inv_norm, keys, aux_sim, nullptr, nullptr, 0, s);
+}
+
+// Joint form: `units` (device) lists {representative frame, candidate frame, member} triples, `n_units_dev`
+// (device) how many; max_units bounds the list (it sizes the launch).  g: one patch per frame.
+oc_status launch_match_joint_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm,
+                                unsigned long long* keys, const int4* units, const int* n_units_dev,
+                                long long max_units, cudaStream_t s) {
+    if (g.gy != 1 || g.gx != 1 || !units || !n_units_dev || max_units <= 0) return OC_ERR_UNSUPPORTED;
+    return launch_tc(ctx, g, x, inv_norm, keys, nullptr, units, n_units_dev, max_units, s);
+}
+
+static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm, unsigned long long* keys,
+                           float* aux_sim, const int4* units, const int* n_units_dev, long long max_units, cudaStream_t s) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return OC_ERR_UNSUPPORTED;
     // once per process: opt in to the large dynamic shared memory, and ask how many CTA pairs fit
@@ -988,7 +1041,7 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
     for (int m = 0; m < n_members + 2; ++m) {
         const bool quantum_map = m >= n_members;
         const int member = quantum_map ? rep_member : m;
-        if (!quantum_map && member == rep_member) continue;              // representatives are never candidates
+        if (!quantum_map && member == rep_member && !units) continue;    // representatives are candidates only across frames
         const int my = member / g.sx, mx = member - my * g.sx;
         void* base = (uint8_t*)x + ((size_t)my * g.W + mx) * g.C * 2;
         CUresult r = enc(quantum_map ? &KP.mapQ[m - n_members] : &KP.mapsA[m], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base,
@@ -1014,11 +1067,14 @@ oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const 
         if (cudaMemsetAsync(P.span, 0, 2 * sizeof(unsigned long long), s) != cudaSuccess) return OC_ERR_CUDA;
     }
     // one walker (CTA or CTA pair) per SM (pair of SMs), or one per piece when there are fewer pieces
-    long long walkers = p.items;
+    P.units = units; P.n_units_dev = n_units_dev;
+    long long walkers = units ? max_units * (long long)p.pieces_per_row * p.n_apairs : p.items;
     const int cap = p.pair ? pair_walkers : ctx->sm_count;
     if (walkers > cap) walkers = cap;
     if (walkers < 1) walkers = 1;
     P.items_base = (int)(p.items / walkers); P.items_rem = (int)(p.items % walkers);
+    P.n_walkers = (unsigned)walkers; P.rcp_walkers = 1.0f / (float)walkers;
+    if (units && max_units * (long long)p.pieces_per_row * p.n_apairs > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
     P.cum[0] = (unsigned)p.pieces_per_row; P.cum[1] = P.cum[0] * (unsigned)p.n_apairs;
     P.cum[2] = P.cum[1] * (unsigned)P.n_cand_lat; P.cum[3] = P.cum[2] * (unsigned)g.gx; P.cum[4] = P.cum[3] * (unsigned)g.gy;
     P.u_step_q = p.n_q_units / p.pieces_per_row; P.u_step_r = p.n_q_units % p.pieces_per_row;

@@ -33,8 +33,19 @@ struct GroupView {
     int w_shift;        // log2(w_local) if it is a power of two, else -1
     int lat_pow2;       // sy and sx are both powers of two
     int contig;         // local units are equally spaced in unit order (FRAME; patches as wide as the frame)
+    long long base1;    // joint form: global index of the second frame's first token
+    int frame_units;    // joint form: tokens per frame (0 otherwise)
+    int rep_half;       // joint form: which of the two frames holds the representatives
     __device__ GroupView(const GroupMap& m, long long g) {
-        if (m.kind != OC_KIND_FRAME) {                  // TOKEN: bt = frame; BLOCK: bt = batch element
+        base1 = 0; frame_units = 0; rep_half = 0;
+        if (m.frames) {                                 // one or two whole frames, in time order
+            const int2 fr = m.frames[g];
+            const int f0 = (fr.y >= 0 && fr.y < fr.x) ? fr.y : fr.x, f1 = (fr.y >= 0 && fr.y < fr.x) ? fr.x : fr.y;
+            frame_units = m.H * m.W;
+            base = (long long)f0 * frame_units; base1 = (long long)f1 * frame_units;
+            rep_half = fr.x == f0 ? 0 : 1;
+            unit_stride = 1; row_pitch = m.W; w_local = m.W;
+        } else if (m.kind != OC_KIND_FRAME) {                  // TOKEN: bt = frame; BLOCK: bt = batch element
             const int px = (int)(g % m.gx), py = (int)((g / m.gx) % m.gy);
             const long long bt = g / ((long long)m.gx * m.gy);
             base = (bt * m.H + (long long)py * m.Hp) * m.W + (long long)px * m.Wp;
@@ -57,11 +68,17 @@ struct GroupView {
         else { ly = u / w_local; lx = u - ly * w_local; }
     }
     __device__ __forceinline__ long long index(const GroupMap& m, int u) const {
+        if (frame_units && u >= frame_units) return base1 + (u - frame_units);
         if (contig) return base + (long long)u * unit_stride;
         int ly, lx; split(u, ly, lx);
         return base + (long long)ly * row_pitch + lx;
     }
     __device__ __forceinline__ bool is_cand(const GroupMap& m, int u) const {
+        if (frame_units) {                              // every token of the partner frame is a candidate
+            const int half = u >= frame_units ? 1 : 0;
+            if (half != rep_half) return true;
+            u -= half * frame_units;
+        }
         if (m.kind == OC_KIND_FRAME) return (u & 1) != 0;
         if (m.self_match) return true;
         int ly, lx; split(u, ly, lx);
@@ -302,9 +319,18 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     __shared__ unsigned sh_kmin, sh_kmax;
 
     const int NT = (int)blockDim.x;                             // 128..1024 threads, chosen by the host for the group size
-    const int U = gm.units_per_group;
+    int U = gm.units_per_group;
     const long long g = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31;
+    if (gm.frames) {                                            // joint form: the slot decides the group's size and budget
+        const int2 fr = gm.frames[g];
+        if (fr.x < 0) {                                         // absorbed into its partner's group: keeps nothing
+            for (int p = tid; p < y_stride; p += NT) kept_idx[g * y_stride + p] = -1;
+            if (tid == 0) kept_count[g] = 0;
+            return;
+        }
+        if (fr.y < 0) { U = gm.H * gm.W; n_reuse = gm.n_reuse_single; }
+    }
     const int n_rounds = (U + NT - 1) / NT;
     const GroupView gv(gm, g);
 
@@ -591,6 +617,33 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
         OC_LAUNCH(select_general_kernel, (unsigned)geo.n_groups, SEL_THREADS, dyn, s, gm, best_sim, best_idx, mode, thr, nr,
                   (int)y_stride, keys_in_smem, kept_idx, kept_count, match_map, slot_of);
     }
+    return last_launch_status();
+}
+
+// Joint form: one CTA per frame slot; pairs are groups of 2*H*W tokens, single frames of H*W.
+oc_status launch_select_joint(oc_ctx* ctx, const Geo& geo, const int2* frames, const float* best_sim,
+                              const int32_t* best_idx, int mode, float thr, int64_t n_reuse_pair,
+                              int64_t n_reuse_single, int64_t y_stride, int32_t* kept_idx, int32_t* kept_count,
+                              int32_t* match_map, int32_t* slot_of, cudaStream_t s) {
+    const long long P = (long long)geo.H * geo.W, slots = (long long)geo.B * geo.T;
+    if (geo.kind != OC_KIND_TOKEN || geo.self_match || geo.gy != 1 || geo.gx != 1) return OC_ERR_UNSUPPORTED;
+    if (2 * P > SEL_SMEM_KEYS) return OC_ERR_UNSUPPORTED;
+    if (slots == 0) return OC_OK;
+    GroupMap gm = make_group_map(geo);
+    gm.frames = frames;
+    gm.units_per_group = (int)(2 * P);
+    gm.n_reuse_single = (int)(n_reuse_single > 0x7FFFFFFF ? 0x7FFFFFFF : n_reuse_single);
+    const int nr = (int)(n_reuse_pair > 0x7FFFFFFF ? 0x7FFFFFFF : n_reuse_pair);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(select_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess)
+            return OC_ERR_CUDA;
+        attr_set = true;
+    }
+    LaunchScope scope(ctx, OC_K_SELECT, s);
+    OC_LAUNCH(select_fast_kernel, (unsigned)slots, SEL_THREADS, (size_t)(2 * P) * sizeof(unsigned), s,
+              gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);
     return last_launch_status();
 }
 

@@ -33,7 +33,7 @@ EXPORTS = (
     "oc_profile_captured_read", "oc_match", "oc_match_frame_levels",
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
     "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
-    "oc_schedule_propose",
+    "oc_schedule_propose", "oc_joint_workspace_bytes", "oc_joint_groups", "oc_match_joint", "oc_select_joint",
 )
 
 
@@ -79,6 +79,10 @@ _lib.oc_profile_captured_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_match.argtypes = [_vp] * 8
 _lib.oc_match_frame_levels.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.oc_select.argtypes = [_vp, _vp, _vp, _vp, _i, _f, _i64, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.oc_joint_workspace_bytes.argtypes = [_vp, _vp]
+_lib.oc_joint_groups.argtypes = [_vp] * 7
+_lib.oc_match_joint.argtypes = [_vp] * 7
+_lib.oc_select_joint.argtypes = [_vp, _vp, _vp, _vp, _vp, _i, _f, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp]
 _lib.oc_gather.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp]
 _lib.oc_restore.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _i, _vp]
 _lib.oc_layer_cache_put.argtypes = [_vp, _i, _i, _vp, C.c_size_t, _vp]
@@ -178,6 +182,13 @@ def match_workspace_bytes(layout: Layout) -> int:
     cl = layout.c()
     n = C.c_size_t()
     _chk(_lib.oc_match_workspace_bytes(C.byref(cl), C.byref(n)), "oc_match_workspace_bytes")
+    return n.value
+
+
+def joint_workspace_bytes(layout: Layout) -> int:
+    cl = layout.c()
+    n = C.c_size_t()
+    _chk(_lib.oc_joint_workspace_bytes(C.byref(cl), C.byref(n)), "oc_joint_workspace_bytes")
     return n.value
 
 
@@ -309,6 +320,34 @@ class Context:
                            _ptr(pair_sim), _stream(stream))
         if check:
             _chk(st, "oc_match")
+        return st
+
+    def joint_groups(self, layout: Layout, frame_best_sim, frame_best_idx, frame_slot_of, frames, stream=None,
+                     check: bool = True) -> int:
+        cl = layout.c()
+        st = _lib.oc_joint_groups(self._h, C.byref(cl), _ptr(frame_best_sim), _ptr(frame_best_idx),
+                                  _ptr(frame_slot_of), _ptr(frames), _stream(stream))
+        if check:
+            _chk(st, "oc_joint_groups")
+        return st
+
+    def match_joint(self, layout: Layout, x, frames, best_sim, best_idx, stream=None, check: bool = True) -> int:
+        cl = layout.c()
+        st = _lib.oc_match_joint(self._h, C.byref(cl), _ptr(x), _ptr(frames), _ptr(best_sim), _ptr(best_idx),
+                                 _stream(stream))
+        if check:
+            _chk(st, "oc_match_joint")
+        return st
+
+    def select_joint(self, layout: Layout, frames, best_sim, best_idx, mode: int, thr: float, n_reuse_pair: int,
+                     n_reuse_single: int, y_stride: int, kept_idx, kept_count, match_map, slot_of, stream=None,
+                     check: bool = True) -> int:
+        cl = layout.c()
+        st = _lib.oc_select_joint(self._h, C.byref(cl), _ptr(frames), _ptr(best_sim), _ptr(best_idx), mode, thr,
+                                  n_reuse_pair, n_reuse_single, y_stride, _ptr(kept_idx), _ptr(kept_count),
+                                  _ptr(match_map), _ptr(slot_of), _stream(stream))
+        if check:
+            _chk(st, "oc_select_joint")
         return st
 
     def match_frame_levels(self, layout: Layout, x, grids, best_sim, best_idx, pos_sim=None, pair_sim=None,

@@ -124,6 +124,10 @@ def test_null_context_and_bad_arguments_are_rejected_before_any_launch(oc):
     assert lib.oc_match(None, C.byref(L), one, one, one, None, None, None) == oc.ERR_INVALID_ARG
     assert lib.oc_match_frame_levels(None, C.byref(L), one, 1, one, one, one, None, None, None) == oc.ERR_INVALID_ARG
     assert lib.oc_select(None, C.byref(L), one, one, 0, 0.5, 0, 64, one, one, one, one, None) == oc.ERR_INVALID_ARG
+    assert lib.oc_joint_groups(None, C.byref(L), one, one, one, one, None) == oc.ERR_INVALID_ARG
+    assert lib.oc_match_joint(None, C.byref(L), one, one, one, one, None) == oc.ERR_INVALID_ARG
+    assert lib.oc_select_joint(None, C.byref(L), one, one, one, 0, 0.5, 0, 0, 64, one, one, one, one, None) == oc.ERR_INVALID_ARG
+    assert lib.oc_joint_workspace_bytes(C.byref(L), None) == oc.ERR_INVALID_ARG
     assert lib.oc_gather(None, C.byref(rows), one, one, 4, one, None) == oc.ERR_INVALID_ARG
     assert lib.oc_restore(None, C.byref(rows), one, one, 4, one, one, one, 0, None) == oc.ERR_INVALID_ARG
     assert lib.oc_layer_cache_put(None, 0, 0, one, 16, None) == oc.ERR_INVALID_ARG

@@ -348,6 +348,144 @@ def test_block_patches_chain(oc, oracle, grid, mode):
         assert rep["reused"] == 7 * grid[0] * grid[1]
 
 
+# ---------------------------------------------------------------------------------------------------
+# Token Cache on the frame pairs of Frame Cache (Section 3.2.3)
+# ---------------------------------------------------------------------------------------------------
+def _joint_case(oc, oracle, x_np, shape, frames_np, mode, thr, n_pair, n_single, lattice=(2, 2, 0, 0)):
+    """match_joint -> select_joint -> gather -> restore on a given frame table, each against the oracle."""
+    B, T, Hh, W, C = shape
+    P = Hh * W
+    sy, sx, oy, ox = lattice
+    L = oc.Layout(oc.KIND_TOKEN, oc.DTYPE_BF16, *shape, sy=sy, sx=sx, oy=oy, ox=ox)
+    Lo = oracle.Layout(0, oracle.DT_BF16, *shape, sy=sy, sx=sx, oy=oy, ox=ox)
+    n = B * T * P
+    x_dev, fr_dev = H.to_dev(x_np), H.to_dev(frames_np)
+    with oc.Context(0, oc.joint_workspace_bytes(L)) as ctx:
+        bs = torch.full((n,), float("nan"), device="cuda")
+        bi = torch.full((n,), -2, device="cuda", dtype=torch.int32)
+        ctx.match_joint(L, x_dev, fr_dev, bs, bi)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == oc.OK
+        ref = oracle.match_joint(Lo, x_np, frames_np)
+        gs, gi = bs.cpu().numpy(), bi.cpu().numpy()
+        H.check_match_against_oracle(oracle, Lo, x_np, gs, gi, ref, TOL[inputs.BF16])
+        # selection on the GPU's own similarities: exact against the oracle given the same arrays
+        stride = 2 * P if mode == oc.SELECT_THRESHOLD else max(2 * P - min(n_pair, 2 * P - P // (sy * sx)),
+                                                                P - min(n_single, P - P // (sy * sx)))
+        F = B * T
+        kept = torch.full((F * stride,), -9, device="cuda", dtype=torch.int32)
+        cnt = torch.full((F,), -9, device="cuda", dtype=torch.int32)
+        mm = torch.full((n,), -9, device="cuda", dtype=torch.int32)
+        so = torch.full((n,), -9, device="cuda", dtype=torch.int32)
+        ctx.select_joint(L, fr_dev, bs, bi, mode, thr, n_pair, n_single, stride, kept, cnt, mm, so)
+        torch.cuda.synchronize()
+        ref_s = oracle.select_joint(Lo, frames_np, gs, gi, mode, thr, n_pair, n_single, stride)
+        for k, t in (("kept_idx", kept), ("kept_count", cnt), ("match_map", mm), ("slot_of", so)):
+            assert np.array_equal(t.cpu().numpy(), ref_s[k]), k
+        # rows: plain token rows
+        Ro = oracle.rows_for(Lo, C, 2)
+        y = torch.full((F * stride, Ro.row_bytes), 0xAB, device="cuda", dtype=torch.uint8)
+        ctx.gather(H.crows(oc, Ro), x_dev, kept, F * stride, y)
+        assert H.dev_bytes(y) == oracle.gather(Ro, x_np, ref_s["kept_idx"], fill=0xAB).tobytes()
+        z_np = inputs.random_rows(5, (F * stride * C,), inputs.BF16)
+        cache_np = inputs.random_rows(6, shape, inputs.BF16)
+        for src_mode in (oc.RESTORE_FROM_CACHE, oc.RESTORE_FROM_REPRESENTATIVE):
+            out = torch.full((cache_np.nbytes,), 0xCD, device="cuda", dtype=torch.uint8)
+            ctx.restore(H.crows(oc, Ro), H.to_dev(z_np), H.to_dev(cache_np), n, so, mm, out, src_mode)
+            want = oracle.restore(Ro, z_np, cache_np, n, ref_s["slot_of"], ref_s["match_map"], src_mode)
+            assert H.dev_bytes(out) == want.tobytes()
+        assert ctx.device_status() == oc.OK
+        return int((ref_s["slot_of"] < 0).sum())
+
+
+@pytest.mark.parametrize("shape,lattice", [((2, 5, 16, 16, 64), (2, 2, 0, 0)), ((1, 6, 12, 24, 72), (2, 2, 1, 0)),
+                                           ((1, 4, 24, 16, 136), (2, 2, 1, 1)), ((2, 3, 8, 32, 40), (2, 2, 0, 1))])
+@pytest.mark.parametrize("mode", ["count", "threshold"])
+def test_joint_token_cache_on_given_frame_tables(oc, oracle, shape, lattice, mode):
+    B, T, Hh, W, C = shape
+    rng = np.random.default_rng(sum(shape))
+    x = np.stack([inputs.ar1_frames(rng, inputs.smooth_field(rng, Hh, W, C, 4.0), T, 0.9) for _ in range(B)])
+    x_np = inputs.to_bf16_bits(np.ascontiguousarray(x.reshape(shape), dtype=np.float32))
+    # every kind of slot: pairs with the partner after and before, unmatched frames, absorbed frames
+    frames = np.array([[f, -1] for f in range(B * T)], np.int32)
+    for b in range(B):
+        o = b * T
+        if b % 2 == 0:
+            frames[o] = (o, o + 1); frames[o + 1] = (-1, -1)            # (0, 1)
+        elif T >= 3:
+            frames[o + 2] = (o + 2, o + 1); frames[o + 1] = (-1, -1)    # (2, 1): partner earlier
+        if T >= 5:
+            frames[o + 4] = (o + 4, o + 3); frames[o + 3] = (-1, -1)
+    P = Hh * W
+    reused = _joint_case(oc, oracle, x_np, shape, frames, oc.SELECT_COUNT if mode == "count" else oc.SELECT_THRESHOLD,
+                         0.97, P // 2 + 3, P // 4 + 1, lattice)
+    assert reused > 0
+
+
+@pytest.mark.parametrize("plan", [None, "0,1,1", "0,2,2", "1,1,1", "1,2,2", "0,2,3"])
+def test_joint_token_cache_svd_level_shapes_every_plan(oc, oracle, plan, monkeypatch):
+    """Several candidate tiles per lattice member, every form of the tensor-core matcher (single CTA / CTA
+    pair, one or two tiles, several pieces per row) on the joint work list."""
+    if plan:
+        monkeypatch.setenv("OC_TC_PLAN", plan)
+    shape = (1, 7, 36, 64, 128)                     # 2304 tokens per frame: 576 per sub-lattice = 4.5 tiles
+    B, T, Hh, W, C = shape
+    rng = np.random.default_rng(17)
+    x = inputs.ar1_frames(rng, inputs.smooth_field(rng, Hh, W, C, 6.0), T, 0.9).reshape(shape)
+    x_np = inputs.to_bf16_bits(np.ascontiguousarray(x, dtype=np.float32))
+    frames = np.array([[0, 1], [-1, -1], [2, -1], [-1, -1], [4, 3], [5, -1], [6, -1]], np.int32)
+    P = Hh * W
+    reused = _joint_case(oc, oracle, x_np, shape, frames, oc.SELECT_COUNT, 0.0, P, P // 3)
+    assert reused == 2 * P + 3 * (P // 3)
+
+
+def test_joint_groups_from_frame_cache_and_full_chain(oc, oracle):
+    """Frame Cache decides the pairs (on the GPU), Token Cache works on them: the whole joint path."""
+    shape = (2, 7, 16, 16, 64)
+    B, T, Hh, W, C = shape
+    rng = np.random.default_rng(5)
+    x = np.stack([inputs.ar1_frames(rng, inputs.smooth_field(rng, Hh, W, C, 4.0), T, 0.93) for _ in range(B)])
+    x_np = inputs.to_bf16_bits(np.ascontiguousarray(x.reshape(shape), dtype=np.float32))
+    Lf = oc.Layout(oc.KIND_FRAME, oc.DTYPE_BF16, *shape)
+    Lfo = oracle.Layout(1, oracle.DT_BF16, *shape)
+    Lt = oc.Layout(oc.KIND_TOKEN, oc.DTYPE_BF16, *shape)
+    x_dev = H.to_dev(x_np)
+    with oc.Context(0, max(oc.match_workspace_bytes(Lf), oc.joint_workspace_bytes(Lt))) as ctx:
+        m = H.gpu_match(oc, ctx, Lf, x_dev)
+        fs = m["best_sim"].cpu().numpy()
+        thr = float(np.median(fs[np.isfinite(fs)]))                    # about half of the candidate frames reused
+        s = H.gpu_select(oc, ctx, Lf, m["best_sim"], m["best_idx"], oc.SELECT_THRESHOLD, thr, 0, T)
+        frames = torch.full((B * T, 2), -9, device="cuda", dtype=torch.int32)
+        ctx.joint_groups(Lt, m["best_sim"], m["best_idx"], s["slot_of"], frames)
+        torch.cuda.synchronize()
+        want = oracle.joint_groups(B, T, fs, m["best_idx"].cpu().numpy(), s["slot_of"].cpu().numpy())
+        assert np.array_equal(frames.cpu().numpy(), want)
+        assert (want[:, 1] >= 0).sum() >= 1 and (want[:, 0] < 0).sum() == (want[:, 1] >= 0).sum()
+    _joint_case(oc, oracle, x_np, shape, want, oc.SELECT_COUNT, 0.0, 200, 60)
+
+
+def test_joint_groups_conflicts_and_ties(oc, oracle):
+    """Random Frame Cache outcomes, many of them with both neighbours claiming the same frame."""
+    rng = np.random.default_rng(9)
+    Lt = oc.Layout(oc.KIND_TOKEN, oc.DTYPE_BF16, 3, 9, 4, 4, 8)
+    B, T = 3, 9
+    with oc.Context(0, 0) as ctx:
+        for trial in range(20):
+            fs = np.full(B * T, -np.inf, np.float32)
+            fi = np.arange(B * T, dtype=np.int32)
+            so = np.arange(B * T, dtype=np.int32)
+            for b in range(B):
+                for t in range(1, T, 2):
+                    f = b * T + t
+                    fs[f] = np.float32(rng.integers(0, 4)) / 4          # few distinct values: ties
+                    fi[f] = f + (1 if (t + 1 < T and rng.random() < 0.5) else -1)
+                    so[f] = -1 if rng.random() < 0.7 else 5
+            frames = torch.full((B * T, 2), -9, device="cuda", dtype=torch.int32)
+            ctx.joint_groups(Lt, H.to_dev(fs), H.to_dev(fi), H.to_dev(so), frames)
+            torch.cuda.synchronize()
+            assert np.array_equal(frames.cpu().numpy(), oracle.joint_groups(B, T, fs, fi, so)), trial
+
+
 def test_config2_sd3_token_cache_full(oc, oracle):
     w = inputs.sd3_token_cache()
     rep = run_chain(oc, oracle, w, full_oracle=True)
