@@ -753,6 +753,119 @@ def _token_groups_one(args, oc, torch, dev, peaks, graph_time_us, label, base, g
 
 
 
+def run_joint(args):
+    """Token Cache on the frame pairs of Frame Cache (Section 3.2.3) on the SVD levels: per-op device time."""
+    import torch
+    from paper_2607_23844_b200 import build
+    build.build()
+    from paper_2607_23844_b200 import omnicache as oc
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+
+    def graph_time_us(fn, reps):
+        fn(); torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        g.replay(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record(); torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / reps
+
+    results = []
+    reps = max(3, args.steps // 10)
+    for lv in (0, 1, 2):
+        base = make_workload(f"svd_token_l{lv}")
+        B, T, Hh, W, C = base.shape
+        P = Hh * W
+        tensor_bytes = int(np.prod(base.shape)) * 2
+        ring = max(2, -(-4 * L2_BYTES // (3 * tensor_bytes)))
+        xs = [torch.from_numpy(base.x.view(np.int16)).to(dev) for _ in range(ring)]
+        caches = [torch.empty_like(xs[0]) for _ in range(ring)]
+        outs = [torch.empty_like(xs[0]) for _ in range(ring)]
+        Lf = oc.Layout(oc.KIND_FRAME, inputs.BF16, *base.shape)
+        Lt = oc.Layout(oc.KIND_TOKEN, inputs.BF16, *base.shape)
+        F, n = B * T, B * T * P
+        ctx = oc.Context(0, max(oc.match_workspace_bytes(Lf), oc.joint_workspace_bytes(Lt), oc.match_workspace_bytes(Lt)))
+        fsim = torch.empty(F, dtype=torch.float32, device=dev); fidx = torch.empty(F, dtype=torch.int32, device=dev)
+        fk = torch.empty(F, dtype=torch.int32, device=dev); fc = torch.empty(B, dtype=torch.int32, device=dev)
+        fmm = torch.empty(F, dtype=torch.int32, device=dev); fso = torch.empty(F, dtype=torch.int32, device=dev)
+        frames = torch.empty((F, 2), dtype=torch.int32, device=dev)
+        ctx.match(Lf, xs[0], fsim, fidx)
+        torch.cuda.synchronize()
+        v = fsim.cpu().numpy()
+        thr = float(np.median(v[np.isfinite(v)]))                      # about half of the candidate frames reused
+        # keep half of each group's candidates
+        n_pair, n_single = (2 * P - P // 4) // 2, (P - P // 4) // 2
+        stride = max(2 * P - n_pair, P - n_single)
+        sims = [torch.empty(n, dtype=torch.float32, device=dev) for _ in range(ring)]
+        idxs = [torch.empty(n, dtype=torch.int32, device=dev) for _ in range(ring)]
+        kept = [torch.empty(F * stride, dtype=torch.int32, device=dev) for _ in range(ring)]
+        cnt = [torch.empty(F, dtype=torch.int32, device=dev) for _ in range(ring)]
+        mm = [torch.empty(n, dtype=torch.int32, device=dev) for _ in range(ring)]
+        so = [torch.empty(n, dtype=torch.int32, device=dev) for _ in range(ring)]
+        rows = oc.rows_from_layout(Lt, C, 2)
+        ys = [torch.empty(F * stride * C * 2, dtype=torch.uint8, device=dev) for _ in range(ring)]
+        cur = torch.cuda.current_stream
+
+        def f_frame():
+            for r in range(ring):
+                ctx.match(Lf, xs[r], fsim, fidx, stream=cur())
+                ctx.select(Lf, fsim, fidx, oc.SELECT_THRESHOLD, thr, 0, T, fk, fc, fmm, fso, stream=cur())
+                ctx.joint_groups(Lt, fsim, fidx, fso, frames, stream=cur())
+
+        def f_match():
+            for r in range(ring):
+                ctx.match_joint(Lt, xs[r], frames, sims[r], idxs[r], stream=cur())
+
+        def f_plain():
+            for r in range(ring):
+                ctx.match(Lt, xs[r], sims[r], idxs[r], stream=cur())
+
+        def f_select():
+            for r in range(ring):
+                ctx.select_joint(Lt, frames, sims[r], idxs[r], oc.SELECT_COUNT, 0.0, n_pair, n_single, stride,
+                                 kept[r], cnt[r], mm[r], so[r], stream=cur())
+
+        def f_gather():
+            for r in range(ring):
+                ctx.gather(rows, xs[r], kept[r], F * stride, ys[r], stream=cur())
+
+        def f_restore():
+            for r in range(ring):
+                ctx.restore(rows, ys[r], caches[r], n, so[r], mm[r], outs[r], stream=cur())
+        t = {k: graph_time_us(f, reps) / ring for k, f in
+             (("frame", f_frame), ("match", f_match), ("plain", f_plain), ("select", f_select), ("gather", f_gather),
+              ("restore", f_restore))}
+        torch.cuda.synchronize()
+        fr = frames.cpu().numpy()
+        n_pairs = int((fr[:, 1] >= 0).sum()); n_groups = int((fr[:, 0] >= 0).sum())
+        n_keep = int(sum(c.item() for c in [cnt[0].sum()]))
+        units = 3 * n_groups + 4 * n_pairs                             # sub-lattices of candidates over all groups
+        flops = 2.0 * units * (P // 4) * (P // 4) * C
+        plain_flops = 2.0 * 3 * F * (P // 4) * (P // 4) * C
+        results.append({
+            "workload": f"svd_l{lv}", "shape": list(base.shape), "frame_threshold": thr, "pairs": n_pairs,
+            "single_frames": n_groups - n_pairs, "kept_tokens": n_keep, "of_tokens": n,
+            "frame_cache_and_pairing_us": t["frame"], "match_joint_us": t["match"], "match_joint_GFLOP": flops / 1e9,
+            "match_joint_TFLOP/s": flops / (t["match"] * 1e-6) / 1e12,
+            "per_frame_token_match_us": t["plain"], "per_frame_token_match_TFLOP/s": plain_flops / (t["plain"] * 1e-6) / 1e12,
+            "select_joint_us": t["select"], "gather_us": t["gather"], "restore_us": t["restore"],
+            "gather_frac_hbm": 2 * n_keep * C * 2 / (t["gather"] * 1e-6) / 1e9 / peaks["hbm_gbs"],
+            "restore_frac_hbm": 2 * n * C * 2 / (t["restore"] * 1e-6) / 1e9 / peaks["hbm_gbs"]})
+        assert ctx.device_status() == oc.OK
+        ctx.close()
+        del xs, caches, outs, sims, idxs, kept, mm, so, ys
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "per-op device time, Token Cache on the frame pairs of Frame Cache (Section 3.2.3), SVD levels",
+                      "unit": "us", "timing": "CUDA-graph replay per op over a ring of buffers larger than 4x L2",
+                      "data": "synthetic", "results": results}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -772,12 +885,14 @@ def main():
     if args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     rank, local_rank, world = sharding.env_rank_world()
-    if args.workload in ("svd_sweep", "sd3_groups", "svd_patches", "frame_block_patches"):
+    if args.workload in ("svd_sweep", "sd3_groups", "svd_patches", "frame_block_patches", "svd_joint"):
         if rank == 0:
             if args.workload == "svd_sweep":
                 run_sweep(args)
             elif args.workload == "sd3_groups":
                 run_token_groups(args)
+            elif args.workload == "svd_joint":
+                run_joint(args)
             elif args.workload == "frame_block_patches":
                 # patch-local Frame Cache (SVD frame tensor) and Block Cache (SVD level 0 and the Latte tensor)
                 blk = make_workload("svd_token_l0")
