@@ -33,6 +33,12 @@
 // its B descriptor 16 rows in), and the pieces are dealt out evenly, in contiguous runs, to one
 // persistent CTA (pair) per SM (pair of SMs).
 // The host picks the form, the tiles per CTA and P with a small cost model.
+// Joint form (Token Cache on the frame pairs of Frame Cache, Section 3.2.3): the rows are not the
+// regular (frame, patch, sub-lattice) enumeration but a list of {representative frame, candidate
+// frame, sub-lattice} units that another kernel wrote; its length exists only on the device, so every
+// walker reads it, takes its share of (unit, tile run, piece) triples and looks a unit up once.  The
+// candidate tiles then come from one frame and the representatives from another -- a different fourth
+// TMA coordinate for the two operands -- and nothing else changes.
 //
 // Warp specialised:
 //   warp 0      TMA producer   (one lane per box; a CTA's candidate tiles are one box, and so are its
