@@ -319,6 +319,7 @@ __device__ __forceinline__ unsigned div_small(unsigned a, unsigned d, float rcp_
 // Pieces are numbered row-major over (frame, patch row, patch column, candidate lattice, tile run,
 // piece of the row); a walker takes a contiguous range.  The first piece is decoded by division,
 // the following ones by counting up.
+template <bool JOINT>
 struct Walk {
     int left;                            // pieces still to hand out
     int j, a_pair, k, px, py, bt;
@@ -330,7 +331,7 @@ struct Walk {
         bt = v.x; bt_a = v.y; member_u = v.z;
     }
     __device__ __forceinline__ Walk(const TcScalars& P, int c) {
-        if (P.units) {
+        if (JOINT) {
             // pieces are numbered (unit, tile run, piece of the row); the list length is read here
             const unsigned total = (unsigned)__ldg(P.n_units_dev) * P.cum[1];
             const unsigned base = div_small(total, P.n_walkers, P.rcp_walkers), rem = total - base * P.n_walkers;
@@ -381,13 +382,13 @@ struct Walk {
         }
         u_cur = u_next; r_cur = r_next;
         p.a_pair = a_pair; p.g = g; p.px = px; p.py = py; p.bt = bt;
-        p.bt_a = P.units ? bt_a : bt;
-        p.member = P.units ? member_u : (k < P.rep_member ? k : k + 1);
+        p.bt_a = JOINT ? bt_a : bt;
+        p.member = JOINT ? member_u : (k < P.rep_member ? k : k + 1);
         if (++j == P.pieces_per_row) {
             j = 0; u_cur = 0; r_cur = 0;
             if (++a_pair == P.n_apairs) {
                 a_pair = 0;
-                if (P.units) {
+                if (JOINT) {
                     ++g;
                     if (left > 0) load_unit(P);
                 } else if (++k == P.n_cand_lat) {
@@ -411,9 +412,11 @@ static constexpr int SMEM_TOTAL = TILE_BYTES + TAIL_BYTES;
 // representative quanta; the tensor cores of both SMs read both halves, so every fetched operand
 // byte feeds twice the FLOPs.  The leader (cluster rank 0) issues all MMAs; both CTAs' copies report
 // to the leader's stage barrier, and the leader's commits free the stage in both CTAs.
-template <bool PAIR, bool AUX>
+// MODE 0: the hot instance; 1: also writes the full similarity rows (parity runs); 2: the joint work list.
+template <bool PAIR, int MODE>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 match_tc_kernel(const __grid_constant__ TcParams KP) {
+    constexpr bool AUX = MODE == 1, JOINT = MODE == 2;
     // The operand ring starts at the base of dynamic shared memory, which must be 1024-byte aligned
     // for the 128-byte swizzle (this kernel has no static shared memory in front of it; checked below).
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -460,7 +463,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         tma_prefetch_map(&KP.mapQ[0]);
         tma_prefetch_map(&KP.mapQ[1]);
         for (int m = 0; m <= KP.s.n_cand_lat; ++m)
-            if (m != KP.s.rep_member || KP.s.units) tma_prefetch_map(&KP.mapsA[m]);
+            if (m != KP.s.rep_member || JOINT) tma_prefetch_map(&KP.mapsA[m]);
     }
     if (warp == 1) {
         if (PAIR) {
@@ -489,8 +492,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     const bool dbl = P.tpp == 1;
 
     // (the joint form's work list is written by a kernel earlier in the stream: wait for it)
-    if (P.units) pdl_wait();
-    Walk walk(P, walker);                  // every role walks the same pieces
+    if (JOINT) pdl_wait();
+    Walk<JOINT> walk(P, walker);                  // every role walks the same pieces
     Piece c;
     const int bwA = 1 << P.bwA_log2, bwQ = 1 << P.bwQ_log2;
     const int my_rep = P.my_rep, mx_rep = P.mx_rep;
@@ -1000,10 +1003,12 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     static bool attr_ok = false;
     static int max_pairs[64];
     std::call_once(attr_once, [] {
-        attr_ok = cudaFuncSetAttribute(match_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
-                  cudaFuncSetAttribute(match_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
-                  cudaFuncSetAttribute(match_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
-                  cudaFuncSetAttribute(match_tc_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess;
+        attr_ok = cudaFuncSetAttribute(match_tc_kernel<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+                  cudaFuncSetAttribute(match_tc_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+                  cudaFuncSetAttribute(match_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+                  cudaFuncSetAttribute(match_tc_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+                  cudaFuncSetAttribute(match_tc_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+                  cudaFuncSetAttribute(match_tc_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess;
         for (int i = 0; i < 64; ++i) max_pairs[i] = -1;
         if (!attr_ok) cudaGetLastError();
     });
@@ -1019,7 +1024,7 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
             q.gridDim = dim3(2 * (unsigned)(ctx->sm_count / 2)); q.blockDim = dim3(TC_THREADS);
             q.dynamicSmemBytes = SMEM_TOTAL; q.attrs = qa; q.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, match_tc_kernel<true, false>, &q) != cudaSuccess) { cudaGetLastError(); n = 0; }
+            if (cudaOccupancyMaxActiveClusters(&n, match_tc_kernel<true, 0>, &q) != cudaSuccess) { cudaGetLastError(); n = 0; }
             if (n > ctx->sm_count / 2) n = ctx->sm_count / 2;
             max_pairs[dev] = n;
         }
@@ -1092,13 +1097,15 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     LaunchScope scope(ctx, OC_K_MATCH_TC, s);
     if (p.pair) {
         PdlLaunch l(dim3(2 * (unsigned)walkers), dim3(TC_THREADS), SMEM_TOTAL, s, 2);
-        const cudaError_t e = aux_sim ? cudaLaunchKernelEx(&l.cfg, match_tc_kernel<true, true>, KP)
-                                      : cudaLaunchKernelEx(&l.cfg, match_tc_kernel<true, false>, KP);
+        const cudaError_t e = units ? cudaLaunchKernelEx(&l.cfg, match_tc_kernel<true, 2>, KP)
+                            : aux_sim ? cudaLaunchKernelEx(&l.cfg, match_tc_kernel<true, 1>, KP)
+                                      : cudaLaunchKernelEx(&l.cfg, match_tc_kernel<true, 0>, KP);
         if (e != cudaSuccess) { cudaGetLastError(); return OC_ERR_CUDA; }
         return OC_OK;
     }
-    if (aux_sim) OC_LAUNCH((match_tc_kernel<false, true>), (unsigned)walkers, TC_THREADS, SMEM_TOTAL, s, KP);
-    else OC_LAUNCH((match_tc_kernel<false, false>), (unsigned)walkers, TC_THREADS, SMEM_TOTAL, s, KP);
+    if (units) OC_LAUNCH((match_tc_kernel<false, 2>), (unsigned)walkers, TC_THREADS, SMEM_TOTAL, s, KP);
+    else if (aux_sim) OC_LAUNCH((match_tc_kernel<false, 1>), (unsigned)walkers, TC_THREADS, SMEM_TOTAL, s, KP);
+    else OC_LAUNCH((match_tc_kernel<false, 0>), (unsigned)walkers, TC_THREADS, SMEM_TOTAL, s, KP);
     return last_launch_status();
 }
 

@@ -25,6 +25,7 @@ static constexpr int SEL_SMEM_KEYS = 40960;          // keys cached in shared me
 // Per-CTA view of one group: unit index and candidate test with as few instructions as possible
 // (one CTA serves a whole group, so the kernel is bound by instruction issue on a single SM):
 // shifts and masks when the row width / lattice strides are powers of two, divisions otherwise.
+template <bool JOINT = false>
 struct GroupView {
     long long base;     // global index of local unit 0 (TOKEN: of the patch's first token)
     int unit_stride;    // FRAME: distance between consecutive frames of a patch position
@@ -38,7 +39,7 @@ struct GroupView {
     int rep_half;       // joint form: which of the two frames holds the representatives
     __device__ GroupView(const GroupMap& m, long long g) {
         base1 = 0; frame_units = 0; rep_half = 0;
-        if (m.frames) {                                 // one or two whole frames, in time order
+        if (JOINT) {                                    // one or two whole frames, in time order
             const int2 fr = m.frames[g];
             const int f0 = (fr.y >= 0 && fr.y < fr.x) ? fr.y : fr.x, f1 = (fr.y >= 0 && fr.y < fr.x) ? fr.x : fr.y;
             frame_units = m.H * m.W;
@@ -68,13 +69,13 @@ struct GroupView {
         else { ly = u / w_local; lx = u - ly * w_local; }
     }
     __device__ __forceinline__ long long index(const GroupMap& m, int u) const {
-        if (frame_units && u >= frame_units) return base1 + (u - frame_units);
+        if (JOINT && u >= frame_units) return base1 + (u - frame_units);
         if (contig) return base + (long long)u * unit_stride;
         int ly, lx; split(u, ly, lx);
         return base + (long long)ly * row_pitch + lx;
     }
     __device__ __forceinline__ bool is_cand(const GroupMap& m, int u) const {
-        if (frame_units) {                              // every token of the partner frame is a candidate
+        if (JOINT) {                                    // every token of the partner frame is a candidate
             const int half = u >= frame_units ? 1 : 0;
             if (half != rep_half) return true;
             u -= half * frame_units;
@@ -128,7 +129,7 @@ select_general_kernel(GroupMap gm, const float* __restrict__ best_sim, const int
     const long long g = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n_rounds = (U + SEL_THREADS - 1) / SEL_THREADS;
-    const GroupView gv(gm, g);
+    const GroupView<> gv(gm, g);
     int scan_flip = 0;
 
     // ---- COUNT mode: value at the cut ----------------------------------------------------------
@@ -305,6 +306,7 @@ __device__ __forceinline__ int block_scan_int(int v, int* sums /*[33]*/, int& to
     return sums[warp] + incl - v;
 }
 
+template <bool JOINT>
 __global__ void __launch_bounds__(1024)
 select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_t* __restrict__ best_idx,
                    int mode, float thr, int n_reuse, int y_stride,
@@ -322,7 +324,7 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
     int U = gm.units_per_group;
     const long long g = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31;
-    if (gm.frames) {                                            // joint form: the slot decides the group's size and budget
+    if (JOINT) {                                                // joint form: the slot decides the group's size and budget
         const int2 fr = gm.frames[g];
         if (fr.x < 0) {                                         // absorbed into its partner's group: keeps nothing
             for (int p = tid; p < y_stride; p += NT) kept_idx[g * y_stride + p] = -1;
@@ -332,7 +334,7 @@ select_fast_kernel(GroupMap gm, const float* __restrict__ best_sim, const int32_
         if (fr.y < 0) { U = gm.H * gm.W; n_reuse = gm.n_reuse_single; }
     }
     const int n_rounds = (U + NT - 1) / NT;
-    const GroupView gv(gm, g);
+    const GroupView<JOINT> gv(gm, g);
 
     // ---- phase 0: every input is read once, coalesced, all loads issued before any is used --------
     // key 0 marks a non-candidate (every real key is >= 1)
@@ -519,7 +521,7 @@ select_small_kernel(GroupMap gm, long long n_groups, const float* __restrict__ b
     if (g >= n_groups) return;                                 // whole warps leave together
     const int lane = threadIdx.x & 31;
     const int U = gm.units_per_group;
-    const GroupView gv(gm, g);
+    const GroupView<> gv(gm, g);
     long long gi[2];
     unsigned key[2];
     int m_idx[2];
@@ -590,7 +592,7 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
     if (!attr_set) {
         if (cudaFuncSetAttribute(select_general_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess ||
-            cudaFuncSetAttribute(select_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaFuncSetAttribute(select_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess)
             return OC_ERR_CUDA;
         attr_set = true;
@@ -609,7 +611,7 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
         while (min_nt < SEL_THREADS && min_nt * 4 < geo.units_per_group) min_nt <<= 1;      // at most ~4 units per thread
         while (nt > min_nt && (long long)geo.n_groups * nt > 2048ll * ctx->sm_count) nt >>= 1;
         while (nt < SEL_THREADS && (geo.units_per_group + nt - 1) / nt > 40) nt <<= 1;
-        OC_LAUNCH(select_fast_kernel, (unsigned)geo.n_groups, nt, (size_t)geo.units_per_group * sizeof(unsigned), s,
+        OC_LAUNCH(select_fast_kernel<false>, (unsigned)geo.n_groups, nt, (size_t)geo.units_per_group * sizeof(unsigned), s,
                   gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);
     } else {
         const int keys_in_smem = (mode == OC_SELECT_COUNT && geo.units_per_group <= SEL_SMEM_KEYS) ? 1 : 0;
@@ -636,13 +638,13 @@ oc_status launch_select_joint(oc_ctx* ctx, const Geo& geo, const int2* frames, c
     const int nr = (int)(n_reuse_pair > 0x7FFFFFFF ? 0x7FFFFFFF : n_reuse_pair);
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(select_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(select_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess)
             return OC_ERR_CUDA;
         attr_set = true;
     }
     LaunchScope scope(ctx, OC_K_SELECT, s);
-    OC_LAUNCH(select_fast_kernel, (unsigned)slots, SEL_THREADS, (size_t)(2 * P) * sizeof(unsigned), s,
+    OC_LAUNCH(select_fast_kernel<true>, (unsigned)slots, SEL_THREADS, (size_t)(2 * P) * sizeof(unsigned), s,
               gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);
     return last_launch_status();
 }
