@@ -316,6 +316,40 @@ def select_joint(L: Layout, frames: np.ndarray, best_sim, best_idx, mode: int, t
     return dict(kept_idx=kept_idx, kept_count=kept_count, match_map=match_map, slot_of=slot_of)
 
 
+def _bf16_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def _f64_to_bf16_rne(v: np.ndarray) -> np.ndarray:
+    """Round float64 values ONCE to bf16 (8 significant bits, ties to even); returns the 16-bit patterns.
+    Normal range only (no subnormal / overflow handling: the tests stay far from both)."""
+    v = np.asarray(v, np.float64)
+    out = np.zeros(v.shape, np.float64)
+    nz = v != 0
+    e = np.floor(np.log2(np.abs(v[nz])))
+    ulp = np.exp2(e - 7)
+    out[nz] = np.rint(v[nz] / ulp) * ulp                 # exact scalings by powers of two; rint = half to even
+    return (out.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+
+
+def linear_gather_scatter(a: np.ndarray, a_idx, n_rows: int, w: np.ndarray, out: np.ndarray, out_idx) -> np.ndarray:
+    """The wrapped layer's projection with the gather folded into its operand load and the restore into
+    its store (Appendix A's compaction and scatter, fused into the layer):
+        out[dst(r), :] = bf16( sum_k a[src(r), k] * w[n, k] ),   r = 0 .. n_rows-1,
+    src(r) = a_idx[r] (r if a_idx is None), dst(r) = out_idx[r] (r if None); a row whose src or dst is
+    negative is skipped; rows of ``out`` that no r writes keep their contents.  bf16 bit patterns in and
+    out, products and sums in float64, one rounding at the end."""
+    a64, w64 = _bf16_to_f64(np.asarray(a, np.uint16)), _bf16_to_f64(np.asarray(w, np.uint16))
+    res = np.array(out, np.uint16, copy=True)
+    for r in range(n_rows):
+        src = r if a_idx is None else int(a_idx[r])
+        dst = r if out_idx is None else int(out_idx[r])
+        if src < 0 or dst < 0:
+            continue
+        res[dst] = _f64_to_bf16_rne(w64 @ a64[src])
+    return res
+
+
 def layer_cache_hit(stored_step: int, step: int, interval: int) -> bool:
     return bool(lib().ocr_layer_cache_hit(stored_step, step, interval))
 

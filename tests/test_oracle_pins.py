@@ -779,6 +779,43 @@ def unit_rows_generic(t, L):
     return np.ascontiguousarray(t.reshape(L.B, L.T, L.H * L.W, Cc).transpose(0, 2, 1, 3)).reshape(L.B * L.H * L.W, -1)
 
 
+def test_linear_gather_scatter_pins(oracle):
+    """bf16 rounding by hand, identity weights, a library matmul, untouched rows."""
+    # rounding to 8 significant bits, ties to even: 1 + 2^-8 is a tie -> 1.0 (even), 1 + 3*2^-8 -> 1 + 2^-6
+    v = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20, -0.3, 3.0e5, 0.0])
+    bits = oracle._f64_to_bf16_rne(v)
+    back = oracle._bf16_to_f64(bits)
+    assert back[0] == 1.0 and back[1] == 1.0 and back[2] == 1.0 + 2.0 ** -6 and back[3] == 1.0 + 2.0 ** -7
+    assert back[6] == 0.0 and abs(back[4] + 0.3) <= 0.3 * 2.0 ** -8 and abs(back[5] - 3.0e5) <= 3.0e5 * 2.0 ** -8
+    assert np.array_equal(oracle._f64_to_bf16_rne(back), bits)                 # bf16 values are fixed points
+    rng = np.random.default_rng(12)
+    Ra, K, N, Ro = 20, 24, 16, 30
+    a = inputs.to_bf16_bits(rng.standard_normal((Ra, K)).astype(np.float32))
+    w = inputs.to_bf16_bits(rng.standard_normal((N, K)).astype(np.float32))
+    out0 = inputs.to_bf16_bits(rng.standard_normal((Ro, N)).astype(np.float32))
+    a_idx = np.array([3, 7, -1, 19, 0, 7], np.int32)
+    out_idx = np.array([5, 29, 2, -1, 11, 0], np.int32)
+    got = oracle.linear_gather_scatter(a, a_idx, 6, w, out0, out_idx)
+    a64, w64 = oracle._bf16_to_f64(a), oracle._bf16_to_f64(w)
+    written = {5: 3, 29: 7, 11: 0, 0: 7}                                        # dst -> src (rows 2 and 3 skipped)
+    for dst in range(Ro):
+        if dst in written:
+            exact = a64[written[dst]] @ w64.T                                   # library matmul in float64
+            y = oracle._bf16_to_f64(got[dst])
+            assert np.all(np.abs(y - exact) <= np.abs(exact) * 2.0 ** -8 + 1e-30)
+        else:
+            assert np.array_equal(got[dst], out0[dst])
+    # identity weights: the output rows ARE the gathered rows; no index arrays: plain rows
+    eye = inputs.to_bf16_bits(np.eye(K, dtype=np.float32))
+    y = oracle.linear_gather_scatter(a, None, Ra, eye, np.zeros((Ra, K), np.uint16), None)
+    assert np.array_equal(y, a)
+    # one hand case: [1, 2] . [[3, 4], [0.5, -1]] = [11, -1.5]
+    ah = inputs.to_bf16_bits(np.array([[1.0, 2.0]], np.float32))
+    wh = inputs.to_bf16_bits(np.array([[3.0, 4.0], [0.5, -1.0]], np.float32))
+    yh = oracle._bf16_to_f64(oracle.linear_gather_scatter(ah, None, 1, wh, np.zeros((1, 2), np.uint16), None))
+    assert yh.tolist() == [[11.0, -1.5]]
+
+
 def test_layer_cache_rule(oracle):
     lc = oracle.LayerCache()
     a = np.arange(100, dtype=np.float32)
