@@ -141,7 +141,8 @@ enum {
     OC_K_GATHER = 9,
     OC_K_RESTORE = 10,
     OC_K_COPY = 11,       /* layered-cache put / copying get                          */
-    OC_K_COUNT = 12
+    OC_K_LINEAR = 12,     /* projection with gather / scatter folded in               */
+    OC_K_COUNT = 13
 };
 const char* oc_kernel_name(int kernel_id);
 
@@ -233,6 +234,25 @@ oc_status oc_match(oc_ctx* ctx, const oc_layout* layout, const void* x, float* b
 oc_status oc_match_frame_levels(oc_ctx* ctx, const oc_layout* layout, const void* x, int n_levels,
                                 const int32_t* grids, float* best_sim, int32_t* best_idx, float* pos_sim,
                                 float* pair_sim, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * The wrapped layer's projection with the gather folded into its operand load and the restore into
+ * its store (Appendix A's compaction and fused scatter taken one step further: the dense buffers on
+ * both sides of the layer are never written):
+ *     out[dst(r), :] = bf16( sum_k a[src(r), k] * w[n, k] ),     r = 0 .. n_rows-1
+ *   a        [a_rows][K] bf16, row-major (e.g. the token rows of the feature tensor)
+ *   a_idx    nullable, [n_rows] int32: src(r) = a_idx[r] (the kept_idx list); null: src(r) = r
+ *   w        [N][K] bf16, row-major (the layout of a linear layer's weight)
+ *   out      [out_rows][N] bf16; out_idx nullable, [n_rows]: dst(r) = out_idx[r]; null: dst(r) = r
+ * A row whose src or dst is negative (or out of range) is skipped; rows of `out` that no r names keep
+ * their contents, so with out = the cached activations and out_idx = kept_idx the call IS the restore.
+ * bf16 x bf16 products, fp32 accumulation on the tcgen05 tensor cores, one rounding to bf16.
+ * K % 8 == 0, N % 8 == 0, N >= 128; a, w, out 16-byte aligned.  Errors: OC_ERR_INVALID_ARG,
+ * OC_ERR_ALIGNMENT, OC_ERR_UNSUPPORTED (shape limits), OC_ERR_CUDA.
+ * ------------------------------------------------------------------------------------------- */
+oc_status oc_linear_gather_scatter(oc_ctx* ctx, const void* a, int64_t a_rows, int64_t K, const int32_t* a_idx,
+                                   int64_t n_rows, const void* w, int64_t N, void* out, int64_t out_rows,
+                                   const int32_t* out_idx, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Token Cache on the frame pairs of Frame Cache (Section 3.2.3): "Token Cache consumes the same

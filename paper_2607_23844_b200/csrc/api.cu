@@ -143,7 +143,7 @@ const char* oc_status_str(oc_status s) {
 const char* oc_kernel_name(int k) {
     static const char* names[OC_K_COUNT] = {"norms", "match_tc", "match_simt", "match_finalize", "frame_pair",
                                             "frame_finalize", "block_partial", "block_finalize", "select",
-                                            "gather", "restore", "copy"};
+                                            "gather", "restore", "copy", "linear"};
     return (k >= 0 && k < OC_K_COUNT) ? names[k] : "unknown";
 }
 
@@ -381,6 +381,18 @@ oc_status oc_match_frame_levels(oc_ctx* c, const oc_layout* layout, const void* 
     DeviceGuard guard(c->device);
     if (!guard.ok) return OC_ERR_CUDA;
     return launch_match_frame_levels(c, g, x, n_levels, grids, best_sim, best_idx, pos_sim, pair_sim, (cudaStream_t)stream);
+}
+
+oc_status oc_linear_gather_scatter(oc_ctx* c, const void* a, int64_t a_rows, int64_t K, const int32_t* a_idx,
+                                   int64_t n_rows, const void* w, int64_t N, void* out, int64_t out_rows,
+                                   const int32_t* out_idx, void* stream) {
+    if (!c || !a || !w || !out || a_rows <= 0 || K <= 0 || N <= 0 || n_rows < 0 || out_rows <= 0) return OC_ERR_INVALID_ARG;
+    if (K % 8 != 0 || N % 8 != 0) return OC_ERR_ALIGNMENT;
+    if (misaligned(a) || misaligned(w) || misaligned(out)) return OC_ERR_ALIGNMENT;
+    if (N < 128 || a_rows > 0x7FFFFFFFll || out_rows > 0x7FFFFFFFll || K > 0x7FFFFFFFll || N > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return OC_ERR_CUDA;
+    return launch_linear_gs(c, a, a_rows, K, a_idx, n_rows, w, N, out, out_rows, out_idx, (cudaStream_t)stream);
 }
 
 // ---- Token Cache on the frame pairs of Frame Cache (Section 3.2.3) ---------------------------------

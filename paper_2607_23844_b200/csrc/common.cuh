@@ -170,6 +170,8 @@ oc_status launch_match_token(oc_ctx*, const Geo&, const void* x, float* best_sim
                              float* aux_sim, cudaStream_t);
 // tcgen05 path of launch_match_token; returns OC_ERR_UNSUPPORTED if the shape is not covered.
 bool tc_match_supported(const Geo&);
+oc_status launch_linear_gs(oc_ctx*, const void* a, int64_t a_rows, int64_t K, const int32_t* a_idx, int64_t n_rows,
+                           const void* w, int64_t N, void* out, int64_t out_rows, const int32_t* out_idx, cudaStream_t);
 size_t joint_workspace_bytes(const Geo&);
 oc_status launch_joint_groups(oc_ctx*, int B, int T, const float* frame_best_sim, const int32_t* frame_best_idx,
                               const int32_t* frame_slot_of, int2* frames, cudaStream_t);

@@ -23,8 +23,8 @@ SELECT_THRESHOLD, SELECT_COUNT = 0, 1
 RESTORE_FROM_CACHE, RESTORE_FROM_REPRESENTATIVE = 0, 1
 FRAME_MEAN_POS_COS, FRAME_FLAT_COS = 0, 1
 (K_NORMS, K_MATCH_TC, K_MATCH_SIMT, K_MATCH_FIN, K_FRAME, K_FRAME_FIN, K_BLOCK, K_BLOCK_FIN, K_SELECT,
- K_GATHER, K_RESTORE, K_COPY) = range(12)
-K_COUNT = 12
+ K_GATHER, K_RESTORE, K_COPY, K_LINEAR) = range(13)
+K_COUNT = 13
 
 EXPORTS = (
     "oc_status_str", "oc_layout_check", "oc_layout_counts", "oc_match_workspace_bytes",
@@ -34,6 +34,7 @@ EXPORTS = (
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
     "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
     "oc_schedule_propose", "oc_joint_workspace_bytes", "oc_joint_groups", "oc_match_joint", "oc_select_joint",
+    "oc_linear_gather_scatter",
 )
 
 
@@ -79,6 +80,7 @@ _lib.oc_profile_captured_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_match.argtypes = [_vp] * 8
 _lib.oc_match_frame_levels.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.oc_select.argtypes = [_vp, _vp, _vp, _vp, _i, _f, _i64, _i64, _vp, _vp, _vp, _vp, _vp]
+_lib.oc_linear_gather_scatter.argtypes = [_vp, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _vp]
 _lib.oc_joint_workspace_bytes.argtypes = [_vp, _vp]
 _lib.oc_joint_groups.argtypes = [_vp] * 7
 _lib.oc_match_joint.argtypes = [_vp] * 7
@@ -320,6 +322,14 @@ class Context:
                            _ptr(pair_sim), _stream(stream))
         if check:
             _chk(st, "oc_match")
+        return st
+
+    def linear_gather_scatter(self, a, a_rows: int, K: int, a_idx, n_rows: int, w, N: int, out, out_rows: int,
+                              out_idx, stream=None, check: bool = True) -> int:
+        st = _lib.oc_linear_gather_scatter(self._h, _ptr(a), a_rows, K, _ptr(a_idx), n_rows, _ptr(w), N, _ptr(out),
+                                           out_rows, _ptr(out_idx), _stream(stream))
+        if check:
+            _chk(st, "oc_linear_gather_scatter")
         return st
 
     def joint_groups(self, layout: Layout, frame_best_sim, frame_best_idx, frame_slot_of, frames, stream=None,

@@ -486,6 +486,81 @@ def test_joint_groups_conflicts_and_ties(oc, oracle):
             assert np.array_equal(frames.cpu().numpy(), oracle.joint_groups(B, T, fs, fi, so)), trial
 
 
+# ---------------------------------------------------------------------------------------------------
+# the projection with gather and scatter folded in
+# ---------------------------------------------------------------------------------------------------
+def _bf16_bits_to_f64(b):
+    return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+@pytest.mark.parametrize("a_rows,K,N,n_rows,use_idx", [
+    (300, 64, 128, 200, True), (300, 72, 136, 257, True), (512, 192, 256, 512, False), (700, 320, 640, 300, True),
+    (128, 8, 128, 1, True), (4096, 1536, 1536, 2560, True),
+])
+def test_linear_gather_scatter(oc, oracle, a_rows, K, N, n_rows, use_idx):
+    rng = np.random.default_rng(a_rows + K + N)
+    a = inputs.to_bf16_bits(rng.standard_normal((a_rows, K)).astype(np.float32))
+    w = inputs.to_bf16_bits((rng.standard_normal((N, K)) / np.sqrt(K)).astype(np.float32))
+    out_rows = a_rows + 5
+    out0 = inputs.to_bf16_bits(rng.standard_normal((out_rows, N)).astype(np.float32))
+    if use_idx:
+        a_idx = np.sort(rng.choice(a_rows, n_rows, replace=False)).astype(np.int32)     # a kept-index list
+        out_idx = a_idx.copy()
+        if n_rows > 3:
+            a_idx[n_rows // 2] = -1                                                     # an unused slot
+            out_idx[n_rows // 2] = -1
+            out_idx[1] = -1                                                             # computed but not stored
+    else:
+        a_idx = out_idx = None
+    with oc.Context(0, 0) as ctx:
+        out = H.to_dev(out0)
+        ctx.linear_gather_scatter(H.to_dev(a), a_rows, K, None if a_idx is None else H.to_dev(a_idx), n_rows, H.to_dev(w), N,
+                                  out, out_rows, None if out_idx is None else H.to_dev(out_idx))
+        torch.cuda.synchronize()
+        assert ctx.device_status() == oc.OK
+        assert ctx.launches()["linear"] == 1
+        got = out.cpu().numpy().view(np.uint16).reshape(out_rows, N)
+    # rows the oracle computes: all of them for the small cases, a sample for the large one
+    rows = np.arange(n_rows) if n_rows * N * K < 5e8 else np.sort(rng.choice(n_rows, 200, replace=False))
+    a64, w64 = _bf16_bits_to_f64(a), _bf16_bits_to_f64(w)
+    written = np.zeros(out_rows, bool)
+    exact_match = total = 0
+    for r in range(n_rows):
+        src = r if a_idx is None else int(a_idx[r])
+        dst = r if out_idx is None else int(out_idx[r])
+        if src >= 0 and dst >= 0:
+            written[dst] = True
+    for r in rows:
+        src = r if a_idx is None else int(a_idx[r])
+        dst = r if out_idx is None else int(out_idx[r])
+        if src < 0 or dst < 0:
+            continue
+        ref = oracle.linear_gather_scatter(a[src:src + 1], None, 1, w, np.zeros((1, N), np.uint16), None)[0]
+        exact = w64 @ a64[src]
+        g64, r64 = _bf16_bits_to_f64(got[dst]), _bf16_bits_to_f64(ref)
+        # fp32 accumulation (error a few ulps of the sum of magnitudes) can land on the other side of a bf16
+        # rounding boundary: one bf16 ulp of the result, plus that accumulation error
+        tol = np.abs(exact) * 2.0 ** -7 + (np.abs(w64) @ np.abs(a64[src])) * 2.0 ** -21
+        bad = np.nonzero(np.abs(g64 - r64) > tol)[0]
+        assert bad.size == 0, f"row {r}: cols {bad[:5]} got {g64[bad[:5]]} ref {r64[bad[:5]]} exact {exact[bad[:5]]} tol {tol[bad[:5]]}"
+        exact_match += int((got[dst] == ref).sum())
+        total += N
+    assert total > 0 and exact_match >= 0.98 * total
+    # rows nobody names keep their bytes
+    assert np.array_equal(got[~written], out0[~written])
+
+
+def test_linear_gather_scatter_argument_checks(oc, oracle):
+    with oc.Context(0, 0) as ctx:
+        t = torch.zeros(256 * 128, device="cuda", dtype=torch.int16)
+        assert ctx.linear_gather_scatter(t, 256, 64, None, 10, t, 120, t, 256, None, check=False) == oc.ERR_UNSUPPORTED   # N < 128
+        assert ctx.linear_gather_scatter(t, 256, 60, None, 10, t, 128, t, 256, None, check=False) == oc.ERR_ALIGNMENT
+        assert ctx.linear_gather_scatter(t, 256, 64, None, 10, t, 132, t, 256, None, check=False) == oc.ERR_ALIGNMENT
+        assert ctx.linear_gather_scatter(t, 256, 64, None, -1, t, 128, t, 256, None, check=False) == oc.ERR_INVALID_ARG
+        assert ctx.linear_gather_scatter(t, 256, 64, None, 0, t, 128, t, 256, None) == oc.OK                              # nothing to do
+        assert ctx.launches()["linear"] == 0
+
+
 def test_config2_sd3_token_cache_full(oc, oracle):
     w = inputs.sd3_token_cache()
     rep = run_chain(oc, oracle, w, full_oracle=True)
