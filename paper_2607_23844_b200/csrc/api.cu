@@ -389,6 +389,7 @@ oc_status oc_linear_gather_scatter(oc_ctx* c, const void* a, int64_t a_rows, int
     if (!c || !a || !w || !out || a_rows <= 0 || K <= 0 || N <= 0 || n_rows < 0 || out_rows <= 0) return OC_ERR_INVALID_ARG;
     if (K % 8 != 0 || N % 8 != 0) return OC_ERR_ALIGNMENT;
     if (misaligned(a) || misaligned(w) || misaligned(out)) return OC_ERR_ALIGNMENT;
+    if (!a_idx && n_rows > a_rows) return OC_ERR_INVALID_ARG;
     if (N < 128 || a_rows > 0x7FFFFFFFll || out_rows > 0x7FFFFFFFll || K > 0x7FFFFFFFll || N > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
     DeviceGuard guard(c->device);
     if (!guard.ok) return OC_ERR_CUDA;

@@ -495,7 +495,7 @@ def _bf16_bits_to_f64(b):
 
 @pytest.mark.parametrize("a_rows,K,N,n_rows,use_idx", [
     (300, 64, 128, 200, True), (300, 72, 136, 257, True), (512, 192, 256, 512, False), (700, 320, 640, 300, True),
-    (128, 8, 128, 1, True), (4096, 1536, 1536, 2560, True),
+    (128, 8, 128, 1, True), (4096, 1536, 1536, 2560, True), (600, 200, 384, 600, "scatter"), (300, 64, 256, 290, "scatter"),
 ])
 def test_linear_gather_scatter(oc, oracle, a_rows, K, N, n_rows, use_idx):
     rng = np.random.default_rng(a_rows + K + N)
@@ -512,6 +512,10 @@ def test_linear_gather_scatter(oc, oracle, a_rows, K, N, n_rows, use_idx):
             out_idx[1] = -1                                                             # computed but not stored
     else:
         a_idx = out_idx = None
+    if use_idx == "scatter":                         # dense rows in, scattered rows out (the restore half alone)
+        a_idx = None
+        out_idx = rng.permutation(out_rows)[:n_rows].astype(np.int32)
+        out_idx[3] = -1
     with oc.Context(0, 0) as ctx:
         out = H.to_dev(out0)
         ctx.linear_gather_scatter(H.to_dev(a), a_rows, K, None if a_idx is None else H.to_dev(a_idx), n_rows, H.to_dev(w), N,
