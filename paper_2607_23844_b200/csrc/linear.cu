@@ -7,8 +7,8 @@
 // go straight to their positions in the restored tensor, which already holds the cached rows).
 //
 // One CTA per (128 or 256) x N_TILE output tile: two 128-row tiles share the weight tile whenever that
-// still leaves enough CTAs (the kernel is bound by the L2 -> shared-memory traffic of its operands and
-// by the turnaround of a 3-4 stage ring; 256 rows per CTA are 1.5x the FLOP per fetched byte).
+// still leaves enough CTAs (the kernel is bound by the turnaround of its 3-4 stage ring -- copy latency,
+// proxy fence, hand-over, MMA, commit -- and 256 rows per CTA put twice the MMA work into a stage).
 // Rows that are not gathered (a_idx null: only the restore is folded in) travel as plain TMA boxes.
 // Warp-specialised like the matcher:
 //   warps 0..3  A producers: the gathered rows arrive by 16-byte asynchronous copies (cp.async), eight
@@ -294,8 +294,8 @@ oc_status launch_linear_gs(oc_ctx* ctx, const void* a, int64_t a_rows, int64_t K
     P.n_rows = n_rows; P.N = N; P.K = K; P.a_rows = a_rows; P.out_rows = out_rows;
     P.kblocks = (int)((K + LIN_BK - 1) / LIN_BK);
     P.n_tile = n_tile;
-    // two 128-row tiles per CTA share the weight tile (1.5x the FLOP per fetched byte: the kernel is bound by
-    // the L2 -> shared-memory traffic of its operands) whenever that still leaves enough CTAs for the device
+    // two 128-row tiles per CTA share the weight tile (twice the MMA work per ring stage, whose turnaround
+    // bounds the kernel) whenever that still leaves enough CTAs for the device
     const int m_tiles_per_cta = (n_tile == 256 && ((n_rows + 255) / 256) * ((N + n_tile - 1) / n_tile) >= (ctx->sm_count * 3) / 4) ? 2 : 1;
     P.stage_bytes = m_tiles_per_cta * LIN_A_BYTES + n_tile * LIN_BK * 2;
     const int smem_budget = 200 * 1024;
