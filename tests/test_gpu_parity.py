@@ -308,6 +308,42 @@ def test_frame_hierarchy_levels_from_one_pass(oc, oracle, dtype, stat):
         assert ctx.match_frame_levels(L, H.to_dev(w.x), [(1, 1)] * 9, bs, bi, check=False) == oc.ERR_INVALID_ARG
 
 
+def _random_frame_block_layouts(n, seed):
+    """Seeded random Frame / Block Cache shapes with patch grids: (kind, shape, grid, dtype, stat, mode)."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < n:
+        kind = "frame" if len(out) % 2 == 0 else "block"
+        gy, gx = int(rng.choice([1, 2, 3])), int(rng.choice([1, 2, 4]))
+        hp, wp = 2 * int(rng.integers(1, 6)), 2 * int(rng.integers(1, 9))
+        C = int(rng.choice([8, 24, 40, 64, 200, 320]))
+        B, T = int(rng.integers(1, 3)), int(rng.integers(1, 10))
+        if B * T * gy * hp * gx * wp * C > 3_000_000:
+            continue
+        out.append((kind, (B, T, gy * hp, gx * wp, C), (gy, gx), int(rng.choice([inputs.BF16, inputs.F32])),
+                    int(rng.integers(0, 2)), str(rng.choice(["count", "threshold"]))))
+    return out
+
+
+@pytest.mark.parametrize("kind,shape,grid,dtype,stat,mode", _random_frame_block_layouts(24, seed=424242))
+def test_frame_block_patch_chain_random_layouts(oc, oracle, kind, shape, grid, dtype, stat, mode):
+    """Patch-local Frame and Block Cache, the whole chain, on shapes nobody picked by hand."""
+    B, T, Hh, W, C = shape
+    rng = np.random.default_rng(int(np.prod(shape)) % 7919)
+    x = np.stack([inputs.ar1_frames(rng, inputs.smooth_field(rng, Hh, W, C, 3.0), T, 0.9) for _ in range(B)])
+    x = np.ascontiguousarray(x.reshape(shape), dtype=np.float32)
+    w = inputs.Workload(f"{kind}_random", kind, dtype, shape, x if dtype == inputs.F32 else inputs.to_bf16_bits(x),
+                        mode=mode, thr=0.9, n_reuse=1)
+    w.groups = grid
+    if kind == "block":
+        cand = (Hh // grid[0]) * (W // grid[1]) * 3 // 4
+        w.n_reuse = max(1, cand // 2)
+        run_chain(oc, oracle, w, Cout=16)
+    else:
+        w.n_reuse = max(1, (T // 2) // 2)
+        run_chain(oc, oracle, w, Cout=16, want_aux=True, frame_stat=stat)
+
+
 def test_frame_patch_chain_long_rows(oc, oracle):
     """Rows too long for the time-marching kernel: the pair kernel's tiles follow the patches too."""
     w = _frame_patch_workload(5, 1, 4, 4, 6, 2176, inputs.BF16, (2, 3), "threshold")
