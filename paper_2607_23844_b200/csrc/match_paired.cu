@@ -123,8 +123,9 @@ frame_pair_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float ep
 // Time-marching variant: a thread-group owns ONE position and walks a segment of frames, keeping the
 // previous frame's row in registers and prefetching the next one, so every row is read exactly once
 // (the pair kernel above reads each row twice, the second time out of L2).  Segments overlap by one
-// frame.  Per pair and CTA the groups' values are combined in a fixed order (shuffles inside a warp,
-// then the warps in index order), written as one partial record per (pair, position tile).
+// frame.  Inside the frame loop a thread-group only leaves {dot, norm} of its position in shared memory;
+// the cosines and, per pair, the tile's sums (a fixed-order shuffle tree) are taken once at the end,
+// written as one partial record per (pair, position tile).
 static constexpr int MARCH_CPL = 8;      // most 16-byte chunks a lane may hold per row (instantiated for 5 and 8)
 
 template <int DT, int LPR, int CPL>
@@ -132,8 +133,12 @@ __global__ void __launch_bounds__(PAIR_THREADS, CPL <= 5 ? 3 : 2)
 frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float eps, int seg_len, int n_seg,
                    float* __restrict__ pos_sim, float4* __restrict__ partial, PatchGrid pg) {
     pdl_enter();
-    extern __shared__ float4 warp_part[];                 // [seg_len][PAIR_THREADS / 32]
+    // per (pair of the segment, position of the tile): {dot, |frame t|^2}; and |frame t0|^2 per position.  The
+    // cosines and the per-pair sums are taken from these at the end, with every lane busy, instead of by one
+    // lane per thread-group inside the frame loop (the kernel is bound by instruction issue as much as by HBM).
+    extern __shared__ float2 pair_dn[];                    // [seg_len][GROUPS], then float n0[GROUPS]
     constexpr int GROUPS = PAIR_THREADS / LPR, WARPS = PAIR_THREADS / 32;
+    float* n0 = (float*)(pair_dn + (size_t)seg_len * GROUPS);
     const int b = blockIdx.y / n_seg, seg = blockIdx.y - b * n_seg;
     const int t0 = seg * seg_len;                         // first frame of the segment (as "previous")
     const int t1 = min(T - 1, t0 + seg_len);              // last frame of the segment
@@ -154,12 +159,14 @@ frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float e
     };
     load_row(prev, t0);
     if (t0 + 1 <= t1) load_row(cur, t0 + 1);
-    float n_prev = 0.f;
+    {
+        float n_first = 0.f;
 #pragma unroll
-    for (int k = 0; k < CPL; ++k)
-        if (lane + k * LPR < cpr) Chunk<DT>::sq(prev[k], n_prev);
-    n_prev = group_sum<LPR>(n_prev);
-
+        for (int k = 0; k < CPL; ++k)
+            if (lane + k * LPR < cpr) Chunk<DT>::sq(prev[k], n_first);
+        n_first = group_sum<LPR>(n_first);
+        if (lane == 0) n0[grp] = n_first;
+    }
     for (int t = t0 + 1; t <= t1; ++t) {
         if (t + 1 <= t1) load_row(nxt, t + 1);            // in flight while frame t is reduced
         float dot = 0.f, n_cur = 0.f;
@@ -167,32 +174,30 @@ frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float e
         for (int k = 0; k < CPL; ++k)
             if (lane + k * LPR < cpr) Chunk<DT>::acc2(cur[k], prev[k], dot, n_cur);
         dot = group_sum<LPR>(dot); n_cur = group_sum<LPR>(n_cur);
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (valid && lane == 0) {
-            const float cs = clamp_unit(dot / (fmaxf(sqrtf(n_cur), eps) * fmaxf(sqrtf(n_prev), eps)));
-            if (pos_sim) pos_sim[((long long)b * (T - 1) + (t - 1)) * P + p] = cs;
-            v = make_float4(cs, dot, n_cur, n_prev);
-        }
-        // groups of one warp, fixed order
-#pragma unroll
-        for (int d = 16; d >= LPR; d >>= 1) {
-            v.x += __shfl_xor_sync(0xFFFFFFFFu, v.x, d); v.y += __shfl_xor_sync(0xFFFFFFFFu, v.y, d);
-            v.z += __shfl_xor_sync(0xFFFFFFFFu, v.z, d); v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, d);
-        }
-        if (wl == 0) warp_part[(t - t0 - 1) * WARPS + warp] = v;
-        n_prev = n_cur;
+        if (lane == 0) pair_dn[(t - t0 - 1) * GROUPS + grp] = make_float2(dot, n_cur);
 #pragma unroll
         for (int k = 0; k < CPL; ++k) { prev[k] = cur[k]; cur[k] = nxt[k]; }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < t1 - t0; i += PAIR_THREADS) {
-        float4 a = warp_part[i * WARPS];
-        for (int w = 1; w < WARPS; ++w) {
-            const float4 c = warp_part[i * WARPS + w];
-            a.x += c.x; a.y += c.y; a.z += c.z; a.w += c.w;
+    // one warp per pair of the segment: lanes take the tile's positions (two each when a tile has 64), the
+    // cosine of every position, then a fixed-order sum of {cos, dot, |a|^2, |b|^2} over the tile
+    const int n_here = min(GROUPS, pg.Pp - tile * GROUPS);            // positions of this tile
+    for (int i = warp; i < t1 - t0; i += WARPS) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int gq = wl; gq < n_here; gq += 32) {
+            const float2 dn = pair_dn[i * GROUPS + gq];
+            const float n_prev = i == 0 ? n0[gq] : pair_dn[(i - 1) * GROUPS + gq].y;
+            const float cs = clamp_unit(dn.x / (fmaxf(sqrtf(dn.y), eps) * fmaxf(sqrtf(n_prev), eps)));
+            if (pos_sim) pos_sim[((long long)b * (T - 1) + t0 + i) * P + patch_position(pg, patch, tile * GROUPS + gq)] = cs;
+            v.x += cs; v.y += dn.x; v.z += dn.y; v.w += n_prev;
+        }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            v.x += __shfl_xor_sync(0xFFFFFFFFu, v.x, d); v.y += __shfl_xor_sync(0xFFFFFFFFu, v.y, d);
+            v.z += __shfl_xor_sync(0xFFFFFFFFu, v.z, d); v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, d);
         }
         const int q = b * (T - 1) + t0 + i;               // pair (t0+i+1, t0+i)
-        partial[(long long)q * gridDim.x + blockIdx.x] = a;
+        if (wl == 0) partial[(long long)q * gridDim.x + blockIdx.x] = v;
     }
 }
 
@@ -334,7 +339,8 @@ static FramePlan frame_plan(const Geo& g) {
         int n_seg = 1;
         while ((long long)f.n_tiles * g.B * n_seg < 148 * 4 && (g.T - 1) / (n_seg + 1) >= 6) ++n_seg;
         f.seg_len = (g.T - 1 + n_seg - 1) / n_seg;
-        if (f.seg_len > 256) f.seg_len = 256;            // per-pair warp records live in shared memory
+        const int seg_cap = 40960 / ((PAIR_THREADS / l) * (int)sizeof(float2));   // per-pair, per-position values live in shared memory
+        if (f.seg_len > seg_cap) f.seg_len = seg_cap;
         f.n_seg = (g.T - 1 + f.seg_len - 1) / f.seg_len;
     } else {
         f.lpr = lanes_per_row(cpr);
@@ -381,7 +387,7 @@ static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, co
         Scope scope(ctx, OC_K_FRAME, s);
         if (f.march) {
             dim3 grid((unsigned)f.n_tiles, (unsigned)(g.B * f.n_seg));
-            const size_t smem = (size_t)f.seg_len * (PAIR_THREADS / 32) * sizeof(float4);
+            const size_t smem = ((size_t)f.seg_len * sizeof(float2) + sizeof(float)) * (size_t)(PAIR_THREADS / f.lpr);
             if (g.dtype == OC_DTYPE_BF16)
                 march_dispatch<OC_DTYPE_BF16>(f.lpr, grid, smem, s, (const uint8_t*)x, g.T, P, cpr, g.eps, f.seg_len, f.n_seg, pos_sim, partial, f.pg);
             else
