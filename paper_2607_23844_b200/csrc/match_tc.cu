@@ -20,8 +20,9 @@
 //
 // Tile.  One CTA multiplies ONE or TWO 128-row candidate tiles by the same N <= 256 representatives.
 // Two tiles (M = 256 per CTA, 128 FLOP/B at N = 256) use all 512 TMEM columns as two accumulators;
-// one tile leaves half of TMEM free, so two accumulators take turns and the epilogue of a piece runs
-// under the MMAs of the next.  Optionally two CTAs of a cluster form a pair (cta_group::2): each
+// one tile - or two tiles whose pieces are at most 128 columns wide - leave half of TMEM free, so two
+// sets of accumulators take turns and the epilogue of a piece runs under the MMAs of the next (what
+// pays on short-K problems, where the arg-max epilogue is a third of the time).  Optionally two CTAs of a cluster form a pair (cta_group::2): each
 // holds its own candidate tiles and fetches HALF of the representatives, and the tensor cores of
 // both SMs read both halves: the same MMA work per SM for fewer fetched bytes.
 //
@@ -94,6 +95,8 @@ struct TcScalars {
     int kblocks;
     int bwA_log2, bhA, n_wtA, n_tilesA;  // candidate box: (1 << bwA_log2) x bhA lattice points = 128 rows
     int tpp;                             // candidate tiles per piece: 2 (M = 256), or 1 for small problems
+    int narrow;                          // tpp == 2 and no piece wider than 128 columns: the two tiles' accumulators
+                                         // are 128 columns apart and take 256 columns, so two sets take turns
     int n_apairs;                        // tile rows per lattice member = ceil(n_tilesA / tpp)
     int bwQ_log2, bhQ, n_wq, n_quanta;   // quantum box:   (1 << bwQ_log2) x bhQ lattice points = 32 rows
     int pieces_per_row, total_items;     // a row = the candidate tiles of one piece against all representatives
@@ -322,7 +325,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         tc_fence_after();
     }
     const int STAGES = P.n_stages, STAGE_BYTES = P.stage_bytes;
-    const bool dbl = P.tpp == 1;
+    const bool dbl = P.tpp == 1 || P.narrow;                  // two accumulator sets take turns
+    const uint32_t tile_stride = P.narrow ? 128u : 256u;      // TMEM columns between the two tiles' accumulators
 
     // (the joint form's work list is written by a kernel earlier in the stream: wait for it)
     if (JOINT) pdl_wait();
@@ -434,7 +438,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     if (nstage == STAGES) { nstage = 0; nphase ^= 1u; }
                     // UMMA K = 16 is 32 bytes along the swizzled row: +2 in the descriptor's address field
                     peeked = tc_mma_stage<PAIR>(d_tmem, a0_desc, a1_desc, b_desc, idesc, (uint32_t)(kb != 0), issue,
-                                                two_tiles, bar_full + 8 * nstage, nphase) != 0;
+                                                two_tiles, bar_full + 8 * nstage, nphase, tile_stride) != 0;
                     // frees the stage (in both CTAs of a pair) when the MMAs retire
                     tc_commit<PAIR>(PAIR ? map_to_cta(bar_empty + 8 * stage, 0) : bar_empty + 8 * stage, issue);
                     if (PAIR) tc_commit<PAIR>(map_to_cta(bar_empty + 8 * stage, 1), issue);
@@ -539,7 +543,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     // which a chain last rose.
                     float bm0 = -INFINITY, bm1 = -INFINITY;
                     int bc0 = -1, bc1 = -1;
-                    const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)(t * 256) + buf * 256u;
+                    const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)t * tile_stride + buf * 256u;
                     // two register buffers: the TMEM load of the next step is in flight while this one is reduced
                     uint32_t va[32], vb[32];
 #define OC_KEY(v, s, j) __uint_as_float((__float_as_uint(__uint_as_float(v) * (s)) & 0xFFFFFFE0u) | (uint32_t)(31 - (j)))
@@ -682,7 +686,7 @@ static int pow2_ceil_log2(int v) { int l = 0; while ((1 << l) < v) ++l; return l
 struct TcPlan {
     int bwA_log2, bhA, n_wtA, n_tilesA, tpp, n_apairs, bwQ_log2, bhQ, n_wq, n_quanta;
     int pair, q_unit, n_q_units, half_units, a_merged, q_merged, q_lo, q_hi;
-    int pieces_per_row, qmax, n_stages, stage_bytes;
+    int pieces_per_row, qmax, n_stages, stage_bytes, narrow;
     long long rows, items;
 };
 
@@ -707,8 +711,10 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
     //     has been drained - the refill round trip (MMAs + ~330 + ~1500 cycles of copy latency, ~1000
     //     more in a pair) divided by the stages that fit in the ring;
     //   * the epilogue costs ~250 + ~410 cycles per 32 columns of each thread's half, per tile; with two
-    //     tiles per CTA it follows the MMAs of the piece, with one tile it runs under the next piece's
-    //     MMAs, where the two slow each other down (~0.8 of the shorter one is not hidden);
+    //     tiles per CTA it follows the MMAs of the piece, with one tile - or with two tiles and pieces of
+    //     at most 128 columns, which leave room for a second set of accumulators - it runs under the
+    //     next piece's MMAs, where the two slow each other down (~0.8, resp. ~0.4, of the shorter one is
+    //     not hidden);
     //   * ~6500 cycles before a CTA's first MMA and after its last.
     const int kblocks = (g.C + BK - 1) / BK;
     // Single-CTA pieces are cut in units of HALF a quantum (16 columns) whenever that is valid: no piece
@@ -746,15 +752,19 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
                 const double slow = refill > fast ? refill : fast;
                 const double epi = tpp * (246.0 + 413.0 * ((q + 1) / 2));
                 double piece;
-                if (tpp == 1) {
+                // (two tiles whose pieces are at most 128 columns wide leave room for a second set of
+                //  accumulators, like one tile does)
+                const bool overlapped = tpp == 1 || (hw ? hw * 16 : q * 32) <= 128;
+                if (overlapped) {
                     const double loop = kblocks * slow;
-                    piece = (loop + 440.0 > epi ? loop + 440.0 : epi) + 0.79 * (loop < epi ? loop : epi);
+                    // (the part of the shorter of the two that is not hidden: fitted, one tile 0.79, two narrow tiles 0.36)
+                    piece = (loop + 440.0 > epi ? loop + 440.0 : epi) + (tpp == 1 ? 0.79 : 0.36) * (loop < epi ? loop : epi);
                 } else {
                     const int nf = kblocks < stages ? kblocks : stages;
                     piece = nf * fast + (kblocks - nf) * slow + epi + 534.0;
                 }
                 if (pair) piece += 850.0;
-                const double cost = 6550.0 + (pair ? 616.0 : 0.0) + per_walker * piece + (tpp == 1 ? epi : 0.0);
+                const double cost = 6550.0 + (pair ? 616.0 : 0.0) + per_walker * piece + (overlapped ? epi : 0.0);
                 if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; best_tpp = tpp; best_pair = pair; }
             }
         }
@@ -786,6 +796,11 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
         if (nq > q_max) q_max = nq;
     }
     p.qmax = q_max * ncta;
+    {   // widest piece in columns
+        const int hw = p.half_units ? half_widest(best_P) : 0;
+        const int cols = hw ? hw * 16 : ((p.n_q_units + best_P - 1) / best_P) * p.q_unit * 32;
+        p.narrow = (p.tpp == 2 && cols <= 128 && !getenv("OC_TC_NO_NARROW")) ? 1 : 0;
+    }
     p.stage_bytes = p.tpp * A_BYTES + q_max * Q_BYTES;
     p.n_stages = TILE_BYTES / p.stage_bytes;
     if (p.n_stages > MAX_STAGES) p.n_stages = MAX_STAGES;
@@ -897,7 +912,7 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     P.Hp = g.Hp; P.Wp = g.Wp; P.Hs = g.Hs; P.Ws = g.Ws;
     P.rep_member = rep_member; P.n_cand_lat = g.sy * g.sx - 1;
     P.kblocks = (g.C + BK - 1) / BK;
-    P.bwA_log2 = p.bwA_log2; P.bhA = p.bhA; P.n_wtA = p.n_wtA; P.n_tilesA = p.n_tilesA; P.tpp = p.tpp; P.n_apairs = p.n_apairs;
+    P.bwA_log2 = p.bwA_log2; P.bhA = p.bhA; P.n_wtA = p.n_wtA; P.n_tilesA = p.n_tilesA; P.tpp = p.tpp; P.narrow = p.narrow; P.n_apairs = p.n_apairs;
     P.bwQ_log2 = p.bwQ_log2; P.bhQ = p.bhQ; P.n_wq = p.n_wq; P.n_quanta = p.n_quanta;
     P.pieces_per_row = p.pieces_per_row; P.total_items = (int)p.items;
     P.q_unit = p.q_unit; P.n_q_units = p.n_q_units; P.half_units = p.half_units;

@@ -125,6 +125,7 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
 // after them, so the ~150 cycles it takes to come back pass while those MMAs queue up instead of
 // between two stages (the tensor pipe accepts an MMA only about when the previous one starts, so
 // nothing else hides that gap).
+// tile_stride: TMEM columns between the accumulators of the two candidate tiles.
 // Returns non-zero when the next stage was already full.
 #define OC_MMA_STAGE_ASM(CG, TWO)                                                                        \
     asm volatile(                                                                                       \
@@ -135,7 +136,7 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
         "setp.ne.b32 pa, %5, 0;\n\t"                                                                    \
         "setp.ne.b32 e, %6, 0;\n\t"                                                                     \
         "setp.eq.b32 pt, 0, 0;\n\t"                                                                     \
-        "add.u32 d1, %1, 256;\n\t"                                                                      \
+        "add.u32 d1, %1, %10;\n\t"                                                                      \
         "@e tcgen05.mma.cta_group::" CG ".kind::f16 [%1], %2, %4, %9, pa;\n\t"                          \
         TWO("@e tcgen05.mma.cta_group::" CG ".kind::f16 [d1], %3, %4, %9, pa;\n\t")                     \
         "add.u64 a0, %2, 2;\n\tadd.u64 a1, %3, 2;\n\tadd.u64 bb, %4, 2;\n\t"                          \
@@ -152,14 +153,14 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
         "}"                                                                                             \
         : "=r"(ready)                                                                                   \
         : "r"(d_tmem), "l"(a0_desc), "l"(a1_desc), "l"(b_desc), "r"(accumulate), "r"(issue), "r"(next_bar), \
-          "r"(next_parity), "r"(idesc)                                                                  \
+          "r"(next_parity), "r"(idesc), "r"(tile_stride)                                                \
         : "memory")
 #define OC_KEEP(x) x
 #define OC_DROP(x)
 template <bool PAIR>
 __device__ __forceinline__ uint32_t tc_mma_stage(uint32_t d_tmem, uint64_t a0_desc, uint64_t a1_desc, uint64_t b_desc,
                                                  uint32_t idesc, uint32_t accumulate, uint32_t issue, bool two_tiles,
-                                                 uint32_t next_bar, uint32_t next_parity) {
+                                                 uint32_t next_bar, uint32_t next_parity, uint32_t tile_stride) {
     uint32_t ready;
     if (two_tiles) {
         if (PAIR) OC_MMA_STAGE_ASM("2", OC_KEEP); else OC_MMA_STAGE_ASM("1", OC_KEEP);
