@@ -52,7 +52,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if failed:
         raise RuntimeError("nvcc failed")
     tmp = LIB + f".{os.getpid()}.tmp"
-    subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart_static", "-ldl", "-lrt", "-lpthread"], check=True)
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs +
+                   ["-lcudart_static", "-ldl", "-lrt", "-lpthread"], check=True)
     os.replace(tmp, LIB)
     return LIB
 
