@@ -147,7 +147,6 @@ linear_gs_kernel(const __grid_constant__ LinParams P) {
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
-            int issued = 0;
             for (int kb = 0; kb < P.kblocks; ++kb) {
                 if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                 // rows that are not gathered travel as plain 128-row boxes (rows past the end read as zeros)
@@ -157,7 +156,6 @@ linear_gs_kernel(const __grid_constant__ LinParams P) {
                     for (int mt = 0; mt < M_TILES; ++mt)
                         tma_load_2d(tiles + (uint32_t)(stage * P.stage_bytes) + mt * LIN_A_BYTES, &P.mapA, kb * LIN_BK,
                                     (int)(m0 + mt * LIN_BM), bar_full + 8 * stage);
-                ++issued;
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
             if (!ok) {
@@ -166,7 +164,6 @@ linear_gs_kernel(const __grid_constant__ LinParams P) {
                 const unsigned long long t0 = global_ns();             // boxes already issued: a bounded chance to land
                 while (global_ns() - t0 < 2000000ull) {}
             }
-            (void)issued;
         }
     } else if (warp == 5) {
         // ================================ MMA issuer ============================================
