@@ -475,6 +475,26 @@ def test_joint_token_cache_svd_level_shapes_every_plan(oc, oracle, plan, monkeyp
     assert reused == 2 * P + 3 * (P // 3)
 
 
+def test_joint_many_short_frames(oc, oracle):
+    """More frame slots than one pass of the work-list kernel takes (1100 > 1024), tiny frames."""
+    shape = (1, 1100, 4, 4, 8)
+    B, T, Hh, W, C = shape
+    rng = np.random.default_rng(2)
+    x = inputs.ar1_frames(rng, rng.standard_normal((Hh, W, C), dtype=np.float32), T, 0.8).reshape(shape)
+    x_np = inputs.to_bf16_bits(np.ascontiguousarray(x, dtype=np.float32))
+    frames = np.array([[f, -1] for f in range(T)], np.int32)
+    for u in range(0, T - 1, 2):                       # every third representative frame takes a partner
+        if (u // 2) % 3 == 0:
+            frames[u] = (u, u + 1); frames[u + 1] = (-1, -1)
+        elif (u // 2) % 3 == 1 and u >= 2 and frames[u - 1][0] >= 0:
+            frames[u] = (u, u - 1); frames[u - 1] = (-1, -1)
+    P = Hh * W
+    reused = _joint_case(oc, oracle, x_np, shape, frames, oc.SELECT_COUNT, 0.0, 9, 5)
+    n_pairs = int((frames[:, 1] >= 0).sum())
+    n_single = int((frames[:, 0] >= 0).sum()) - n_pairs
+    assert reused == 9 * n_pairs + 5 * n_single
+
+
 def test_joint_groups_from_frame_cache_and_full_chain(oc, oracle):
     """Frame Cache decides the pairs (on the GPU), Token Cache works on them: the whole joint path."""
     shape = (2, 7, 16, 16, 64)
