@@ -344,6 +344,16 @@ def test_frame_block_patch_chain_random_layouts(oc, oracle, kind, shape, grid, d
         run_chain(oc, oracle, w, Cout=16, want_aux=True, frame_stat=stat)
 
 
+@pytest.mark.parametrize("grid", [(1, 1), (2, 3)])
+def test_frame_chain_long_clip(oc, oracle, grid):
+    """600 frames: the marching kernel cuts the clip into several segments (its per-pair records live
+    in shared memory) and the select sees groups of 600 units."""
+    w = _frame_patch_workload(9, 1, 600, 4, 6, 8, inputs.BF16, grid, "count", rho=0.9)
+    w.n_reuse = 140
+    rep = run_chain(oc, oracle, w, Cout=8, want_aux=True)
+    assert rep["reused"] == 140 * grid[0] * grid[1]
+
+
 def test_frame_patch_chain_long_rows(oc, oracle):
     """Rows too long for the time-marching kernel: the pair kernel's tiles follow the patches too."""
     w = _frame_patch_workload(5, 1, 4, 4, 6, 2176, inputs.BF16, (2, 3), "threshold")
