@@ -796,7 +796,7 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
         if (nq > q_max) q_max = nq;
     }
     p.qmax = q_max * ncta;
-    {   // widest piece in columns
+    {   // widest piece in columns (experiments may set OC_TC_NO_NARROW to keep such plans on one accumulator set)
         const int hw = p.half_units ? half_widest(best_P) : 0;
         const int cols = hw ? hw * 16 : ((p.n_q_units + best_P - 1) / best_P) * p.q_unit * 32;
         p.narrow = (p.tpp == 2 && cols <= 128 && !getenv("OC_TC_NO_NARROW")) ? 1 : 0;
