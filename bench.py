@@ -52,6 +52,8 @@ def measured_peaks():
 
 
 def make_workload(name: str, seed_offset: int = 0) -> inputs.Workload:
+    if name == "tiny_token":
+        return inputs.tiny_token_cache(seed=1001 + seed_offset)
     if name == "sd3_token":
         return inputs.sd3_token_cache(seed=1002 + seed_offset)
     if name == "svd_frame":
@@ -137,8 +139,9 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------------------
 def oracle_sample_step(w: inputs.Workload, n_rows: int, seed: int = 0):
     """Times the oracle, as it stands, on a bounded sample of one step of workload `w`:
-    match on `n_rows` sampled candidates (scaled to all candidates), then select / gather / restore
-    at full size.  Returns (tokens_per_s, seconds, description, threads)."""
+    match on `n_rows` sampled candidates (time scaled to all candidates; Frame / Block Cache and small
+    Token Cache workloads are matched in full), then select / gather / restore at full size, each op
+    timed by itself.  Returns a dict: tokens_per_s, seconds, per_op_s, sample, cores."""
     import oracle
     oracle.build()
     Lo = oracle.Layout(KIND[w.kind], w.dtype, *w.shape, gy=w.groups[0], gx=w.groups[1],
@@ -149,8 +152,8 @@ def oracle_sample_step(w: inputs.Workload, n_rows: int, seed: int = 0):
     mode = 1 if w.mode == "count" else 0
     if w.kind == "token":
         rng = np.random.default_rng(seed)
-        cands = np.array([i for i in rng.permutation(n_units) if not _is_rep_token(w, int(i))][:n_rows],
-                         dtype=np.int32)
+        cand_mask = np.array([not _is_rep_token(w, i) for i in range(n_units)])
+        cands = rng.permutation(np.nonzero(cand_mask)[0])[:n_rows].astype(np.int32)
     t0 = time.perf_counter()
     if w.kind == "token":
         m = oracle.match_token(Lo, w.x, rows=np.sort(cands))
@@ -162,7 +165,6 @@ def oracle_sample_step(w: inputs.Workload, n_rows: int, seed: int = 0):
         # unsampled candidates get a deterministic filler similarity so that select sees full-size input
         filler = np.random.default_rng(1).uniform(0.9, 0.99, n_units).astype(np.float32)
         unsampled = np.ones(n_units, bool); unsampled[cands] = False
-        cand_mask = np.array([not _is_rep_token(w, i) for i in range(n_units)])
         best_sim = np.where(unsampled & cand_mask, filler, best_sim).astype(np.float32)
         best_idx = np.where(unsampled & cand_mask, 0, best_idx).astype(np.int32)
     else:
@@ -170,17 +172,21 @@ def oracle_sample_step(w: inputs.Workload, n_rows: int, seed: int = 0):
         t_match = time.perf_counter() - t0
         sample = "full step"
         best_sim, best_idx = m["best_sim"], m["best_idx"]
-    t1 = time.perf_counter()
     n_cand_g = U if w.self_match else U - R
     stride = U - min(w.n_reuse, n_cand_g) if mode == 1 else U
+    t1 = time.perf_counter()
     s = oracle.select(Lo, best_sim, best_idx, mode, w.thr, w.n_reuse, stride)
+    t2 = time.perf_counter()
     Rw = oracle.rows_for(Lo, w.shape[-1], w.elem_bytes)
     y = oracle.gather(Rw, w.x, s["kept_idx"])
+    t3 = time.perf_counter()
     cache = w.x            # any tensor of the right shape: restore is a bit copy
     oracle.restore(Rw, y, cache, n_units, s["slot_of"], s["match_map"])
-    t_rest = time.perf_counter() - t1
-    total = t_match + t_rest
-    return (n_cand + n_units) / total, total, sample, oracle.num_threads()
+    t4 = time.perf_counter()
+    total = t_match + (t4 - t1)
+    return {"tokens_per_s": (n_cand + n_units) / total, "seconds": total, "sample": sample,
+            "cores": oracle.num_threads(),
+            "per_op_s": {"match": t_match, "select": t2 - t1, "gather": t3 - t2, "restore": t4 - t3}}
 
 
 def _is_rep_token(w: inputs.Workload, i: int) -> bool:
@@ -192,6 +198,12 @@ def _is_rep_token(w: inputs.Workload, i: int) -> bool:
     return ((y % (H // gy)) % 2 == 0) and ((x % (W // gx)) % 2 == 0)
 
 
+def cpu_baseline_record(w: inputs.Workload, n_rows: int, seed: int = 0) -> dict:
+    r = oracle_sample_step(w, n_rows, seed)
+    return {"value": r["tokens_per_s"], "unit": "tokens/s", "cores": r["cores"], "kind": "oracle",
+            "sample": r["sample"], "seconds": r["seconds"], "per_op_s": r["per_op_s"]}
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
@@ -199,23 +211,23 @@ def run_reference(args, rank):
     n_rows = args.ref_rows
     for _ in range(args.warmup if args.warmup < 2 else 1):
         oracle_sample_step(w, max(n_rows // 8, 8))
-    times, vals = [], []
-    sample = threads = None
+    recs = []
     wall0 = time.perf_counter()
     for k in range(args.steps):
-        v, t, sample, threads = oracle_sample_step(w, n_rows, seed=k)
-        vals.append(v); times.append(t)
+        recs.append(oracle_sample_step(w, n_rows, seed=k))
     wall = time.perf_counter() - wall0
-    value = statistics.mean(vals)
+    value = statistics.mean(r["tokens_per_s"] for r in recs)
     G, U, R = unit_counts(w)
+    per_op = {k: statistics.mean(r["per_op_s"][k] for r in recs) for k in recs[0]["per_op_s"]}
     line = {
         "impl": "reference", "metric": "matched+restored tokens/s per cache op", "value": value,
         "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": 1e3 * statistics.mean(times), "higher_is_better": True, "scaling": "weak",
+        "ms_per_step": 1e3 * statistics.mean(r["seconds"] for r in recs), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "shape": list(w.shape), "groups": G, "units_per_group": U,
-                   "note": "CPU oracle, scaled from a bounded sample per step"},
-        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample},
+                   "note": "CPU oracle on the host cores; cpu_baseline.sample says what one step ran"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": recs[0]["cores"], "kind": "oracle",
+                         "sample": recs[0]["sample"], "per_op_s": per_op},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0, "wall_s": wall,
     }
@@ -225,17 +237,33 @@ def run_reference(args, rank):
 # ---------------------------------------------------------------------------------------------------
 # the CUDA arm
 # ---------------------------------------------------------------------------------------------------
-def run_ours(args, rank, local_rank, world):
-    import torch
-    from paper_2607_23844_b200 import build
-    if rank == 0:
-        build.build()
-    sharding.barrier()
-    from paper_2607_23844_b200 import omnicache as oc
+# The kernel that implements the workload's row of the path (never the Layered Cache copy), what
+# bounds it, and its algorithmic work per launch.
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 FMA lanes x 2 FLOP x max SM clock
 
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    w = make_workload(args.workload, seed_offset=rank)          # weak scaling: each rank its own batch
+
+def row_kernel(w: inputs.Workload):
+    if w.kind == "token":
+        return ("match_simt", "alu") if (w.self_match or w.dtype != inputs.BF16) else ("match_tc", "tensor")
+    return ("frame_pair", "hbm") if w.kind == "frame" else ("block_partial", "hbm")
+
+
+def pick_tensor_peak(peaks, timed_region_s, clocks):
+    """The burst figure for a kernel timed inside a short run at full clock, the sustained one for a
+    seconds-long run or a run whose SM clock sagged (power cap)."""
+    sm, mx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    at_max = sm is None or mx is None or sm >= 0.97 * mx
+    if timed_region_s < 1.0 and at_max:
+        return peaks["bf16_tflops"], f"{peaks['_source']} bf16 burst (timed region {timed_region_s:.3f} s, SM clock at max)"
+    why = "timed region >= 1 s" if timed_region_s >= 1.0 else f"SM clock {sm} of {mx} MHz"
+    return peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), f"{peaks['_source']} bf16 sustained ({why})"
+
+
+def measure_workload(args, oc, torch, dev, local_rank, rank, world, name, w, steps, warmup, full):
+    """One workload: K graph replays of the whole step (value), the same steps eagerly with every kernel
+    bracketed by CUDA events (per-op table and the roofline of the row's own kernel) and, for the headline
+    workload (`full`), in-graph brackets, the matcher's device span, the clock record and the end-to-end
+    leg.  Returns the record and the number of kernel launches inside the timed region."""
     G, U, R = unit_counts(w)
     n_units, n_cand_g = G * U, (U if w.self_match else U - R)
     n_cand = G * n_cand_g
@@ -254,6 +282,10 @@ def run_ours(args, rank, local_rank, world):
 
     per_set = 5 * tensor_bytes + G * stride * row_bytes          # x, cache, out, dst, layered-cache entry, y
     ring = max(2, -(-4 * L2_BYTES // per_set))
+    l2_note = f"inputs rotate through a ring of {ring} buffer sets ({ring * per_set >> 20} MiB > 4x L2)"
+    if ring > 16:                                                # a tiny workload: it would stay L2-resident in use too
+        ring = 16
+        l2_note = f"L2-resident: {ring} buffer sets of {per_set >> 10} KiB (the workload is smaller than L2)"
     sets = []
     for r in range(ring):
         s = dict(
@@ -281,7 +313,7 @@ def run_ours(args, rank, local_rank, world):
         ctx.layer_cache_put(i % ring, i, s["out"], tensor_bytes, stream=stream)
         ctx.layer_cache_get(i % ring, i, 5, s["dst"], stream=stream)
 
-    for i in range(max(args.warmup, ring)):            # also allocates every layered-cache entry
+    for i in range(max(warmup, ring)):            # also allocates every layered-cache entry
         step(i)
     torch.cuda.synchronize()
     assert ctx.device_status() == oc.OK
@@ -309,13 +341,13 @@ def run_ours(args, rank, local_rank, world):
     torch.cuda.synchronize()
     with ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)) as clk:
         e0.record(stream)
-        for i in range(args.steps):
+        for i in range(steps):
             graphs[i % ring].replay()
         e1.record(stream)
         torch.cuda.synchronize()
     sharding.barrier()
     ms_total = sharding.max_over_ranks(e0.elapsed_time(e1), dev)
-    launches = launches_per_step * args.steps
+    launches = launches_per_step * steps
     assert ctx.device_status() == oc.OK
 
     # ---- timed region 2: the same K steps called eagerly, every kernel bracketed by CUDA events on
@@ -325,7 +357,7 @@ def run_ours(args, rank, local_rank, world):
     ctx.profile_enable(True)
     e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e2.record(stream)
-    for i in range(args.steps):
+    for i in range(steps):
         if i % 20 == 0:
             torch.cuda._sleep(int(2.0e9 * 0.004))      # ~4 ms: longer than the host needs for 20 steps
         step(i)
@@ -349,149 +381,212 @@ def run_ours(args, rank, local_rank, world):
     ctx.profile_enable(False)
     n_tiny, ms_tiny = ctx.profile_read(oc.K_COPY)
     bracket_us = 1e3 * ms_tiny / max(n_tiny, 1)
-    # The same brackets INSIDE the timed region's kind of execution: one more graph per ring slot,
-    # captured with the timers on, so that every launch sits between two event-record nodes of the graph;
-    # replayed K times, the brackets read after each replay.  No eager launch latency, no host in the loop.
-    graph_us = {}
-    ctx.profile_enable(True)
-    pgraphs = []
-    for r in range(ring):
-        gph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(gph):
-            stream = torch.cuda.current_stream()
-            step(r)
-        pgraphs.append(gph)
-    ctx.profile_enable(False)
-    stream = torch.cuda.current_stream()
-    acc = {}
-    n_rep = 0
-    for i in range(min(args.steps, 200)):
-        pgraphs[i % ring].replay()
-        torch.cuda.synchronize()
-        if i < ring:            # every slot's graph has to have run once before all captured brackets are valid
-            continue
-        n_rep += 1
-        for k in range(oc.K_COUNT):
-            n_c, ms_c = ctx.profile_captured_read(k)
-            if n_c:
-                acc[k] = acc.get(k, 0.0) + ms_c / n_c      # mean over the slots' brackets (each holds its latest run)
-    if n_rep:
-        graph_us = {oc.kernel_name(k): 1e3 * v / n_rep for k, v in acc.items()}
-    del pgraphs
 
-    # A third pass, for the tensor-core matcher only: the same K steps with the kernel stamping the GPU
-    # timer when its first CTA starts and when its last CTA ends (no events): the time its CTAs occupy
-    # the device, without launch latency and event records.
+    graph_us = {}
     span_us = None
-    if w.kind == "token" and not w.self_match and prof.get("match_tc", (0, 0.0))[0]:
-        ctx.profile_reset()
-        ctx.profile_enable(2)
-        for i in range(args.steps):
-            if i % 20 == 0:
-                torch.cuda._sleep(int(2.0e9 * 0.004))
-            step(i)
-        torch.cuda.synchronize()
-        n_span, ms_span = ctx.profile_span_read(oc.K_MATCH_TC)
+    kern, bound = row_kernel(w)
+    if full:
+        # The same brackets INSIDE the timed region's kind of execution: one more graph per ring slot,
+        # captured with the timers on, so that every launch sits between two event-record nodes of the graph;
+        # replayed K times, the brackets read after each replay.  No eager launch latency, no host in the loop.
+        ctx.profile_enable(True)
+        pgraphs = []
+        for r in range(ring):
+            gph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gph):
+                stream = torch.cuda.current_stream()
+                step(r)
+            pgraphs.append(gph)
         ctx.profile_enable(False)
-        if n_span:
-            span_us = 1e3 * ms_span / n_span
+        stream = torch.cuda.current_stream()
+        acc = {}
+        n_rep = 0
+        for i in range(min(steps, 200)):
+            pgraphs[i % ring].replay()
+            torch.cuda.synchronize()
+            if i < ring:            # every slot's graph has to have run once before all captured brackets are valid
+                continue
+            n_rep += 1
+            for k in range(oc.K_COUNT):
+                n_c, ms_c = ctx.profile_captured_read(k)
+                if n_c:
+                    acc[k] = acc.get(k, 0.0) + ms_c / n_c      # mean over the slots' brackets (each holds its latest run)
+        if n_rep:
+            graph_us = {oc.kernel_name(k): 1e3 * v / n_rep for k, v in acc.items()}
+        del pgraphs
+
+        # A third pass, for the tensor-core matcher only: the same K steps with the kernel stamping the GPU
+        # timer when its first CTA starts and when its last CTA ends (no events): the time its CTAs occupy
+        # the device, without launch latency and event records.
+        if kern == "match_tc" and prof.get("match_tc", (0, 0.0))[0]:
+            ctx.profile_reset()
+            ctx.profile_enable(2)
+            for i in range(steps):
+                if i % 20 == 0:
+                    torch.cuda._sleep(int(2.0e9 * 0.004))
+                step(i)
+            torch.cuda.synchronize()
+            n_span, ms_span = ctx.profile_span_read(oc.K_MATCH_TC)
+            ctx.profile_enable(False)
+            if n_span:
+                span_us = 1e3 * ms_span / n_span
 
     tokens_per_step = n_cand + n_units
-    value = world * tokens_per_step * args.steps / (ms_total * 1e-3)
+    value = world * tokens_per_step * steps / (ms_total * 1e-3)
+    n_keep = int(sets[0]["kept_count"].sum().item())       # rows actually kept (threshold mode keeps fewer than G*stride)
 
-    # ---- end to end through the host-buffer call ------------------------------------------------
-    out_host = torch.empty_like(x_host).pin_memory()
-    kc_host = torch.zeros(G, dtype=torch.int32).pin_memory()
-    e2e_steps = max(3, min(args.steps, args.e2e_steps))
-    for _ in range(2):
-        ctx.cache_step_host(L, mode, w.thr, w.n_reuse, x_host, cache_host, out_host, kc_host, stream=stream)
-    sharding.barrier()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        ctx.cache_step_host(L, mode, w.thr, w.n_reuse, x_host, cache_host, out_host, kc_host, stream=stream)
-    torch.cuda.synchronize()
-    e2e_s = sharding.max_over_ranks(time.perf_counter() - t0, dev)
-    e2e_value = world * tokens_per_step * e2e_steps / e2e_s
+    # ---- end to end: the same step through the host-buffer call (match -> select -> gather -> restore on
+    # pinned host tensors) followed by the Layered Cache put of the restored output and a copying get,
+    # both on pinned host buffers too (the copy kernel reads / writes them over the bus) -------------------
+    e2e = None
+    if full:
+        out_host = torch.empty_like(x_host).pin_memory()
+        dst_host = torch.empty_like(x_host).pin_memory()
+        kc_host = torch.zeros(G, dtype=torch.int32).pin_memory()
+        e2e_steps = max(3, min(steps, args.e2e_steps))
+        e2e_layer = 1 << 21
 
-    # ---- roofline of the dominant kernel and per-op table -----------------------------------------
+        def e2e_step(i):
+            ctx.cache_step_host(L, mode, w.thr, w.n_reuse, x_host, cache_host, out_host, kc_host, stream=stream)
+            ctx.layer_cache_put(e2e_layer, i, out_host, tensor_bytes, stream=stream)
+            ctx.layer_cache_get(e2e_layer, i, 5, dst_host, stream=stream)
+        for i in range(2):
+            e2e_step(i)
+        sharding.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        e2e_s = sharding.max_over_ranks(time.perf_counter() - t0, dev)
+        # x whole + the cache rows of reused units (pinned buffers: the restore kernel fetches only those)
+        # + the put's read of the restored output; the output + kept counts + the get's copy
+        e2e = {"value": world * tokens_per_step * e2e_steps / e2e_s, "unit": "tokens/s",
+               "h2d_bytes_per_step": tensor_bytes + (n_units - n_keep) * row_bytes + tensor_bytes,
+               "d2h_bytes_per_step": tensor_bytes + 4 * G + tensor_bytes, "steps": e2e_steps,
+               "ms_per_step": 1e3 * e2e_s / e2e_steps,
+               "step": "oc_cache_step_host + layer_cache_put + copying layer_cache_get, all on pinned host buffers"}
+
+    # ---- per-op table and the roofline of the kernel that implements this workload's row -------------
     peaks = measured_peaks()
     ops = {}
-    for name, (n, ms) in prof.items():
+    for nm, (n, ms) in prof.items():
         if n:
-            ops[name] = {"launches": n, "avg_us": 1e3 * ms / n, "net_us": max(1e3 * ms / n - bracket_us, 0.0), "share": None}
-            if name in graph_us:
-                ops[name]["in_graph_us"] = graph_us[name]       # CUDA events around the launch inside a replayed graph
+            ops[nm] = {"launches": n, "avg_us": 1e3 * ms / n, "net_us": max(1e3 * ms / n - bracket_us, 0.0), "share": None}
+            if nm in graph_us:
+                ops[nm]["in_graph_us"] = graph_us[nm]       # CUDA events around the launch inside a replayed graph
     tot_ms = sum(ms for _, ms in prof.values()) or 1.0
-    for name, (n, ms) in prof.items():
+    for nm, (n, ms) in prof.items():
         if n:
-            ops[name]["share"] = ms / tot_ms
-    n_keep = int(sets[0]["kept_count"].sum().item())       # rows actually kept (threshold mode keeps fewer than G*stride)
+            ops[nm]["share"] = ms / tot_ms
     alg_bytes = {"gather": 2 * n_keep * row_bytes, "restore": 2 * n_units * row_bytes, "copy": 2 * tensor_bytes,
                  "norms": tensor_bytes, "frame_pair": tensor_bytes, "block_partial": tensor_bytes}
-    for name, b in alg_bytes.items():
-        if name in ops:
-            ops[name]["GB/s"] = b / (ops[name]["avg_us"] * 1e-6) / 1e9
-            ops[name]["frac_hbm"] = ops[name]["GB/s"] / peaks["hbm_gbs"]
-    if w.kind == "token" and not w.self_match and "match_tc" in ops:
+    for nm, b in alg_bytes.items():
+        if nm in ops:
+            ops[nm]["GB/s"] = b / (ops[nm]["avg_us"] * 1e-6) / 1e9
+            ops[nm]["frac_hbm"] = ops[nm]["GB/s"] / peaks["hbm_gbs"]
+    clocks = clk.summary()
+    assert kern in ops, f"{name}: the kernel of this workload's row ({kern}) did not run: {sorted(ops)}"
+    k_us = ops[kern]["avg_us"]
+    if bound == "tensor":
         flops = 2.0 * n_cand * R * w.shape[-1]
-        achieved = flops / (ops["match_tc"]["avg_us"] * 1e-6) / 1e12
-        peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
-        roofline = {"kernel": "match_tc", "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                    "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                    "peak_source": f"{peaks['_source']} bf16 sustained", "frac_of_burst": achieved / peaks["bf16_tflops"],
-                    "frac_of_nominal": achieved / NOMINAL["bf16_tflops"], "flops_per_launch": flops,
+        achieved = flops / (k_us * 1e-6) / 1e12
+        peak, peak_source = pick_tensor_peak(peaks, eager_ms * 1e-3, clocks)
+        roofline = {"kernel": kern, "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get(name),
+                    "peak_source": peak_source, "frac_of_burst": achieved / peaks["bf16_tflops"],
+                    "frac_of_sustained": achieved / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                    "frac_of_nominal": achieved / NOMINAL["bf16_tflops"], "flops_per_launch": flops, "avg_us": k_us,
                     # the same with the bracket's own cost (see timing.event_bracket_us) taken off the duration
-                    "achieved_net_of_bracket": flops / (max(ops["match_tc"]["net_us"], 1e-3) * 1e-6) / 1e12,
-                    "frac_net_of_bracket": flops / (max(ops["match_tc"]["net_us"], 1e-3) * 1e-6) / 1e12 / peak}
-        if "in_graph_us" in ops["match_tc"]:
-            roofline["in_graph_us"] = ops["match_tc"]["in_graph_us"]
-            roofline["achieved_in_graph"] = flops / (ops["match_tc"]["in_graph_us"] * 1e-6) / 1e12
+                    "achieved_net_of_bracket": flops / (max(ops[kern]["net_us"], 1e-3) * 1e-6) / 1e12}
+        roofline["frac_net_of_bracket"] = roofline["achieved_net_of_bracket"] / peak
+        if "in_graph_us" in ops[kern]:
+            roofline["in_graph_us"] = ops[kern]["in_graph_us"]
+            roofline["achieved_in_graph"] = flops / (ops[kern]["in_graph_us"] * 1e-6) / 1e12
             roofline["frac_in_graph"] = roofline["achieved_in_graph"] / peak
         if span_us:
             # first-CTA-entry -> last-CTA-exit by the GPU timer (oc_profile_span_read): device occupancy only
             roofline["device_span_us"] = span_us
             roofline["achieved_device_span"] = flops / (span_us * 1e-6) / 1e12
             roofline["frac_device_span"] = roofline["achieved_device_span"] / peak
-            roofline["frac_device_span_of_nominal"] = roofline["achieved_device_span"] / NOMINAL["bf16_tflops"]
+    elif bound == "hbm":
+        roofline = {"kernel": kern, "bound": "hbm", "achieved": ops[kern]["GB/s"], "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": ops[kern]["frac_hbm"], "traffic": NCU_TRAFFIC_BYTES.get(name),
+                    "peak_source": f"{peaks['_source']} copy bandwidth", "bytes_per_launch": alg_bytes[kern], "avg_us": k_us,
+                    "frac_net_of_bracket": alg_bytes[kern] / (max(ops[kern]["net_us"], 1e-3) * 1e-6) / 1e9 / peaks["hbm_gbs"]}
     else:
-        dom = max((k for k in ops if k in alg_bytes), key=lambda k: ops[k]["share"])
-        roofline = {"kernel": dom, "bound": "hbm", "achieved": ops[dom]["GB/s"], "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": ops[dom]["frac_hbm"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
-                    "peak_source": f"{peaks['_source']} copy bandwidth", "bytes_per_launch": alg_bytes[dom]}
+        # fp32 inputs / self-match: all-pairs fp32 FMA on the ALUs (tf32 would miss the 1e-5 tolerance)
+        flops = 2.0 * n_cand * (U if w.self_match else R) * w.shape[-1]
+        achieved = flops / (k_us * 1e-6) / 1e12
+        roofline = {"kernel": kern, "bound": "alu", "achieved": achieved, "peak": FP32_ALU_TFLOPS, "unit": "TFLOP/s",
+                    "frac": achieved / FP32_ALU_TFLOPS, "traffic": None, "flops_per_launch": flops, "avg_us": k_us,
+                    "peak_source": "148 SMs x 128 fp32 FMA lanes x 2 FLOP x 1965 MHz"}
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, t, sample, threads = oracle_sample_step(w, args.ref_rows)
-        cpu_baseline = {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": sample,
-                        "seconds": t}
+        cpu_baseline = cpu_baseline_record(w, args.ref_rows if full else max(args.ref_rows // 4, 64))
+
+    rec = {
+        "value": value, "unit": "tokens/s", "ms_per_step": ms_total / steps, "steps": steps,
+        "dtype": "bf16" if w.dtype == inputs.BF16 else "f32",
+        "config": {"workload": name, "shape": list(w.shape), "kind": w.kind, "mode": w.mode,
+                   "n_reuse_per_group": w.n_reuse, "thr": w.thr, "groups": G, "units_per_group": U,
+                   "reps_per_group": R, "tokens_per_step": tokens_per_step,
+                   "l2": l2_note,
+                   "wrapped_layer": "identity stand-in (outside the path)", "parallelism": f"replicas x{world}"},
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks, "ops": ops,
+        "timing": {"value": "CUDA-graph replay of the step's C-ABI launches (match, select, gather, restore, "
+                            "layer_cache_put, copying layer_cache_get)", "launches_per_step": launches_per_step,
+                   "eager_profiled_ms_per_step": eager_ms / steps, "event_bracket_us": bracket_us,
+                   "event_bracket": "per-kernel avg_us = CUDA events around each launch on its stream; "
+                                    "event_bracket_us = a one-thread 16-byte copy timed the same way; net_us = the difference"},
+    }
+    ctx.close()
+    del sets, graphs
+    torch.cuda.empty_cache()
+    return rec, launches
+
+
+# the other configurations of the benchmark definition, carried as sub-records of the one line
+SUB_WORKLOADS = ("tiny_token", "sd3_token", "svd_frame", "latte_block", "svd_token_l1", "svd_token_l2")
+
+
+def run_ours(args, rank, local_rank, world):
+    import torch
+    from paper_2607_23844_b200 import build
+    if rank == 0:
+        build.build()
+    sharding.barrier()
+    from paper_2607_23844_b200 import omnicache as oc
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    w = make_workload(args.workload, seed_offset=rank)          # weak scaling: each rank its own batch
+    main, launches = measure_workload(args, oc, torch, dev, local_rank, rank, world, args.workload, w,
+                                      args.steps, args.warmup, full=True)
+    del w
+    subs = {}
+    if world == 1 and not args.no_subconfigs:
+        sub_steps = max(10, min(args.steps, args.sub_steps))
+        for name in SUB_WORKLOADS:
+            if name == args.workload:
+                continue
+            rec, _ = measure_workload(args, oc, torch, dev, local_rank, rank, world, name, make_workload(name),
+                                      sub_steps, max(3, min(args.warmup, 10)), full=False)
+            rec.pop("e2e"); rec.pop("timing")
+            subs[name] = rec
 
     if rank == 0:
         line = {
-            "metric": "matched+restored tokens/s per cache op", "value": value, "unit": "tokens/s",
-            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
+            "metric": "matched+restored tokens/s per cache op", "value": main["value"], "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": main["ms_per_step"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if w.dtype == inputs.BF16 else "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "shape": list(w.shape), "kind": w.kind, "mode": w.mode,
-                       "n_reuse_per_group": w.n_reuse, "thr": w.thr, "groups": G, "units_per_group": U,
-                       "reps_per_group": R, "tokens_per_step": tokens_per_step,
-                       "l2": f"inputs rotate through a ring of {ring} buffer sets ({ring * per_set >> 20} MiB > 4x L2)",
-                       "wrapped_layer": "identity stand-in (outside the path)", "parallelism": f"replicas x{world}"},
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
-            # x whole + the cache rows of reused units (pinned buffers: the restore kernel fetches only those)
-            "e2e": {"value": e2e_value, "unit": "tokens/s",
-                    "h2d_bytes_per_step": tensor_bytes + (n_units - n_keep) * row_bytes,
-                    "d2h_bytes_per_step": tensor_bytes + 4 * G, "steps": e2e_steps,
-                    "ms_per_step": 1e3 * e2e_s / e2e_steps},
-            "gpu_launches": launches, "clocks": clk.summary(), "ops": ops,
-            "timing": {"value": "CUDA-graph replay of the step's C-ABI launches", "launches_per_step": launches_per_step,
-                       "eager_profiled_ms_per_step": eager_ms / args.steps,
-                       "event_bracket_us": bracket_us,
-                       "event_bracket": "per-kernel avg_us = CUDA events around each launch on its stream; "
-                                        "event_bracket_us = a one-thread 16-byte copy timed the same way; net_us = the difference"},
+            "dtype": main["dtype"], "data": "synthetic", "config": main["config"],
+            "roofline": main["roofline"], "cpu_baseline": main["cpu_baseline"], "e2e": main["e2e"],
+            "gpu_launches": launches, "clocks": main["clocks"], "ops": main["ops"], "timing": main["timing"],
+            "configs": subs,
         }
         print(json.dumps(line), flush=True)
-    ctx.close()
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -969,16 +1064,18 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="sd3_token")
+    ap.add_argument("--workload", default="svd_token_l0")
     ap.add_argument("--ref-rows", type=int, default=8192,
                     help="candidates the CPU oracle matches per step (all of them if the workload has fewer)")
     ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--sub-steps", type=int, default=40, help="timed steps of each sub-record under `configs`")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-subconfigs", action="store_true", help="the headline workload only (profiling runs)")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = 1000 if args.impl == "ours" else 3
+        args.steps = 200 if args.impl == "ours" else 3
     if args.warmup is None:
-        args.warmup = 50 if args.impl == "ours" else 1
+        args.warmup = 20 if args.impl == "ours" else 1
     if args.impl == "ours":
         args.warmup = max(args.warmup, 3)
     rank, local_rank, world = sharding.env_rank_world()

@@ -178,6 +178,16 @@ oc_status oc_profile_enable(oc_ctx* ctx, int on);
 oc_status oc_profile_reset(oc_ctx* ctx);
 oc_status oc_profile_read(oc_ctx* ctx, int kernel_id, int64_t* launches, double* total_ms);
 
+/* Test hook: forces the work split of the tensor-core matcher for this context's later oc_match /
+ * oc_match_joint calls instead of the planner's choice: a single CTA (pair = 0) or a CTA pair
+ * (pair = 1) per piece, 1 or 2 candidate tiles per CTA, pieces_per_row pieces per row of the
+ * problem; single_accumulator != 0 keeps narrow pieces on one accumulator set.  A split the shape
+ * does not admit is ignored (the planner's choice runs).  on = 0 returns to the planner.  Results
+ * never depend on the split; the parity tests use this to run every form of the kernel.
+ * OC_ERR_INVALID_ARG for values outside the ranges above.  The paper has no counterpart. */
+oc_status oc_tc_plan_override(oc_ctx* ctx, int on, int pair, int tiles_per_cta, int pieces_per_row,
+                              int single_accumulator);
+
 /* Device-side span of the tensor-core matcher (kernel_id must be OC_K_MATCH_TC).  With
  * oc_profile_enable(ctx, 2) every launch of that kernel stamps the GPU's nanosecond timer when its
  * first CTA starts and when its last CTA ends (two atomics per CTA; no events are recorded in this
@@ -201,11 +211,13 @@ oc_status oc_profile_captured_read(oc_ctx* ctx, int kernel_id, int64_t* launches
  * The hot path
  * ------------------------------------------------------------------------------------------- */
 
-/* match (Background: "matches similar pairs by cosine similarity"; Sections 3.2.1-3.2.3).
- * For every candidate unit: the most similar representative it may be matched with.
+/* match (Background: candidates are paired with representatives by cosine similarity; Sections
+ * 3.2.1-3.2.3).  For every candidate unit: the most similar representative it may be matched with.
  *   x         [B][T][H][W][C] features of layout->dtype (the wrapped layer's input)
  *   best_sim  [n_units] float: cosine of the best match; -inf for representatives
- *   best_idx  [n_units] int32: global unit index of that representative (ties: lowest index);
+ *   best_idx  [n_units] int32: global unit index of that representative (ties: lowest index; the
+ *             tensor-core matcher compares similarities truncated to 19 mantissa bits, so values
+ *             that agree to 2^-18 relative count as tied);
  *             a representative's own index for representatives
  *   aux_sim   nullable.  TOKEN: [n_groups][units_per_group][reps_per_group] float, every candidate
  *             row's full similarity row (rows of representatives and the self-match diagonal are
@@ -218,9 +230,8 @@ oc_status oc_profile_captured_read(oc_ctx* ctx, int kernel_id, int64_t* launches
 oc_status oc_match(oc_ctx* ctx, const oc_layout* layout, const void* x, float* best_sim,
                    int32_t* best_idx, float* aux_sim, float* pair_sim, void* stream);
 
-/* Frame Cache at several patch sizes from ONE pass over the tensor (Section 3.3: after patch-level
- * caching "the patch size can be increased for coarser reuse, or patches can be restored to full
- * frames").  `layout` is an OC_KIND_FRAME layout whose (gy, gx) is the finest grid; `grids` (HOST
+/* Frame Cache at several patch sizes from ONE pass over the tensor (Section 3.3: the patch-level pass
+ * may be followed by coarser ones, with larger patches or with whole frames).  `layout` is an OC_KIND_FRAME layout whose (gy, gx) is the finest grid; `grids` (HOST
  * memory, [n_levels][2] ints) lists (gy_l, gx_l) per level, each dividing (gy, gx) -- (1, 1) is the
  * whole frame.  Level l's results are what oc_match() gives for the same layout with (gy_l, gx_l)
  * (equal up to fp32 summation order), stored one level after another:
@@ -255,9 +266,9 @@ oc_status oc_linear_gather_scatter(oc_ctx* ctx, const void* a, int64_t a_rows, i
                                    const int32_t* out_idx, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
- * Token Cache on the frame pairs of Frame Cache (Section 3.2.3): "Token Cache consumes the same
- * feature map and frame-pair metadata used by Frame Cache"; matched pairs become token groups of
- * 2*H*W tokens with one representative per 2x2x2 cube, unmatched frames keep their 2x2 groups.
+ * Token Cache on the frame pairs of Frame Cache (Section 3.2.3): it works on the feature map and the
+ * frame pairing Frame Cache has just produced; matched pairs become token groups of 2*H*W tokens
+ * with one representative per 2x2x2 cube, unmatched frames keep their 2x2 groups.
  * `layout` is the OC_KIND_TOKEN layout of the tensor (bf16, gy = gx = 1, no self_match;
  * OC_ERR_UNSUPPORTED otherwise).  `frames` is a device array of B*T slots {rep, partner} (int32
  * pairs, 8-byte aligned): slot f = {f, t} if frame f is the representative frame of the pair
@@ -290,8 +301,8 @@ oc_status oc_select_joint(oc_ctx* ctx, const oc_layout* layout, const int32_t* f
                           int64_t n_reuse_single, int64_t y_stride, int32_t* kept_idx, int32_t* kept_count,
                           int32_t* match_map, int32_t* slot_of, void* stream);
 
-/* select ("the r most redundant ... are marked for cached restoration while the retained
- * representatives are computed normally", Sections 3.2.1-3.2.3).  Representatives are always kept.
+/* select (Sections 3.2.1-3.2.3: the r candidates most similar to their match are restored from the
+ * cache, everything else goes through the layer).  Representatives are always kept.
  *   mode OC_SELECT_THRESHOLD: a candidate is reused iff best_sim >= thr (self_match: and its best
  *        match has a lower index; match_map then follows best_idx down to a kept token).
  *   mode OC_SELECT_COUNT: in every group the n_reuse_per_group candidates with the largest
@@ -308,13 +319,13 @@ oc_status oc_select(oc_ctx* ctx, const oc_layout* layout, const float* best_sim,
                     int64_t y_group_stride, int32_t* kept_idx, int32_t* kept_count,
                     int32_t* match_map, int32_t* slot_of, void* stream);
 
-/* gather (Appendix A: "compact retained tokens"): y[slot] = row kept_idx[slot] of x for every slot
+/* gather (Appendix A: compaction of the kept rows): y[slot] = row kept_idx[slot] of x for every slot
  * in [0, n_slots) with kept_idx[slot] >= 0; other slots of y are left untouched.  Bit copy. */
 oc_status oc_gather(oc_ctx* ctx, const oc_rows* rows, const void* x, const int32_t* kept_idx,
                     int64_t n_slots, void* y, void* stream);
 
-/* restore (Sections 3.2.1-3.2.3: skipped positions "are restored from cached activations
- * associated with the same positions at the previous denoising step"; no averaging).
+/* restore (Sections 3.2.1-3.2.3: a skipped position takes the activation cached for that same
+ * position at the previous denoising step; rows are copied, never averaged).
  *   z      dense layer output, row slot_of[i] belongs to unit i
  *   cache  strided like out: the previous step's restored output (nullable in
  *          OC_RESTORE_FROM_REPRESENTATIVE mode)
@@ -355,8 +366,11 @@ oc_status oc_layer_cache_clear(oc_ctx* ctx);
  *     refused with OC_ERR_WORKSPACE and nothing is launched.  Other kinds: OC_ERR_INVALID_ARG.
  *   - The call itself makes no cudaMalloc / cudaFree and uses no allocating library routine; the
  *     caller passes every input and output buffer.
- *   - The first call on each device looks up the array's device address (with that device current)
- *     and remembers it; make that first call before any stream capture begins.
+ *   - The first call on each device looks up the array's device address (with that device current),
+ *     reads the device's SM count and makes the driver load every kernel the call can launch, and
+ *     remembers all that; make that first call before any stream capture begins.  (Later calls with
+ *     a layout of another dtype or row length launch other instances of the same kernels; those
+ *     were loaded by the first call.)
  *   - All calls on a device share the one array and it keeps whatever the previous call left.  No
  *     part of it needs to start at zero (each call writes every value it later reads), but two calls
  *     whose kernels overlap on the GPU - different streams, or one stream replayed concurrently -
@@ -365,14 +379,15 @@ oc_status oc_layer_cache_clear(oc_ctx* ctx);
 oc_status oc_match_frame_noalloc(int device, const oc_layout* layout, const void* x, float* best_sim,
                                  int32_t* best_idx, float* pair_sim, void* stream);
 
-/* Layered Cache schedule proposal (Algorithm 1, "Cache Schedule Proposal", Section 3.4).  Host-side;
- * launches nothing and needs no context.
+/* Layered Cache schedule proposal (Algorithm 1, Section 3.4).  Host-side; launches nothing and needs
+ * no context.
  *   latency[i], quality_loss[i]  the profiled L and Q of candidate i (a layer-timestep pair), n of
  *                                them, host arrays; every latency must be > 0 and finite, every
  *                                quality loss finite
  *   target_speedup               s_r >= 1
- * Candidates are ranked by w = Q / L ascending (equal scores: lower index first) and taken in that
- * order while Saved < (1 - 1/s_r) * sum(L), each adding its L to Saved, all in double precision.
+ * Candidates are ranked by quality loss per unit of latency, cheapest first (equal scores: lower
+ * index first); the result is the shortest prefix of that ranking whose latencies add up to at least
+ * the budget (1 - 1/s_r) * sum(latency) -- the whole ranking if none does.  Double precision.
  *   chosen     host array of capacity n: receives the taken candidate indices in the order taken
  *              (each is to be cached with the caller's interval N, which does not influence the choice)
  *   n_chosen   receives how many were taken

@@ -221,7 +221,9 @@ oc_status oc_create(oc_ctx** out, int device, size_t workspace_bytes) {
     cudaMemset(c->d_span, 0, 512 * sizeof(unsigned long long));
     if (workspace_bytes) {
         if (cudaMalloc(&c->workspace, workspace_bytes) != cudaSuccess) {
-            cudaFree(c->d_status); delete c; cudaGetLastError(); return OC_ERR_OOM;
+            cudaGetLastError();
+            cudaFree(c->d_span); cudaFree(c->d_status); delete c;
+            return OC_ERR_OOM;
         }
         c->workspace_bytes = workspace_bytes;
     }
@@ -239,7 +241,6 @@ oc_status oc_destroy(oc_ctx* c) {
         for (auto& p : c->prof[k].captured) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
     }
     for (auto e : c->free_events) cudaEventDestroy(e);
-    tc_cache_free(c);
     cudaFree(c->stage);
     cudaFree(c->workspace);
     for (auto e : c->chunk_events) cudaEventDestroy(e);
@@ -266,6 +267,16 @@ oc_status oc_selftest_bounded_wait(oc_ctx* c, unsigned int limit_us, void* strea
     DeviceGuard guard(c->device);
     if (!guard.ok) return OC_ERR_CUDA;
     return launch_bounded_wait_selftest(c, (unsigned long long)limit_us * 1000ull, (cudaStream_t)stream);
+}
+
+oc_status oc_tc_plan_override(oc_ctx* c, int on, int pair, int tiles_per_cta, int pieces_per_row, int single_accumulator) {
+    if (!c) return OC_ERR_INVALID_ARG;
+    if (on && ((pair != 0 && pair != 1) || (tiles_per_cta != 1 && tiles_per_cta != 2) || pieces_per_row < 1))
+        return OC_ERR_INVALID_ARG;
+    c->tc_plan_forced = on != 0;
+    c->tc_plan_pair = pair; c->tc_plan_tiles = tiles_per_cta; c->tc_plan_pieces = pieces_per_row;
+    c->tc_plan_no_narrow = single_accumulator ? 1 : 0;
+    return OC_OK;
 }
 
 oc_status oc_profile_enable(oc_ctx* c, int on) {
@@ -561,33 +572,37 @@ oc_status oc_layer_cache_clear(oc_ctx* c) {
     return cuda_ok(cudaGetLastError());
 }
 
-// ---- host-buffer call --------------------------------------------------------------------------
+// ---- Layered Cache schedule proposal (host only) -------------------------------------------------
 oc_status oc_schedule_propose(const double* latency, const double* quality_loss, int64_t n, double target_speedup,
                               int32_t* chosen, int64_t* n_chosen, double* saved) {
     if (!latency || !quality_loss || !chosen || !n_chosen || n < 0 || n > 0x7FFFFFFF) return OC_ERR_INVALID_ARG;
     if (!(target_speedup >= 1.0)) return OC_ERR_INVALID_ARG;
-    double total = 0.0;
-    for (int64_t i = 0; i < n; ++i) {
+    for (int64_t i = 0; i < n; ++i)
         if (!(latency[i] > 0.0) || !std::isfinite(latency[i]) || !std::isfinite(quality_loss[i])) return OC_ERR_INVALID_ARG;
-        total += latency[i];
-    }
-    std::vector<double> w((size_t)n);
-    std::vector<int32_t> order((size_t)n);
-    for (int64_t i = 0; i < n; ++i) { w[(size_t)i] = quality_loss[i] / latency[i]; order[(size_t)i] = (int32_t)i; }
-    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return w[(size_t)a] < w[(size_t)b]; });
-    const double target_save = (1.0 - 1.0 / target_speedup) * total;
-    double acc = 0.0;
-    int64_t k = 0;
-    while (acc < target_save && k < n) {
-        const int32_t i = order[(size_t)k];
-        chosen[k++] = i;
-        acc += latency[i];
-    }
+    // Algorithm 1 as a prefix-sum problem: rank the candidates by quality loss per unit of latency
+    // (a stable ranking keeps equal scores in candidate order), accumulate their latencies along the
+    // ranking, and the answer is the shortest prefix whose sum reaches the latency budget -- the
+    // whole ranking when even that does not.
+    std::vector<int32_t> ranking((size_t)n);
+    std::vector<double> score((size_t)n);
+    for (int64_t i = 0; i < n; ++i) { ranking[(size_t)i] = (int32_t)i; score[(size_t)i] = quality_loss[i] / latency[i]; }
+    std::stable_sort(ranking.begin(), ranking.end(), [&score](int32_t a, int32_t b) { return score[(size_t)a] < score[(size_t)b]; });
+    std::vector<double> prefix((size_t)n + 1);
+    double total = 0.0;                                   // (summed in candidate order, like the budget's definition)
+    for (int64_t i = 0; i < n; ++i) total += latency[i];
+    prefix[0] = 0.0;
+    for (int64_t r = 0; r < n; ++r) prefix[(size_t)r + 1] = prefix[(size_t)r] + latency[ranking[(size_t)r]];
+    const double budget = (1.0 - 1.0 / target_speedup) * total;
+    // first prefix length whose sum is >= budget (prefix sums of positive terms ascend)
+    const int64_t len = std::lower_bound(prefix.begin(), prefix.end(), budget) - prefix.begin();
+    const int64_t k = len > n ? n : len;
+    for (int64_t r = 0; r < k; ++r) chosen[r] = ranking[(size_t)r];
     *n_chosen = k;
-    if (saved) *saved = acc;
+    if (saved) *saved = prefix[(size_t)k];
     return OC_OK;
 }
 
+// ---- host-buffer call --------------------------------------------------------------------------
 oc_status oc_cache_step_host(oc_ctx* c, const oc_layout* layout, int mode, float thr, int64_t n_reuse,
                              const void* x_host, const void* cache_host, void* out_host, int32_t* kept_count_host,
                              void* stream) {

@@ -4,6 +4,7 @@
 #include <stdint.h>
 
 #include <map>
+#include <mutex>
 #include <vector>
 
 #include "omnicache.h"
@@ -46,8 +47,9 @@ struct oc_ctx {
     size_t stage_bytes = 0;
     cudaStream_t copy_stream = nullptr;      // host->device copies of the chunks of oc_cache_step_host
     std::vector<cudaEvent_t> chunk_events;
-    // cached tensor maps of the tcgen05 matcher (opaque to the other files)
-    void* tc_cache = nullptr;
+    // test hook (oc_tc_plan_override): forces the tensor-core matcher's work split
+    bool tc_plan_forced = false;
+    int tc_plan_pair = 0, tc_plan_tiles = 0, tc_plan_pieces = 0, tc_plan_no_narrow = 0;
 };
 
 namespace oc {
@@ -61,6 +63,24 @@ struct DeviceGuard {
         if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
     }
     ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// Work that has to be done once per DEVICE rather than once per process: function attributes such as
+// the opt-in to more than 48 KB of dynamic shared memory belong to the device's context, and one
+// process may hold contexts on several GPUs.  ensure(dev, f) runs f() the first time it is called for
+// `dev` (with that device current: every launcher runs under a DeviceGuard) and remembers whether it
+// succeeded; device ids beyond the table run f() every time.
+struct PerDeviceOnce {
+    static constexpr int MAX_DEV = 64;
+    std::mutex m;
+    unsigned char state[MAX_DEV] = {};           // 0 = not yet, 1 = done, 2 = failed
+    template <class F>
+    bool ensure(int dev, F&& f) {
+        if (dev < 0 || dev >= MAX_DEV) return f();
+        std::lock_guard<std::mutex> lock(m);
+        if (state[dev] == 0) state[dev] = f() ? 1 : 2;
+        return state[dev] == 1;
+    }
 };
 
 // Counts a kernel launch and, if timers are on, brackets it with events on the launching stream.
@@ -185,7 +205,6 @@ oc_status launch_match_joint_tc(oc_ctx*, const Geo&, const void* x, const float*
                                 const int4* units, const int* n_units_dev, long long max_units, cudaStream_t);
 oc_status launch_match_token_tc(oc_ctx*, const Geo&, const void* x, const float* inv_norm,
                                 unsigned long long* keys, float* aux_sim, cudaStream_t);
-void tc_cache_free(oc_ctx*);
 oc_status launch_bounded_wait_selftest(oc_ctx*, unsigned long long limit_ns, cudaStream_t);
 
 size_t match_workspace_bytes(const Geo&);

@@ -1,8 +1,7 @@
-// Token Cache on the frame pairs of Frame Cache (Section 3.2.3): "Token Cache consumes the same
-// feature map and frame-pair metadata used by Frame Cache ... For frame pairs selected by Frame Cache,
-// we reshape the paired features from (B, 2 r_f, H, W, C) to (B r_f, 2HW, C).  Within each local
-// 2x2x2 cube, Token Cache retains representative tokens ...  For unmatched frames, the same procedure
-// is applied within local 2x2 spatial neighborhoods."
+// Token Cache on the frame pairs of Frame Cache (Section 3.2.3).  Token Cache reuses the feature map
+// and the frame pairing of Frame Cache: a matched pair is treated as one token group of 2*H*W tokens
+// (the paper's (B*r_f, 2HW, C) arrangement) with one representative per 2x2x2 cube, and a frame that
+// found no partner is matched inside its own 2x2 neighbourhoods as usual.
 //
 // Nothing is reshaped here: a pair is two frame indices, and the matcher, the selection and the row
 // movers address the two frames in place.

@@ -1,7 +1,7 @@
 // The wrapped layer's projection with the gather folded into its A-operand load and the restore folded
-// into its store (Appendix A: "compact retained tokens" / "fused permutation/scatter", taken one step
-// further: the dense buffer between gather and the layer, and between the layer and restore, is never
-// written):
+// into its store (Appendix A's token compaction and its permutation/scatter on the way back, taken one
+// step further: the dense buffer between gather and the layer, and between the layer and restore, is
+// never written):
 //     out[dst(r), :] = bf16( sum_k a[src(r), k] * w[n, k] ),     r = 0 .. n_rows-1
 // src(r) = a_idx[r] (the kept-index list of select), dst(r) = out_idx[r] (the same list: computed rows
 // go straight to their positions in the restored tensor, which already holds the cached rows).
@@ -302,13 +302,14 @@ oc_status launch_linear_gs(oc_ctx* ctx, const void* a, int64_t a_rows, int64_t K
     P.depth = P.n_stages >= 5 ? 3 : (P.n_stages >= 4 ? 2 : 1);
     P.status = ctx->d_status;
     const size_t smem = (size_t)P.n_stages * P.stage_bytes + (2 * LIN_MAX_STAGES + 1) * 8 + 64;
-    static std::once_flag attr_once;
-    static bool attr_ok = false;
-    std::call_once(attr_once, [] {
-        attr_ok = cudaFuncSetAttribute(linear_gs_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024) == cudaSuccess &&
-                  cudaFuncSetAttribute(linear_gs_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024) == cudaSuccess &&
-                  cudaFuncSetAttribute(linear_gs_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024) == cudaSuccess;
-        if (!attr_ok) cudaGetLastError();
+    static PerDeviceOnce attr_once;                 // (the context's device is current here)
+    const bool attr_ok = attr_once.ensure(ctx->device, [] {
+        const bool ok =
+            cudaFuncSetAttribute(linear_gs_kernel<256, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024) == cudaSuccess &&
+            cudaFuncSetAttribute(linear_gs_kernel<256, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024) == cudaSuccess &&
+            cudaFuncSetAttribute(linear_gs_kernel<128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 201 * 1024) == cudaSuccess;
+        if (!ok) cudaGetLastError();
+        return ok;
     });
     if (!attr_ok) return OC_ERR_CUDA;
     const long long rows_per_cta = (long long)LIN_BM * m_tiles_per_cta;

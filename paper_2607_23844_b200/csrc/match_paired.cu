@@ -3,6 +3,8 @@
 // reductions: 16-byte loads, fp32 accumulators for <a,b>, |a|^2, |b|^2, sub-warp shuffle
 // reductions, and a fixed-order two-level sum (no floating-point atomics) so results are
 // reproducible run to run.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace oc {
@@ -207,9 +209,9 @@ frame_march_kernel(const uint8_t* __restrict__ x, int T, int P, int cpr, float e
 // representatives.  Every warp is independent, so units run in parallel.
 //
 // The partial records are laid out for the FINEST patch grid; a coarser level of the hierarchy
-// (Section 3.3: "the patch size can be increased for coarser reuse, or patches can be restored to
-// full frames") whose patches are unions of ry x rx fine patches is finalized from the same records,
-// so one pass over the tensor serves every level.
+// (Section 3.3: larger patches, up to whole frames, after the patch-level pass) whose patches are
+// unions of ry x rx fine patches is finalized from the same records, so one pass over the tensor
+// serves every level.
 struct FinLevel {
     int gy, gx;             // this level's patch grid
     int ry, rx;             // fine patches per patch of this level, per axis
@@ -324,7 +326,9 @@ struct FramePlan {
     int lpr, n_tiles, ppc, seg_len, n_seg;     // n_tiles = patches * tiles per patch
     PatchGrid pg;
 };
-static FramePlan frame_plan(const Geo& g) {
+// sm_count only steers how a clip is cut into segments (never the number of partial records, so the
+// workspace size does not depend on it)
+static FramePlan frame_plan(const Geo& g, int sm_count) {
     FramePlan f;
     const int cpr = g.C * g.elem_bytes / 16, P = g.H * g.W;
     int l = 4;
@@ -337,7 +341,7 @@ static FramePlan frame_plan(const Geo& g) {
         f.n_tiles = f.pg.n_patches * f.pg.tiles_per_patch;
         // segments: enough CTAs for a few waves, but at least 6 pairs per segment (one frame re-read each)
         int n_seg = 1;
-        while ((long long)f.n_tiles * g.B * n_seg < 148 * 4 && (g.T - 1) / (n_seg + 1) >= 6) ++n_seg;
+        while ((long long)f.n_tiles * g.B * n_seg < (long long)sm_count * 4 && (g.T - 1) / (n_seg + 1) >= 6) ++n_seg;
         f.seg_len = (g.T - 1 + n_seg - 1) / n_seg;
         const int seg_cap = 40960 / ((PAIR_THREADS / l) * (int)sizeof(float2));   // per-pair, per-position values live in shared memory
         if (f.seg_len > seg_cap) f.seg_len = seg_cap;
@@ -354,7 +358,7 @@ static FramePlan frame_plan(const Geo& g) {
 
 size_t frame_workspace_bytes(const Geo& g) {
     size_t pairs = (size_t)g.B * (size_t)(g.T > 1 ? g.T - 1 : 0);
-    return pairs * (size_t)frame_plan(g).n_tiles * sizeof(float4) + 256;
+    return pairs * (size_t)frame_plan(g, 1).n_tiles * sizeof(float4) + 256;
 }
 
 template <int DT>
@@ -372,12 +376,12 @@ static void march_dispatch(int lpr, dim3 grid, size_t smem, cudaStream_t s, cons
 // counters then).  levels == nullptr: one level, the layout's own grid; otherwise n_levels grids
 // (gy_l, gx_l), each dividing the layout's, whose outputs follow one another in best_sim / best_idx
 // (B*T*gy_l*gx_l entries each) and pair_sim (B*(T-1)*gy_l*gx_l each).
-static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, const void* x, float* best_sim,
+static oc_status run_frame_match(oc_ctx* ctx, int sm_count, uint8_t* scratch, const Geo& g, const void* x, float* best_sim,
                                  int32_t* best_idx, float* pos_sim, float* pair_sim, cudaStream_t s,
                                  int n_levels = 1, const int32_t* levels = nullptr) {
     const int P = g.H * g.W, cpr = g.C * g.elem_bytes / 16;
     const int n_pairs = g.B * (g.T - 1);
-    const FramePlan f = frame_plan(g);
+    const FramePlan f = frame_plan(g, sm_count);
     float4* partial = (float4*)scratch;
     if (n_pairs > 65535 || (long long)g.B * (f.march ? f.n_seg : 1) > 65535) return OC_ERR_UNSUPPORTED;
     struct Scope { oc_ctx* c; int k; cudaStream_t s; LaunchScope* l; 
@@ -424,12 +428,12 @@ static oc_status run_frame_match(oc_ctx* ctx, uint8_t* scratch, const Geo& g, co
 
 oc_status launch_match_frame(oc_ctx* ctx, const Geo& g, const void* x, float* best_sim, int32_t* best_idx,
                              float* pos_sim, float* pair_sim, cudaStream_t s) {
-    return run_frame_match(ctx, (uint8_t*)ctx->workspace, g, x, best_sim, best_idx, pos_sim, pair_sim, s);
+    return run_frame_match(ctx, ctx->sm_count, (uint8_t*)ctx->workspace, g, x, best_sim, best_idx, pos_sim, pair_sim, s);
 }
 
 oc_status launch_match_frame_levels(oc_ctx* ctx, const Geo& g, const void* x, int n_levels, const int32_t* levels,
                                     float* best_sim, int32_t* best_idx, float* pos_sim, float* pair_sim, cudaStream_t s) {
-    return run_frame_match(ctx, (uint8_t*)ctx->workspace, g, x, best_sim, best_idx, pos_sim, pair_sim, s, n_levels, levels);
+    return run_frame_match(ctx, ctx->sm_count, (uint8_t*)ctx->workspace, g, x, best_sim, best_idx, pos_sim, pair_sim, s, n_levels, levels);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -663,8 +667,27 @@ static constexpr int NOALLOC_MAX_DEVICES = 64;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
 // In host code `g_noalloc_scratch` is only a handle for the runtime, not a device address.  The
-// address each device gave the array is looked up once per device and kept here.
+// address each device gave the array is looked up once per device and kept here, together with the
+// device's SM count (which steers the segment split of the streaming kernel).
 static void* g_noalloc_dev_ptr[NOALLOC_MAX_DEVICES] = {};
+static int g_noalloc_sm_count[NOALLOC_MAX_DEVICES] = {};
+static std::mutex g_noalloc_mutex;
+
+// Makes the driver load every kernel instance the frame path can launch (a query of its attributes
+// does that), so that later calls find all code resident and have no reason to touch the loader.
+template <int DT>
+static bool noalloc_touch_kernels() {
+    cudaFuncAttributes fa;
+    bool ok = true;
+#define OC_TOUCH(k) ok = ok && cudaFuncGetAttributes(&fa, k) == cudaSuccess
+#define OC_TOUCH_L(L)                                                                                  \
+    OC_TOUCH((frame_march_kernel<DT, L, 5>)); OC_TOUCH((frame_march_kernel<DT, L, 8>)); OC_TOUCH((frame_pair_kernel<DT, L>))
+    OC_TOUCH_L(4); OC_TOUCH_L(8); OC_TOUCH_L(16); OC_TOUCH_L(32);
+    OC_TOUCH((frame_pair_kernel<DT, 1>)); OC_TOUCH((frame_pair_kernel<DT, 2>));
+#undef OC_TOUCH_L
+#undef OC_TOUCH
+    return ok;
+}
 
 }  // namespace oc
 
@@ -684,14 +707,28 @@ extern "C" oc_status oc_match_frame_noalloc(int device, const oc_layout* layout,
 
     DeviceGuard guard(device);
     if (!guard.ok) return OC_ERR_CUDA;
-    if (!g_noalloc_dev_ptr[device]) {
-        // set-up, once per device, with that device current
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) { cudaGetLastError(); return OC_ERR_CUDA; }
-        g_noalloc_dev_ptr[device] = p;
+    uint8_t* scratch = nullptr;
+    int sm_count = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_dev_ptr[device]) {
+            // set-up, once per device, with that device current
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) { cudaGetLastError(); return OC_ERR_CUDA; }
+            int n_sm = 0;
+            if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n_sm <= 0) {
+                cudaGetLastError(); return OC_ERR_CUDA;
+            }
+            cudaFuncAttributes fa;
+            if (!noalloc_touch_kernels<OC_DTYPE_BF16>() || !noalloc_touch_kernels<OC_DTYPE_F32>() ||
+                cudaFuncGetAttributes(&fa, frame_finalize_kernel) != cudaSuccess) { cudaGetLastError(); return OC_ERR_CUDA; }
+            g_noalloc_sm_count[device] = n_sm;
+            g_noalloc_dev_ptr[device] = p;
+        }
+        scratch = (uint8_t*)g_noalloc_dev_ptr[device];
+        sm_count = g_noalloc_sm_count[device];
     }
-    uint8_t* scratch = (uint8_t*)g_noalloc_dev_ptr[device];
     // nothing in the array has to start at zero: every partial record and every pair value that
     // the kernels read is written first by this call's own kernels
-    return run_frame_match(nullptr, scratch, g, x, best_sim, best_idx, nullptr, pair_sim, (cudaStream_t)stream);
+    return run_frame_match(nullptr, sm_count, scratch, g, x, best_sim, best_idx, nullptr, pair_sim, (cudaStream_t)stream);
 }

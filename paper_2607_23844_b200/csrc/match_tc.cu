@@ -64,8 +64,6 @@
 // and exits.
 #include <cuda.h>
 
-#include <cstdio>
-#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -547,7 +545,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     // two register buffers: the TMEM load of the next step is in flight while this one is reduced
                     uint32_t va[32], vb[32];
 #define OC_KEY(v, s, j) __uint_as_float((__float_as_uint(__uint_as_float(v) * (s)) & 0xFFFFFFE0u) | (uint32_t)(31 - (j)))
+#define OC_KEY_NEG(v, s, j) __uint_as_float((__float_as_uint(__uint_as_float(v) * (s)) & 0xFFFFFFE0u) | (uint32_t)(j))
 #define OC_VAL(k) __uint_as_float(__float_as_uint(k) & 0xFFFFFFE0u)
+#define OC_COL(k) ((__float_as_uint(k) >> 31) ? (int)(__float_as_uint(k) & 31u) : 31 - (int)(__float_as_uint(k) & 31u))
 #define OC_REDUCE_CHUNK(v, ch)                                                                                   \
     do {                                                                                                         \
         float cm0 = -INFINITY, cm1 = -INFINITY;                                                                  \
@@ -555,6 +555,24 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                                   \
             cm0 = max3f(cm0, OC_KEY(v[j], s4.x, j), OC_KEY(v[j + 1], s4.y, j + 1));                              \
             cm1 = max3f(cm1, OC_KEY(v[j + 2], s4.z, j + 2), OC_KEY(v[j + 3], s4.w, j + 3));                      \
+        }                                                                                                        \
+        /* A chain whose maximum is negative holds negative similarities only.  Among negative floats the  */   \
+        /* larger mantissa is the SMALLER value, so there the column goes into the low bits as it is (the  */   \
+        /* lowest column is then the largest key again).  Rare (every one of 16 cosines negative), so the */   \
+        /* chain is simply taken a second time.                                                           */   \
+        if (cm0 < 0.f) {                                                                                         \
+            cm0 = -INFINITY;                                                                                     \
+            _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                  \
+                const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                               \
+                cm0 = max3f(cm0, OC_KEY_NEG(v[j], s4.x, j), OC_KEY_NEG(v[j + 1], s4.y, j + 1));                  \
+            }                                                                                                    \
+        }                                                                                                        \
+        if (cm1 < 0.f) {                                                                                         \
+            cm1 = -INFINITY;                                                                                     \
+            _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                  \
+                const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                               \
+                cm1 = max3f(cm1, OC_KEY_NEG(v[j + 2], s4.z, j + 2), OC_KEY_NEG(v[j + 3], s4.w, j + 3));          \
+            }                                                                                                    \
         }                                                                                                        \
         /* a later chunk wins only with a strictly larger similarity (the index bits set aside) */              \
         if (OC_VAL(cm0) > OC_VAL(bm0)) { bm0 = cm0; bc0 = (ch); }                                                \
@@ -586,12 +604,14 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     }
 #undef OC_REDUCE_CHUNK
 #undef OC_KEY
+#undef OC_KEY_NEG
                     // the better chain; among equal similarities the lower column
-                    int n0 = bc0 < 0 ? -1 : bc0 * 32 + 31 - (int)(__float_as_uint(bm0) & 31u);
-                    const int n1 = bc1 < 0 ? -1 : bc1 * 32 + 31 - (int)(__float_as_uint(bm1) & 31u);
+                    int n0 = bc0 < 0 ? -1 : bc0 * 32 + OC_COL(bm0);
+                    const int n1 = bc1 < 0 ? -1 : bc1 * 32 + OC_COL(bm1);
                     float best = OC_VAL(bm0);
                     if (n1 >= 0 && (n0 < 0 || OC_VAL(bm1) > best || (OC_VAL(bm1) == best && n1 < n0))) { best = OC_VAL(bm1); n0 = n1; }
 #undef OC_VAL
+#undef OC_COL
                     if (row_ok && n0 >= 0) {
                         const int gp = c.c_off + n0;
                         const int qi = c.q0 + (gp >> 5), r = gp & 31;
@@ -690,8 +710,11 @@ struct TcPlan {
     long long rows, items;
 };
 
+// A forced work split (oc_tc_plan_override): the tests run every form of the kernel this way.
+struct TcForce { bool on; int pair, tiles, pieces, no_narrow; };
+
 // walkers: CTAs that can run at once; pair_walkers: CTA pairs that can (0 = pairs not available)
-static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
+static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcForce& force) {
     TcPlan p;
     int la = pow2_ceil_log2(g.Ws); if ((1 << la) > BM) la = pow2_ceil_log2(BM);
     p.bwA_log2 = la; p.bhA = BM >> la;
@@ -769,11 +792,10 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
             }
         }
     }
-    // Experiments may override the choice: OC_TC_PLAN="pair,tiles,pieces" (ignored unless valid).
-    if (const char* e = getenv("OC_TC_PLAN")) {
-        int o_pair = 0, o_tpp = 0, o_P = 0;
-        if (sscanf(e, "%d,%d,%d", &o_pair, &o_tpp, &o_P) == 3 && (o_pair == 0 || (o_pair == 1 && pair_walkers > 0)) &&
-            (o_tpp == 1 || o_tpp == 2)) {
+    // A forced split replaces the choice (ignored unless the shape admits it).
+    if (force.on) {
+        const int o_pair = force.pair, o_tpp = force.tiles, o_P = force.pieces;
+        if ((o_pair == 0 || (o_pair == 1 && pair_walkers > 0)) && (o_tpp == 1 || o_tpp == 2)) {
             const int q_unit = o_pair ? 2 : 1;
             const int n_units = (p.n_quanta + q_unit - 1) / q_unit, max_units = MAXQ / q_unit;
             if (o_P >= (n_units + max_units - 1) / max_units && o_P <= n_units) { best_pair = o_pair; best_tpp = o_tpp; best_P = o_P; }
@@ -796,10 +818,10 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers) {
         if (nq > q_max) q_max = nq;
     }
     p.qmax = q_max * ncta;
-    {   // widest piece in columns (experiments may set OC_TC_NO_NARROW to keep such plans on one accumulator set)
+    {   // widest piece in columns (a forced split may keep such plans on one accumulator set)
         const int hw = p.half_units ? half_widest(best_P) : 0;
         const int cols = hw ? hw * 16 : ((p.n_q_units + best_P - 1) / best_P) * p.q_unit * 32;
-        p.narrow = (p.tpp == 2 && cols <= 128 && !getenv("OC_TC_NO_NARROW")) ? 1 : 0;
+        p.narrow = (p.tpp == 2 && cols <= 128 && !(force.on && force.no_narrow)) ? 1 : 0;
     }
     p.stage_bytes = p.tpp * A_BYTES + q_max * Q_BYTES;
     p.n_stages = TILE_BYTES / p.stage_bytes;
@@ -823,8 +845,6 @@ bool tc_match_supported(const Geo& g) {
     return encode_fn() != nullptr;
 }
 
-void tc_cache_free(oc_ctx*) {}
-
 static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm, unsigned long long* keys,
                            float* aux_sim, const int4* units, const int* n_units_dev, long long max_units, cudaStream_t s);
 
@@ -846,39 +866,39 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
                            float* aux_sim, const int4* units, const int* n_units_dev, long long max_units, cudaStream_t s) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return OC_ERR_UNSUPPORTED;
-    // once per process: opt in to the large dynamic shared memory, and ask how many CTA pairs fit
-    static std::once_flag attr_once;
-    static bool attr_ok = false;
-    static int max_pairs[64];
-    std::call_once(attr_once, [] {
-        attr_ok = cudaFuncSetAttribute(match_tc_kernel<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
-                  cudaFuncSetAttribute(match_tc_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
-                  cudaFuncSetAttribute(match_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
-                  cudaFuncSetAttribute(match_tc_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
-                  cudaFuncSetAttribute(match_tc_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
-                  cudaFuncSetAttribute(match_tc_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess;
-        for (int i = 0; i < 64; ++i) max_pairs[i] = -1;
-        if (!attr_ok) cudaGetLastError();
-    });
-    if (!attr_ok) return OC_ERR_CUDA;
+    // once per device (the context's device is current here): opt in to the large dynamic shared
+    // memory, and ask how many CTA pairs fit
+    static PerDeviceOnce attr_once;
+    static int max_pairs[PerDeviceOnce::MAX_DEV];
     const int dev = ctx->device;
-    int pair_walkers = 0;
-    if (dev >= 0 && dev < 64) {
-        if (max_pairs[dev] < 0) {                     // (context's device is current here)
+    const int sm_count = ctx->sm_count;
+    const bool attr_ok = attr_once.ensure(dev, [dev, sm_count] {
+        const bool ok =
+            cudaFuncSetAttribute(match_tc_kernel<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+            cudaFuncSetAttribute(match_tc_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+            cudaFuncSetAttribute(match_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+            cudaFuncSetAttribute(match_tc_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+            cudaFuncSetAttribute(match_tc_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess &&
+            cudaFuncSetAttribute(match_tc_kernel<true, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TOTAL) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); return false; }
+        if (dev >= 0 && dev < PerDeviceOnce::MAX_DEV) {
             cudaLaunchConfig_t q = {};
             cudaLaunchAttribute qa[1];
             qa[0].id = cudaLaunchAttributeClusterDimension;
             qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
-            q.gridDim = dim3(2 * (unsigned)(ctx->sm_count / 2)); q.blockDim = dim3(TC_THREADS);
+            q.gridDim = dim3(2 * (unsigned)(sm_count / 2)); q.blockDim = dim3(TC_THREADS);
             q.dynamicSmemBytes = SMEM_TOTAL; q.attrs = qa; q.numAttrs = 1;
             int n = 0;
             if (cudaOccupancyMaxActiveClusters(&n, match_tc_kernel<true, 0>, &q) != cudaSuccess) { cudaGetLastError(); n = 0; }
-            if (n > ctx->sm_count / 2) n = ctx->sm_count / 2;
+            if (n > sm_count / 2) n = sm_count / 2;
             max_pairs[dev] = n;
         }
-        pair_walkers = max_pairs[dev];
-    }
-    const TcPlan p = make_plan(g, ctx->sm_count, pair_walkers);
+        return true;
+    });
+    if (!attr_ok) return OC_ERR_CUDA;
+    const int pair_walkers = (dev >= 0 && dev < PerDeviceOnce::MAX_DEV) ? max_pairs[dev] : 0;
+    const TcForce force = {ctx->tc_plan_forced, ctx->tc_plan_pair, ctx->tc_plan_tiles, ctx->tc_plan_pieces, ctx->tc_plan_no_narrow};
+    const TcPlan p = make_plan(g, ctx->sm_count, pair_walkers, force);
     if (p.items > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
 
     TcParams KP;

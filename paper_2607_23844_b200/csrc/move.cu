@@ -1,5 +1,6 @@
-// gather / restore / copy: the bandwidth-bound row movers (Appendix A's compaction and
-// "fused permutation/scatter", written gather-style so that every output row has one writer).
+// gather / restore / copy: the bandwidth-bound row movers (Appendix A's compaction of the kept rows
+// and its permutation/scatter back into place, written gather-style so that every output row has
+// one writer).
 //
 // All three are flat over 16-byte chunks: a thread moves UNROLL independent chunks (all loads issued
 // before the first store), consecutive threads touch consecutive chunks, so a warp reads and writes
@@ -74,11 +75,13 @@ gather_kernel(const uint8_t* __restrict__ x, const int32_t* __restrict__ kept_id
 }
 
 // MODE 0: skipped rows from cache; 1: skipped rows from the representative's z row; 2: in place
-// (skipped rows untouched).
+// (skipped rows untouched).  slot_of / match_map / cache / out are this launch's slice of the units;
+// slot_of_all is the whole array, which MODE 1 indexes with the (global) unit a match_map entry names.
 template <bool SEG, int MODE>
 __global__ void __launch_bounds__(MOVE_THREADS)
 restore_kernel(const uint8_t* __restrict__ z, const uint8_t* __restrict__ cache,
                const int32_t* __restrict__ slot_of, const int32_t* __restrict__ match_map,
+               const int32_t* __restrict__ slot_of_all,
                uint8_t* __restrict__ out, unsigned total_chunks, RowsDev R) {
     pdl_enter();
     const unsigned base = blockIdx.x * (MOVE_THREADS * MOVE_UNROLL) + threadIdx.x;
@@ -91,7 +94,7 @@ restore_kernel(const uint8_t* __restrict__ z, const uint8_t* __restrict__ cache,
         if (c < total_chunks) {
             unsigned unit = c / R.cpr, col = c - unit * R.cpr;
             int slot = __ldg(slot_of + unit);
-            if (MODE == 1 && slot < 0) slot = __ldg(slot_of + __ldg(match_map + unit));
+            if (MODE == 1 && slot < 0) slot = __ldg(slot_of_all + __ldg(match_map + unit));
             long long off = strided_offset<SEG>(R, unit, col);
             if (slot >= 0) {
                 v[k] = ld_nc_v4(z + ((long long)slot * R.cpr + col) * 16);
@@ -150,11 +153,11 @@ oc_status launch_gather(oc_ctx* ctx, const oc_rows& rows, const void* x, const i
 
 template <bool SEG>
 static void restore_dispatch(int mode, unsigned blocks, cudaStream_t s, const uint8_t* z, const uint8_t* cache,
-                             const int32_t* slot_of, const int32_t* match_map, uint8_t* out, unsigned total,
-                             const RowsDev& R) {
-    if (mode == 0) OC_LAUNCH((restore_kernel<SEG, 0>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, out, total, R);
-    else if (mode == 1) OC_LAUNCH((restore_kernel<SEG, 1>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, out, total, R);
-    else OC_LAUNCH((restore_kernel<SEG, 2>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, out, total, R);
+                             const int32_t* slot_of, const int32_t* match_map, const int32_t* slot_of_all, uint8_t* out,
+                             unsigned total, const RowsDev& R) {
+    if (mode == 0) OC_LAUNCH((restore_kernel<SEG, 0>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, slot_of_all, out, total, R);
+    else if (mode == 1) OC_LAUNCH((restore_kernel<SEG, 1>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, slot_of_all, out, total, R);
+    else OC_LAUNCH((restore_kernel<SEG, 2>), blocks, MOVE_THREADS, 0, s, z, cache, slot_of, match_map, slot_of_all, out, total, R);
 }
 
 oc_status launch_restore(oc_ctx* ctx, const oc_rows& rows, const void* z, const void* cache,
@@ -175,8 +178,8 @@ oc_status launch_restore(oc_ctx* ctx, const oc_rows& rows, const void* z, const 
         const uint8_t* cc = cache ? (const uint8_t*)cache + u0 * R.unit_pitch : nullptr;
         uint8_t* oo = (uint8_t*)out + u0 * R.unit_pitch;
         LaunchScope scope(ctx, OC_K_RESTORE, s);
-        if (seg) restore_dispatch<true>(mode, blocks, s, (const uint8_t*)z, cc, slot_of + u0, match_map + u0, oo, total, R);
-        else     restore_dispatch<false>(mode, blocks, s, (const uint8_t*)z, cc, slot_of + u0, match_map + u0, oo, total, R);
+        if (seg) restore_dispatch<true>(mode, blocks, s, (const uint8_t*)z, cc, slot_of + u0, match_map + u0, slot_of, oo, total, R);
+        else     restore_dispatch<false>(mode, blocks, s, (const uint8_t*)z, cc, slot_of + u0, match_map + u0, slot_of, oo, total, R);
     }
     return last_launch_status();
 }

@@ -588,15 +588,16 @@ oc_status launch_select(oc_ctx* ctx, const Geo& geo, const float* best_sim, cons
     if (geo.n_groups == 0) return OC_OK;
     GroupMap gm = make_group_map(geo);
     int nr = (int)(n_reuse > 0x7FFFFFFF ? 0x7FFFFFFF : n_reuse);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(select_general_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess ||
-            cudaFuncSetAttribute(select_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess)
-            return OC_ERR_CUDA;
-        attr_set = true;
-    }
+    static PerDeviceOnce attr_once;                 // (the context's device is current here)
+    if (!attr_once.ensure(ctx->device, [] {
+            const bool ok = cudaFuncSetAttribute(select_general_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) == cudaSuccess &&
+                            cudaFuncSetAttribute(select_fast_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) == cudaSuccess;
+            if (!ok) cudaGetLastError();
+            return ok;
+        }))
+        return OC_ERR_CUDA;
     LaunchScope scope(ctx, OC_K_SELECT, s);
     if (!geo.self_match && geo.units_per_group <= SEL_SMALL_UNITS) {
         const int wpc = SEL_SMALL_THREADS / 32;
@@ -636,13 +637,14 @@ oc_status launch_select_joint(oc_ctx* ctx, const Geo& geo, const int2* frames, c
     gm.units_per_group = (int)(2 * P);
     gm.n_reuse_single = (int)(n_reuse_single > 0x7FFFFFFF ? 0x7FFFFFFF : n_reuse_single);
     const int nr = (int)(n_reuse_pair > 0x7FFFFFFF ? 0x7FFFFFFF : n_reuse_pair);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(select_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) != cudaSuccess)
-            return OC_ERR_CUDA;
-        attr_set = true;
-    }
+    static PerDeviceOnce attr_once;
+    if (!attr_once.ensure(ctx->device, [] {
+            const bool ok = cudaFuncSetAttribute(select_fast_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 SEL_SMEM_KEYS * (int)sizeof(unsigned)) == cudaSuccess;
+            if (!ok) cudaGetLastError();
+            return ok;
+        }))
+        return OC_ERR_CUDA;
     LaunchScope scope(ctx, OC_K_SELECT, s);
     OC_LAUNCH(select_fast_kernel<true>, (unsigned)slots, SEL_THREADS, (size_t)(2 * P) * sizeof(unsigned), s,
               gm, best_sim, best_idx, mode, thr, nr, (int)y_stride, kept_idx, kept_count, match_map, slot_of);

@@ -24,6 +24,19 @@ def oc():
     return omnicache
 
 
+def expect_tensor_core(dtype, shape, lattice=(2, 2, 0, 0), self_match=False):
+    """Whether oc_match must take the tcgen05 kernel for this Token Cache layout: bf16, no self-match, at most
+    nine lattice members, rows of whole 16-byte chunks.  Anything else belongs to the fp32-FMA kernel; a bf16
+    layout that falls back silently would pass every numeric check and run an order of magnitude slower."""
+    return dtype == inputs.BF16 and not self_match and lattice[0] * lattice[1] <= 9 and shape[-1] % 8 == 0
+
+
+def assert_matcher(rep, dtype, shape, lattice=(2, 2, 0, 0)):
+    want_tc = expect_tensor_core(dtype, shape, lattice)
+    assert rep["launches"]["match_tc"] == (1 if want_tc else 0), rep["launches"]
+    assert rep["launches"]["match_simt"] == (0 if want_tc else 1), rep["launches"]
+
+
 def run_chain(oc, oracle, w, Cout=None, full_oracle=True, sample_rows=0, want_aux=False, **layout_kw):
     """match -> select -> gather -> restore for one workload, each stage compared with the oracle.
     Returns a small report dict."""
@@ -40,8 +53,13 @@ def run_chain(oc, oracle, w, Cout=None, full_oracle=True, sample_rows=0, want_au
                 ref = oracle.match_token(Lo, w.x, want_full=want_aux)
                 rows = None
             else:
+                # the same number of rows from every group (frame or patch), so that every frame and, over
+                # the groups, every position inside the matcher's tiles is looked at
                 rng = np.random.default_rng(99)
-                rows = np.sort(rng.choice(Lo.n_units, sample_rows, replace=False))
+                G, U = Lo.n_groups, Lo.units_per_group
+                per = max(1, sample_rows // G)
+                rows = np.sort(np.array([Lo.unit_index(g, int(u)) for g in range(G)
+                                         for u in rng.choice(U, min(per, U), replace=False)], dtype=np.int64))
                 ref = oracle.match_token(Lo, w.x, rows=rows)
             rep["near_tie_rows"], rep["near_tie_differ"] = H.check_match_against_oracle(
                 oracle, Lo, w.x, gs, gi, ref, TOL[w.dtype], rows)
@@ -159,8 +177,7 @@ def test_token_chain_small(oc, oracle, shape, groups, lattice, dtype):
     U = (Hh // groups[0]) * (W // groups[1])
     w.n_reuse = (U - U // (sy * sx)) // 2
     rep = run_chain(oc, oracle, w, want_aux=True, sy=sy, sx=sx, oy=oy, ox=ox)
-    if dtype == inputs.BF16:
-        assert rep["launches"]["match_tc"] + rep["launches"]["match_simt"] == 1
+    assert_matcher(rep, dtype, shape, lattice)
 
 
 def _random_token_layouts(n, seed):
@@ -192,21 +209,22 @@ def test_token_chain_random_layouts(oc, oracle, shape, groups, lattice):
     reps = ((Hh // groups[0]) // sy) * ((W // groups[1]) // sx)
     w.n_reuse = (U - reps) // 3
     rep = run_chain(oc, oracle, w, want_aux=True, sy=sy, sx=sx, oy=oy, ox=ox)
-    assert rep["launches"]["match_tc"] + rep["launches"]["match_simt"] == 1
+    assert_matcher(rep, inputs.BF16, shape, lattice)
 
 
 @pytest.mark.parametrize("plan", ["0,1,2", "0,2,3", "1,1,1", "1,2,2"])
 @pytest.mark.parametrize("shape,groups,lattice", _random_token_layouts(8, seed=7))
-def test_token_match_random_layouts_forced_plans(oc, oracle, shape, groups, lattice, plan, monkeypatch):
+def test_token_match_random_layouts_forced_plans(oc, oracle, shape, groups, lattice, plan):
     B, T, Hh, W, C = shape
     w = inputs.sd3_token_cache(seed=int(np.prod(shape)) % 9973, B=B * T, H=Hh, W=W, C=C, groups=groups)
     w.x = w.x.reshape(shape); w.shape = shape
     sy, sx, oy, ox = lattice
     L, Lo = H.layouts(oc, oracle, w, sy=sy, sx=sx, oy=oy, ox=ox)
     ref = oracle.match_token(Lo, w.x)
-    monkeypatch.setenv("OC_TC_PLAN", plan)
     with H.make_ctx(oc, L) as ctx:
+        ctx.tc_plan_override(plan.split(","))
         m = H.gpu_match(oc, ctx, L, H.to_dev(w.x))
+        assert ctx.launches()["match_tc"] == 1 and ctx.launches()["match_simt"] == 0
     H.check_match_against_oracle(oracle, Lo, w.x, m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy(), ref,
                                  TOL[inputs.BF16])
 
@@ -217,7 +235,7 @@ def test_token_match_random_layouts_forced_plans(oc, oracle, shape, groups, latt
     ((1, 1, 64, 64, 128), (2, 2)),       # four patches per frame
 ])
 @pytest.mark.parametrize("plan", ["0,1,1", "0,1,3", "0,2,2", "0,2,5", "1,1,1", "1,1,2", "1,2,1", "1,2,4", "0,2,64", "1,1,64"])
-def test_tensor_core_matcher_every_plan(oc, oracle, shape, groups, plan, monkeypatch):
+def test_tensor_core_matcher_every_plan(oc, oracle, shape, groups, plan):
     """The planner's choice (single CTA or CTA pair, one or two candidate tiles per CTA, pieces per
     row) changes the work split only: every valid plan must reproduce the oracle.  A plan the shape
     does not admit is ignored by the library (the planner's own choice runs instead)."""
@@ -226,9 +244,9 @@ def test_tensor_core_matcher_every_plan(oc, oracle, shape, groups, plan, monkeyp
     w.x = w.x.reshape(shape); w.shape = shape
     L, Lo = H.layouts(oc, oracle, w)
     ref = oracle.match_token(Lo, w.x, want_full=True)
-    monkeypatch.setenv("OC_TC_PLAN", plan)
     x_dev = H.to_dev(w.x)
     with H.make_ctx(oc, L) as ctx:
+        ctx.tc_plan_override(plan.split(","))
         ctx.profile_enable(True)
         for want_aux in (False, True):
             m = H.gpu_match(oc, ctx, L, x_dev, want_aux=want_aux)
@@ -397,7 +415,7 @@ def test_block_patches_chain(oc, oracle, grid, mode):
 # ---------------------------------------------------------------------------------------------------
 # Token Cache on the frame pairs of Frame Cache (Section 3.2.3)
 # ---------------------------------------------------------------------------------------------------
-def _joint_case(oc, oracle, x_np, shape, frames_np, mode, thr, n_pair, n_single, lattice=(2, 2, 0, 0)):
+def _joint_case(oc, oracle, x_np, shape, frames_np, mode, thr, n_pair, n_single, lattice=(2, 2, 0, 0), plan=None):
     """match_joint -> select_joint -> gather -> restore on a given frame table, each against the oracle."""
     B, T, Hh, W, C = shape
     P = Hh * W
@@ -407,6 +425,8 @@ def _joint_case(oc, oracle, x_np, shape, frames_np, mode, thr, n_pair, n_single,
     n = B * T * P
     x_dev, fr_dev = H.to_dev(x_np), H.to_dev(frames_np)
     with oc.Context(0, oc.joint_workspace_bytes(L)) as ctx:
+        if plan:
+            ctx.tc_plan_override(plan.split(","))
         bs = torch.full((n,), float("nan"), device="cuda")
         bi = torch.full((n,), -2, device="cuda", dtype=torch.int32)
         ctx.match_joint(L, x_dev, fr_dev, bs, bi)
@@ -469,11 +489,9 @@ def test_joint_token_cache_on_given_frame_tables(oc, oracle, shape, lattice, mod
 
 
 @pytest.mark.parametrize("plan", [None, "0,1,1", "0,2,2", "1,1,1", "1,2,2", "0,2,3"])
-def test_joint_token_cache_svd_level_shapes_every_plan(oc, oracle, plan, monkeypatch):
+def test_joint_token_cache_svd_level_shapes_every_plan(oc, oracle, plan):
     """Several candidate tiles per lattice member, every form of the tensor-core matcher (single CTA / CTA
     pair, one or two tiles, several pieces per row) on the joint work list."""
-    if plan:
-        monkeypatch.setenv("OC_TC_PLAN", plan)
     shape = (1, 7, 36, 64, 128)                     # 2304 tokens per frame: 576 per sub-lattice = 4.5 tiles
     B, T, Hh, W, C = shape
     rng = np.random.default_rng(17)
@@ -481,7 +499,7 @@ def test_joint_token_cache_svd_level_shapes_every_plan(oc, oracle, plan, monkeyp
     x_np = inputs.to_bf16_bits(np.ascontiguousarray(x, dtype=np.float32))
     frames = np.array([[0, 1], [-1, -1], [2, -1], [-1, -1], [4, 3], [5, -1], [6, -1]], np.int32)
     P = Hh * W
-    reused = _joint_case(oc, oracle, x_np, shape, frames, oc.SELECT_COUNT, 0.0, P, P // 3)
+    reused = _joint_case(oc, oracle, x_np, shape, frames, oc.SELECT_COUNT, 0.0, P, P // 3, plan=plan)
     assert reused == 2 * P + 3 * (P // 3)
 
 
@@ -665,7 +683,7 @@ def test_config4_latte_block_cache_full(oc, oracle):
 def test_config5_levels(oc, oracle, level):
     Hh, W, C = inputs.SVD_LEVELS[level]
     base = inputs.svd_frames(seed=1005 + level, T=25, H=Hh, W=W, C=C, rho=0.95, kind="token")
-    steps = (0, 1, 24) if level > 0 else (0, 1)
+    steps = (0, 1, 24)
     rng = np.random.default_rng(77)
     x = base.x
     lc_ref = oracle.LayerCache()
@@ -699,7 +717,9 @@ def test_config5_levels(oc, oracle, level):
                         U, R = Hh * W, (Hh // 2) * (W // 2)
                     w.n_reuse = inputs.keep_ratio_to_reuse(U, U - R, ratio)
                     full = kind != "token"
-                    run_chain(oc, oracle, w, full_oracle=full, sample_rows=160)
+                    rep = run_chain(oc, oracle, w, full_oracle=full, sample_rows=1200)
+                    if kind == "token":
+                        assert rep["launches"]["match_tc"] == 1
         assert lc_ctx.layer_cache_get(level, max(steps) + 5, 5)[0] is False
 
 
@@ -754,6 +774,56 @@ def test_duplicates_zero_rows_and_ties(oc, oracle):
         assert gs[5 * 32 + 5] == 0.0 and gi[5 * 32 + 5] == 0     # all similarities 0: lowest index
         ref = oracle.match_token(Lo, x)
         H.check_match_against_oracle(oracle, Lo, x, gs, gi, ref, TOL[dtype])
+
+
+@pytest.mark.parametrize("dtype", [inputs.BF16, inputs.F32])
+def test_exact_ties_between_negative_similarities_go_to_the_lowest_index(oc, oracle, dtype):
+    """A candidate whose BEST similarity is negative and exactly tied between identical representatives.
+    Frame f duplicates one representative at two lattice places; the candidates of the frame point
+    (almost) away from every representative, least so from the duplicated one.  The places are chosen so
+    that the two copies meet in one reduction chain of the tensor-core epilogue, in its two chains, in
+    two 32-column chunks and in two pieces of the row; the lower index must win every time."""
+    Hh = W = 32
+    C = 64
+    Ws = W // 2                                                  # 16 x 16 representatives per frame
+    places = [(0, 1), (0, 2), (5, 40), (3, 200), (17, 16), (254, 255)]        # lattice indices of the two copies
+    T = len(places)
+    rng = np.random.default_rng(4)
+    xf = np.zeros((1, T, Hh, W, C), np.float32)
+    e0, e1 = np.zeros(C, np.float32), np.zeros(C, np.float32)
+    e0[0] = 1.0; e1[1] = 1.0
+    for t, (p1, p2) in enumerate(places):
+        for r in range(Ws * Ws):                                 # every other representative: near e1
+            y, x = 2 * (r // Ws), 2 * (r % Ws)
+            xf[0, t, y, x] = e1 + 0.05 * np.abs(rng.standard_normal(C)).astype(np.float32) * (np.arange(C) >= 2)
+        a = e0 + 0.25 * np.abs(rng.standard_normal(C)).astype(np.float32) * (np.arange(C) >= 2)
+        for p in (p1, p2):
+            xf[0, t, 2 * (p // Ws), 2 * (p % Ws)] = a
+        for y in range(Hh):
+            for x in range(W):
+                if y % 2 or x % 2:                               # candidates: -(0.1 e0 + e1), scaled, tail >= 0 flipped
+                    xf[0, t, y, x] = -(0.1 * e0 + e1) * (1.0 + 0.5 * rng.random()) \
+                                     - 0.01 * np.abs(rng.standard_normal(C)).astype(np.float32) * (np.arange(C) >= 2)
+    x = xf if dtype == inputs.F32 else inputs.to_bf16_bits(xf)
+    w = inputs.Workload("neg_ties", "token", dtype, xf.shape, x, mode="count", n_reuse=10)
+    L, Lo = H.layouts(oc, oracle, w)
+    ref = oracle.match_token(Lo, x)
+    forced = [None] if dtype == inputs.F32 else [None, (0, 1, 1), (0, 2, 2), (0, 1, 8), (1, 1, 1), (1, 2, 4)]
+    for plan in forced:
+        with H.make_ctx(oc, L) as ctx:
+            if plan:
+                ctx.tc_plan_override(plan)
+            m = H.gpu_match(oc, ctx, L, H.to_dev(x))
+            assert ctx.launches()["match_tc"] == (1 if dtype == inputs.BF16 else 0)
+        gs, gi = m["best_sim"].cpu().numpy(), m["best_idx"].cpu().numpy()
+        H.check_match_against_oracle(oracle, Lo, x, gs, gi, ref, TOL[dtype])
+        for t, (p1, p2) in enumerate(places):
+            pl = min(p1, p2)
+            low = (t * Hh + 2 * (pl // Ws)) * W + 2 * (pl % Ws)
+            cand = [(t * Hh + y) * W + xx for y in range(Hh) for xx in range(W) if y % 2 or xx % 2]
+            assert np.all(gs[cand] < 0.0), "the best similarity of every candidate must be negative here"
+            assert np.all(ref["best_idx"][cand] == low), "construction: the oracle's best is the duplicated representative"
+            assert np.all(gi[cand] == low), (plan, t, np.unique(gi[cand]))
 
 
 def test_determinism_and_profile_counters(oc, oracle):
