@@ -1065,7 +1065,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="svd_token_l0")
-    ap.add_argument("--ref-rows", type=int, default=8192,
+    ap.add_argument("--ref-rows", type=int, default=65536,
                     help="candidates the CPU oracle matches per step (all of them if the workload has fewer)")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--sub-steps", type=int, default=40, help="timed steps of each sub-record under `configs`")

@@ -181,12 +181,21 @@ oc_status oc_profile_read(oc_ctx* ctx, int kernel_id, int64_t* launches, double*
 /* Test hook: forces the work split of the tensor-core matcher for this context's later oc_match /
  * oc_match_joint calls instead of the planner's choice: a single CTA (pair = 0) or a CTA pair
  * (pair = 1) per piece, 1 or 2 candidate tiles per CTA, pieces_per_row pieces per row of the
- * problem; single_accumulator != 0 keeps narrow pieces on one accumulator set.  A split the shape
- * does not admit is ignored (the planner's choice runs).  on = 0 returns to the planner.  Results
- * never depend on the split; the parity tests use this to run every form of the kernel.
- * OC_ERR_INVALID_ARG for values outside the ranges above.  The paper has no counterpart. */
+ * problem; single_accumulator != 0 keeps narrow pieces on one accumulator set; candidates_resident
+ * 1 / 0 turns on / off keeping a CTA's candidate tiles in shared memory for all pieces of a row
+ * (only where they fit), -1 leaves that to the planner.  A split the shape does not admit is ignored
+ * (the planner's choice runs).  on = 0 returns to the planner.  Results never depend on the split;
+ * the parity tests use this to run every form of the kernel.  OC_ERR_INVALID_ARG for values outside
+ * the ranges above.  The paper has no counterpart. */
 oc_status oc_tc_plan_override(oc_ctx* ctx, int on, int pair, int tiles_per_cta, int pieces_per_row,
-                              int single_accumulator);
+                              int single_accumulator, int candidates_resident);
+
+/* Test hook: the work split oc_match would use for this (bf16, no self-match) OC_KIND_TOKEN layout on
+ * this context, forced split included.  out receives 12 ints: pair, tiles per CTA, pieces per row,
+ * two accumulator sets (0/1), ring stages, bytes per stage, candidate tiles resident (0/1), pieces in
+ * total, walkers (CTAs or CTA pairs launched), widest piece in columns, 64-channel steps, reserved.
+ * Host only.  OC_ERR_UNSUPPORTED when the layout does not take the tensor-core kernel. */
+oc_status oc_tc_plan_describe(oc_ctx* ctx, const oc_layout* layout, int32_t* out);
 
 /* Device-side span of the tensor-core matcher (kernel_id must be OC_K_MATCH_TC).  With
  * oc_profile_enable(ctx, 2) every launch of that kernel stamps the GPU's nanosecond timer when its

@@ -41,6 +41,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
                "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
+        cmd[1:1] = os.environ.get("OC_NVCC_EXTRA", "").split()      # e.g. -DNAME=value for an experiment build
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
         objs.append(obj)
     failed = False

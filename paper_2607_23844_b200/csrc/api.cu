@@ -269,14 +269,26 @@ oc_status oc_selftest_bounded_wait(oc_ctx* c, unsigned int limit_us, void* strea
     return launch_bounded_wait_selftest(c, (unsigned long long)limit_us * 1000ull, (cudaStream_t)stream);
 }
 
-oc_status oc_tc_plan_override(oc_ctx* c, int on, int pair, int tiles_per_cta, int pieces_per_row, int single_accumulator) {
+oc_status oc_tc_plan_override(oc_ctx* c, int on, int pair, int tiles_per_cta, int pieces_per_row, int single_accumulator,
+                              int candidates_resident) {
     if (!c) return OC_ERR_INVALID_ARG;
     if (on && ((pair != 0 && pair != 1) || (tiles_per_cta != 1 && tiles_per_cta != 2) || pieces_per_row < 1))
         return OC_ERR_INVALID_ARG;
     c->tc_plan_forced = on != 0;
     c->tc_plan_pair = pair; c->tc_plan_tiles = tiles_per_cta; c->tc_plan_pieces = pieces_per_row;
     c->tc_plan_no_narrow = single_accumulator ? 1 : 0;
+    c->tc_plan_a_res = candidates_resident < 0 ? -1 : (candidates_resident ? 1 : 0);
     return OC_OK;
+}
+
+oc_status oc_tc_plan_describe(oc_ctx* c, const oc_layout* layout, int32_t* out) {
+    if (!c || !out) return OC_ERR_INVALID_ARG;
+    Geo g;
+    oc_status st = make_geo(layout, &g);
+    if (st != OC_OK) return st;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return OC_ERR_CUDA;
+    return tc_plan_describe(c, g, out);
 }
 
 oc_status oc_profile_enable(oc_ctx* c, int on) {

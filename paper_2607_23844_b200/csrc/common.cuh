@@ -49,7 +49,7 @@ struct oc_ctx {
     std::vector<cudaEvent_t> chunk_events;
     // test hook (oc_tc_plan_override): forces the tensor-core matcher's work split
     bool tc_plan_forced = false;
-    int tc_plan_pair = 0, tc_plan_tiles = 0, tc_plan_pieces = 0, tc_plan_no_narrow = 0;
+    int tc_plan_pair = 0, tc_plan_tiles = 0, tc_plan_pieces = 0, tc_plan_no_narrow = 0, tc_plan_a_res = -1;
 };
 
 namespace oc {
@@ -205,6 +205,7 @@ oc_status launch_match_joint_tc(oc_ctx*, const Geo&, const void* x, const float*
                                 const int4* units, const int* n_units_dev, long long max_units, cudaStream_t);
 oc_status launch_match_token_tc(oc_ctx*, const Geo&, const void* x, const float* inv_norm,
                                 unsigned long long* keys, float* aux_sim, cudaStream_t);
+oc_status tc_plan_describe(oc_ctx*, const Geo&, int32_t* out12);
 oc_status launch_bounded_wait_selftest(oc_ctx*, unsigned long long limit_ns, cudaStream_t);
 
 size_t match_workspace_bytes(const Geo&);
@@ -241,11 +242,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 // One look at a barrier, never suspending the thread.
 __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -255,6 +251,11 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
 }
 // Bounded wait: false if the phase did not complete within WAIT_LIMIT_NS or another role gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {

@@ -78,9 +78,14 @@ static constexpr int BK = 64;            // channels per stage: 128 bytes of bf1
 static constexpr int A_BYTES = BM * BK * 2;
 static constexpr int Q_BYTES = QN * BK * 2;
 static constexpr int MAX_STAGES = 8;
+static constexpr int MAX_AKB = 10;       // most 64-channel steps whose candidate tiles may stay resident
 static constexpr int SMEM_LIMIT = 232448;         // 227 KB: the most dynamic shared memory a CTA may have
-static constexpr int TC_THREADS = 320;   // producer warp, MMA warp, 8 epilogue warps
-static constexpr int EPI_THREADS = 256;
+#ifndef OC_EPI_WARPS
+#define OC_EPI_WARPS 8
+#endif
+static constexpr int EPI_WARPS = OC_EPI_WARPS;            // 8 or 16: two or four per TMEM lane quarter
+static constexpr int EPI_PARTS = EPI_WARPS / 4;           // a piece's columns are cut into this many parts
+static constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;    // producer warp, MMA warp, the epilogue warps
 static constexpr int MAX_LATTICES = 9;
 static constexpr uint32_t TMEM_COLS = 512;
 
@@ -109,6 +114,9 @@ struct TcScalars {
     int sx_magic;                        // ceil(65536 / sx): (m * sx_magic) >> 16 == m / sx for m < 256
     int u_step_q, u_step_r;              // n_q_units / pieces_per_row and the remainder
     int n_stages, stage_bytes;           // operand ring of this launch
+    int a_res, a_region_bytes;           // candidate tiles resident: all 64-channel steps of a CTA's candidate tiles
+                                         // sit in front of the ring (one slot per step) for all pieces of a row, and
+                                         // the ring carries representatives only
     int units_per_group, reps_per_group;
     // Joint form (Token Cache on the frame pairs of Frame Cache, Section 3.2.3): the work is a list of
     // units {representative frame, candidate frame, candidate sub-lattice member} written by another
@@ -138,6 +146,8 @@ struct Piece {
     int q0, nq;                          // quanta [q0, q0 + nq) of the group's representatives are fetched
     int c_off, ncol;                     // of which columns [c_off, c_off + ncol) are the piece (c_off is 0 or 16,
                                          // ncol a multiple of 16: pieces may begin and end in mid-quantum)
+    int first, last;                     // the first / last piece this walker has of the piece's row (the same
+                                         // candidate tiles serve all pieces of a row)
     long long g;
 };
 // floor(a / d) for a < 2^22 from the float reciprocal (one multiply and a fix-up; an integer division
@@ -159,12 +169,14 @@ struct Walk {
     int j, a_pair, k, px, py, bt;
     int u_cur, r_cur;                    // floor(j * n_q_units / pieces_per_row) and the remainder
     int bt_a, member_u;                  // joint form: the current unit's candidate frame and member
+    int fresh;                           // nothing handed out yet
     long long g;
     __device__ __forceinline__ void load_unit(const TcScalars& P) {
         const int4 v = __ldg(P.units + g);
         bt = v.x; bt_a = v.y; member_u = v.z;
     }
     __device__ __forceinline__ Walk(const TcScalars& P, int c) {
+        fresh = 1;
         if (JOINT) {
             // pieces are numbered (unit, tile run, piece of the row); the list length is read here
             const unsigned total = (unsigned)__ldg(P.n_units_dev) * P.cum[1];
@@ -215,6 +227,8 @@ struct Walk {
             p.ncol = p.nq * QN;
         }
         u_cur = u_next; r_cur = r_next;
+        p.first = (j == 0) | fresh; fresh = 0;
+        p.last = (j + 1 == P.pieces_per_row) | (left == 0);
         p.a_pair = a_pair; p.g = g; p.px = px; p.py = py; p.bt = bt;
         p.bt_a = JOINT ? bt_a : bt;
         p.member = JOINT ? member_u : (k < P.rep_member ? k : k + 1);
@@ -235,8 +249,39 @@ struct Walk {
     }
 };
 
+// Maximum of 32 arg-max keys by a tree of three-input maxima: 16 instructions, four levels deep.  (NaN keys,
+// the masked columns, never win: max.f32 returns its non-NaN operand.)
+__device__ __forceinline__ float key_tree_max(const float (&k)[32]) {
+    float a[11];
+#pragma unroll
+    for (int i = 0; i < 10; ++i) a[i] = max3f(k[3 * i], k[3 * i + 1], k[3 * i + 2]);
+    a[10] = fmaxf(k[30], k[31]);
+    const float b0 = max3f(a[0], a[1], a[2]), b1 = max3f(a[3], a[4], a[5]), b2 = max3f(a[6], a[7], a[8]);
+    const float c0 = max3f(b0, b1, b2);
+    return max3f(c0, a[9], a[10]);
+}
+
+// Arg-max key of the epilogue's second look at a row (see there): the value with its 5 low mantissa bits
+// replaced by the column, stored so that the LOWEST column is the largest key whatever the sign.
+__device__ __forceinline__ float oc_key_any(float x, int j) {
+    const uint32_t b = __float_as_uint(x);
+    return __uint_as_float((b & 0xFFFFFFE0u) | (uint32_t)((b >> 31) ? j : 31 - j));
+}
+
+#ifdef OC_TC_TRACE
+// scratch instrumentation (experiment builds only): SM cycle counter at a few points of every piece of one CTA
+__device__ unsigned long long g_tc_trace[4][128][4];
+__device__ unsigned long long g_tc_stage[8][512];
+#define OC_TS(k, n, who) do { if (blockIdx.x == OC_TC_TRACE && (who) && (n) < 512) g_tc_stage[k][n] = clock64(); } while (0)
+#define OC_TR(role, piece, k, who)                                                                                  \
+    do { if (blockIdx.x == OC_TC_TRACE && (who) && (piece) < 128) g_tc_trace[role][piece][k] = clock64(); } while (0)
+#else
+#define OC_TR(role, piece, k, who)
+#define OC_TS(k, n, who)
+#endif
+
 static constexpr int COL_BYTES = 256 * 8;                               // {scale, bias} per column of a piece
-static constexpr int N_BARS = 2 * MAX_STAGES + 5;                       // full[], empty[], acc_full[2], acc_empty[2], drain
+static constexpr int N_BARS = 2 * MAX_STAGES + 5 + MAX_AKB;             // full[], empty[], acc_full[2], acc_empty[2], drain, a_empty[]
 static constexpr int TAIL_BYTES = COL_BYTES + N_BARS * 8 + 32;        // column table, barriers, TMEM slot, flags
 static constexpr int TILE_BYTES = (SMEM_LIMIT - TAIL_BYTES) / 1024 * 1024;   // operand ring: everything else
 static constexpr int SMEM_TOTAL = TILE_BYTES + TAIL_BYTES;
@@ -260,6 +305,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * MAX_STAGES;
     const uint32_t bar_acc_full = bar_empty + 8 * MAX_STAGES, bar_acc_empty = bar_acc_full + 16;   // two of each
     const uint32_t bar_drain = bar_acc_empty + 16;
+    const uint32_t bar_a_empty = bar_drain + 8;                        // resident candidate slots, one per 64-channel step
     uint32_t* tmem_slot = (uint32_t*)(bars + N_BARS);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     const uint32_t tiles_base = smem_u32(smem);
@@ -286,9 +332,10 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
-            mbar_init(bar_acc_empty + 8 * b, PAIR ? 16 : 8);            // one arrival per epilogue warp (of both CTAs)
+            mbar_init(bar_acc_empty + 8 * b, PAIR ? 2 * EPI_WARPS : EPI_WARPS);   // one arrival per epilogue warp (of both CTAs)
         }
         mbar_init(bar_drain, 1);
+        for (int k = 0; k < MAX_AKB; ++k) mbar_init(bar_a_empty + 8 * k, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -336,51 +383,109 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
 
     if (warp == 0) {
         // ================================ TMA producer ==========================================
-        // One lane per box: the first tpp lanes fetch this CTA's candidate tiles, the next lanes one
-        // quantum each (in a pair: this CTA's half of the piece's quanta), so a stage costs one
-        // barrier wait plus one copy instruction per lane.
+        // Every stage costs the issuing thread one look at the stage's "empty" barrier, its copies and one
+        // arrive on the "full" barrier.  When a CTA's candidate tiles are one box and its quanta of a piece
+        // are one box (the usual case: see a_merged / q_merged) lane 0 does all of that by itself, with no
+        // warp-wide exchange per stage; otherwise one lane per box: the first tpp lanes fetch the candidate
+        // tiles, the next lanes one quantum each (in a pair: this CTA's half of the piece's quanta).
         int stage = 0; uint32_t phase = 0;
+        uint32_t a_phase = 0;                         // resident candidate slots: flips with every row loaded
         uint32_t armed = 0;                           // stages with a copy possibly still in flight
         bool ok = true;
         bool joined = !early_producer;                // whether this warp has met the set-up barrier yet
+        const uint32_t ring_base = tiles_base + (uint32_t)P.a_region_bytes;       // (a_region_bytes is 0 unless a_res)
+        const bool solo = P.a_merged && P.q_merged;
+        const uint32_t a_step = P.a_res ? (uint32_t)(P.tpp * A_BYTES) : 0u;     // resident slot pitch
+        const uint32_t q_off = (uint32_t)(P.a_res ? 0 : P.tpp * A_BYTES);       // quanta inside a ring stage
+        int trp = -1;
         while (ok && walk.next(P, c)) {
+            ++trp;
             const int nq_mine = PAIR ? (c.nq >> 1) : c.nq;             // quanta this CTA fetches
             const int nA = P.a_merged ? 1 : P.tpp, nQ = P.q_merged ? 1 : nq_mine;   // boxes per stage
-            const CUtensorMap* map;
-            int w, h;
-            uint32_t dst_off;
-            if (lane < nA) {
-                map = &KP.mapsA[c.member];
-                // (tiles past the lattice are fetched as zeros and masked in the epilogue)
-                const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + lane;
-                const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
-                w = c.px * P.Ws + wtA * bwA; h = c.py * P.Hs + htA * P.bhA;
-                dst_off = (uint32_t)(lane * A_BYTES);
-            } else {
-                map = &KP.mapQ[(P.q_merged && nq_mine != P.q_lo) ? 1 : 0];
-                const int qi = c.q0 + (int)rank * nq_mine + lane - nA;
-                const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
-                w = c.px * P.Ws + wq * bwQ; h = c.py * P.Hs + hq * P.bhQ;
-                dst_off = (uint32_t)(P.tpp * A_BYTES + (lane - nA) * Q_BYTES);
-            }
-            const bool active = lane < nA + nQ;
+            // resident candidate tiles are fetched with the first piece of a row only, each 64-channel step
+            // into its own slot, and reported to the barrier of the ring stage that carries the same step
+            const bool load_a = !P.a_res || c.first;
             // what the leader's barrier expects per stage: the copies of both CTAs
-            const uint32_t bytes = (uint32_t)((PAIR ? 2 : 1) * (P.tpp * A_BYTES + nq_mine * Q_BYTES));
-            for (int kb = 0; kb < P.kblocks; ++kb) {
-                const uint32_t full_local = bar_full + 8 * stage;
-                const uint32_t full = PAIR ? map_to_cta(full_local, 0) : full_local;
-                bool go = true;
-                if (lane == 0) {
-                    go = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
-                    if (go && leader) mbar_arrive_expect_tx(full_local, bytes);
+            const uint32_t bytes = (uint32_t)((PAIR ? 2 : 1) * ((load_a ? P.tpp * A_BYTES : 0) + nq_mine * Q_BYTES));
+            if (solo) {
+                // (tiles past the lattice are fetched as zeros and masked in the epilogue)
+                const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp;
+                const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
+                const int wA = c.px * P.Ws + wtA * bwA, hA = c.py * P.Hs + htA * P.bhA;
+                const int qi = c.q0 + (int)rank * nq_mine;
+                const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
+                const int wQ = c.px * P.Ws + wq * bwQ, hQ = c.py * P.Hs + hq * P.bhQ;
+                const CUtensorMap* mapA = &KP.mapsA[c.member];
+                const CUtensorMap* mapQ = &KP.mapQ[nq_mine != P.q_lo ? 1 : 0];
+                for (int kb = 0; kb < P.kblocks; ++kb) {
+                    if (lane == 0 && ok) {
+                        const uint32_t full_local = bar_full + 8 * stage;
+                        const uint32_t full = PAIR ? map_to_cta(full_local, 0) : full_local;
+                        bool go = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
+                        // the slot of this step is free once the MMAs of the previous row's last piece have read it
+                        if (go && P.a_res && load_a) go = mbar_wait(bar_a_empty + 8 * kb, a_phase ^ 1u, abort_flag);
+                        if (go) {
+                            // the copies first, the arrival that carries their byte count after them: the barrier
+                            // cannot complete before that arrival, and the copies are on their way sooner
+                            tma_load_4d<PAIR>(ring_base + stage * STAGE_BYTES + q_off, mapQ, kb * BK, wQ, hQ, c.bt, full);
+                            if (load_a)
+                                tma_load_4d<PAIR>(P.a_res ? tiles_base + (uint32_t)kb * a_step : ring_base + stage * STAGE_BYTES,
+                                                  mapA, kb * BK, wA, hA, c.bt_a, full);
+                            if (leader) mbar_arrive_expect_tx(full_local, bytes);
+                        } else {
+                            ok = false;
+                        }
+                    }
+                    if (kb == 0) OC_TR(0, trp, 0, lane == 0);
+                    if (kb == P.kblocks - 1) OC_TR(0, trp, 1, lane == 0);
+                    armed |= 1u << stage;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    if (!joined) { __syncwarp(); __syncthreads(); joined = true; }   // first stage on its way: meet the others
                 }
-                go = __shfl_sync(0xFFFFFFFFu, (int)go, 0) != 0;
-                if (!go) { ok = false; break; }
-                if (active) tma_load_4d<PAIR>(tiles_base + stage * STAGE_BYTES + dst_off, map, kb * BK, w, h, lane < nA ? c.bt_a : c.bt, full);
-                armed |= 1u << stage;
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                if (!joined) { __syncthreads(); joined = true; }   // first stage on its way: meet the others
+                __syncwarp();
+                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;        // (lane 0 alone knows; once per piece)
+            } else {
+                const CUtensorMap* map;
+                int w, h;
+                uint32_t dst_off;
+                if (lane < nA) {
+                    map = &KP.mapsA[c.member];
+                    const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + lane;
+                    const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
+                    w = c.px * P.Ws + wtA * bwA; h = c.py * P.Hs + htA * P.bhA;
+                    dst_off = (uint32_t)(lane * A_BYTES);
+                } else {
+                    map = &KP.mapQ[(P.q_merged && nq_mine != P.q_lo) ? 1 : 0];
+                    const int qi = c.q0 + (int)rank * nq_mine + lane - nA;
+                    const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
+                    w = c.px * P.Ws + wq * bwQ; h = c.py * P.Hs + hq * P.bhQ;
+                    dst_off = q_off + (uint32_t)((lane - nA) * Q_BYTES);
+                }
+                const bool active = lane < nA ? load_a : lane < nA + nQ;
+                for (int kb = 0; kb < P.kblocks; ++kb) {
+                    const uint32_t full_local = bar_full + 8 * stage;
+                    const uint32_t full = PAIR ? map_to_cta(full_local, 0) : full_local;
+                    bool go = true;
+                    if (lane == 0) {
+                        go = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
+                        if (go && P.a_res && load_a) go = mbar_wait(bar_a_empty + 8 * kb, a_phase ^ 1u, abort_flag);
+                        if (go && leader) mbar_arrive_expect_tx(full_local, bytes);
+                    }
+                    go = __shfl_sync(0xFFFFFFFFu, (int)go, 0) != 0;
+                    if (!go) { ok = false; break; }
+                    if (kb == 0) OC_TR(0, trp, 0, lane == 0);
+                    if (kb == P.kblocks - 1) OC_TR(0, trp, 1, lane == 0);
+                    if (active) {
+                        const uint32_t dst = (lane < nA && P.a_res) ? tiles_base + (uint32_t)kb * a_step + dst_off
+                                                                    : ring_base + stage * STAGE_BYTES + dst_off;
+                        tma_load_4d<PAIR>(dst, map, kb * BK, w, h, lane < nA ? c.bt_a : c.bt, full);
+                    }
+                    armed |= 1u << stage;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    if (!joined) { __syncthreads(); joined = true; }   // first stage on its way: meet the others
+                }
             }
+            if (P.a_res && load_a) a_phase ^= 1u;
         }
         if (!joined) { __syncthreads(); joined = true; }
         if (!ok && lane == 0) {
@@ -414,7 +519,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 // epilogue of a piece runs under the MMAs of the next one
                 const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
                 ++it;
+                OC_TR(1, (int)it - 1, 0, lane == 0);
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_empty + 8 * buf, acc_phase ^ 1u, abort_flag))) { ok = false; break; }
+                OC_TR(1, (int)it - 1, 1, lane == 0);
                 const uint32_t d_tmem = tmem_base + buf * 256u;
                 tc_fence_after();
                 const uint32_t idesc = IDESC_BASE | ((uint32_t)(c.ncol >> 3) << 17);
@@ -426,12 +533,14 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     //  full stays right, and the others wait here)
                     if (!peeked && !mbar_wait(bar_full + 8 * stage, phase, abort_flag)) ok = false;
                     if (!__all_sync(0xFFFFFFFFu, ok)) { ok = false; break; }
-                    const uint32_t a_addr = tiles_base + stage * STAGE_BYTES;
+                    if (kb == 0) OC_TR(1, (int)it - 1, 2, lane == 0);
+                    const uint32_t s_addr = tiles_base + (uint32_t)P.a_region_bytes + stage * STAGE_BYTES;
+                    const uint32_t a_addr = P.a_res ? tiles_base + (uint32_t)(kb * P.tpp * A_BYTES) : s_addr;
                     const uint64_t a0_desc = make_smem_desc(a_addr);
                     const uint64_t a1_desc = make_smem_desc(a_addr + A_BYTES);
                     // (a piece that begins in mid-quantum skips 16 rows = 2 KB of its first box: a whole number
                     //  of 8-row swizzle groups)
-                    const uint64_t b_desc = make_smem_desc(a_addr + P.tpp * A_BYTES + (uint32_t)c.c_off * 128u);
+                    const uint64_t b_desc = make_smem_desc(s_addr + (P.a_res ? 0 : P.tpp * A_BYTES) + (uint32_t)c.c_off * 128u);
                     int nstage = stage + 1; uint32_t nphase = phase;
                     if (nstage == STAGES) { nstage = 0; nphase ^= 1u; }
                     // UMMA K = 16 is 32 bytes along the swizzled row: +2 in the descriptor's address field
@@ -440,8 +549,13 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     // frees the stage (in both CTAs of a pair) when the MMAs retire
                     tc_commit<PAIR>(PAIR ? map_to_cta(bar_empty + 8 * stage, 0) : bar_empty + 8 * stage, issue);
                     if (PAIR) tc_commit<PAIR>(map_to_cta(bar_empty + 8 * stage, 1), issue);
+                    if (P.a_res && c.last) {         // the row's candidate tiles of this step have been read for the last time
+                        tc_commit<PAIR>(PAIR ? map_to_cta(bar_a_empty + 8 * kb, 0) : bar_a_empty + 8 * kb, issue);
+                        if (PAIR) tc_commit<PAIR>(map_to_cta(bar_a_empty + 8 * kb, 1), issue);
+                    }
                     stage = nstage; phase = nphase;
                 }
+                OC_TR(1, (int)it - 1, 3, lane == 0);
                 if (ok) {
                     tc_commit<PAIR>(PAIR ? map_to_cta(bar_acc_full + 8 * buf, 0) : bar_acc_full + 8 * buf, issue);
                     if (PAIR) tc_commit<PAIR>(map_to_cta(bar_acc_full + 8 * buf, 1), issue);
@@ -456,7 +570,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     } else {
         // ================================ epilogue ==============================================
         const int et = threadIdx.x - 64;                               // 0..255
-        const int half = et >> 7;                                      // which half of the piece's columns
+        const int part = et >> 7;                                      // which part of the piece's columns
         const int lane_group = warp & 3;                               // TMEM lanes this warp may read
         const int row = lane_group * 32 + lane;                        // tile row owned by this thread
         bool ok = true;
@@ -484,15 +598,15 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         if (et == 0) pdl_launch_dependents();
         Piece nx;
         bool have = walk.next(P, c);
-        if (have) col_scale[et] = table_entry(c);
-        if (!epilogue_barrier_all(ok)) { ok = false; have = false; }
+        if (have && et < 256) col_scale[et] = table_entry(c);
+        if (!epilogue_barrier_all<32 * EPI_WARPS>(ok)) { ok = false; have = false; }
         while (have) {
             const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
             const float4* col_scale4 = (const float4*)(col_scale + (it & 1u) * 256);
             const float* col_scale1 = col_scale + (it & 1u) * 256;
             const bool have_nx = walk.next(P, nx);
             float sc_nx = 0.f;
-            if (have_nx) sc_nx = table_entry(nx);                      // in flight until the end of this piece
+            if (have_nx && et < 256) sc_nx = table_entry(nx);          // in flight until the end of this piece
             const int my = (c.member * P.sx_magic) >> 16, mx = c.member - my * P.sx;
             long long tokA0, tokA1; bool row_ok0, row_ok1;
             {
@@ -513,10 +627,12 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             }
             // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
             const int n_ch = (c.ncol + 31) >> 5;                        // (a last half chunk reads 16 columns of
-            const int ch_split = (n_ch + 1) >> 1;                      //  nothing: their table entries are NaN)
-            const int ch_begin = half ? ch_split : 0, ch_end = half ? n_ch : ch_split;
+            const int ch_begin = (part * n_ch + EPI_PARTS - 1) / EPI_PARTS;      //  nothing: their table entries are NaN)
+            const int ch_end = ((part + 1) * n_ch + EPI_PARTS - 1) / EPI_PARTS;
             // warp-uniform outcome: the TMEM loads below are warp-collective
+            OC_TR(2, (int)it, 0, et == 0);
             const bool ready = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * buf, acc_phase, abort_flag));
+            OC_TR(2, (int)it, 1, et == 0);
             if (ready) {
                 tc_fence_after();
 #pragma unroll 1
@@ -537,46 +653,30 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     // replaced by 31 - (column within the chunk), so that ONE three-input max per two
                     // columns carries the arg max along (among equal similarities the lowest column has
                     // the largest key).  The similarity loses 5 of its 24 mantissa bits (2^-18 relative),
-                    // far inside the tolerance of a bf16 match.  Two independent chains; bc = the chunk in
-                    // which a chain last rose.
-                    float bm0 = -INFINITY, bm1 = -INFINITY;
-                    int bc0 = -1, bc1 = -1;
+                    // far inside the tolerance of a bf16 match.  The 32 keys of a chunk are reduced by a tree
+                    // of depth 4 (a running maximum would be a chain of 16 dependent instructions, and with two
+                    // epilogue warps per scheduler nothing else hides that latency); bc = the chunk in which the
+                    // row's maximum last rose.
+                    float bm = -INFINITY;
+                    int bc = -1;
                     const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)t * tile_stride + buf * 256u;
                     // two register buffers: the TMEM load of the next step is in flight while this one is reduced
                     uint32_t va[32], vb[32];
 #define OC_KEY(v, s, j) __uint_as_float((__float_as_uint(__uint_as_float(v) * (s)) & 0xFFFFFFE0u) | (uint32_t)(31 - (j)))
-#define OC_KEY_NEG(v, s, j) __uint_as_float((__float_as_uint(__uint_as_float(v) * (s)) & 0xFFFFFFE0u) | (uint32_t)(j))
+#define OC_KEY_ANY(v, s, j) oc_key_any(__uint_as_float(v) * (s), (j))
 #define OC_VAL(k) __uint_as_float(__float_as_uint(k) & 0xFFFFFFE0u)
 #define OC_COL(k) ((__float_as_uint(k) >> 31) ? (int)(__float_as_uint(k) & 31u) : 31 - (int)(__float_as_uint(k) & 31u))
 #define OC_REDUCE_CHUNK(v, ch)                                                                                   \
     do {                                                                                                         \
-        float cm0 = -INFINITY, cm1 = -INFINITY;                                                                  \
+        float kf[32];                                                                                            \
         _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
             const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                                   \
-            cm0 = max3f(cm0, OC_KEY(v[j], s4.x, j), OC_KEY(v[j + 1], s4.y, j + 1));                              \
-            cm1 = max3f(cm1, OC_KEY(v[j + 2], s4.z, j + 2), OC_KEY(v[j + 3], s4.w, j + 3));                      \
+            kf[j] = OC_KEY(v[j], s4.x, j); kf[j + 1] = OC_KEY(v[j + 1], s4.y, j + 1);                            \
+            kf[j + 2] = OC_KEY(v[j + 2], s4.z, j + 2); kf[j + 3] = OC_KEY(v[j + 3], s4.w, j + 3);                \
         }                                                                                                        \
-        /* A chain whose maximum is negative holds negative similarities only.  Among negative floats the  */   \
-        /* larger mantissa is the SMALLER value, so there the column goes into the low bits as it is (the  */   \
-        /* lowest column is then the largest key again).  Rare (every one of 16 cosines negative), so the */   \
-        /* chain is simply taken a second time.                                                           */   \
-        if (cm0 < 0.f) {                                                                                         \
-            cm0 = -INFINITY;                                                                                     \
-            _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                  \
-                const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                               \
-                cm0 = max3f(cm0, OC_KEY_NEG(v[j], s4.x, j), OC_KEY_NEG(v[j + 1], s4.y, j + 1));                  \
-            }                                                                                                    \
-        }                                                                                                        \
-        if (cm1 < 0.f) {                                                                                         \
-            cm1 = -INFINITY;                                                                                     \
-            _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                  \
-                const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                               \
-                cm1 = max3f(cm1, OC_KEY_NEG(v[j + 2], s4.z, j + 2), OC_KEY_NEG(v[j + 3], s4.w, j + 3));          \
-            }                                                                                                    \
-        }                                                                                                        \
+        const float cm = key_tree_max(kf);                                                                       \
         /* a later chunk wins only with a strictly larger similarity (the index bits set aside) */              \
-        if (OC_VAL(cm0) > OC_VAL(bm0)) { bm0 = cm0; bc0 = (ch); }                                                \
-        if (OC_VAL(cm1) > OC_VAL(bm1)) { bm1 = cm1; bc1 = (ch); }                                                \
+        if (OC_VAL(cm) > OC_VAL(bm)) { bm = cm; bc = (ch); }                                                     \
         if (AUX && aux_row) {                                                                                    \
             for (int j = 0; j < 32; ++j) {                                                                       \
                 const float sc = col_scale1[(ch) * 32 + j];                                                      \
@@ -590,26 +690,49 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             }                                                                                                    \
         }                                                                                                        \
     } while (0)
+                    if (t == 0) OC_TR(3, (int)it, 0, et == 0);
                     if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
 #pragma unroll 1
                     for (int ch = ch_begin; ch < ch_end; ch += 2) {
                         tmem_ld_wait();
+                        if (t == 0 && ch == ch_begin) OC_TR(3, (int)it, 1, et == 0);
                         if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);
                         OC_REDUCE_CHUNK(va, ch);
+                        if (t == 0 && ch == ch_begin) OC_TR(3, (int)it, 2, et == 0);
                         if (ch + 1 < ch_end) {
                             tmem_ld_wait();
+                            if (t == 0 && ch == ch_begin) OC_TR(3, (int)it, 3, et == 0);
                             if (ch + 2 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), va);
                             OC_REDUCE_CHUNK(vb, ch + 1);
                         }
                     }
 #undef OC_REDUCE_CHUNK
+                    // A chain whose maximum is negative has seen negative similarities only, and among negative
+                    // floats the larger mantissa is the SMALLER value: the keys above then prefer the highest
+                    // column among equal similarities.  Such a row is taken again from TMEM (the accumulators are
+                    // still there) with keys that store the column itself under a negative value.  Rare -- all
+                    // of a row's cosines negative -- and warp-uniform, because the TMEM loads are collective.
+                    if (__any_sync(0xFFFFFFFFu, bc >= 0 && bm < 0.f)) {
+                        bm = -INFINITY; bc = -1;
+#pragma unroll 1
+                        for (int ch = ch_begin; ch < ch_end; ++ch) {
+                            tmem_ld32(t_row + (uint32_t)(ch * 32), va);
+                            tmem_ld_wait();
+                            float kf[32];
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                const float4 s4 = col_scale4[ch * 8 + (j >> 2)];
+                                kf[j] = OC_KEY_ANY(va[j], s4.x, j); kf[j + 1] = OC_KEY_ANY(va[j + 1], s4.y, j + 1);
+                                kf[j + 2] = OC_KEY_ANY(va[j + 2], s4.z, j + 2); kf[j + 3] = OC_KEY_ANY(va[j + 3], s4.w, j + 3);
+                            }
+                            const float cm = key_tree_max(kf);
+                            if (OC_VAL(cm) > OC_VAL(bm)) { bm = cm; bc = ch; }
+                        }
+                    }
 #undef OC_KEY
-#undef OC_KEY_NEG
-                    // the better chain; among equal similarities the lower column
-                    int n0 = bc0 < 0 ? -1 : bc0 * 32 + OC_COL(bm0);
-                    const int n1 = bc1 < 0 ? -1 : bc1 * 32 + OC_COL(bm1);
-                    float best = OC_VAL(bm0);
-                    if (n1 >= 0 && (n0 < 0 || OC_VAL(bm1) > best || (OC_VAL(bm1) == best && n1 < n0))) { best = OC_VAL(bm1); n0 = n1; }
+#undef OC_KEY_ANY
+                    const int n0 = bc < 0 ? -1 : bc * 32 + OC_COL(bm);
+                    const float best = OC_VAL(bm);
 #undef OC_VAL
 #undef OC_COL
                     if (row_ok && n0 >= 0) {
@@ -624,6 +747,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 }
                 tc_fence_before();
                 __syncwarp();
+                OC_TR(2, (int)it, 2, et == 0);
                 if (lane == 0) {                                       // both accumulators may be overwritten
                     if (PAIR) mbar_arrive_cluster(acc_empty + 8 * buf); else mbar_arrive(bar_acc_empty + 8 * buf);
                 }
@@ -632,8 +756,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             }
             // the next piece's table entries; the barrier publishes them, and keeps the table just read
             // from being overwritten (in the next turn) while a slower warp still reads it
-            if (have_nx) col_scale[((it + 1u) & 1u) * 256 + et] = sc_nx;
-            if (!epilogue_barrier_all(ok)) { ok = false; break; }
+            if (have_nx && et < 256) col_scale[((it + 1u) & 1u) * 256 + et] = sc_nx;
+            if (!epilogue_barrier_all<32 * EPI_WARPS>(ok)) { ok = false; break; }
+            OC_TR(2, (int)it, 3, et == 0);
             c = nx; have = have_nx;
             ++it;
         }
@@ -705,13 +830,14 @@ static int pow2_ceil_log2(int v) { int l = 0; while ((1 << l) < v) ++l; return l
 
 struct TcPlan {
     int bwA_log2, bhA, n_wtA, n_tilesA, tpp, n_apairs, bwQ_log2, bhQ, n_wq, n_quanta;
-    int pair, q_unit, n_q_units, half_units, a_merged, q_merged, q_lo, q_hi;
+    int pair, q_unit, n_q_units, half_units, a_merged, q_merged, q_lo, q_hi, q_rows;
     int pieces_per_row, qmax, n_stages, stage_bytes, narrow;
+    int a_res, a_region_bytes;
     long long rows, items;
 };
 
 // A forced work split (oc_tc_plan_override): the tests run every form of the kernel this way.
-struct TcForce { bool on; int pair, tiles, pieces, no_narrow; };
+struct TcForce { bool on; int pair, tiles, pieces, no_narrow, a_res /* -1: the planner's choice */; };
 
 // walkers: CTAs that can run at once; pair_walkers: CTA pairs that can (0 = pairs not available)
 static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcForce& force) {
@@ -724,21 +850,19 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
     p.bwQ_log2 = lq; p.bhQ = QN >> lq;
     p.n_wq = (g.Ws + (1 << lq) - 1) >> lq;
     p.n_quanta = p.n_wq * ((g.Hs + p.bhQ - 1) / p.bhQ);
-    // Form (single CTA or CTA pair), candidate tiles per CTA (1 or 2) and pieces per row, by estimated
-    // cycles of the busiest walker.  The shape of the estimate follows the kernel; its constants were
-    // fitted to timed sweeps of all valid plans on six workloads (SD3-shaped token cache at 1/4/8
-    // token groups per image, the three SVD UNet levels):
-    //   * per 64-channel stage a CTA fetches tpp*16 KB of candidates plus 4 KB per quantum it loads
-    //     (all q of the piece, or q/2 in a pair) and issues tpp*64*q tensor cycles; the stage takes the
-    //     longest of the MMAs (+~50 cycles between stages), the fetch at ~74 B/clk, and - once the ring
-    //     has been drained - the refill round trip (MMAs + ~330 + ~1500 cycles of copy latency, ~1000
-    //     more in a pair) divided by the stages that fit in the ring;
-    //   * the epilogue costs ~250 + ~410 cycles per 32 columns of each thread's half, per tile; with two
-    //     tiles per CTA it follows the MMAs of the piece, with one tile - or with two tiles and pieces of
-    //     at most 128 columns, which leave room for a second set of accumulators - it runs under the
-    //     next piece's MMAs, where the two slow each other down (~0.8, resp. ~0.4, of the shorter one is
-    //     not hidden);
-    //   * ~6500 cycles before a CTA's first MMA and after its last.
+    // Form (single CTA or CTA pair), candidate tiles per CTA (1 or 2), pieces per row and whether the
+    // candidate tiles stay resident, by estimated cycles of the busiest walker.  The shape of the estimate
+    // follows the kernel; its constants were fitted (least squares on the logarithm, over 60 timed plans)
+    // to sweeps of forced plans on four workloads (the SD3-shaped token cache and the three SVD UNet
+    // levels) and reproduce every one of those times within a few per cent:
+    //   * a 64-channel stage issues tpp*64*q tensor cycles and cannot go faster than the hand-over of a
+    //     ring slot between the copy producer and the MMA issuer (~650 cycles while the epilogue runs
+    //     beside the MMAs, ~950 when it follows them), nor than its bytes at ~58 B/clk;
+    //   * the epilogue costs ~420 + ~370 cycles per 32 columns of each thread's half, per tile; with two
+    //     accumulator sets (one tile, or two tiles and pieces of at most 128 columns) it runs under the
+    //     next piece's MMAs and the piece takes the longer of the two plus ~13 % of the shorter,
+    //     otherwise it follows them;
+    //   * ~2500 cycles before a CTA's first MMA and after its last.
     const int kblocks = (g.C + BK - 1) / BK;
     // Single-CTA pieces are cut in units of HALF a quantum (16 columns) whenever that is valid: no piece
     // wider than 256 columns, none that would have to fetch more than MAXQ quanta (one that begins in
@@ -751,7 +875,7 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
         if (h_max == 2 * MAXQ && !(n_half % P == 0 && (h_max & 1) == 0)) return 0;   // 256 columns only from even starts
         return h_max;
     };
-    double best_cost = 0; int best_P = 0, best_tpp = 2, best_pair = 0;
+    double best_cost = 0; int best_P = 0, best_tpp = 2, best_pair = 0, best_ar = 0;
     for (int pair = 0; pair <= (pair_walkers > 0 ? 1 : 0); ++pair) {
         const int ncta = pair ? 2 : 1, q_unit = pair ? 2 : 1;
         const int n_units = (p.n_quanta + q_unit - 1) / q_unit, max_units = MAXQ / q_unit;
@@ -766,29 +890,29 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
                 if (hw) { q_load = (hw + 2) >> 1; if (q_load > MAXQ) q_load = MAXQ; }
                 const double qe = hw ? hw * 0.5 : (double)q;          // width in quanta (may end in a half)
                 if (hw) q = (hw + 1) >> 1;
-                const double stage_kb = tpp * 16.0 + 4.0 * q_load / ncta;
-                int stages = (int)(TILE_BYTES / 1024 / stage_kb); if (stages > MAX_STAGES) stages = MAX_STAGES;
                 const long long per_walker = (rows * P + nw - 1) / nw;
-                const double mma = tpp * 64.0 * qe, fetch = stage_kb * 1024.0 / 74.0;
-                const double refill = (mma + 330.0 + 1450.0 + 1.35 * stage_kb + (pair ? 980.0 : 0.0)) / stages;
-                double fast = mma + 53.0; if (fetch > fast) fast = fetch;
-                const double slow = refill > fast ? refill : fast;
-                const double epi = tpp * (246.0 + 413.0 * ((q + 1) / 2));
-                double piece;
+                const double mma = tpp * 64.0 * qe;
+                const double epi = tpp * (420.0 + 370.0 * ((q + 1) / 2));
                 // (two tiles whose pieces are at most 128 columns wide leave room for a second set of
                 //  accumulators, like one tile does)
                 const bool overlapped = tpp == 1 || (hw ? hw * 16 : q * 32) <= 128;
-                if (overlapped) {
-                    const double loop = kblocks * slow;
-                    // (the part of the shorter of the two that is not hidden: fitted, one tile 0.79, two narrow tiles 0.36)
-                    piece = (loop + 440.0 > epi ? loop + 440.0 : epi) + (tpp == 1 ? 0.79 : 0.36) * (loop < epi ? loop : epi);
-                } else {
-                    const int nf = kblocks < stages ? kblocks : stages;
-                    piece = nf * fast + (kblocks - nf) * slow + epi + 534.0;
+                for (int ar = 0; ar <= 1; ++ar) {
+                    const double a_kb = tpp * 16.0, q_kb = 4.0 * q_load / ncta;
+                    if (ar && (kblocks > MAX_AKB || a_kb * kblocks + 3 * q_kb > TILE_BYTES / 1024 || P == 1)) continue;
+                    const double feed = ((ar ? 0.0 : a_kb) + q_kb) * 1024.0 / 58.4;
+                    double piece;
+                    if (overlapped) {
+                        double stage = mma + 46.0; if (stage < 648.0) stage = 648.0; if (stage < feed) stage = feed;
+                        const double loop = kblocks * stage + 904.0, tail = epi + 2919.0;
+                        piece = (loop > tail ? loop : tail) + 0.13 * (kblocks * stage < epi ? kblocks * stage : epi);
+                    } else {
+                        double stage = mma + 480.0; if (stage < 948.0) stage = 948.0; if (stage < feed) stage = feed;
+                        piece = kblocks * stage + epi + 1022.0;
+                    }
+                    if (pair) piece += 850.0;
+                    const double cost = 2450.0 + per_walker * piece + (overlapped ? epi : 0.0);
+                    if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; best_tpp = tpp; best_pair = pair; best_ar = ar; }
                 }
-                if (pair) piece += 850.0;
-                const double cost = 6550.0 + (pair ? 616.0 : 0.0) + per_walker * piece + (overlapped ? epi : 0.0);
-                if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; best_tpp = tpp; best_pair = pair; }
             }
         }
     }
@@ -809,13 +933,18 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
     p.n_apairs = (p.n_tilesA + p.tpp * ncta - 1) / (p.tpp * ncta);
     p.rows = g.n_groups * (long long)(g.sy * g.sx - 1) * p.n_apairs;
     p.pieces_per_row = best_P;
-    // fewest and most quanta any piece fetches (per CTA)
+    // fewest and most quanta any piece fetches (per CTA); and whether every CTA's run of quanta is a whole
+    // number of lattice rows (lattices wider than one quantum: the run is then one rectangle of rows)
     int q_min = 1 << 30, q_max = 0;
+    bool whole_rows = p.n_wq > 1 && p.bhQ == 1 && p.n_wq * QN <= 256;
     for (int j = 0; j < best_P; ++j) {
         const int u0 = (int)((long long)j * p.n_q_units / best_P), u1 = (int)((long long)(j + 1) * p.n_q_units / best_P);
+        const int q0 = p.half_units ? (u0 >> 1) : u0 * p.q_unit;
         int nq = p.half_units ? ((u1 - 1) >> 1) - (u0 >> 1) + 1 : (u1 - u0) * p.q_unit / ncta;
         if (nq < q_min) q_min = nq;
         if (nq > q_max) q_max = nq;
+        for (int r = 0; r < ncta; ++r)
+            if ((q0 + r * nq) % p.n_wq != 0 || nq % p.n_wq != 0) whole_rows = false;
     }
     p.qmax = q_max * ncta;
     {   // widest piece in columns (a forced split may keep such plans on one accumulator set)
@@ -823,16 +952,24 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
         const int cols = hw ? hw * 16 : ((p.n_q_units + best_P - 1) / best_P) * p.q_unit * 32;
         p.narrow = (p.tpp == 2 && cols <= 128 && !(force.on && force.no_narrow)) ? 1 : 0;
     }
-    p.stage_bytes = p.tpp * A_BYTES + q_max * Q_BYTES;
-    p.n_stages = TILE_BYTES / p.stage_bytes;
+    // Candidate tiles resident (all 64-channel steps of a CTA's tiles in front of the ring, fetched once per
+    // row instead of once per piece): possible when they leave room for at least three ring stages of
+    // representatives.
+    const int a_region = p.tpp * A_BYTES * kblocks;
+    const bool a_res_ok = kblocks <= MAX_AKB && a_region + 3 * q_max * Q_BYTES <= TILE_BYTES && best_P > 1;
+    p.a_res = a_res_ok ? (force.on ? (force.a_res != 0) : (best_ar != 0)) : 0;
+    p.a_region_bytes = p.a_res ? a_region : 0;
+    p.stage_bytes = (p.a_res ? 0 : p.tpp * A_BYTES) + q_max * Q_BYTES;
+    p.n_stages = (TILE_BYTES - p.a_region_bytes) / p.stage_bytes;
     if (p.n_stages > MAX_STAGES) p.n_stages = MAX_STAGES;
     p.items = p.rows * p.pieces_per_row;
     // One copy instruction costs the producer ~100 cycles whatever the box size, so a CTA's candidate
     // tiles, and its quanta of a piece, travel as ONE box each whenever they stack into a rectangle
     // of lattice rows (always the case when the patch's lattice is at most one box wide).
     p.a_merged = (p.tpp == 1 || p.n_wtA == 1) ? 1 : 0;
-    p.q_merged = p.n_wq == 1 ? 1 : 0;
-    p.q_lo = q_min;                           // merged boxes come in two heights: q_lo and q_lo + 1 quanta
+    p.q_rows = whole_rows ? 1 : 0;            // ... or when every run of quanta is a rectangle of whole lattice rows
+    p.q_merged = (p.n_wq == 1 || whole_rows) ? 1 : 0;
+    p.q_lo = q_min;                           // merged boxes come in two heights: q_lo and q_hi quanta
     p.q_hi = q_max;
     return p;
 }
@@ -845,29 +982,9 @@ bool tc_match_supported(const Geo& g) {
     return encode_fn() != nullptr;
 }
 
-static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm, unsigned long long* keys,
-                           float* aux_sim, const int4* units, const int* n_units_dev, long long max_units, cudaStream_t s);
-
-oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm,
-                                unsigned long long* keys, float* aux_sim, cudaStream_t s) {
-    return launch_tc(ctx, g, x, inv_norm, keys, aux_sim, nullptr, nullptr, 0, s);
-}
-
-// Joint form: `units` (device) lists {representative frame, candidate frame, member} triples, `n_units_dev`
-// (device) how many; max_units bounds the list (it sizes the launch).  g: one patch per frame.
-oc_status launch_match_joint_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm,
-                                unsigned long long* keys, const int4* units, const int* n_units_dev,
-                                long long max_units, cudaStream_t s) {
-    if (g.gy != 1 || g.gx != 1 || !units || !n_units_dev || max_units <= 0) return OC_ERR_UNSUPPORTED;
-    return launch_tc(ctx, g, x, inv_norm, keys, nullptr, units, n_units_dev, max_units, s);
-}
-
-static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm, unsigned long long* keys,
-                           float* aux_sim, const int4* units, const int* n_units_dev, long long max_units, cudaStream_t s) {
-    EncodeTiledFn enc = encode_fn();
-    if (!enc) return OC_ERR_UNSUPPORTED;
-    // once per device (the context's device is current here): opt in to the large dynamic shared
-    // memory, and ask how many CTA pairs fit
+// Once per device (the context's device is current): opt in to the large dynamic shared memory and ask
+// how many CTA pairs fit.  False if the attributes could not be set.
+static bool tc_device_setup(oc_ctx* ctx, int* pair_walkers_out) {
     static PerDeviceOnce attr_once;
     static int max_pairs[PerDeviceOnce::MAX_DEV];
     const int dev = ctx->device;
@@ -895,9 +1012,53 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
         }
         return true;
     });
-    if (!attr_ok) return OC_ERR_CUDA;
-    const int pair_walkers = (dev >= 0 && dev < PerDeviceOnce::MAX_DEV) ? max_pairs[dev] : 0;
-    const TcForce force = {ctx->tc_plan_forced, ctx->tc_plan_pair, ctx->tc_plan_tiles, ctx->tc_plan_pieces, ctx->tc_plan_no_narrow};
+    *pair_walkers_out = (attr_ok && dev >= 0 && dev < PerDeviceOnce::MAX_DEV) ? max_pairs[dev] : 0;
+    return attr_ok;
+}
+
+oc_status tc_plan_describe(oc_ctx* ctx, const Geo& g, int32_t* out) {
+    if (!tc_match_supported(g)) return OC_ERR_UNSUPPORTED;
+    int pair_walkers = 0;
+    if (!tc_device_setup(ctx, &pair_walkers)) return OC_ERR_CUDA;
+    const TcForce force = {ctx->tc_plan_forced, ctx->tc_plan_pair, ctx->tc_plan_tiles, ctx->tc_plan_pieces, ctx->tc_plan_no_narrow,
+                           ctx->tc_plan_a_res};
+    const TcPlan p = make_plan(g, ctx->sm_count, pair_walkers, force);
+    long long walkers = p.items;
+    const int cap = p.pair ? pair_walkers : ctx->sm_count;
+    if (walkers > cap) walkers = cap;
+    const int widest = p.half_units ? ((2 * p.n_quanta + p.pieces_per_row - 1) / p.pieces_per_row) * 16
+                                    : ((p.n_q_units + p.pieces_per_row - 1) / p.pieces_per_row) * p.q_unit * 32;
+    const int v[12] = {p.pair, p.tpp, p.pieces_per_row, (p.tpp == 1 || p.narrow) ? 1 : 0, p.n_stages, p.stage_bytes, p.a_res,
+                       (int)(p.items > 0x7FFFFFFFll ? 0x7FFFFFFF : p.items), (int)walkers, widest, (g.C + BK - 1) / BK, 0};
+    for (int i = 0; i < 12; ++i) out[i] = v[i];
+    return OC_OK;
+}
+
+static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm, unsigned long long* keys,
+                           float* aux_sim, const int4* units, const int* n_units_dev, long long max_units, cudaStream_t s);
+
+oc_status launch_match_token_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm,
+                                unsigned long long* keys, float* aux_sim, cudaStream_t s) {
+    return launch_tc(ctx, g, x, inv_norm, keys, aux_sim, nullptr, nullptr, 0, s);
+}
+
+// Joint form: `units` (device) lists {representative frame, candidate frame, member} triples, `n_units_dev`
+// (device) how many; max_units bounds the list (it sizes the launch).  g: one patch per frame.
+oc_status launch_match_joint_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm,
+                                unsigned long long* keys, const int4* units, const int* n_units_dev,
+                                long long max_units, cudaStream_t s) {
+    if (g.gy != 1 || g.gx != 1 || !units || !n_units_dev || max_units <= 0) return OC_ERR_UNSUPPORTED;
+    return launch_tc(ctx, g, x, inv_norm, keys, nullptr, units, n_units_dev, max_units, s);
+}
+
+static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float* inv_norm, unsigned long long* keys,
+                           float* aux_sim, const int4* units, const int* n_units_dev, long long max_units, cudaStream_t s) {
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return OC_ERR_UNSUPPORTED;
+    int pair_walkers = 0;
+    if (!tc_device_setup(ctx, &pair_walkers)) return OC_ERR_CUDA;
+    const TcForce force = {ctx->tc_plan_forced, ctx->tc_plan_pair, ctx->tc_plan_tiles, ctx->tc_plan_pieces, ctx->tc_plan_no_narrow,
+                           ctx->tc_plan_a_res};
     const TcPlan p = make_plan(g, ctx->sm_count, pair_walkers, force);
     if (p.items > 0x7FFFFFFFll) return OC_ERR_UNSUPPORTED;
 
@@ -912,9 +1073,12 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     const cuuint32_t boxA[4] = {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwA_log2),
                                 (cuuint32_t)(p.bhA * (p.a_merged ? p.tpp : 1)), 1};
     const int q_hi = p.q_hi;
+    // (a run of whole lattice rows: the box is n_wq quanta wide and one lattice row per n_wq quanta high)
+    const cuuint32_t q_box_w = (cuuint32_t)(p.q_rows ? p.n_wq * QN : (1 << p.bwQ_log2));
+    const int q_per_h = p.q_rows ? p.n_wq : 1;
     const cuuint32_t boxQ[2][4] = {
-        {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwQ_log2), (cuuint32_t)(p.bhQ * (p.q_merged ? p.q_lo : 1)), 1},
-        {(cuuint32_t)BK, (cuuint32_t)(1 << p.bwQ_log2), (cuuint32_t)(p.bhQ * (p.q_merged ? q_hi : 1)), 1}};
+        {(cuuint32_t)BK, q_box_w, (cuuint32_t)(p.bhQ * (p.q_merged ? p.q_lo / q_per_h : 1)), 1},
+        {(cuuint32_t)BK, q_box_w, (cuuint32_t)(p.bhQ * (p.q_merged ? q_hi / q_per_h : 1)), 1}};
     const int rep_member = g.oy * g.sx + g.ox;
     const int n_members = g.sy * g.sx;
     for (int m = 0; m < n_members + 2; ++m) {
@@ -938,6 +1102,7 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     P.q_unit = p.q_unit; P.n_q_units = p.n_q_units; P.half_units = p.half_units;
     P.a_merged = p.a_merged; P.q_merged = p.q_merged; P.q_lo = p.q_lo;
     P.n_stages = p.n_stages; P.stage_bytes = p.stage_bytes;
+    P.a_res = p.a_res; P.a_region_bytes = p.a_region_bytes;
     P.units_per_group = (int)g.units_per_group; P.reps_per_group = (int)g.reps_per_group;
     P.inv_norm = inv_norm; P.keys = keys; P.aux = aux_sim; P.status = ctx->d_status;
     if (ctx->span_on) {
@@ -978,3 +1143,12 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
 }
 
 }  // namespace oc
+
+#ifdef OC_TC_TRACE
+extern "C" int oc_debug_tc_trace_read(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, oc::g_tc_trace, sizeof(oc::g_tc_trace));
+}
+extern "C" int oc_debug_tc_stage_read(unsigned long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, oc::g_tc_stage, sizeof(oc::g_tc_stage));
+}
+#endif

@@ -107,16 +107,17 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
     return d;
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Barrier over the 256 epilogue threads that also ANDs a flag: every thread learns whether any
+// Barrier over the NT epilogue threads that also ANDs a flag: every thread learns whether any
 // thread has given up, so they all leave the piece loop together.
+template <int NT>
 __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 1, 256, q;\n\t"
+        "bar.red.and.pred p, 1, %2, q;\n\t"
         "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(r) : "r"((uint32_t)ok) : "memory");
+        : "=r"(r) : "r"((uint32_t)ok), "n"(NT) : "memory");
     return r != 0;
 }
 

@@ -34,7 +34,7 @@ EXPORTS = (
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
     "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
     "oc_schedule_propose", "oc_joint_workspace_bytes", "oc_joint_groups", "oc_match_joint", "oc_select_joint",
-    "oc_linear_gather_scatter", "oc_tc_plan_override",
+    "oc_linear_gather_scatter", "oc_tc_plan_override", "oc_tc_plan_describe",
 )
 
 
@@ -73,7 +73,8 @@ _lib.oc_destroy.argtypes = [_vp]
 _lib.oc_device_status.argtypes = [_vp, _vp]
 _lib.oc_selftest_bounded_wait.argtypes = [_vp, C.c_uint, _vp]
 _lib.oc_profile_enable.argtypes = [_vp, _i]
-_lib.oc_tc_plan_override.argtypes = [_vp, _i, _i, _i, _i, _i]
+_lib.oc_tc_plan_override.argtypes = [_vp, _i, _i, _i, _i, _i, _i]
+_lib.oc_tc_plan_describe.argtypes = [_vp, _vp, _vp]
 _lib.oc_profile_reset.argtypes = [_vp]
 _lib.oc_profile_read.argtypes = [_vp, _i, _vp, _vp]
 _lib.oc_profile_span_read.argtypes = [_vp, _i, _vp, _vp]
@@ -287,14 +288,27 @@ class Context:
         """Makes a bounded device-side wait run out on purpose (see oc_selftest_bounded_wait)."""
         _chk(_lib.oc_selftest_bounded_wait(self._h, limit_us, _stream(stream)), "oc_selftest_bounded_wait")
 
-    def tc_plan_override(self, plan=None, single_accumulator: bool = False) -> None:
-        """Test hook (oc_tc_plan_override): ``plan`` = (pair, tiles per CTA, pieces per row) forces the
-        tensor-core matcher's work split; None returns to the planner."""
+    def tc_plan_override(self, plan=None, single_accumulator: bool = False, candidates_resident: int = -1) -> None:
+        """Test hook (oc_tc_plan_override): ``plan`` = (pair, tiles per CTA, pieces per row[, candidates
+        resident]) forces the tensor-core matcher's work split; None returns to the planner."""
         if plan is None:
-            _chk(_lib.oc_tc_plan_override(self._h, 0, 0, 1, 1, 0), "oc_tc_plan_override")
+            _chk(_lib.oc_tc_plan_override(self._h, 0, 0, 1, 1, 0, -1), "oc_tc_plan_override")
         else:
-            pair, tiles, pieces = (int(v) for v in plan)
-            _chk(_lib.oc_tc_plan_override(self._h, 1, pair, tiles, pieces, int(single_accumulator)), "oc_tc_plan_override")
+            vals = [int(v) for v in plan]
+            if len(vals) == 4:
+                candidates_resident = vals[3]
+            pair, tiles, pieces = vals[:3]
+            _chk(_lib.oc_tc_plan_override(self._h, 1, pair, tiles, pieces, int(single_accumulator), int(candidates_resident)),
+                 "oc_tc_plan_override")
+
+    def tc_plan_describe(self, layout: Layout) -> dict:
+        """Test hook (oc_tc_plan_describe): the tensor-core matcher's work split for this layout."""
+        cl = layout.c()
+        out = (C.c_int32 * 12)()
+        _chk(_lib.oc_tc_plan_describe(self._h, C.byref(cl), out), "oc_tc_plan_describe")
+        keys = ("pair", "tiles", "pieces_per_row", "two_acc_sets", "stages", "stage_bytes", "a_resident", "pieces",
+                "walkers", "widest_cols", "kblocks")
+        return dict(zip(keys, list(out)))
 
     def profile_enable(self, on) -> None:
         """False/0: timers off; True/1: CUDA events around every launch; 2: device-side spans of the

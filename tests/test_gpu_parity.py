@@ -212,7 +212,7 @@ def test_token_chain_random_layouts(oc, oracle, shape, groups, lattice):
     assert_matcher(rep, inputs.BF16, shape, lattice)
 
 
-@pytest.mark.parametrize("plan", ["0,1,2", "0,2,3", "1,1,1", "1,2,2"])
+@pytest.mark.parametrize("plan", ["0,1,2", "0,2,3", "1,1,1", "1,2,2", "0,2,3,1", "1,1,2,1", "0,1,4,1"])
 @pytest.mark.parametrize("shape,groups,lattice", _random_token_layouts(8, seed=7))
 def test_token_match_random_layouts_forced_plans(oc, oracle, shape, groups, lattice, plan):
     B, T, Hh, W, C = shape
@@ -234,7 +234,10 @@ def test_token_match_random_layouts_forced_plans(oc, oracle, shape, groups, latt
     ((1, 3, 40, 56, 136), (1, 1)),       # ragged 20 x 28 lattice, K tail, three frames
     ((1, 1, 64, 64, 128), (2, 2)),       # four patches per frame
 ])
-@pytest.mark.parametrize("plan", ["0,1,1", "0,1,3", "0,2,2", "0,2,5", "1,1,1", "1,1,2", "1,2,1", "1,2,4", "0,2,64", "1,1,64"])
+@pytest.mark.parametrize("plan", ["0,1,1", "0,1,3", "0,2,2", "0,2,5", "1,1,1", "1,1,2", "1,2,1", "1,2,4", "0,2,64", "1,1,64",
+                                  # the same with the candidate tiles resident in shared memory for a whole row
+                                  "0,1,3,1", "0,2,2,1", "0,2,5,1", "1,1,2,1", "1,2,4,1", "0,1,7,1", "1,2,2,1",
+                                  "0,2,5,0", "1,1,2,0"])
 def test_tensor_core_matcher_every_plan(oc, oracle, shape, groups, plan):
     """The planner's choice (single CTA or CTA pair, one or two candidate tiles per CTA, pieces per
     row) changes the work split only: every valid plan must reproduce the oracle.  A plan the shape
@@ -488,7 +491,7 @@ def test_joint_token_cache_on_given_frame_tables(oc, oracle, shape, lattice, mod
     assert reused > 0
 
 
-@pytest.mark.parametrize("plan", [None, "0,1,1", "0,2,2", "1,1,1", "1,2,2", "0,2,3"])
+@pytest.mark.parametrize("plan", [None, "0,1,1", "0,2,2", "1,1,1", "1,2,2", "0,2,3", "0,2,3,1", "0,1,2,1", "1,2,2,1", "1,1,3,1"])
 def test_joint_token_cache_svd_level_shapes_every_plan(oc, oracle, plan):
     """Several candidate tiles per lattice member, every form of the tensor-core matcher (single CTA / CTA
     pair, one or two tiles, several pieces per row) on the joint work list."""
