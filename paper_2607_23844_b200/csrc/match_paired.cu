@@ -562,6 +562,91 @@ block_partial_reg_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int
     }
 }
 
+// Fused variant of the two kernels around it, for clips whose T frames fit the thread-groups of one CTA
+// (T <= threads / LPR): a thread-group still handles one (cell, t) with every load issued up front, but
+// all T groups of a cell sit in the same CTA, leave their partial sums in shared memory, and the cell's
+// candidates are finished right there -- the T partials never travel through global memory and the
+// finalize launch disappears (what matters on small tensors, where a launch costs more than the work).
+// The sums over t are taken in the same order as block_finalize_kernel takes them: same bits.
+template <int DT, int LPR, int CPL, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+block_fused_kernel(const uint8_t* __restrict__ x, int T, int H, int W, int cpr, int sy, int sx, int oy, int ox,
+                   int cells_per_cta, float eps, float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
+    pdl_enter();
+    constexpr int NC = 3, REC = 1 + 2 * NC, GROUPS = THREADS / LPR;
+    __shared__ float rec[GROUPS][REC];
+    const int b = blockIdx.y;
+    const int cells_x = W / sx, cells = (H / sy) * cells_x;
+    const int grp = threadIdx.x / LPR, lane = threadIdx.x % LPR;
+    const int lc = grp / T, t = grp - lc * T;                       // local cell, frame
+    const int cell_raw = blockIdx.x * cells_per_cta + lc;
+    const bool valid = lc < cells_per_cta && cell_raw < cells;      // idle groups redo cell 0 and publish nothing
+    const int cell = valid ? cell_raw : 0;
+    const int cy = cell / cells_x, cx = cell - cy * cells_x;
+    const long long row_bytes = (long long)cpr * 16;
+    const uint8_t* frame = x + ((long long)b * T + (valid ? t : 0)) * H * W * row_bytes;
+    const uint8_t* rep = frame + ((long long)(cy * sy + oy) * W + (cx * sx + ox)) * row_bytes;
+    const int nc = sy * sx - 1, rep_m = oy * sx + ox;
+    const uint8_t* cand[NC];
+#pragma unroll
+    for (int k = 0; k < NC; ++k) {
+        const int m = k + (k >= rep_m ? 1 : 0);
+        const int my = m / sx, mx = m - my * sx;
+        cand[k] = k < nc ? frame + ((long long)(cy * sy + my) * W + (cx * sx + mx)) * row_bytes : rep;
+    }
+    uint4 r[CPL], a[NC][CPL];
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) {
+        const int c = lane + j * LPR;
+        if (c < cpr) {
+            r[j] = ld_nc_v4(rep + (long long)c * 16);
+#pragma unroll
+            for (int k = 0; k < NC; ++k)
+                if (k < nc) a[k][j] = ld_nc_v4(cand[k] + (long long)c * 16);
+        }
+    }
+    float rn = 0.f, dot[NC] = {0.f, 0.f, 0.f}, na[NC] = {0.f, 0.f, 0.f};
+#pragma unroll
+    for (int j = 0; j < CPL; ++j) {
+        if (lane + j * LPR < cpr) {
+            Chunk<DT>::sq(r[j], rn);
+#pragma unroll
+            for (int k = 0; k < NC; ++k)
+                if (k < nc) Chunk<DT>::acc2(a[k][j], r[j], dot[k], na[k]);
+        }
+    }
+    rn = group_sum<LPR>(rn);
+    if (lane == 0) rec[grp][0] = rn;
+#pragma unroll
+    for (int k = 0; k < NC; ++k) {
+        const float d = group_sum<LPR>(dot[k]), n = group_sum<LPR>(na[k]);
+        if (lane == 0) { rec[grp][1 + 2 * k] = d; rec[grp][2 + 2 * k] = n; }
+    }
+    __syncthreads();
+    // one thread per (local cell, member of the neighbourhood): the representative's own entry, or a
+    // candidate's cosine from the T partials added in order of t
+    const int members = sy * sx;
+    for (int i = threadIdx.x; i < cells_per_cta * members; i += THREADS) {
+        const int c_l = i / members, m = i - c_l * members;
+        const int c_g = blockIdx.x * cells_per_cta + c_l;
+        if (c_g >= cells) continue;
+        const int gy = c_g / cells_x, gx = c_g - gy * cells_x;
+        const int my = m / sx, mx = m - my * sx;
+        const long long P = (long long)H * W;
+        const long long pos = (long long)b * P + (long long)(gy * sy + my) * W + (gx * sx + mx);
+        const long long rep_pos = (long long)b * P + (long long)(gy * sy + oy) * W + (gx * sx + ox);
+        if (m == rep_m) { best_sim[pos] = -INFINITY; best_idx[pos] = (int32_t)pos; continue; }
+        const int k = m > rep_m ? m - 1 : m;
+        float s_rn = 0.f, s_dot = 0.f, s_na = 0.f;
+        for (int tt = 0; tt < T; ++tt) {
+            const float* q = rec[c_l * T + tt];
+            s_rn += q[0]; s_dot += q[1 + 2 * k]; s_na += q[2 + 2 * k];
+        }
+        best_sim[pos] = clamp_unit(s_dot / (fmaxf(sqrtf(s_na), eps) * fmaxf(sqrtf(s_rn), eps)));
+        best_idx[pos] = (int32_t)rep_pos;
+    }
+}
+
 __global__ void __launch_bounds__(PAIR_THREADS)
 block_finalize_kernel(const float* __restrict__ partial, int B, int T, int H, int W, int sy, int sx, int oy, int ox,
                       int rec, float eps, float* __restrict__ best_sim, int32_t* __restrict__ best_idx) {
@@ -619,6 +704,24 @@ oc_status launch_match_block(oc_ctx* ctx, const Geo& g, const void* x, float* be
     while (lr < 32 && lr * 5 < cpr) lr <<= 1;
     const bool reg_variant = g.sy * g.sx - 1 <= 3 && cpr <= 5 * lr;
     const int lpr = reg_variant ? lr : lanes_per_row(cpr);
+    // one launch instead of two when a cell's T frames fit one CTA's thread-groups and the whole grid is
+    // small enough that the second launch would cost more than it saves (large tensors keep the two-kernel
+    // form: its first kernel has no CTA-wide barrier and more CTAs in flight)
+    const int fused_threads = g.T * lpr <= PAIR_THREADS ? PAIR_THREADS : 512;
+    const bool fused = reg_variant && g.T * lpr <= 512 && (long long)cells * g.B * g.T * lpr <= 512ll * 4 * ctx->sm_count;
+    if (fused) {
+        const int groups = fused_threads / lpr, cells_per_cta = groups / g.T;
+        dim3 grid((unsigned)((cells + cells_per_cta - 1) / cells_per_cta), (unsigned)g.B);
+        LaunchScope scope(ctx, OC_K_BLOCK, s);
+        const uint8_t* xb = (const uint8_t*)x;
+#define OC_BLKF(DTV, L, TH) OC_LAUNCH((block_fused_kernel<DTV, L, 5, TH>), grid, TH, 0, s, xb, g.T, g.H, g.W, cpr, g.sy, g.sx, g.oy, g.ox, cells_per_cta, g.eps, best_sim, best_idx)
+#define OC_BLKF_L(DTV, TH) switch (lpr) { case 4: OC_BLKF(DTV, 4, TH); break; case 8: OC_BLKF(DTV, 8, TH); break; case 16: OC_BLKF(DTV, 16, TH); break; default: OC_BLKF(DTV, 32, TH); break; }
+        if (g.dtype == OC_DTYPE_BF16) { if (fused_threads == 256) { OC_BLKF_L(OC_DTYPE_BF16, 256) } else { OC_BLKF_L(OC_DTYPE_BF16, 512) } }
+        else { if (fused_threads == 256) { OC_BLKF_L(OC_DTYPE_F32, 256) } else { OC_BLKF_L(OC_DTYPE_F32, 512) } }
+#undef OC_BLKF_L
+#undef OC_BLKF
+        return last_launch_status();
+    }
     {
         const int groups = PAIR_THREADS / lpr;
         dim3 grid((unsigned)((cells + groups - 1) / groups), (unsigned)(g.B * g.T));

@@ -42,7 +42,8 @@
 // TMA coordinate for the two operands -- and nothing else changes.
 //
 // Warp specialised:
-//   warp 0      TMA producer   (one lane per box; a CTA's candidate tiles are one box, and so are its
+//   warp 0 (and, for one-tile plans, the last warp, taking turns with it stage by stage)
+//               TMA producer   (one lane per box; a CTA's candidate tiles are one box, and so are its
 //               quanta of a piece, whenever they stack into a rectangle of lattice rows): global ->
 //               smem ring (as many stages as fit in 224 KB), mbarrier complete_tx
 //   warp 1      MMA issuer     (all lanes walk the loop so that addresses stay warp-uniform, one
@@ -85,7 +86,12 @@ static constexpr int SMEM_LIMIT = 232448;         // 227 KB: the most dynamic sh
 #endif
 static constexpr int EPI_WARPS = OC_EPI_WARPS;            // 8 or 16: two or four per TMEM lane quarter
 static constexpr int EPI_PARTS = EPI_WARPS / 4;           // a piece's columns are cut into this many parts
-static constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;    // producer warp, MMA warp, the epilogue warps
+#ifndef OC_PRODUCERS
+#define OC_PRODUCERS 2
+#endif
+static constexpr int N_PRODUCERS = OC_PRODUCERS;          // copy-producer warps: warp 0 and, with two, the last warp
+static constexpr int PRODUCER2_WARP = 2 + EPI_WARPS;
+static constexpr int TC_THREADS = 64 + 32 * EPI_WARPS + 32 * (N_PRODUCERS - 1);   // producer, MMA, epilogue warps[, producer]
 static constexpr int MAX_LATTICES = 9;
 static constexpr uint32_t TMEM_COLS = 512;
 
@@ -114,6 +120,7 @@ struct TcScalars {
     int sx_magic;                        // ceil(65536 / sx): (m * sx_magic) >> 16 == m / sx for m < 256
     int u_step_q, u_step_r;              // n_q_units / pieces_per_row and the remainder
     int n_stages, stage_bytes;           // operand ring of this launch
+    int n_prod;                          // copy-producer warps at work: 1, or 2 taking turns stage by stage
     int a_res, a_region_bytes;           // candidate tiles resident: all 64-channel steps of a CTA's candidate tiles
                                          // sit in front of the ring (one slot per step) for all pieces of a row, and
                                          // the ring carries representatives only
@@ -279,6 +286,13 @@ __device__ unsigned long long g_tc_stage[8][512];
 #define OC_TR(role, piece, k, who)
 #define OC_TS(k, n, who)
 #endif
+#ifdef OC_TC_TRACE
+#define OC_ACC_BEGIN(v) const unsigned long long v##_t0 = clock64()
+#define OC_ACC_END(v) v += clock64() - v##_t0
+#else
+#define OC_ACC_BEGIN(v)
+#define OC_ACC_END(v)
+#endif
 
 static constexpr int COL_BYTES = 256 * 8;                               // {scale, bias} per column of a piece
 static constexpr int N_BARS = 2 * MAX_STAGES + 5 + MAX_AKB;             // full[], empty[], acc_full[2], acc_empty[2], drain, a_empty[]
@@ -381,8 +395,16 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     const int my_rep = P.my_rep, mx_rep = P.mx_rep;
     const uint32_t tmem_base = early_producer ? 0u : *tmem_slot;    // (the producer warp never touches TMEM)
 
-    if (warp == 0) {
+    if (warp == PRODUCER2_WARP && P.n_prod < 2) {
+        // (the second producer warp sits this launch out)
+    } else if (warp == 0 || warp == PRODUCER2_WARP) {
         // ================================ TMA producer ==========================================
+        // Two producer warps take turns, stage by stage (the producer's own work per stage -- a look at a
+        // barrier, one or two copy instructions, an arrival, all of them slow to issue beside the epilogue
+        // warps -- is longer than the MMAs of a short stage; two of them halve it).  Each walks all pieces
+        // and all stages, and acts on every other stage.
+        const uint32_t my_turn = warp == 0 ? 0u : 1u;
+        uint32_t gstage = 0;                          // stages handed out so far, over all pieces
         // Every stage costs the issuing thread one look at the stage's "empty" barrier, its copies and one
         // arrive on the "full" barrier.  When a CTA's candidate tiles are one box and its quanta of a piece
         // are one box (the usual case: see a_merged / q_merged) lane 0 does all of that by itself, with no
@@ -395,6 +417,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         bool joined = !early_producer;                // whether this warp has met the set-up barrier yet
         const uint32_t ring_base = tiles_base + (uint32_t)P.a_region_bytes;       // (a_region_bytes is 0 unless a_res)
         const bool solo = P.a_merged && P.q_merged;
+#ifdef OC_TC_TRACE
+        unsigned long long acc_pw = 0, acc_pt = 0, acc_pe = 0, acc_pp = 0; const unsigned long long acc_p0 = clock64();
+#endif
         const uint32_t a_step = P.a_res ? (uint32_t)(P.tpp * A_BYTES) : 0u;     // resident slot pitch
         const uint32_t q_off = (uint32_t)(P.a_res ? 0 : P.tpp * A_BYTES);       // quanta inside a ring stage
         int trp = -1;
@@ -408,6 +433,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             // what the leader's barrier expects per stage: the copies of both CTAs
             const uint32_t bytes = (uint32_t)((PAIR ? 2 : 1) * ((load_a ? P.tpp * A_BYTES : 0) + nq_mine * Q_BYTES));
             if (solo) {
+                OC_ACC_BEGIN(acc_pp);
                 // (tiles past the lattice are fetched as zeros and masked in the epilogue)
                 const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp;
                 const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
@@ -417,21 +443,28 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 const int wQ = c.px * P.Ws + wq * bwQ, hQ = c.py * P.Hs + hq * P.bhQ;
                 const CUtensorMap* mapA = &KP.mapsA[c.member];
                 const CUtensorMap* mapQ = &KP.mapQ[nq_mine != P.q_lo ? 1 : 0];
-                for (int kb = 0; kb < P.kblocks; ++kb) {
-                    if (lane == 0 && ok) {
+                OC_ACC_END(acc_pp);
+                for (int kb = 0; kb < P.kblocks; ++kb, ++gstage) {
+                    if (lane == 0 && ok && (P.n_prod < 2 || (gstage & 1u) == my_turn)) {
                         const uint32_t full_local = bar_full + 8 * stage;
                         const uint32_t full = PAIR ? map_to_cta(full_local, 0) : full_local;
+                        OC_ACC_BEGIN(acc_pw);
                         bool go = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
+                        OC_ACC_END(acc_pw);
                         // the slot of this step is free once the MMAs of the previous row's last piece have read it
                         if (go && P.a_res && load_a) go = mbar_wait(bar_a_empty + 8 * kb, a_phase ^ 1u, abort_flag);
                         if (go) {
                             // the copies first, the arrival that carries their byte count after them: the barrier
                             // cannot complete before that arrival, and the copies are on their way sooner
+                            OC_ACC_BEGIN(acc_pt);
                             tma_load_4d<PAIR>(ring_base + stage * STAGE_BYTES + q_off, mapQ, kb * BK, wQ, hQ, c.bt, full);
                             if (load_a)
                                 tma_load_4d<PAIR>(P.a_res ? tiles_base + (uint32_t)kb * a_step : ring_base + stage * STAGE_BYTES,
                                                   mapA, kb * BK, wA, hA, c.bt_a, full);
+                            OC_ACC_END(acc_pt);
+                            OC_ACC_BEGIN(acc_pe);
                             if (leader) mbar_arrive_expect_tx(full_local, bytes);
+                            OC_ACC_END(acc_pe);
                         } else {
                             ok = false;
                         }
@@ -462,7 +495,11 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     dst_off = q_off + (uint32_t)((lane - nA) * Q_BYTES);
                 }
                 const bool active = lane < nA ? load_a : lane < nA + nQ;
-                for (int kb = 0; kb < P.kblocks; ++kb) {
+                for (int kb = 0; kb < P.kblocks; ++kb, ++gstage) {
+                    if (P.n_prod > 1 && (gstage & 1u) != my_turn) {             // the other producer's stage
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     const uint32_t full_local = bar_full + 8 * stage;
                     const uint32_t full = PAIR ? map_to_cta(full_local, 0) : full_local;
                     bool go = true;
@@ -488,6 +525,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             if (P.a_res && load_a) a_phase ^= 1u;
         }
         if (!joined) { __syncthreads(); joined = true; }
+#ifdef OC_TC_TRACE
+        if (blockIdx.x == OC_TC_TRACE && lane == 0 && warp == 0) { g_tc_stage[0][0] = acc_pw; g_tc_stage[0][1] = clock64() - acc_p0; g_tc_stage[0][2] = trp + 1; g_tc_stage[0][3] = acc_pt; g_tc_stage[0][4] = acc_pe; g_tc_stage[0][5] = acc_pp; }
+#endif
         if (!ok && lane == 0) {
             atomicCAS(P.status, 0, OC_ERR_TIMEOUT);
             *abort_flag = 1;
@@ -514,13 +554,18 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             int stage = 0; uint32_t phase = 0;
             bool ok = true, peeked = false;
             uint32_t it = 0;
+#ifdef OC_TC_TRACE
+            unsigned long long acc_mf = 0, acc_ma = 0, acc_mi = 0; const unsigned long long acc_m0 = clock64();
+#endif
             while (ok && walk.next(P, c)) {
                 // one candidate tile per CTA leaves half of TMEM free: two accumulators take turns, and the
                 // epilogue of a piece runs under the MMAs of the next one
                 const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
                 ++it;
                 OC_TR(1, (int)it - 1, 0, lane == 0);
+                OC_ACC_BEGIN(acc_ma);
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_empty + 8 * buf, acc_phase ^ 1u, abort_flag))) { ok = false; break; }
+                OC_ACC_END(acc_ma);
                 OC_TR(1, (int)it - 1, 1, lane == 0);
                 const uint32_t d_tmem = tmem_base + buf * 256u;
                 tc_fence_after();
@@ -531,8 +576,11 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 for (int kb = 0; kb < P.kblocks; ++kb) {
                     // (each lane looked for itself; the barrier's phase cannot go back, so a lane that saw it
                     //  full stays right, and the others wait here)
+                    OC_ACC_BEGIN(acc_mf);
                     if (!peeked && !mbar_wait(bar_full + 8 * stage, phase, abort_flag)) ok = false;
                     if (!__all_sync(0xFFFFFFFFu, ok)) { ok = false; break; }
+                    OC_ACC_END(acc_mf);
+                    OC_ACC_BEGIN(acc_mi);
                     if (kb == 0) OC_TR(1, (int)it - 1, 2, lane == 0);
                     const uint32_t s_addr = tiles_base + (uint32_t)P.a_region_bytes + stage * STAGE_BYTES;
                     const uint32_t a_addr = P.a_res ? tiles_base + (uint32_t)(kb * P.tpp * A_BYTES) : s_addr;
@@ -549,6 +597,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     // frees the stage (in both CTAs of a pair) when the MMAs retire
                     tc_commit<PAIR>(PAIR ? map_to_cta(bar_empty + 8 * stage, 0) : bar_empty + 8 * stage, issue);
                     if (PAIR) tc_commit<PAIR>(map_to_cta(bar_empty + 8 * stage, 1), issue);
+                    OC_ACC_END(acc_mi);
                     if (P.a_res && c.last) {         // the row's candidate tiles of this step have been read for the last time
                         tc_commit<PAIR>(PAIR ? map_to_cta(bar_a_empty + 8 * kb, 0) : bar_a_empty + 8 * kb, issue);
                         if (PAIR) tc_commit<PAIR>(map_to_cta(bar_a_empty + 8 * kb, 1), issue);
@@ -561,6 +610,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     if (PAIR) tc_commit<PAIR>(map_to_cta(bar_acc_full + 8 * buf, 1), issue);
                 }
             }
+#ifdef OC_TC_TRACE
+            if (blockIdx.x == OC_TC_TRACE && lane == 0) { g_tc_stage[1][0] = acc_mf; g_tc_stage[1][1] = acc_ma; g_tc_stage[1][2] = acc_mi; g_tc_stage[1][3] = clock64() - acc_m0; g_tc_stage[1][4] = it; }
+#endif
             if (!ok && lane == 0) { atomicCAS(P.status, 0, OC_ERR_TIMEOUT); *abort_flag = 1; }
             // all MMAs issued by this warp must retire before TMEM is released
             tc_commit<PAIR>(PAIR ? map_to_cta(bar_drain, 0) : bar_drain, issue);
@@ -1103,6 +1155,9 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     P.a_merged = p.a_merged; P.q_merged = p.q_merged; P.q_lo = p.q_lo;
     P.n_stages = p.n_stages; P.stage_bytes = p.stage_bytes;
     P.a_res = p.a_res; P.a_region_bytes = p.a_region_bytes;
+    // two producers pay where a stage is short (one candidate tile per CTA); with two tiles the MMAs of a
+    // stage cover one producer's work and the second warp only competes for issue slots
+    P.n_prod = (N_PRODUCERS > 1 && p.tpp == 1) ? 2 : 1;
     P.units_per_group = (int)g.units_per_group; P.reps_per_group = (int)g.reps_per_group;
     P.inv_norm = inv_norm; P.keys = keys; P.aux = aux_sim; P.status = ctx->d_status;
     if (ctx->span_on) {
