@@ -225,8 +225,8 @@ oc_status oc_profile_captured_read(oc_ctx* ctx, int kernel_id, int64_t* launches
  *   x         [B][T][H][W][C] features of layout->dtype (the wrapped layer's input)
  *   best_sim  [n_units] float: cosine of the best match; -inf for representatives
  *   best_idx  [n_units] int32: global unit index of that representative (ties: lowest index; the
- *             tensor-core matcher compares similarities truncated to 19 mantissa bits, so values
- *             that agree to 2^-18 relative count as tied);
+ *             tensor-core matcher compares cosines truncated by up to 8e-6, so values that agree to
+ *             that precision count as tied);
  *             a representative's own index for representatives
  *   aux_sim   nullable.  TOKEN: [n_groups][units_per_group][reps_per_group] float, every candidate
  *             row's full similarity row (rows of representatives and the self-match diagonal are

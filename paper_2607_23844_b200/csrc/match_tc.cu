@@ -54,11 +54,13 @@
 //               tiles for the first / second half of the piece's columns: tcgen05.ld 32 columns at a
 //               time (double buffered), scale by the representative's inverse norm, and a running
 //               maximum over keys that carry the column in their 5 low mantissa bits (one three-input
-//               max per two columns, no compare-and-select per element, no cross-thread reduction);
+//               max per three keys, no compare-and-select per element, no cross-thread reduction; the
+//               values are lifted to be non-negative first, so that the lowest column wins among equal
+//               similarities whatever their sign);
 //               then ONE 64-bit atomicMax per row merges the piece into the packed key array (largest
 //               value, then lowest index: independent of arrival order, hence deterministic).
-//               The reported similarity is thereby truncated by at most 2^-18 relative, and among
-//               representatives whose similarities agree to that precision the lowest index wins.
+//               The reported cosine is thereby truncated by at most 8e-6, and among representatives
+//               whose similarities agree to that precision the lowest index wins.
 // Rows / columns of a box that fall outside the patch are masked in the epilogue (a NaN scale never
 // wins a max), so ragged lattices need no padding.  Every mbarrier wait is bounded: on expiry the CTA
 // records OC_ERR_TIMEOUT in the context's status word, lets its outstanding copies land, frees TMEM
@@ -266,13 +268,6 @@ __device__ __forceinline__ float key_tree_max(const float (&k)[32]) {
     const float b0 = max3f(a[0], a[1], a[2]), b1 = max3f(a[3], a[4], a[5]), b2 = max3f(a[6], a[7], a[8]);
     const float c0 = max3f(b0, b1, b2);
     return max3f(c0, a[9], a[10]);
-}
-
-// Arg-max key of the epilogue's second look at a row (see there): the value with its 5 low mantissa bits
-// replaced by the column, stored so that the LOWEST column is the largest key whatever the sign.
-__device__ __forceinline__ float oc_key_any(float x, int j) {
-    const uint32_t b = __float_as_uint(x);
-    return __uint_as_float((b & 0xFFFFFFE0u) | (uint32_t)((b >> 31) ? j : 31 - j));
 }
 
 #ifdef OC_TC_TRACE
@@ -677,6 +672,14 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 const int yA = (c.py * P.Hs + hsA) * P.sy + my, xA = (c.px * P.Ws + wsA) * P.sx + mx;
                 tokA1 = ((long long)c.bt_a * P.H + yA) * P.W + xA;
             }
+            // The keys below want non-negative values (among negative floats the larger mantissa is the
+            // SMALLER value, which would turn the tie rule round): every scaled similarity of a row is
+            // lifted by a little more than the row's own norm -- |<a, b>| / |b| <= |a| -- inside the same
+            // FMA that applies the scale, and the lift is taken off the one value that is reported.
+            float lift0 = 0.f, lift1 = 0.f;
+            // (its own low bits cleared, so that a similarity of exactly zero is reported as exactly zero)
+            if (row_ok0) lift0 = __uint_as_float(__float_as_uint(1.001f / __ldg(P.inv_norm + tokA0)) & 0xFFFFFFE0u);
+            if (row_ok1) lift1 = __uint_as_float(__float_as_uint(1.001f / __ldg(P.inv_norm + tokA1)) & 0xFFFFFFE0u);
             // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
             const int n_ch = (c.ncol + 31) >> 5;                        // (a last half chunk reads 16 columns of
             const int ch_begin = (part * n_ch + EPI_PARTS - 1) / EPI_PARTS;      //  nothing: their table entries are NaN)
@@ -702,22 +705,23 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                         aux_row = P.aux + ((long long)c.g * P.units_per_group + u_local) * P.reps_per_group;
                     }
                     // Running maximum over "keys": the scaled similarity with its 5 low mantissa bits
-                    // replaced by 31 - (column within the chunk), so that ONE three-input max per two
-                    // columns carries the arg max along (among equal similarities the lowest column has
-                    // the largest key).  The similarity loses 5 of its 24 mantissa bits (2^-18 relative),
-                    // far inside the tolerance of a bf16 match.  The 32 keys of a chunk are reduced by a tree
+                    // replaced by 31 - (column within the chunk), so that ONE three-input max per three
+                    // keys carries the arg max along (among equal similarities the lowest column has the
+                    // largest key).  The lifted similarity loses 5 of its 24 mantissa bits (2^-18 of at most
+                    // twice the row's norm: 8e-6 in units of the cosine), far inside the tolerance of a bf16
+                    // match.  The 32 keys of a chunk are reduced by a tree
                     // of depth 4 (a running maximum would be a chain of 16 dependent instructions, and with two
                     // epilogue warps per scheduler nothing else hides that latency); bc = the chunk in which the
                     // row's maximum last rose.
                     float bm = -INFINITY;
                     int bc = -1;
+                    const float row_lift = t ? lift1 : lift0;
                     const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)t * tile_stride + buf * 256u;
                     // two register buffers: the TMEM load of the next step is in flight while this one is reduced
                     uint32_t va[32], vb[32];
-#define OC_KEY(v, s, j) __uint_as_float((__float_as_uint(__uint_as_float(v) * (s)) & 0xFFFFFFE0u) | (uint32_t)(31 - (j)))
-#define OC_KEY_ANY(v, s, j) oc_key_any(__uint_as_float(v) * (s), (j))
+#define OC_KEY(v, s, j) __uint_as_float((__float_as_uint(fmaf(__uint_as_float(v), (s), row_lift)) & 0xFFFFFFE0u) | (uint32_t)(31 - (j)))
 #define OC_VAL(k) __uint_as_float(__float_as_uint(k) & 0xFFFFFFE0u)
-#define OC_COL(k) ((__float_as_uint(k) >> 31) ? (int)(__float_as_uint(k) & 31u) : 31 - (int)(__float_as_uint(k) & 31u))
+#define OC_COL(k) (31 - (int)(__float_as_uint(k) & 31u))
 #define OC_REDUCE_CHUNK(v, ch)                                                                                   \
     do {                                                                                                         \
         float kf[32];                                                                                            \
@@ -759,32 +763,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                         }
                     }
 #undef OC_REDUCE_CHUNK
-                    // A chain whose maximum is negative has seen negative similarities only, and among negative
-                    // floats the larger mantissa is the SMALLER value: the keys above then prefer the highest
-                    // column among equal similarities.  Such a row is taken again from TMEM (the accumulators are
-                    // still there) with keys that store the column itself under a negative value.  Rare -- all
-                    // of a row's cosines negative -- and warp-uniform, because the TMEM loads are collective.
-                    if (__any_sync(0xFFFFFFFFu, bc >= 0 && bm < 0.f)) {
-                        bm = -INFINITY; bc = -1;
-#pragma unroll 1
-                        for (int ch = ch_begin; ch < ch_end; ++ch) {
-                            tmem_ld32(t_row + (uint32_t)(ch * 32), va);
-                            tmem_ld_wait();
-                            float kf[32];
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                const float4 s4 = col_scale4[ch * 8 + (j >> 2)];
-                                kf[j] = OC_KEY_ANY(va[j], s4.x, j); kf[j + 1] = OC_KEY_ANY(va[j + 1], s4.y, j + 1);
-                                kf[j + 2] = OC_KEY_ANY(va[j + 2], s4.z, j + 2); kf[j + 3] = OC_KEY_ANY(va[j + 3], s4.w, j + 3);
-                            }
-                            const float cm = key_tree_max(kf);
-                            if (OC_VAL(cm) > OC_VAL(bm)) { bm = cm; bc = ch; }
-                        }
-                    }
 #undef OC_KEY
-#undef OC_KEY_ANY
                     const int n0 = bc < 0 ? -1 : bc * 32 + OC_COL(bm);
-                    const float best = OC_VAL(bm);
+                    const float best = OC_VAL(bm) - row_lift;      // (exact: both are multiples of the key's last kept bit or larger)
 #undef OC_VAL
 #undef OC_COL
                     if (row_ok && n0 >= 0) {
