@@ -225,7 +225,7 @@ oc_status oc_profile_captured_read(oc_ctx* ctx, int kernel_id, int64_t* launches
  *   x         [B][T][H][W][C] features of layout->dtype (the wrapped layer's input)
  *   best_sim  [n_units] float: cosine of the best match; -inf for representatives
  *   best_idx  [n_units] int32: global unit index of that representative (ties: lowest index; the
- *             tensor-core matcher compares cosines truncated by up to 8e-6, so values that agree to
+ *             tensor-core matcher compares cosines rounded to within 2.4e-7, so values that agree to
  *             that precision count as tied);
  *             a representative's own index for representatives
  *   aux_sim   nullable.  TOKEN: [n_groups][units_per_group][reps_per_group] float, every candidate

@@ -53,14 +53,15 @@
 //   warps 2..9  epilogue: thread r of warps 2..5 / 6..9 owns row r (= TMEM lane r) of the candidate
 //               tiles for the first / second half of the piece's columns: tcgen05.ld 32 columns at a
 //               time (double buffered), scale by the representative's inverse norm, and a running
-//               maximum over keys that carry the column in their 5 low mantissa bits (one three-input
-//               max per three keys, no compare-and-select per element, no cross-thread reduction; the
-//               values are lifted to be non-negative first, so that the lowest column wins among equal
-//               similarities whatever their sign);
+//               maximum over integer keys: the scaled similarity, lifted into one binade (where a
+//               float's bits are linear in its value), times 32, plus 31 - column (one three-input max
+//               per three keys, no compare-and-select per element, no cross-thread reduction; the
+//               lowest column wins among equal similarities whatever their sign);
 //               then ONE 64-bit atomicMax per row merges the piece into the packed key array (largest
 //               value, then lowest index: independent of arrival order, hence deterministic).
-//               The reported cosine is thereby truncated by at most 8e-6, and among representatives
-//               whose similarities agree to that precision the lowest index wins.
+//               The lift rounds the reported cosine by at most 2.4e-7, and among representatives
+//               whose similarities agree to that precision the lowest index wins.  The epilogue warps
+//               never wait for one another: each keeps the column scales of its own chunks.
 // Rows / columns of a box that fall outside the patch are masked in the epilogue (a NaN scale never
 // wins a max), so ragged lattices need no padding.  Every mbarrier wait is bounded: on expiry the CTA
 // records OC_ERR_TIMEOUT in the context's status word, lets its outstanding copies land, frees TMEM
@@ -123,6 +124,7 @@ struct TcScalars {
     int u_step_q, u_step_r;              // n_q_units / pieces_per_row and the remainder
     int n_stages, stage_bytes;           // operand ring of this launch
     int n_prod;                          // copy-producer warps at work: 1, or 2 taking turns stage by stage
+    unsigned key_mul;                    // 32, as a run-time value: keeps half of the key multiplies on the FMA pipe
     int a_res, a_region_bytes;           // candidate tiles resident: all 64-channel steps of a CTA's candidate tiles
                                          // sit in front of the ring (one slot per step) for all pieces of a row, and
                                          // the ring carries representatives only
@@ -258,16 +260,25 @@ struct Walk {
     }
 };
 
-// Maximum of 32 arg-max keys by a tree of three-input maxima: 16 instructions, four levels deep.  (NaN keys,
-// the masked columns, never win: max.f32 returns its non-NaN operand.)
-__device__ __forceinline__ float key_tree_max(const float (&k)[32]) {
-    float a[11];
+// Maximum of 32 arg-max keys by a tree of three-input maxima: 16 instructions, four levels deep.
+__device__ __forceinline__ uint32_t key_tree_max(const uint32_t (&k)[32]) {
+    uint32_t a[11];
 #pragma unroll
-    for (int i = 0; i < 10; ++i) a[i] = max3f(k[3 * i], k[3 * i + 1], k[3 * i + 2]);
-    a[10] = fmaxf(k[30], k[31]);
-    const float b0 = max3f(a[0], a[1], a[2]), b1 = max3f(a[3], a[4], a[5]), b2 = max3f(a[6], a[7], a[8]);
-    const float c0 = max3f(b0, b1, b2);
-    return max3f(c0, a[9], a[10]);
+    for (int i = 0; i < 10; ++i) a[i] = __vimax3_u32(k[3 * i], k[3 * i + 1], k[3 * i + 2]);
+    a[10] = max(k[30], k[31]);
+    const uint32_t b0 = __vimax3_u32(a[0], a[1], a[2]), b1 = __vimax3_u32(a[3], a[4], a[5]), b2 = __vimax3_u32(a[6], a[7], a[8]);
+    const uint32_t c0 = __vimax3_u32(b0, b1, b2);
+    return __vimax3_u32(c0, a[9], a[10]);
+}
+
+// d = a * b + {c, c} on two packed fp32 lanes: one FMA-pipe instruction for two columns
+__device__ __forceinline__ void fma_pair(float& d0, float& d1, uint32_t a0, uint32_t a1, float b0, float b1, float c) {
+    unsigned long long a, b, cc, d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(a) : "r"(a0), "r"(a1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(b) : "f"(b0), "f"(b1));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(cc) : "f"(c));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(cc));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
 }
 
 #ifdef OC_TC_TRACE
@@ -289,9 +300,9 @@ __device__ unsigned long long g_tc_stage[8][512];
 #define OC_ACC_END(v)
 #endif
 
-static constexpr int COL_BYTES = 256 * 8;                               // {scale, bias} per column of a piece
+static constexpr int COL_BYTES = EPI_WARPS * 128 * 4;                   // per epilogue warp: the scales of its (at most 128) columns
 static constexpr int N_BARS = 2 * MAX_STAGES + 5 + MAX_AKB;             // full[], empty[], acc_full[2], acc_empty[2], drain, a_empty[]
-static constexpr int TAIL_BYTES = COL_BYTES + N_BARS * 8 + 32;        // column table, barriers, TMEM slot, flags
+static constexpr int TAIL_BYTES = COL_BYTES + N_BARS * 8 + 32 + EPI_WARPS * 16;   // column tables, barriers, TMEM slot, flags, masks
 static constexpr int TILE_BYTES = (SMEM_LIMIT - TAIL_BYTES) / 1024 * 1024;   // operand ring: everything else
 static constexpr int SMEM_TOTAL = TILE_BYTES + TAIL_BYTES;
 
@@ -317,6 +328,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     const uint32_t bar_a_empty = bar_drain + 8;                        // resident candidate slots, one per 64-channel step
     uint32_t* tmem_slot = (uint32_t*)(bars + N_BARS);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+    uint32_t* col_masked = tmem_slot + 8;                              // [warp][4]: per 32-column chunk, its columns that are no representative
     const uint32_t tiles_base = smem_u32(smem);
     const TcScalars& P = KP.s;
     if (P.span && threadIdx.x == 0) atomicMax(P.span, ~global_ns());
@@ -624,66 +636,127 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         uint32_t it = 0;
         const uint32_t acc_empty = PAIR ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;   // the leader's
         // Per column of a piece: the representative's inverse norm (NaN where the column is not a
-        // representative of this patch: a NaN product never wins a max).  Two tables take turns: the
-        // entries of the NEXT piece are fetched (one per thread) before this piece's accumulators are
-        // read and stored after, so their global-memory latency is never waited for.
-        float* col_scale = (float*)colsb;                              // [2][256]
+        // representative of this patch; each chunk of 32 columns also has a bit mask of those, and
+        // their keys are zeroed).  Every epilogue warp keeps a table of its OWN columns -- at most four
+        // chunks of 32 -- so the warps never wait for one another: a piece costs a warp its reduction
+        // and nothing else.  What the NEXT piece needs (the table entries, four per lane; each row's own
+        // norm) is fetched before this piece's accumulators are waited for and used after, so that
+        // global-memory latency is never waited for either.
+        const int ew = et >> 5;                                        // this warp among the epilogue warps
+        float* my_scale = (float*)colsb + ew * 128;
+        uint32_t* my_masked = col_masked + ew * 4;
+        const uint32_t key_mul = P.key_mul;
         const int rowh = row >> P.bwA_log2, roww = row & (bwA - 1);
-        auto table_entry = [&](const Piece& pc) -> float {
-            if (et >= pc.ncol) return __int_as_float(0x7FC00000);
-            const int gp = pc.c_off + et;
-            const int qi = pc.q0 + (gp >> 5), r = gp & 31;
-            const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
-            const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));
-            if (hs >= P.Hs || ws >= P.Ws) return __int_as_float(0x7FC00000);
-            const int y = (pc.py * P.Hs + hs) * P.sy + my_rep, x = (pc.px * P.Ws + ws) * P.sx + mx_rep;
-            return __ldg(P.inv_norm + ((long long)pc.bt * P.H + y) * P.W + x);
+        // What a warp needs of a piece, gathered ahead of time.  A lone warp runs dependent integer
+        // arithmetic at its full latency and pays for every branch, and this is on the one path that
+        // bounds the kernel, so: no branches (selects and a clamped address instead), one division per
+        // piece (the lane's four columns lie in four consecutive quanta), and the row part only when
+        // the row changes (the pieces of a row share their candidate tiles).
+        struct Cols {
+            int ch_begin, ch_end;            // this warp's chunks of 32 columns
+            float sc[4];                     // lane's table entries: column (ch_begin + i) * 32 + lane
+        };
+        struct Rows {
+            int tokA[2];                     // the rows (candidate tokens) this thread owns in the piece's tiles
+            bool row_ok[2];
+            float inv_a[2];                  // their inverse norms
+            float lift[2];
+            int my, mx;
+        };
+        // floor(a / d) for 0 <= a < 2^22 from the float reciprocal, without a branch
+        auto div_fast = [](int a, int d, float rcp_d) {
+            int q = (int)((float)a * rcp_d);
+            const int r = a - q * d;
+            q += (r >= d ? 1 : 0) - (r < 0 ? 1 : 0);
+            return q;
+        };
+        const float quiet_nan = __int_as_float(0x7FC00000);
+        const int tok_per_lattice_row = P.sy * P.W;
+        auto gather_cols = [&](const Piece& pc, Cols& a) {
+            // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
+            const int n_ch = (pc.ncol + 31) >> 5;                       // (a last half chunk reads 16 columns of
+            a.ch_begin = (part * n_ch + EPI_PARTS - 1) / EPI_PARTS;     //  nothing: their table entries are NaN)
+            a.ch_end = ((part + 1) * n_ch + EPI_PARTS - 1) / EPI_PARTS;
+            const int g0 = pc.c_off + lane;                             // the lane's column, counted from the piece's first quantum
+            const int r = g0 & 31, rh = r >> P.bwQ_log2, rw = r & (bwQ - 1);
+            const int qi = pc.q0 + (g0 >> 5) + a.ch_begin;
+            int hq = div_fast(qi, P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
+            // token of the patch's lattice point (0, 0) of the representatives' member
+            const int tok0 = (pc.bt * P.H + pc.py * P.Hs * P.sy + my_rep) * P.W + pc.px * P.Ws * P.sx + mx_rep;
+            const int col0 = a.ch_begin * 32 + lane;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int hs = hq * P.bhQ + rh, ws = wq * bwQ + rw;
+                const bool valid = (a.ch_begin + i < a.ch_end) & (col0 + 32 * i < pc.ncol) & (hs < P.Hs) & (ws < P.Ws);
+                const int tok = valid ? tok0 + hs * tok_per_lattice_row + ws * P.sx : 0;
+                const float v = __ldg(P.inv_norm + tok);
+                a.sc[i] = valid ? v : quiet_nan;
+                ++wq;
+                const bool wrap = wq == P.n_wq;
+                wq = wrap ? 0 : wq; hq += wrap ? 1 : 0;
+            }
+        };
+        auto gather_rows = [&](const Piece& pc, Rows& a) {
+            a.my = (pc.member * P.sx_magic) >> 16; a.mx = pc.member - a.my * P.sx;
+            const int tok0 = (pc.bt_a * P.H + pc.py * P.Hs * P.sy + a.my) * P.W + pc.px * P.Ws * P.sx + a.mx;
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int ta = (PAIR ? 2 : 1) * P.tpp * pc.a_pair + (int)rank * P.tpp + t;
+                const int htA = div_fast(ta, P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
+                const int hsA = htA * P.bhA + rowh, wsA = wtA * bwA + roww;
+                a.row_ok[t] = (t < P.tpp) & (hsA < P.Hs) & (wsA < P.Ws);
+                a.tokA[t] = a.row_ok[t] ? tok0 + hsA * tok_per_lattice_row + wsA * P.sx : 0;
+                a.inv_a[t] = __ldg(P.inv_norm + a.tokA[t]);
+            }
+        };
+        // The keys below want every scaled similarity of a row inside ONE binade, where the bits of a
+        // float are linear in its value: the FMA that applies the scale also adds a lift of 3 * 2^k,
+        // with 2^k the power of two at or above 1.001 x the row's own norm.  |<a, b>| / |b| <= |a|, so
+        // the lifted values lie in [2^(k+1), 2^(k+2)); the lift is taken off the one value reported.
+        auto set_lifts = [&](Rows& a) {
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const float bound = 1.001f / a.inv_a[t];
+                a.lift[t] = 3.0f * __uint_as_float((__float_as_uint(bound) + 0x007FFFFFu) & 0x7F800000u);
+            }
+        };
+        // the warp's table: written only when every lane is done with the one before
+        auto publish = [&](const Cols& a) {
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                my_scale[i * 32 + lane] = a.sc[i];
+                const uint32_t masked = __ballot_sync(0xFFFFFFFFu, a.sc[i] != a.sc[i]);
+                if (lane == 0) my_masked[i] = masked;
+            }
+            __syncwarp();
         };
         // Only from here on does this kernel touch what the norm pre-pass (the kernel before it in the
         // stream) writes: its operand copies and MMAs may run while that kernel still does.
         pdl_wait();
         if (et == 0) pdl_launch_dependents();
         Piece nx;
+        Cols cols, cols_ahead;
+        Rows cur, rows_ahead;
         bool have = walk.next(P, c);
-        if (have && et < 256) col_scale[et] = table_entry(c);
-        if (!epilogue_barrier_all<32 * EPI_WARPS>(ok)) { ok = false; have = false; }
+        if (have) { gather_cols(c, cols); gather_rows(c, cur); publish(cols); set_lifts(cur); }
         while (have) {
             const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
-            const float4* col_scale4 = (const float4*)(col_scale + (it & 1u) * 256);
-            const float* col_scale1 = col_scale + (it & 1u) * 256;
+            const float4* col_scale4 = (const float4*)my_scale;
+            const float* col_scale1 = my_scale;
+            OC_TR(3, (int)it, 0, et == 0);
             const bool have_nx = walk.next(P, nx);
-            float sc_nx = 0.f;
-            if (have_nx && et < 256) sc_nx = table_entry(nx);          // in flight until the end of this piece
-            const int my = (c.member * P.sx_magic) >> 16, mx = c.member - my * P.sx;
-            long long tokA0, tokA1; bool row_ok0, row_ok1;
-            {
-                const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp;
-                const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
-                const int hsA = htA * P.bhA + rowh, wsA = wtA * bwA + roww;
-                row_ok0 = hsA < P.Hs && wsA < P.Ws;
-                const int yA = (c.py * P.Hs + hsA) * P.sy + my, xA = (c.px * P.Ws + wsA) * P.sx + mx;
-                tokA0 = ((long long)c.bt_a * P.H + yA) * P.W + xA;
+            OC_TR(3, (int)it, 1, et == 0);
+            if (have_nx) {                                             // in flight until the end of this piece
+                gather_cols(nx, cols_ahead);
+                if (nx.first) gather_rows(nx, rows_ahead);
             }
-            {
-                const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + 1;
-                const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
-                const int hsA = htA * P.bhA + rowh, wsA = wtA * bwA + roww;
-                row_ok1 = P.tpp == 2 && hsA < P.Hs && wsA < P.Ws;
-                const int yA = (c.py * P.Hs + hsA) * P.sy + my, xA = (c.px * P.Ws + wsA) * P.sx + mx;
-                tokA1 = ((long long)c.bt_a * P.H + yA) * P.W + xA;
-            }
-            // The keys below want non-negative values (among negative floats the larger mantissa is the
-            // SMALLER value, which would turn the tie rule round): every scaled similarity of a row is
-            // lifted by a little more than the row's own norm -- |<a, b>| / |b| <= |a| -- inside the same
-            // FMA that applies the scale, and the lift is taken off the one value that is reported.
-            float lift0 = 0.f, lift1 = 0.f;
-            // (its own low bits cleared, so that a similarity of exactly zero is reported as exactly zero)
-            if (row_ok0) lift0 = __uint_as_float(__float_as_uint(1.001f / __ldg(P.inv_norm + tokA0)) & 0xFFFFFFE0u);
-            if (row_ok1) lift1 = __uint_as_float(__float_as_uint(1.001f / __ldg(P.inv_norm + tokA1)) & 0xFFFFFFE0u);
-            // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
-            const int n_ch = (c.ncol + 31) >> 5;                        // (a last half chunk reads 16 columns of
-            const int ch_begin = (part * n_ch + EPI_PARTS - 1) / EPI_PARTS;      //  nothing: their table entries are NaN)
-            const int ch_end = ((part + 1) * n_ch + EPI_PARTS - 1) / EPI_PARTS;
+            OC_TR(3, (int)it, 2, et == 0);
+            const int my = cur.my, mx = cur.mx;
+            const float lift0 = cur.lift[0], lift1 = cur.lift[1];
+            const int ch_begin = cols.ch_begin, ch_end = cols.ch_end;
+            OC_TR(3, (int)it, 3, et == 0);
+
             // warp-uniform outcome: the TMEM loads below are warp-collective
             OC_TR(2, (int)it, 0, et == 0);
             const bool ready = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * buf, acc_phase, abort_flag));
@@ -693,49 +766,60 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
 #pragma unroll 1
                 for (int t = 0; t < P.tpp; ++t) {                      // the piece's candidate tiles
                     if ((PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + t >= P.n_tilesA) continue;   // past the lattice
-                    const long long tokA = t ? tokA1 : tokA0;
-                    const bool row_ok = t ? row_ok1 : row_ok0;
+                    const int tokA = (t ? cur.tokA[1] : cur.tokA[0]);
+                    const bool row_ok = (t ? cur.row_ok[1] : cur.row_ok[0]);
                     float inv_a = 0.f;
                     float* aux_row = nullptr;
                     if (AUX && P.aux && row_ok) {
-                        inv_a = __ldg(P.inv_norm + tokA);
+                        inv_a = (t ? cur.inv_a[1] : cur.inv_a[0]);
                         const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + t;
                         const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
                         const int u_local = ((htA * P.bhA + rowh) * P.sy + my) * P.Wp + (wtA * bwA + roww) * P.sx + mx;
                         aux_row = P.aux + ((long long)c.g * P.units_per_group + u_local) * P.reps_per_group;
                     }
-                    // Running maximum over "keys": the scaled similarity with its 5 low mantissa bits
-                    // replaced by 31 - (column within the chunk), so that ONE three-input max per three
-                    // keys carries the arg max along (among equal similarities the lowest column has the
-                    // largest key).  The lifted similarity loses 5 of its 24 mantissa bits (2^-18 of at most
-                    // twice the row's norm: 8e-6 in units of the cosine), far inside the tolerance of a bf16
-                    // match.  The 32 keys of a chunk are reduced by a tree
-                    // of depth 4 (a running maximum would be a chain of 16 dependent instructions, and with two
-                    // epilogue warps per scheduler nothing else hides that latency); bc = the chunk in which the
-                    // row's maximum last rose.
-                    float bm = -INFINITY;
+                    // Running maximum over "keys".  A key is the lifted similarity's bit pattern times 32
+                    // plus 31 - (column within the chunk): the multiply drops the sign and the four high
+                    // exponent bits, which all lifted values of a row share, and keeps every mantissa bit, so
+                    // unsigned order of keys is order of similarity and then lowest column first, and ONE
+                    // three-input integer max per three keys carries the arg max along.  Nothing is lost
+                    // beyond the rounding of the FMA at the lift's magnitude (2^-23 of at most 4 x the row's
+                    // norm: 5e-7 in units of the cosine).  Per element that is half a packed FMA, one
+                    // multiply-add (every other one with a run-time factor, so that the compiler's shift-add
+                    // on the ALU pipe and the integer FMA pipe share them) and half a max.  The 32 keys of a
+                    // chunk are reduced by a tree of depth 4 (a running maximum would be a chain of 16
+                    // dependent instructions, and with two epilogue warps per scheduler nothing else hides
+                    // that latency); bc = the chunk in which the row's maximum last rose.
+                    uint32_t bm = 0;
                     int bc = -1;
                     const float row_lift = t ? lift1 : lift0;
                     const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)t * tile_stride + buf * 256u;
                     // two register buffers: the TMEM load of the next step is in flight while this one is reduced
                     uint32_t va[32], vb[32];
-#define OC_KEY(v, s, j) __uint_as_float((__float_as_uint(fmaf(__uint_as_float(v), (s), row_lift)) & 0xFFFFFFE0u) | (uint32_t)(31 - (j)))
-#define OC_VAL(k) __uint_as_float(__float_as_uint(k) & 0xFFFFFFE0u)
-#define OC_COL(k) (31 - (int)(__float_as_uint(k) & 31u))
 #define OC_REDUCE_CHUNK(v, ch)                                                                                   \
     do {                                                                                                         \
-        float kf[32];                                                                                            \
+        uint32_t kf[32];                                                                                         \
         _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
-            const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                                   \
-            kf[j] = OC_KEY(v[j], s4.x, j); kf[j + 1] = OC_KEY(v[j + 1], s4.y, j + 1);                            \
-            kf[j + 2] = OC_KEY(v[j + 2], s4.z, j + 2); kf[j + 3] = OC_KEY(v[j + 3], s4.w, j + 3);                \
+            const float4 s4 = col_scale4[((ch) - ch_begin) * 8 + (j >> 2)];                                      \
+            float x0, x1, x2, x3;                                                                                \
+            fma_pair(x0, x1, v[j], v[j + 1], s4.x, s4.y, row_lift);                                              \
+            fma_pair(x2, x3, v[j + 2], v[j + 3], s4.z, s4.w, row_lift);                                          \
+            kf[j] = __float_as_uint(x0) * 32u + (uint32_t)(31 - j);                                              \
+            kf[j + 1] = __float_as_uint(x1) * key_mul + (uint32_t)(30 - j);                                      \
+            kf[j + 2] = __float_as_uint(x2) * 32u + (uint32_t)(29 - j);                                          \
+            kf[j + 3] = __float_as_uint(x3) * key_mul + (uint32_t)(28 - j);                                      \
         }                                                                                                        \
-        const float cm = key_tree_max(kf);                                                                       \
-        /* a later chunk wins only with a strictly larger similarity (the index bits set aside) */              \
-        if (OC_VAL(cm) > OC_VAL(bm)) { bm = cm; bc = (ch); }                                                     \
+        const uint32_t masked = my_masked[(ch) - ch_begin];            /* warp-uniform, almost always zero */    \
+        if (masked) {                                                                                            \
+            _Pragma("unroll") for (int j = 0; j < 32; ++j)                                                       \
+                if ((masked >> j) & 1u) kf[j] = 0u;                                                              \
+        }                                                                                                        \
+        const uint32_t cm = key_tree_max(kf);                                                                    \
+        /* a later chunk wins only with a strictly larger similarity (the index bits set aside); a zeroed     */ \
+        /* key never does: a lifted similarity lies strictly above the binade's lower end, so a key is > 31  */ \
+        if (cm > (bm | 31u)) { bm = cm; bc = (ch); }                                                             \
         if (AUX && aux_row) {                                                                                    \
             for (int j = 0; j < 32; ++j) {                                                                       \
-                const float sc = col_scale1[(ch) * 32 + j];                                                      \
+                const float sc = col_scale1[((ch) - ch_begin) * 32 + j];                                         \
                 if (sc == sc) {                                                                                  \
                     const int gp_ = c.c_off + (ch) * 32 + j;                                                     \
                     const int qi = c.q0 + (gp_ >> 5), r = gp_ & 31;                                              \
@@ -746,28 +830,22 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             }                                                                                                    \
         }                                                                                                        \
     } while (0)
-                    if (t == 0) OC_TR(3, (int)it, 0, et == 0);
                     if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
 #pragma unroll 1
                     for (int ch = ch_begin; ch < ch_end; ch += 2) {
                         tmem_ld_wait();
-                        if (t == 0 && ch == ch_begin) OC_TR(3, (int)it, 1, et == 0);
                         if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);
                         OC_REDUCE_CHUNK(va, ch);
-                        if (t == 0 && ch == ch_begin) OC_TR(3, (int)it, 2, et == 0);
                         if (ch + 1 < ch_end) {
                             tmem_ld_wait();
-                            if (t == 0 && ch == ch_begin) OC_TR(3, (int)it, 3, et == 0);
                             if (ch + 2 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), va);
                             OC_REDUCE_CHUNK(vb, ch + 1);
                         }
                     }
 #undef OC_REDUCE_CHUNK
-#undef OC_KEY
-                    const int n0 = bc < 0 ? -1 : bc * 32 + OC_COL(bm);
-                    const float best = OC_VAL(bm) - row_lift;      // (exact: both are multiples of the key's last kept bit or larger)
-#undef OC_VAL
-#undef OC_COL
+                    const int n0 = bc < 0 ? -1 : bc * 32 + 31 - (int)(bm & 31u);
+                    // the winner's bits again: what the multiply dropped is what the lift's own bits have there
+                    const float best = __uint_as_float((bm >> 5) | (__float_as_uint(row_lift) & 0xF8000000u)) - row_lift;   // (exact)
                     if (row_ok && n0 >= 0) {
                         const int gp = c.c_off + n0;
                         const int qi = c.q0 + (gp >> 5), r = gp & 31;
@@ -787,10 +865,12 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             } else {
                 ok = false;
             }
-            // the next piece's table entries; the barrier publishes them, and keeps the table just read
-            // from being overwritten (in the next turn) while a slower warp still reads it
-            if (have_nx && et < 256) col_scale[((it + 1u) & 1u) * 256 + et] = sc_nx;
-            if (!epilogue_barrier_all<32 * EPI_WARPS>(ok)) { ok = false; break; }
+            if (!ok) break;
+            if (have_nx) {
+                publish(cols_ahead);
+                cols.ch_begin = cols_ahead.ch_begin; cols.ch_end = cols_ahead.ch_end;
+                if (nx.first) { cur = rows_ahead; set_lifts(cur); }
+            }
             OC_TR(2, (int)it, 3, et == 0);
             c = nx; have = have_nx;
             ++it;
@@ -1139,6 +1219,7 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     // two producers pay where a stage is short (one candidate tile per CTA); with two tiles the MMAs of a
     // stage cover one producer's work and the second warp only competes for issue slots
     P.n_prod = (N_PRODUCERS > 1 && p.tpp == 1) ? 2 : 1;
+    P.key_mul = 32u;
     P.units_per_group = (int)g.units_per_group; P.reps_per_group = (int)g.reps_per_group;
     P.inv_norm = inv_norm; P.keys = keys; P.aux = aux_sim; P.status = ctx->d_status;
     if (ctx->span_on) {
