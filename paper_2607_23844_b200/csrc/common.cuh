@@ -259,13 +259,16 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait: false if the phase did not complete within WAIT_LIMIT_NS or another role gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
+    // (the clock is first read after 256 failed tries: reading %globaltimer is slow, and nearly every wait
+    //  of the hot loops ends long before that)
+    unsigned long long t0 = 0;
     unsigned spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 255u) == 0) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) return false;
         }
     }
     return true;

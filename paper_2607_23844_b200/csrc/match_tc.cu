@@ -94,6 +94,11 @@ static constexpr int EPI_PARTS = EPI_WARPS / 4;           // a piece's columns a
 #endif
 static constexpr int N_PRODUCERS = OC_PRODUCERS;          // copy-producer warps: warp 0 and, with two, the last warp
 static constexpr int PRODUCER2_WARP = 2 + EPI_WARPS;
+// The epilogue warps come in two halves (each with one warp per TMEM lane quarter).  With two accumulator
+// sets the halves take alternate pieces (set = piece parity), each warp all columns of its rows; with one
+// set of two tiles, one tile each; with one set of one tile, half of the columns each.  The first two
+// give a warp twice the columns per piece it touches and half the pieces: its per-piece overhead halves.
+enum { EPI_BY_COLUMNS = 0, EPI_BY_PIECE = 1, EPI_BY_TILE = 2 };
 static constexpr int TC_THREADS = 64 + 32 * EPI_WARPS + 32 * (N_PRODUCERS - 1);   // producer, MMA, epilogue warps[, producer]
 static constexpr int MAX_LATTICES = 9;
 static constexpr uint32_t TMEM_COLS = 512;
@@ -125,6 +130,7 @@ struct TcScalars {
     int n_stages, stage_bytes;           // operand ring of this launch
     int n_prod;                          // copy-producer warps at work: 1, or 2 taking turns stage by stage
     unsigned key_mul;                    // 32, as a run-time value: keeps half of the key multiplies on the FMA pipe
+    int epi_split;                       // how the two halves of the epilogue warps share the work (EPI_BY_*)
     int a_res, a_region_bytes;           // candidate tiles resident: all 64-channel steps of a CTA's candidate tiles
                                          // sit in front of the ring (one slot per step) for all pieces of a row, and
                                          // the ring carries representatives only
@@ -300,9 +306,9 @@ __device__ unsigned long long g_tc_stage[8][512];
 #define OC_ACC_END(v)
 #endif
 
-static constexpr int COL_BYTES = EPI_WARPS * 128 * 4;                   // per epilogue warp: the scales of its (at most 128) columns
+static constexpr int COL_BYTES = EPI_WARPS * 256 * 4;                   // per epilogue warp: the scales of its (at most 256) columns
 static constexpr int N_BARS = 2 * MAX_STAGES + 5 + MAX_AKB;             // full[], empty[], acc_full[2], acc_empty[2], drain, a_empty[]
-static constexpr int TAIL_BYTES = COL_BYTES + N_BARS * 8 + 32 + EPI_WARPS * 16;   // column tables, barriers, TMEM slot, flags, masks
+static constexpr int TAIL_BYTES = COL_BYTES + N_BARS * 8 + 32 + EPI_WARPS * 32;   // column tables, barriers, TMEM slot, flags, masks
 static constexpr int TILE_BYTES = (SMEM_LIMIT - TAIL_BYTES) / 1024 * 1024;   // operand ring: everything else
 static constexpr int SMEM_TOTAL = TILE_BYTES + TAIL_BYTES;
 
@@ -328,7 +334,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     const uint32_t bar_a_empty = bar_drain + 8;                        // resident candidate slots, one per 64-channel step
     uint32_t* tmem_slot = (uint32_t*)(bars + N_BARS);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
-    uint32_t* col_masked = tmem_slot + 8;                              // [warp][4]: per 32-column chunk, its columns that are no representative
+    uint32_t* col_masked = tmem_slot + 8;                              // [warp][8]: per 32-column chunk, its columns that are no representative
     const uint32_t tiles_base = smem_u32(smem);
     const TcScalars& P = KP.s;
     if (P.span && threadIdx.x == 0) atomicMax(P.span, ~global_ns());
@@ -353,7 +359,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_acc_full + 8 * b, 1);
-            mbar_init(bar_acc_empty + 8 * b, PAIR ? 2 * EPI_WARPS : EPI_WARPS);   // one arrival per epilogue warp (of both CTAs)
+            // one arrival per epilogue warp (of both CTAs) that reads the accumulator set
+            mbar_init(bar_acc_empty + 8 * b, (PAIR ? 2 : 1) * (KP.s.epi_split == EPI_BY_PIECE ? EPI_WARPS / 2 : EPI_WARPS));
         }
         mbar_init(bar_drain, 1);
         for (int k = 0; k < MAX_AKB; ++k) mbar_init(bar_a_empty + 8 * k, 1);
@@ -464,13 +471,19 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                             // the copies first, the arrival that carries their byte count after them: the barrier
                             // cannot complete before that arrival, and the copies are on their way sooner
                             OC_ACC_BEGIN(acc_pt);
+#ifndef OC_EXP_NOTMA
                             tma_load_4d<PAIR>(ring_base + stage * STAGE_BYTES + q_off, mapQ, kb * BK, wQ, hQ, c.bt, full);
                             if (load_a)
                                 tma_load_4d<PAIR>(P.a_res ? tiles_base + (uint32_t)kb * a_step : ring_base + stage * STAGE_BYTES,
                                                   mapA, kb * BK, wA, hA, c.bt_a, full);
+#endif
                             OC_ACC_END(acc_pt);
                             OC_ACC_BEGIN(acc_pe);
+#ifdef OC_EXP_NOTMA
+                            if (leader) mbar_arrive(full_local);
+#else
                             if (leader) mbar_arrive_expect_tx(full_local, bytes);
+#endif
                             OC_ACC_END(acc_pe);
                         } else {
                             ok = false;
@@ -637,24 +650,26 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         const uint32_t acc_empty = PAIR ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;   // the leader's
         // Per column of a piece: the representative's inverse norm (NaN where the column is not a
         // representative of this patch; each chunk of 32 columns also has a bit mask of those, and
-        // their keys are zeroed).  Every epilogue warp keeps a table of its OWN columns -- at most four
+        // their keys are zeroed).  Every epilogue warp keeps a table of its OWN columns -- at most eight
         // chunks of 32 -- so the warps never wait for one another: a piece costs a warp its reduction
-        // and nothing else.  What the NEXT piece needs (the table entries, four per lane; each row's own
+        // and nothing else.  What its NEXT piece needs (the table entries, eight per lane; each row's own
         // norm) is fetched before this piece's accumulators are waited for and used after, so that
         // global-memory latency is never waited for either.
         const int ew = et >> 5;                                        // this warp among the epilogue warps
-        float* my_scale = (float*)colsb + ew * 128;
-        uint32_t* my_masked = col_masked + ew * 4;
+        float* my_scale = (float*)colsb + ew * 256;
+        uint32_t* my_masked = col_masked + ew * 8;
+        const int split = P.epi_split;
+        const int t_begin = split == EPI_BY_TILE ? part : 0, t_end = split == EPI_BY_TILE ? part + 1 : P.tpp;
         const uint32_t key_mul = P.key_mul;
         const int rowh = row >> P.bwA_log2, roww = row & (bwA - 1);
         // What a warp needs of a piece, gathered ahead of time.  A lone warp runs dependent integer
         // arithmetic at its full latency and pays for every branch, and this is on the one path that
         // bounds the kernel, so: no branches (selects and a clamped address instead), one division per
-        // piece (the lane's four columns lie in four consecutive quanta), and the row part only when
+        // piece (the lane's eight columns lie in eight consecutive quanta), and the row part only when
         // the row changes (the pieces of a row share their candidate tiles).
         struct Cols {
             int ch_begin, ch_end;            // this warp's chunks of 32 columns
-            float sc[4];                     // lane's table entries: column (ch_begin + i) * 32 + lane
+            float sc[8];                     // lane's table entries: column (ch_begin + i) * 32 + lane
         };
         struct Rows {
             int tokA[2];                     // the rows (candidate tokens) this thread owns in the piece's tiles
@@ -673,10 +688,13 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         const float quiet_nan = __int_as_float(0x7FC00000);
         const int tok_per_lattice_row = P.sy * P.W;
         auto gather_cols = [&](const Piece& pc, Cols& a) {
-            // chunks of 32 columns: the first half of them to warps 2..5, the rest to warps 6..9
+            // chunks of 32 columns: all of them, or the first half to warps 2..5 and the rest to warps 6..9
             const int n_ch = (pc.ncol + 31) >> 5;                       // (a last half chunk reads 16 columns of
-            a.ch_begin = (part * n_ch + EPI_PARTS - 1) / EPI_PARTS;     //  nothing: their table entries are NaN)
-            a.ch_end = ((part + 1) * n_ch + EPI_PARTS - 1) / EPI_PARTS;
+            a.ch_begin = 0; a.ch_end = n_ch;                            //  nothing: their table entries are NaN)
+            if (split == EPI_BY_COLUMNS) {
+                a.ch_begin = (part * n_ch + EPI_PARTS - 1) / EPI_PARTS;
+                a.ch_end = ((part + 1) * n_ch + EPI_PARTS - 1) / EPI_PARTS;
+            }
             const int g0 = pc.c_off + lane;                             // the lane's column, counted from the piece's first quantum
             const int r = g0 & 31, rh = r >> P.bwQ_log2, rw = r & (bwQ - 1);
             const int qi = pc.q0 + (g0 >> 5) + a.ch_begin;
@@ -685,7 +703,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             const int tok0 = (pc.bt * P.H + pc.py * P.Hs * P.sy + my_rep) * P.W + pc.px * P.Ws * P.sx + mx_rep;
             const int col0 = a.ch_begin * 32 + lane;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 8; ++i) {
                 const int hs = hq * P.bhQ + rh, ws = wq * bwQ + rw;
                 const bool valid = (a.ch_begin + i < a.ch_end) & (col0 + 32 * i < pc.ncol) & (hs < P.Hs) & (ws < P.Ws);
                 const int tok = valid ? tok0 + hs * tok_per_lattice_row + ws * P.sx : 0;
@@ -724,7 +742,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         auto publish = [&](const Cols& a) {
             __syncwarp();
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < 8; ++i) {
                 my_scale[i * 32 + lane] = a.sc[i];
                 const uint32_t masked = __ballot_sync(0xFFFFFFFFu, a.sc[i] != a.sc[i]);
                 if (lane == 0) my_masked[i] = masked;
@@ -738,18 +756,31 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         Piece nx;
         Cols cols, cols_ahead;
         Rows cur, rows_ahead;
-        bool have = walk.next(P, c);
+        // this warp's next piece: every piece, or (EPI_BY_PIECE) every other one
+        uint32_t handed = 0;                                           // pieces the walk has handed out
+        auto next_mine = [&](Piece& pc, uint32_t& index, bool& new_row) -> bool {
+            new_row = false;
+            for (;;) {
+                if (!walk.next(P, pc)) return false;
+                index = handed++;
+                new_row |= pc.first != 0;
+                if (split != EPI_BY_PIECE || (index & 1u) == (uint32_t)part) return true;
+            }
+        };
+        uint32_t it_nx = 0;
+        bool new_row = false;
+        bool have = next_mine(c, it, new_row);
         if (have) { gather_cols(c, cols); gather_rows(c, cur); publish(cols); set_lifts(cur); }
         while (have) {
             const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
             const float4* col_scale4 = (const float4*)my_scale;
             const float* col_scale1 = my_scale;
             OC_TR(3, (int)it, 0, et == 0);
-            const bool have_nx = walk.next(P, nx);
+            const bool have_nx = next_mine(nx, it_nx, new_row);
             OC_TR(3, (int)it, 1, et == 0);
             if (have_nx) {                                             // in flight until the end of this piece
                 gather_cols(nx, cols_ahead);
-                if (nx.first) gather_rows(nx, rows_ahead);
+                if (new_row) gather_rows(nx, rows_ahead);
             }
             OC_TR(3, (int)it, 2, et == 0);
             const int my = cur.my, mx = cur.mx;
@@ -763,10 +794,11 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             OC_TR(2, (int)it, 1, et == 0);
             if (ready) {
                 tc_fence_after();
+                uint32_t won_key0 = 0, won_key1 = 0;                   // per tile: the row's largest key and its chunk
+                int won_ch0 = -1, won_ch1 = -1;
 #pragma unroll 1
-                for (int t = 0; t < P.tpp; ++t) {                      // the piece's candidate tiles
+                for (int t = t_begin; t < t_end; ++t) {                // the piece's candidate tiles (of this warp)
                     if ((PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + t >= P.n_tilesA) continue;   // past the lattice
-                    const int tokA = (t ? cur.tokA[1] : cur.tokA[0]);
                     const bool row_ok = (t ? cur.row_ok[1] : cur.row_ok[0]);
                     float inv_a = 0.f;
                     float* aux_row = nullptr;
@@ -830,9 +862,15 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             }                                                                                                    \
         }                                                                                                        \
     } while (0)
+#ifndef OC_EXP_NOEPI
                     if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
+#endif
 #pragma unroll 1
+#ifdef OC_EXP_NOEPI
+                    for (int ch = ch_begin; ch < ch_begin; ch += 2) {
+#else
                     for (int ch = ch_begin; ch < ch_end; ch += 2) {
+#endif
                         tmem_ld_wait();
                         if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);
                         OC_REDUCE_CHUNK(va, ch);
@@ -843,24 +881,32 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                         }
                     }
 #undef OC_REDUCE_CHUNK
-                    const int n0 = bc < 0 ? -1 : bc * 32 + 31 - (int)(bm & 31u);
-                    // the winner's bits again: what the multiply dropped is what the lift's own bits have there
-                    const float best = __uint_as_float((bm >> 5) | (__float_as_uint(row_lift) & 0xF8000000u)) - row_lift;   // (exact)
-                    if (row_ok && n0 >= 0) {
-                        const int gp = c.c_off + n0;
-                        const int qi = c.q0 + (gp >> 5), r = gp & 31;
-                        const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
-                        const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));
-                        const int y = (c.py * P.Hs + hs) * P.sy + my_rep, x = (c.px * P.Ws + ws) * P.sx + mx_rep;
-                        const long long tokB = ((long long)c.bt * P.H + y) * P.W + x;
-                        atomicMax(P.keys + tokA, pack_key(best, (uint32_t)tokB));
-                    }
+                    if (t) { won_key1 = bm; won_ch1 = row_ok ? bc : -1; } else { won_key0 = bm; won_ch0 = row_ok ? bc : -1; }
                 }
                 tc_fence_before();
                 __syncwarp();
                 OC_TR(2, (int)it, 2, et == 0);
                 if (lane == 0) {                                       // both accumulators may be overwritten
                     if (PAIR) mbar_arrive_cluster(acc_empty + 8 * buf); else mbar_arrive(bar_acc_empty + 8 * buf);
+                }
+                // The rows' results go out only now: the arrival above releases (at cluster scope, in a
+                // pair) what its thread wrote before it, and would wait for these atomics to be performed.
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    const uint32_t bm = t ? won_key1 : won_key0;
+                    const int bc = t ? won_ch1 : won_ch0;
+                    if (bc < 0) continue;
+                    const float row_lift = t ? lift1 : lift0;
+                    const int n0 = bc * 32 + 31 - (int)(bm & 31u);
+                    // the winner's bits again: what the multiply dropped is what the lift's own bits have there
+                    const float best = __uint_as_float((bm >> 5) | (__float_as_uint(row_lift) & 0xF8000000u)) - row_lift;   // (exact)
+                    const int gp = c.c_off + n0;
+                    const int qi = c.q0 + (gp >> 5), r = gp & 31;
+                    const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
+                    const int hs = hq * P.bhQ + (r >> P.bwQ_log2), ws = wq * bwQ + (r & (bwQ - 1));
+                    const int y = (c.py * P.Hs + hs) * P.sy + my_rep, x = (c.px * P.Ws + ws) * P.sx + mx_rep;
+                    const long long tokB = ((long long)c.bt * P.H + y) * P.W + x;
+                    atomicMax(P.keys + (t ? cur.tokA[1] : cur.tokA[0]), pack_key(best, (uint32_t)tokB));
                 }
             } else {
                 ok = false;
@@ -869,11 +915,11 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             if (have_nx) {
                 publish(cols_ahead);
                 cols.ch_begin = cols_ahead.ch_begin; cols.ch_end = cols_ahead.ch_end;
-                if (nx.first) { cur = rows_ahead; set_lifts(cur); }
+                if (new_row) { cur = rows_ahead; set_lifts(cur); }
             }
             OC_TR(2, (int)it, 3, et == 0);
             c = nx; have = have_nx;
-            ++it;
+            it = it_nx;
         }
         if (!ok) { atomicCAS(P.status, 0, OC_ERR_TIMEOUT); *abort_flag = 1; }
     }
@@ -1220,6 +1266,7 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     // stage cover one producer's work and the second warp only competes for issue slots
     P.n_prod = (N_PRODUCERS > 1 && p.tpp == 1) ? 2 : 1;
     P.key_mul = 32u;
+    P.epi_split = (p.tpp == 1 || p.narrow) ? EPI_BY_PIECE : (p.tpp == 2 ? EPI_BY_TILE : EPI_BY_COLUMNS);
     P.units_per_group = (int)g.units_per_group; P.reps_per_group = (int)g.reps_per_group;
     P.inv_norm = inv_norm; P.keys = keys; P.aux = aux_sim; P.status = ctx->d_status;
     if (ctx->span_on) {
