@@ -431,6 +431,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         bool joined = !early_producer;                // whether this warp has met the set-up barrier yet
         const uint32_t ring_base = tiles_base + (uint32_t)P.a_region_bytes;       // (a_region_bytes is 0 unless a_res)
         const bool solo = P.a_merged && P.q_merged;
+        const uint32_t issue = elect_one();
 #ifdef OC_TC_TRACE
         unsigned long long acc_pw = 0, acc_pt = 0, acc_pe = 0, acc_pp = 0; const unsigned long long acc_p0 = clock64();
 #endif
@@ -459,31 +460,31 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 const CUtensorMap* mapQ = &KP.mapQ[nq_mine != P.q_lo ? 1 : 0];
                 OC_ACC_END(acc_pp);
                 for (int kb = 0; kb < P.kblocks; ++kb, ++gstage) {
-                    if (lane == 0 && ok && (P.n_prod < 2 || (gstage & 1u) == my_turn)) {
+                    // (the whole warp runs this; the elected lane issues)
+                    if (ok && (P.n_prod < 2 || (gstage & 1u) == my_turn)) {
                         const uint32_t full_local = bar_full + 8 * stage;
                         const uint32_t full = PAIR ? map_to_cta(full_local, 0) : full_local;
                         OC_ACC_BEGIN(acc_pw);
+                        OC_TS(2, gstage, lane == 0);
                         bool go = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
+                        OC_TS(7, gstage, lane == 0);
                         OC_ACC_END(acc_pw);
                         // the slot of this step is free once the MMAs of the previous row's last piece have read it
                         if (go && P.a_res && load_a) go = mbar_wait(bar_a_empty + 8 * kb, a_phase ^ 1u, abort_flag);
-                        if (go) {
+                        if (__all_sync(0xFFFFFFFFu, go)) {
                             // the copies first, the arrival that carries their byte count after them: the barrier
                             // cannot complete before that arrival, and the copies are on their way sooner
                             OC_ACC_BEGIN(acc_pt);
 #ifndef OC_EXP_NOTMA
-                            tma_load_4d<PAIR>(ring_base + stage * STAGE_BYTES + q_off, mapQ, kb * BK, wQ, hQ, c.bt, full);
+                            tma_load_4d_elected<PAIR>(ring_base + stage * STAGE_BYTES + q_off, mapQ, kb * BK, wQ, hQ, c.bt, full, issue);
                             if (load_a)
-                                tma_load_4d<PAIR>(P.a_res ? tiles_base + (uint32_t)kb * a_step : ring_base + stage * STAGE_BYTES,
-                                                  mapA, kb * BK, wA, hA, c.bt_a, full);
+                                tma_load_4d_elected<PAIR>(P.a_res ? tiles_base + (uint32_t)kb * a_step : ring_base + stage * STAGE_BYTES,
+                                                          mapA, kb * BK, wA, hA, c.bt_a, full, issue);
 #endif
                             OC_ACC_END(acc_pt);
                             OC_ACC_BEGIN(acc_pe);
-#ifdef OC_EXP_NOTMA
-                            if (leader) mbar_arrive(full_local);
-#else
-                            if (leader) mbar_arrive_expect_tx(full_local, bytes);
-#endif
+                            if (leader) mbar_arrive_expect_tx_elected(full_local, bytes, issue);
+                            OC_TS(3, gstage, lane == 0);
                             OC_ACC_END(acc_pe);
                         } else {
                             ok = false;
@@ -495,8 +496,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     if (!joined) { __syncwarp(); __syncthreads(); joined = true; }   // first stage on its way: meet the others
                 }
-                __syncwarp();
-                ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;        // (lane 0 alone knows; once per piece)
             } else {
                 const CUtensorMap* map;
                 int w, h;
@@ -572,10 +571,18 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                                             ((uint32_t)((PAIR ? 2 * BM : BM) >> 4) << 24);   // M=128 (256 across a pair)
             const uint32_t issue = elect_one();        // all lanes walk the loop, this one issues
             int stage = 0; uint32_t phase = 0;
+            // K-major, 128-byte swizzle (as make_smem_desc): the constant part of every operand descriptor,
+            // and the parts of the address field (16-byte units) that the loop adds up
+            const uint64_t desc_hi = make_smem_desc(0);
+            const bool a_res = P.a_res != 0;
+            const int kblocks = P.kblocks;
+            const uint32_t res_lo = (tiles_base >> 4) & 0x3FFFu, ring_lo = ((tiles_base + (uint32_t)P.a_region_bytes) >> 4) & 0x3FFFu;
+            const uint32_t stage16 = (uint32_t)STAGE_BYTES >> 4, a_tile16 = (uint32_t)A_BYTES >> 4;
+            const uint32_t a_slot16 = (uint32_t)(P.tpp * A_BYTES) >> 4, q_off16 = a_res ? 0u : a_slot16;
             bool ok = true, peeked = false;
             uint32_t it = 0;
 #ifdef OC_TC_TRACE
-            unsigned long long acc_mf = 0, acc_ma = 0, acc_mi = 0; const unsigned long long acc_m0 = clock64();
+            unsigned long long acc_mf = 0, acc_ma = 0, acc_mi = 0; const unsigned long long acc_m0 = clock64(); unsigned mstage = 0;
 #endif
             while (ok && walk.next(P, c)) {
                 // one candidate tile per CTA leaves half of TMEM free: two accumulators take turns, and the
@@ -593,35 +600,42 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 // an odd number of candidate tiles leaves the last run with an empty second tile (in a pair:
                 // empty in both CTAs): its MMAs are not issued, and the epilogue skips it likewise
                 const bool two_tiles = P.tpp == 2 && (PAIR ? 2 : 1) * P.tpp * c.a_pair + 1 < P.n_tilesA;
-                for (int kb = 0; kb < P.kblocks; ++kb) {
+                // descriptors of the piece's operands: low words only (the high word is one constant), kept
+                // up to date by additions -- between two stages the tensor pipe runs dry unless this warp is
+                // back with the next MMA within about one MMA's time
+                const uint32_t c_off16 = (uint32_t)c.c_off * 8u;        // (c_off rows of 128 bytes, in 16-byte units)
+                const uint32_t free_a = (a_res && c.last) ? 1u : 0u;
+                for (int kb = 0; kb < kblocks; ++kb) {
                     // (each lane looked for itself; the barrier's phase cannot go back, so a lane that saw it
                     //  full stays right, and the others wait here)
                     OC_ACC_BEGIN(acc_mf);
-                    if (!peeked && !mbar_wait(bar_full + 8 * stage, phase, abort_flag)) ok = false;
-                    if (!__all_sync(0xFFFFFFFFu, ok)) { ok = false; break; }
+                    OC_TS(4, mstage, lane == 0);
+                    if (!peeked) {
+                        if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) ok = false;
+                        if (!__all_sync(0xFFFFFFFFu, ok)) { ok = false; break; }
+                    }
+                    OC_TS(5, mstage, lane == 0);
                     OC_ACC_END(acc_mf);
                     OC_ACC_BEGIN(acc_mi);
                     if (kb == 0) OC_TR(1, (int)it - 1, 2, lane == 0);
-                    const uint32_t s_addr = tiles_base + (uint32_t)P.a_region_bytes + stage * STAGE_BYTES;
-                    const uint32_t a_addr = P.a_res ? tiles_base + (uint32_t)(kb * P.tpp * A_BYTES) : s_addr;
-                    const uint64_t a0_desc = make_smem_desc(a_addr);
-                    const uint64_t a1_desc = make_smem_desc(a_addr + A_BYTES);
+                    const uint32_t s_lo = ring_lo + (uint32_t)stage * stage16;
+                    const uint32_t a_lo = a_res ? res_lo + (uint32_t)kb * a_slot16 : s_lo;
                     // (a piece that begins in mid-quantum skips 16 rows = 2 KB of its first box: a whole number
                     //  of 8-row swizzle groups)
-                    const uint64_t b_desc = make_smem_desc(s_addr + (P.a_res ? 0 : P.tpp * A_BYTES) + (uint32_t)c.c_off * 128u);
+                    const uint32_t b_lo = s_lo + q_off16 + c_off16;
                     int nstage = stage + 1; uint32_t nphase = phase;
                     if (nstage == STAGES) { nstage = 0; nphase ^= 1u; }
-                    // UMMA K = 16 is 32 bytes along the swizzled row: +2 in the descriptor's address field
-                    peeked = tc_mma_stage<PAIR>(d_tmem, a0_desc, a1_desc, b_desc, idesc, (uint32_t)(kb != 0), issue,
-                                                two_tiles, bar_full + 8 * nstage, nphase, tile_stride) != 0;
-                    // frees the stage (in both CTAs of a pair) when the MMAs retire
-                    tc_commit<PAIR>(PAIR ? map_to_cta(bar_empty + 8 * stage, 0) : bar_empty + 8 * stage, issue);
-                    if (PAIR) tc_commit<PAIR>(map_to_cta(bar_empty + 8 * stage, 1), issue);
+                    // UMMA K = 16 is 32 bytes along the swizzled row: +2 in the descriptor's address field.
+                    // The commits free the stage (in both CTAs of a pair) when the MMAs retire, and with the
+                    // row's last piece the resident candidate slot of this step.
+                    peeked = tc_mma_stage<PAIR>(d_tmem, desc_hi | a_lo, desc_hi | (a_lo + a_tile16), desc_hi | b_lo, idesc,
+                                                (uint32_t)(kb != 0), issue, two_tiles, bar_full + 8 * nstage, nphase, tile_stride,
+                                                bar_empty + 8 * stage, free_a ? bar_a_empty + 8 * kb : 0u) != 0;
                     OC_ACC_END(acc_mi);
-                    if (P.a_res && c.last) {         // the row's candidate tiles of this step have been read for the last time
-                        tc_commit<PAIR>(PAIR ? map_to_cta(bar_a_empty + 8 * kb, 0) : bar_a_empty + 8 * kb, issue);
-                        if (PAIR) tc_commit<PAIR>(map_to_cta(bar_a_empty + 8 * kb, 1), issue);
-                    }
+                    OC_TS(6, mstage, lane == 0);
+#ifdef OC_TC_TRACE
+                    ++mstage;
+#endif
                     stage = nstage; phase = nphase;
                 }
                 OC_TR(1, (int)it - 1, 3, lane == 0);

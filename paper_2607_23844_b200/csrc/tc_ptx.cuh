@@ -12,9 +12,12 @@ namespace oc {
 __device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" :: "l"(map) : "memory");
 }
-// arrive on a barrier given by its cluster-wide shared address (own CTA or the other CTA of a pair)
+// arrive on a barrier given by its cluster-wide shared address (own CTA or the other CTA of a pair).
+// What the arrival orders here are reads of tensor memory, which the tcgen05 fences around it cover; it
+// publishes no ordinary memory to the other CTA, so the default (CTA-scope) release is enough, and a
+// cluster-scope one would wait for the thread's outstanding global-memory traffic first.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" :: "r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" :: "r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -42,6 +45,27 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         asm volatile(
             "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
             :: "r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+// The same copy issued by the one lane whose `issue` is non-zero, from code that the whole warp runs:
+// addresses and coordinates then stay warp-uniform values (a lone diverged lane would have them moved
+// from per-thread to uniform registers before every instruction, which costs it hundreds of cycles).
+template <bool PAIR>
+__device__ __forceinline__ void tma_load_4d_elected(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                    uint32_t bar, uint32_t issue) {
+    if (PAIR)
+        asm volatile(
+            "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %7, 0;\n\t"
+            "@e cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n\t}"
+            :: "r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar), "r"(issue) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %7, 0;\n\t"
+            "@e cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n\t}"
+            :: "r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar), "r"(issue) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_elected(uint32_t bar, uint32_t bytes, uint32_t issue) {
+    asm volatile("{\n\t.reg .pred e;\n\tsetp.ne.b32 e, %2, 0;\n\t"
+                 "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t}" :: "r"(bar), "r"(bytes), "r"(issue) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -127,11 +151,19 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
 // between two stages (the tensor pipe accepts an MMA only about when the previous one starts, so
 // nothing else hides that gap).
 // tile_stride: TMEM columns between the accumulators of the two candidate tiles.
+// The commits that follow a stage's MMAs are part of the same block -- the one that frees the stage's
+// ring slot and, when a_empty_bar is non-zero, the one that frees a resident candidate slot -- so that
+// nothing the compiler schedules comes between them: in a pair ONE commit with a CTA mask signals the
+// barrier at the same address in both CTAs.
 // Returns non-zero when the next stage was already full.
-#define OC_MMA_STAGE_ASM(CG, TWO)                                                                        \
+#define OC_COMMIT_CG1(bar, pred) "@" pred " tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [" bar "];\n\t"
+#define OC_COMMIT_CG2(bar, pred) "@" pred " tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [" bar "], both;\n\t"
+#define OC_MMA_STAGE_ASM(CG, TWO, COMMIT)                                                                \
     asm volatile(                                                                                       \
         "{\n\t"                                                                                         \
-        ".reg .pred pa, pt, e, r;\n\t"                                                                  \
+        ".reg .pred pa, pt, e, r, ea;\n\t"                                                              \
+        ".reg .b16 both;\n\t"                                                                           \
+        "mov.b16 both, 3;\n\t"                                                                          \
         ".reg .b64 a0, a1, bb;\n\t"                                                                     \
         ".reg .b32 d1;\n\t"                                                                             \
         "setp.ne.b32 pa, %5, 0;\n\t"                                                                    \
@@ -150,23 +182,28 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
         "add.u64 a0, %2, 6;\n\tadd.u64 a1, %3, 6;\n\tadd.u64 bb, %4, 6;\n\t"                          \
         "@e tcgen05.mma.cta_group::" CG ".kind::f16 [%1], a0, bb, %9, pt;\n\t"                          \
         TWO("@e tcgen05.mma.cta_group::" CG ".kind::f16 [d1], a1, bb, %9, pt;\n\t")                     \
+        COMMIT("%11", "e")                                                                              \
+        "setp.ne.b32 ea, %12, 0;\n\t"                                                                   \
+        "and.pred ea, ea, e;\n\t"                                                                       \
+        COMMIT("%12", "ea")                                                                             \
         "selp.b32 %0, 1, 0, r;\n\t"                                                                     \
         "}"                                                                                             \
         : "=r"(ready)                                                                                   \
         : "r"(d_tmem), "l"(a0_desc), "l"(a1_desc), "l"(b_desc), "r"(accumulate), "r"(issue), "r"(next_bar), \
-          "r"(next_parity), "r"(idesc), "r"(tile_stride)                                                \
+          "r"(next_parity), "r"(idesc), "r"(tile_stride), "r"(empty_bar), "r"(a_empty_bar)              \
         : "memory")
 #define OC_KEEP(x) x
 #define OC_DROP(x)
 template <bool PAIR>
 __device__ __forceinline__ uint32_t tc_mma_stage(uint32_t d_tmem, uint64_t a0_desc, uint64_t a1_desc, uint64_t b_desc,
                                                  uint32_t idesc, uint32_t accumulate, uint32_t issue, bool two_tiles,
-                                                 uint32_t next_bar, uint32_t next_parity, uint32_t tile_stride) {
+                                                 uint32_t next_bar, uint32_t next_parity, uint32_t tile_stride,
+                                                 uint32_t empty_bar, uint32_t a_empty_bar) {
     uint32_t ready;
     if (two_tiles) {
-        if (PAIR) OC_MMA_STAGE_ASM("2", OC_KEEP); else OC_MMA_STAGE_ASM("1", OC_KEEP);
+        if (PAIR) OC_MMA_STAGE_ASM("2", OC_KEEP, OC_COMMIT_CG2); else OC_MMA_STAGE_ASM("1", OC_KEEP, OC_COMMIT_CG1);
     } else {
-        if (PAIR) OC_MMA_STAGE_ASM("2", OC_DROP); else OC_MMA_STAGE_ASM("1", OC_DROP);
+        if (PAIR) OC_MMA_STAGE_ASM("2", OC_DROP, OC_COMMIT_CG2); else OC_MMA_STAGE_ASM("1", OC_DROP, OC_COMMIT_CG1);
     }
     return ready;
 }
