@@ -584,6 +584,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
 #ifdef OC_TC_TRACE
             unsigned long long acc_mf = 0, acc_ma = 0, acc_mi = 0; const unsigned long long acc_m0 = clock64(); unsigned mstage = 0;
 #endif
+            // (the commit that hands the accumulators to the epilogue is part of the last stage's block; taking
+            //  the walk to the next piece between two stages instead of between two pieces measured slower)
             while (ok && walk.next(P, c)) {
                 // one candidate tile per CTA leaves half of TMEM free: two accumulators take turns, and the
                 // epilogue of a piece runs under the MMAs of the next one
@@ -630,7 +632,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     // row's last piece the resident candidate slot of this step.
                     peeked = tc_mma_stage<PAIR>(d_tmem, desc_hi | a_lo, desc_hi | (a_lo + a_tile16), desc_hi | b_lo, idesc,
                                                 (uint32_t)(kb != 0), issue, two_tiles, bar_full + 8 * nstage, nphase, tile_stride,
-                                                bar_empty + 8 * stage, free_a ? bar_a_empty + 8 * kb : 0u) != 0;
+                                                bar_empty + 8 * stage, free_a ? bar_a_empty + 8 * kb : 0u,
+                                                kb + 1 == kblocks ? bar_acc_full + 8 * buf : 0u) != 0;
                     OC_ACC_END(acc_mi);
                     OC_TS(6, mstage, lane == 0);
 #ifdef OC_TC_TRACE
@@ -639,10 +642,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     stage = nstage; phase = nphase;
                 }
                 OC_TR(1, (int)it - 1, 3, lane == 0);
-                if (ok) {
-                    tc_commit<PAIR>(PAIR ? map_to_cta(bar_acc_full + 8 * buf, 0) : bar_acc_full + 8 * buf, issue);
-                    if (PAIR) tc_commit<PAIR>(map_to_cta(bar_acc_full + 8 * buf, 1), issue);
-                }
             }
 #ifdef OC_TC_TRACE
             if (blockIdx.x == OC_TC_TRACE && lane == 0) { g_tc_stage[1][0] = acc_mf; g_tc_stage[1][1] = acc_ma; g_tc_stage[1][2] = acc_mi; g_tc_stage[1][3] = clock64() - acc_m0; g_tc_stage[1][4] = it; }
@@ -1025,17 +1024,20 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
     p.n_quanta = p.n_wq * ((g.Hs + p.bhQ - 1) / p.bhQ);
     // Form (single CTA or CTA pair), candidate tiles per CTA (1 or 2), pieces per row and whether the
     // candidate tiles stay resident, by estimated cycles of the busiest walker.  The shape of the estimate
-    // follows the kernel; its constants were fitted (least squares on the logarithm, over 60 timed plans)
+    // follows the kernel; its constants were fitted (least squares on the logarithm, over 40 timed plans)
     // to sweeps of forced plans on four workloads (the SD3-shaped token cache and the three SVD UNet
-    // levels) and reproduce every one of those times within a few per cent:
-    //   * a 64-channel stage issues tpp*64*q tensor cycles and cannot go faster than the hand-over of a
-    //     ring slot between the copy producer and the MMA issuer (~650 cycles while the epilogue runs
-    //     beside the MMAs, ~950 when it follows them), nor than its bytes at ~58 B/clk;
-    //   * the epilogue costs ~420 + ~370 cycles per 32 columns of each thread's half, per tile; with two
-    //     accumulator sets (one tile, or two tiles and pieces of at most 128 columns) it runs under the
-    //     next piece's MMAs and the piece takes the longer of the two plus ~13 % of the shorter,
-    //     otherwise it follows them;
-    //   * ~2500 cycles before a CTA's first MMA and after its last.
+    // levels); the estimate picks the fastest measured plan on each of them:
+    //   * a 64-channel stage issues tpp*64*q tensor cycles (x0.9 as fitted) and cannot go faster than
+    //     the hand-over of a ring slot (~490 cycles), than its copies arrive (~81 B/clk), nor than shared
+    //     memory serves the copies' writes and the MMAs' operand reads together (~138 B/clk: one tile of
+    //     256 columns reads 48 KB and is sent 32 KB per stage; a CTA pair halves the representatives' part
+    //     of both, which is what makes the pair faster on wide pieces);
+    //   * the epilogue costs ~340 cycles per 32 columns per tile.  With two accumulator sets (one tile, or
+    //     two tiles and pieces of at most 128 columns) each half of its warps takes every other piece and
+    //     runs under the MMAs of the next one: the piece takes the longest of its MMAs, half its epilogue,
+    //     and half of (epilogue + MMAs) plus ~720 (a set is not reused before its epilogue is over);
+    //     otherwise the epilogue follows the MMAs;
+    //   * ~3400 cycles before a CTA's first MMA and after its last.
     const int kblocks = (g.C + BK - 1) / BK;
     // Single-CTA pieces are cut in units of HALF a quantum (16 columns) whenever that is valid: no piece
     // wider than 256 columns, none that would have to fetch more than MAXQ quanta (one that begins in
@@ -1064,26 +1066,29 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
                 const double qe = hw ? hw * 0.5 : (double)q;          // width in quanta (may end in a half)
                 if (hw) q = (hw + 1) >> 1;
                 const long long per_walker = (rows * P + nw - 1) / nw;
-                const double mma = tpp * 64.0 * qe;
-                const double epi = tpp * (420.0 + 370.0 * ((q + 1) / 2));
+                const double mma = tpp * 64.0 * qe * 0.897;
                 // (two tiles whose pieces are at most 128 columns wide leave room for a second set of
                 //  accumulators, like one tile does)
-                const bool overlapped = tpp == 1 || (hw ? hw * 16 : q * 32) <= 128;
-                for (int ar = 0; ar <= 1; ++ar) {
+                const int cols = hw ? hw * 16 : q * 32, chunks = (cols + 31) / 32;
+                const bool overlapped = tpp == 1 || cols <= 128;
+                const double epi_all = 338.4 * (overlapped ? tpp * chunks : (tpp == 2 ? chunks : (chunks + 1) / 2));
+                const double epi = overlapped ? 0.5 * epi_all : epi_all;   // per piece and warp
+                for (int ar = 1; ar >= 0; --ar) {                           // (equal estimates: fewer bytes fetched wins)
                     const double a_kb = tpp * 16.0, q_kb = 4.0 * q_load / ncta;
                     if (ar && (kblocks > MAX_AKB || a_kb * kblocks + 3 * q_kb > TILE_BYTES / 1024 || P == 1)) continue;
-                    const double feed = ((ar ? 0.0 : a_kb) + q_kb) * 1024.0 / 58.4;
+                    const double sent_kb = (ar ? 0.0 : a_kb) + q_kb, read_kb = tpp * (16.0 + 4.0 * qe / ncta);
+                    const double feed = sent_kb * 1024.0 / 80.7, smem = (sent_kb + read_kb) * 7.42;
                     double piece;
                     if (overlapped) {
-                        double stage = mma + 46.0; if (stage < 648.0) stage = 648.0; if (stage < feed) stage = feed;
-                        const double loop = kblocks * stage + 904.0, tail = epi + 2919.0;
-                        piece = (loop > tail ? loop : tail) + 0.13 * (kblocks * stage < epi ? kblocks * stage : epi);
+                        double stage = mma + 54.0; if (stage < 488.0) stage = 488.0; if (stage < feed) stage = feed; if (stage < smem) stage = smem;
+                        const double loop = kblocks * stage + 530.0, reuse = 0.5 * (epi_all + loop) + 723.0;
+                        piece = loop; if (piece < epi + 66.0) piece = epi + 66.0; if (piece < reuse) piece = reuse;
                     } else {
-                        double stage = mma + 480.0; if (stage < 948.0) stage = 948.0; if (stage < feed) stage = feed;
-                        piece = kblocks * stage + epi + 1022.0;
+                        double stage = mma + 213.0; if (stage < 307.0) stage = 307.0; if (stage < feed) stage = feed; if (stage < smem) stage = smem;
+                        piece = kblocks * stage + epi + 955.0;
                     }
-                    if (pair) piece += 850.0;
-                    const double cost = 2450.0 + per_walker * piece + (overlapped ? epi : 0.0);
+                    if (pair) piece += 123.0;
+                    const double cost = 3377.0 + per_walker * piece + (overlapped ? epi_all : 0.0);
                     if (best_P == 0 || cost < best_cost) { best_cost = cost; best_P = P; best_tpp = tpp; best_pair = pair; best_ar = ar; }
                 }
             }

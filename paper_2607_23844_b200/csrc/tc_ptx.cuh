@@ -152,7 +152,8 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
 // nothing else hides that gap).
 // tile_stride: TMEM columns between the accumulators of the two candidate tiles.
 // The commits that follow a stage's MMAs are part of the same block -- the one that frees the stage's
-// ring slot and, when a_empty_bar is non-zero, the one that frees a resident candidate slot -- so that
+// ring slot, when a_empty_bar is non-zero the one that frees a resident candidate slot, and when
+// acc_full_bar is non-zero (the piece's last stage) the one that hands the accumulators over -- so that
 // nothing the compiler schedules comes between them: in a pair ONE commit with a CTA mask signals the
 // barrier at the same address in both CTAs.
 // Returns non-zero when the next stage was already full.
@@ -161,7 +162,7 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
 #define OC_MMA_STAGE_ASM(CG, TWO, COMMIT)                                                                \
     asm volatile(                                                                                       \
         "{\n\t"                                                                                         \
-        ".reg .pred pa, pt, e, r, ea;\n\t"                                                              \
+        ".reg .pred pa, pt, e, r, ea, ef;\n\t"                                                          \
         ".reg .b16 both;\n\t"                                                                           \
         "mov.b16 both, 3;\n\t"                                                                          \
         ".reg .b64 a0, a1, bb;\n\t"                                                                     \
@@ -186,11 +187,14 @@ __device__ __forceinline__ bool epilogue_barrier_all(bool ok) {
         "setp.ne.b32 ea, %12, 0;\n\t"                                                                   \
         "and.pred ea, ea, e;\n\t"                                                                       \
         COMMIT("%12", "ea")                                                                             \
+        "setp.ne.b32 ef, %13, 0;\n\t"                                                                   \
+        "and.pred ef, ef, e;\n\t"                                                                       \
+        COMMIT("%13", "ef")                                                                             \
         "selp.b32 %0, 1, 0, r;\n\t"                                                                     \
         "}"                                                                                             \
         : "=r"(ready)                                                                                   \
         : "r"(d_tmem), "l"(a0_desc), "l"(a1_desc), "l"(b_desc), "r"(accumulate), "r"(issue), "r"(next_bar), \
-          "r"(next_parity), "r"(idesc), "r"(tile_stride), "r"(empty_bar), "r"(a_empty_bar)              \
+          "r"(next_parity), "r"(idesc), "r"(tile_stride), "r"(empty_bar), "r"(a_empty_bar), "r"(acc_full_bar) \
         : "memory")
 #define OC_KEEP(x) x
 #define OC_DROP(x)
@@ -198,7 +202,7 @@ template <bool PAIR>
 __device__ __forceinline__ uint32_t tc_mma_stage(uint32_t d_tmem, uint64_t a0_desc, uint64_t a1_desc, uint64_t b_desc,
                                                  uint32_t idesc, uint32_t accumulate, uint32_t issue, bool two_tiles,
                                                  uint32_t next_bar, uint32_t next_parity, uint32_t tile_stride,
-                                                 uint32_t empty_bar, uint32_t a_empty_bar) {
+                                                 uint32_t empty_bar, uint32_t a_empty_bar, uint32_t acc_full_bar) {
     uint32_t ready;
     if (two_tiles) {
         if (PAIR) OC_MMA_STAGE_ASM("2", OC_KEEP, OC_COMMIT_CG2); else OC_MMA_STAGE_ASM("1", OC_KEEP, OC_COMMIT_CG1);
