@@ -37,7 +37,8 @@ FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1
 
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES = {"sd3_token": 25325568}     # profiles/match_tc_sd3_token.md
+# (profiles/step_kernels_<workload>.md: the row kernel's DRAM read + write of one cold launch)
+NCU_TRAFFIC_BYTES = {"svd_token_l0": 179428096, "sd3_token": 25328384, "svd_token_l1": 76260352, "svd_token_l2": 37098752, "svd_frame": 150800128, "latte_block": 9459456, "tiny_token": 106752}
 
 
 def measured_peaks():

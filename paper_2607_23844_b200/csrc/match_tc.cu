@@ -6,17 +6,25 @@
 // 4-D TMA tensor map {C, W/sx, H/sy, B*T}, so a box {64 channels, bw, bh, 1} lands in shared memory
 // as a canonical K-major, 128-byte-swizzled tile.  No operand is gathered or copied beforehand.
 //
-// What bounds it.  Measured on B200 (in-kernel timestamps and a copy-only micro-benchmark):
-//   * a TMA box costs the issuing warp ~50-100 cycles whatever its size, and the L2 -> shared-memory
-//     path delivers ~80 B/clk/SM to all SMs at once, with ~2000 cycles from issue to "stage full" for
-//     a 56 KB stage under load.  With 224 KB of ring the loop is therefore bound by bytes in flight
-//     (Little's law) unless a stage carries enough MMA work: the tile is chosen for FLOP per fetched
-//     byte, and a stage is fetched with as few boxes as possible;
-//   * the tensor pipe accepts an MMA only about when the previous one starts, so whatever the issuing
-//     warp does between two stages (finding out that the next stage is full takes ~150 cycles) is
-//     time the pipe idles, unless it is folded in between the MMAs of a stage;
-//   * a lone warp pays several hundred cycles per integer division and per first touch of code or
-//     parameters, which is what the first piece of a CTA costs before its first copy is issued.
+// What bounds it.  Measured on B200 (in-kernel timestamps, timing-only builds with the copies or the
+// epilogue's arithmetic left out, and micro-benchmarks of the copy ring, the MMA issue and the key
+// arithmetic):
+//   * the L2 -> shared-memory path delivers ~70-80 B/clk/SM to all SMs at once, some 500-800 cycles
+//     after the copy is issued; an MMA of 128 x 256 x 16 takes ~140 cycles;
+//   * shared memory serves the copies' writes AND the MMAs' operand reads: one tile of 128 rows against
+//     256 columns reads 12 KB per MMA and is sent 8 KB, which is more than 128 B/clk -- a single CTA's
+//     stage then takes ~700 cycles for 560 of MMA.  In a CTA pair each CTA reads and is sent half of the
+//     representatives, and the tensor pipe is the bound again;
+//   * the tensor pipe runs dry while the issuing warp is between two stages or two pieces unless that
+//     warp is back within about one MMA's time: the look at the next stage's barrier and all commits
+//     of a stage sit inside the block that issues its MMAs, and descriptors are kept by additions;
+//   * a lone warp runs dependent integer arithmetic at full latency (~6 cycles an instruction) and pays
+//     for every branch; a lone diverged LANE also has its operands moved into uniform registers before
+//     every copy or MMA.  So the producer and the MMA issuer run their loops with the whole warp and
+//     elect the lane that issues, and the epilogue's per-piece index arithmetic is branch-free, done
+//     ahead of time and only for what changed;
+//   * the arg-max epilogue is bound by the ALU and FMA pipes (two warps per scheduler): per element
+//     half a packed FMA, one integer multiply-add and half a three-input maximum.
 //
 // Tile.  One CTA multiplies ONE or TWO 128-row candidate tiles by the same N <= 256 representatives.
 // Two tiles (M = 256 per CTA, 128 FLOP/B at N = 256) use all 512 TMEM columns as two accumulators;
@@ -43,16 +51,21 @@
 //
 // Warp specialised:
 //   warp 0 (and, for one-tile plans, the last warp, taking turns with it stage by stage)
-//               TMA producer   (one lane per box; a CTA's candidate tiles are one box, and so are its
-//               quanta of a piece, whenever they stack into a rectangle of lattice rows): global ->
-//               smem ring (as many stages as fit in 224 KB), mbarrier complete_tx
+//               TMA producer: global -> smem ring (as many stages as fit), mbarrier complete_tx.  A
+//               CTA's candidate tiles are one box, and so are its quanta of a piece, whenever they
+//               stack into a rectangle of lattice rows: the whole warp then walks the loop and one
+//               elected lane issues; otherwise one lane per box.  With "resident" candidate tiles
+//               (plans whose rows have several pieces and few channels) all 64-channel steps of a row's
+//               tiles sit in front of the ring and are fetched once per row.
 //   warp 1      MMA issuer     (all lanes walk the loop so that addresses stay warp-uniform, one
 //               elected lane issues): tcgen05.mma kind::f16 (bf16 x bf16 -> fp32 in TMEM), all MMAs
-//               of a stage in one instruction block with the look at the next stage's barrier
-//               folded in; owns tcgen05.alloc / dealloc
-//   warps 2..9  epilogue: thread r of warps 2..5 / 6..9 owns row r (= TMEM lane r) of the candidate
-//               tiles for the first / second half of the piece's columns: tcgen05.ld 32 columns at a
-//               time (double buffered), scale by the representative's inverse norm, and a running
+//               of a stage in one instruction block with the look at the next stage's barrier and
+//               the stage's commits folded in; owns tcgen05.alloc / dealloc
+//   warps 2..9  epilogue, two halves of four warps (one warp per TMEM lane quarter, thread r owns row
+//               r of the candidate tiles).  With two accumulator sets the halves take alternate
+//               pieces; with one set of two tiles one tile each; with one set of one tile half of
+//               the columns each.  tcgen05.ld 32 columns at a time (double buffered), scale by the
+//               representative's inverse norm, and a running
 //               maximum over integer keys: the scaled similarity, lifted into one binade (where a
 //               float's bits are linear in its value), times 32, plus 31 - column (one three-input max
 //               per three keys, no compare-and-select per element, no cross-thread reduction; the
@@ -61,9 +74,10 @@
 //               value, then lowest index: independent of arrival order, hence deterministic).
 //               The lift rounds the reported cosine by at most 2.4e-7, and among representatives
 //               whose similarities agree to that precision the lowest index wins.  The epilogue warps
-//               never wait for one another: each keeps the column scales of its own chunks.
-// Rows / columns of a box that fall outside the patch are masked in the epilogue (a NaN scale never
-// wins a max), so ragged lattices need no padding.  Every mbarrier wait is bounded: on expiry the CTA
+//               never wait for one another: each keeps the column scales of its own chunks, fetched
+//               while the piece before is reduced.
+// Rows / columns of a box that fall outside the patch are masked in the epilogue (their scale is NaN
+// and their key is zeroed), so ragged lattices need no padding.  Every mbarrier wait is bounded: on expiry the CTA
 // records OC_ERR_TIMEOUT in the context's status word, lets its outstanding copies land, frees TMEM
 // and exits.
 #include <cuda.h>
@@ -287,24 +301,6 @@ __device__ __forceinline__ void fma_pair(float& d0, float& d1, uint32_t a0, uint
     asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
 }
 
-#ifdef OC_TC_TRACE
-// scratch instrumentation (experiment builds only): SM cycle counter at a few points of every piece of one CTA
-__device__ unsigned long long g_tc_trace[4][128][4];
-__device__ unsigned long long g_tc_stage[8][512];
-#define OC_TS(k, n, who) do { if (blockIdx.x == OC_TC_TRACE && (who) && (n) < 512) g_tc_stage[k][n] = clock64(); } while (0)
-#define OC_TR(role, piece, k, who)                                                                                  \
-    do { if (blockIdx.x == OC_TC_TRACE && (who) && (piece) < 128) g_tc_trace[role][piece][k] = clock64(); } while (0)
-#else
-#define OC_TR(role, piece, k, who)
-#define OC_TS(k, n, who)
-#endif
-#ifdef OC_TC_TRACE
-#define OC_ACC_BEGIN(v) const unsigned long long v##_t0 = clock64()
-#define OC_ACC_END(v) v += clock64() - v##_t0
-#else
-#define OC_ACC_BEGIN(v)
-#define OC_ACC_END(v)
-#endif
 
 static constexpr int COL_BYTES = EPI_WARPS * 256 * 4;                   // per epilogue warp: the scales of its (at most 256) columns
 static constexpr int N_BARS = 2 * MAX_STAGES + 5 + MAX_AKB;             // full[], empty[], acc_full[2], acc_empty[2], drain, a_empty[]
@@ -432,9 +428,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         const uint32_t ring_base = tiles_base + (uint32_t)P.a_region_bytes;       // (a_region_bytes is 0 unless a_res)
         const bool solo = P.a_merged && P.q_merged;
         const uint32_t issue = elect_one();
-#ifdef OC_TC_TRACE
-        unsigned long long acc_pw = 0, acc_pt = 0, acc_pe = 0, acc_pp = 0; const unsigned long long acc_p0 = clock64();
-#endif
         const uint32_t a_step = P.a_res ? (uint32_t)(P.tpp * A_BYTES) : 0u;     // resident slot pitch
         const uint32_t q_off = (uint32_t)(P.a_res ? 0 : P.tpp * A_BYTES);       // quanta inside a ring stage
         int trp = -1;
@@ -448,7 +441,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             // what the leader's barrier expects per stage: the copies of both CTAs
             const uint32_t bytes = (uint32_t)((PAIR ? 2 : 1) * ((load_a ? P.tpp * A_BYTES : 0) + nq_mine * Q_BYTES));
             if (solo) {
-                OC_ACC_BEGIN(acc_pp);
                 // (tiles past the lattice are fetched as zeros and masked in the epilogue)
                 const int ta = (PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp;
                 const int htA = (int)div_small((unsigned)ta, (unsigned)P.n_wtA, P.rcp_n_wtA), wtA = ta - htA * P.n_wtA;
@@ -458,40 +450,26 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 const int wQ = c.px * P.Ws + wq * bwQ, hQ = c.py * P.Hs + hq * P.bhQ;
                 const CUtensorMap* mapA = &KP.mapsA[c.member];
                 const CUtensorMap* mapQ = &KP.mapQ[nq_mine != P.q_lo ? 1 : 0];
-                OC_ACC_END(acc_pp);
                 for (int kb = 0; kb < P.kblocks; ++kb, ++gstage) {
                     // (the whole warp runs this; the elected lane issues)
                     if (ok && (P.n_prod < 2 || (gstage & 1u) == my_turn)) {
                         const uint32_t full_local = bar_full + 8 * stage;
                         const uint32_t full = PAIR ? map_to_cta(full_local, 0) : full_local;
-                        OC_ACC_BEGIN(acc_pw);
-                        OC_TS(2, gstage, lane == 0);
                         bool go = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag);
-                        OC_TS(7, gstage, lane == 0);
-                        OC_ACC_END(acc_pw);
                         // the slot of this step is free once the MMAs of the previous row's last piece have read it
                         if (go && P.a_res && load_a) go = mbar_wait(bar_a_empty + 8 * kb, a_phase ^ 1u, abort_flag);
                         if (__all_sync(0xFFFFFFFFu, go)) {
                             // the copies first, the arrival that carries their byte count after them: the barrier
                             // cannot complete before that arrival, and the copies are on their way sooner
-                            OC_ACC_BEGIN(acc_pt);
-#ifndef OC_EXP_NOTMA
                             tma_load_4d_elected<PAIR>(ring_base + stage * STAGE_BYTES + q_off, mapQ, kb * BK, wQ, hQ, c.bt, full, issue);
                             if (load_a)
                                 tma_load_4d_elected<PAIR>(P.a_res ? tiles_base + (uint32_t)kb * a_step : ring_base + stage * STAGE_BYTES,
                                                           mapA, kb * BK, wA, hA, c.bt_a, full, issue);
-#endif
-                            OC_ACC_END(acc_pt);
-                            OC_ACC_BEGIN(acc_pe);
                             if (leader) mbar_arrive_expect_tx_elected(full_local, bytes, issue);
-                            OC_TS(3, gstage, lane == 0);
-                            OC_ACC_END(acc_pe);
                         } else {
                             ok = false;
                         }
                     }
-                    if (kb == 0) OC_TR(0, trp, 0, lane == 0);
-                    if (kb == P.kblocks - 1) OC_TR(0, trp, 1, lane == 0);
                     armed |= 1u << stage;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     if (!joined) { __syncwarp(); __syncthreads(); joined = true; }   // first stage on its way: meet the others
@@ -529,8 +507,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     }
                     go = __shfl_sync(0xFFFFFFFFu, (int)go, 0) != 0;
                     if (!go) { ok = false; break; }
-                    if (kb == 0) OC_TR(0, trp, 0, lane == 0);
-                    if (kb == P.kblocks - 1) OC_TR(0, trp, 1, lane == 0);
                     if (active) {
                         const uint32_t dst = (lane < nA && P.a_res) ? tiles_base + (uint32_t)kb * a_step + dst_off
                                                                     : ring_base + stage * STAGE_BYTES + dst_off;
@@ -544,9 +520,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             if (P.a_res && load_a) a_phase ^= 1u;
         }
         if (!joined) { __syncthreads(); joined = true; }
-#ifdef OC_TC_TRACE
-        if (blockIdx.x == OC_TC_TRACE && lane == 0 && warp == 0) { g_tc_stage[0][0] = acc_pw; g_tc_stage[0][1] = clock64() - acc_p0; g_tc_stage[0][2] = trp + 1; g_tc_stage[0][3] = acc_pt; g_tc_stage[0][4] = acc_pe; g_tc_stage[0][5] = acc_pp; }
-#endif
         if (!ok && lane == 0) {
             atomicCAS(P.status, 0, OC_ERR_TIMEOUT);
             *abort_flag = 1;
@@ -581,9 +554,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             const uint32_t a_slot16 = (uint32_t)(P.tpp * A_BYTES) >> 4, q_off16 = a_res ? 0u : a_slot16;
             bool ok = true, peeked = false;
             uint32_t it = 0;
-#ifdef OC_TC_TRACE
-            unsigned long long acc_mf = 0, acc_ma = 0, acc_mi = 0; const unsigned long long acc_m0 = clock64(); unsigned mstage = 0;
-#endif
             // (the commit that hands the accumulators to the epilogue is part of the last stage's block; taking
             //  the walk to the next piece between two stages instead of between two pieces measured slower)
             while (ok && walk.next(P, c)) {
@@ -591,11 +561,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 // epilogue of a piece runs under the MMAs of the next one
                 const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
                 ++it;
-                OC_TR(1, (int)it - 1, 0, lane == 0);
-                OC_ACC_BEGIN(acc_ma);
                 if (!__all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_empty + 8 * buf, acc_phase ^ 1u, abort_flag))) { ok = false; break; }
-                OC_ACC_END(acc_ma);
-                OC_TR(1, (int)it - 1, 1, lane == 0);
                 const uint32_t d_tmem = tmem_base + buf * 256u;
                 tc_fence_after();
                 const uint32_t idesc = IDESC_BASE | ((uint32_t)(c.ncol >> 3) << 17);
@@ -610,16 +576,10 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 for (int kb = 0; kb < kblocks; ++kb) {
                     // (each lane looked for itself; the barrier's phase cannot go back, so a lane that saw it
                     //  full stays right, and the others wait here)
-                    OC_ACC_BEGIN(acc_mf);
-                    OC_TS(4, mstage, lane == 0);
                     if (!peeked) {
                         if (!mbar_wait(bar_full + 8 * stage, phase, abort_flag)) ok = false;
                         if (!__all_sync(0xFFFFFFFFu, ok)) { ok = false; break; }
                     }
-                    OC_TS(5, mstage, lane == 0);
-                    OC_ACC_END(acc_mf);
-                    OC_ACC_BEGIN(acc_mi);
-                    if (kb == 0) OC_TR(1, (int)it - 1, 2, lane == 0);
                     const uint32_t s_lo = ring_lo + (uint32_t)stage * stage16;
                     const uint32_t a_lo = a_res ? res_lo + (uint32_t)kb * a_slot16 : s_lo;
                     // (a piece that begins in mid-quantum skips 16 rows = 2 KB of its first box: a whole number
@@ -634,18 +594,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                                                 (uint32_t)(kb != 0), issue, two_tiles, bar_full + 8 * nstage, nphase, tile_stride,
                                                 bar_empty + 8 * stage, free_a ? bar_a_empty + 8 * kb : 0u,
                                                 kb + 1 == kblocks ? bar_acc_full + 8 * buf : 0u) != 0;
-                    OC_ACC_END(acc_mi);
-                    OC_TS(6, mstage, lane == 0);
-#ifdef OC_TC_TRACE
-                    ++mstage;
-#endif
                     stage = nstage; phase = nphase;
                 }
-                OC_TR(1, (int)it - 1, 3, lane == 0);
             }
-#ifdef OC_TC_TRACE
-            if (blockIdx.x == OC_TC_TRACE && lane == 0) { g_tc_stage[1][0] = acc_mf; g_tc_stage[1][1] = acc_ma; g_tc_stage[1][2] = acc_mi; g_tc_stage[1][3] = clock64() - acc_m0; g_tc_stage[1][4] = it; }
-#endif
             if (!ok && lane == 0) { atomicCAS(P.status, 0, OC_ERR_TIMEOUT); *abort_flag = 1; }
             // all MMAs issued by this warp must retire before TMEM is released
             tc_commit<PAIR>(PAIR ? map_to_cta(bar_drain, 0) : bar_drain, issue);
@@ -788,23 +739,17 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
             const float4* col_scale4 = (const float4*)my_scale;
             const float* col_scale1 = my_scale;
-            OC_TR(3, (int)it, 0, et == 0);
             const bool have_nx = next_mine(nx, it_nx, new_row);
-            OC_TR(3, (int)it, 1, et == 0);
             if (have_nx) {                                             // in flight until the end of this piece
                 gather_cols(nx, cols_ahead);
                 if (new_row) gather_rows(nx, rows_ahead);
             }
-            OC_TR(3, (int)it, 2, et == 0);
             const int my = cur.my, mx = cur.mx;
             const float lift0 = cur.lift[0], lift1 = cur.lift[1];
             const int ch_begin = cols.ch_begin, ch_end = cols.ch_end;
-            OC_TR(3, (int)it, 3, et == 0);
 
             // warp-uniform outcome: the TMEM loads below are warp-collective
-            OC_TR(2, (int)it, 0, et == 0);
             const bool ready = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * buf, acc_phase, abort_flag));
-            OC_TR(2, (int)it, 1, et == 0);
             if (ready) {
                 tc_fence_after();
                 uint32_t won_key0 = 0, won_key1 = 0;                   // per tile: the row's largest key and its chunk
@@ -875,15 +820,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             }                                                                                                    \
         }                                                                                                        \
     } while (0)
-#ifndef OC_EXP_NOEPI
                     if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
-#endif
 #pragma unroll 1
-#ifdef OC_EXP_NOEPI
-                    for (int ch = ch_begin; ch < ch_begin; ch += 2) {
-#else
                     for (int ch = ch_begin; ch < ch_end; ch += 2) {
-#endif
                         tmem_ld_wait();
                         if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);
                         OC_REDUCE_CHUNK(va, ch);
@@ -898,7 +837,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 }
                 tc_fence_before();
                 __syncwarp();
-                OC_TR(2, (int)it, 2, et == 0);
                 if (lane == 0) {                                       // both accumulators may be overwritten
                     if (PAIR) mbar_arrive_cluster(acc_empty + 8 * buf); else mbar_arrive(bar_acc_empty + 8 * buf);
                 }
@@ -930,7 +868,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 cols.ch_begin = cols_ahead.ch_begin; cols.ch_end = cols_ahead.ch_end;
                 if (new_row) { cur = rows_ahead; set_lifts(cur); }
             }
-            OC_TR(2, (int)it, 3, et == 0);
             c = nx; have = have_nx;
             it = it_nx;
         }
@@ -1327,11 +1264,3 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
 
 }  // namespace oc
 
-#ifdef OC_TC_TRACE
-extern "C" int oc_debug_tc_trace_read(unsigned long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, oc::g_tc_trace, sizeof(oc::g_tc_trace));
-}
-extern "C" int oc_debug_tc_stage_read(unsigned long long* out) {
-    return (int)cudaMemcpyFromSymbol(out, oc::g_tc_stage, sizeof(oc::g_tc_stage));
-}
-#endif
