@@ -21,8 +21,8 @@
 //   * a lone warp runs dependent integer arithmetic at full latency (~6 cycles an instruction) and pays
 //     for every branch; a lone diverged LANE also has its operands moved into uniform registers before
 //     every copy or MMA.  So the producer and the MMA issuer run their loops with the whole warp and
-//     elect the lane that issues, and the epilogue's per-piece index arithmetic is branch-free, done
-//     ahead of time and only for what changed;
+//     elect the lane that issues, and the epilogue does index arithmetic per group and per row, not
+//     per piece, branch-free and ahead of time;
 //   * the arg-max epilogue is bound by the ALU and FMA pipes (two warps per scheduler): per element
 //     half a packed FMA, one integer multiply-add and half a three-input maximum.
 //
@@ -74,8 +74,10 @@
 //               value, then lowest index: independent of arrival order, hence deterministic).
 //               The lift rounds the reported cosine by at most 2.4e-7, and among representatives
 //               whose similarities agree to that precision the lowest index wins.  The epilogue warps
-//               never wait for one another: each keeps the column scales of its own chunks, fetched
-//               while the piece before is reduced.
+//               never wait for one another from piece to piece: each half keeps the column scales of
+//               the whole group in shared memory (rebuilt, behind a barrier over the half's four warps,
+//               only when its pieces move to another group), and a row's own norms are fetched while
+//               the piece before is reduced.
 // Rows / columns of a box that fall outside the patch are masked in the epilogue (their scale is NaN
 // and their key is zeroed), so ragged lattices need no padding.  Every mbarrier wait is bounded: on expiry the CTA
 // records OC_ERR_TIMEOUT in the context's status word, lets its outstanding copies land, frees TMEM
@@ -145,6 +147,8 @@ struct TcScalars {
     int n_prod;                          // copy-producer warps at work: 1, or 2 taking turns stage by stage
     unsigned key_mul;                    // 32, as a run-time value: keeps half of the key multiplies on the FMA pipe
     int epi_split;                       // how the two halves of the epilogue warps share the work (EPI_BY_*)
+    int gt_off, gt_half_bytes, gt_quanta; // the group's column-scale tables (one per half of the epilogue warps):
+                                         // byte offset in shared memory, size of one, quanta per group
     int a_res, a_region_bytes;           // candidate tiles resident: all 64-channel steps of a CTA's candidate tiles
                                          // sit in front of the ring (one slot per step) for all pieces of a row, and
                                          // the ring carries representatives only
@@ -302,9 +306,9 @@ __device__ __forceinline__ void fma_pair(float& d0, float& d1, uint32_t a0, uint
 }
 
 
-static constexpr int COL_BYTES = EPI_WARPS * 256 * 4;                   // per epilogue warp: the scales of its (at most 256) columns
+static constexpr int GT_MAX_QUANTA = 150;                               // largest group whose scale tables fit beside the ring
 static constexpr int N_BARS = 2 * MAX_STAGES + 5 + MAX_AKB;             // full[], empty[], acc_full[2], acc_empty[2], drain, a_empty[]
-static constexpr int TAIL_BYTES = COL_BYTES + N_BARS * 8 + 32 + EPI_WARPS * 32;   // column tables, barriers, TMEM slot, flags, masks
+static constexpr int TAIL_BYTES = N_BARS * 8 + 32;                      // barriers, TMEM slot, flags
 static constexpr int TILE_BYTES = (SMEM_LIMIT - TAIL_BYTES) / 1024 * 1024;   // operand ring: everything else
 static constexpr int SMEM_TOTAL = TILE_BYTES + TAIL_BYTES;
 
@@ -322,15 +326,13 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     // for the 128-byte swizzle (this kernel has no static shared memory in front of it; checked below).
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = smem_raw;
-    float4* colsb = (float4*)(smem + TILE_BYTES);                      // per column: scale[256], then token[256]
-    uint64_t* bars = (uint64_t*)(smem + TILE_BYTES + COL_BYTES);
+    uint64_t* bars = (uint64_t*)(smem + TILE_BYTES);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * MAX_STAGES;
     const uint32_t bar_acc_full = bar_empty + 8 * MAX_STAGES, bar_acc_empty = bar_acc_full + 16;   // two of each
     const uint32_t bar_drain = bar_acc_empty + 16;
     const uint32_t bar_a_empty = bar_drain + 8;                        // resident candidate slots, one per 64-channel step
     uint32_t* tmem_slot = (uint32_t*)(bars + N_BARS);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
-    uint32_t* col_masked = tmem_slot + 8;                              // [warp][8]: per 32-column chunk, its columns that are no representative
     const uint32_t tiles_base = smem_u32(smem);
     const TcScalars& P = KP.s;
     if (P.span && threadIdx.x == 0) atomicMax(P.span, ~global_ns());
@@ -612,16 +614,15 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         bool ok = true;
         uint32_t it = 0;
         const uint32_t acc_empty = PAIR ? map_to_cta(bar_acc_empty, 0) : bar_acc_empty;   // the leader's
-        // Per column of a piece: the representative's inverse norm (NaN where the column is not a
-        // representative of this patch; each chunk of 32 columns also has a bit mask of those, and
-        // their keys are zeroed).  Every epilogue warp keeps a table of its OWN columns -- at most eight
-        // chunks of 32 -- so the warps never wait for one another: a piece costs a warp its reduction
-        // and nothing else.  What its NEXT piece needs (the table entries, eight per lane; each row's own
-        // norm) is fetched before this piece's accumulators are waited for and used after, so that
-        // global-memory latency is never waited for either.
+        // Per representative slot of the GROUP (quantum by quantum, 32 lattice points each): the
+        // representative's inverse norm, NaN where the slot is no representative of this patch, and per
+        // quantum a bit mask of those slots (their keys are zeroed).  Each half of the epilogue warps
+        // keeps its own table and rebuilds it when its pieces move on to another group (a barrier over
+        // the half's four warps on either side: rare); a piece then costs a warp no table work at all,
+        // its columns are a window into the table.
         const int ew = et >> 5;                                        // this warp among the epilogue warps
-        float* my_scale = (float*)colsb + ew * 256;
-        uint32_t* my_masked = col_masked + ew * 8;
+        float* gt_scale = (float*)(smem + P.gt_off + part * P.gt_half_bytes);
+        uint32_t* gt_mask = (uint32_t*)(gt_scale + P.gt_quanta * QN);  // [gt_quanta + 1]
         const int split = P.epi_split;
         const int t_begin = split == EPI_BY_TILE ? part : 0, t_end = split == EPI_BY_TILE ? part + 1 : P.tpp;
         const uint32_t key_mul = P.key_mul;
@@ -629,12 +630,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         // What a warp needs of a piece, gathered ahead of time.  A lone warp runs dependent integer
         // arithmetic at its full latency and pays for every branch, and this is on the one path that
         // bounds the kernel, so: no branches (selects and a clamped address instead), one division per
-        // piece (the lane's eight columns lie in eight consecutive quanta), and the row part only when
-        // the row changes (the pieces of a row share their candidate tiles).
-        struct Cols {
-            int ch_begin, ch_end;            // this warp's chunks of 32 columns
-            float sc[8];                     // lane's table entries: column (ch_begin + i) * 32 + lane
-        };
+        // lookup, and that only when the row changes (the pieces of a row share their candidate tiles).
         struct Rows {
             int tokA[2];                     // the rows (candidate tokens) this thread owns in the piece's tiles
             bool row_ok[2];
@@ -651,32 +647,25 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         };
         const float quiet_nan = __int_as_float(0x7FC00000);
         const int tok_per_lattice_row = P.sy * P.W;
-        auto gather_cols = [&](const Piece& pc, Cols& a) {
-            // chunks of 32 columns: all of them, or the first half to warps 2..5 and the rest to warps 6..9
-            const int n_ch = (pc.ncol + 31) >> 5;                       // (a last half chunk reads 16 columns of
-            a.ch_begin = 0; a.ch_end = n_ch;                            //  nothing: their table entries are NaN)
-            if (split == EPI_BY_COLUMNS) {
-                a.ch_begin = (part * n_ch + EPI_PARTS - 1) / EPI_PARTS;
-                a.ch_end = ((part + 1) * n_ch + EPI_PARTS - 1) / EPI_PARTS;
-            }
-            const int g0 = pc.c_off + lane;                             // the lane's column, counted from the piece's first quantum
-            const int r = g0 & 31, rh = r >> P.bwQ_log2, rw = r & (bwQ - 1);
-            const int qi = pc.q0 + (g0 >> 5) + a.ch_begin;
-            int hq = div_fast(qi, P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;
-            // token of the patch's lattice point (0, 0) of the representatives' member
+        // The group's table: warp w of the half fills quanta w, w + 4, ...  Every warp of the half comes
+        // here at the same piece (they take the same pieces), also one that has given up: it must not
+        // leave the others waiting at the barriers.
+        int table_bt = -1, table_py = -1, table_px = -1;
+        auto rebuild_table = [&](const Piece& pc) {
+            asm volatile("bar.sync %0, 128;" :: "r"(1 + part) : "memory");     // the old table is no longer read
             const int tok0 = (pc.bt * P.H + pc.py * P.Hs * P.sy + my_rep) * P.W + pc.px * P.Ws * P.sx + mx_rep;
-            const int col0 = a.ch_begin * 32 + lane;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int hs = hq * P.bhQ + rh, ws = wq * bwQ + rw;
-                const bool valid = (a.ch_begin + i < a.ch_end) & (col0 + 32 * i < pc.ncol) & (hs < P.Hs) & (ws < P.Ws);
-                const int tok = valid ? tok0 + hs * tok_per_lattice_row + ws * P.sx : 0;
-                const float v = __ldg(P.inv_norm + tok);
-                a.sc[i] = valid ? v : quiet_nan;
-                ++wq;
-                const bool wrap = wq == P.n_wq;
-                wq = wrap ? 0 : wq; hq += wrap ? 1 : 0;
+            for (int q = ew & 3; q < P.gt_quanta; q += 4) {
+                const int hq = div_fast(q, P.n_wq, P.rcp_n_wq), wq = q - hq * P.n_wq;
+                const int hs = hq * P.bhQ + (lane >> P.bwQ_log2), ws = wq * bwQ + (lane & (bwQ - 1));
+                const bool valid = (hs < P.Hs) & (ws < P.Ws);
+                const float v = __ldg(P.inv_norm + (valid ? tok0 + hs * tok_per_lattice_row + ws * P.sx : 0));
+                gt_scale[q * QN + lane] = valid ? v : quiet_nan;
+                const uint32_t masked = __ballot_sync(0xFFFFFFFFu, !valid);
+                if (lane == 0) gt_mask[q] = masked;
             }
+            if ((ew & 3) == 0 && lane == 0) gt_mask[P.gt_quanta] = 0xFFFFFFFFu;     // (read with the last quantum's word)
+            asm volatile("bar.sync %0, 128;" :: "r"(1 + part) : "memory");
+            table_bt = pc.bt; table_py = pc.py; table_px = pc.px;
         };
         auto gather_rows = [&](const Piece& pc, Rows& a) {
             a.my = (pc.member * P.sx_magic) >> 16; a.mx = pc.member - a.my * P.sx;
@@ -702,23 +691,11 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 a.lift[t] = 3.0f * __uint_as_float((__float_as_uint(bound) + 0x007FFFFFu) & 0x7F800000u);
             }
         };
-        // the warp's table: written only when every lane is done with the one before
-        auto publish = [&](const Cols& a) {
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                my_scale[i * 32 + lane] = a.sc[i];
-                const uint32_t masked = __ballot_sync(0xFFFFFFFFu, a.sc[i] != a.sc[i]);
-                if (lane == 0) my_masked[i] = masked;
-            }
-            __syncwarp();
-        };
         // Only from here on does this kernel touch what the norm pre-pass (the kernel before it in the
         // stream) writes: its operand copies and MMAs may run while that kernel still does.
         pdl_wait();
         if (et == 0) pdl_launch_dependents();
         Piece nx;
-        Cols cols, cols_ahead;
         Rows cur, rows_ahead;
         // this warp's next piece: every piece, or (EPI_BY_PIECE) every other one
         uint32_t handed = 0;                                           // pieces the walk has handed out
@@ -734,22 +711,31 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         uint32_t it_nx = 0;
         bool new_row = false;
         bool have = next_mine(c, it, new_row);
-        if (have) { gather_cols(c, cols); gather_rows(c, cur); publish(cols); set_lifts(cur); }
+        if (have) { gather_rows(c, cur); set_lifts(cur); }
         while (have) {
             const uint32_t buf = dbl ? (it & 1u) : 0u, acc_phase = dbl ? ((it >> 1) & 1u) : (it & 1u);
-            const float4* col_scale4 = (const float4*)my_scale;
-            const float* col_scale1 = my_scale;
             const bool have_nx = next_mine(nx, it_nx, new_row);
-            if (have_nx) {                                             // in flight until the end of this piece
-                gather_cols(nx, cols_ahead);
-                if (new_row) gather_rows(nx, rows_ahead);
-            }
+            if (have_nx && new_row) gather_rows(nx, rows_ahead);       // in flight until the end of this piece
+            if ((c.bt != table_bt) | (c.py != table_py) | (c.px != table_px)) rebuild_table(c);
             const int my = cur.my, mx = cur.mx;
             const float lift0 = cur.lift[0], lift1 = cur.lift[1];
-            const int ch_begin = cols.ch_begin, ch_end = cols.ch_end;
+            // chunks of 32 columns: all of them, or the first half to warps 2..5 and the rest to warps 6..9
+            // (a last half chunk reads 16 columns of nothing: they are masked)
+            const int n_ch = (c.ncol + 31) >> 5;
+            const int ch_begin = split == EPI_BY_COLUMNS ? (part * n_ch + EPI_PARTS - 1) / EPI_PARTS : 0;
+            const int ch_end = split == EPI_BY_COLUMNS ? ((part + 1) * n_ch + EPI_PARTS - 1) / EPI_PARTS : n_ch;
+            // the piece's columns in the group's table (a piece may begin in mid-quantum)
+            const int col0 = c.q0 * QN + c.c_off;
+            const float* col_scale1 = gt_scale + col0;
+            const float4* col_scale4 = (const float4*)col_scale1;
+            // whether any column of the piece is masked: a slot outside the patch, or the tail of a last,
+            // partial chunk (one mask word per lane)
+            const int w_first = col0 >> 5, w_last = (col0 + c.ncol - 1) >> 5;
+            const bool piece_masked = (c.ncol & 31) != 0 ||
+                                      __any_sync(0xFFFFFFFFu, w_first + lane <= w_last && gt_mask[w_first + lane] != 0u);
 
             // warp-uniform outcome: the TMEM loads below are warp-collective
-            const bool ready = __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * buf, acc_phase, abort_flag));
+            const bool ready = ok && __all_sync(0xFFFFFFFFu, mbar_wait(bar_acc_full + 8 * buf, acc_phase, abort_flag));
             if (ready) {
                 tc_fence_after();
                 uint32_t won_key0 = 0, won_key1 = 0;                   // per tile: the row's largest key and its chunk
@@ -789,7 +775,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     do {                                                                                                         \
         uint32_t kf[32];                                                                                         \
         _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
-            const float4 s4 = col_scale4[((ch) - ch_begin) * 8 + (j >> 2)];                                      \
+            const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                                   \
             float x0, x1, x2, x3;                                                                                \
             fma_pair(x0, x1, v[j], v[j + 1], s4.x, s4.y, row_lift);                                              \
             fma_pair(x2, x3, v[j + 2], v[j + 3], s4.z, s4.w, row_lift);                                          \
@@ -798,8 +784,11 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             kf[j + 2] = __float_as_uint(x2) * 32u + (uint32_t)(29 - j);                                          \
             kf[j + 3] = __float_as_uint(x3) * key_mul + (uint32_t)(28 - j);                                      \
         }                                                                                                        \
-        const uint32_t masked = my_masked[(ch) - ch_begin];            /* warp-uniform, almost always zero */    \
-        if (masked) {                                                                                            \
+        if (piece_masked) {                                            /* warp-uniform, almost always false */   \
+            const int gcol = col0 + (ch) * 32, left = c.ncol - (ch) * 32;                                        \
+            uint32_t masked = gt_mask[gcol >> 5];                                                                \
+            if (gcol & 16) masked = (masked >> 16) | (gt_mask[(gcol >> 5) + 1] << 16);                           \
+            if (left < 32) masked |= 0xFFFFFFFFu << left;              /* columns of the next piece */          \
             _Pragma("unroll") for (int j = 0; j < 32; ++j)                                                       \
                 if ((masked >> j) & 1u) kf[j] = 0u;                                                              \
         }                                                                                                        \
@@ -809,8 +798,8 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         if (cm > (bm | 31u)) { bm = cm; bc = (ch); }                                                             \
         if (AUX && aux_row) {                                                                                    \
             for (int j = 0; j < 32; ++j) {                                                                       \
-                const float sc = col_scale1[((ch) - ch_begin) * 32 + j];                                         \
-                if (sc == sc) {                                                                                  \
+                const float sc = col_scale1[(ch) * 32 + j];                                                      \
+                if ((ch) * 32 + j < c.ncol && sc == sc) {                                                        \
                     const int gp_ = c.c_off + (ch) * 32 + j;                                                     \
                     const int qi = c.q0 + (gp_ >> 5), r = gp_ & 31;                                              \
                     const int hq = (int)div_small((unsigned)qi, (unsigned)P.n_wq, P.rcp_n_wq), wq = qi - hq * P.n_wq;                                           \
@@ -859,15 +848,14 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     const long long tokB = ((long long)c.bt * P.H + y) * P.W + x;
                     atomicMax(P.keys + (t ? cur.tokA[1] : cur.tokA[0]), pack_key(best, (uint32_t)tokB));
                 }
-            } else {
+            } else if (ok) {
                 ok = false;
+                atomicCAS(P.status, 0, OC_ERR_TIMEOUT);
+                *abort_flag = 1;                                       // the other roles give up at their next wait
             }
-            if (!ok) break;
-            if (have_nx) {
-                publish(cols_ahead);
-                cols.ch_begin = cols_ahead.ch_begin; cols.ch_end = cols_ahead.ch_end;
-                if (new_row) { cur = rows_ahead; set_lifts(cur); }
-            }
+            // (a warp that has given up still walks its remaining pieces, without waiting for anything: the
+            //  other warps of its half may be at a table's barriers, which want all four of them)
+            if (have_nx && new_row) { cur = rows_ahead; set_lifts(cur); }
             c = nx; have = have_nx;
             it = it_nx;
         }
@@ -942,8 +930,15 @@ struct TcPlan {
     int pair, q_unit, n_q_units, half_units, a_merged, q_merged, q_lo, q_hi, q_rows;
     int pieces_per_row, qmax, n_stages, stage_bytes, narrow;
     int a_res, a_region_bytes;
+    int gt_half_bytes;                   // one group table: a scale per representative slot and a mask word per quantum (+1)
     long long rows, items;
 };
+// quanta of 32 lattice points that cover one group's representatives
+static int group_quanta(const Geo& g) {
+    int lq = pow2_ceil_log2(g.Ws); if ((1 << lq) > QN) lq = pow2_ceil_log2(QN);
+    const int bhQ = QN >> lq;
+    return ((g.Ws + (1 << lq) - 1) >> lq) * ((g.Hs + bhQ - 1) / bhQ);
+}
 
 // A forced work split (oc_tc_plan_override): the tests run every form of the kernel this way.
 struct TcForce { bool on; int pair, tiles, pieces, no_narrow, a_res /* -1: the planner's choice */; };
@@ -959,6 +954,9 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
     p.bwQ_log2 = lq; p.bhQ = QN >> lq;
     p.n_wq = (g.Ws + (1 << lq) - 1) >> lq;
     p.n_quanta = p.n_wq * ((g.Hs + p.bhQ - 1) / p.bhQ);
+    // two tables (one per half of the epilogue warps) at the end of the operand region: the ring gets the rest
+    p.gt_half_bytes = (p.n_quanta * (QN * 4 + 4) + 4 + 15) / 16 * 16;
+    const int ring_cap = TILE_BYTES - 2 * p.gt_half_bytes;
     // Form (single CTA or CTA pair), candidate tiles per CTA (1 or 2), pieces per row and whether the
     // candidate tiles stay resident, by estimated cycles of the busiest walker.  The shape of the estimate
     // follows the kernel; its constants were fitted (least squares on the logarithm, over 40 timed plans)
@@ -1012,7 +1010,7 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
                 const double epi = overlapped ? 0.5 * epi_all : epi_all;   // per piece and warp
                 for (int ar = 1; ar >= 0; --ar) {                           // (equal estimates: fewer bytes fetched wins)
                     const double a_kb = tpp * 16.0, q_kb = 4.0 * q_load / ncta;
-                    if (ar && (kblocks > MAX_AKB || a_kb * kblocks + 3 * q_kb > TILE_BYTES / 1024 || P == 1)) continue;
+                    if (ar && (kblocks > MAX_AKB || a_kb * kblocks + 3 * q_kb > ring_cap / 1024 || P == 1)) continue;
                     const double sent_kb = (ar ? 0.0 : a_kb) + q_kb, read_kb = tpp * (16.0 + 4.0 * qe / ncta);
                     const double feed = sent_kb * 1024.0 / 80.7, smem = (sent_kb + read_kb) * 7.42;
                     double piece;
@@ -1071,11 +1069,11 @@ static TcPlan make_plan(const Geo& g, int walkers, int pair_walkers, const TcFor
     // row instead of once per piece): possible when they leave room for at least three ring stages of
     // representatives.
     const int a_region = p.tpp * A_BYTES * kblocks;
-    const bool a_res_ok = kblocks <= MAX_AKB && a_region + 3 * q_max * Q_BYTES <= TILE_BYTES && best_P > 1;
+    const bool a_res_ok = kblocks <= MAX_AKB && a_region + 3 * q_max * Q_BYTES <= ring_cap && best_P > 1;
     p.a_res = a_res_ok ? (force.on ? (force.a_res != 0) : (best_ar != 0)) : 0;
     p.a_region_bytes = p.a_res ? a_region : 0;
     p.stage_bytes = (p.a_res ? 0 : p.tpp * A_BYTES) + q_max * Q_BYTES;
-    p.n_stages = (TILE_BYTES - p.a_region_bytes) / p.stage_bytes;
+    p.n_stages = (ring_cap - p.a_region_bytes) / p.stage_bytes;
     if (p.n_stages > MAX_STAGES) p.n_stages = MAX_STAGES;
     p.items = p.rows * p.pieces_per_row;
     // One copy instruction costs the producer ~100 cycles whatever the box size, so a CTA's candidate
@@ -1094,6 +1092,7 @@ bool tc_match_supported(const Geo& g) {
     if (g.sy * g.sx > MAX_LATTICES) return false;
     if (g.C % 8 != 0) return false;
     if ((long long)g.B * g.T > 0x7FFFFFFFll) return false;
+    if (group_quanta(g) > GT_MAX_QUANTA) return false;           // the group's scale tables would not fit beside the ring
     return encode_fn() != nullptr;
 }
 
@@ -1222,6 +1221,7 @@ static oc_status launch_tc(oc_ctx* ctx, const Geo& g, const void* x, const float
     // stage cover one producer's work and the second warp only competes for issue slots
     P.n_prod = (N_PRODUCERS > 1 && p.tpp == 1) ? 2 : 1;
     P.key_mul = 32u;
+    P.gt_half_bytes = p.gt_half_bytes; P.gt_off = TILE_BYTES - 2 * p.gt_half_bytes; P.gt_quanta = p.n_quanta;
     P.epi_split = (p.tpp == 1 || p.narrow) ? EPI_BY_PIECE : (p.tpp == 2 ? EPI_BY_TILE : EPI_BY_COLUMNS);
     P.units_per_group = (int)g.units_per_group; P.reps_per_group = (int)g.reps_per_group;
     P.inv_norm = inv_norm; P.keys = keys; P.aux = aux_sim; P.status = ctx->d_status;
