@@ -24,15 +24,29 @@ def oc():
     return omnicache
 
 
-def expect_tensor_core(dtype, shape, lattice=(2, 2, 0, 0), self_match=False):
+def group_quanta(shape, groups=(1, 1), lattice=(2, 2, 0, 0)):
+    """Boxes of 32 lattice points (2^k wide, at most 32) that cover one group's representative lattice."""
+    sy, sx, oy, ox = lattice
+    hp, wp = shape[2] // groups[0], shape[3] // groups[1]
+    hs, ws = (hp - oy + sy - 1) // sy, (wp - ox + sx - 1) // sx
+    bw = 1
+    while bw < min(ws, 32):
+        bw *= 2
+    bh = 32 // bw
+    return -(-ws // bw) * -(-hs // bh)
+
+
+def expect_tensor_core(dtype, shape, lattice=(2, 2, 0, 0), self_match=False, groups=(1, 1)):
     """Whether oc_match must take the tcgen05 kernel for this Token Cache layout: bf16, no self-match, at most
-    nine lattice members, rows of whole 16-byte chunks.  Anything else belongs to the fp32-FMA kernel; a bf16
+    nine lattice members, rows of whole 16-byte chunks, a group whose column-scale tables fit beside the
+    operand ring (150 boxes of 32 representatives).  Anything else belongs to the fp32-FMA kernel; a bf16
     layout that falls back silently would pass every numeric check and run an order of magnitude slower."""
-    return dtype == inputs.BF16 and not self_match and lattice[0] * lattice[1] <= 9 and shape[-1] % 8 == 0
+    return (dtype == inputs.BF16 and not self_match and lattice[0] * lattice[1] <= 9 and shape[-1] % 8 == 0
+            and group_quanta(shape, groups, lattice) <= 150)
 
 
-def assert_matcher(rep, dtype, shape, lattice=(2, 2, 0, 0)):
-    want_tc = expect_tensor_core(dtype, shape, lattice)
+def assert_matcher(rep, dtype, shape, lattice=(2, 2, 0, 0), groups=(1, 1)):
+    want_tc = expect_tensor_core(dtype, shape, lattice, groups=groups)
     assert rep["launches"]["match_tc"] == (1 if want_tc else 0), rep["launches"]
     assert rep["launches"]["match_simt"] == (0 if want_tc else 1), rep["launches"]
 
@@ -177,7 +191,7 @@ def test_token_chain_small(oc, oracle, shape, groups, lattice, dtype):
     U = (Hh // groups[0]) * (W // groups[1])
     w.n_reuse = (U - U // (sy * sx)) // 2
     rep = run_chain(oc, oracle, w, want_aux=True, sy=sy, sx=sx, oy=oy, ox=ox)
-    assert_matcher(rep, dtype, shape, lattice)
+    assert_matcher(rep, dtype, shape, lattice, groups)
 
 
 def _random_token_layouts(n, seed):
@@ -209,7 +223,24 @@ def test_token_chain_random_layouts(oc, oracle, shape, groups, lattice):
     reps = ((Hh // groups[0]) // sy) * ((W // groups[1]) // sx)
     w.n_reuse = (U - reps) // 3
     rep = run_chain(oc, oracle, w, want_aux=True, sy=sy, sx=sx, oy=oy, ox=ox)
-    assert_matcher(rep, inputs.BF16, shape, lattice)
+    assert_matcher(rep, inputs.BF16, shape, lattice, groups)
+
+
+@pytest.mark.parametrize("shape,want_tc", [
+    ((1, 1, 128, 128, 64), True),      # 64 x 64 representatives: 128 boxes, the largest tables in use here
+    ((1, 1, 160, 128, 64), False),     # 80 x 64 representatives: 160 boxes, past the tables -> the FMA matcher
+])
+def test_token_group_tables_limit_and_fallback(oc, oracle, shape, want_tc):
+    """The tensor-core matcher keeps the inverse norms of a whole group's representatives in shared memory;
+    groups too large for that must fall back to the FMA matcher, not fail and not compute garbage."""
+    B, T, Hh, W, C = shape
+    assert expect_tensor_core(inputs.BF16, shape) == want_tc
+    w = inputs.sd3_token_cache(seed=33, B=B * T, H=Hh, W=W, C=C, groups=(1, 1), dtype=inputs.BF16)
+    w.x = w.x.reshape(shape); w.shape = shape
+    U = Hh * W
+    w.n_reuse = (U - U // 4) // 2
+    rep = run_chain(oc, oracle, w, full_oracle=False, sample_rows=400)
+    assert_matcher(rep, inputs.BF16, shape)
 
 
 @pytest.mark.parametrize("plan", ["0,1,2", "0,2,3", "1,1,1", "1,2,2", "0,2,3,1", "1,1,2,1", "0,1,4,1"])
