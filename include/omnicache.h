@@ -169,6 +169,16 @@ oc_status oc_device_status(oc_ctx* ctx, int* code);
  * afterwards oc_device_status() reports OC_ERR_TIMEOUT once, and the context works as before. */
 oc_status oc_selftest_bounded_wait(oc_ctx* ctx, unsigned int limit_us, void* stream);
 
+/* Self-test of the once-per-device bookkeeping (host only: no CUDA call, no device needed).  Kernel
+ * attributes such as the opt-in to large dynamic shared memory belong to a device, and one process may
+ * use the library on several; the launchers therefore run their set-up once per DEVICE.  This call
+ * drives a fresh instance of that bookkeeping: for round = 0 .. n_rounds-1 and dev = 0 .. n_devices-1
+ * it asks for the set-up of `dev`, with a set-up routine that counts its runs per device and fails on
+ * device fail_dev (-1: never).  runs[dev] receives how often the routine ran (1 for every device, also
+ * the failing one: a failure is remembered, not retried), ok[dev] how often the request succeeded
+ * (n_rounds, or 0 for fail_dev).  Both arrays are host memory of n_devices ints (1 .. 64 devices). */
+oc_status oc_selftest_per_device_once(int n_devices, int n_rounds, int fail_dev, int* runs, int* ok);
+
 /* Launch counters and optional per-kernel timers.  Counters always run.  oc_profile_enable takes
  * 0 (timers off), 1 (each kernel launch is bracketed by CUDA events on the caller's stream) or 2
  * (device-side spans of the tensor-core matcher, see oc_profile_span_read; no events).

@@ -262,6 +262,16 @@ oc_status oc_device_status(oc_ctx* c, int* code) {
     return OC_OK;
 }
 
+oc_status oc_selftest_per_device_once(int n_devices, int n_rounds, int fail_dev, int* runs, int* ok) {
+    if (n_devices < 1 || n_devices > oc::PerDeviceOnce::MAX_DEV || n_rounds < 1 || !runs || !ok) return OC_ERR_INVALID_ARG;
+    oc::PerDeviceOnce once;
+    for (int d = 0; d < n_devices; ++d) { runs[d] = 0; ok[d] = 0; }
+    for (int r = 0; r < n_rounds; ++r)
+        for (int d = 0; d < n_devices; ++d)
+            if (once.ensure(d, [&] { ++runs[d]; return d != fail_dev; })) ++ok[d];
+    return OC_OK;
+}
+
 oc_status oc_selftest_bounded_wait(oc_ctx* c, unsigned int limit_us, void* stream) {
     if (!c || limit_us == 0 || limit_us > 1000000u) return OC_ERR_INVALID_ARG;
     DeviceGuard guard(c->device);

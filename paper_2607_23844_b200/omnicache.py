@@ -32,7 +32,7 @@ EXPORTS = (
     "oc_device_status", "oc_profile_enable", "oc_profile_reset", "oc_profile_read", "oc_profile_span_read",
     "oc_profile_captured_read", "oc_match", "oc_match_frame_levels",
     "oc_select", "oc_gather", "oc_restore", "oc_layer_cache_put", "oc_layer_cache_get",
-    "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait",
+    "oc_layer_cache_clear", "oc_cache_step_host", "oc_match_frame_noalloc", "oc_selftest_bounded_wait", "oc_selftest_per_device_once",
     "oc_schedule_propose", "oc_joint_workspace_bytes", "oc_joint_groups", "oc_match_joint", "oc_select_joint",
     "oc_linear_gather_scatter", "oc_tc_plan_override", "oc_tc_plan_describe",
 )
@@ -72,6 +72,7 @@ _lib.oc_create.argtypes = [_vp, _i, C.c_size_t]
 _lib.oc_destroy.argtypes = [_vp]
 _lib.oc_device_status.argtypes = [_vp, _vp]
 _lib.oc_selftest_bounded_wait.argtypes = [_vp, C.c_uint, _vp]
+_lib.oc_selftest_per_device_once.argtypes = [C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
 _lib.oc_profile_enable.argtypes = [_vp, _i]
 _lib.oc_tc_plan_override.argtypes = [_vp, _i, _i, _i, _i, _i, _i]
 _lib.oc_tc_plan_describe.argtypes = [_vp, _vp, _vp]

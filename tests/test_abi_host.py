@@ -146,6 +146,23 @@ def test_null_context_and_bad_arguments_are_rejected_before_any_launch(oc):
     assert lib.oc_create(C.byref(h), -1, 0) == oc.ERR_INVALID_ARG
 
 
+def test_kernel_setup_runs_once_per_device_not_once_per_process(oc):
+    """Kernel attributes (the opt-in to large dynamic shared memory) belong to a device; a process may use
+    several.  The launchers' bookkeeping must run the set-up once for EVERY device it is asked about, remember
+    a failure without retrying it, and refuse nothing else (host-only: a counting set-up routine stands in)."""
+    lib = oc._lib
+    n = 5
+    runs, ok = (C.c_int * n)(), (C.c_int * n)()
+    assert lib.oc_selftest_per_device_once(n, 4, -1, runs, ok) == oc.OK
+    assert list(runs) == [1] * n and list(ok) == [4] * n
+    assert lib.oc_selftest_per_device_once(n, 3, 2, runs, ok) == oc.OK
+    assert list(runs) == [1] * n                       # the failing device's set-up is not run again either
+    assert list(ok) == [3, 3, 0, 3, 3]
+    assert lib.oc_selftest_per_device_once(0, 1, -1, runs, ok) == oc.ERR_INVALID_ARG
+    assert lib.oc_selftest_per_device_once(65, 1, -1, runs, ok) == oc.ERR_INVALID_ARG
+    assert lib.oc_selftest_per_device_once(n, 1, -1, None, ok) == oc.ERR_INVALID_ARG
+
+
 def test_schedule_proposal_matches_oracle(oc, oracle):
     """Algorithm 1 is host logic: the library's answer must equal the oracle's to the index."""
     import numpy as np
