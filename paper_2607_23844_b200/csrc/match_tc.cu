@@ -740,6 +740,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                 tc_fence_after();
                 uint32_t won_key0 = 0, won_key1 = 0;                   // per tile: the row's largest key and its chunk
                 int won_ch0 = -1, won_ch1 = -1;
+                bool released = false;
 #pragma unroll 1
                 for (int t = t_begin; t < t_end; ++t) {                // the piece's candidate tiles (of this warp)
                     if ((PAIR ? 2 : 1) * P.tpp * c.a_pair + (int)rank * P.tpp + t >= P.n_tilesA) continue;   // past the lattice
@@ -809,28 +810,39 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             }                                                                                                    \
         }                                                                                                        \
     } while (0)
+                    // The accumulators are handed back as soon as this warp's LAST load of them has landed in
+                    // registers, before that chunk is reduced: the MMAs of the piece after next wait for it.
+                    const bool last_tile = t + 1 == t_end;
+#define OC_RELEASE_ACCUMULATORS()                                                                                \
+    do {                                                                                                         \
+        tc_fence_before();                                                                                       \
+        __syncwarp();                                                                                            \
+        if (lane == 0) {                                                                                         \
+            if (PAIR) mbar_arrive_cluster(acc_empty + 8 * buf); else mbar_arrive(bar_acc_empty + 8 * buf);       \
+        }                                                                                                        \
+        released = true;                                                                                         \
+    } while (0)
                     if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
 #pragma unroll 1
                     for (int ch = ch_begin; ch < ch_end; ch += 2) {
                         tmem_ld_wait();
                         if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);
+                        else if (last_tile) OC_RELEASE_ACCUMULATORS();
                         OC_REDUCE_CHUNK(va, ch);
                         if (ch + 1 < ch_end) {
                             tmem_ld_wait();
                             if (ch + 2 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), va);
+                            else if (last_tile) OC_RELEASE_ACCUMULATORS();
                             OC_REDUCE_CHUNK(vb, ch + 1);
                         }
                     }
 #undef OC_REDUCE_CHUNK
                     if (t) { won_key1 = bm; won_ch1 = row_ok ? bc : -1; } else { won_key0 = bm; won_ch0 = row_ok ? bc : -1; }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {                                       // both accumulators may be overwritten
-                    if (PAIR) mbar_arrive_cluster(acc_empty + 8 * buf); else mbar_arrive(bar_acc_empty + 8 * buf);
-                }
-                // The rows' results go out only now: the arrival above releases (at cluster scope, in a
-                // pair) what its thread wrote before it, and would wait for these atomics to be performed.
+                if (!released) OC_RELEASE_ACCUMULATORS();              // (no chunk of a last tile: nothing was loaded)
+#undef OC_RELEASE_ACCUMULATORS
+                // The rows' results go out only after the arrival: it releases what its thread wrote before
+                // it, and would wait for these atomics to be performed.
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     const uint32_t bm = t ? won_key1 : won_key0;
