@@ -772,11 +772,17 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)t * tile_stride + buf * 256u;
                     // two register buffers: the TMEM load of the next step is in flight while this one is reduced
                     uint32_t va[32], vb[32];
+// (the scales of a chunk are asked for before the wait for its accumulators: shared memory is busy with
+//  the MMAs' operand reads, and the answers take a few hundred cycles)
+#define OC_LOAD_SCALES(ch)                                                                                       \
+    do {                                                                                                         \
+        _Pragma("unroll") for (int q = 0; q < 8; ++q) sc4[q] = col_scale4[(ch) * 8 + q];                         \
+    } while (0)
 #define OC_REDUCE_CHUNK(v, ch)                                                                                   \
     do {                                                                                                         \
         uint32_t kf[32];                                                                                         \
         _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
-            const float4 s4 = col_scale4[(ch) * 8 + (j >> 2)];                                                   \
+            const float4 s4 = sc4[j >> 2];                                                                       \
             float x0, x1, x2, x3;                                                                                \
             fma_pair(x0, x1, v[j], v[j + 1], s4.x, s4.y, row_lift);                                              \
             fma_pair(x2, x3, v[j + 2], v[j + 3], s4.z, s4.w, row_lift);                                          \
@@ -822,20 +828,24 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         }                                                                                                        \
         released = true;                                                                                         \
     } while (0)
+                    float4 sc4[8];
                     if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
 #pragma unroll 1
                     for (int ch = ch_begin; ch < ch_end; ch += 2) {
+                        OC_LOAD_SCALES(ch);
                         tmem_ld_wait();
                         if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);
                         else if (last_tile) OC_RELEASE_ACCUMULATORS();
                         OC_REDUCE_CHUNK(va, ch);
                         if (ch + 1 < ch_end) {
+                            OC_LOAD_SCALES(ch + 1);
                             tmem_ld_wait();
                             if (ch + 2 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), va);
                             else if (last_tile) OC_RELEASE_ACCUMULATORS();
                             OC_REDUCE_CHUNK(vb, ch + 1);
                         }
                     }
+#undef OC_LOAD_SCALES
 #undef OC_REDUCE_CHUNK
                     if (t) { won_key1 = bm; won_ch1 = row_ok ? bc : -1; } else { won_key0 = bm; won_ch0 = row_ok ? bc : -1; }
                 }
