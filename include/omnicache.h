@@ -243,8 +243,10 @@ oc_status oc_profile_captured_read(oc_ctx* ctx, int kernel_id, int64_t* launches
  *             not written).  FRAME: [B][T-1][H*W] per-position cosines of frame t vs t-1.
  *   pair_sim  nullable, FRAME only: [B][T-1][gy*gx] statistic of every adjacent pair (t, t-1),
  *             per patch.
- * bf16 TOKEN layouts without self_match run on the tcgen05 tensor cores (fp32 accumulation);
- * everything else on fp32 FMA pipelines.  Needs oc_match_workspace_bytes() of context workspace
+ * bf16 TOKEN layouts without self_match run on the tcgen05 tensor cores (fp32 accumulation) when the
+ * lattice has at most 9 members, C is a multiple of 8 and a group has at most 4800 representative
+ * slots (150 boxes of 32 lattice points; the SVD-XT frame has 2304, the SD3 image 1024);
+ * everything else on fp32 FMA pipelines, with the same results up to the tolerances above.  Needs oc_match_workspace_bytes() of context workspace
  * (OC_ERR_WORKSPACE otherwise).  Calls on one context must not overlap on the device. */
 oc_status oc_match(oc_ctx* ctx, const oc_layout* layout, const void* x, float* best_sim,
                    int32_t* best_idx, float* aux_sim, float* pair_sim, void* stream);
@@ -288,8 +290,8 @@ oc_status oc_linear_gather_scatter(oc_ctx* ctx, const void* a, int64_t a_rows, i
  * Token Cache on the frame pairs of Frame Cache (Section 3.2.3): it works on the feature map and the
  * frame pairing Frame Cache has just produced; matched pairs become token groups of 2*H*W tokens
  * with one representative per 2x2x2 cube, unmatched frames keep their 2x2 groups.
- * `layout` is the OC_KIND_TOKEN layout of the tensor (bf16, gy = gx = 1, no self_match;
- * OC_ERR_UNSUPPORTED otherwise).  `frames` is a device array of B*T slots {rep, partner} (int32
+ * `layout` is the OC_KIND_TOKEN layout of the tensor (bf16, gy = gx = 1, no self_match, a layout
+ * that oc_match runs on the tensor cores; OC_ERR_UNSUPPORTED otherwise).  `frames` is a device array of B*T slots {rep, partner} (int32
  * pairs, 8-byte aligned): slot f = {f, t} if frame f is the representative frame of the pair
  * (f, t), {f, -1} if frame f is a group of its own, {-1, -1} if frame f was absorbed into its
  * partner's group.
