@@ -778,7 +778,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     do {                                                                                                         \
         _Pragma("unroll") for (int q = 0; q < 8; ++q) sc4[q] = col_scale4[(ch) * 8 + q];                         \
     } while (0)
-#define OC_REDUCE_CHUNK(v, ch)                                                                                   \
+#define OC_REDUCE_CHUNK(v, ch, MASKED)                                                                           \
     do {                                                                                                         \
         uint32_t kf[32];                                                                                         \
         _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
@@ -791,7 +791,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             kf[j + 2] = __float_as_uint(x2) * 32u + (uint32_t)(29 - j);                                          \
             kf[j + 3] = __float_as_uint(x3) * key_mul + (uint32_t)(28 - j);                                      \
         }                                                                                                        \
-        if (piece_masked) {                                            /* warp-uniform, almost always false */   \
+        if (MASKED) {                                                  /* (a literal: two copies of the loop) */ \
             const int gcol = col0 + (ch) * 32, left = c.ncol - (ch) * 32;                                        \
             uint32_t masked = gt_mask[gcol >> 5];                                                                \
             if (gcol & 16) masked = (masked >> 16) | (gt_mask[(gcol >> 5) + 1] << 16);                           \
@@ -830,21 +830,31 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
     } while (0)
                     float4 sc4[8];
                     if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
-#pragma unroll 1
-                    for (int ch = ch_begin; ch < ch_end; ch += 2) {
-                        OC_LOAD_SCALES(ch);
-                        tmem_ld_wait();
-                        if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);
-                        else if (last_tile) OC_RELEASE_ACCUMULATORS();
-                        OC_REDUCE_CHUNK(va, ch);
-                        if (ch + 1 < ch_end) {
-                            OC_LOAD_SCALES(ch + 1);
-                            tmem_ld_wait();
-                            if (ch + 2 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), va);
-                            else if (last_tile) OC_RELEASE_ACCUMULATORS();
-                            OC_REDUCE_CHUNK(vb, ch + 1);
-                        }
+                    // (two copies of the loop: with the mask test inside it every key of a chunk has to sit in a
+                    //  register before the first maximum is taken)
+#define OC_CHUNK_LOOP(MASKED)                                                                                    \
+                    for (int ch = ch_begin; ch < ch_end; ch += 2) {                                              \
+                        OC_LOAD_SCALES(ch);                                                                      \
+                        tmem_ld_wait();                                                                          \
+                        if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);                   \
+                        else if (last_tile) OC_RELEASE_ACCUMULATORS();                                           \
+                        OC_REDUCE_CHUNK(va, ch, MASKED);                                                         \
+                        if (ch + 1 < ch_end) {                                                                   \
+                            OC_LOAD_SCALES(ch + 1);                                                              \
+                            tmem_ld_wait();                                                                      \
+                            if (ch + 2 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), va);               \
+                            else if (last_tile) OC_RELEASE_ACCUMULATORS();                                       \
+                            OC_REDUCE_CHUNK(vb, ch + 1, MASKED);                                                 \
+                        }                                                                                        \
                     }
+                    if (piece_masked) {
+#pragma unroll 1
+                        OC_CHUNK_LOOP(1)
+                    } else {
+#pragma unroll 1
+                        OC_CHUNK_LOOP(0)
+                    }
+#undef OC_CHUNK_LOOP
 #undef OC_LOAD_SCALES
 #undef OC_REDUCE_CHUNK
                     if (t) { won_key1 = bm; won_ch1 = row_ok ? bc : -1; } else { won_key0 = bm; won_ch0 = row_ok ? bc : -1; }
