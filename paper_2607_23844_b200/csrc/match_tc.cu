@@ -64,7 +64,7 @@
 //   warps 2..9  epilogue, two halves of four warps (one warp per TMEM lane quarter, thread r owns row
 //               r of the candidate tiles).  With two accumulator sets the halves take alternate
 //               pieces; with one set of two tiles one tile each; with one set of one tile half of
-//               the columns each.  tcgen05.ld 32 columns at a time (double buffered), scale by the
+//               the columns each.  tcgen05.ld 32 columns at a time, scale by the
 //               representative's inverse norm, and a running
 //               maximum over integer keys: the scaled similarity, lifted into one binade (where a
 //               float's bits are linear in its value), times 32, plus 31 - column (one three-input max
@@ -770,17 +770,17 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     int bc = -1;
                     const float row_lift = t ? lift1 : lift0;
                     const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)t * tile_stride + buf * 256u;
-                    // two register buffers: the TMEM load of the next step is in flight while this one is reduced
-                    uint32_t va[32], vb[32];
+                    uint32_t va[32];
 // (the scales of a chunk are asked for before the wait for its accumulators: shared memory is busy with
 //  the MMAs' operand reads, and the answers take a few hundred cycles)
 #define OC_LOAD_SCALES(ch)                                                                                       \
     do {                                                                                                         \
         _Pragma("unroll") for (int q = 0; q < 8; ++q) sc4[q] = col_scale4[(ch) * 8 + q];                         \
     } while (0)
-#define OC_REDUCE_CHUNK(v, ch, MASKED)                                                                           \
+// The keys of a chunk (and, in the parity instance, its row of the full similarity matrix): everything
+// that reads the loaded accumulators and the scales, so that both registers sets are free afterwards.
+#define OC_KEYS(v, ch, MASKED)                                                                                   \
     do {                                                                                                         \
-        uint32_t kf[32];                                                                                         \
         _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
             const float4 s4 = sc4[j >> 2];                                                                       \
             float x0, x1, x2, x3;                                                                                \
@@ -799,10 +799,6 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
             _Pragma("unroll") for (int j = 0; j < 32; ++j)                                                       \
                 if ((masked >> j) & 1u) kf[j] = 0u;                                                              \
         }                                                                                                        \
-        const uint32_t cm = key_tree_max(kf);                                                                    \
-        /* a later chunk wins only with a strictly larger similarity (the index bits set aside); a zeroed     */ \
-        /* key never does: a lifted similarity lies strictly above the binade's lower end, so a key is > 31  */ \
-        if (cm > (bm | 31u)) { bm = cm; bc = (ch); }                                                             \
         if (AUX && aux_row) {                                                                                    \
             for (int j = 0; j < 32; ++j) {                                                                       \
                 const float sc = col_scale1[(ch) * 32 + j];                                                      \
@@ -829,24 +825,23 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
         released = true;                                                                                         \
     } while (0)
                     float4 sc4[8];
-                    if (ch_begin < ch_end) tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va);
-                    // (two copies of the loop: with the mask test inside it every key of a chunk has to sit in a
-                    //  register before the first maximum is taken)
+                    uint32_t kf[32];
+                    // One register buffer for the accumulators: the next chunk's load and its scales are asked for
+                    // as soon as this chunk's keys are formed, and arrive under the maximum tree.  The loop exists
+                    // twice (with the mask test inside it every key of a chunk has to sit in a register before the
+                    // first maximum is taken, masked columns or not).  A later chunk wins only with a strictly
+                    // larger similarity (the index bits set aside); a zeroed key never does: a lifted similarity
+                    // lies strictly above the binade's lower end, so a key is > 31.
 #define OC_CHUNK_LOOP(MASKED)                                                                                    \
-                    for (int ch = ch_begin; ch < ch_end; ch += 2) {                                              \
-                        OC_LOAD_SCALES(ch);                                                                      \
+                    for (int ch = ch_begin; ch < ch_end; ++ch) {                                                 \
                         tmem_ld_wait();                                                                          \
-                        if (ch + 1 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), vb);                   \
+                        OC_KEYS(va, ch, MASKED);                                                                 \
+                        if (ch + 1 < ch_end) { tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), va); OC_LOAD_SCALES(ch + 1); } \
                         else if (last_tile) OC_RELEASE_ACCUMULATORS();                                           \
-                        OC_REDUCE_CHUNK(va, ch, MASKED);                                                         \
-                        if (ch + 1 < ch_end) {                                                                   \
-                            OC_LOAD_SCALES(ch + 1);                                                              \
-                            tmem_ld_wait();                                                                      \
-                            if (ch + 2 < ch_end) tmem_ld32(t_row + (uint32_t)((ch + 2) * 32), va);               \
-                            else if (last_tile) OC_RELEASE_ACCUMULATORS();                                       \
-                            OC_REDUCE_CHUNK(vb, ch + 1, MASKED);                                                 \
-                        }                                                                                        \
+                        const uint32_t cm = key_tree_max(kf);                                                    \
+                        if (cm > (bm | 31u)) { bm = cm; bc = ch; }                                               \
                     }
+                    if (ch_begin < ch_end) { tmem_ld32(t_row + (uint32_t)(ch_begin * 32), va); OC_LOAD_SCALES(ch_begin); }
                     if (piece_masked) {
 #pragma unroll 1
                         OC_CHUNK_LOOP(1)
@@ -856,7 +851,7 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
                     }
 #undef OC_CHUNK_LOOP
 #undef OC_LOAD_SCALES
-#undef OC_REDUCE_CHUNK
+#undef OC_KEYS
                     if (t) { won_key1 = bm; won_ch1 = row_ok ? bc : -1; } else { won_key0 = bm; won_ch0 = row_ok ? bc : -1; }
                 }
                 if (!released) OC_RELEASE_ACCUMULATORS();              // (no chunk of a last tile: nothing was loaded)
