@@ -835,9 +835,9 @@ match_tc_kernel(const __grid_constant__ TcParams KP) {
 #define OC_CHUNK_LOOP(MASKED)                                                                                    \
                     for (int ch = ch_begin; ch < ch_end; ++ch) {                                                 \
                         tmem_ld_wait();                                                                          \
+                        if (ch + 1 == ch_end && last_tile) OC_RELEASE_ACCUMULATORS();                            \
                         OC_KEYS(va, ch, MASKED);                                                                 \
                         if (ch + 1 < ch_end) { tmem_ld32(t_row + (uint32_t)((ch + 1) * 32), va); OC_LOAD_SCALES(ch + 1); } \
-                        else if (last_tile) OC_RELEASE_ACCUMULATORS();                                           \
                         const uint32_t cm = key_tree_max(kf);                                                    \
                         if (cm > (bm | 31u)) { bm = cm; bc = ch; }                                               \
                     }
