@@ -38,7 +38,7 @@ FALLBACK = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1
 # DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists for the workload.
 # (profiles/step_kernels_<workload>.md: the row kernel's DRAM read + write of one cold launch)
-NCU_TRAFFIC_BYTES = {"svd_token_l0": 178078976, "sd3_token": 25320448, "svd_token_l1": 76370176, "svd_token_l2": 37090816, "svd_frame": 150526464, "latte_block": 9459712, "tiny_token": 106240}
+NCU_TRAFFIC_BYTES = {"svd_token_l0": 174840576, "sd3_token": 25319424, "svd_token_l1": 76274432, "svd_token_l2": 37090048, "svd_frame": 150985216, "latte_block": 9469184, "tiny_token": 106240}
 
 
 def measured_peaks():
