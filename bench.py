@@ -510,6 +510,21 @@ def measure_workload(args, oc, torch, dev, local_rank, rank, world, name, w, ste
             roofline["device_span_us"] = span_us
             roofline["achieved_device_span"] = flops / (span_us * 1e-6) / 1e12
             roofline["frac_device_span"] = roofline["achieved_device_span"] / peak
+        # Below the ridge (FLOP per compulsory byte under tensor peak / copy bandwidth: the smallest SVD level,
+        # 108 FLOP/B against ~250) the matcher's roof is HBM: the tensor figures stay beside it.
+        ridge = peak * 1e12 / (peaks["hbm_gbs"] * 1e9)
+        if flops / tensor_bytes < ridge:
+            gbs = tensor_bytes / (k_us * 1e-6) / 1e9
+            tensor_side = {k: roofline[k] for k in ("achieved", "peak", "frac", "peak_source", "frac_of_burst",
+                                                    "frac_of_sustained", "frac_of_nominal")}
+            roofline.update({"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": gbs / peaks["hbm_gbs"], "peak_source": f"{peaks['_source']} copy bandwidth",
+                             "bytes_per_launch": tensor_bytes, "flop_per_byte": flops / tensor_bytes,
+                             "ridge_flop_per_byte": ridge, "tensor": tensor_side,
+                             "frac_net_of_bracket": tensor_bytes / (max(ops[kern]["net_us"], 1e-3) * 1e-6) / 1e9 / peaks["hbm_gbs"]})
+            if span_us:
+                roofline["frac_device_span"] = tensor_bytes / (span_us * 1e-6) / 1e9 / peaks["hbm_gbs"]
+                roofline["achieved_device_span"] = tensor_bytes / (span_us * 1e-6) / 1e9
     elif bound == "hbm":
         roofline = {"kernel": kern, "bound": "hbm", "achieved": ops[kern]["GB/s"], "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "frac": ops[kern]["frac_hbm"], "traffic": NCU_TRAFFIC_BYTES.get(name),
